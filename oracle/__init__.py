@@ -1,0 +1,231 @@
+"""ctypes access to the CPU oracle (``dspark_oracle.c``) -- test infrastructure only.
+
+Only tests, the smoke check and the benchmark's CPU-baseline / reference legs
+may import this package.  It never imports the CUDA package and the CUDA
+package never imports it.  Arrays are numpy; bf16 logits are passed as their
+raw 16-bit patterns (``uint16``).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dspark_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+F32, BF16 = 0, 1
+MODE_EARLY_STOP, MODE_GLOBAL, MODE_TOPK = 0, 1, 2
+ST_BAD_OFFSETS, ST_BAD_TOKEN, ST_BAD_ROW = 1, 2, 4
+ST_CONF_CLAMPED, ST_BUDGET_LT_R, ST_ALL_NEG_INF = 16, 32, 64
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no contraction, no fast-math) next to its source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-Wall", "-shared", "-fPIC",
+             "-pthread", _SRC, "-o", tmp, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+class _SchedInfo(C.Structure):
+    _fields_ = [("B", C.c_int32), ("n_admitted", C.c_int32), ("status", C.c_int32),
+                ("n_candidates", C.c_int32), ("tau", C.c_double), ("theta", C.c_double)]
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+    return _lib
+
+
+def _p(a, ctype=C.c_void_p):
+    return None if a is None else a.ctypes.data_as(ctype)
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.uint16:
+        return BF16
+    raise TypeError(f"logits must be float32 or uint16 (bf16 bits), got {a.dtype}")
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    c = (C.c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in ctr])
+    k = (C.c_uint32 * 2)(*[int(x) & 0xFFFFFFFF for x in key])
+    o = (C.c_uint32 * 4)()
+    lib().orc_philox4x32_10(c, k, o)
+    return np.array(list(o), dtype=np.uint32)
+
+
+def uniforms(seed: int, r: int, j: int):
+    ua, ur = C.c_float(), C.c_float()
+    lib().orc_uniforms(C.c_uint64(seed), C.c_uint32(r), C.c_uint32(j), C.byref(ua), C.byref(ur))
+    return ua.value, ur.value
+
+
+def sps_table(bp_tokens, bp_sps, max_tokens: int) -> np.ndarray:
+    bt = np.ascontiguousarray(bp_tokens, dtype=np.int32)
+    bs = np.ascontiguousarray(bp_sps, dtype=np.float64)
+    out = np.empty(max_tokens + 1, dtype=np.float64)
+    rc = lib().orc_sps_table(_p(bt), _p(bs), C.c_int(len(bt)), C.c_int(max_tokens), _p(out))
+    if rc != 0:
+        raise ValueError("invalid breakpoints")
+    return out
+
+
+@dataclass
+class ScheduleResult:
+    lengths: np.ndarray
+    survival: np.ndarray
+    expected_len: np.ndarray
+    B: int
+    n_admitted: int
+    n_candidates: int
+    status: int
+    tau: float
+    theta: float
+    theta_path: np.ndarray
+
+
+def schedule(conf, table, budget_tokens: int, mode: int = MODE_EARLY_STOP, topk_K: int = 0,
+             draft_len=None) -> ScheduleResult:
+    conf = np.ascontiguousarray(conf, dtype=np.float32)
+    R, gamma = conf.shape
+    table = np.ascontiguousarray(table, dtype=np.float64)
+    dl = None if draft_len is None else np.ascontiguousarray(draft_len, dtype=np.int32)
+    out_len = np.zeros(R, dtype=np.int32)
+    surv = np.zeros((R, max(gamma, 1)), dtype=np.float32)[:, :gamma].copy()
+    exp_len = np.zeros(R, dtype=np.float32)
+    path = np.full(R * gamma + 1, np.nan, dtype=np.float64)
+    info = _SchedInfo()
+    rc = lib().orc_schedule(_p(conf), _p(dl), C.c_int(R), C.c_int(gamma), C.c_int(budget_tokens),
+                            C.c_int(mode), C.c_int(topk_K), _p(table), C.c_int(len(table) - 1),
+                            _p(out_len), _p(surv), _p(exp_len), C.byref(info), _p(path))
+    if rc != 0:
+        raise ValueError(f"orc_schedule failed ({rc})")
+    return ScheduleResult(out_len, surv, exp_len, info.B, info.n_admitted, info.n_candidates,
+                          info.status, info.tau, info.theta, path)
+
+
+def schedule_bruteforce(conf, table, budget_tokens: int, draft_len=None):
+    conf = np.ascontiguousarray(conf, dtype=np.float32)
+    R, gamma = conf.shape
+    table = np.ascontiguousarray(table, dtype=np.float64)
+    dl = None if draft_len is None else np.ascontiguousarray(draft_len, dtype=np.int32)
+    best = C.c_double()
+    best_B = C.c_int32()
+    best_len = np.zeros(R, dtype=np.int32)
+    rc = lib().orc_schedule_bruteforce(_p(conf), _p(dl), C.c_int(R), C.c_int(gamma),
+                                       C.c_int(budget_tokens), _p(table), C.c_int(len(table) - 1),
+                                       C.byref(best), C.byref(best_B), _p(best_len))
+    if rc != 0:
+        raise ValueError("brute force limited to R <= 8, gamma <= 8")
+    return best.value, best_B.value, best_len
+
+
+def _logits(a):
+    a = np.asarray(a)
+    if a.ndim != 2 or a.strides[1] != a.itemsize:
+        raise ValueError("logits must be 2-D with unit inner stride")
+    return a, a.strides[0] // a.itemsize
+
+
+def softmax_row(logits, row: int, temperature: float = 1.0):
+    a, stride = _logits(logits)
+    V = a.shape[1]
+    probs = np.empty(V, dtype=np.float64)
+    m, Z = C.c_double(), C.c_double()
+    bad = lib().orc_softmax_row(_p(a), C.c_int(_dtype_code(a)), C.c_int64(row), C.c_int64(stride),
+                                C.c_int(V), C.c_double(temperature), _p(probs), C.byref(m), C.byref(Z))
+    return probs, m.value, Z.value, bool(bad)
+
+
+@dataclass
+class GreedyResult:
+    accepted_len: np.ndarray
+    out_tokens: np.ndarray
+    row_argmax: np.ndarray
+    status: np.ndarray
+
+
+def verify_greedy(target, row_offsets, draft_tokens) -> GreedyResult:
+    t, stride = _logits(target)
+    ro = np.ascontiguousarray(row_offsets, dtype=np.int32)
+    dt = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    R = len(ro) - 1
+    n_rows = t.shape[0]
+    acc = np.zeros(R, dtype=np.int32)
+    out = np.full(n_rows, -1, dtype=np.int32)
+    am = np.full(n_rows, -1, dtype=np.int32)
+    st = np.zeros(R, dtype=np.int32)
+    rc = lib().orc_verify_greedy(_p(t), C.c_int(_dtype_code(t)), C.c_int64(stride), C.c_int(t.shape[1]),
+                                 _p(ro), _p(dt), C.c_int(R), _p(acc), _p(out), _p(am), _p(st))
+    if rc != 0:
+        raise ValueError("orc_verify_greedy failed")
+    return GreedyResult(acc, out, am, st)
+
+
+def verify_greedy_mt(target, row_offsets, draft_tokens, n_threads: int):
+    t, stride = _logits(target)
+    ro = np.ascontiguousarray(row_offsets, dtype=np.int32)
+    dt = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    R = len(ro) - 1
+    acc = np.zeros(R, dtype=np.int32)
+    out = np.full(t.shape[0], -1, dtype=np.int32)
+    st = np.zeros(R, dtype=np.int32)
+    rc = lib().orc_verify_greedy_mt(_p(t), C.c_int(_dtype_code(t)), C.c_int64(stride), C.c_int(t.shape[1]),
+                                    _p(ro), _p(dt), C.c_int(R), C.c_int(n_threads), _p(acc), _p(out), _p(st))
+    if rc != 0:
+        raise ValueError("orc_verify_greedy_mt failed")
+    return acc, out, st
+
+
+@dataclass
+class VerifyResult:
+    accepted_len: np.ndarray
+    out_tokens: np.ndarray
+    p_tok: np.ndarray
+    q_tok: np.ndarray
+    accept_margin: np.ndarray
+    token_margin: np.ndarray
+    status: np.ndarray
+
+
+def verify(target, draft, row_offsets, draft_tokens, temperature: float, seed: int,
+           draft_row_start=None, eval_all: bool = True, n_threads: int = 1) -> VerifyResult:
+    t, ts = _logits(target)
+    d, ds = _logits(draft)
+    if t.dtype != d.dtype:
+        raise TypeError("target and draft logits must share a dtype")
+    ro = np.ascontiguousarray(row_offsets, dtype=np.int32)
+    dt = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    drs = None if draft_row_start is None else np.ascontiguousarray(draft_row_start, dtype=np.int64)
+    R = len(ro) - 1
+    n_rows = t.shape[0]
+    acc = np.zeros(R, dtype=np.int32)
+    out = np.full(n_rows, -1, dtype=np.int32)
+    p = np.full(n_rows, np.nan)
+    q = np.full(n_rows, np.nan)
+    am = np.full(n_rows, np.nan)
+    tm = np.full(R, np.nan)
+    st = np.zeros(R, dtype=np.int32)
+    rc = lib().orc_verify(_p(t), _p(d), C.c_int(_dtype_code(t)), C.c_int64(ts), C.c_int64(ds),
+                          C.c_int(t.shape[1]), _p(ro), _p(drs), _p(dt), C.c_int(R),
+                          C.c_double(temperature), C.c_uint64(seed), C.c_int(int(eval_all)),
+                          C.c_int(n_threads), _p(acc), _p(out), _p(p), _p(q), _p(am), _p(tm), _p(st))
+    if rc != 0:
+        raise ValueError("orc_verify rejected its arguments")
+    return VerifyResult(acc, out, p, q, am, tm, st)

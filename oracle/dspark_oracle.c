@@ -1,0 +1,632 @@
+/*
+ * DSpark CPU oracle -- TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, sequential restatement of what the scheduler and the
+ * speculative verifier compute, in fp64 (except where noted), written from
+ * the paper's definitions.  Only tests, the smoke check and the benchmark's
+ * cpu_baseline / reference legs may call it.  It shares no code, header,
+ * table or constant generator with the CUDA library; the handful of enum
+ * values it repeats (dtype, mode, status bits) are the public API contract.
+ *
+ * Every function names the passage of the paper it follows.  Where the paper
+ * is silent the reading taken is stated next to the code.
+ *
+ * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC -pthread
+ * (no contraction: products and sums round exactly as written).
+ */
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_F32 0
+#define ORC_BF16 1
+
+#define ORC_MODE_EARLY_STOP 0
+#define ORC_MODE_GLOBAL 1
+#define ORC_MODE_TOPK 2
+
+/* status bits (per request in the verifier, global in the scheduler) */
+#define ORC_ST_BAD_OFFSETS 1
+#define ORC_ST_BAD_TOKEN 2
+#define ORC_ST_BAD_ROW 4
+#define ORC_ST_CONF_CLAMPED 16
+#define ORC_ST_BUDGET_LT_R 32
+#define ORC_ST_ALL_NEG_INF 64
+
+/* ------------------------------------------------------------------------ */
+/* Counter-based RNG.  The paper never names a generator; the reading taken  */
+/* is Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): ten rounds of       */
+/*   (c0,c1,c2,c3) <- (hi(M1*c2)^c1^k0, lo(M1*c2), hi(M0*c0)^c3^k1, lo(M0*c0)) */
+/* with the key bumped by the Weyl constants between rounds.                 */
+/* ------------------------------------------------------------------------ */
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t p0 = (uint64_t)M0 * (uint64_t)c0;
+        uint64_t p1 = (uint64_t)M1 * (uint64_t)c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += W0; k1 += W1;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/*
+ * The two uniforms of (seed, request r, position j): counter (j, 0, r, 0),
+ * key (seed low word, seed high word); word 0 drives the accept test, word 1
+ * the residual / bonus draw.  u = (word >> 8) * 2^-24 lies in [0,1) and is
+ * exact in fp32.
+ */
+void orc_uniforms(uint64_t seed, uint32_t r, uint32_t j, float* u_accept, float* u_resample)
+{
+    uint32_t ctr[4] = { j, 0u, r, 0u };
+    uint32_t key[2] = { (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32) };
+    uint32_t w[4];
+    orc_philox4x32_10(ctr, key, w);
+    *u_accept = (float)(w[0] >> 8) * (1.0f / 16777216.0f);
+    *u_resample = (float)(w[1] >> 8) * (1.0f / 16777216.0f);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Engine throughput profile SPS(B) (Section 3.2.2: profiled once, stored as */
+/* a cost table).  Reading: dense fp64 table B = 0..max_tokens, piecewise    */
+/* linear between the given breakpoints, constant outside them.              */
+/* ------------------------------------------------------------------------ */
+int orc_sps_table(const int32_t* bp_tokens, const double* bp_sps, int n_bp,
+                  int max_tokens, double* table)
+{
+    if (n_bp < 1 || max_tokens < 0) return -1;
+    for (int k = 1; k < n_bp; ++k)
+        if (bp_tokens[k] <= bp_tokens[k - 1]) return -1;
+    for (int B = 0; B <= max_tokens; ++B) {
+        double y;
+        if (B <= bp_tokens[0]) {
+            y = bp_sps[0];
+        } else if (B >= bp_tokens[n_bp - 1]) {
+            y = bp_sps[n_bp - 1];
+        } else {
+            int k = 0;
+            while (!(bp_tokens[k] <= B && B < bp_tokens[k + 1])) ++k;
+            double frac = (double)(B - bp_tokens[k]) / (double)(bp_tokens[k + 1] - bp_tokens[k]);
+            double dy = bp_sps[k + 1] - bp_sps[k];
+            double t = dy * frac;
+            y = bp_sps[k] + t;
+        }
+        table[B] = y;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Scheduler (Algorithm 1; definitions of a, B, tau, Theta in Section 3.2.2; */
+/* no-break variant and capacity limit in Section 4.2).                      */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    float a;
+    int32_t j;
+    int32_t r;
+} orc_cand_t;
+
+static int cand_cmp(const void* pa, const void* pb)
+{
+    const orc_cand_t* x = (const orc_cand_t*)pa;
+    const orc_cand_t* y = (const orc_cand_t*)pb;
+    if (x->a > y->a) return -1;       /* survival probability, descending */
+    if (x->a < y->a) return 1;
+    if (x->j != y->j) return x->j < y->j ? -1 : 1;   /* then position ascending */
+    if (x->r != y->r) return x->r < y->r ? -1 : 1;   /* then request ascending  */
+    return 0;
+}
+
+/* Confidence as the scheduler reads it: c in [0,1]; NaN or negative ends the
+ * block (0), above 1 is 1.  Sets *clamped when it changed anything. */
+static float sanitize_conf(float c, int* clamped)
+{
+    if (!(c >= 0.0f)) { *clamped = 1; return 0.0f; }
+    if (c > 1.0f) { *clamped = 1; return 1.0f; }
+    return c;
+}
+
+/* Survival products a_{r,j} = prod_{i<=j} c_{r,i} (Algorithm 1, line 2), as a
+ * left-to-right fp32 product.  Positions at or beyond draft_len[r], and all
+ * positions after the product reaches 0, hold 0 and are not candidates. */
+static void survival_products(const float* conf, const int32_t* draft_len, int R, int gamma,
+                              float* surv, int* clamped)
+{
+    for (int r = 0; r < R; ++r) {
+        int lim = gamma;
+        if (draft_len) { lim = draft_len[r]; if (lim < 0) lim = 0; if (lim > gamma) lim = gamma; }
+        float a = 1.0f;
+        int dead = 0;
+        for (int j = 0; j < gamma; ++j) {
+            if (j >= lim) dead = 1;
+            if (!dead) {
+                a = a * sanitize_conf(conf[(size_t)r * gamma + j], clamped);
+                if (!(a > 0.0f)) dead = 1;
+            }
+            surv[(size_t)r * gamma + j] = dead ? 0.0f : a;
+        }
+    }
+}
+
+/* Expected-accept mass of one candidate in units of 2^-40 (an exact integer
+ * sum keeps tau independent of summation order). */
+static uint64_t fix40(float a)
+{
+    return (uint64_t)((double)a * 1099511627776.0);
+}
+
+typedef struct {
+    int32_t B;           /* batch tokens R + sum l*_r        */
+    int32_t n_admitted;  /* i*                               */
+    int32_t status;      /* warning bits                     */
+    int32_t n_candidates;/* |E|                              */
+    double tau;          /* expected accepted tokens         */
+    double theta;        /* tau * SPS(B)                     */
+} orc_sched_info_t;
+
+/*
+ * table[0..max_tokens] is SPS; lookups beyond max_tokens use the last entry.
+ * theta_path (optional, length >= min(|E|, cap)+1) receives Theta_i * 2^40.
+ */
+int orc_schedule(const float* conf, const int32_t* draft_len, int R, int gamma,
+                 int budget_tokens, int mode, int topk_K,
+                 const double* table, int max_tokens,
+                 int32_t* out_len, float* out_survival, float* out_expected_len,
+                 orc_sched_info_t* info, double* theta_path)
+{
+    if (R <= 0 || gamma < 0 || max_tokens < 0) return -1;
+    size_t n = (size_t)R * (size_t)(gamma > 0 ? gamma : 1);
+    float* surv = (float*)calloc(n, sizeof(float));
+    orc_cand_t* cand = (orc_cand_t*)malloc(n * sizeof(orc_cand_t));
+    if (!surv || !cand) { free(surv); free(cand); return -2; }
+    int clamped = 0;
+    survival_products(conf, draft_len, R, gamma, surv, &clamped);
+
+    /* candidate space E = {(r,j) : a_{r,j} > 0}, sorted descending by a */
+    size_t nE = 0;
+    for (int r = 0; r < R; ++r)
+        for (int j = 0; j < gamma; ++j) {
+            float a = surv[(size_t)r * gamma + j];
+            if (a > 0.0f) { cand[nE].a = a; cand[nE].j = j; cand[nE].r = r; ++nE; }
+        }
+    qsort(cand, nE, sizeof(orc_cand_t), cand_cmp);
+
+    int status = 0;
+    if (clamped) status |= ORC_ST_CONF_CLAMPED;
+    long cap = (long)budget_tokens - (long)R;
+    if (cap < 0) { cap = 0; status |= ORC_ST_BUDGET_LT_R; }
+    size_t N = nE < (size_t)cap ? nE : (size_t)cap;
+
+    /* initial state: l = 0, B = R, tau = R, Theta_best = R * SPS(R) */
+    uint64_t T = (uint64_t)R << 40;
+    int B = R;
+    double theta_best = (double)T * table[B < max_tokens ? B : max_tokens];
+    uint64_t T_best = T;
+    size_t i_star = 0;
+    if (theta_path) theta_path[0] = theta_best;
+
+    for (size_t i = 1; i <= N; ++i) {
+        T += fix40(cand[i - 1].a);
+        B = R + (int)i;
+        double theta = (double)T * table[B < max_tokens ? B : max_tokens];
+        if (theta_path) theta_path[i] = theta;
+        if (mode == ORC_MODE_TOPK) {
+            if ((long)i <= (long)topk_K) { theta_best = theta; T_best = T; i_star = i; }
+            continue;
+        }
+        if (theta > theta_best) {
+            theta_best = theta; T_best = T; i_star = i;
+        } else if (mode == ORC_MODE_EARLY_STOP) {
+            break;                                  /* Algorithm 1: else break */
+        }
+    }
+
+    for (int r = 0; r < R; ++r) out_len[r] = 0;
+    for (size_t k = 0; k < i_star; ++k) out_len[cand[k].r] += 1;
+
+    if (out_survival) memcpy(out_survival, surv, (size_t)R * gamma * sizeof(float));
+    if (out_expected_len)
+        for (int r = 0; r < R; ++r) {
+            double e = 1.0;
+            for (int j = 0; j < out_len[r]; ++j) e += (double)surv[(size_t)r * gamma + j];
+            out_expected_len[r] = (float)e;
+        }
+    if (info) {
+        info->B = R + (int)i_star;
+        info->n_admitted = (int32_t)i_star;
+        info->status = status;
+        info->n_candidates = (int32_t)nE;
+        info->tau = (double)T_best / 1099511627776.0;
+        info->theta = theta_best / 1099511627776.0;
+    }
+    free(surv); free(cand);
+    return 0;
+}
+
+/*
+ * Exhaustive companion for tiny batches: every schedule l in {0..gamma}^R whose
+ * positions are all candidates (a > 0, j < draft_len) and whose admitted count
+ * is within the cap; Theta(l) from the same integer tau and the same table.
+ * Returns the maximum Theta*2^40 and, among maximisers, the smallest batch size.
+ */
+int orc_schedule_bruteforce(const float* conf, const int32_t* draft_len, int R, int gamma,
+                            int budget_tokens, const double* table, int max_tokens,
+                            double* best_theta_scaled, int32_t* best_B, int32_t* best_len)
+{
+    if (R <= 0 || R > 8 || gamma < 0 || gamma > 8) return -1;
+    float surv[64];
+    int clamped = 0;
+    survival_products(conf, draft_len, R, gamma, surv, &clamped);
+    long cap = (long)budget_tokens - (long)R;
+    if (cap < 0) cap = 0;
+    int len[8] = {0};
+    double best = -1.0; int bestB = -1;
+    for (;;) {
+        int ok = 1; long tot = 0;
+        uint64_t T = (uint64_t)R << 40;
+        for (int r = 0; r < R && ok; ++r) {
+            for (int j = 0; j < len[r]; ++j) {
+                float a = surv[r * gamma + j];
+                if (!(a > 0.0f)) { ok = 0; break; }
+                T += fix40(a);
+            }
+            tot += len[r];
+        }
+        if (ok && tot <= cap) {
+            int B = R + (int)tot;
+            double theta = (double)T * table[B < max_tokens ? B : max_tokens];
+            if (theta > best || (theta == best && B < bestB)) {
+                best = theta; bestB = B;
+                if (best_len) for (int r = 0; r < R; ++r) best_len[r] = len[r];
+            }
+        }
+        int r = 0;
+        while (r < R) { if (++len[r] <= gamma) break; len[r] = 0; ++r; }
+        if (r == R) break;
+    }
+    *best_theta_scaled = best; *best_B = bestB;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Logit access: bf16 is storage only; its 16 bits are the high half of the  */
+/* fp32 pattern.                                                             */
+/* ------------------------------------------------------------------------ */
+static inline double logit_at(const void* base, int dtype, int64_t row, int64_t stride, int64_t v)
+{
+    if (dtype == ORC_BF16) {
+        uint16_t h = ((const uint16_t*)base)[row * stride + v];
+        uint32_t bits = (uint32_t)h << 16;
+        float f;
+        memcpy(&f, &bits, 4);
+        return (double)f;
+    }
+    return (double)((const float*)base)[row * stride + v];
+}
+
+/* Lowest-index argmax; NaN never wins a comparison.  Returns 1 when no element
+ * exceeds -inf (index 0 is reported then). */
+static int row_argmax(const void* base, int dtype, int64_t row, int64_t stride, int V, int32_t* idx)
+{
+    double best = -INFINITY;
+    int32_t bi = 0;
+    for (int v = 0; v < V; ++v) {
+        double x = logit_at(base, dtype, row, stride, v);
+        if (x > best) { best = x; bi = v; }
+    }
+    *idx = bi;
+    return best == -INFINITY;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Greedy verification: a draft token is accepted iff it equals the target   */
+/* row's argmax (lowest index on ties); the first mismatch ends the prefix   */
+/* (Section 2.1: the first rejection discards the rest) and the emitted      */
+/* token is the argmax of that row, or of the bonus row when all matched.    */
+/* ------------------------------------------------------------------------ */
+int orc_verify_greedy(const void* target, int dtype, int64_t target_row_stride, int V,
+                      const int32_t* row_offsets, const int32_t* draft_tokens, int R,
+                      int32_t* accepted_len, int32_t* out_tokens, int32_t* row_argmax_out,
+                      int32_t* status /* [R] */)
+{
+    if (R <= 0 || V <= 0) return -1;
+    for (int r = 0; r < R; ++r) {
+        int32_t lo = row_offsets[r], hi = row_offsets[r + 1];
+        int32_t st = 0;
+        if (lo < 0 || hi - lo < 1) { status[r] = ORC_ST_BAD_OFFSETS; accepted_len[r] = 0; continue; }
+        int32_t len = hi - lo - 1;
+        for (int32_t i = lo; i < hi; ++i) out_tokens[i] = -1;
+        int32_t n = len;
+        int32_t emitted = -1;
+        for (int32_t j = 0; j < len; ++j) {
+            int32_t d = draft_tokens[lo + j];
+            if (d < 0 || d >= V) st |= ORC_ST_BAD_TOKEN;
+        }
+        if (st) {                          /* invalid draft token: nothing is emitted */
+            accepted_len[r] = 0; status[r] = st; continue;
+        }
+        for (int32_t j = 0; j <= len; ++j) {
+            int32_t am;
+            if (row_argmax(target, dtype, lo + j, target_row_stride, V, &am)) st |= ORC_ST_ALL_NEG_INF;
+            if (row_argmax_out) row_argmax_out[lo + j] = am;
+            if (j == len) { emitted = am; break; }
+            if (draft_tokens[lo + j] != am) { n = j; emitted = am; break; }
+        }
+        for (int32_t j = 0; j < n; ++j) out_tokens[lo + j] = draft_tokens[lo + j];
+        out_tokens[lo + n] = emitted;
+        accepted_len[r] = n;
+        status[r] = st;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Sampling verification (Section 2.1): accept x_k with probability          */
+/* min(1, p_k^t(x_k)/p_k^d(x_k)), left to right, first rejection discards    */
+/* the suffix; on rejection draw from norm(max(0, p - q)) at that position,  */
+/* otherwise draw the bonus token from p of the last row (Section 1).        */
+/* p = softmax(target/T), q = softmax(draft/T), one temperature for both.    */
+/* ------------------------------------------------------------------------ */
+
+/* m = max_v x_v and Z = sum_v exp(x_v - m) in vocabulary order, x = logit/T.
+ * Returns 1 when the row is unusable (contains NaN, or its max is -inf). */
+static int row_softmax_stats(const void* base, int dtype, int64_t row, int64_t stride, int V,
+                             double T, double* m_out, double* Z_out)
+{
+    double m = -INFINITY;
+    int bad = 0;
+    for (int v = 0; v < V; ++v) {
+        double x = logit_at(base, dtype, row, stride, v) / T;
+        if (x != x) bad = 1;
+        if (x > m) m = x;
+    }
+    double Z = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double x = logit_at(base, dtype, row, stride, v) / T;
+        Z += exp(x - m);
+    }
+    *m_out = m; *Z_out = Z;
+    if (m == -INFINITY || !(Z > 0.0) || Z != Z) bad = 1;
+    return bad;
+}
+
+static inline double prob_at(const void* base, int dtype, int64_t row, int64_t stride, int v,
+                             double T, double m, double Z)
+{
+    return exp(logit_at(base, dtype, row, stride, v) / T - m) / Z;
+}
+
+/* Full probability row (used by the pins and by small-case parity checks). */
+int orc_softmax_row(const void* base, int dtype, int64_t row, int64_t stride, int V,
+                    double temperature, double* probs, double* m_out, double* Z_out)
+{
+    double m, Z;
+    int bad = row_softmax_stats(base, dtype, row, stride, V, temperature, &m, &Z);
+    for (int v = 0; v < V; ++v) probs[v] = prob_at(base, dtype, row, stride, v, temperature, m, Z);
+    if (m_out) *m_out = m;
+    if (Z_out) *Z_out = Z;
+    return bad;
+}
+
+/* Inverse CDF over p in vocabulary order: smallest v with sum_{i<=v} p_i > thr.
+ * If rounding leaves the running sum at or below thr, the last v with p_v > 0. */
+static int32_t sample_from_p(const void* base, int dtype, int64_t row, int64_t stride, int V,
+                             double T, double m, double Z, double thr, double* margin)
+{
+    double cum = 0.0;
+    int32_t last_pos = -1;
+    for (int v = 0; v < V; ++v) {
+        double pv = prob_at(base, dtype, row, stride, v, T, m, Z);
+        double prev = cum;
+        cum += pv;
+        if (pv > 0.0) last_pos = v;
+        if (cum > thr) {
+            double d0 = thr - prev, d1 = cum - thr;
+            *margin = d0 < d1 ? d0 : d1;
+            return v;
+        }
+    }
+    *margin = 0.0;
+    return last_pos;
+}
+
+typedef struct {
+    const void* target; const void* draft; int dtype;
+    int64_t tstride, dstride; int V;
+    const int32_t* row_offsets; const int64_t* draft_row_start; const int32_t* draft_tokens;
+    int R; double T; uint64_t seed; int eval_all;
+    int32_t* accepted_len; int32_t* out_tokens;
+    double* p_tok; double* q_tok; double* accept_margin; double* token_margin;
+    int32_t* status;
+    int r_begin, r_end;
+} verify_job_t;
+
+static void verify_request(const verify_job_t* J, int r)
+{
+    int32_t lo = J->row_offsets[r], hi = J->row_offsets[r + 1];
+    J->token_margin[r] = NAN;
+    if (lo < 0 || hi - lo < 1) { J->status[r] = ORC_ST_BAD_OFFSETS; J->accepted_len[r] = 0; return; }
+    int32_t len = hi - lo - 1;
+    int64_t drow0 = J->draft_row_start ? J->draft_row_start[r] : (int64_t)lo - (int64_t)r;
+    int32_t st = 0;
+    for (int32_t i = lo; i < hi; ++i) {
+        J->out_tokens[i] = -1;
+        if (J->p_tok) J->p_tok[i] = NAN;
+        if (J->q_tok) J->q_tok[i] = NAN;
+        if (J->accept_margin) J->accept_margin[i] = NAN;
+    }
+    for (int32_t j = 0; j < len; ++j) {
+        int32_t d = J->draft_tokens[lo + j];
+        if (d < 0 || d >= J->V) st |= ORC_ST_BAD_TOKEN;
+    }
+    if (st) { J->status[r] = st; J->accepted_len[r] = 0; return; }
+
+    int32_t n = len;           /* first rejected position, or len */
+    for (int32_t j = 0; j < len; ++j) {
+        if (n < len && !J->eval_all) break;   /* verification stops at the first rejection */
+        double mp, Zp, mq, Zq;
+        int bad = row_softmax_stats(J->target, J->dtype, lo + j, J->tstride, J->V, J->T, &mp, &Zp);
+        bad |= row_softmax_stats(J->draft, J->dtype, drow0 + j, J->dstride, J->V, J->T, &mq, &Zq);
+        if (bad) { st |= ORC_ST_BAD_ROW; break; }
+        int32_t d = J->draft_tokens[lo + j];
+        double p = prob_at(J->target, J->dtype, lo + j, J->tstride, d, J->T, mp, Zp);
+        double q = prob_at(J->draft, J->dtype, drow0 + j, J->dstride, d, J->T, mq, Zq);
+        if (J->p_tok) J->p_tok[lo + j] = p;
+        if (J->q_tok) J->q_tok[lo + j] = q;
+        float ua, ur;
+        orc_uniforms(J->seed, (uint32_t)r, (uint32_t)j, &ua, &ur);
+        double lhs = (double)ua * q;
+        if (J->accept_margin) {
+            double big = p > q ? p : q;
+            J->accept_margin[lo + j] = big > 0.0 ? fabs(lhs - p) / big : 0.0;
+        }
+        int accept = lhs < p;      /* u < p/q without the division; u in [0,1) */
+        if (!accept && j < n) n = j;
+    }
+    if (st) { J->status[r] = st; J->accepted_len[r] = 0; return; }
+
+    float ua, ur;
+    orc_uniforms(J->seed, (uint32_t)r, (uint32_t)n, &ua, &ur);
+    int32_t tok = -1;
+    double margin = 0.0;
+    double mp, Zp;
+    if (row_softmax_stats(J->target, J->dtype, lo + n, J->tstride, J->V, J->T, &mp, &Zp)) {
+        J->status[r] = ORC_ST_BAD_ROW; J->accepted_len[r] = 0; return;
+    }
+    int resampled = 0;
+    if (n < len) {
+        /* residual norm(max(0, p - q)) at the rejected position */
+        double mq, Zq;
+        row_softmax_stats(J->draft, J->dtype, drow0 + n, J->dstride, J->V, J->T, &mq, &Zq);
+        double W = 0.0;
+        for (int v = 0; v < J->V; ++v) {
+            double pv = prob_at(J->target, J->dtype, lo + n, J->tstride, v, J->T, mp, Zp);
+            double qv = prob_at(J->draft, J->dtype, drow0 + n, J->dstride, v, J->T, mq, Zq);
+            double w = pv - qv;
+            if (w > 0.0) W += w;
+        }
+        if (W > 0.0) {
+            double thr = (double)ur * W;
+            double cum = 0.0;
+            int32_t last_pos = -1;
+            for (int v = 0; v < J->V; ++v) {
+                double pv = prob_at(J->target, J->dtype, lo + n, J->tstride, v, J->T, mp, Zp);
+                double qv = prob_at(J->draft, J->dtype, drow0 + n, J->dstride, v, J->T, mq, Zq);
+                double w = pv - qv;
+                if (!(w > 0.0)) continue;
+                double prev = cum;
+                cum += w;
+                last_pos = v;
+                if (cum > thr) {
+                    double d0 = thr - prev, d1 = cum - thr;
+                    margin = (d0 < d1 ? d0 : d1) / W;
+                    tok = v;
+                    break;
+                }
+            }
+            if (tok < 0) { tok = last_pos; margin = 0.0; }
+            resampled = 1;
+        }
+    }
+    if (!resampled) {
+        /* bonus token from p of row n (also the fallback when the residual is empty) */
+        tok = sample_from_p(J->target, J->dtype, lo + n, J->tstride, J->V, J->T, mp, Zp, (double)ur, &margin);
+    }
+    for (int32_t j = 0; j < n; ++j) J->out_tokens[lo + j] = J->draft_tokens[lo + j];
+    J->out_tokens[lo + n] = tok;
+    J->accepted_len[r] = n;
+    J->token_margin[r] = margin;
+    J->status[r] = st;
+}
+
+static void* verify_worker(void* arg)
+{
+    const verify_job_t* J = (const verify_job_t*)arg;
+    for (int r = J->r_begin; r < J->r_end; ++r) verify_request(J, r);
+    return NULL;
+}
+
+/*
+ * eval_all != 0 evaluates p(d), q(d) and the accept margin at every draft
+ * position (for parity checks); otherwise evaluation stops at the first
+ * rejection, as verification itself does.  n_threads splits requests over
+ * pthreads (requests are independent); results do not depend on it.
+ */
+int orc_verify(const void* target, const void* draft, int dtype,
+               int64_t target_row_stride, int64_t draft_row_stride, int V,
+               const int32_t* row_offsets, const int64_t* draft_row_start,
+               const int32_t* draft_tokens, int R, double temperature, uint64_t seed,
+               int eval_all, int n_threads,
+               int32_t* accepted_len, int32_t* out_tokens,
+               double* p_tok, double* q_tok, double* accept_margin, double* token_margin,
+               int32_t* status)
+{
+    if (R <= 0 || V <= 0 || !(temperature > 0.0) || !isfinite(temperature)) return -1;
+    if (n_threads < 1) n_threads = 1;
+    if (n_threads > R) n_threads = R;
+    if (n_threads > 256) n_threads = 256;
+    verify_job_t base = { target, draft, dtype, target_row_stride, draft_row_stride, V,
+                          row_offsets, draft_row_start, draft_tokens, R, temperature, seed, eval_all,
+                          accepted_len, out_tokens, p_tok, q_tok, accept_margin, token_margin,
+                          status, 0, R };
+    if (n_threads == 1) { verify_worker(&base); return 0; }
+    pthread_t th[256];
+    verify_job_t jobs[256];
+    for (int t = 0; t < n_threads; ++t) {
+        jobs[t] = base;
+        jobs[t].r_begin = (int)((long)R * t / n_threads);
+        jobs[t].r_end = (int)((long)R * (t + 1) / n_threads);
+        pthread_create(&th[t], NULL, verify_worker, &jobs[t]);
+    }
+    for (int t = 0; t < n_threads; ++t) pthread_join(th[t], NULL);
+    return 0;
+}
+
+/* Threaded wrapper for the greedy verifier's timing leg (same results). */
+typedef struct {
+    const void* target; int dtype; int64_t stride; int V;
+    const int32_t* row_offsets; const int32_t* draft_tokens;
+    int32_t* accepted_len; int32_t* out_tokens; int32_t* status; int r_begin, r_end;
+} greedy_job_t;
+
+static void* greedy_worker(void* arg)
+{
+    greedy_job_t* G = (greedy_job_t*)arg;
+    /* each slice is an independent batch over a window of the offsets array */
+    orc_verify_greedy(G->target, G->dtype, G->stride, G->V, G->row_offsets + G->r_begin,
+                      G->draft_tokens, G->r_end - G->r_begin,
+                      G->accepted_len + G->r_begin, G->out_tokens, NULL, G->status + G->r_begin);
+    return NULL;
+}
+
+int orc_verify_greedy_mt(const void* target, int dtype, int64_t target_row_stride, int V,
+                         const int32_t* row_offsets, const int32_t* draft_tokens, int R,
+                         int n_threads, int32_t* accepted_len, int32_t* out_tokens, int32_t* status)
+{
+    if (R <= 0 || V <= 0) return -1;
+    if (n_threads < 1) n_threads = 1;
+    if (n_threads > R) n_threads = R;
+    if (n_threads > 256) n_threads = 256;
+    pthread_t th[256];
+    greedy_job_t jobs[256];
+    for (int t = 0; t < n_threads; ++t) {
+        greedy_job_t g = { target, dtype, target_row_stride, V, row_offsets, draft_tokens,
+                           accepted_len, out_tokens, status,
+                           (int)((long)R * t / n_threads), (int)((long)R * (t + 1) / n_threads) };
+        jobs[t] = g;
+        if (g.r_end > g.r_begin) pthread_create(&th[t], NULL, greedy_worker, &jobs[t]);
+    }
+    for (int t = 0; t < n_threads; ++t)
+        if (jobs[t].r_end > jobs[t].r_begin) pthread_join(th[t], NULL);
+    return 0;
+}
