@@ -1,0 +1,218 @@
+/*
+ * dspark.h -- C ABI of the B200 (sm_100a) hot path of DSpark's serving step:
+ * the confidence-scheduled verification-length scheduler and the fused
+ * ragged-batch speculative verifier.
+ *
+ * Conventions for every entry point
+ *  - "device" pointers are CUDA global-memory addresses on the current device,
+ *    "host" pointers are ordinary process memory.  The caller owns every buffer;
+ *    the library allocates only inside dspark_profile_create / dspark_ktimer_create.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    Calls enqueue kernels on it and return; they never synchronise and never read
+ *    device data on the host.
+ *  - Return value: DSPARK_OK (0) or one of the positive error codes below.  Host-detectable
+ *    problems (NULL pointers, non-positive sizes, workspace too small, bad
+ *    temperature) return an error and launch nothing.  Problems only visible on the
+ *    device (bad offsets, token id outside [0,V), NaN rows, ...) set bits in the
+ *    int32 that `dev_status` points to (bits are OR-ed in; the caller zeroes it),
+ *    the affected request gets accepted_len = 0 and tokens -1; kernels never trap
+ *    and every device-side wait is bounded.
+ *  - Logit rows are row-major with unit inner stride; `*_row_stride` is in elements.
+ *    The bulk-copy fast path needs 16-byte aligned base pointers, row strides that
+ *    are multiples of 16 bytes and V*sizeof(elem) a multiple of 16; anything else
+ *    takes a slower element-wise path with identical results.
+ */
+#ifndef DSPARK_H
+#define DSPARK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DSPARK_OK = 0,
+    DSPARK_ERR_INVALID_ARG = 1,
+    DSPARK_ERR_SHAPE = 2,
+    DSPARK_ERR_ALIGNMENT = 3,
+    DSPARK_ERR_WORKSPACE = 4,
+    DSPARK_ERR_CUDA = 5,
+    DSPARK_ERR_TIMEOUT = 6
+} dspark_status_t;
+
+typedef enum { DSPARK_F32 = 0, DSPARK_BF16 = 1 } dspark_dtype_t;
+
+typedef enum {
+    DSPARK_SCHED_EARLY_STOP = 0, /* Algorithm 1 as printed: stop at the first non-improving admission */
+    DSPARK_SCHED_GLOBAL = 1,     /* Section 4.2: same path without the break, first maximiser wins */
+    DSPARK_SCHED_TOPK = 2        /* Section 4.2: admit the K most confident candidates (K from the caller) */
+} dspark_sched_mode_t;
+
+/* Bits OR-ed into *dev_status (verifier) and into dspark_sched_info_t.status (scheduler). */
+#define DSPARK_DEV_BAD_OFFSETS 1   /* row_offsets not increasing by >= 1, or beyond the n_rows capacity */
+#define DSPARK_DEV_BAD_TOKEN 2     /* a draft token id outside [0, V) */
+#define DSPARK_DEV_BAD_ROW 4       /* a logit row with NaN, +inf, or no finite element */
+#define DSPARK_DEV_TIMEOUT 8       /* a bounded device-side wait ran out */
+#define DSPARK_DEV_CONF_CLAMPED 16 /* a confidence was NaN, negative or above 1 (read as 0, 0, 1) */
+#define DSPARK_DEV_BUDGET_LT_R 32  /* token budget below the number of requests: every l*_r = 0 */
+#define DSPARK_DEV_ALL_NEG_INF 64  /* greedy: a row without any element above -inf (index 0 reported) */
+
+/* ------------------------------------------------------------------------------------
+ * Engine throughput profile SPS(B), steps per second at B batch tokens (Section 3.2.2:
+ * "profiled once during engine initialization and stored as a lightweight cost table").
+ *
+ * bp_tokens / bp_sps: host arrays of n_bp breakpoints, bp_tokens strictly increasing.
+ * The library builds a dense fp64 device table SPS[0..max_tokens]: piecewise linear
+ * between breakpoints, constant outside them (a step-wise curve is expressed by passing
+ * every B as a breakpoint).  Lookups beyond max_tokens use the last entry.
+ * Allocates device memory (cudaMalloc) and synchronises; call it at start-up.
+ * Errors: INVALID_ARG (NULL, n_bp < 1, max_tokens < 1, non-increasing tokens), CUDA.
+ */
+typedef struct dspark_profile dspark_profile_t;
+int dspark_profile_create(const int32_t* bp_tokens, const double* bp_sps, int n_bp,
+                          int max_tokens, dspark_profile_t** out);
+int dspark_profile_destroy(dspark_profile_t* prof);
+/* Device pointer to the fp64 table (max_tokens + 1 entries); owned by the profile. */
+const double* dspark_profile_table(const dspark_profile_t* prof, int* max_tokens);
+
+/* What the scheduler reports besides the lengths (device struct, 32 bytes). */
+typedef struct {
+    int32_t B;            /* batch tokens R + sum_r l*_r                         */
+    int32_t n_admitted;   /* admitted candidates i*                               */
+    int32_t status;       /* DSPARK_DEV_* warning bits                            */
+    int32_t n_candidates; /* |E|, candidates with positive survival probability   */
+    double tau;           /* expected accepted tokens R + sum of admitted a_{r,j} */
+    double theta;         /* tau * SPS(B), the objective reached                  */
+} dspark_sched_info_t;
+
+/* ------------------------------------------------------------------------------------
+ * dspark_schedule -- hardware-aware prefix scheduler (Algorithm 1; a, B, tau, Theta as
+ * defined in Section 3.2.2; no-break and top-K variants and the capacity limit from
+ * Section 4.2).
+ *
+ * Computes survival products a_{r,j} = prod_{i<=j} c_{r,i} (fp32, left to right), orders
+ * all candidates with a > 0 by (a descending, position ascending, request ascending),
+ * walks the admission path i = 1..min(|E|, budget_tokens - R) with
+ *     tau_i = R + sum of the first i survival values (exact, in units of 2^-40),
+ *     Theta_i = tau_i * SPS(R + i)   (one fp64 multiply),
+ * and stops per `mode`.  l*_r = number of admitted candidates of request r.
+ *
+ *  conf            device [R, gamma] fp32, row-major, c in [0,1] (NaN/<0 -> 0, >1 -> 1 with a warning bit)
+ *  draft_len       device [R] int32 or NULL: positions >= draft_len[r] are not candidates (NULL: gamma)
+ *  budget_tokens   cap on batch tokens B = R + sum l_r
+ *  topk_K          only for DSPARK_SCHED_TOPK
+ *  out_len         device [R] int32: l*_r
+ *  out_row_offsets device [R+1] int32 or NULL: exclusive scan of (l*_r + 1), the verifier's row_offsets
+ *  out_survival    device [R, gamma] fp32 or NULL: a_{r,j} (0 where not a candidate)
+ *  out_expected_len device [R] fp32 or NULL: 1 + sum_{j < l*_r} a_{r,j}
+ *  out_info        device dspark_sched_info_t or NULL
+ *  workspace       device scratch of at least dspark_schedule_workspace_bytes(R, gamma) bytes, 16-byte aligned
+ *
+ * Limits: 1 <= R <= 2^20, 0 <= gamma <= 4096, R*gamma <= 2^20.
+ * Errors: INVALID_ARG, SHAPE (limits), WORKSPACE, CUDA (launch failure).
+ */
+size_t dspark_schedule_workspace_bytes(int R, int gamma);
+int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32_t* draft_len,
+                    int R, int gamma, int budget_tokens, int mode, int topk_K,
+                    int32_t* out_len, int32_t* out_row_offsets, float* out_survival,
+                    float* out_expected_len, dspark_sched_info_t* out_info,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* row_offsets[0..R] = exclusive scan of (lengths[r] + 1): the flat ragged layout of
+ * Section 4.3 (all verified tokens of all requests flattened).  Device in, device out. */
+int dspark_build_offsets(const int32_t* lengths, int R, int32_t* row_offsets, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Ragged verification batch (both verifiers).
+ *  R requests; request r owns target rows [row_offsets[r], row_offsets[r+1]): l_r draft
+ *  positions followed by one bonus row, so row_offsets[r+1] - row_offsets[r] = l_r + 1 >= 1.
+ *  n_rows is the host-known CAPACITY of the flat arrays (target rows, draft_tokens,
+ *  out_tokens, out_p_tok, out_q_tok); the true row count is row_offsets[R] on the device
+ *  and must not exceed it.  draft_tokens[row_offsets[r] + j] is the token proposed at
+ *  position j < l_r (the bonus-row entry is ignored).
+ * Outputs: accepted_len[r] = n_r, the number of accepted draft tokens;
+ *  out_tokens[row_offsets[r] + i] = draft token for i < n_r, the corrected / bonus token
+ *  at i = n_r, -1 for i > n_r.  The request emits n_r + 1 tokens.
+ */
+size_t dspark_verify_workspace_bytes(int R, int n_rows, int V);
+
+/* dspark_verify_greedy -- a draft token is accepted iff it equals the argmax of its
+ * target row (lowest index on ties; NaN never wins; -0.0 ties +0.0); the first mismatch
+ * ends the prefix (Section 2.1: the first rejection discards all later tokens) and the
+ * argmax of that row is emitted; if every token matched, the argmax of the bonus row.
+ * target_logits: device [n_rows, V] of `dtype`.  One pass over the rows, no exponentials.
+ */
+int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_row_stride, int V,
+                         const int32_t* row_offsets, const int32_t* draft_tokens, int R, int n_rows,
+                         int32_t* accepted_len, int32_t* out_tokens, int32_t* dev_status,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* dspark_verify -- lossless sampling verification (Section 2.1): with p = softmax(target/T)
+ * and q = softmax(draft/T) at each position, token x is accepted with probability
+ * min(1, p(x)/q(x)), tested as  u * q(x) < p(x)  with u in [0,1) from Philox4x32-10 keyed by
+ * `seed` at counter (position, 0, request, 0), word 0.  Left to right; at the first rejection
+ * the emitted token is drawn from norm(max(0, p - q)) of that position, otherwise the bonus
+ * token is drawn from p of the last row (Section 1: longest accepted prefix plus one bonus
+ * token); both draws invert the CDF in vocabulary order with u' = word 1 of the same counter
+ * (position n_r): the smallest v whose running sum exceeds u' times the total.
+ *
+ *  draft_logits     device rows of `dtype`, same V.  draft_row_start == NULL: compact layout,
+ *                   the draft row of (r, j) is row_offsets[r] - r + j (needs n_rows - R rows of
+ *                   capacity).  Otherwise device [R] int64: the row of (r, j) is
+ *                   draft_row_start[r] + j (e.g. r * gamma for the drafter's full blocks).
+ *  temperature      T > 0, applied to both distributions.
+ *  out_p_tok/out_q_tok  device [n_rows] fp32 or NULL: p(x), q(x) at every draft position
+ *                   (bonus-row entries are not written).  When NULL, positions after the first
+ *                   rejection are not evaluated.
+ * Streams every target and draft row once (online softmax statistics per 2 KB block), then
+ * re-reads only the rejected position's row pair of each rejected request.
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE, CUDA.
+ */
+int dspark_verify(const void* target_logits, const void* draft_logits, int dtype,
+                  int64_t target_row_stride, int64_t draft_row_stride, int V,
+                  const int32_t* row_offsets, const int64_t* draft_row_start,
+                  const int32_t* draft_tokens, int R, int n_rows,
+                  float temperature, uint64_t seed,
+                  int32_t* accepted_len, int32_t* out_tokens,
+                  float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* The two uniforms of (seed, request, position) exactly as the verifier draws them
+ * (host computation; for tests and for replaying a step). */
+void dspark_uniforms(uint64_t seed, uint32_t request, uint32_t position,
+                     float* u_accept, float* u_resample);
+
+/* ------------------------------------------------------------------------------------
+ * Per-kernel device timing (measurement aid; the paper has no counterpart).
+ * While a timer is attached, every kernel the library launches is bracketed by a pair
+ * of CUDA events on the caller's stream; dspark_ktimer_read synchronises on them and
+ * returns, for one kernel id, the summed milliseconds and the number of launches.
+ * Not thread-safe; attach NULL to detach.  Launches beyond `capacity` are not recorded.
+ */
+typedef struct dspark_ktimer dspark_ktimer_t;
+enum {
+    DSPARK_K_SCHEDULE = 0, DSPARK_K_OFFSETS = 1, DSPARK_K_STREAM = 2, DSPARK_K_DECIDE = 3,
+    DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6,
+    DSPARK_K_GREEDY_DECIDE = 7, DSPARK_K_COUNT = 8
+};
+int dspark_ktimer_create(int capacity, dspark_ktimer_t** out);
+int dspark_ktimer_destroy(dspark_ktimer_t* t);
+int dspark_ktimer_attach(dspark_ktimer_t* t);
+int dspark_ktimer_reset(dspark_ktimer_t* t);
+int dspark_ktimer_read(dspark_ktimer_t* t, int kernel_id, float* total_ms, int* launches);
+
+/* Diagnostic switch for the streamed passes: 0 = automatic (bulk-copy pipeline when the
+ * 16-byte rules hold, direct loads otherwise), 1 = always direct loads.  Results are the
+ * same either way up to fp32 summation order.  Process-wide; the paper has no counterpart. */
+int dspark_set_stream_path(int path);
+
+const char* dspark_status_string(int status);
+const char* dspark_kernel_name(int kernel_id);
+int dspark_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSPARK_H */

@@ -1,0 +1,271 @@
+"""Thin ctypes binding over ``libdspark.so`` (declared in ``include/dspark.h``).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels.  The
+functions keep the C names and take torch CUDA tensors (device memory and streams
+are PyTorch's), returning the library's status code turned into an exception.
+There is no CPU fallback: a missing library or a CPU tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdspark.so")
+_lib: Optional[C.CDLL] = None
+
+DSPARK_F32, DSPARK_BF16 = 0, 1
+DSPARK_SCHED_EARLY_STOP, DSPARK_SCHED_GLOBAL, DSPARK_SCHED_TOPK = 0, 1, 2
+DEV_BAD_OFFSETS, DEV_BAD_TOKEN, DEV_BAD_ROW, DEV_TIMEOUT = 1, 2, 4, 8
+DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF = 16, 32, 64
+(K_SCHEDULE, K_OFFSETS, K_STREAM, K_DECIDE, K_RESIDUAL, K_FINALIZE,
+ K_GREEDY_STREAM, K_GREEDY_DECIDE, K_COUNT) = range(9)
+
+EXPORTS = [
+    "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",
+    "dspark_schedule_workspace_bytes", "dspark_schedule", "dspark_build_offsets",
+    "dspark_verify_workspace_bytes", "dspark_verify_greedy", "dspark_verify", "dspark_uniforms",
+    "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
+    "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
+    "dspark_version",
+]
+
+
+class DsparkError(RuntimeError):
+    pass
+
+
+class SchedInfo(C.Structure):
+    _fields_ = [("B", C.c_int32), ("n_admitted", C.c_int32), ("status", C.c_int32),
+                ("n_candidates", C.c_int32), ("tau", C.c_double), ("theta", C.c_double)]
+
+
+def lib() -> C.CDLL:
+    """Loads the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise DsparkError(f"{_LIB_PATH} is missing: run `python -m paper_2607_05147_b200.build` "
+                              "(there is no CPU fallback)")
+        L = C.CDLL(_LIB_PATH)
+        vp, i32, i64, u64, sz = C.c_void_p, C.c_int, C.c_int64, C.c_uint64, C.c_size_t
+        L.dspark_profile_create.argtypes = [vp, vp, i32, i32, C.POINTER(vp)]
+        L.dspark_profile_destroy.argtypes = [vp]
+        L.dspark_profile_table.argtypes = [vp, C.POINTER(C.c_int)]
+        L.dspark_profile_table.restype = vp
+        L.dspark_schedule_workspace_bytes.argtypes = [i32, i32]
+        L.dspark_schedule_workspace_bytes.restype = sz
+        L.dspark_schedule.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.dspark_build_offsets.argtypes = [vp, i32, vp, vp]
+        L.dspark_verify_workspace_bytes.argtypes = [i32, i32, i32]
+        L.dspark_verify_workspace_bytes.restype = sz
+        L.dspark_verify_greedy.argtypes = [vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.dspark_verify.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, C.c_float, u64,
+                                    vp, vp, vp, vp, vp, vp, sz, vp]
+        L.dspark_uniforms.argtypes = [u64, C.c_uint32, C.c_uint32, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+        L.dspark_uniforms.restype = None
+        L.dspark_ktimer_create.argtypes = [i32, C.POINTER(vp)]
+        L.dspark_ktimer_destroy.argtypes = [vp]
+        L.dspark_ktimer_attach.argtypes = [vp]
+        L.dspark_ktimer_reset.argtypes = [vp]
+        L.dspark_ktimer_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int)]
+        L.dspark_set_stream_path.argtypes = [i32]
+        L.dspark_status_string.argtypes = [i32]
+        L.dspark_status_string.restype = C.c_char_p
+        L.dspark_kernel_name.argtypes = [i32]
+        L.dspark_kernel_name.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise DsparkError(f"{what}: {lib().dspark_status_string(rc).decode()} ({rc})")
+
+
+def _dev(t: Optional[torch.Tensor], name: str, dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise DsparkError(f"{name} must be a CUDA tensor (no CPU path exists)")
+    if dtype is not None and t.dtype != dtype:
+        raise DsparkError(f"{name} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous() and t.dim() <= 1:
+        raise DsparkError(f"{name} must be contiguous")
+    return t.data_ptr()
+
+
+def _logits(t: torch.Tensor, name: str):
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise DsparkError(f"{name} must be 2-D with unit inner stride")
+    if t.dtype == torch.float32:
+        code = DSPARK_F32
+    elif t.dtype == torch.bfloat16:
+        code = DSPARK_BF16
+    else:
+        raise DsparkError(f"{name} must be float32 or bfloat16")
+    return _dev(t, name), code, t.stride(0)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+# ------------------------------------------------------------------------------- profile ----
+class Profile:
+    """Owner of a ``dspark_profile_t`` (device SPS table)."""
+
+    def __init__(self, bp_tokens, bp_sps, max_tokens: int):
+        n = len(bp_tokens)
+        bt = (C.c_int32 * n)(*[int(x) for x in bp_tokens])
+        bs = (C.c_double * n)(*[float(x) for x in bp_sps])
+        h = C.c_void_p()
+        _check(lib().dspark_profile_create(bt, bs, n, int(max_tokens), C.byref(h)), "dspark_profile_create")
+        self.handle = h
+        self.max_tokens = int(max_tokens)
+
+    def table(self) -> torch.Tensor:
+        """Copy of the device table as a host fp64 tensor (tests)."""
+        mt = C.c_int()
+        ptr = lib().dspark_profile_table(self.handle, C.byref(mt))
+
+        class _Raw:   # view of the library-owned device table through the CUDA array interface
+            __cuda_array_interface__ = {"shape": (mt.value + 1,), "typestr": "<f8", "data": (ptr, True), "version": 2}
+        return torch.as_tensor(_Raw(), device="cuda").clone().cpu()
+
+    def close(self):
+        if self.handle:
+            lib().dspark_profile_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def dspark_schedule_workspace_bytes(R: int, gamma: int) -> int:
+    return int(lib().dspark_schedule_workspace_bytes(R, gamma))
+
+
+def dspark_schedule(prof: Profile, conf: torch.Tensor, budget_tokens: int, mode: int = DSPARK_SCHED_EARLY_STOP,
+                    topk_K: int = 0, draft_len: Optional[torch.Tensor] = None, *, out_len: torch.Tensor,
+                    out_row_offsets: Optional[torch.Tensor] = None, out_survival: Optional[torch.Tensor] = None,
+                    out_expected_len: Optional[torch.Tensor] = None, out_info: Optional[torch.Tensor] = None,
+                    workspace: torch.Tensor) -> None:
+    """out_info: a 32-byte CUDA uint8 tensor receiving dspark_sched_info_t."""
+    if conf.dim() != 2 or not conf.is_contiguous():
+        raise DsparkError("conf must be a contiguous [R, gamma] tensor")
+    R, gamma = conf.shape
+    rc = lib().dspark_schedule(prof.handle, _dev(conf, "conf", torch.float32), _dev(draft_len, "draft_len", torch.int32),
+                               R, gamma, int(budget_tokens), int(mode), int(topk_K),
+                               _dev(out_len, "out_len", torch.int32), _dev(out_row_offsets, "out_row_offsets", torch.int32),
+                               _dev(out_survival, "out_survival", torch.float32),
+                               _dev(out_expected_len, "out_expected_len", torch.float32),
+                               _dev(out_info, "out_info", torch.uint8), _dev(workspace, "workspace"),
+                               workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_schedule")
+
+
+def read_sched_info(out_info: torch.Tensor) -> SchedInfo:
+    raw = bytes(out_info.cpu().numpy().tobytes())
+    return SchedInfo.from_buffer_copy(raw)
+
+
+def dspark_build_offsets(lengths: torch.Tensor, row_offsets: torch.Tensor) -> None:
+    _check(lib().dspark_build_offsets(_dev(lengths, "lengths", torch.int32), lengths.numel(),
+                                      _dev(row_offsets, "row_offsets", torch.int32), _stream()), "dspark_build_offsets")
+
+
+def dspark_verify_workspace_bytes(R: int, n_rows: int, V: int) -> int:
+    return int(lib().dspark_verify_workspace_bytes(R, n_rows, V))
+
+
+def dspark_verify_greedy(target: torch.Tensor, row_offsets: torch.Tensor, draft_tokens: torch.Tensor, *,
+                         accepted_len: torch.Tensor, out_tokens: torch.Tensor,
+                         dev_status: Optional[torch.Tensor], workspace: torch.Tensor,
+                         n_rows: Optional[int] = None) -> None:
+    tp, code, ts = _logits(target, "target")
+    R = row_offsets.numel() - 1
+    n_rows = target.shape[0] if n_rows is None else n_rows
+    rc = lib().dspark_verify_greedy(tp, code, ts, target.shape[1], _dev(row_offsets, "row_offsets", torch.int32),
+                                    _dev(draft_tokens, "draft_tokens", torch.int32), R, n_rows,
+                                    _dev(accepted_len, "accepted_len", torch.int32),
+                                    _dev(out_tokens, "out_tokens", torch.int32),
+                                    _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+                                    workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_verify_greedy")
+
+
+def dspark_verify(target: torch.Tensor, draft: torch.Tensor, row_offsets: torch.Tensor,
+                  draft_tokens: torch.Tensor, temperature: float, seed: int, *,
+                  draft_row_start: Optional[torch.Tensor] = None,
+                  accepted_len: torch.Tensor, out_tokens: torch.Tensor,
+                  out_p_tok: Optional[torch.Tensor] = None, out_q_tok: Optional[torch.Tensor] = None,
+                  dev_status: Optional[torch.Tensor], workspace: torch.Tensor,
+                  n_rows: Optional[int] = None) -> None:
+    tp, code, ts = _logits(target, "target")
+    dp, dcode, ds = _logits(draft, "draft")
+    if code != dcode or target.shape[1] != draft.shape[1]:
+        raise DsparkError("target and draft logits must share dtype and vocabulary size")
+    R = row_offsets.numel() - 1
+    n_rows = target.shape[0] if n_rows is None else n_rows
+    rc = lib().dspark_verify(tp, dp, code, ts, ds, target.shape[1], _dev(row_offsets, "row_offsets", torch.int32),
+                             _dev(draft_row_start, "draft_row_start", torch.int64),
+                             _dev(draft_tokens, "draft_tokens", torch.int32), R, n_rows,
+                             float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF,
+                             _dev(accepted_len, "accepted_len", torch.int32), _dev(out_tokens, "out_tokens", torch.int32),
+                             _dev(out_p_tok, "out_p_tok", torch.float32), _dev(out_q_tok, "out_q_tok", torch.float32),
+                             _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+                             workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_verify")
+
+
+def dspark_uniforms(seed: int, request: int, position: int):
+    a, b = C.c_float(), C.c_float()
+    lib().dspark_uniforms(int(seed) & 0xFFFFFFFFFFFFFFFF, request, position, C.byref(a), C.byref(b))
+    return a.value, b.value
+
+
+def dspark_set_stream_path(path: int) -> None:
+    _check(lib().dspark_set_stream_path(path), "dspark_set_stream_path")
+
+
+class KernelTimer:
+    """Per-kernel CUDA-event timing of the library's launches (measurement aid)."""
+
+    def __init__(self, capacity: int):
+        h = C.c_void_p()
+        _check(lib().dspark_ktimer_create(capacity, C.byref(h)), "dspark_ktimer_create")
+        self.handle = h
+
+    def attach(self):
+        lib().dspark_ktimer_reset(self.handle)
+        lib().dspark_ktimer_attach(self.handle)
+
+    def detach(self):
+        lib().dspark_ktimer_attach(None)
+
+    def read(self) -> dict:
+        out = {}
+        for k in range(K_COUNT):
+            ms, n = C.c_float(), C.c_int()
+            _check(lib().dspark_ktimer_read(self.handle, k, C.byref(ms), C.byref(n)), "dspark_ktimer_read")
+            if n.value:
+                out[lib().dspark_kernel_name(k).decode()] = {"ms": ms.value, "launches": n.value}
+        return out
+
+    def close(self):
+        if self.handle:
+            self.detach()
+            lib().dspark_ktimer_destroy(self.handle)
+            self.handle = None
+
+
+def workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A 256-byte aligned scratch buffer (torch allocations are 512-byte aligned)."""
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)

@@ -1,0 +1,165 @@
+// Shared device helpers for the DSpark sm_100a kernels: PTX wrappers (mbarrier,
+// bulk async copy, warp reductions), the counter-based RNG, launch bookkeeping.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dspark.h"
+
+namespace dspark {
+
+// ---------------------------------------------------------------------------------
+// Geometry of the streamed passes.  A logit row is cut into 2 KB blocks (one warp
+// each: 4 x 16 B per lane); 8 blocks form a 16 KB piece, the unit one bulk async
+// copy brings into one pipeline stage.
+// ---------------------------------------------------------------------------------
+constexpr int kBlockBytes = 2048;
+constexpr int kConsumerWarps = 8;
+constexpr int kPieceBytes = kBlockBytes * kConsumerWarps;   // 16 KB
+constexpr int kVecPerLane = kBlockBytes / (32 * 16);        // 4
+constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;   // + one producer warp
+
+// Upper bound on polls of one mbarrier phase before a kernel gives up (each poll may
+// itself block for a short hardware-defined time, so this is on the order of a second).
+constexpr uint32_t kWaitPollLimit = 1u << 22;
+
+__host__ __device__ inline int blocks_per_row(int V, int elem_bytes)
+{
+    long long bytes = (long long)V * elem_bytes;
+    return (int)((bytes + kBlockBytes - 1) / kBlockBytes);
+}
+__host__ __device__ inline int pieces_per_row(int V, int elem_bytes)
+{
+    return (blocks_per_row(V, elem_bytes) + kConsumerWarps - 1) / kConsumerWarps;
+}
+
+// ---------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_fence_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the poll limit ran out.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity)
+{
+    for (uint32_t i = 0; i < kWaitPollLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// 1-D bulk async copy global -> this CTA's shared memory, completion counted on `bar`.
+// dst, src 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2_approx(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// Warp-wide float max in one instruction (sm_100a redux); NaN inputs are ignored.
+__device__ __forceinline__ float warp_max_f32(float x)
+{
+    float y;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float warp_sum_f32(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+__device__ __forceinline__ double warp_sum_f64(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// ---------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11).  counter = (position, 0, request, 0), key = seed.
+// Word 0 -> accept uniform, word 1 -> resample uniform; u = (word >> 8) * 2^-24.
+// ---------------------------------------------------------------------------------
+__host__ __device__ inline void philox_round(uint32_t& c0, uint32_t& c1, uint32_t& c2, uint32_t& c3,
+                                             uint32_t k0, uint32_t k1)
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+#ifdef __CUDA_ARCH__
+    uint32_t hi0 = __umulhi(M0, c0), hi1 = __umulhi(M1, c2);
+#else
+    uint32_t hi0 = (uint32_t)(((uint64_t)M0 * c0) >> 32), hi1 = (uint32_t)(((uint64_t)M1 * c2) >> 32);
+#endif
+    uint32_t lo0 = M0 * c0, lo1 = M1 * c2;
+    uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+}
+__host__ __device__ inline void philox_uniforms(uint64_t seed, uint32_t request, uint32_t position,
+                                                float& u_accept, float& u_resample)
+{
+    uint32_t c0 = position, c1 = 0u, c2 = request, c3 = 0u;
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        philox_round(c0, c1, c2, c3, k0, k1);
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    u_accept = (float)(c0 >> 8) * (1.0f / 16777216.0f);
+    u_resample = (float)(c1 >> 8) * (1.0f / 16777216.0f);
+}
+
+// ---------------------------------------------------------------------------------
+// Host-side launch bookkeeping (per-kernel event timing, error mapping)
+// ---------------------------------------------------------------------------------
+struct KernelTimerScope {
+    KernelTimerScope(int kernel_id, cudaStream_t stream);
+    ~KernelTimerScope();
+    int slot;
+    cudaStream_t stream;
+};
+int launch_status();   // maps cudaGetLastError() to DSPARK_OK / DSPARK_ERR_CUDA
+
+}  // namespace dspark

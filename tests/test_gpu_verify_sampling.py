@@ -1,0 +1,169 @@
+"""GPU sampling verifier vs the CPU oracle.  Bars: accepted lengths and tokens bit-exact except
+where the oracle's margin to a decision boundary is below 1e-6 (counted and printed);
+p(x), q(x) within 1e-5 relative."""
+import numpy as np
+import pytest
+import torch
+from scipy import stats
+
+import helpers as H
+from paper_2607_05147_b200 import binding as B
+from paper_2607_05147_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _report(name, batch, g, mism):
+    lens = batch.meta["lengths"].cpu().numpy()
+    print(f"[{name}] requests={batch.R} rows={batch.n_rows} mean_len={lens.mean():.2f} "
+          f"mean_accepted={g['acc'].mean():.2f} rejected={(g['acc'] < lens).mean():.2f} "
+          f"boundary_mismatches={mism} ({mism / batch.R:.2e} per request)")
+
+
+def test_config_2_reduced():
+    batch = W.config_2("cuda", R=16)
+    g, o, mism = H.check_sampling(batch)
+    _report("cfg2/R=16", batch, g, mism)
+
+
+def test_config_2_full_size():
+    batch = W.config_2("cuda")
+    g, o, mism = H.check_sampling(batch)
+    _report("cfg2", batch, g, mism)
+    assert mism <= 1
+    # the run without probability outputs (stops at the first rejection) gives the same tokens
+    g2 = H.gpu_verify(batch, want_probs=False)
+    np.testing.assert_array_equal(g2["acc"], g["acc"])
+    np.testing.assert_array_equal(g2["out"], g["out"])
+
+
+def test_config_3_full_size_scheduled_then_verified():
+    sched = W.config_3_schedule("cuda")
+    gs, _ = H.check_schedule(sched, B.DSPARK_SCHED_EARLY_STOP)
+    batch = W.config_3_batch(torch.from_numpy(gs["lengths"]), "cuda")
+    assert torch.equal(batch.row_offsets.cpu(), torch.from_numpy(gs["offsets"]))
+    g, o, mism = H.check_sampling(batch)
+    _report("cfg3", batch, g, mism)
+    assert mism <= 2
+
+
+def test_config_5_full_size_scheduled_then_verified():
+    sched = W.config_5_schedule("cuda")
+    gs, _ = H.check_schedule(sched, B.DSPARK_SCHED_EARLY_STOP)
+    batch = W.config_5_batch(torch.from_numpy(gs["lengths"]), "cuda")
+    g, o, mism = H.check_sampling(batch)
+    _report("cfg5", batch, g, mism)
+    assert mism <= 3
+    lens = gs["lengths"]
+    assert (g["acc"] < lens).mean() > 0.3          # high rejection rate: the residual pass is exercised
+
+
+@pytest.mark.parametrize("V", [2, 16, 1000, 4097, 129281])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_odd_vocabularies_dtypes_and_paths(V, dtype):
+    lengths = torch.tensor([3, 0, 1, 6, 2, 0, 4, 8, 1])
+    batch = W.sampling_batch(lengths, V, 70 + V, "cuda", dtype=dtype, temperature=0.9, verify_seed=V)
+    g, o, mism = H.check_sampling(batch)
+    B.dspark_set_stream_path(1)
+    try:
+        g1, o1, mism1 = H.check_sampling(batch)
+    finally:
+        B.dspark_set_stream_path(0)
+    assert mism + mism1 <= 1
+    np.testing.assert_array_equal(g["acc"], g1["acc"])
+
+
+def test_compact_and_block_layouts_agree():
+    lengths = torch.tensor([2, 5, 0, 3, 1, 7])
+    a = W.sampling_batch(lengths, 20000, 3, "cuda", verify_seed=5)
+    b = W.sampling_batch(lengths, 20000, 3, "cuda", verify_seed=5, block=8)
+    ga, _, _ = H.check_sampling(a)
+    gb, _, _ = H.check_sampling(b)
+    np.testing.assert_array_equal(ga["acc"], gb["acc"])
+    np.testing.assert_array_equal(ga["out"], gb["out"])
+
+
+def test_padded_strides_and_capacity():
+    lengths = torch.tensor([2, 0, 4, 1])
+    b = W.sampling_batch(lengths, 3000, 8, "cuda", verify_seed=3)
+    tp = torch.zeros(b.n_rows + 3, 3080, dtype=torch.bfloat16, device="cuda"); tp[: b.n_rows, :3000] = b.target
+    dp = torch.zeros(b.draft.shape[0], 3008, dtype=torch.bfloat16, device="cuda"); dp[:, :3000] = b.draft
+    toks = torch.zeros(b.n_rows + 3, dtype=torch.int32, device="cuda"); toks[: b.n_rows] = b.draft_tokens
+    padded = W.VerifyBatch(tp[:, :3000], dp[:, :3000], b.row_offsets, toks, None, b.temperature, b.seed, b.meta)
+    g0, _, _ = H.check_sampling(b)
+    g1 = H.gpu_verify(padded)
+    np.testing.assert_array_equal(g0["acc"], g1["acc"])
+    np.testing.assert_array_equal(g0["out"][: b.n_rows], g1["out"][: b.n_rows])
+    assert (g1["out"][b.n_rows:] == -7).all()
+
+
+def test_degenerate_batches():
+    V = 5000
+    lengths = torch.tensor([4, 4, 4, 0, 0])
+    b = W.sampling_batch(lengths, V, 21, "cuda", verify_seed=9)
+    # draft == target: every token accepted (u < 1), bonus from p
+    same = W.VerifyBatch(b.target, b.target[[0, 1, 2, 3, 5, 6, 7, 8, 10, 11, 12, 13]].contiguous(), b.row_offsets,
+                         b.draft_tokens, None, 1.0, 9, b.meta)
+    g, o, _ = H.check_sampling(same)
+    assert (g["acc"] == lengths.numpy()).all()
+    # target -inf at the draft token: p(x) = 0, always rejected, residual never returns x
+    t = b.target.clone()
+    off = b.row_offsets.cpu().numpy()
+    for r in range(3):
+        t[off[r], b.draft_tokens[off[r]].item()] = float("-inf")
+    rej = W.VerifyBatch(t, b.draft, b.row_offsets, b.draft_tokens, None, 1.0, 9, b.meta)
+    g, o, _ = H.check_sampling(rej)
+    assert (g["acc"][:3] == 0).all()
+    for r in range(3):
+        assert g["out"][off[r]] != b.draft_tokens[off[r]].item()
+    # NaN row, +inf row, all -inf row, bad token: flagged, nothing emitted, others unaffected
+    t2 = b.target.clone(); t2[off[0] + 1, 17] = float("nan"); t2[off[1], :] = float("-inf"); t2[off[2], 5] = float("inf")
+    toks = b.draft_tokens.clone(); toks[off[4] - 1] = 0
+    bad = W.VerifyBatch(t2, b.draft, b.row_offsets, toks, None, 1.0, 9, b.meta)
+    g, o, _ = H.check_sampling(bad)
+    assert g["status"] & B.DEV_BAD_ROW and (g["acc"][:3] == 0).all() and g["out"][off[3]] >= 0
+    toks[off[0]] = V
+    g, o, _ = H.check_sampling(W.VerifyBatch(b.target, b.draft, b.row_offsets, toks, None, 1.0, 9, b.meta))
+    assert g["status"] & B.DEV_BAD_TOKEN
+
+
+def test_lossless_invariant_on_the_gpu():
+    # first emitted token ~ p whatever q is (chi-square, V = 16, 60k single-position requests)
+    rng = np.random.default_rng(5)
+    V, n = 16, 60_000
+    p = rng.dirichlet(np.ones(V) * 0.6); q = rng.dirichlet(np.ones(V) * 0.6)
+    tl = torch.tensor(np.log(p), dtype=torch.float32); ql = torch.tensor(np.log(q), dtype=torch.float32)
+    target = tl.repeat(2 * n, 1).cuda(); draft = ql.repeat(n, 1).cuda()
+    pp = torch.softmax(tl.double(), 0).numpy(); qq = torch.softmax(ql.double(), 0).numpy()
+    toks = torch.zeros(2 * n, dtype=torch.int32); toks[0::2] = torch.from_numpy(rng.choice(V, size=n, p=qq)).int()
+    off = (2 * torch.arange(n + 1)).int()
+    batch = W.VerifyBatch(target, draft, off.cuda(), toks.cuda(), None, 1.0, 123, {"lengths": torch.ones(n)})
+    g = H.gpu_verify(batch, want_probs=False)
+    first = g["out"][0::2]
+    assert stats.chisquare(np.bincount(first, minlength=V), pp * n).pvalue > 1e-3
+    want = 1 - 0.5 * np.abs(pp - qq).sum()
+    assert abs(g["acc"].mean() - want) < 4 * np.sqrt(want * (1 - want) / n)
+    bonus = g["out"][1::2][g["acc"] == 1]
+    assert stats.chisquare(np.bincount(bonus, minlength=V), pp * len(bonus)).pvalue > 1e-3
+
+
+def test_results_are_reproducible_run_to_run():
+    batch = W.config_2("cuda", R=24)
+    a = H.gpu_verify(batch)
+    for _ in range(3):
+        b = H.gpu_verify(batch)
+        for k in ("acc", "out", "p", "q"):
+            np.testing.assert_array_equal(a[k], b[k])
+
+
+def test_host_side_errors():
+    b = W.sampling_batch(torch.tensor([1, 2]), 512, 1, "cuda")
+    acc = torch.zeros(2, dtype=torch.int32, device="cuda"); out = torch.zeros(5, dtype=torch.int32, device="cuda")
+    ws = B.workspace(B.dspark_verify_workspace_bytes(2, 5, 512))
+    for T in (0.0, -1.0, float("nan"), float("inf")):
+        with pytest.raises(B.DsparkError, match="invalid"):
+            B.dspark_verify(b.target, b.draft, b.row_offsets, b.draft_tokens, T, 1, accepted_len=acc,
+                            out_tokens=out, dev_status=None, workspace=ws)
+    with pytest.raises(B.DsparkError, match="workspace"):
+        B.dspark_verify(b.target, b.draft, b.row_offsets, b.draft_tokens, 1.0, 1, accepted_len=acc,
+                        out_tokens=out, dev_status=None, workspace=torch.empty(512, dtype=torch.uint8, device="cuda"))
