@@ -133,7 +133,7 @@ class Profile:
         ptr = lib().dspark_profile_table(self.handle, C.byref(mt))
 
         class _Raw:   # view of the library-owned device table through the CUDA array interface
-            __cuda_array_interface__ = {"shape": (mt.value + 1,), "typestr": "<f8", "data": (ptr, True), "version": 2}
+            __cuda_array_interface__ = {"shape": (mt.value + 1,), "typestr": "<f8", "data": (ptr, False), "version": 2}
         return torch.as_tensor(_Raw(), device="cuda").clone().cpu()
 
     def close(self):

@@ -182,7 +182,7 @@ def greedy_batch(lengths: torch.Tensor, V: int, seed: int, device, *, sigma=4.0,
         keep = u < torch.as_tensor(match_prob, device=device, dtype=torch.float32)[pos.clamp_max(len(match_prob) - 1)]
     else:
         keep = u >= (perturb or 0.0)
-    other = (am.to(torch.int64) + torch.randint(1, V, (n_rows,), generator=g, device=device)) % V
+    other = (am.to(torch.int64) + torch.randint(1, max(V, 2), (n_rows,), generator=g, device=device)) % V
     tokens = torch.where(keep, am, other.to(torch.int32))
     tokens[pos == lengths[req]] = 0                             # bonus-row entries are ignored
     return VerifyBatch(target, None, off, tokens.contiguous(), None, 1.0, seed, {"lengths": lengths})

@@ -67,9 +67,10 @@ def test_special_values_and_device_errors():
     b = W.greedy_batch(lengths, 5000, 9, "cuda", perturb=0.0)
     t = b.target
     t[0, 7] = float("nan"); t[1, :] = float("-inf"); t[2, 100] = float("inf")
-    t[4] = -1.0; t[4, 4000] = 0.0; t[4, 3000] = -0.0            # -0.0 ties +0.0: lowest index wins
+    i4 = int(b.row_offsets[4])
+    t[i4] = -1.0; t[i4, 4000] = 0.0; t[i4, 3000] = -0.0         # -0.0 ties +0.0: lowest index wins
     acc, out, o = H.check_greedy(b)
-    assert out[int(b.row_offsets[4])] == 3000
+    assert out[i4] == 3000
     b.draft_tokens[0] = 5000                                     # token id out of range
     acc, out, _ = H.check_greedy(b)
     assert acc[0] == 0 and out[0] == -1
