@@ -1,0 +1,506 @@
+#!/usr/bin/env python
+"""Benchmark of the DSpark hot path on B200: one step = schedule -> ragged offsets ->
+fused verification of one synthetic batch, through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is verified target rows per second over all GPUs with the
+inputs resident in HBM; `e2e` is the same metric with the step's inputs copied from pinned
+host memory and its results copied back inside the timed region; `roofline` is the dominant
+kernel against the measured HBM peak; `cpu_baseline` times the CPU oracle on the same batch.
+Multi-GPU runs are independent replicas (requests are independent and the scheduler is per
+engine), one process per GPU under torchrun; time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "verified rows/sec and achieved HBM GB/s (% of B200 peak) at V=129280, 1 GPU"
+UNIT = "rows/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126 * 1024 * 1024
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture of that workload exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+# ----------------------------------------------------------------------------- workloads ----
+def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=False):
+    """Returns a dict describing the step: schedule input (or None) and a list of batches that
+    differ only in their logits (rotated so consecutive steps never touch the same bytes).
+    n_sets None: as many batches as it takes to exceed four times the L2 capacity."""
+    from paper_2607_05147_b200 import workloads as W
+    sched = None
+    greedy = False
+    if name == "cfg3":
+        sched = W.config_3_schedule(device)
+        desc = "Confidence-scheduled, high concurrency: 256 requests, V=129280, blocks of 16, budget 1024, bf16 sampling"
+    elif name == "cfg5":
+        sched = W.config_5_schedule(device)
+        desc = "Long-block stress: 512 requests, V=129280, blocks of 32, budget 4096, bf16 sampling T=0.7"
+    elif name == "cfg2":
+        desc = "Sampling, moderate batch: 64 requests, V=129280, ragged k~U{1..8}, bf16, T=1"
+    elif name == "cfg4":
+        greedy = True
+        desc = "Large batch greedy: 1024 requests, V=129280, ragged k~U{0..8}, fp32"
+    else:
+        raise SystemExit(f"unknown workload {name}")
+
+    lengths = None
+    prof = None
+    if sched is not None:
+        # the schedule is fixed by the confidences: run it once to size the logits
+        if oracle_schedule:
+            import oracle
+            tab = oracle.sps_table(sched.bp_tokens, sched.bp_sps, sched.max_tokens)
+            lengths = torch.from_numpy(oracle.schedule(sched.conf.cpu().numpy(), tab, sched.budget_tokens,
+                                                       oracle.MODE_EARLY_STOP).lengths)
+        else:
+            from paper_2607_05147_b200 import binding as B
+            prof = B.Profile(sched.bp_tokens, sched.bp_sps, sched.max_tokens)
+            R, gamma = sched.conf.shape
+            out_len = torch.zeros(R, dtype=torch.int32, device=device)
+            ws = B.workspace(B.dspark_schedule_workspace_bytes(R, gamma))
+            B.dspark_schedule(prof, sched.conf, sched.budget_tokens, B.DSPARK_SCHED_EARLY_STOP, out_len=out_len,
+                              workspace=ws)
+            torch.cuda.synchronize()
+            lengths = out_len.cpu()
+
+    def one(k):
+        seed = 5000 + 97 * rank + k
+        if name == "cfg3":
+            return W.sampling_batch(lengths, W.V_FULL, seed, device, temperature=1.0, draft_noise=1.0, verify_seed=2)
+        if name == "cfg5":
+            return W.sampling_batch(lengths, W.V_FULL, seed, device, temperature=0.7, draft_noise=2.0, verify_seed=4)
+        if name == "cfg2":
+            g = torch.Generator(device="cpu"); g.manual_seed(1)
+            ln = torch.randint(1, 9, (64,), generator=g)
+            return W.sampling_batch(ln, W.V_FULL, seed, device, temperature=1.0, draft_noise=1.0, verify_seed=1)
+        g = torch.Generator(device="cpu"); g.manual_seed(3)
+        ln = torch.randint(0, 9, (1024,), generator=g)
+        return W.greedy_batch(ln, W.V_FULL, seed, device, sigma=4.0, tie_frac=0.01,
+                              match_prob=[0.85 ** (j + 1) for j in range(8)])
+
+    batches = [one(0)]
+    if n_sets is None:
+        stream_b, _ = algorithmic_bytes(batches[0], greedy, 0)
+        n_sets = max(2, min(8, -(-4 * L2_BYTES // stream_b)))
+    for k in range(1, n_sets):
+        batches.append(one(k))
+    return dict(name=name, desc=desc, sched=sched, prof=prof, batches=batches, greedy=greedy)
+
+
+class Step:
+    """Device buffers + the calls of one step (all through the C ABI binding)."""
+
+    def __init__(self, wl, device):
+        from paper_2607_05147_b200 import binding as B
+        self.B = B
+        self.wl = wl
+        b0 = wl["batches"][0]
+        self.R, self.n_rows, self.V = b0.R, b0.n_rows, b0.V
+        self.acc = torch.zeros(self.R, dtype=torch.int32, device=device)
+        self.out = torch.zeros(self.n_rows, dtype=torch.int32, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.ws = B.workspace(B.dspark_verify_workspace_bytes(self.R, self.n_rows, self.V))
+        self.sched = wl["sched"]
+        if self.sched is not None:
+            R, gamma = self.sched.conf.shape
+            self.out_len = torch.zeros(R, dtype=torch.int32, device=device)
+            self.offsets = torch.zeros(R + 1, dtype=torch.int32, device=device)
+            self.sws = B.workspace(B.dspark_schedule_workspace_bytes(R, gamma))
+        self.launches_per_step = (1 if self.sched is not None else 0) + (2 if wl["greedy"] else 4)
+
+    def run(self, batch, conf=None):
+        B = self.B
+        offsets = batch.row_offsets
+        if self.sched is not None:
+            B.dspark_schedule(self.wl["prof"], self.sched.conf if conf is None else conf, self.sched.budget_tokens,
+                              B.DSPARK_SCHED_EARLY_STOP, out_len=self.out_len, out_row_offsets=self.offsets,
+                              workspace=self.sws)
+            offsets = self.offsets            # the verifier reads the schedule's offsets from device memory
+        if self.wl["greedy"]:
+            B.dspark_verify_greedy(batch.target, offsets, batch.draft_tokens, accepted_len=self.acc,
+                                   out_tokens=self.out, dev_status=self.status, workspace=self.ws, n_rows=self.n_rows)
+        else:
+            B.dspark_verify(batch.target, batch.draft, offsets, batch.draft_tokens, batch.temperature, batch.seed,
+                            draft_row_start=batch.draft_row_start, accepted_len=self.acc, out_tokens=self.out,
+                            dev_status=self.status, workspace=self.ws, n_rows=self.n_rows)
+
+
+def algorithmic_bytes(batch, greedy, n_rejected):
+    """Bytes the method must move: every target and draft row once, plus one re-read of the
+    rejected position's row pair per rejected request."""
+    elem = batch.target.element_size()
+    n_draft = batch.n_rows - batch.R
+    stream = elem * batch.V * (batch.n_rows + (0 if greedy else n_draft))
+    return stream, stream + (0 if greedy else 2 * elem * batch.V * n_rejected)
+
+
+# -------------------------------------------------------------------------------- clocks ----
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the GPU is busy."""
+
+    def __init__(self, index: int, period=0.02):
+        super().__init__(daemon=True)
+        self.period = period
+        self.samples, self.reasons = [], set()
+        self.stop_flag = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.max_mhz = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+        }
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, nm in names.items():
+                    if mask & bit:
+                        self.reasons.add(nm)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def finish(self):
+        self.stop_flag.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# -------------------------------------------------------------------------- reference arm ----
+def oracle_step(wl, batch, n_requests, threads):
+    """The CPU oracle over the first n_requests requests of the batch (schedule on all of them:
+    it is cheap and not separable)."""
+    import numpy as np
+    import oracle
+    from paper_2607_05147_b200 import workloads as W
+    host = wl["host"]
+    if wl["sched"] is not None:
+        oracle.schedule(host["conf"], host["table"], wl["sched"].budget_tokens, oracle.MODE_EARLY_STOP)
+    off = host["offsets"][: n_requests + 1]
+    if wl["greedy"]:
+        oracle.verify_greedy_mt(host["target"], off, host["tokens"], threads)
+    else:
+        oracle.verify(host["target"], host["draft"], off, host["tokens"], batch.temperature, batch.seed,
+                      eval_all=False, n_threads=threads)
+    return int(off[-1])
+
+
+def host_copy(wl):
+    import oracle
+    from paper_2607_05147_b200 import workloads as W
+    b = wl["batches"][0]
+    host = dict(target=W.bf16_bits(b.target), draft=None if b.draft is None else W.bf16_bits(b.draft),
+                offsets=b.row_offsets.cpu().numpy(), tokens=b.draft_tokens.cpu().numpy())
+    if wl["sched"] is not None:
+        host["conf"] = wl["sched"].conf.cpu().numpy()
+        host["table"] = oracle.sps_table(wl["sched"].bp_tokens, wl["sched"].bp_sps, wl["sched"].max_tokens)
+    wl["host"] = host
+
+
+def run_reference(args, rank):
+    """--impl reference: the CPU oracle, as it stands, on the machine's host cores."""
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    device = "cuda" if torch.cuda.is_available() else "cpu"     # only to draw the synthetic batch faster
+    wl = make_workload(args.workload, device, 0, 1, oracle_schedule=True)
+    host_copy(wl)
+    b = wl["batches"][0]
+    threads = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    oracle_step(wl, b, b.R, threads)
+    t1 = time.perf_counter() - t0
+    budget_s = 150.0
+    frac = min(1.0, budget_s / max(1e-9, (args.steps + args.warmup) * t1))
+    n_req = max(1, int(b.R * frac))
+    for _ in range(args.warmup):
+        oracle_step(wl, b, n_req, threads)
+    t0 = time.perf_counter()
+    rows = 0
+    for _ in range(args.steps):
+        rows += oracle_step(wl, b, n_req, threads)
+    dt = time.perf_counter() - t0
+    value = rows / dt
+    sample = f"first {n_req} of {b.R} requests per step ({rows // max(1, args.steps)} rows), schedule over all requests"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": wl["desc"], "name": wl["name"]},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------- main ----
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--all-workloads", action="store_true", help="also time the other V=129280 configurations")
+    ap.add_argument("--quick", action="store_true",
+                    help="timed steps only (no clock probe, per-kernel timing, e2e or CPU legs): for profiler captures")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2607_05147_b200 import binding as B
+    B.lib()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def time_workload(name, steps, warmup, with_e2e, with_cpu):
+        # enough distinct batches that consecutive steps cannot be served from the 126 MB L2
+        wl = make_workload(name, device, rank)
+        step = Step(wl, device)
+        batches = wl["batches"]
+        n_sets = len(batches)
+        for i in range(warmup):
+            step.run(batches[i % n_sets])
+        torch.cuda.synchronize()
+        dev_status = int(step.status.item())
+        n_rows = batches[0].n_rows
+        lens = batches[0].meta["lengths"].to(device)
+        n_rejected = int((step.acc < lens).sum().item()) if not wl["greedy"] else 0
+        if wl["sched"] is not None:
+            assert torch.equal(step.offsets, batches[0].row_offsets), "scheduled offsets differ from the generated batch"
+
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        for i in range(steps):
+            step.run(batches[i % n_sets])
+        ev1.record()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if args.quick:
+            sampler.finish()
+            return dict(wl=wl, step=step, ms=ms, n_rows=n_rows, n_rejected=n_rejected, quick=True)
+        # keep the same load running for ~1.5 s so the clock sampler sees it (not timed)
+        t_end = time.perf_counter() + 1.5
+        i = 0
+        while time.perf_counter() < t_end:
+            step.run(batches[i % n_sets]); i += 1
+            if i % 64 == 0:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        clocks = sampler.finish()
+
+        # per-kernel timing of the same steps (events around every launch of the library)
+        timer = B.KernelTimer(steps * 8)
+        timer.attach()
+        for i in range(steps):
+            step.run(batches[i % n_sets])
+        torch.cuda.synchronize()
+        timer.detach()
+        kernels = timer.read()
+        timer.close()
+
+        res = dict(wl=wl, step=step, ms=ms, n_rows=n_rows, n_rejected=n_rejected, kernels=kernels,
+                   clocks=clocks, dev_status=dev_status, n_sets=n_sets)
+
+        if with_e2e:
+            # end to end: inputs start in pinned host memory, results end in host memory, every step
+            b = batches[0]
+            host_in = [t.cpu().pin_memory() for t in (b.target, b.draft, b.draft_tokens) if t is not None]
+            conf_h = wl["sched"].conf.cpu().pin_memory() if wl["sched"] is not None else None
+            off_h = None if wl["sched"] is not None else b.row_offsets.cpu().pin_memory()
+            dev_in = [torch.empty_like(t, device=device) for t in host_in]
+            conf_d = torch.empty_like(wl["sched"].conf) if conf_h is not None else None
+            off_d = torch.empty_like(b.row_offsets) if off_h is not None else None
+            acc_h = torch.empty(step.R, dtype=torch.int32).pin_memory()
+            out_h = torch.empty(step.n_rows, dtype=torch.int32).pin_memory()
+            from paper_2607_05147_b200 import workloads as W
+            h2d = sum(t.numel() * t.element_size() for t in host_in)
+            h2d += conf_h.numel() * 4 if conf_h is not None else off_h.numel() * 4
+            d2h = acc_h.numel() * 4 + out_h.numel() * 4
+
+            def e2e_step():
+                for h, d in zip(host_in, dev_in):
+                    d.copy_(h, non_blocking=True)
+                if conf_h is not None:
+                    conf_d.copy_(conf_h, non_blocking=True)
+                else:
+                    off_d.copy_(off_h, non_blocking=True)
+                if wl["greedy"]:
+                    eb = W.VerifyBatch(dev_in[0], None, off_d if off_d is not None else b.row_offsets, dev_in[1],
+                                       None, b.temperature, b.seed)
+                else:
+                    eb = W.VerifyBatch(dev_in[0], dev_in[1], off_d if off_d is not None else b.row_offsets,
+                                       dev_in[2], None, b.temperature, b.seed)
+                step.run(eb, conf=conf_d)
+                acc_h.copy_(step.acc, non_blocking=True)
+                out_h.copy_(step.out, non_blocking=True)
+
+            e2e_steps = max(3, min(steps, 20))
+            for _ in range(3):
+                e2e_step()
+            barrier()
+            ev0.record()
+            for _ in range(e2e_steps):
+                e2e_step()
+            ev1.record()
+            barrier()
+            e2e_ms = ev0.elapsed_time(ev1)
+            res["e2e"] = dict(ms=e2e_ms, steps=e2e_steps, h2d=h2d, d2h=d2h)
+
+        if with_cpu and rank == 0:
+            import oracle
+            oracle.build()
+            host_copy(wl)
+            threads = os.cpu_count() or 1
+            t0 = time.perf_counter()
+            rows = oracle_step(wl, batches[0], batches[0].R, threads)
+            dt = time.perf_counter() - t0
+            res["cpu"] = {"value": rows / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                          "sample": f"whole batch once ({batches[0].R} requests, {rows} rows, {dt:.2f} s), "
+                                    "pthreads over requests"}
+        return res
+
+    res = time_workload(args.workload, args.steps, args.warmup, True, world == 1 or rank == 0)
+    wl = res["wl"]
+    if res.get("quick"):
+        print(json.dumps({"quick": True, "workload": wl["name"], "ms_per_step": res["ms"] / args.steps,
+                          "rows_per_s": res["n_rows"] * args.steps / (res["ms"] * 1e-3)}), flush=True)
+        return
+
+    # max over ranks of the device time
+    ms = res["ms"]
+    e2e_ms = res["e2e"]["ms"]
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+
+    b0 = wl["batches"][0]
+    stream_bytes, all_bytes = algorithmic_bytes(b0, wl["greedy"], res["n_rejected"])
+    value = world * res["n_rows"] * args.steps / (ms * 1e-3)
+    e2e_value = world * res["n_rows"] * res["e2e"]["steps"] / (e2e_ms * 1e-3)
+
+    peaks_file = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_file):
+        peak, peak_src = float(json.load(open(peaks_file))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+    dom = "greedy_stream" if wl["greedy"] else "stream_stats"
+    k = res["kernels"].get(dom, {"ms": float("nan"), "launches": 1})
+    dom_ms = k["ms"] / max(1, k["launches"])
+    achieved = stream_bytes / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "traffic": NCU_TRAFFIC_BYTES.get(wl["name"]), "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": stream_bytes, "us_per_launch": dom_ms * 1e3}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl["desc"], "name": wl["name"], "requests": b0.R, "rows_per_step": res["n_rows"],
+                       "draft_rows_per_step": b0.n_rows - b0.R, "rejected_requests": res["n_rejected"],
+                       "logit_dtype": "fp32" if wl["greedy"] else "bf16",
+                       "l2": f"inputs larger than L2: {res['n_sets']} distinct batches rotated "
+                             f"({res['n_sets'] * stream_bytes / 1e6:.0f} MB of logits)",
+                       "parallelism": "replicas only (one engine per GPU, no collective)"},
+            "step_algorithmic_bytes": all_bytes,
+            "step_effective_gbs": all_bytes / (ms / args.steps * 1e-3) / 1e9,
+            "step_frac_of_peak": all_bytes / (ms / args.steps * 1e-3) / 1e9 / peak,
+            "roofline": roofline,
+            "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in res["kernels"].items()},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": res["e2e"]["h2d"],
+                    "d2h_bytes_per_step": res["e2e"]["d2h"], "ms_per_step": e2e_ms / res["e2e"]["steps"],
+                    "steps": res["e2e"]["steps"]},
+            "gpu_launches": res["step"].launches_per_step * args.steps,
+            "clocks": res["clocks"], "dev_status": res["dev_status"],
+            "cpu_baseline": res.get("cpu"),
+        }
+        if args.all_workloads and world == 1:
+            others = {}
+            for name in ["cfg2", "cfg3", "cfg4", "cfg5"]:
+                if name == args.workload:
+                    continue
+                del res, wl
+                torch.cuda.empty_cache()
+                res = time_workload(name, args.steps, args.warmup, False, False)
+                wl = res["wl"]
+                sb, ab = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
+                d = "greedy_stream" if wl["greedy"] else "stream_stats"
+                kk = res["kernels"][d]
+                dms = kk["ms"] / kk["launches"]
+                others[name] = {"rows_per_s": res["n_rows"] * args.steps / (res["ms"] * 1e-3),
+                                "ms_per_step": res["ms"] / args.steps,
+                                "step_effective_gbs": ab / (res["ms"] / args.steps * 1e-3) / 1e9,
+                                "dominant_kernel_gbs": sb / (dms * 1e-3) / 1e9,
+                                "dominant_kernel_frac": sb / (dms * 1e-3) / 1e9 / peak,
+                                "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in res["kernels"].items()}}
+            line["other_workloads"] = others
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
