@@ -10,28 +10,28 @@
 namespace dspark {
 
 // ---------------------------------------------------------------------------------
-// Geometry of the streamed passes.  A logit row is cut into 2 KB blocks (one warp
-// each: 4 x 16 B per lane); 8 blocks form a 16 KB piece, the unit one bulk async
-// copy brings into one pipeline stage.
+// Geometry of the streamed passes.  A logit row is cut into blocks, one warp each
+// (16 B per lane per vector).  The statistics / argmax passes use 4 KB blocks
+// (8 vectors per lane), the residual pass 2 KB blocks of each of its two rows.
+// Eight blocks form a piece, the unit one bulk async copy brings into one stage.
 // ---------------------------------------------------------------------------------
-constexpr int kBlockBytes = 2048;
 constexpr int kConsumerWarps = 8;
-constexpr int kPieceBytes = kBlockBytes * kConsumerWarps;   // 16 KB
-constexpr int kVecPerLane = kBlockBytes / (32 * 16);        // 4
 constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;   // + one producer warp
+constexpr int kStatVec = 8;                                 // vectors per lane, statistics / argmax
+constexpr int kResidVec = 4;                                // vectors per lane and row, residual
+constexpr int kStatBlockBytes = kStatVec * 512;             // 4 KB
+constexpr int kResidBlockBytes = kResidVec * 512;           // 2 KB
+constexpr int kStageBytes = 32768;                          // one pipeline stage in every mode
+constexpr int kStages = 3;
 
 // Upper bound on polls of one mbarrier phase before a kernel gives up (each poll may
 // itself block for a short hardware-defined time, so this is on the order of a second).
 constexpr uint32_t kWaitPollLimit = 1u << 22;
 
-__host__ __device__ inline int blocks_per_row(int V, int elem_bytes)
+__host__ __device__ inline int blocks_per_row(int V, int elem_bytes, int block_bytes)
 {
     long long bytes = (long long)V * elem_bytes;
-    return (int)((bytes + kBlockBytes - 1) / kBlockBytes);
-}
-__host__ __device__ inline int pieces_per_row(int V, int elem_bytes)
-{
-    return (blocks_per_row(V, elem_bytes) + kConsumerWarps - 1) / kConsumerWarps;
+    return (int)((bytes + block_bytes - 1) / block_bytes);
 }
 
 // ---------------------------------------------------------------------------------
@@ -97,6 +97,35 @@ __device__ __forceinline__ float lg2_approx(float x)
     float y;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// Packed pairs of fp32 (sm_100 f32x2 arithmetic: one instruction, two IEEE-rounded results).
+__device__ __forceinline__ uint64_t pack2(float a, float b)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
 }
 // Warp-wide float max in one instruction (sm_100a redux); NaN inputs are ignored.
 __device__ __forceinline__ float warp_max_f32(float x)

@@ -3,14 +3,14 @@
 //
 // Pass structure (all on the caller's stream, no host round trip):
 //   stream   every target / draft row is read from HBM exactly once.  A row is cut into
-//            2 KB blocks; one warp reduces one block to (reference, sum of 2^(x*scale-ref))
+//            4 KB blocks; one warp reduces one block to (reference, sum of 2^(x*scale-ref))
 //            [sampling] or (max, lowest argmax) [greedy].  Persistent CTAs; a producer warp
-//            feeds a ring of 16 KB shared-memory stages with 1-D bulk async copies
+//            feeds a ring of 32 KB shared-memory stages with 1-D bulk async copies
 //            (cp.async.bulk + mbarrier), eight consumer warps drain it.
 //   decide   one CTA per request: combines block statistics into row statistics, gathers
 //            p(x), q(x), runs the accept tests (Philox), finds the first rejection, writes
 //            the accepted prefix, and queues the rejected position for the residual pass.
-//   residual second read of the rejected position's row pair only: per-block sums of
+//   residual second read of the rejected position's row pair only: per-2KB-block sums of
 //            max(0, p - q), same bulk-copy pipeline with two sources per stage.
 //   finalize one warp per request: inverse CDF over block sums, then inside one block.
 #include <cuda_bf16.h>
@@ -23,7 +23,7 @@ namespace dspark {
 constexpr int kModeStats = 0, kModeGreedy = 1, kModeResid = 2;
 constexpr int kTaskNone = 0, kTaskResid = 1, kTaskBonus = 2;
 constexpr int kDecideThreads = 256;
-constexpr int kFinalizeThreads = 256;
+constexpr int kFinalizeThreads = 128;
 constexpr float kNegInf = -INFINITY;
 
 struct __align__(16) ResidTask {     // one rejected request queued for the residual pass
@@ -46,7 +46,9 @@ struct VerifyParams {
     const unsigned char* target;
     const unsigned char* draft;
     long long tstride_bytes, dstride_bytes;
-    int V, elem, row_bytes, nblk, ppr, epb;   // epb = elements per block
+    int V, elem, row_bytes;
+    int nblk, epb;                            // statistics blocks per row, elements per block
+    int nblk_r, epb_r;                        // residual blocks per row, elements per block
     const int32_t* row_offsets;
     const int64_t* draft_row_start;
     const int32_t* draft_tokens;
@@ -65,6 +67,14 @@ struct VerifyParams {
     ResidTask* resid;
     RequestTask* req;
     float* wblk;
+};
+
+template <int kMode> struct ModeCfg {
+    static constexpr int kSrc = (kMode == kModeResid) ? 2 : 1;
+    static constexpr int kVec = (kMode == kModeResid) ? kResidVec : kStatVec;
+    static constexpr int kBlockBytes = kVec * 512;
+    static constexpr int kPieceBytes = kBlockBytes * kConsumerWarps;   // per source
+    static_assert(kPieceBytes * kSrc == kStageBytes, "a stage holds one piece of every source");
 };
 
 // ---------------------------------------------------------------------------------------
@@ -92,56 +102,35 @@ __device__ __forceinline__ long long draft_phys_row(const VerifyParams& P, int d
     return P.draft_row_start[lo] + j;
 }
 
-struct Unit {
-    const unsigned char* src0;
-    const unsigned char* src1;
-    int piece;          // piece index inside the row
-    int bytes;          // bytes of this piece (per source)
-    long long out_row;  // row index into the statistics array (or residual slot)
-    int is_draft;
-    ResidTask task;
+// Number of row streams a streamed pass walks.
+template <int kMode>
+__device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
+{
+    if (kMode == kModeStats) return n_rows + (n_rows > P.R ? n_rows - P.R : 0);
+    if (kMode == kModeGreedy) return n_rows;
+    int nq = __ldcg(&P.counters[0]);
+    return nq > P.R ? P.R : (nq < 0 ? 0 : nq);
+}
+
+// Walks the units (stream s, piece) owned by this CTA: unit index = s * ppr + piece, advancing by
+// gridDim.x units per step without divisions.
+struct UnitCursor {
+    int s, piece, step_s, step_p, ppr;
+    __device__ __forceinline__ void init(int ppr_)
+    {
+        ppr = ppr_;
+        s = (int)blockIdx.x / ppr; piece = (int)blockIdx.x - s * ppr;
+        step_s = (int)gridDim.x / ppr; step_p = (int)gridDim.x - step_s * ppr;
+    }
+    __device__ __forceinline__ void next()
+    {
+        s += step_s; piece += step_p;
+        if (piece >= ppr) { piece -= ppr; ++s; }
+    }
 };
 
-template <int kMode>
-__device__ __forceinline__ int total_units(const VerifyParams& P, int n_rows)
-{
-    if (kMode == kModeStats) return (n_rows + (n_rows > P.R ? n_rows - P.R : 0)) * P.ppr;
-    if (kMode == kModeGreedy) return n_rows * P.ppr;
-    int nq = __ldcg(&P.counters[0]);
-    return (nq > P.R ? P.R : nq) * P.ppr;
-}
-
-template <int kMode>
-__device__ __forceinline__ void decode_unit(const VerifyParams& P, int u, int n_rows, bool need_src, Unit& U)
-{
-    const int s = u / P.ppr;
-    U.piece = u - s * P.ppr;
-    const long long off = (long long)U.piece * kPieceBytes;
-    const long long rem = (long long)P.row_bytes - off;
-    U.bytes = (int)(rem < kPieceBytes ? rem : kPieceBytes);
-    U.src1 = nullptr;
-    U.is_draft = 0;
-    if (kMode == kModeResid) {
-        U.task = P.resid[s];
-        U.out_row = s;
-        U.src0 = P.target + (long long)U.task.row_t * P.tstride_bytes + off;
-        U.src1 = P.draft + U.task.row_d * P.dstride_bytes + off;
-        return;
-    }
-    if (s < n_rows) {
-        U.out_row = s;
-        U.src0 = P.target + (long long)s * P.tstride_bytes + off;
-    } else {
-        const int ds = s - n_rows;
-        U.out_row = ds;
-        U.is_draft = 1;
-        long long phys = need_src ? draft_phys_row(P, ds) : 0;
-        U.src0 = (phys >= 0 ? P.draft + phys * P.dstride_bytes : P.target) + off;
-    }
-}
-
 // ---------------------------------------------------------------------------------------
-// Per-lane view of one 2 KB block: 4 x 16 B, vector k of lane l is vector k*32+l of the block
+// Per-lane view of one block: kVec x 16 B, vector k of lane l is vector k*32+l of the block
 // ---------------------------------------------------------------------------------------
 template <int kElem> __device__ __forceinline__ uint32_t fill_word() { return kElem == 2 ? 0xFF80FF80u : 0xFF800000u; }
 
@@ -175,14 +164,19 @@ struct GlobalFetch {
     }
 };
 
-template <int kElem, typename Fetch>
-__device__ __forceinline__ void load_block(const Fetch& f, int nbytes, int lane, uint4 (&v)[kVecPerLane])
+template <int kElem, int kVec, typename Fetch>
+__device__ __forceinline__ void load_block(const Fetch& f, int nbytes, int lane, uint4 (&v)[kVec])
 {
+    if (nbytes == kVec * 512) {                  // full block: no per-vector tests
 #pragma unroll
-    for (int k = 0; k < kVecPerLane; ++k) {
-        const int vec = k * 32 + lane;
-        const uint32_t fw = fill_word<kElem>();
-        v[k] = (vec * 16 < nbytes) ? f(vec, nbytes) : make_uint4(fw, fw, fw, fw);
+        for (int k = 0; k < kVec; ++k) v[k] = f(k * 32 + lane, nbytes);
+    } else {
+#pragma unroll
+        for (int k = 0; k < kVec; ++k) {
+            const int vec = k * 32 + lane;
+            const uint32_t fw = fill_word<kElem>();
+            v[k] = (vec * 16 < nbytes) ? f(vec, nbytes) : make_uint4(fw, fw, fw, fw);
+        }
     }
 }
 
@@ -190,61 +184,77 @@ __device__ __forceinline__ uint32_t word_of(const uint4& q, int i)
 {
     return i == 0 ? q.x : (i == 1 ? q.y : (i == 2 ? q.z : q.w));
 }
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
+{
+    __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+}
 
 // Sampling statistics of one block: reference c = max(x) * scale (warp-uniform) and
-// s = sum over the block of 2^(x*scale - c): exactly one exponential per element.
-template <int kElem>
-__device__ __forceinline__ float2 block_stats(const uint4 (&v)[kVecPerLane], float scale)
+// s = sum over the block of 2^(x*scale - c): exactly one exponential per element; the
+// multiply-adds and the accumulation run as packed f32x2 instructions.
+template <int kElem, int kVec>
+__device__ __forceinline__ float2 block_stats(const uint4 (&v)[kVec], float scale)
 {
     float mx;
     if (kElem == 2) {
-        __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&v[0].x);
+        uint32_t m0 = v[0].x, m1 = v[0].y;
 #pragma unroll
-        for (int k = 0; k < kVecPerLane; ++k)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t w = word_of(v[k], i);
-                m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162*>(&w));
-            }
-        uint32_t mw = *reinterpret_cast<uint32_t*>(&m2);
-        mx = fmaxf(bf16lo(mw), bf16hi(mw));
+        for (int k = 0; k < kVec; ++k) {
+            m0 = bf16x2_max(m0, v[k].x); m1 = bf16x2_max(m1, v[k].y);
+            m0 = bf16x2_max(m0, v[k].z); m1 = bf16x2_max(m1, v[k].w);
+        }
+        m0 = bf16x2_max(m0, m1);
+        mx = fmaxf(bf16lo(m0), bf16hi(m0));
     } else {
-        mx = kNegInf;
+        float a = kNegInf, b = kNegInf;
 #pragma unroll
-        for (int k = 0; k < kVecPerLane; ++k)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) mx = fmaxf(mx, __uint_as_float(word_of(v[k], i)));
+        for (int k = 0; k < kVec; ++k) {
+            a = fmaxf(a, __uint_as_float(v[k].x)); b = fmaxf(b, __uint_as_float(v[k].y));
+            a = fmaxf(a, __uint_as_float(v[k].z)); b = fmaxf(b, __uint_as_float(v[k].w));
+        }
+        mx = fmaxf(a, b);
     }
     const float wmax = warp_max_f32(mx);
     if (wmax == kNegInf) return make_float2(kNegInf, 0.0f);
     const float c = __fmul_rn(wmax, scale);
-    const float nc = -c;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint64_t s2 = pack2(scale, scale), nc2 = pack2(-c, -c);
+    uint64_t acc0 = pack2(0.f, 0.f), acc1 = acc0;
 #pragma unroll
-    for (int k = 0; k < kVecPerLane; ++k)
+    for (int k = 0; k < kVec; ++k) {
+        if (kElem == 2) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t w = word_of(v[k], i);
-            if (kElem == 2) {
-                acc[i] += ex2_approx(__fmaf_rn(bf16lo(w), scale, nc));
-                acc[i] += ex2_approx(__fmaf_rn(bf16hi(w), scale, nc));
-            } else {
-                acc[i] += ex2_approx(__fmaf_rn(__uint_as_float(w), scale, nc));
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t w = word_of(v[k], i);
+                float t0, t1;
+                unpack2(fma2(pack2(bf16lo(w), bf16hi(w)), s2, nc2), t0, t1);
+                const uint64_t e2 = pack2(ex2_approx(t0), ex2_approx(t1));
+                if (i & 1) acc1 = add2(acc1, e2); else acc0 = add2(acc0, e2);
             }
+        } else {
+            float t0, t1, t2, t3;
+            unpack2(fma2(pack2(__uint_as_float(v[k].x), __uint_as_float(v[k].y)), s2, nc2), t0, t1);
+            unpack2(fma2(pack2(__uint_as_float(v[k].z), __uint_as_float(v[k].w)), s2, nc2), t2, t3);
+            acc0 = add2(acc0, pack2(ex2_approx(t0), ex2_approx(t1)));
+            acc1 = add2(acc1, pack2(ex2_approx(t2), ex2_approx(t3)));
         }
-    const float s = warp_sum_f32((acc[0] + acc[1]) + (acc[2] + acc[3]));
+    }
+    float a0, a1, b0, b1;
+    unpack2(acc0, a0, a1);
+    unpack2(acc1, b0, b1);
+    const float s = warp_sum_f32((a0 + a1) + (b0 + b1));
     return make_float2(c, s);
 }
 
 // Greedy statistics of one block: (max, lowest index attaining it); NaN never wins.
-template <int kElem>
-__device__ __forceinline__ float2 block_argmax(const uint4 (&v)[kVecPerLane], int elem_base, int lane)
+template <int kElem, int kVec>
+__device__ __forceinline__ float2 block_argmax(const uint4 (&v)[kVec], int elem_base, int lane)
 {
     constexpr int kPerVec = 16 / kElem;
     float best = kNegInf;
     int bi = 0x7fffffff;
 #pragma unroll
-    for (int k = 0; k < kVecPerLane; ++k) {
+    for (int k = 0; k < kVec; ++k) {
         const int base = elem_base + (k * 32 + lane) * kPerVec;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -265,84 +275,133 @@ __device__ __forceinline__ float2 block_argmax(const uint4 (&v)[kVecPerLane], in
     return make_float2(wmax, __int_as_float((int)widx));
 }
 
-// One element of the residual max(0, p - q), with the exact operation sequence the
-// finalize kernel repeats.
-__device__ __forceinline__ float resid_elem(float xt, float xd, float scale, const ResidTask& t)
+// Residual max(0, p - q) of two neighbouring elements, packed; p = 2^(xt*scale-cp) * inv_zp,
+// q likewise.  Every operation is a single IEEE-rounded step, so the scalar form below gives
+// bit-identical values (the finalize kernel relies on that).
+struct ResidConst {
+    uint64_t s2, ncp2, ncq2, izp2, nizq2;
+    float scale, cp, cq, inv_zp, inv_zq;
+    __device__ __forceinline__ void set(float scale_, float cp_, float inv_zp_, float cq_, float inv_zq_)
+    {
+        scale = scale_; cp = cp_; cq = cq_; inv_zp = inv_zp_; inv_zq = inv_zq_;
+        s2 = pack2(scale, scale); ncp2 = pack2(-cp, -cp); ncq2 = pack2(-cq, -cq);
+        izp2 = pack2(inv_zp, inv_zp); nizq2 = pack2(-inv_zq, -inv_zq);
+    }
+};
+__device__ __forceinline__ uint64_t resid_pair(uint64_t xt2, uint64_t xd2, const ResidConst& K)
 {
-    const float ep = ex2_approx(__fmaf_rn(xt, scale, -t.cp));
-    const float eq = ex2_approx(__fmaf_rn(xd, scale, -t.cq));
-    const float q = __fmul_rn(eq, t.inv_zq);
-    return fmaxf(__fmaf_rn(ep, t.inv_zp, -q), 0.0f);
+    float a0, a1, b0, b1;
+    unpack2(fma2(xt2, K.s2, K.ncp2), a0, a1);
+    unpack2(fma2(xd2, K.s2, K.ncq2), b0, b1);
+    const uint64_t ep2 = pack2(ex2_approx(a0), ex2_approx(a1));
+    const uint64_t eq2 = pack2(ex2_approx(b0), ex2_approx(b1));
+    float w0, w1;
+    unpack2(fma2(ep2, K.izp2, mul2(eq2, K.nizq2)), w0, w1);
+    return pack2(fmaxf(w0, 0.0f), fmaxf(w1, 0.0f));
+}
+__device__ __forceinline__ float resid_elem(float xt, float xd, const ResidConst& K)
+{
+    const float ep = ex2_approx(__fmaf_rn(xt, K.scale, -K.cp));
+    const float eq = ex2_approx(__fmaf_rn(xd, K.scale, -K.cq));
+    return fmaxf(__fmaf_rn(ep, K.inv_zp, __fmul_rn(eq, -K.inv_zq)), 0.0f);
 }
 
-template <int kElem>
-__device__ __forceinline__ float block_resid(const uint4 (&vt)[kVecPerLane], const uint4 (&vd)[kVecPerLane],
-                                             float scale, const ResidTask& t)
+template <int kElem, int kVec>
+__device__ __forceinline__ float block_resid(const uint4 (&vt)[kVec], const uint4 (&vd)[kVec], const ResidConst& K)
 {
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    uint64_t acc0 = pack2(0.f, 0.f), acc1 = acc0;
 #pragma unroll
-    for (int k = 0; k < kVecPerLane; ++k)
+    for (int k = 0; k < kVec; ++k) {
+        if (kElem == 2) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t a = word_of(vt[k], i), b = word_of(vd[k], i);
-            if (kElem == 2) {
-                acc[i] += resid_elem(bf16lo(a), bf16lo(b), scale, t);
-                acc[i] += resid_elem(bf16hi(a), bf16hi(b), scale, t);
-            } else {
-                acc[i] += resid_elem(__uint_as_float(a), __uint_as_float(b), scale, t);
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t a = word_of(vt[k], i), b = word_of(vd[k], i);
+                const uint64_t w2 = resid_pair(pack2(bf16lo(a), bf16hi(a)), pack2(bf16lo(b), bf16hi(b)), K);
+                if (i & 1) acc1 = add2(acc1, w2); else acc0 = add2(acc0, w2);
             }
+        } else {
+            acc0 = add2(acc0, resid_pair(pack2(__uint_as_float(vt[k].x), __uint_as_float(vt[k].y)),
+                                         pack2(__uint_as_float(vd[k].x), __uint_as_float(vd[k].y)), K));
+            acc1 = add2(acc1, resid_pair(pack2(__uint_as_float(vt[k].z), __uint_as_float(vt[k].w)),
+                                         pack2(__uint_as_float(vd[k].z), __uint_as_float(vd[k].w)), K));
         }
-    return warp_sum_f32((acc[0] + acc[1]) + (acc[2] + acc[3]));
+    }
+    float a0, a1, b0, b1;
+    unpack2(acc0, a0, a1);
+    unpack2(acc1, b0, b1);
+    return warp_sum_f32((a0 + a1) + (b0 + b1));
 }
 
-// What a consumer warp does with its block of a unit.
+// What a consumer warp does with its block of the unit (stream s, piece).
 template <int kElem, int kMode, typename Fetch>
-__device__ __forceinline__ void consume_block(const VerifyParams& P, const Unit& U, int warp, int lane,
-                                              const Fetch& f0, const Fetch& f1)
+__device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int piece, int n_rows,
+                                              int warp, int lane, const Fetch& f0, const Fetch& f1)
 {
-    const int b = U.piece * kConsumerWarps + warp;
-    if (b >= P.nblk) return;
-    const int blk_off = warp * kBlockBytes;
-    const int nbytes = (U.bytes - blk_off) < kBlockBytes ? (U.bytes - blk_off) : kBlockBytes;
-    uint4 v[kVecPerLane];
-    load_block<kElem>(f0, nbytes, lane, v);
+    using M = ModeCfg<kMode>;
+    const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
+    const int b = piece * kConsumerWarps + warp;
+    if (b >= nblk) return;
+    const int rem = P.row_bytes - b * M::kBlockBytes;
+    const int nbytes = rem < M::kBlockBytes ? rem : M::kBlockBytes;
+    uint4 v[M::kVec];
+    load_block<kElem, M::kVec>(f0, nbytes, lane, v);
     if (kMode == kModeStats) {
-        const float2 st = block_stats<kElem>(v, P.scale);
-        if (lane == 0) (U.is_draft ? P.stats_d : P.stats_t)[U.out_row * P.nblk + b] = st;
+        const float2 st = block_stats<kElem, M::kVec>(v, P.scale);
+        if (lane == 0) {
+            float2* dst = (s < n_rows) ? P.stats_t + (long long)s * nblk : P.stats_d + (long long)(s - n_rows) * nblk;
+            dst[b] = st;
+        }
     } else if (kMode == kModeGreedy) {
-        const float2 st = block_argmax<kElem>(v, b * P.epb, lane);
-        if (lane == 0) P.stats_t[U.out_row * P.nblk + b] = st;
+        const float2 st = block_argmax<kElem, M::kVec>(v, b * P.epb, lane);
+        if (lane == 0) P.stats_t[(long long)s * nblk + b] = st;
     } else {
-        uint4 vd[kVecPerLane];
-        load_block<kElem>(f1, nbytes, lane, vd);
-        const float w = block_resid<kElem>(v, vd, P.scale, U.task);
-        if (lane == 0) P.wblk[U.out_row * P.nblk + b] = w;
+        uint4 vd[M::kVec];
+        load_block<kElem, M::kVec>(f1, nbytes, lane, vd);
+        const float4 c = *reinterpret_cast<const float4*>(&P.resid[s].cp);
+        ResidConst K;
+        K.set(P.scale, c.x, c.y, c.z, c.w);
+        const float w = block_resid<kElem, M::kVec>(v, vd, K);
+        if (lane == 0) P.wblk[(long long)s * nblk + b] = w;
+    }
+}
+
+// Source addresses of a unit (producer / direct path).
+template <int kMode>
+__device__ __forceinline__ void unit_sources(const VerifyParams& P, int s, int piece, int n_rows,
+                                             const unsigned char*& src0, const unsigned char*& src1, int& bytes)
+{
+    using M = ModeCfg<kMode>;
+    const long long off = (long long)piece * M::kPieceBytes;
+    const long long rem = (long long)P.row_bytes - off;
+    bytes = (int)(rem < M::kPieceBytes ? rem : M::kPieceBytes);
+    src1 = nullptr;
+    if (kMode == kModeResid) {
+        const ResidTask t = P.resid[s];
+        src0 = P.target + (long long)t.row_t * P.tstride_bytes + off;
+        src1 = P.draft + t.row_d * P.dstride_bytes + off;
+    } else if (s < n_rows) {
+        src0 = P.target + (long long)s * P.tstride_bytes + off;
+    } else {
+        const long long phys = draft_phys_row(P, s - n_rows);
+        src0 = (phys >= 0 ? P.draft + phys * P.dstride_bytes : P.target) + off;
     }
 }
 
 // ---------------------------------------------------------------------------------------
-// Streamed pass, bulk-copy pipeline.  kStages x kSrc x 16 KB of shared memory per CTA.
+// Streamed pass, bulk-copy pipeline: kStages x 32 KB of shared memory per CTA.
 // ---------------------------------------------------------------------------------------
-template <int kElem, int kMode>
-struct StreamCfg {
-    static constexpr int kSrc = (kMode == kModeResid) ? 2 : 1;
-    static constexpr int kStages = 6 / kSrc;
-    static constexpr int kStageBytes = kSrc * kPieceBytes;
-    static constexpr int kSmemBytes = kStages * kStageBytes;
-};
-
 template <int kElem, int kMode>
 __global__ void __launch_bounds__(kStreamThreads, 2) stream_bulk_kernel(VerifyParams P)
 {
-    using Cfg = StreamCfg<kElem, kMode>;
+    using M = ModeCfg<kMode>;
     extern __shared__ __align__(128) unsigned char stage_mem[];
-    __shared__ __align__(8) uint64_t full_bar[Cfg::kStages];
-    __shared__ __align__(8) uint64_t empty_bar[Cfg::kStages];
+    __shared__ __align__(8) uint64_t full_bar[kStages];
+    __shared__ __align__(8) uint64_t empty_bar[kStages];
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kConsumerWarps); }
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kConsumerWarps); }
         s_abort = 0;
         mbar_fence_init();
     }
@@ -354,55 +413,57 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_bulk_kernel(VerifyPa
         P.counters[0] = 0;                       // residual queue, filled by the decide kernel
         if (bad_rows) atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS);
     }
-    const int total = total_units<kMode>(P, n_rows);
+    const int n_streams = stream_count<kMode>(P, n_rows);
+    const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
+    UnitCursor cur;
+    cur.init((nblk + kConsumerWarps - 1) / kConsumerWarps);
     volatile int* abort_flag = &s_abort;
 
     if (warp == kConsumerWarps) {
         // ---------------- producer warp: lane 0 issues the copies -----------------------
         int it = 0;
-        for (int u = blockIdx.x; u < total; u += gridDim.x, ++it) {
-            const int s = it % Cfg::kStages;
-            const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
+        for (; cur.s < n_streams; cur.next(), ++it) {
+            const int st = it % kStages;
+            const uint32_t ph = (uint32_t)(it / kStages) & 1u;
             if (*abort_flag) break;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(&empty_bar[s], ph ^ 1u))) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(&empty_bar[st], ph ^ 1u))) {
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
                 break;
             }
-            Unit U;
-            decode_unit<kMode>(P, u, n_rows, true, U);
             if (lane == 0) {
-                unsigned char* dst = stage_mem + s * Cfg::kStageBytes;
-                mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(U.bytes * Cfg::kSrc));
-                bulk_g2s(dst, U.src0, (uint32_t)U.bytes, &full_bar[s]);
-                if (Cfg::kSrc == 2) bulk_g2s(dst + kPieceBytes, U.src1, (uint32_t)U.bytes, &full_bar[s]);
+                const unsigned char *src0, *src1;
+                int bytes;
+                unit_sources<kMode>(P, cur.s, cur.piece, n_rows, src0, src1, bytes);
+                unsigned char* dst = stage_mem + st * kStageBytes;
+                mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(bytes * M::kSrc));
+                bulk_g2s(dst, src0, (uint32_t)bytes, &full_bar[st]);
+                if (M::kSrc == 2) bulk_g2s(dst + M::kPieceBytes, src1, (uint32_t)bytes, &full_bar[st]);
             }
             __syncwarp();
         }
         if (*abort_flag) {
             // leave only after every copy already issued has landed (bounded)
-            for (int k = 0; k < Cfg::kStages && k < it; ++k) {
+            for (int k = 0; k < kStages && k < it; ++k) {
                 const int jt = it - 1 - k;
-                mbar_wait_bounded(&full_bar[jt % Cfg::kStages], (uint32_t)(jt / Cfg::kStages) & 1u);
+                mbar_wait_bounded(&full_bar[jt % kStages], (uint32_t)(jt / kStages) & 1u);
             }
         }
     } else {
         // ---------------- consumer warps --------------------------------------------------
         int it = 0;
-        for (int u = blockIdx.x; u < total; u += gridDim.x, ++it) {
-            const int s = it % Cfg::kStages;
-            const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
+        for (; cur.s < n_streams; cur.next(), ++it) {
+            const int st = it % kStages;
+            const uint32_t ph = (uint32_t)(it / kStages) & 1u;
             if (*abort_flag) break;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(&full_bar[s], ph))) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(&full_bar[st], ph))) {
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
                 break;
             }
-            Unit U;
-            decode_unit<kMode>(P, u, n_rows, false, U);
-            const unsigned char* st = stage_mem + s * Cfg::kStageBytes + warp * kBlockBytes;
-            SmemFetch f0{st}, f1{st + kPieceBytes};
-            consume_block<kElem, kMode>(P, U, warp, lane, f0, f1);
+            const unsigned char* sp = stage_mem + st * kStageBytes + warp * M::kBlockBytes;
+            SmemFetch f0{sp}, f1{sp + M::kPieceBytes};
+            consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1);
             __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[s]);
+            if (lane == 0) mbar_arrive(&empty_bar[st]);
         }
     }
 }
@@ -413,6 +474,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_bulk_kernel(VerifyPa
 template <int kElem, int kMode>
 __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(VerifyParams P)
 {
+    using M = ModeCfg<kMode>;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
@@ -420,39 +482,62 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
         P.counters[0] = 0;
         if (bad_rows) atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS);
     }
-    const int total = total_units<kMode>(P, n_rows);
-    for (int u = blockIdx.x; u < total; u += gridDim.x) {
-        Unit U;
-        decode_unit<kMode>(P, u, n_rows, true, U);
-        GlobalFetch<kElem> f0{U.src0 + warp * kBlockBytes};
-        GlobalFetch<kElem> f1{(kMode == kModeResid ? U.src1 : U.src0) + warp * kBlockBytes};
-        consume_block<kElem, kMode>(P, U, warp, lane, f0, f1);
+    const int n_streams = stream_count<kMode>(P, n_rows);
+    const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
+    UnitCursor cur;
+    cur.init((nblk + kConsumerWarps - 1) / kConsumerWarps);
+    for (; cur.s < n_streams; cur.next()) {
+        const unsigned char *src0, *src1;
+        int bytes;
+        unit_sources<kMode>(P, cur.s, cur.piece, n_rows, src0, src1, bytes);
+        GlobalFetch<kElem> f0{src0 + warp * M::kBlockBytes};
+        GlobalFetch<kElem> f1{(kMode == kModeResid ? src1 : src0) + warp * M::kBlockBytes};
+        consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1);
     }
 }
 
 // ---------------------------------------------------------------------------------------
 // Row statistics from block statistics: reference C = max_b c_b, sum S = sum_b s_b 2^(c_b-C).
-// Called by one full warp; result valid in every lane.
+// One pass over the entries (4 per lane in flight), online rescaling per lane, then a warp
+// combine.  Called by one full warp; the result is valid in every lane.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void combine_row(const float2* __restrict__ st, int nblk, int lane, float& C, double& S)
+struct RowAcc {
+    float C;
+    double S;
+    __device__ __forceinline__ void init() { C = kNegInf; S = 0.0; }
+    __device__ __forceinline__ void add(float2 e)
+    {
+        if (e.x != e.x || e.y != e.y) { S = NAN; return; }      // a NaN anywhere must survive
+        if (!(e.x > kNegInf)) return;                           // empty block
+        if (e.x > C) { S *= (double)ex2_approx(C - e.x); C = e.x; }   // C = -inf: factor 0, S was 0
+        S += (double)(e.y * ex2_approx(e.x - C));
+    }
+    __device__ __forceinline__ void finish()
+    {
+        const float Cw = warp_max_f32(C);
+        double s = (C > kNegInf) ? S * (double)ex2_approx(C - Cw) : (S != S ? S : 0.0);
+        S = warp_sum_f64(s);
+        C = Cw;
+    }
+};
+
+__device__ __forceinline__ void combine_rows(const float2* __restrict__ a, const float2* __restrict__ b,
+                                             int nblk, int lane, RowAcc& A, RowAcc& Bc)
 {
-    float c = kNegInf;
-    for (int b = lane; b < nblk; b += 32) c = fmaxf(c, __ldcg(&st[b]).x);
-    C = warp_max_f32(c);
-    double s = 0.0;
-    if (C > kNegInf) {
-        for (int b = lane; b < nblk; b += 32) {
-            const float2 e = __ldcg(&st[b]);
-            if (e.x > kNegInf) s += (double)(e.y * ex2_approx(e.x - C));
-            else if (e.y != e.y) s += (double)e.y;
+    A.init(); Bc.init();
+    for (int base = 0; base < nblk; base += 128) {
+        float2 ea[4], eb[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int i = base + k * 32 + lane;
+            ea[k] = (i < nblk) ? __ldcg(&a[i]) : make_float2(kNegInf, 0.f);
+            eb[k] = (b && i < nblk) ? __ldcg(&b[i]) : make_float2(kNegInf, 0.f);
         }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { A.add(ea[k]); Bc.add(eb[k]); }
     }
-    // a NaN anywhere (NaN reference or NaN sum) must survive
-    for (int b = lane; b < nblk; b += 32) {
-        const float2 e = __ldcg(&st[b]);
-        if (e.x != e.x || e.y != e.y) s = NAN;
-    }
-    S = warp_sum_f64(s);
+    A.finish();
+    if (b) Bc.finish();
 }
 
 __device__ __forceinline__ float load_logit(const unsigned char* base, long long row, long long stride_bytes,
@@ -469,14 +554,20 @@ __device__ __forceinline__ bool row_usable(float C, double S)
 }
 
 // ---------------------------------------------------------------------------------------
-// decide: one CTA per request.
+// decide: one CTA per request, one warp per position (eight positions per round).
+// Position j = len is the bonus row (statistics only).
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
 {
+    constexpr int kWarps = kDecideThreads / 32;
     __shared__ int s_first, s_bad;
+    __shared__ float s_Ct[kWarps], s_Cd[kWarps];
+    __shared__ double s_St[kWarps], s_Sd[kWarps];
+    __shared__ float s_fin_C[2];     // [0] target, [1] draft statistics of the row that emits the token
+    __shared__ double s_fin_S[2];
+    __shared__ int s_have_fin;
     const int r = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    constexpr int kWarps = kDecideThreads / 32;
 
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
@@ -492,7 +583,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     }
     const int len = hi - lo - 1;
     const long long drow0 = P.draft_row_start ? P.draft_row_start[r] : (long long)(lo - r);
-    if (tid == 0) { s_first = len; s_bad = 0; }
+    if (tid == 0) { s_first = len; s_bad = 0; s_have_fin = 0; }
     __syncthreads();
     for (int i = tid; i <= len; i += kDecideThreads) {
         P.out_tokens[lo + i] = -1;
@@ -509,90 +600,103 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     const bool want_all = (P.out_p != nullptr) || (P.out_q != nullptr);
     const double scale_d = (double)P.scale;
 
-    for (int j0 = 0; j0 < len; j0 += kWarps) {
+    for (int j0 = 0; j0 <= len; j0 += kWarps) {
         const int j = j0 + warp;
-        if (j < len) {
-            float Cp, Cq; double Sp, Sq;
-            combine_row(P.stats_t + (long long)(lo + j) * P.nblk, P.nblk, lane, Cp, Sp);
-            combine_row(P.stats_d + (long long)(lo - r + j) * P.nblk, P.nblk, lane, Cq, Sq);
+        if (j <= len) {
+            const bool is_draft_pos = j < len;
+            // the two logits at the draft token do not depend on the statistics: fetch them first
+            float xt = 0.f, xd = 0.f;
+            if (is_draft_pos && lane == 0) {
+                const int d = P.draft_tokens[lo + j];
+                xt = load_logit(P.target, lo + j, P.tstride_bytes, P.elem, d);
+                xd = load_logit(P.draft, drow0 + j, P.dstride_bytes, P.elem, d);
+            }
+            RowAcc A, D;
+            combine_rows(P.stats_t + (long long)(lo + j) * P.nblk,
+                         is_draft_pos ? P.stats_d + (long long)(lo - r + j) * P.nblk : nullptr, P.nblk, lane, A, D);
             if (lane == 0) {
-                if (!row_usable(Cp, Sp) || !row_usable(Cq, Sq)) {
-                    atomicOr(&s_bad, DSPARK_DEV_BAD_ROW);
-                } else {
-                    const int d = P.draft_tokens[lo + j];
-                    const double xt = (double)load_logit(P.target, lo + j, P.tstride_bytes, P.elem, d);
-                    const double xd = (double)load_logit(P.draft, drow0 + j, P.dstride_bytes, P.elem, d);
-                    const double p = exp2(xt * scale_d - (double)Cp) / Sp;
-                    const double q = exp2(xd * scale_d - (double)Cq) / Sq;
-                    if (P.out_p) P.out_p[lo + j] = (float)p;
-                    if (P.out_q) P.out_q[lo + j] = (float)q;
-                    float ua, ur;
-                    philox_uniforms(P.seed, (uint32_t)r, (uint32_t)j, ua, ur);
-                    if (!((double)ua * q < p)) atomicMin(&s_first, j);     // rejected
+                s_Ct[warp] = A.C; s_St[warp] = A.S; s_Cd[warp] = D.C; s_Sd[warp] = D.S;
+                if (is_draft_pos) {
+                    if (!row_usable(A.C, A.S) || !row_usable(D.C, D.S)) {
+                        atomicOr(&s_bad, DSPARK_DEV_BAD_ROW);
+                    } else {
+                        const double p = exp2((double)xt * scale_d - (double)A.C) / A.S;
+                        const double q = exp2((double)xd * scale_d - (double)D.C) / D.S;
+                        if (P.out_p) P.out_p[lo + j] = (float)p;
+                        if (P.out_q) P.out_q[lo + j] = (float)q;
+                        float ua, ur;
+                        philox_uniforms(P.seed, (uint32_t)r, (uint32_t)j, ua, ur);
+                        if (!((double)ua * q < p)) atomicMin(&s_first, j);     // rejected
+                    }
                 }
             }
         }
         __syncthreads();
-        const bool stop = s_bad || (!want_all && s_first < len);
+        const int first = s_first;
+        const bool in_round = first >= j0 && first < j0 + kWarps;
+        if (tid == 0 && in_round && !s_have_fin) {      // the row that emits the token sits in this round
+            const int w = first - j0;
+            s_fin_C[0] = s_Ct[w]; s_fin_S[0] = s_St[w]; s_fin_C[1] = s_Cd[w]; s_fin_S[1] = s_Sd[w];
+            s_have_fin = 1;
+        }
+        const bool stop = s_bad || (!want_all && first < len);
         __syncthreads();                         // everyone has read the flags before the next round updates them
         if (stop) break;
     }
-    if (warp != 0) return;
+    if (tid != 0) return;
 
     if (s_bad) {
-        if (lane == 0) { atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
+        atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone;
         return;
     }
     const int n = s_first;
-    float Cp; double Sp;
-    combine_row(P.stats_t + (long long)(lo + n) * P.nblk, P.nblk, lane, Cp, Sp);
-    if (!row_usable(Cp, Sp)) {
-        if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
+    const float Cp = s_fin_C[0];
+    const double Sp = s_fin_S[0];
+    if (!s_have_fin || !row_usable(Cp, Sp)) {
+        atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone;
         return;
     }
-    float Cq = 0.f; double Sq = 1.0;
-    if (n < len) combine_row(P.stats_d + (long long)(lo - r + n) * P.nblk, P.nblk, lane, Cq, Sq);
-    for (int i = lane; i < n; i += 32) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
-    if (lane == 0) {
-        float ua, ur;
-        philox_uniforms(P.seed, (uint32_t)r, (uint32_t)n, ua, ur);
-        RequestTask t;
-        t.n = n; t.u = ur; t.slot = -1;
-        t.cp = Cp; t.inv_zp = (float)(1.0 / Sp);
-        t.cq = Cq; t.inv_zq = (float)(1.0 / Sq);
-        t.row_d = drow0 + n;
-        if (n < len) {
-            const int slot = atomicAdd(&P.counters[0], 1);
-            ResidTask q;
-            q.request = r; q.row_t = lo + n; q.row_d = t.row_d;
-            q.cp = t.cp; q.inv_zp = t.inv_zp; q.cq = t.cq; q.inv_zq = t.inv_zq;
-            P.resid[slot] = q;
-            t.kind = kTaskResid; t.slot = slot;
-        } else {
-            t.kind = kTaskBonus;
-        }
-        P.req[r] = t;
-        P.accepted_len[r] = n;
+    for (int i = 0; i < n; ++i) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
+    float ua, ur;
+    philox_uniforms(P.seed, (uint32_t)r, (uint32_t)n, ua, ur);
+    RequestTask t;
+    t.n = n; t.u = ur; t.slot = -1;
+    t.cp = Cp; t.inv_zp = (float)(1.0 / Sp);
+    t.cq = 0.f; t.inv_zq = 1.f;
+    t.row_d = drow0 + n;
+    if (n < len) {
+        t.cq = s_fin_C[1]; t.inv_zq = (float)(1.0 / s_fin_S[1]);
+        const int slot = atomicAdd(&P.counters[0], 1);
+        ResidTask q;
+        q.request = r; q.row_t = lo + n; q.row_d = t.row_d;
+        q.cp = t.cp; q.inv_zp = t.inv_zp; q.cq = t.cq; q.inv_zq = t.inv_zq;
+        P.resid[slot] = q;
+        t.kind = kTaskResid; t.slot = slot;
+    } else {
+        t.kind = kTaskBonus;
     }
+    P.req[r] = t;
+    P.accepted_len[r] = n;
 }
 
 // ---------------------------------------------------------------------------------------
 // finalize: one warp per request.  Inverse CDF in vocabulary order: first over per-block
 // sums (fp64 running sum), then over the elements of the one block that holds the crossing.
+// Each lane owns a contiguous run; values are held in registers.
 // ---------------------------------------------------------------------------------------
 
-// Finds, over values val(b) for b in [0, n) taken in index order, the first index whose
-// inclusive running sum exceeds thr.  Each lane owns a contiguous run.  Returns the index
-// (or -1), the exclusive sum before it, and the grand total.
-template <typename F>
-__device__ __forceinline__ int warp_first_crossing(int n, int lane, double thr, F val, double& before, double& total,
-                                                   int& last_positive)
+// Over values x[0..cnt) of each lane (lane-major order = index order), finds the first index whose
+// inclusive running sum exceeds thr(total).  kMax values per lane.  Returns the global index
+// lane*per + k (or -1), the exclusive sum before it, the total and the last positive index.
+template <int kMax, typename Thr>
+__device__ __forceinline__ int warp_crossing(const float (&x)[kMax], int per, int cnt, int lane, Thr thr_of,
+                                             double& before, double& total, int& last_positive)
 {
-    const int per = (n + 31) / 32;
-    const int b0 = lane * per, b1 = (b0 + per < n) ? b0 + per : n;
     double mine = 0.0;
     int lastp = -1;
-    for (int b = b0; b < b1; ++b) { const double x = val(b); mine += x; if (x > 0.0) lastp = b; }
+#pragma unroll
+    for (int k = 0; k < kMax; ++k)
+        if (k < cnt) { mine += (double)x[k]; if (x[k] > 0.f) lastp = lane * per + k; }
     double incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -600,8 +704,8 @@ __device__ __forceinline__ int warp_first_crossing(int n, int lane, double thr, 
         if (lane >= o) incl += t;
     }
     total = __shfl_sync(0xffffffffu, incl, 31);
-    const double excl = incl - mine;
-    const unsigned hit = __ballot_sync(0xffffffffu, incl > thr && b0 < b1);
+    const double thr = thr_of(total);
+    const unsigned hit = __ballot_sync(0xffffffffu, incl > thr && cnt > 0);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) lastp = max(lastp, __shfl_xor_sync(0xffffffffu, lastp, o));
     last_positive = lastp;
@@ -610,21 +714,96 @@ __device__ __forceinline__ int warp_first_crossing(int n, int lane, double thr, 
     int found = -1;
     double bef = 0.0;
     if (lane == src) {
-        double run = excl;
-        for (int b = b0; b < b1; ++b) {
-            const double x = val(b);
-            if (run + x > thr) { found = b; bef = run; break; }
-            run += x;
+        double run = incl - mine;
+#pragma unroll
+        for (int k = 0; k < kMax; ++k) {
+            if (k < cnt && found < 0) {
+                if (run + (double)x[k] > thr) { found = lane * per + k; bef = run; }
+                else run += (double)x[k];
+            }
         }
-        if (found < 0) { found = b1 - 1; bef = run; }   // only by rounding between the two sums
+        if (found < 0) { found = lane * per + cnt - 1; bef = run; }   // only by rounding between the two sums
     }
     found = __shfl_sync(0xffffffffu, found, src);
     before = __shfl_sync(0xffffffffu, bef, src);
     return found;
 }
 
+// Loads this lane's contiguous run of a block: `per` elements starting at element e_begin of the
+// row, as fp32 values; elements at or beyond V read -inf.  16-byte loads when the address allows.
+template <int kElem, int kPer>
+__device__ __forceinline__ void load_run(const unsigned char* row, int e_begin, int V, float (&x)[kPer])
+{
+    const unsigned char* p = row + (long long)e_begin * kElem;
+    constexpr int kBytes = kPer * kElem;
+    if (e_begin + kPer <= V && ((uintptr_t)p & 15u) == 0) {
+#pragma unroll
+        for (int k = 0; k < kBytes / 16; ++k) {
+            const uint4 q = __ldg((const uint4*)(p + 16 * k));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t w = word_of(q, i);
+                if (kElem == 2) { x[k * 8 + 2 * i] = bf16lo(w); x[k * 8 + 2 * i + 1] = bf16hi(w); }
+                else x[k * 4 + i] = __uint_as_float(w);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < kPer; ++k) {
+            float val = kNegInf;
+            if (e_begin + k < V) {
+                if (kElem == 2) val = __uint_as_float((uint32_t)__ldg((const unsigned short*)(p + 2 * k)) << 16);
+                else val = __ldg((const float*)(p + 4 * k));
+            }
+            x[k] = val;
+        }
+    }
+}
+
+// Level 1 of the inverse CDF: over n block values val(i) in index order, the first block whose
+// inclusive running sum exceeds u * total.  Up to 256 blocks are held in registers (8 per lane);
+// longer rows take the total first and then walk chunks of 256 blocks in order.
+template <typename F>
+__device__ __forceinline__ int block_crossing(int n, int lane, double u, F val, double& before, double& total,
+                                              int& last_positive)
+{
+    int b = -1;
+    last_positive = -1;
+    before = 0.0;
+    if (n <= 256) {
+        const int per = (n + 31) / 32;
+        float x[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { const int i = lane * per + k; x[k] = (k < per && i < n) ? val(i) : 0.f; }
+        int cnt = n - lane * per; cnt = cnt < 0 ? 0 : (cnt > per ? per : cnt);
+        b = warp_crossing<8>(x, per, cnt, lane, [&](double tot) { return u * tot; }, before, total, last_positive);
+    } else {
+        double tot = 0.0;
+        for (int i = lane; i < n; i += 32) tot += (double)val(i);
+        total = warp_sum_f64(tot);
+        const double thr = u * total;
+        double run = 0.0;
+        for (int base = 0; base < n && b < 0; base += 256) {
+            float x[8];
+            int cnt = n - base - lane * 8; cnt = cnt < 0 ? 0 : (cnt > 8 ? 8 : cnt);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) x[k] = (k < cnt) ? val(base + lane * 8 + k) : 0.f;
+            double bef, tot_c;
+            int lp;
+            const int f = warp_crossing<8>(x, 8, cnt, lane, [&](double) { return thr - run; }, bef, tot_c, lp);
+            if (lp >= 0) last_positive = base + lp;
+            if (f >= 0) { b = base + f; before = run + bef; }
+            run += tot_c;
+        }
+    }
+    return b;
+}
+
+template <int kElem>
 __global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(VerifyParams P)
 {
+    constexpr int kPerStat = kStatBlockBytes / kElem / 32;     // elements per lane in a statistics block
+    constexpr int kPerResid = kResidBlockBytes / kElem / 32;   // elements per lane in a residual block
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * (kFinalizeThreads / 32) + (threadIdx.x >> 5);
     if (r >= P.R) return;
@@ -632,72 +811,70 @@ __global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(VerifyParams
     if (t.kind == kTaskNone) return;
     const int lo = P.row_offsets[r];
     const int row_t = lo + t.n;
+    const unsigned char* trow = P.target + (long long)row_t * P.tstride_bytes;
     int token = -1;
     bool from_p = (t.kind == kTaskBonus);
-
-    ResidTask rt;
-    rt.cp = t.cp; rt.inv_zp = t.inv_zp; rt.cq = t.cq; rt.inv_zq = t.inv_zq;
+    const double u = (double)t.u;
 
     if (t.kind == kTaskResid) {
-        const float* wb = P.wblk + (long long)t.slot * P.nblk;
+        const float* wb = P.wblk + (long long)t.slot * P.nblk_r;
+        const unsigned char* drow = P.draft + t.row_d * P.dstride_bytes;
+        ResidConst K;
+        K.set(P.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
         double before, W;
         int lastp;
-        // total first (thr depends on it), then the crossing
-        warp_first_crossing(P.nblk, lane, INFINITY, [&](int b) { return (double)__ldcg(&wb[b]); }, before, W, lastp);
+        int b = block_crossing(P.nblk_r, lane, u, [&](int i) { return __ldcg(&wb[i]); }, before, W, lastp);
         if (!(W > 0.0) || !(W < INFINITY)) {
             from_p = true;                                   // empty residual: draw from p with the same u
         } else {
-            const double thr = (double)t.u * W;
-            int b = warp_first_crossing(P.nblk, lane, thr, [&](int bb) { return (double)__ldcg(&wb[bb]); }, before, W, lastp);
             if (b < 0) b = lastp;
-            const int e0 = b * P.epb;
-            const int ne = (P.V - e0) < P.epb ? (P.V - e0) : P.epb;
-            auto w_of = [&](int e) {
-                const float xt = load_logit(P.target, row_t, P.tstride_bytes, P.elem, e0 + e);
-                const float xd = load_logit(P.draft, t.row_d, P.dstride_bytes, P.elem, e0 + e);
-                return (double)resid_elem(xt, xd, P.scale, rt);
-            };
+            const int e0 = b * P.epb_r + lane * kPerResid;
+            float xt[kPerResid], xd[kPerResid], w[kPerResid];
+            load_run<kElem, kPerResid>(trow, e0, P.V, xt);
+            load_run<kElem, kPerResid>(drow, e0, P.V, xd);
+#pragma unroll
+            for (int k = 0; k < kPerResid; ++k) w[k] = resid_elem(xt[k], xd[k], K);
+            int cnt = P.V - e0; cnt = cnt < 0 ? 0 : (cnt > kPerResid ? kPerResid : cnt);
+            const double thr_local = u * W - before;
             double bef2, tot2;
             int lp2;
-            int e = warp_first_crossing(ne, lane, thr - before, w_of, bef2, tot2, lp2);
+            int e = warp_crossing<kPerResid>(w, kPerResid, cnt, lane, [&](double) { return thr_local; }, bef2, tot2, lp2);
             if (e < 0) e = lp2 >= 0 ? lp2 : 0;
-            token = e0 + e;
+            token = b * P.epb_r + e;
         }
     }
     if (from_p) {
         const float2* st = P.stats_t + (long long)row_t * P.nblk;
         const float C = t.cp;
-        auto mass = [&](int b) {
-            const float2 e = __ldcg(&st[b]);
-            return e.x > kNegInf ? (double)(e.y * ex2_approx(e.x - C)) : 0.0;
+        auto mass = [&](int i) {
+            const float2 e = __ldcg(&st[i]);
+            return e.x > kNegInf ? e.y * ex2_approx(e.x - C) : 0.f;
         };
         double before, Z;
         int lastp;
-        warp_first_crossing(P.nblk, lane, INFINITY, mass, before, Z, lastp);
-        const double thr = (double)t.u * Z;
-        int b = warp_first_crossing(P.nblk, lane, thr, mass, before, Z, lastp);
+        int b = block_crossing(P.nblk, lane, u, mass, before, Z, lastp);
         if (b < 0) b = lastp >= 0 ? lastp : 0;
         const float2 sb = __ldcg(&st[b]);
-        const int e0 = b * P.epb;
-        const int ne = (P.V - e0) < P.epb ? (P.V - e0) : P.epb;
+        const int e0 = b * P.epb + lane * kPerStat;
+        float x[kPerStat];
+        load_run<kElem, kPerStat>(trow, e0, P.V, x);
         // inside the block work in the block's own reference: divide the remaining mass by 2^(c_b - C)
-        const double thr_local = (thr - before) / (double)ex2_approx(sb.x - C);
+        const double thr_local = (u * Z - before) / (double)ex2_approx(sb.x - C);
         const float nc = -sb.x;
-        auto e_of = [&](int e) {
-            const float x = load_logit(P.target, row_t, P.tstride_bytes, P.elem, e0 + e);
-            return (double)ex2_approx(__fmaf_rn(x, P.scale, nc));
-        };
+#pragma unroll
+        for (int k = 0; k < kPerStat; ++k) x[k] = ex2_approx(__fmaf_rn(x[k], P.scale, nc));
+        int cnt = P.V - e0; cnt = cnt < 0 ? 0 : (cnt > kPerStat ? kPerStat : cnt);
         double bef2, tot2;
         int lp2;
-        int e = warp_first_crossing(ne, lane, thr_local, e_of, bef2, tot2, lp2);
+        int e = warp_crossing<kPerStat>(x, kPerStat, cnt, lane, [&](double) { return thr_local; }, bef2, tot2, lp2);
         if (e < 0) e = lp2 >= 0 ? lp2 : 0;
-        token = e0 + e;
+        token = b * P.epb + e;
     }
     if (lane == 0) P.out_tokens[row_t] = token;
 }
 
 // ---------------------------------------------------------------------------------------
-// greedy decide: one warp per request.
+// greedy decide: one warp per request, one lane per row (all rows of a request in flight).
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kDecideThreads) greedy_decide_kernel(VerifyParams P)
 {
@@ -723,25 +900,34 @@ __global__ void __launch_bounds__(kDecideThreads) greedy_decide_kernel(VerifyPar
     }
     __syncwarp();
     int n = len, emitted = -1, status = 0;
-    for (int j = 0; j <= len; ++j) {
-        const float2* st = P.stats_t + (long long)(lo + j) * P.nblk;
-        float best = kNegInf;
-        int bi = 0x7fffffff;
-        for (int b = lane; b < P.nblk; b += 32) {
-            const float2 e = __ldcg(&st[b]);
-            const int idx = __float_as_int(e.y);
-            if (e.x > best || (e.x == best && idx < bi)) { best = e.x; bi = idx; }
+    bool done = false;
+    for (int j0 = 0; j0 <= len && !done; j0 += 32) {
+        const int j = j0 + lane;
+        int am = -1, neg = 0;
+        if (j <= len) {
+            const float2* st = P.stats_t + (long long)(lo + j) * P.nblk;
+            float best = kNegInf;
+            int bi = 0x7fffffff;
+#pragma unroll 4
+            for (int b = 0; b < P.nblk; ++b) {
+                const float2 e = __ldcg(&st[b]);
+                const int idx = __float_as_int(e.y);
+                if (e.x > best || (e.x == best && idx < bi)) { best = e.x; bi = idx; }
+            }
+            am = bi;
+            if (best == kNegInf) { am = 0; neg = 1; }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+        const bool ends = (j < len) ? (P.draft_tokens[lo + j] != am) : (j == len);   // mismatch, or the bonus row
+        const unsigned mm = __ballot_sync(0xffffffffu, ends);
+        unsigned negs = __ballot_sync(0xffffffffu, neg);
+        if (mm) {
+            const int src = __ffs(mm) - 1;
+            n = j0 + src;
+            emitted = __shfl_sync(0xffffffffu, am, src);
+            negs &= (src == 31) ? 0xffffffffu : ((2u << src) - 1u);   // only rows up to the one that emits
+            done = true;
         }
-        int am = bi;
-        if (best == kNegInf) { am = 0; status |= DSPARK_DEV_ALL_NEG_INF; }
-        if (j == len) { emitted = am; break; }
-        if (P.draft_tokens[lo + j] != am) { n = j; emitted = am; break; }
+        if (negs) status |= DSPARK_DEV_ALL_NEG_INF;
     }
     for (int i = lane; i < n; i += 32) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
     if (lane == 0) {
@@ -771,7 +957,7 @@ template <int kElem, int kMode>
 static cudaError_t set_smem_attr()
 {
     return cudaFuncSetAttribute(stream_bulk_kernel<kElem, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                StreamCfg<kElem, kMode>::kSmemBytes);
+                                kStages * kStageBytes);
 }
 
 static bool ensure_attrs()
@@ -793,7 +979,7 @@ static void launch_stream(const VerifyParams& P, bool bulk, long long max_units,
         long long g = (long long)sms * 2;
         if (g > max_units) g = max_units;
         if (g < 1) g = 1;
-        stream_bulk_kernel<kElem, kMode><<<(int)g, kStreamThreads, StreamCfg<kElem, kMode>::kSmemBytes, s>>>(P);
+        stream_bulk_kernel<kElem, kMode><<<(int)g, kStreamThreads, kStages * kStageBytes, s>>>(P);
     } else {
         long long g = (long long)sms * 8;
         if (g > max_units) g = max_units;
@@ -815,7 +1001,8 @@ struct Workspace {
 static Workspace workspace_layout(int R, int n_rows, int V)
 {
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
-    const size_t nblk = (size_t)blocks_per_row(V, 4);
+    const size_t nblk = (size_t)blocks_per_row(V, 4, kStatBlockBytes);
+    const size_t nblk_r = (size_t)blocks_per_row(V, 4, kResidBlockBytes);
     Workspace w;
     size_t o = 0;
     w.counters = o; o += up(64 * sizeof(int));
@@ -823,7 +1010,7 @@ static Workspace workspace_layout(int R, int n_rows, int V)
     w.stats_d = o;  o += up((size_t)n_rows * nblk * sizeof(float2));
     w.resid = o;    o += up((size_t)R * sizeof(ResidTask));
     w.req = o;      o += up((size_t)R * sizeof(RequestTask));
-    w.wblk = o;     o += up((size_t)R * nblk * sizeof(float));
+    w.wblk = o;     o += up((size_t)R * nblk_r * sizeof(float));
     w.total = o;
     return w;
 }
@@ -853,9 +1040,10 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.tstride_bytes = (long long)tstride * elem;
     P.dstride_bytes = (long long)dstride * elem;
     P.V = V; P.elem = elem; P.row_bytes = V * elem;
-    P.nblk = blocks_per_row(V, elem);
-    P.ppr = pieces_per_row(V, elem);
-    P.epb = kBlockBytes / elem;
+    P.nblk = blocks_per_row(V, elem, kStatBlockBytes);
+    P.epb = kStatBlockBytes / elem;
+    P.nblk_r = blocks_per_row(V, elem, kResidBlockBytes);
+    P.epb_r = kResidBlockBytes / elem;
     P.row_offsets = row_offsets; P.draft_row_start = draft_row_start; P.draft_tokens = draft_tokens;
     P.R = R; P.n_rows_cap = n_rows;
     P.scale = 1.0f; P.seed = 0;
@@ -869,6 +1057,8 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.wblk = (float*)(ws + w.wblk);
     return DSPARK_OK;
 }
+
+static long long pieces(int nblk) { return (nblk + kConsumerWarps - 1) / kConsumerWarps; }
 
 }  // namespace dspark
 
@@ -903,7 +1093,7 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
     const bool bulk = !g_force_direct && aligned16(P.target, P.tstride_bytes, P.row_bytes);
     {
         KernelTimerScope timer(DSPARK_K_GREEDY_STREAM, s);
-        launch_stream_dtype<kModeGreedy>(P, bulk, (long long)n_rows * P.ppr, s);
+        launch_stream_dtype<kModeGreedy>(P, bulk, (long long)n_rows * pieces(P.nblk), s);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
@@ -941,7 +1131,7 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
                       aligned16(P.draft, P.dstride_bytes, P.row_bytes);
     {
         KernelTimerScope timer(DSPARK_K_STREAM, s);
-        launch_stream_dtype<kModeStats>(P, bulk, (long long)(2ll * n_rows - R > 0 ? 2ll * n_rows - R : n_rows) * P.ppr, s);
+        launch_stream_dtype<kModeStats>(P, bulk, (2ll * n_rows - R) * pieces(P.nblk), s);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
@@ -951,13 +1141,15 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_RESIDUAL, s);
-        launch_stream_dtype<kModeResid>(P, bulk, (long long)R * P.ppr, s);
+        launch_stream_dtype<kModeResid>(P, bulk, (long long)R * pieces(P.nblk_r), s);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_FINALIZE, s);
         const int warps_per_cta = kFinalizeThreads / 32;
-        finalize_kernel<<<(R + warps_per_cta - 1) / warps_per_cta, kFinalizeThreads, 0, s>>>(P);
+        const int grid = (R + warps_per_cta - 1) / warps_per_cta;
+        if (P.elem == 2) finalize_kernel<2><<<grid, kFinalizeThreads, 0, s>>>(P);
+        else finalize_kernel<4><<<grid, kFinalizeThreads, 0, s>>>(P);
     }
     return launch_status();
 }
