@@ -122,7 +122,7 @@ class Step:
             self.out_len = torch.zeros(R, dtype=torch.int32, device=device)
             self.offsets = torch.zeros(R + 1, dtype=torch.int32, device=device)
             self.sws = B.workspace(B.dspark_schedule_workspace_bytes(R, gamma))
-        self.launches_per_step = (1 if self.sched is not None else 0) + (2 if wl["greedy"] else 4)
+        self.launches_per_step = (2 if self.sched is not None else 0) + (2 if wl["greedy"] else 4)
 
     def run(self, batch, conf=None):
         B = self.B

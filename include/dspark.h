@@ -166,7 +166,7 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
  *  out_p_tok/out_q_tok  device [n_rows] fp32 or NULL: p(x), q(x) at every draft position
  *                   (bonus-row entries are not written).  When NULL, positions after the first
  *                   rejection are not evaluated.
- * Streams every target and draft row once (online softmax statistics per 2 KB block), then
+ * Streams every target and draft row once (online softmax statistics per 4 KB block), then
  * re-reads only the rejected position's row pair of each rejected request.
  * Errors: INVALID_ARG, SHAPE, WORKSPACE, CUDA.
  */
@@ -194,8 +194,8 @@ void dspark_uniforms(uint64_t seed, uint32_t request, uint32_t position,
 typedef struct dspark_ktimer dspark_ktimer_t;
 enum {
     DSPARK_K_SCHEDULE = 0, DSPARK_K_OFFSETS = 1, DSPARK_K_STREAM = 2, DSPARK_K_DECIDE = 3,
-    DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6,
-    DSPARK_K_GREEDY_DECIDE = 7, DSPARK_K_COUNT = 8
+    DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6, DSPARK_K_GREEDY_DECIDE = 7,
+    DSPARK_K_COUNT = 8
 };
 int dspark_ktimer_create(int capacity, dspark_ktimer_t** out);
 int dspark_ktimer_destroy(dspark_ktimer_t* t);

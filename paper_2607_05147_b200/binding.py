@@ -21,8 +21,8 @@ DSPARK_F32, DSPARK_BF16 = 0, 1
 DSPARK_SCHED_EARLY_STOP, DSPARK_SCHED_GLOBAL, DSPARK_SCHED_TOPK = 0, 1, 2
 DEV_BAD_OFFSETS, DEV_BAD_TOKEN, DEV_BAD_ROW, DEV_TIMEOUT = 1, 2, 4, 8
 DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF = 16, 32, 64
-(K_SCHEDULE, K_OFFSETS, K_STREAM, K_DECIDE, K_RESIDUAL, K_FINALIZE,
- K_GREEDY_STREAM, K_GREEDY_DECIDE, K_COUNT) = range(9)
+(K_SCHEDULE, K_OFFSETS, K_STREAM, K_DECIDE, K_RESIDUAL, K_FINALIZE, K_GREEDY_STREAM, K_GREEDY_DECIDE,
+ K_COUNT) = range(9)
 
 EXPORTS = [
     "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",

@@ -98,6 +98,12 @@ __device__ __forceinline__ float lg2_approx(float x)
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Programmatic dependent launch: every kernel of the library is launched so that its CTAs may be
+// scheduled while the previous kernel on the stream drains; pdl_wait() returns once that kernel
+// has completed and its writes are visible, and must precede any read of its results.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Packed pairs of fp32 (sm_100 f32x2 arithmetic: one instruction, two IEEE-rounded results).
 __device__ __forceinline__ uint64_t pack2(float a, float b)
 {
@@ -190,5 +196,22 @@ struct KernelTimerScope {
     cudaStream_t stream;
 };
 int launch_status();   // maps cudaGetLastError() to DSPARK_OK / DSPARK_ERR_CUDA
+
+// Launch with programmatic stream serialization (the kernel must call pdl_wait() first).
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, args...);
+}
 
 }  // namespace dspark

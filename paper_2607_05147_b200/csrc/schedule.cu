@@ -1,15 +1,25 @@
-// dspark_schedule: the hardware-aware prefix scheduler (Algorithm 1; Sections 3.2.2, 4.2)
-// as one single-CTA kernel: survival products -> 64-bit key sort in shared memory ->
-// exact integer prefix sums of the expected-accept mass -> Theta path and stop rule ->
-// per-request lengths, row offsets, expected lengths.  The problem is a few thousand
-// keys: latency-bound, so everything stays inside one CTA with no host round trip.
+// dspark_schedule: the hardware-aware prefix scheduler (Algorithm 1; Sections 3.2.2, 4.2).
+//
+// Algorithm 1 sorts all candidates (r, j) by survival probability and walks the sorted
+// list.  Here nothing is sorted: every request's survival products are already in
+// descending order (a_{r,j} is non-increasing in j), so the position of a candidate in the
+// global order, and the exact expected-accept mass admitted up to it, are sums over all
+// requests of one binary search each.  Two kernels on the caller's stream:
+//   prep   one warp per request: a_{r,j} as a left-to-right fp32 product, per-tile inclusive
+//          prefix sums of the fixed-point mass (units of 2^-40, exact integers);
+//   rank   one CTA per tile of 32 candidates, 32 warps each searching a slice of all tiles
+//          (tiles are loaded coalesced and searched with warp shuffles): candidate c gets
+//          rank_c = #{keys <= key_c} and T_c = R*2^40 + mass of those keys, scattered to
+//          by-rank arrays; the CTA that finishes last (a ticket counter, nobody waits) then
+//          walks the path: Theta_i = T_i * SPS(R + i), stop rule, lengths, offsets.
+// Integer sums are associative, so the result is bit-identical to the sequential walk.
 #include "common.cuh"
 
 namespace dspark {
 
 constexpr int kSchedThreads = 1024;
-constexpr int kSmemKeyCap = 16384;          // 128 KB of 64-bit keys in shared memory
-constexpr unsigned long long kPadKey = ~0ull;
+constexpr int kPrepThreads = 128;
+constexpr int kSmemLenCap = 4096;
 
 struct SchedParams {
     const float* conf;
@@ -22,8 +32,16 @@ struct SchedParams {
     float* out_surv;
     float* out_exp;
     dspark_sched_info_t* info;
-    unsigned long long* keys_global;
-    int n_pad;
+    // geometry: gpad = positions per request after padding (power of two <= 32, or a multiple of 32),
+    // seg = min(gpad, 32) entries per sorted segment, n_tiles tiles of 32 entries
+    int gpad, seg, n_tiles, R_pad;
+    // workspace
+    uint32_t* akey;                 // [n_tiles*32] fp32 bits of a_{r,j}, 0 where not a candidate
+    unsigned long long* pfix;       // [n_tiles*32] inclusive prefix of fix40(a) inside the segment
+    int32_t* cnt;                   // [R] candidates of request r (bit 30: a confidence was clamped)
+    unsigned long long* t_by_rank;  // [N+1] T_i
+    int32_t* owner_by_rank;         // [N+1] request of the i-th admitted candidate
+    int* ticket;                    // counts finished rank CTAs (zeroed by the prep kernel)
 };
 
 __device__ __forceinline__ float sanitize_conf(float c, int& clamped)
@@ -36,9 +54,161 @@ __device__ __forceinline__ unsigned long long fix40(float a)
 {
     return __double2ull_rz(__dmul_rn((double)a, 1099511627776.0));
 }
-__device__ __forceinline__ float key_survival(unsigned long long key)
+
+// ---- S1: survival products (fp32, left to right), segment-local prefix sums ----------------
+// One warp per 32/seg requests (seg = entries per segment): confidences are loaded coalesced,
+// the product chain runs in request order through warp shuffles (every lane follows the same
+// chain and keeps the value of its own position), the mass prefix is a segmented warp scan.
+__global__ void __launch_bounds__(kPrepThreads) sched_prep_kernel(SchedParams P)
 {
-    return __uint_as_float(~(uint32_t)(key >> 32));
+    pdl_launch_dependents();
+    pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0) *P.ticket = 0;
+    const int lane = threadIdx.x & 31;
+    const int wid = blockIdx.x * (kPrepThreads / 32) + (threadIdx.x >> 5);
+    const int gamma = P.gamma, gpad = P.gpad, seg = P.seg;
+    const int req_per_warp = 32 / seg;
+    const int chunks = gpad / seg;                       // 32-entry tiles per request (1 when gpad <= 32)
+    const int sub = lane / seg, k_in_seg = lane - sub * seg;
+    const int r = wid * req_per_warp + sub;
+    if (wid * req_per_warp >= P.R_pad) return;
+    const bool real = r < P.R;
+    int lim = 0;
+    if (real) {
+        lim = gamma;
+        if (P.draft_len) { lim = P.draft_len[r]; lim = lim < 0 ? 0 : (lim > gamma ? gamma : lim); }
+    }
+    float a_run = 1.0f;
+    bool dead = false;
+    int clamped = 0, n = 0;
+    for (int q = 0; q < chunks; ++q) {
+        const int j = q * seg + k_in_seg;
+        float c = 0.0f;
+        if (real && j < lim) c = P.conf[(size_t)r * gamma + j];
+        float mine = 0.0f;
+        for (int k = 0; k < seg; ++k) {
+            const float ck = __shfl_sync(0xffffffffu, c, sub * seg + k);
+            if (q * seg + k >= lim) dead = true;
+            if (!dead) {                                  // only confidences actually multiplied are judged
+                a_run = __fmul_rn(a_run, sanitize_conf(ck, clamped));
+                if (!(a_run > 0.0f)) dead = true;
+            }
+            if (k == k_in_seg) mine = dead ? 0.0f : a_run;
+        }
+        unsigned long long pre = mine > 0.0f ? fix40(mine) : 0ull;
+        for (int o = 1; o < seg; o <<= 1) {
+            const unsigned long long up = __shfl_up_sync(0xffffffffu, pre, o, seg);
+            if (k_in_seg >= o) pre += up;
+        }
+        const unsigned live = __ballot_sync(0xffffffffu, mine > 0.0f);
+        const unsigned segmask = (seg == 32) ? 0xffffffffu : (((1u << seg) - 1u) << (sub * seg));
+        n += __popc(live & segmask);
+        const size_t e = (size_t)r * gpad + j;
+        P.akey[e] = __float_as_uint(mine);
+        P.pfix[e] = pre;
+        if (real && j < gamma && P.out_surv) P.out_surv[(size_t)r * gamma + j] = mine;
+    }
+    if (real && k_in_seg == 0) P.cnt[r] = n | (clamped ? (1 << 30) : 0);
+}
+
+// ---- S2 + S3 without a sort: rank and admitted mass of every candidate ------------------------
+// key order: a descending, then position ascending, then request ascending.
+__device__ __forceinline__ bool key_le(uint32_t a2, int j2, int r2, uint32_t a1, int j1, int r1)
+{
+    // is key (a2, j2, r2) at or before key (a1, j1, r1) in the admission order?
+    return a2 > a1 || (a2 == a1 && (j2 < j1 || (j2 == j1 && r2 <= r1)));
+}
+
+// Searches one sorted segment (SEG entries held one per lane starting at lane `base`, the first
+// `cnt` of them candidates) for the number of entries at or before my key.  The common case needs
+// only the strict comparison on a; a warp that sees an exact tie redoes the search with the full key.
+template <int SEG>
+__device__ __forceinline__ int segment_search(uint32_t ak, int base, int cnt, uint32_t a1, int j1, int r1,
+                                              int j_base, int r2)
+{
+    int pos = 0;
+#pragma unroll
+    for (int step = SEG; step >= 1; step >>= 1) {
+        const int probe = pos + step;
+        const uint32_t a2 = __shfl_sync(0xffffffffu, ak, base + (probe <= SEG ? probe : SEG) - 1);
+        if (probe <= cnt && a2 > a1) pos = probe;
+    }
+    const uint32_t a_next = __shfl_sync(0xffffffffu, ak, base + (pos < SEG ? pos : SEG - 1));
+    if (__any_sync(0xffffffffu, pos < cnt && a_next == a1)) {
+        pos = 0;
+#pragma unroll
+        for (int step = SEG; step >= 1; step >>= 1) {
+            const int probe = pos + step;
+            const uint32_t a2 = __shfl_sync(0xffffffffu, ak, base + (probe <= SEG ? probe : SEG) - 1);
+            if (probe <= cnt && key_le(a2, j_base + probe - 1, r2, a1, j1, r1)) pos = probe;
+        }
+    }
+    return pos;
+}
+
+__device__ void sched_final_stage(const SchedParams& P);
+
+template <int SEG>
+__global__ void __launch_bounds__(kSchedThreads, 1) sched_rank_kernel(SchedParams P)
+{
+    constexpr int kWarps = kSchedThreads / 32;
+    constexpr int kSegsPerTile = 32 / SEG;
+    __shared__ unsigned int s_rank[kWarps][32];
+    __shared__ unsigned long long s_mass[kWarps][32];
+    __shared__ int s_is_last;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int tile = blockIdx.x;
+    const int tiles_per_req = P.gpad > 32 ? P.gpad / 32 : 1;
+
+    // my candidate
+    const int e = tile * 32 + lane;            // flat padded entry index
+    const uint32_t a1 = P.akey[e];
+    const int r1 = P.gpad > 32 ? tile / tiles_per_req : e / P.gpad;
+    const int j1 = e - r1 * P.gpad;
+
+    unsigned int rank = 0;
+    unsigned long long mass = 0ull;
+    for (int t = warp; t < P.n_tiles; t += kWarps) {
+        const uint32_t ak = P.akey[t * 32 + lane];
+        const unsigned long long pf = P.pfix[t * 32 + lane];
+        const unsigned valid = __ballot_sync(0xffffffffu, ak != 0u);
+        if (valid == 0u) continue;
+#pragma unroll
+        for (int sgi = 0; sgi < kSegsPerTile; ++sgi) {
+            const int base = sgi * SEG;
+            const unsigned segmask = (SEG == 32) ? 0xffffffffu : (((1u << SEG) - 1u) << base);
+            const int cnt = __popc(valid & segmask);      // candidates form a prefix of the segment
+            const int r2 = P.gpad > 32 ? t / tiles_per_req : (t * 32 + base) / P.gpad;
+            const int j_base = P.gpad > 32 ? (t - r2 * tiles_per_req) * 32 : 0;
+            const int pos = segment_search<SEG>(ak, base, cnt, a1, j1, r1, j_base, r2);
+            const unsigned long long m = __shfl_sync(0xffffffffu, pf, base + (pos > 0 ? pos - 1 : 0));
+            if (pos > 0) { rank += (unsigned)pos; mass += m; }
+        }
+    }
+    s_rank[warp][lane] = rank;
+    s_mass[warp][lane] = mass;
+    __syncthreads();
+    if (warp == 0 && a1 != 0u) {
+        unsigned int rk = 0;
+        unsigned long long ms = (unsigned long long)P.R << 40;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { rk += s_rank[w][lane]; ms += s_mass[w][lane]; }
+        // rk is the 1-based place of this candidate on the admission path, ms is T at that place
+        P.t_by_rank[rk] = ms;
+        P.owner_by_rank[rk] = r1;
+    }
+    // the CTA that finishes last walks the path (no CTA ever waits for another)
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_is_last = (atomicAdd(P.ticket, 1) == (int)gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    __threadfence();
+    sched_final_stage(P);
 }
 
 // Inclusive scan of one 64-bit value per thread over the CTA (1024 threads).
@@ -67,11 +237,9 @@ __device__ __forceinline__ unsigned long long block_scan_u64(unsigned long long 
     return v;
 }
 
-template <bool kSmemKeys>
-__global__ void __launch_bounds__(kSchedThreads, 1) schedule_kernel(SchedParams P)
+// ---- S3 + S4: Theta path, stop rule, lengths, offsets (one CTA of 1024 threads) -------------
+__device__ void sched_final_stage(const SchedParams& P)
 {
-    extern __shared__ __align__(16) unsigned long long smem_keys[];
-    unsigned long long* keys = kSmemKeys ? smem_keys : P.keys_global;
     __shared__ unsigned long long s_warp_tot[32];
     __shared__ unsigned long long s_carry, s_T_best;
     __shared__ double s_theta_best;
@@ -80,60 +248,26 @@ __global__ void __launch_bounds__(kSchedThreads, 1) schedule_kernel(SchedParams 
     __shared__ int s_red_i[32];
     __shared__ unsigned long long s_red_T[32];
 
+    __shared__ int s_len[kSmemLenCap];        // per-request lengths while R fits (else global out_len)
     const int tid = threadIdx.x;
-    const int R = P.R, gamma = P.gamma;
-    const int n = R * gamma;
-
+    const int R = P.R;
+    const bool len_in_smem = R <= kSmemLenCap;
+    int* len_arr = len_in_smem ? s_len : P.out_len;
     if (tid == 0) { s_nE = 0; s_status = 0; s_first_bad = 0x7fffffff; s_done = 0; }
     __syncthreads();
-
-    // ---- S1: survival products a_{r,j} (fp32, left to right) and sort keys --------------
     {
-        int my_cand = 0, clamped = 0;
+        int n = 0, cl = 0;
         for (int r = tid; r < R; r += kSchedThreads) {
-            int lim = gamma;
-            if (P.draft_len) { lim = P.draft_len[r]; lim = lim < 0 ? 0 : (lim > gamma ? gamma : lim); }
-            float a = 1.0f;
-            bool dead = false;
-            for (int j = 0; j < gamma; ++j) {
-                if (j >= lim) dead = true;
-                if (!dead) {
-                    a = __fmul_rn(a, sanitize_conf(P.conf[(size_t)r * gamma + j], clamped));
-                    if (!(a > 0.0f)) dead = true;
-                }
-                float s = dead ? 0.0f : a;
-                if (P.out_surv) P.out_surv[(size_t)r * gamma + j] = s;
-                unsigned long long key = kPadKey;
-                if (!dead) {
-                    // ascending key order == (a descending, position ascending, request ascending)
-                    key = ((unsigned long long)(~__float_as_uint(s)) << 32) | ((unsigned)j << 20) | (unsigned)r;
-                    ++my_cand;
-                }
-                keys[(size_t)r * gamma + j] = key;
-            }
+            const int c = P.cnt[r];
+            n += c & 0x3fffffff;
+            cl |= c >> 30;
+            len_arr[r] = 0;
         }
-        for (int i = n + tid; i < P.n_pad; i += kSchedThreads) keys[i] = kPadKey;
-        if (my_cand) atomicAdd(&s_nE, my_cand);
-        if (clamped) atomicOr(&s_status, DSPARK_DEV_CONF_CLAMPED);
+        if (n) atomicAdd(&s_nE, n);
+        if (cl) atomicOr(&s_status, DSPARK_DEV_CONF_CLAMPED);
     }
     __syncthreads();
 
-    // ---- S2: bitonic sort, ascending ----------------------------------------------------
-    const int np = P.n_pad;
-    for (int k = 2; k <= np; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = tid; i < (np >> 1); i += kSchedThreads) {
-                int lo = ((i & ~(j - 1)) << 1) | (i & (j - 1));
-                int hi = lo + j;
-                unsigned long long x = keys[lo], y = keys[hi];
-                bool up = (lo & k) == 0;
-                if ((x > y) == up) { keys[lo] = y; keys[hi] = x; }
-            }
-            __syncthreads();
-        }
-    }
-
-    // ---- S3 + S4: admission path, Theta_i = tau_i * SPS(R + i), stop rule -----------------
     const int nE = s_nE;
     long long cap = (long long)P.budget - (long long)R;
     if (cap < 0) { cap = 0; if (tid == 0) s_status |= DSPARK_DEV_BUDGET_LT_R; }
@@ -141,7 +275,6 @@ __global__ void __launch_bounds__(kSchedThreads, 1) schedule_kernel(SchedParams 
     const unsigned long long T0 = (unsigned long long)R << 40;
     const int mt = P.max_tokens;
     if (tid == 0) {
-        s_carry = T0;
         s_T_best = T0;
         s_theta_best = __dmul_rn(__ull2double_rn(T0), P.table[R < mt ? R : mt]);
         s_istar = 0;
@@ -151,17 +284,18 @@ __global__ void __launch_bounds__(kSchedThreads, 1) schedule_kernel(SchedParams 
     for (int base = 0; base < N; base += kSchedThreads) {
         const int i = base + tid + 1;                 // 1-based admitted count
         const bool valid = i <= N;
-        unsigned long long v = valid ? fix40(key_survival(keys[i - 1])) : 0ull;
-        unsigned long long Ti = block_scan_u64(v, s_warp_tot) + s_carry;
+        unsigned long long Ti = 0ull, Tp = 0ull;
         double theta_i = 0.0;
         if (valid) {
-            int B = R + i;
+            Ti = P.t_by_rank[i];
+            Tp = (i == 1) ? T0 : P.t_by_rank[i - 1];
+            const int B = R + i;
             theta_i = __dmul_rn(__ull2double_rn(Ti), P.table[B < mt ? B : mt]);
         }
         if (P.mode == DSPARK_SCHED_EARLY_STOP) {
             if (valid) {
-                int Bp = R + i - 1;
-                double theta_prev = __dmul_rn(__ull2double_rn(Ti - v), P.table[Bp < mt ? Bp : mt]);
+                const int Bp = R + i - 1;
+                const double theta_prev = __dmul_rn(__ull2double_rn(Tp), P.table[Bp < mt ? Bp : mt]);
                 if (!(theta_i > theta_prev)) atomicMin(&s_first_bad, i);
             }
             __syncthreads();
@@ -201,26 +335,26 @@ __global__ void __launch_bounds__(kSchedThreads, 1) schedule_kernel(SchedParams 
             const int istar = N < K ? N : K;
             if (valid && i == istar) { s_T_best = Ti; s_theta_best = theta_i; s_istar = i; }
         }
-        if (tid == kSchedThreads - 1) s_carry = Ti;
         __syncthreads();
         if (s_done) break;
     }
     __syncthreads();
     const int istar = s_istar;
 
-    // ---- lengths l*_r = admitted candidates of request r ---------------------------------
-    for (int r = tid; r < R; r += kSchedThreads) P.out_len[r] = 0;
+    // ---- lengths l*_r = admitted candidates of request r -----------------------------------
+    for (int k = tid + 1; k <= istar; k += kSchedThreads) atomicAdd(&len_arr[P.owner_by_rank[k]], 1);
     __syncthreads();
-    for (int k = tid; k < istar; k += kSchedThreads) atomicAdd(&P.out_len[(int)(keys[k] & 0xFFFFFu)], 1);
-    __syncthreads();
+    if (len_in_smem)
+        for (int r = tid; r < R; r += kSchedThreads) P.out_len[r] = s_len[r];
 
-    // ---- row offsets: exclusive scan of (l*_r + 1) ---------------------------------------
+    // ---- row offsets: exclusive scan of (l*_r + 1) -------------------------------------------
     if (P.out_offsets) {
         if (tid == 0) s_carry = 0ull;
         __syncthreads();
         for (int base = 0; base < R; base += kSchedThreads) {
             const int r = base + tid;
-            unsigned long long v = r < R ? (unsigned long long)(__ldcg(&P.out_len[r]) + 1) : 0ull;
+            unsigned long long v = 0ull;
+            if (r < R) v = (unsigned long long)((len_in_smem ? s_len[r] : __ldcg(&P.out_len[r])) + 1);
             unsigned long long incl = block_scan_u64(v, s_warp_tot) + s_carry;
             if (r < R) P.out_offsets[r] = (int32_t)(incl - v);
             if (r == R - 1) P.out_offsets[R] = (int32_t)incl;
@@ -230,17 +364,13 @@ __global__ void __launch_bounds__(kSchedThreads, 1) schedule_kernel(SchedParams 
         }
     }
 
-    // ---- expected accepted length 1 + sum_{j < l*_r} a_{r,j} -----------------------------
+    // ---- expected accepted length 1 + sum_{j < l*_r} a_{r,j} ---------------------------------
     if (P.out_exp) {
         for (int r = tid; r < R; r += kSchedThreads) {
-            const int len = __ldcg(&P.out_len[r]);
-            float a = 1.0f;
+            const int len = len_in_smem ? s_len[r] : __ldcg(&P.out_len[r]);
             double e = 1.0;
-            int dummy = 0;
-            for (int j = 0; j < len; ++j) {
-                a = __fmul_rn(a, sanitize_conf(P.conf[(size_t)r * gamma + j], dummy));
-                e = __dadd_rn(e, (double)a);
-            }
+            for (int j = 0; j < len; ++j)
+                e = __dadd_rn(e, (double)__uint_as_float(P.akey[(size_t)r * P.gpad + j]));
             P.out_exp[r] = (float)e;
         }
     }
@@ -256,11 +386,21 @@ __global__ void __launch_bounds__(kSchedThreads, 1) schedule_kernel(SchedParams 
     }
 }
 
+// No candidates at all (gamma = 0): only the final stage runs.
+__global__ void __launch_bounds__(kSchedThreads, 1) sched_final_only_kernel(SchedParams P)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    sched_final_stage(P);
+}
+
 __global__ void __launch_bounds__(kSchedThreads, 1)
 build_offsets_kernel(const int32_t* __restrict__ lengths, int R, int32_t* __restrict__ offsets)
 {
     __shared__ unsigned long long s_warp_tot[32];
     __shared__ unsigned long long s_carry;
+    pdl_launch_dependents();
+    pdl_wait();
     const int tid = threadIdx.x;
     if (tid == 0) s_carry = 0ull;
     __syncthreads();
@@ -278,11 +418,29 @@ build_offsets_kernel(const int32_t* __restrict__ lengths, int R, int32_t* __rest
     }
 }
 
-static int next_pow2(int x)
+// Padded geometry: positions per request, requests after padding, tiles of 32 entries.
+struct SchedGeom { int gpad, seg, R_pad, n_tiles; size_t akey, pfix, cnt, tbr, obr, ticket, total; };
+static SchedGeom sched_geom(int R, int gamma)
 {
-    int p = 2;
-    while (p < x) p <<= 1;
-    return p;
+    SchedGeom g;
+    int gp = 1;
+    if (gamma <= 32) { while (gp < gamma) gp <<= 1; } else { gp = (gamma + 31) / 32 * 32; }
+    g.gpad = gp;
+    g.seg = gp < 32 ? gp : 32;
+    const int req_per_tile = gp < 32 ? 32 / gp : 1;
+    g.R_pad = (R + req_per_tile - 1) / req_per_tile * req_per_tile;
+    const size_t n_entries = (size_t)g.R_pad * gp;
+    g.n_tiles = (int)(n_entries / 32);
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    size_t o = 0;
+    g.akey = o; o += up(n_entries * sizeof(uint32_t));
+    g.pfix = o; o += up(n_entries * sizeof(unsigned long long));
+    g.cnt = o;  o += up((size_t)R * sizeof(int32_t));
+    g.tbr = o;  o += up((n_entries + 1) * sizeof(unsigned long long));
+    g.obr = o;  o += up((n_entries + 1) * sizeof(int32_t));
+    g.ticket = o; o += up(sizeof(int));
+    g.total = o;
+    return g;
 }
 
 }  // namespace dspark
@@ -294,9 +452,8 @@ extern "C" {
 size_t dspark_schedule_workspace_bytes(int R, int gamma)
 {
     if (R < 1 || gamma < 0) return 0;
-    long long n = (long long)R * gamma;
-    if (n > (1 << 20)) return 0;
-    return (size_t)next_pow2((int)(n > 2 ? n : 2)) * sizeof(unsigned long long);
+    if (R > (1 << 20) || gamma > 4096 || (long long)R * gamma > (1 << 20)) return 0;
+    return sched_geom(R, gamma).total;
 }
 
 int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32_t* draft_len,
@@ -310,35 +467,44 @@ int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32
         return DSPARK_ERR_INVALID_ARG;
     if (R < 1 || gamma < 0) return DSPARK_ERR_INVALID_ARG;
     if (R > (1 << 20) || gamma > 4096 || (long long)R * gamma > (1 << 20)) return DSPARK_ERR_SHAPE;
-    const size_t need = dspark_schedule_workspace_bytes(R, gamma);
-    if (!workspace || workspace_bytes < need) return DSPARK_ERR_WORKSPACE;
-    if (((uintptr_t)workspace & 15u) != 0) return DSPARK_ERR_ALIGNMENT;
+    const SchedGeom g = sched_geom(R, gamma);
+    if (!workspace || workspace_bytes < g.total) return DSPARK_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255u) != 0) return DSPARK_ERR_ALIGNMENT;
 
     int max_tokens = 0;
     const double* table = dspark_profile_table(prof, &max_tokens);
+    unsigned char* ws = (unsigned char*)workspace;
     SchedParams P;
     P.conf = conf; P.draft_len = draft_len;
     P.R = R; P.gamma = gamma; P.budget = budget_tokens; P.mode = mode; P.topk = topk_K;
     P.table = table; P.max_tokens = max_tokens;
     P.out_len = out_len; P.out_offsets = out_row_offsets; P.out_surv = out_survival;
     P.out_exp = out_expected_len; P.info = out_info;
-    P.keys_global = (unsigned long long*)workspace;
-    P.n_pad = next_pow2(R * gamma > 2 ? R * gamma : 2);
+    P.gpad = g.gpad; P.seg = g.seg; P.n_tiles = g.n_tiles; P.R_pad = g.R_pad;
+    P.akey = (uint32_t*)(ws + g.akey);
+    P.pfix = (unsigned long long*)(ws + g.pfix);
+    P.cnt = (int32_t*)(ws + g.cnt);
+    P.t_by_rank = (unsigned long long*)(ws + g.tbr);
+    P.owner_by_rank = (int32_t*)(ws + g.obr);
+    P.ticket = (int*)(ws + g.ticket);
 
     cudaStream_t s = (cudaStream_t)stream;
     KernelTimerScope timer(DSPARK_K_SCHEDULE, s);
-    if (P.n_pad <= kSmemKeyCap) {
-        const size_t smem = (size_t)P.n_pad * sizeof(unsigned long long);
-        static bool attr_set = false;
-        if (!attr_set) {
-            if (cudaFuncSetAttribute(schedule_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kSmemKeyCap * (int)sizeof(unsigned long long)) != cudaSuccess)
-                return launch_status();
-            attr_set = true;
+    const int prep_warps = g.R_pad / (32 / g.seg);
+    const int prep_ctas = (prep_warps + kPrepThreads / 32 - 1) / (kPrepThreads / 32);
+    launch_pdl(sched_prep_kernel, dim3(prep_ctas), dim3(kPrepThreads), 0, s, P);
+    if (g.n_tiles > 0 && gamma > 0) {
+        const dim3 grid(g.n_tiles), block(kSchedThreads);
+        switch (g.seg) {
+            case 1: launch_pdl(sched_rank_kernel<1>, grid, block, 0, s, P); break;
+            case 2: launch_pdl(sched_rank_kernel<2>, grid, block, 0, s, P); break;
+            case 4: launch_pdl(sched_rank_kernel<4>, grid, block, 0, s, P); break;
+            case 8: launch_pdl(sched_rank_kernel<8>, grid, block, 0, s, P); break;
+            case 16: launch_pdl(sched_rank_kernel<16>, grid, block, 0, s, P); break;
+            default: launch_pdl(sched_rank_kernel<32>, grid, block, 0, s, P); break;
         }
-        schedule_kernel<true><<<1, kSchedThreads, smem, s>>>(P);
     } else {
-        schedule_kernel<false><<<1, kSchedThreads, 0, s>>>(P);
+        launch_pdl(sched_final_only_kernel, dim3(1), dim3(kSchedThreads), 0, s, P);
     }
     return launch_status();
 }
@@ -348,7 +514,7 @@ int dspark_build_offsets(const int32_t* lengths, int R, int32_t* row_offsets, vo
     if (!lengths || !row_offsets || R < 1) return DSPARK_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
     KernelTimerScope timer(DSPARK_K_OFFSETS, s);
-    build_offsets_kernel<<<1, kSchedThreads, 0, s>>>(lengths, R, row_offsets);
+    launch_pdl(build_offsets_kernel, dim3(1), dim3(kSchedThreads), 0, s, lengths, R, row_offsets);
     return launch_status();
 }
 

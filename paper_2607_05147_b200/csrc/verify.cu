@@ -8,11 +8,12 @@
 //            feeds a ring of 32 KB shared-memory stages with 1-D bulk async copies
 //            (cp.async.bulk + mbarrier), eight consumer warps drain it.
 //   decide   one CTA per request: combines block statistics into row statistics, gathers
-//            p(x), q(x), runs the accept tests (Philox), finds the first rejection, writes
-//            the accepted prefix, and queues the rejected position for the residual pass.
+//            p(x), q(x), runs the accept tests (Philox), finds the first rejection, writes the
+//            accepted prefix; a fully accepted request draws its bonus token here (inverse CDF
+//            over the saved block statistics, one block re-read); a rejected one is queued.
 //   residual second read of the rejected position's row pair only: per-2KB-block sums of
 //            max(0, p - q), same bulk-copy pipeline with two sources per stage.
-//   finalize one warp per request: inverse CDF over block sums, then inside one block.
+//   finalize one warp per rejected request: inverse CDF over block sums, then inside one block.
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -23,7 +24,6 @@ namespace dspark {
 constexpr int kModeStats = 0, kModeGreedy = 1, kModeResid = 2;
 constexpr int kTaskNone = 0, kTaskResid = 1, kTaskBonus = 2;
 constexpr int kDecideThreads = 256;
-constexpr int kFinalizeThreads = 128;
 constexpr float kNegInf = -INFINITY;
 
 struct __align__(16) ResidTask {     // one rejected request queued for the residual pass
@@ -31,15 +31,8 @@ struct __align__(16) ResidTask {     // one rejected request queued for the resi
     int32_t row_t;                   // target row of the rejected position
     int64_t row_d;                   // physical draft row
     float cp, inv_zp, cq, inv_zq;    // row references (log2 domain) and 1 / row sums
-};
-
-struct __align__(16) RequestTask {   // what finalize needs per request
-    int32_t kind;                    // kTaskNone / kTaskResid / kTaskBonus
-    int32_t n;                       // accepted length
-    int32_t slot;                    // index into the residual list (kTaskResid)
-    float u;                         // resample uniform
-    int64_t row_d;
-    float cp, inv_zp, cq, inv_zq;
+    float u;                         // resample uniform of the rejected position
+    int32_t pad[3];
 };
 
 struct VerifyParams {
@@ -61,12 +54,11 @@ struct VerifyParams {
     float* out_q;
     int32_t* dev_status;
     // workspace
-    int* counters;                            // [0] number of queued residual tasks
+    int* counters;                            // [0] queued residual tasks, [1] dev_status stand-in
     float2* stats_t;
     float2* stats_d;
-    ResidTask* resid;
-    RequestTask* req;
-    float* wblk;
+    ResidTask* resid;                         // queue of rejected requests (decide -> residual pass)
+    float* wblk;                              // per queue slot: residual block sums
 };
 
 template <int kMode> struct ModeCfg {
@@ -108,7 +100,7 @@ __device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
 {
     if (kMode == kModeStats) return n_rows + (n_rows > P.R ? n_rows - P.R : 0);
     if (kMode == kModeGreedy) return n_rows;
-    int nq = __ldcg(&P.counters[0]);
+    const int nq = __ldcg(&P.counters[0]);
     return nq > P.R ? P.R : (nq < 0 ? 0 : nq);
 }
 
@@ -357,9 +349,9 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
     } else {
         uint4 vd[M::kVec];
         load_block<kElem, M::kVec>(f1, nbytes, lane, vd);
-        const float4 c = *reinterpret_cast<const float4*>(&P.resid[s].cp);
+        const ResidTask t = P.resid[s];
         ResidConst K;
-        K.set(P.scale, c.x, c.y, c.z, c.w);
+        K.set(P.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
         const float w = block_resid<kElem, M::kVec>(v, vd, K);
         if (lane == 0) P.wblk[(long long)s * nblk + b] = w;
     }
@@ -400,12 +392,14 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_bulk_kernel(VerifyPa
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kConsumerWarps); }
         s_abort = 0;
         mbar_fence_init();
     }
     __syncthreads();
+    pdl_wait();                                  // everything below reads what earlier kernels wrote
 
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
@@ -459,7 +453,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_bulk_kernel(VerifyPa
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
                 break;
             }
-            const unsigned char* sp = stage_mem + st * kStageBytes + warp * M::kBlockBytes;
+            unsigned char* sp = stage_mem + st * kStageBytes + warp * M::kBlockBytes;
             SmemFetch f0{sp}, f1{sp + M::kPieceBytes};
             consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1);
             __syncwarp();
@@ -476,6 +470,8 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
 {
     using M = ModeCfg<kMode>;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_launch_dependents();
+    pdl_wait();
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
     if (kMode != kModeResid && blockIdx.x == 0 && tid == 0) {
@@ -554,18 +550,242 @@ __device__ __forceinline__ bool row_usable(float C, double S)
 }
 
 // ---------------------------------------------------------------------------------------
-// decide: one CTA per request, one warp per position (eight positions per round).
-// Position j = len is the bonus row (statistics only).
+// Inverse CDF in vocabulary order, two levels, one warp, registers and a 2 KB scratch only:
+//   level 1  over per-block values (residual block sums, or block masses of p): chunks of 32
+//            consecutive blocks are read coalesced, chunk totals reduced with shuffles;
+//   level 2  inside the one block that holds the crossing: its raw logits are staged into
+//            shared memory and every lane walks a contiguous run (rolled loops, small code).
+// All running sums are fp64 sums of the fp32 values in index order.
 // ---------------------------------------------------------------------------------------
+template <typename F>
+__device__ __forceinline__ double warp_total(int n, int lane, F val)
+{
+    double t = 0.0;
+#pragma unroll 4
+    for (int i = lane; i < n; i += 32) t += (double)val(i);
+    return warp_sum_f64(t);
+}
+
+// First index i in [0, n) whose inclusive running sum exceeds thr; -1 if none (then `before` is the
+// total).  `last_positive` = last index with a positive value.
+template <typename F>
+__device__ __forceinline__ int chunked_search(int n, int lane, F val, double thr, double& before, int& last_positive)
+{
+    double run = 0.0;
+    int lastp = -1;
+    for (int g0 = 0; g0 < n; g0 += 1024) {
+        // totals of the 32 chunks of this group: lane c keeps the total of chunk c
+        double mine = 0.0;
+#pragma unroll 2
+        for (int c = 0; c < 32; ++c) {
+            const int i = g0 + c * 32 + lane;
+            if (g0 + c * 32 >= n) break;
+            const float x = i < n ? val(i) : 0.f;
+            const double t = warp_sum_f64((double)x);
+            if (lane == c) mine = t;
+            const unsigned pos = __ballot_sync(0xffffffffu, x > 0.f);
+            if (pos) lastp = g0 + c * 32 + (31 - __clz(pos));
+        }
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        const unsigned hit = __ballot_sync(0xffffffffu, run + incl > thr);
+        if (hit) {
+            const int c = __ffs(hit) - 1;
+            const double bef_chunk = run + __shfl_sync(0xffffffffu, incl - mine, c);
+            const int i = g0 + c * 32 + lane;
+            const float x = i < n ? val(i) : 0.f;
+            double inc2 = (double)x;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double t = __shfl_up_sync(0xffffffffu, inc2, o);
+                if (lane >= o) inc2 += t;
+            }
+            const unsigned hit2 = __ballot_sync(0xffffffffu, bef_chunk + inc2 > thr && i < n);
+            int l = hit2 ? __ffs(hit2) - 1 : -1;
+            if (l < 0) {                                  // only by rounding between the two sums
+                const unsigned pos = __ballot_sync(0xffffffffu, x > 0.f);
+                l = pos ? 31 - __clz(pos) : 0;
+            }
+            before = bef_chunk + __shfl_sync(0xffffffffu, inc2 - (double)x, l);
+            last_positive = lastp;
+            return g0 + c * 32 + l;
+        }
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    before = run;
+    last_positive = lastp;
+    return -1;
+}
+
+// Copies the raw bytes of `cnt` elements of a row (from element e_begin) into shared memory.
+template <int kElem>
+__device__ __forceinline__ void stage_raw(const unsigned char* row, int e_begin, int cnt, unsigned char* dst, int lane)
+{
+    const unsigned char* p = row + (long long)e_begin * kElem;
+    const int bytes = cnt * kElem;
+    int done = 0;
+    if (((uintptr_t)p & 15u) == 0) {
+        const int nvec = bytes >> 4;
+#pragma unroll 4
+        for (int v = lane; v < nvec; v += 32) *reinterpret_cast<uint4*>(dst + 16 * v) = __ldg((const uint4*)(p + 16 * v));
+        done = nvec << 4;
+    }
+    if (kElem == 2) {
+        for (int o = done + 2 * lane; o < bytes; o += 64)
+            *reinterpret_cast<unsigned short*>(dst + o) = __ldg((const unsigned short*)(p + o));
+    } else {
+        for (int o = done + 4 * lane; o < bytes; o += 128)
+            *reinterpret_cast<uint32_t*>(dst + o) = __ldg((const uint32_t*)(p + o));
+    }
+}
+template <int kElem>
+__device__ __forceinline__ float raw_elem(const unsigned char* raw, int i)
+{
+    if (kElem == 2) return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short*>(raw + 2 * i)) << 16);
+    return *reinterpret_cast<const float*>(raw + 4 * i);
+}
+
+// Level 2 over one staged unit of at most 2 KB per row: lane l owns elements [l*per, (l+1)*per).
+// f(xt, xd) is the value of an element.  Returns the element index (or -1), the unit total and the
+// last positive index.
+template <int kElem, typename F>
+__device__ __forceinline__ int raw_unit_search(const unsigned char* t_raw, const unsigned char* d_raw, int cnt, int lane,
+                                               double thr, F f, double& total, int& last_positive)
+{
+    constexpr int kPer = kResidBlockBytes / kElem / 32;
+    const int i0 = lane * kPer;
+    int n_mine = cnt - i0;
+    n_mine = n_mine < 0 ? 0 : (n_mine > kPer ? kPer : n_mine);
+    double mine = 0.0;
+    int lastp = -1;
+#pragma unroll 1
+    for (int k = 0; k < n_mine; ++k) {
+        const float w = f(raw_elem<kElem>(t_raw, i0 + k), d_raw ? raw_elem<kElem>(d_raw, i0 + k) : 0.f);
+        mine += (double)w;
+        if (w > 0.f) lastp = i0 + k;
+    }
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    total = __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) lastp = max(lastp, __shfl_xor_sync(0xffffffffu, lastp, o));
+    last_positive = lastp;
+    const unsigned hit = __ballot_sync(0xffffffffu, incl > thr && n_mine > 0);
+    if (!hit) return -1;
+    const int src = __ffs(hit) - 1;
+    int found = -1;
+    if (lane == src) {
+        double run = incl - mine;
+#pragma unroll 1
+        for (int k = 0; k < n_mine; ++k) {
+            const float w = f(raw_elem<kElem>(t_raw, i0 + k), d_raw ? raw_elem<kElem>(d_raw, i0 + k) : 0.f);
+            if (run + (double)w > thr) { found = i0 + k; break; }
+            run += (double)w;
+        }
+        if (found < 0) found = i0 + n_mine - 1;          // only by rounding between the two sums
+    }
+    return __shfl_sync(0xffffffffu, found, src);
+}
+
+// Draws from p = softmax of target row `row_t` with uniform u, using the block statistics saved by
+// the streamed pass (reference Cp = row reference).  One warp; scratch = 2 KB of shared memory.
+template <int kElem>
+__device__ __forceinline__ int sample_from_p(const VerifyParams& P, int row_t, float Cp, double u,
+                                             unsigned char* scratch, int lane)
+{
+    const float2* st = P.stats_t + (long long)row_t * P.nblk;
+    const unsigned char* trow = P.target + (long long)row_t * P.tstride_bytes;
+    auto mass = [&](int i) {
+        const float2 e = __ldcg(&st[i]);
+        return e.x > kNegInf ? e.y * ex2_approx(e.x - Cp) : 0.f;
+    };
+    const double Z = warp_total(P.nblk, lane, mass);
+    double before;
+    int lastp;
+    int b = chunked_search(P.nblk, lane, mass, u * Z, before, lastp);
+    if (b < 0) { b = lastp >= 0 ? lastp : 0; before = u * Z; }
+    const float2 sb = __ldcg(&st[b]);
+    // inside the block work in the block's own reference: divide the remaining mass by 2^(c_b - C)
+    double thr_local = (u * Z - before) / (double)ex2_approx(sb.x - Cp);
+    const float nc = -sb.x, scale = P.scale;
+    auto ev = [&](float xt, float) { return ex2_approx(__fmaf_rn(xt, scale, nc)); };
+    int token = -1, fallback = b * P.epb;
+    for (int h = 0; h < kStatBlockBytes / kResidBlockBytes; ++h) {
+        const int e0 = b * P.epb + h * P.epb_r;
+        const int cnt = (P.V - e0) < P.epb_r ? (P.V - e0) : P.epb_r;
+        if (cnt <= 0) break;
+        __syncwarp();
+        stage_raw<kElem>(trow, e0, cnt, scratch, lane);
+        __syncwarp();
+        double tot;
+        int lp;
+        const int e = raw_unit_search<kElem>(scratch, nullptr, cnt, lane, thr_local, ev, tot, lp);
+        if (lp >= 0) fallback = e0 + lp;
+        if (e >= 0) { token = e0 + e; break; }
+        thr_local -= tot;
+    }
+    return token >= 0 ? token : fallback;
+}
+
+// Draws the corrected token of a rejected position from norm(max(0, p - q)) given the per-block
+// sums of the residual pass.  One warp; scratch = 2 KB + 2 KB of shared memory.
+template <int kElem>
+__device__ __forceinline__ int sample_from_residual(const VerifyParams& P, const ResidTask& t, const float* wb,
+                                                    unsigned char* scr_t, unsigned char* scr_d, int lane)
+{
+    const double u = (double)t.u;
+    auto wv = [&](int i) { return __ldcg(&wb[i]); };
+    const double W = warp_total(P.nblk_r, lane, wv);
+    if (!(W > 0.0) || !(W < INFINITY))                       // empty residual: draw from p with the same u
+        return sample_from_p<kElem>(P, t.row_t, t.cp, u, scr_t, lane);
+    double before;
+    int lastp;
+    int b = chunked_search(P.nblk_r, lane, wv, u * W, before, lastp);
+    if (b < 0) { b = lastp >= 0 ? lastp : 0; before = u * W; }
+    const int e0 = b * P.epb_r;
+    const int cnt = (P.V - e0) < P.epb_r ? (P.V - e0) : P.epb_r;
+    __syncwarp();
+    stage_raw<kElem>(P.target + (long long)t.row_t * P.tstride_bytes, e0, cnt, scr_t, lane);
+    stage_raw<kElem>(P.draft + t.row_d * P.dstride_bytes, e0, cnt, scr_d, lane);
+    __syncwarp();
+    ResidConst K;
+    K.set(P.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
+    double tot;
+    int lp;
+    int e = raw_unit_search<kElem>(scr_t, scr_d, cnt, lane, u * W - before,
+                                   [&](float xt, float xd) { return resid_elem(xt, xd, K); }, tot, lp);
+    if (e < 0) e = lp >= 0 ? lp : 0;
+    return e0 + e;
+}
+
+// ---------------------------------------------------------------------------------------
+// decide: one CTA per request, one warp per position (eight per round): row statistics from
+// block statistics, p(x), q(x), accept test, first rejection n_r; the accepted prefix is written.
+// Position j = len is the bonus row (statistics only).  A fully accepted request draws its bonus
+// token here; a rejected one is queued for the residual pass.
+// ---------------------------------------------------------------------------------------
+template <int kElem>
 __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
 {
     constexpr int kWarps = kDecideThreads / 32;
-    __shared__ int s_first, s_bad;
+    __shared__ int s_first, s_bad, s_have_fin, s_kind;
     __shared__ float s_Ct[kWarps], s_Cd[kWarps];
     __shared__ double s_St[kWarps], s_Sd[kWarps];
     __shared__ float s_fin_C[2];     // [0] target, [1] draft statistics of the row that emits the token
     __shared__ double s_fin_S[2];
-    __shared__ int s_have_fin;
+    __shared__ float s_u;
+    __shared__ __align__(16) unsigned char s_scratch[kResidBlockBytes];
+
+    pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -574,16 +794,12 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     const int lo = P.row_offsets[r], hi = P.row_offsets[r + 1];
     // the request's rows must lie inside the batch, and so must its draft rows (compact index lo - r)
     if (lo < 0 || hi - lo < 1 || hi > n_rows || lo - r < 0 || (hi - 1 - r) > n_rows - P.R) {
-        if (tid == 0) {
-            atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS);
-            P.accepted_len[r] = 0;
-            P.req[r].kind = kTaskNone;
-        }
+        if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS); P.accepted_len[r] = 0; }
         return;
     }
     const int len = hi - lo - 1;
     const long long drow0 = P.draft_row_start ? P.draft_row_start[r] : (long long)(lo - r);
-    if (tid == 0) { s_first = len; s_bad = 0; s_have_fin = 0; }
+    if (tid == 0) { s_first = len; s_bad = 0; s_have_fin = 0; s_kind = kTaskNone; }
     __syncthreads();
     for (int i = tid; i <= len; i += kDecideThreads) {
         P.out_tokens[lo + i] = -1;
@@ -594,7 +810,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     }
     __syncthreads();
     if (s_bad) {
-        if (tid == 0) { atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
+        if (tid == 0) { atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; }
         return;
     }
     const bool want_all = (P.out_p != nullptr) || (P.out_q != nullptr);
@@ -643,234 +859,58 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
         __syncthreads();                         // everyone has read the flags before the next round updates them
         if (stop) break;
     }
-    if (tid != 0) return;
 
-    if (s_bad) {
-        atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone;
-        return;
-    }
     const int n = s_first;
-    const float Cp = s_fin_C[0];
-    const double Sp = s_fin_S[0];
-    if (!s_have_fin || !row_usable(Cp, Sp)) {
-        atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone;
-        return;
+    if (tid == 0) {
+        if (s_bad || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
+            (n < len && !row_usable(s_fin_C[1], s_fin_S[1]))) {
+            atomicOr(P.dev_status, s_bad ? s_bad : DSPARK_DEV_BAD_ROW);
+            P.accepted_len[r] = 0;
+        } else {
+            for (int i = 0; i < n; ++i) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
+            float ua, ur;
+            philox_uniforms(P.seed, (uint32_t)r, (uint32_t)n, ua, ur);
+            s_u = ur;
+            P.accepted_len[r] = n;
+            if (n < len) {
+                const int slot = atomicAdd(&P.counters[0], 1);
+                ResidTask q;
+                q.request = r; q.row_t = lo + n; q.row_d = drow0 + n;
+                q.cp = s_fin_C[0]; q.inv_zp = (float)(1.0 / s_fin_S[0]);
+                q.cq = s_fin_C[1]; q.inv_zq = (float)(1.0 / s_fin_S[1]);
+                q.u = ur; q.pad[0] = q.pad[1] = q.pad[2] = 0;
+                P.resid[slot] = q;
+                s_kind = kTaskResid;
+            } else {
+                s_kind = kTaskBonus;
+            }
+        }
     }
-    for (int i = 0; i < n; ++i) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
-    float ua, ur;
-    philox_uniforms(P.seed, (uint32_t)r, (uint32_t)n, ua, ur);
-    RequestTask t;
-    t.n = n; t.u = ur; t.slot = -1;
-    t.cp = Cp; t.inv_zp = (float)(1.0 / Sp);
-    t.cq = 0.f; t.inv_zq = 1.f;
-    t.row_d = drow0 + n;
-    if (n < len) {
-        t.cq = s_fin_C[1]; t.inv_zq = (float)(1.0 / s_fin_S[1]);
-        const int slot = atomicAdd(&P.counters[0], 1);
-        ResidTask q;
-        q.request = r; q.row_t = lo + n; q.row_d = t.row_d;
-        q.cp = t.cp; q.inv_zp = t.inv_zp; q.cq = t.cq; q.inv_zq = t.inv_zq;
-        P.resid[slot] = q;
-        t.kind = kTaskResid; t.slot = slot;
-    } else {
-        t.kind = kTaskBonus;
-    }
-    P.req[r] = t;
-    P.accepted_len[r] = n;
+    __syncthreads();
+    if (s_kind != kTaskBonus || warp != 0) return;
+    const int token = sample_from_p<kElem>(P, lo + n, s_fin_C[0], (double)s_u, s_scratch, lane);
+    if (lane == 0) P.out_tokens[lo + n] = token;
 }
 
 // ---------------------------------------------------------------------------------------
-// finalize: one warp per request.  Inverse CDF in vocabulary order: first over per-block
-// sums (fp64 running sum), then over the elements of the one block that holds the crossing.
-// Each lane owns a contiguous run; values are held in registers.
+// finalize: one warp per queued (rejected) request draws the corrected token from the residual.
 // ---------------------------------------------------------------------------------------
-
-// Over values x[0..cnt) of each lane (lane-major order = index order), finds the first index whose
-// inclusive running sum exceeds thr(total).  kMax values per lane.  Returns the global index
-// lane*per + k (or -1), the exclusive sum before it, the total and the last positive index.
-template <int kMax, typename Thr>
-__device__ __forceinline__ int warp_crossing(const float (&x)[kMax], int per, int cnt, int lane, Thr thr_of,
-                                             double& before, double& total, int& last_positive)
-{
-    double mine = 0.0;
-    int lastp = -1;
-#pragma unroll
-    for (int k = 0; k < kMax; ++k)
-        if (k < cnt) { mine += (double)x[k]; if (x[k] > 0.f) lastp = lane * per + k; }
-    double incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    total = __shfl_sync(0xffffffffu, incl, 31);
-    const double thr = thr_of(total);
-    const unsigned hit = __ballot_sync(0xffffffffu, incl > thr && cnt > 0);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) lastp = max(lastp, __shfl_xor_sync(0xffffffffu, lastp, o));
-    last_positive = lastp;
-    if (!hit) { before = total; return -1; }
-    const int src = __ffs(hit) - 1;
-    int found = -1;
-    double bef = 0.0;
-    if (lane == src) {
-        double run = incl - mine;
-#pragma unroll
-        for (int k = 0; k < kMax; ++k) {
-            if (k < cnt && found < 0) {
-                if (run + (double)x[k] > thr) { found = lane * per + k; bef = run; }
-                else run += (double)x[k];
-            }
-        }
-        if (found < 0) { found = lane * per + cnt - 1; bef = run; }   // only by rounding between the two sums
-    }
-    found = __shfl_sync(0xffffffffu, found, src);
-    before = __shfl_sync(0xffffffffu, bef, src);
-    return found;
-}
-
-// Loads this lane's contiguous run of a block: `per` elements starting at element e_begin of the
-// row, as fp32 values; elements at or beyond V read -inf.  16-byte loads when the address allows.
-template <int kElem, int kPer>
-__device__ __forceinline__ void load_run(const unsigned char* row, int e_begin, int V, float (&x)[kPer])
-{
-    const unsigned char* p = row + (long long)e_begin * kElem;
-    constexpr int kBytes = kPer * kElem;
-    if (e_begin + kPer <= V && ((uintptr_t)p & 15u) == 0) {
-#pragma unroll
-        for (int k = 0; k < kBytes / 16; ++k) {
-            const uint4 q = __ldg((const uint4*)(p + 16 * k));
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t w = word_of(q, i);
-                if (kElem == 2) { x[k * 8 + 2 * i] = bf16lo(w); x[k * 8 + 2 * i + 1] = bf16hi(w); }
-                else x[k * 4 + i] = __uint_as_float(w);
-            }
-        }
-    } else {
-#pragma unroll
-        for (int k = 0; k < kPer; ++k) {
-            float val = kNegInf;
-            if (e_begin + k < V) {
-                if (kElem == 2) val = __uint_as_float((uint32_t)__ldg((const unsigned short*)(p + 2 * k)) << 16);
-                else val = __ldg((const float*)(p + 4 * k));
-            }
-            x[k] = val;
-        }
-    }
-}
-
-// Level 1 of the inverse CDF: over n block values val(i) in index order, the first block whose
-// inclusive running sum exceeds u * total.  Up to 256 blocks are held in registers (8 per lane);
-// longer rows take the total first and then walk chunks of 256 blocks in order.
-template <typename F>
-__device__ __forceinline__ int block_crossing(int n, int lane, double u, F val, double& before, double& total,
-                                              int& last_positive)
-{
-    int b = -1;
-    last_positive = -1;
-    before = 0.0;
-    if (n <= 256) {
-        const int per = (n + 31) / 32;
-        float x[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { const int i = lane * per + k; x[k] = (k < per && i < n) ? val(i) : 0.f; }
-        int cnt = n - lane * per; cnt = cnt < 0 ? 0 : (cnt > per ? per : cnt);
-        b = warp_crossing<8>(x, per, cnt, lane, [&](double tot) { return u * tot; }, before, total, last_positive);
-    } else {
-        double tot = 0.0;
-        for (int i = lane; i < n; i += 32) tot += (double)val(i);
-        total = warp_sum_f64(tot);
-        const double thr = u * total;
-        double run = 0.0;
-        for (int base = 0; base < n && b < 0; base += 256) {
-            float x[8];
-            int cnt = n - base - lane * 8; cnt = cnt < 0 ? 0 : (cnt > 8 ? 8 : cnt);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) x[k] = (k < cnt) ? val(base + lane * 8 + k) : 0.f;
-            double bef, tot_c;
-            int lp;
-            const int f = warp_crossing<8>(x, 8, cnt, lane, [&](double) { return thr - run; }, bef, tot_c, lp);
-            if (lp >= 0) last_positive = base + lp;
-            if (f >= 0) { b = base + f; before = run + bef; }
-            run += tot_c;
-        }
-    }
-    return b;
-}
-
+constexpr int kFinalizeThreads = 128;
 template <int kElem>
 __global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(VerifyParams P)
 {
-    constexpr int kPerStat = kStatBlockBytes / kElem / 32;     // elements per lane in a statistics block
-    constexpr int kPerResid = kResidBlockBytes / kElem / 32;   // elements per lane in a residual block
-    const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * (kFinalizeThreads / 32) + (threadIdx.x >> 5);
-    if (r >= P.R) return;
-    const RequestTask t = P.req[r];
-    if (t.kind == kTaskNone) return;
-    const int lo = P.row_offsets[r];
-    const int row_t = lo + t.n;
-    const unsigned char* trow = P.target + (long long)row_t * P.tstride_bytes;
-    int token = -1;
-    bool from_p = (t.kind == kTaskBonus);
-    const double u = (double)t.u;
-
-    if (t.kind == kTaskResid) {
-        const float* wb = P.wblk + (long long)t.slot * P.nblk_r;
-        const unsigned char* drow = P.draft + t.row_d * P.dstride_bytes;
-        ResidConst K;
-        K.set(P.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
-        double before, W;
-        int lastp;
-        int b = block_crossing(P.nblk_r, lane, u, [&](int i) { return __ldcg(&wb[i]); }, before, W, lastp);
-        if (!(W > 0.0) || !(W < INFINITY)) {
-            from_p = true;                                   // empty residual: draw from p with the same u
-        } else {
-            if (b < 0) b = lastp;
-            const int e0 = b * P.epb_r + lane * kPerResid;
-            float xt[kPerResid], xd[kPerResid], w[kPerResid];
-            load_run<kElem, kPerResid>(trow, e0, P.V, xt);
-            load_run<kElem, kPerResid>(drow, e0, P.V, xd);
-#pragma unroll
-            for (int k = 0; k < kPerResid; ++k) w[k] = resid_elem(xt[k], xd[k], K);
-            int cnt = P.V - e0; cnt = cnt < 0 ? 0 : (cnt > kPerResid ? kPerResid : cnt);
-            const double thr_local = u * W - before;
-            double bef2, tot2;
-            int lp2;
-            int e = warp_crossing<kPerResid>(w, kPerResid, cnt, lane, [&](double) { return thr_local; }, bef2, tot2, lp2);
-            if (e < 0) e = lp2 >= 0 ? lp2 : 0;
-            token = b * P.epb_r + e;
-        }
-    }
-    if (from_p) {
-        const float2* st = P.stats_t + (long long)row_t * P.nblk;
-        const float C = t.cp;
-        auto mass = [&](int i) {
-            const float2 e = __ldcg(&st[i]);
-            return e.x > kNegInf ? e.y * ex2_approx(e.x - C) : 0.f;
-        };
-        double before, Z;
-        int lastp;
-        int b = block_crossing(P.nblk, lane, u, mass, before, Z, lastp);
-        if (b < 0) b = lastp >= 0 ? lastp : 0;
-        const float2 sb = __ldcg(&st[b]);
-        const int e0 = b * P.epb + lane * kPerStat;
-        float x[kPerStat];
-        load_run<kElem, kPerStat>(trow, e0, P.V, x);
-        // inside the block work in the block's own reference: divide the remaining mass by 2^(c_b - C)
-        const double thr_local = (u * Z - before) / (double)ex2_approx(sb.x - C);
-        const float nc = -sb.x;
-#pragma unroll
-        for (int k = 0; k < kPerStat; ++k) x[k] = ex2_approx(__fmaf_rn(x[k], P.scale, nc));
-        int cnt = P.V - e0; cnt = cnt < 0 ? 0 : (cnt > kPerStat ? kPerStat : cnt);
-        double bef2, tot2;
-        int lp2;
-        int e = warp_crossing<kPerStat>(x, kPerStat, cnt, lane, [&](double) { return thr_local; }, bef2, tot2, lp2);
-        if (e < 0) e = lp2 >= 0 ? lp2 : 0;
-        token = b * P.epb + e;
-    }
-    if (lane == 0) P.out_tokens[row_t] = token;
+    __shared__ __align__(16) unsigned char s_scratch[kFinalizeThreads / 32][2 * kResidBlockBytes];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int slot = blockIdx.x * (kFinalizeThreads / 32) + warp;
+    int nq = __ldcg(&P.counters[0]);
+    nq = nq > P.R ? P.R : nq;
+    if (slot >= nq) return;
+    const ResidTask t = P.resid[slot];
+    const int token = sample_from_residual<kElem>(P, t, P.wblk + (long long)slot * P.nblk_r, s_scratch[warp],
+                                                  s_scratch[warp] + kResidBlockBytes, lane);
+    if (lane == 0) P.out_tokens[t.row_t] = token;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -878,6 +918,8 @@ __global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(VerifyParams
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kDecideThreads) greedy_decide_kernel(VerifyParams P)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * (kDecideThreads / 32) + (threadIdx.x >> 5);
     if (r >= P.R) return;
@@ -979,12 +1021,12 @@ static void launch_stream(const VerifyParams& P, bool bulk, long long max_units,
         long long g = (long long)sms * 2;
         if (g > max_units) g = max_units;
         if (g < 1) g = 1;
-        stream_bulk_kernel<kElem, kMode><<<(int)g, kStreamThreads, kStages * kStageBytes, s>>>(P);
+        launch_pdl(stream_bulk_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kStreamThreads), kStages * kStageBytes, s, P);
     } else {
         long long g = (long long)sms * 8;
         if (g > max_units) g = max_units;
         if (g < 1) g = 1;
-        stream_direct_kernel<kElem, kMode><<<(int)g, kConsumerWarps * 32, 0, s>>>(P);
+        launch_pdl(stream_direct_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kConsumerWarps * 32), 0, s, P);
     }
 }
 
@@ -996,7 +1038,7 @@ static void launch_stream_dtype(const VerifyParams& P, bool bulk, long long max_
 }
 
 struct Workspace {
-    size_t counters, stats_t, stats_d, resid, req, wblk, total;
+    size_t counters, stats_t, stats_d, resid, wblk, total;
 };
 static Workspace workspace_layout(int R, int n_rows, int V)
 {
@@ -1009,7 +1051,6 @@ static Workspace workspace_layout(int R, int n_rows, int V)
     w.stats_t = o;  o += up((size_t)n_rows * nblk * sizeof(float2));
     w.stats_d = o;  o += up((size_t)n_rows * nblk * sizeof(float2));
     w.resid = o;    o += up((size_t)R * sizeof(ResidTask));
-    w.req = o;      o += up((size_t)R * sizeof(RequestTask));
     w.wblk = o;     o += up((size_t)R * nblk_r * sizeof(float));
     w.total = o;
     return w;
@@ -1053,7 +1094,6 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.stats_t = (float2*)(ws + w.stats_t);
     P.stats_d = (float2*)(ws + w.stats_d);
     P.resid = (ResidTask*)(ws + w.resid);
-    P.req = (RequestTask*)(ws + w.req);
     P.wblk = (float*)(ws + w.wblk);
     return DSPARK_OK;
 }
@@ -1099,7 +1139,7 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
     {
         KernelTimerScope timer(DSPARK_K_GREEDY_DECIDE, s);
         const int warps_per_cta = kDecideThreads / 32;
-        greedy_decide_kernel<<<(R + warps_per_cta - 1) / warps_per_cta, kDecideThreads, 0, s>>>(P);
+        launch_pdl(greedy_decide_kernel, dim3((R + warps_per_cta - 1) / warps_per_cta), dim3(kDecideThreads), 0, s, P);
     }
     return launch_status();
 }
@@ -1136,7 +1176,8 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_DECIDE, s);
-        decide_kernel<<<R, kDecideThreads, 0, s>>>(P);
+        if (P.elem == 2) launch_pdl(decide_kernel<2>, dim3(R), dim3(kDecideThreads), 0, s, P);
+        else launch_pdl(decide_kernel<4>, dim3(R), dim3(kDecideThreads), 0, s, P);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
@@ -1146,10 +1187,9 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_FINALIZE, s);
-        const int warps_per_cta = kFinalizeThreads / 32;
-        const int grid = (R + warps_per_cta - 1) / warps_per_cta;
-        if (P.elem == 2) finalize_kernel<2><<<grid, kFinalizeThreads, 0, s>>>(P);
-        else finalize_kernel<4><<<grid, kFinalizeThreads, 0, s>>>(P);
+        const int grid = (R + kFinalizeThreads / 32 - 1) / (kFinalizeThreads / 32);
+        if (P.elem == 2) launch_pdl(finalize_kernel<2>, dim3(grid), dim3(kFinalizeThreads), 0, s, P);
+        else launch_pdl(finalize_kernel<4>, dim3(grid), dim3(kFinalizeThreads), 0, s, P);
     }
     return launch_status();
 }

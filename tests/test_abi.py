@@ -34,7 +34,7 @@ def test_host_only_entry_points():
     # workspace queries are pure host arithmetic
     assert B.dspark_verify_workspace_bytes(64, 352, 129280) > 2 * 352 * 127 * 8
     assert B.dspark_verify_workspace_bytes(0, 1, 10) == 0
-    assert B.dspark_schedule_workspace_bytes(512, 32) == 16384 * 8
+    assert B.dspark_schedule_workspace_bytes(512, 32) >= 16384 * (4 + 8 + 8 + 4)
     assert B.dspark_schedule_workspace_bytes(1 << 20, 2) == 0          # beyond the supported size
 
 
