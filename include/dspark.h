@@ -39,7 +39,8 @@ typedef enum {
     DSPARK_ERR_ALIGNMENT = 3,
     DSPARK_ERR_WORKSPACE = 4,
     DSPARK_ERR_CUDA = 5,
-    DSPARK_ERR_TIMEOUT = 6
+    DSPARK_ERR_TIMEOUT = 6,
+    DSPARK_ERR_STATIC_LIMIT = 7
 } dspark_status_t;
 
 typedef enum { DSPARK_F32 = 0, DSPARK_BF16 = 1 } dspark_dtype_t;
@@ -148,6 +149,42 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
                          const int32_t* row_offsets, const int32_t* draft_tokens, int R, int n_rows,
                          int32_t* accepted_len, int32_t* out_tokens, int32_t* dev_status,
                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* dspark_verify_greedy_static -- the same greedy verification for callers that are not
+ * allowed to allocate device memory.  (The paper has no counterpart; this is a packaging
+ * variant of dspark_verify_greedy.)
+ *
+ * Who needs it: a serving engine once it has entered its steady-state loop usually cannot call
+ * cudaMalloc any more -- every byte of HBM is already promised to weights and KV cache, an
+ * allocation would synchronise the whole device in the middle of a step, and code that runs as
+ * a plug-in of another runtime may simply be forbidden to allocate after start-up.  Such a
+ * caller has nowhere to get a workspace from, so this entry point takes none: the per-block
+ * (max, argmax) statistics go into a fixed array of DSPARK_STATIC_SCRATCH_BYTES that is part
+ * of the library image.  Every GPU that loads the library carries that array until the
+ * process exits, whether or not this function is ever called.
+ *
+ * Arguments, outputs and device-side error reporting are those of dspark_verify_greedy, minus
+ * the workspace.  Differences a caller has to know:
+ *  - Size limit.  A batch whose scratch need (dspark_verify_workspace_bytes(R, n_rows, V))
+ *    exceeds dspark_verify_greedy_static_capacity() is refused with DSPARK_ERR_STATIC_LIMIT and a
+ *    message on stderr; nothing is launched.  8 MiB covers about 8 000 fp32 rows or 16 000
+ *    bf16 rows at V = 129 280.
+ *  - First call on a device.  It looks up the device address of the array
+ *    (cudaGetSymbolAddress) with that device current and caches it; later calls on that
+ *    device do no set-up.  Make that first call during initialisation, before any stream
+ *    capture begins.
+ *  - One array for everybody.  All calls in the process, on every stream, share it, and it keeps
+ *    whatever the previous call left.  That is harmless for results (each call rewrites every
+ *    entry it later reads), but two calls that overlap in time on the GPU race on it: run them
+ *    on one stream, or order them yourself.
+ *  - It calls no cudaMalloc, cudaFree or other allocating routine.
+ */
+#define DSPARK_STATIC_SCRATCH_BYTES (8u << 20)
+size_t dspark_verify_greedy_static_capacity(void);
+int dspark_verify_greedy_static(const void* target_logits, int dtype, int64_t target_row_stride, int V,
+                                const int32_t* row_offsets, const int32_t* draft_tokens, int R, int n_rows,
+                                int32_t* accepted_len, int32_t* out_tokens, int32_t* dev_status,
+                                void* stream);
 
 /* dspark_verify -- lossless sampling verification (Section 2.1): with p = softmax(target/T)
  * and q = softmax(draft/T) at each position, token x is accepted with probability

@@ -28,6 +28,7 @@ EXPORTS = [
     "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",
     "dspark_schedule_workspace_bytes", "dspark_schedule", "dspark_build_offsets",
     "dspark_verify_workspace_bytes", "dspark_verify_greedy", "dspark_verify", "dspark_uniforms",
+    "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
     "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
     "dspark_version",
@@ -63,6 +64,9 @@ def lib() -> C.CDLL:
         L.dspark_verify_workspace_bytes.argtypes = [i32, i32, i32]
         L.dspark_verify_workspace_bytes.restype = sz
         L.dspark_verify_greedy.argtypes = [vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.dspark_verify_greedy_static.argtypes = [vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp]
+        L.dspark_verify_greedy_static_capacity.argtypes = []
+        L.dspark_verify_greedy_static_capacity.restype = sz
         L.dspark_verify.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, C.c_float, u64,
                                     vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_uniforms.argtypes = [u64, C.c_uint32, C.c_uint32, C.POINTER(C.c_float), C.POINTER(C.c_float)]
@@ -199,6 +203,27 @@ def dspark_verify_greedy(target: torch.Tensor, row_offsets: torch.Tensor, draft_
                                     _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
                                     workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_verify_greedy")
+
+
+def dspark_verify_greedy_static_capacity() -> int:
+    return int(lib().dspark_verify_greedy_static_capacity())
+
+
+def dspark_verify_greedy_static(target: torch.Tensor, row_offsets: torch.Tensor, draft_tokens: torch.Tensor, *,
+                                accepted_len: torch.Tensor, out_tokens: torch.Tensor,
+                                dev_status: Optional[torch.Tensor], n_rows: Optional[int] = None) -> None:
+    """Greedy verification without a caller workspace, for callers that may not allocate device
+    memory: the scratch is a fixed array inside the library.  Raises when the batch is larger than
+    that array (see dspark_verify_greedy_static_capacity)."""
+    tp, code, ts = _logits(target, "target")
+    R = row_offsets.numel() - 1
+    n_rows = target.shape[0] if n_rows is None else n_rows
+    rc = lib().dspark_verify_greedy_static(tp, code, ts, target.shape[1], _dev(row_offsets, "row_offsets", torch.int32),
+                                           _dev(draft_tokens, "draft_tokens", torch.int32), R, n_rows,
+                                           _dev(accepted_len, "accepted_len", torch.int32),
+                                           _dev(out_tokens, "out_tokens", torch.int32),
+                                           _dev(dev_status, "dev_status", torch.int32), _stream())
+    _check(rc, "dspark_verify_greedy_static")
 
 
 def dspark_verify(target: torch.Tensor, draft: torch.Tensor, row_offsets: torch.Tensor,

@@ -15,6 +15,7 @@
 //            max(0, p - q), same bulk-copy pipeline with two sources per stage.
 //   finalize one warp per rejected request: inverse CDF over block sums, then inside one block.
 #include <cuda_bf16.h>
+#include <cstdio>
 #include <math.h>
 
 #include "common.cuh"
@@ -1192,6 +1193,66 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
         else launch_pdl(finalize_kernel<4>, dim3(grid), dim3(kFinalizeThreads), 0, s, P);
     }
     return launch_status();
+}
+
+
+// ---------------------------------------------------------------------------------------
+// dspark_verify_greedy_static: greedy verification for callers that must not allocate.
+// Its scratch is this fixed array inside the library image instead of a caller workspace.
+// ---------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace dspark {
+
+constexpr size_t kStaticScratchBytes = DSPARK_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// The array's name is only a host-side handle; kernels need its device address, which is looked
+// up once per device (with that device current) and cached.
+static void* g_static_scratch_ptr[64] = {};
+
+static int static_scratch_address(void** out)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return DSPARK_ERR_CUDA; }
+    if (!g_static_scratch_ptr[dev]) {
+        void* ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr) {
+            fprintf(stderr, "dspark: cudaGetSymbolAddress(static scratch) failed: %s\n", cudaGetErrorString(e));
+            cudaGetLastError();
+            return DSPARK_ERR_CUDA;
+        }
+        g_static_scratch_ptr[dev] = ptr;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return DSPARK_OK;
+}
+
+}  // namespace dspark
+
+extern "C" {
+
+size_t dspark_verify_greedy_static_capacity(void) { return kStaticScratchBytes; }
+
+int dspark_verify_greedy_static(const void* target_logits, int dtype, int64_t target_row_stride, int V,
+                                const int32_t* row_offsets, const int32_t* draft_tokens, int R, int n_rows,
+                                int32_t* accepted_len, int32_t* out_tokens, int32_t* dev_status, void* stream)
+{
+    if (R < 1 || n_rows < R || V < 1) return DSPARK_ERR_INVALID_ARG;
+    const size_t need = workspace_layout(R, n_rows, V).total;
+    if (need > kStaticScratchBytes) {
+        fprintf(stderr, "dspark_verify_greedy_static: this batch needs %zu bytes of scratch, the built-in array "
+                        "holds %zu; use dspark_verify_greedy with a caller workspace\n", need, kStaticScratchBytes);
+        return DSPARK_ERR_STATIC_LIMIT;
+    }
+    void* scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc != DSPARK_OK) return rc;
+    // every statistic the decide kernel reads is rewritten by the stream kernel of this same call,
+    // so nothing left by an earlier call needs clearing
+    return dspark_verify_greedy(target_logits, dtype, target_row_stride, V, row_offsets, draft_tokens, R, n_rows,
+                                accepted_len, out_tokens, dev_status, scratch, kStaticScratchBytes, stream);
 }
 
 }  // extern "C"
