@@ -22,7 +22,7 @@ constexpr int kResidVec = 4;                                // vectors per lane 
 constexpr int kStatBlockBytes = kStatVec * 512;             // 4 KB
 constexpr int kResidBlockBytes = kResidVec * 512;           // 2 KB
 constexpr int kStageBytes = 32768;                          // one pipeline stage in every mode
-constexpr int kStages = 3;
+constexpr int kStages = 2;
 
 // Upper bound on polls of one mbarrier phase before a kernel gives up (each poll may
 // itself block for a short hardware-defined time, so this is on the order of a second).

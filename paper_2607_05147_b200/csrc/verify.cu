@@ -9,11 +9,11 @@
 //            (cp.async.bulk + mbarrier), eight consumer warps drain it.
 //   decide   one CTA per request: combines block statistics into row statistics, gathers
 //            p(x), q(x), runs the accept tests (Philox), finds the first rejection, writes the
-//            accepted prefix; a fully accepted request draws its bonus token here (inverse CDF
-//            over the saved block statistics, one block re-read); a rejected one is queued.
+//            accepted prefix, and queues a rejected position for the residual pass.
 //   residual second read of the rejected position's row pair only: per-2KB-block sums of
 //            max(0, p - q), same bulk-copy pipeline with two sources per stage.
-//   finalize one warp per rejected request: inverse CDF over block sums, then inside one block.
+//   finalize one warp per request: inverse CDF over block values (residual sums, or the saved
+//            statistics of the bonus row), then inside the one block that holds the crossing.
 #include <cuda_bf16.h>
 #include <cstdio>
 #include <math.h>
@@ -33,6 +33,15 @@ struct __align__(16) ResidTask {     // one rejected request queued for the resi
     int64_t row_d;                   // physical draft row
     float cp, inv_zp, cq, inv_zq;    // row references (log2 domain) and 1 / row sums
     float u;                         // resample uniform of the rejected position
+    int32_t pad[3];
+};
+
+struct __align__(16) RequestRec {    // what the finalize kernel needs per request (written by decide)
+    int32_t kind;                    // kTaskNone / kTaskResid / kTaskBonus
+    int32_t row_t;                   // target row that emits the token
+    int64_t row_d;                   // physical draft row of the rejected position
+    float cp, inv_zp, cq, inv_zq;    // row references (log2 domain) and 1 / row sums
+    float u;                         // resample uniform
     int32_t pad[3];
 };
 
@@ -59,7 +68,8 @@ struct VerifyParams {
     float2* stats_t;
     float2* stats_d;
     ResidTask* resid;                         // queue of rejected requests (decide -> residual pass)
-    float* wblk;                              // per queue slot: residual block sums
+    RequestRec* req;                          // per request: outcome of decide for the finalize kernel
+    float* wblk;                              // per request: residual block sums
 };
 
 template <int kMode> struct ModeCfg {
@@ -354,7 +364,7 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
         ResidConst K;
         K.set(P.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
         const float w = block_resid<kElem, M::kVec>(v, vd, K);
-        if (lane == 0) P.wblk[(long long)s * nblk + b] = w;
+        if (lane == 0) P.wblk[(long long)t.request * nblk + b] = w;
     }
 }
 
@@ -384,7 +394,7 @@ __device__ __forceinline__ void unit_sources(const VerifyParams& P, int s, int p
 // Streamed pass, bulk-copy pipeline: kStages x 32 KB of shared memory per CTA.
 // ---------------------------------------------------------------------------------------
 template <int kElem, int kMode>
-__global__ void __launch_bounds__(kStreamThreads, 2) stream_bulk_kernel(VerifyParams P)
+__global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyParams P)
 {
     using M = ModeCfg<kMode>;
     extern __shared__ __align__(128) unsigned char stage_mem[];
@@ -551,11 +561,14 @@ __device__ __forceinline__ bool row_usable(float C, double S)
 }
 
 // ---------------------------------------------------------------------------------------
-// Inverse CDF in vocabulary order, two levels, one warp, registers and a 2 KB scratch only:
-//   level 1  over per-block values (residual block sums, or block masses of p): chunks of 32
-//            consecutive blocks are read coalesced, chunk totals reduced with shuffles;
-//   level 2  inside the one block that holds the crossing: its raw logits are staged into
-//            shared memory and every lane walks a contiguous run (rolled loops, small code).
+// Inverse CDF in vocabulary order, two levels, one warp:
+//   level 1  over per-block values (residual block sums, or block masses of p).  Up to 256 blocks
+//            are held in registers, lane-strided (value k of lane l is block k*32+l): chunk totals
+//            by warp reduction, then one warp scan inside the chunk that holds the crossing.
+//            Longer rows walk memory in chunks of 32 blocks.
+//   level 2  inside that one block: every lane copies its own contiguous run of raw logits into a
+//            padded (bank-conflict-free) strip of shared memory, sums its values, the warp scans
+//            the lane sums, and the lane that holds the crossing walks its cached values.
 // All running sums are fp64 sums of the fp32 values in index order.
 // ---------------------------------------------------------------------------------------
 template <typename F>
@@ -567,223 +580,184 @@ __device__ __forceinline__ double warp_total(int n, int lane, F val)
     return warp_sum_f64(t);
 }
 
-// First index i in [0, n) whose inclusive running sum exceeds thr; -1 if none (then `before` is the
-// total).  `last_positive` = last index with a positive value.
+__device__ __forceinline__ double warp_incl_scan_f64(double x, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += t;
+    }
+    return x;
+}
+
+// Level 1 from registers: x[k] = value of block k*32+lane (0 beyond n), n <= 256.  thr = u * total.
+// Returns the block index (never -1 when total > 0: falls back to the last positive block), and the
+// exclusive sum before it.
+__device__ __forceinline__ int level1_registers(const float (&x)[8], int n, int lane, double u, double& before,
+                                                double& total)
+{
+    double ct[8];
+    total = 0.0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { ct[k] = (k * 32 < n) ? warp_sum_f64((double)x[k]) : 0.0; total += ct[k]; }
+    const double thr = u * total;
+    double run = 0.0;
+    int kc = -1;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        if (kc < 0 && k * 32 < n) {
+            if (run + ct[k] > thr) kc = k; else run += ct[k];
+        }
+    }
+    int lastp = -1;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const unsigned pos = __ballot_sync(0xffffffffu, x[k] > 0.f);
+        if (pos) lastp = k * 32 + (31 - __clz(pos));
+    }
+    if (kc < 0) { before = total; return lastp >= 0 ? lastp : 0; }      // only by rounding
+    float xc = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) if (k == kc) xc = x[k];
+    const double incl = warp_incl_scan_f64((double)xc, lane);
+    const unsigned hit = __ballot_sync(0xffffffffu, run + incl > thr && kc * 32 + lane < n);
+    int l;
+    if (hit) l = __ffs(hit) - 1;
+    else { const unsigned pos = __ballot_sync(0xffffffffu, xc > 0.f); l = pos ? 31 - __clz(pos) : 0; }
+    before = run + __shfl_sync(0xffffffffu, incl - (double)xc, l);
+    return kc * 32 + l;
+}
+
+// Level 1 from memory for rows with more than 256 blocks: first index i in [0, n) whose inclusive
+// running sum exceeds thr, else the last positive index.
 template <typename F>
-__device__ __forceinline__ int chunked_search(int n, int lane, F val, double thr, double& before, int& last_positive)
+__device__ __forceinline__ int level1_memory(int n, int lane, F val, double thr, double& before)
 {
     double run = 0.0;
     int lastp = -1;
-    for (int g0 = 0; g0 < n; g0 += 1024) {
-        // totals of the 32 chunks of this group: lane c keeps the total of chunk c
-        double mine = 0.0;
-#pragma unroll 2
-        for (int c = 0; c < 32; ++c) {
-            const int i = g0 + c * 32 + lane;
-            if (g0 + c * 32 >= n) break;
-            const float x = i < n ? val(i) : 0.f;
-            const double t = warp_sum_f64((double)x);
-            if (lane == c) mine = t;
-            const unsigned pos = __ballot_sync(0xffffffffu, x > 0.f);
-            if (pos) lastp = g0 + c * 32 + (31 - __clz(pos));
-        }
-        double incl = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const double t = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += t;
-        }
-        const unsigned hit = __ballot_sync(0xffffffffu, run + incl > thr);
+    for (int c0 = 0; c0 < n; c0 += 32) {
+        const int i = c0 + lane;
+        const float x = i < n ? val(i) : 0.f;
+        const double incl = warp_incl_scan_f64((double)x, lane);
+        const unsigned pos = __ballot_sync(0xffffffffu, x > 0.f);
+        if (pos) lastp = c0 + (31 - __clz(pos));
+        const unsigned hit = __ballot_sync(0xffffffffu, run + incl > thr && i < n);
         if (hit) {
-            const int c = __ffs(hit) - 1;
-            const double bef_chunk = run + __shfl_sync(0xffffffffu, incl - mine, c);
-            const int i = g0 + c * 32 + lane;
-            const float x = i < n ? val(i) : 0.f;
-            double inc2 = (double)x;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double t = __shfl_up_sync(0xffffffffu, inc2, o);
-                if (lane >= o) inc2 += t;
-            }
-            const unsigned hit2 = __ballot_sync(0xffffffffu, bef_chunk + inc2 > thr && i < n);
-            int l = hit2 ? __ffs(hit2) - 1 : -1;
-            if (l < 0) {                                  // only by rounding between the two sums
-                const unsigned pos = __ballot_sync(0xffffffffu, x > 0.f);
-                l = pos ? 31 - __clz(pos) : 0;
-            }
-            before = bef_chunk + __shfl_sync(0xffffffffu, inc2 - (double)x, l);
-            last_positive = lastp;
-            return g0 + c * 32 + l;
+            const int l = __ffs(hit) - 1;
+            before = run + __shfl_sync(0xffffffffu, incl - (double)x, l);
+            return c0 + l;
         }
         run += __shfl_sync(0xffffffffu, incl, 31);
     }
     before = run;
-    last_positive = lastp;
-    return -1;
+    return lastp >= 0 ? lastp : 0;
 }
 
-// Copies the raw bytes of `cnt` elements of a row (from element e_begin) into shared memory.
+// Shared-memory strip of one warp for level 2.
 template <int kElem>
-__device__ __forceinline__ void stage_raw(const unsigned char* row, int e_begin, int cnt, unsigned char* dst, int lane)
+struct Level2Scratch {
+    static constexpr int kWordsStat = kStatBlockBytes / 32 / 4;      // raw words per lane, 4 KB block
+    static constexpr int kPerStat = kStatBlockBytes / 32 / kElem;    // elements per lane, 4 KB block
+    uint32_t raw_t[32 * (kWordsStat + 1)];
+    uint32_t raw_d[32 * (kWordsStat / 2 + 1)];
+    float w[32 * (kPerStat + 1)];
+};
+
+// Copies this lane's run (kWords 32-bit words starting at element e_lane of `row`) into its strip.
+template <int kElem, int kWords>
+__device__ __forceinline__ void stage_own_run(const unsigned char* row, int e_lane, int n_mine, uint32_t* strip)
 {
-    const unsigned char* p = row + (long long)e_begin * kElem;
-    const int bytes = cnt * kElem;
-    int done = 0;
-    if (((uintptr_t)p & 15u) == 0) {
-        const int nvec = bytes >> 4;
-#pragma unroll 4
-        for (int v = lane; v < nvec; v += 32) *reinterpret_cast<uint4*>(dst + 16 * v) = __ldg((const uint4*)(p + 16 * v));
-        done = nvec << 4;
-    }
-    if (kElem == 2) {
-        for (int o = done + 2 * lane; o < bytes; o += 64)
-            *reinterpret_cast<unsigned short*>(dst + o) = __ldg((const unsigned short*)(p + o));
+    const unsigned char* p = row + (long long)e_lane * kElem;
+    constexpr int kPer = kWords * 4 / kElem;
+    if (n_mine == kPer && ((uintptr_t)p & 15u) == 0) {
+#pragma unroll
+        for (int v = 0; v < kWords / 4; ++v) {
+            const uint4 q = __ldg((const uint4*)(p + 16 * v));
+            strip[4 * v] = q.x; strip[4 * v + 1] = q.y; strip[4 * v + 2] = q.z; strip[4 * v + 3] = q.w;
+        }
+    } else if (kElem == 4) {
+        for (int k = 0; k < n_mine; ++k) strip[k] = __ldg((const uint32_t*)(p + 4 * k));
     } else {
-        for (int o = done + 4 * lane; o < bytes; o += 128)
-            *reinterpret_cast<uint32_t*>(dst + o) = __ldg((const uint32_t*)(p + o));
+        for (int k = 0; k < n_mine; k += 2) {
+            uint32_t lo = __ldg((const unsigned short*)(p + 2 * k));
+            uint32_t hi = (k + 1 < n_mine) ? __ldg((const unsigned short*)(p + 2 * k + 2)) : 0xFF80u;
+            strip[k >> 1] = lo | (hi << 16);
+        }
     }
 }
 template <int kElem>
-__device__ __forceinline__ float raw_elem(const unsigned char* raw, int i)
+__device__ __forceinline__ float strip_elem(const uint32_t* strip, int k)
 {
-    if (kElem == 2) return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short*>(raw + 2 * i)) << 16);
-    return *reinterpret_cast<const float*>(raw + 4 * i);
+    if (kElem == 4) return __uint_as_float(strip[k]);
+    const uint32_t w = strip[k >> 1];
+    return (k & 1) ? bf16hi(w) : bf16lo(w);
 }
 
-// Level 2 over one staged unit of at most 2 KB per row: lane l owns elements [l*per, (l+1)*per).
-// f(xt, xd) is the value of an element.  Returns the element index (or -1), the unit total and the
-// last positive index.
-template <int kElem, typename F>
-__device__ __forceinline__ int raw_unit_search(const unsigned char* t_raw, const unsigned char* d_raw, int cnt, int lane,
-                                               double thr, F f, double& total, int& last_positive)
+// Level 2 over one block of kBlockBytes per row starting at element e0 (cnt valid elements): lane l
+// owns elements [l*per, (l+1)*per).  f(xt, xd) is the value of an element.  Returns the element
+// index inside the block.
+template <int kElem, int kBlockBytes, bool kTwoRows, typename F>
+__device__ __forceinline__ int level2_block(const unsigned char* trow, const unsigned char* drow, int e0, int cnt,
+                                            int lane, double thr, F f, Level2Scratch<kElem>& S)
 {
-    constexpr int kPer = kResidBlockBytes / kElem / 32;
+    constexpr int kWords = kBlockBytes / 32 / 4;
+    constexpr int kPer = kBlockBytes / 32 / kElem;
     const int i0 = lane * kPer;
     int n_mine = cnt - i0;
     n_mine = n_mine < 0 ? 0 : (n_mine > kPer ? kPer : n_mine);
+    uint32_t* st = S.raw_t + lane * (kWords + 1);
+    uint32_t* sd = S.raw_d + lane * (kWords + 1);
+    float* sw = S.w + lane * (kPer + 1);
+    stage_own_run<kElem, kWords>(trow, e0 + i0, n_mine, st);
+    if (kTwoRows) stage_own_run<kElem, kWords>(drow, e0 + i0, n_mine, sd);
     double mine = 0.0;
     int lastp = -1;
-#pragma unroll 1
+#pragma unroll 4
     for (int k = 0; k < n_mine; ++k) {
-        const float w = f(raw_elem<kElem>(t_raw, i0 + k), d_raw ? raw_elem<kElem>(d_raw, i0 + k) : 0.f);
+        const float w = f(strip_elem<kElem>(st, k), kTwoRows ? strip_elem<kElem>(sd, k) : 0.f);
+        sw[k] = w;
         mine += (double)w;
         if (w > 0.f) lastp = i0 + k;
     }
-    double incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    total = __shfl_sync(0xffffffffu, incl, 31);
+    const double incl = warp_incl_scan_f64(mine, lane);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) lastp = max(lastp, __shfl_xor_sync(0xffffffffu, lastp, o));
-    last_positive = lastp;
     const unsigned hit = __ballot_sync(0xffffffffu, incl > thr && n_mine > 0);
-    if (!hit) return -1;
+    if (!hit) return lastp >= 0 ? lastp : 0;              // only by rounding between the two levels
+    // the whole warp scans the cached values of the lane that holds the crossing
     const int src = __ffs(hit) - 1;
+    const double run0 = __shfl_sync(0xffffffffu, incl - mine, src);
+    const int n_src = __shfl_sync(0xffffffffu, n_mine, src);
+    const float* ssrc = S.w + src * (kPer + 1);
+    __syncwarp();
+    double run = run0;
     int found = -1;
-    if (lane == src) {
-        double run = incl - mine;
-#pragma unroll 1
-        for (int k = 0; k < n_mine; ++k) {
-            const float w = f(raw_elem<kElem>(t_raw, i0 + k), d_raw ? raw_elem<kElem>(d_raw, i0 + k) : 0.f);
-            if (run + (double)w > thr) { found = i0 + k; break; }
-            run += (double)w;
-        }
-        if (found < 0) found = i0 + n_mine - 1;          // only by rounding between the two sums
+#pragma unroll
+    for (int c = 0; c < kPer; c += 32) {
+        const float w = (c + lane < n_src) ? ssrc[c + lane] : 0.f;
+        const double inc = warp_incl_scan_f64((double)w, lane);
+        const unsigned h2 = __ballot_sync(0xffffffffu, run + inc > thr && c + lane < n_src);
+        if (found < 0 && h2) found = c + __ffs(h2) - 1;
+        run += __shfl_sync(0xffffffffu, inc, 31);
     }
-    return __shfl_sync(0xffffffffu, found, src);
-}
-
-// Draws from p = softmax of target row `row_t` with uniform u, using the block statistics saved by
-// the streamed pass (reference Cp = row reference).  One warp; scratch = 2 KB of shared memory.
-template <int kElem>
-__device__ __forceinline__ int sample_from_p(const VerifyParams& P, int row_t, float Cp, double u,
-                                             unsigned char* scratch, int lane)
-{
-    const float2* st = P.stats_t + (long long)row_t * P.nblk;
-    const unsigned char* trow = P.target + (long long)row_t * P.tstride_bytes;
-    auto mass = [&](int i) {
-        const float2 e = __ldcg(&st[i]);
-        return e.x > kNegInf ? e.y * ex2_approx(e.x - Cp) : 0.f;
-    };
-    const double Z = warp_total(P.nblk, lane, mass);
-    double before;
-    int lastp;
-    int b = chunked_search(P.nblk, lane, mass, u * Z, before, lastp);
-    if (b < 0) { b = lastp >= 0 ? lastp : 0; before = u * Z; }
-    const float2 sb = __ldcg(&st[b]);
-    // inside the block work in the block's own reference: divide the remaining mass by 2^(c_b - C)
-    double thr_local = (u * Z - before) / (double)ex2_approx(sb.x - Cp);
-    const float nc = -sb.x, scale = P.scale;
-    auto ev = [&](float xt, float) { return ex2_approx(__fmaf_rn(xt, scale, nc)); };
-    int token = -1, fallback = b * P.epb;
-    for (int h = 0; h < kStatBlockBytes / kResidBlockBytes; ++h) {
-        const int e0 = b * P.epb + h * P.epb_r;
-        const int cnt = (P.V - e0) < P.epb_r ? (P.V - e0) : P.epb_r;
-        if (cnt <= 0) break;
-        __syncwarp();
-        stage_raw<kElem>(trow, e0, cnt, scratch, lane);
-        __syncwarp();
-        double tot;
-        int lp;
-        const int e = raw_unit_search<kElem>(scratch, nullptr, cnt, lane, thr_local, ev, tot, lp);
-        if (lp >= 0) fallback = e0 + lp;
-        if (e >= 0) { token = e0 + e; break; }
-        thr_local -= tot;
-    }
-    return token >= 0 ? token : fallback;
-}
-
-// Draws the corrected token of a rejected position from norm(max(0, p - q)) given the per-block
-// sums of the residual pass.  One warp; scratch = 2 KB + 2 KB of shared memory.
-template <int kElem>
-__device__ __forceinline__ int sample_from_residual(const VerifyParams& P, const ResidTask& t, const float* wb,
-                                                    unsigned char* scr_t, unsigned char* scr_d, int lane)
-{
-    const double u = (double)t.u;
-    auto wv = [&](int i) { return __ldcg(&wb[i]); };
-    const double W = warp_total(P.nblk_r, lane, wv);
-    if (!(W > 0.0) || !(W < INFINITY))                       // empty residual: draw from p with the same u
-        return sample_from_p<kElem>(P, t.row_t, t.cp, u, scr_t, lane);
-    double before;
-    int lastp;
-    int b = chunked_search(P.nblk_r, lane, wv, u * W, before, lastp);
-    if (b < 0) { b = lastp >= 0 ? lastp : 0; before = u * W; }
-    const int e0 = b * P.epb_r;
-    const int cnt = (P.V - e0) < P.epb_r ? (P.V - e0) : P.epb_r;
-    __syncwarp();
-    stage_raw<kElem>(P.target + (long long)t.row_t * P.tstride_bytes, e0, cnt, scr_t, lane);
-    stage_raw<kElem>(P.draft + t.row_d * P.dstride_bytes, e0, cnt, scr_d, lane);
-    __syncwarp();
-    ResidConst K;
-    K.set(P.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
-    double tot;
-    int lp;
-    int e = raw_unit_search<kElem>(scr_t, scr_d, cnt, lane, u * W - before,
-                                   [&](float xt, float xd) { return resid_elem(xt, xd, K); }, tot, lp);
-    if (e < 0) e = lp >= 0 ? lp : 0;
-    return e0 + e;
+    if (found < 0) found = n_src - 1;                     // only by rounding between the two sums
+    return src * kPer + found;
 }
 
 // ---------------------------------------------------------------------------------------
 // decide: one CTA per request, one warp per position (eight per round): row statistics from
 // block statistics, p(x), q(x), accept test, first rejection n_r; the accepted prefix is written.
-// Position j = len is the bonus row (statistics only).  A fully accepted request draws its bonus
-// token here; a rejected one is queued for the residual pass.
+// Position j = len is the bonus row (statistics only).  Every request leaves a record for the
+// finalize kernel; a rejected one is also queued for the residual pass.
 // ---------------------------------------------------------------------------------------
-template <int kElem>
 __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
 {
     constexpr int kWarps = kDecideThreads / 32;
-    __shared__ int s_first, s_bad, s_have_fin, s_kind;
+    __shared__ int s_first, s_bad, s_have_fin;
     __shared__ float s_Ct[kWarps], s_Cd[kWarps];
     __shared__ double s_St[kWarps], s_Sd[kWarps];
     __shared__ float s_fin_C[2];     // [0] target, [1] draft statistics of the row that emits the token
     __shared__ double s_fin_S[2];
-    __shared__ float s_u;
-    __shared__ __align__(16) unsigned char s_scratch[kResidBlockBytes];
 
     pdl_launch_dependents();
     pdl_wait();
@@ -795,12 +769,12 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     const int lo = P.row_offsets[r], hi = P.row_offsets[r + 1];
     // the request's rows must lie inside the batch, and so must its draft rows (compact index lo - r)
     if (lo < 0 || hi - lo < 1 || hi > n_rows || lo - r < 0 || (hi - 1 - r) > n_rows - P.R) {
-        if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS); P.accepted_len[r] = 0; }
+        if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
         return;
     }
     const int len = hi - lo - 1;
     const long long drow0 = P.draft_row_start ? P.draft_row_start[r] : (long long)(lo - r);
-    if (tid == 0) { s_first = len; s_bad = 0; s_have_fin = 0; s_kind = kTaskNone; }
+    if (tid == 0) { s_first = len; s_bad = 0; s_have_fin = 0; }
     __syncthreads();
     for (int i = tid; i <= len; i += kDecideThreads) {
         P.out_tokens[lo + i] = -1;
@@ -811,7 +785,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     }
     __syncthreads();
     if (s_bad) {
-        if (tid == 0) { atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; }
+        if (tid == 0) { atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
         return;
     }
     const bool want_all = (P.out_p != nullptr) || (P.out_q != nullptr);
@@ -831,6 +805,16 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             RowAcc A, D;
             combine_rows(P.stats_t + (long long)(lo + j) * P.nblk,
                          is_draft_pos ? P.stats_d + (long long)(lo - r + j) * P.nblk : nullptr, P.nblk, lane, A, D);
+            if (!is_draft_pos) {
+                // bonus row: leave its block masses (relative to the row reference) where the finalize
+                // kernel looks for block values; a rejected request overwrites them in the residual pass
+                const float2* st = P.stats_t + (long long)(lo + j) * P.nblk;
+                float* wb = P.wblk + (long long)r * P.nblk_r;
+                for (int b = lane; b < P.nblk; b += 32) {
+                    const float2 e = __ldcg(&st[b]);
+                    wb[b] = (e.x > kNegInf && A.C > kNegInf) ? e.y * ex2_approx(e.x - A.C) : 0.f;
+                }
+            }
             if (lane == 0) {
                 s_Ct[warp] = A.C; s_St[warp] = A.S; s_Cd[warp] = D.C; s_Sd[warp] = D.S;
                 if (is_draft_pos) {
@@ -861,57 +845,121 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
         if (stop) break;
     }
 
+    if (tid != 0) return;
     const int n = s_first;
-    if (tid == 0) {
-        if (s_bad || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
-            (n < len && !row_usable(s_fin_C[1], s_fin_S[1]))) {
-            atomicOr(P.dev_status, s_bad ? s_bad : DSPARK_DEV_BAD_ROW);
-            P.accepted_len[r] = 0;
+    RequestRec rec;
+    rec.kind = kTaskNone; rec.row_t = lo + n; rec.row_d = drow0 + n;
+    rec.cp = rec.cq = 0.f; rec.inv_zp = rec.inv_zq = 1.f; rec.u = 0.f; rec.pad[0] = rec.pad[1] = rec.pad[2] = 0;
+    if (s_bad || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
+        (n < len && !row_usable(s_fin_C[1], s_fin_S[1]))) {
+        atomicOr(P.dev_status, s_bad ? s_bad : DSPARK_DEV_BAD_ROW);
+        P.accepted_len[r] = 0;
+    } else {
+        for (int i = 0; i < n; ++i) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
+        float ua, ur;
+        philox_uniforms(P.seed, (uint32_t)r, (uint32_t)n, ua, ur);
+        P.accepted_len[r] = n;
+        rec.u = ur;
+        rec.cp = s_fin_C[0]; rec.inv_zp = (float)(1.0 / s_fin_S[0]);
+        if (n < len) {
+            rec.cq = s_fin_C[1]; rec.inv_zq = (float)(1.0 / s_fin_S[1]);
+            rec.kind = kTaskResid;
+            const int slot = atomicAdd(&P.counters[0], 1);
+            ResidTask q;
+            q.request = r; q.row_t = rec.row_t; q.row_d = rec.row_d;
+            q.cp = rec.cp; q.inv_zp = rec.inv_zp; q.cq = rec.cq; q.inv_zq = rec.inv_zq;
+            q.u = ur; q.pad[0] = q.pad[1] = q.pad[2] = 0;
+            P.resid[slot] = q;
         } else {
-            for (int i = 0; i < n; ++i) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
-            float ua, ur;
-            philox_uniforms(P.seed, (uint32_t)r, (uint32_t)n, ua, ur);
-            s_u = ur;
-            P.accepted_len[r] = n;
-            if (n < len) {
-                const int slot = atomicAdd(&P.counters[0], 1);
-                ResidTask q;
-                q.request = r; q.row_t = lo + n; q.row_d = drow0 + n;
-                q.cp = s_fin_C[0]; q.inv_zp = (float)(1.0 / s_fin_S[0]);
-                q.cq = s_fin_C[1]; q.inv_zq = (float)(1.0 / s_fin_S[1]);
-                q.u = ur; q.pad[0] = q.pad[1] = q.pad[2] = 0;
-                P.resid[slot] = q;
-                s_kind = kTaskResid;
-            } else {
-                s_kind = kTaskBonus;
-            }
+            rec.kind = kTaskBonus;
         }
     }
-    __syncthreads();
-    if (s_kind != kTaskBonus || warp != 0) return;
-    const int token = sample_from_p<kElem>(P, lo + n, s_fin_C[0], (double)s_u, s_scratch, lane);
-    if (lane == 0) P.out_tokens[lo + n] = token;
+    P.req[r] = rec;
 }
 
 // ---------------------------------------------------------------------------------------
-// finalize: one warp per queued (rejected) request draws the corrected token from the residual.
+// finalize: one warp per request draws the token that follows the accepted prefix: from
+// norm(max(0, p - q)) of the rejected position (block sums from the residual pass), or the bonus
+// token from p of the last row (block statistics saved by the streamed pass).
 // ---------------------------------------------------------------------------------------
-constexpr int kFinalizeThreads = 128;
+constexpr int kFinalizeWarps = 2;
 template <int kElem>
-__global__ void __launch_bounds__(kFinalizeThreads) finalize_kernel(VerifyParams P)
+__global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyParams P)
 {
-    __shared__ __align__(16) unsigned char s_scratch[kFinalizeThreads / 32][2 * kResidBlockBytes];
+    __shared__ Level2Scratch<kElem> s_scr[kFinalizeWarps];
     pdl_launch_dependents();
     pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int slot = blockIdx.x * (kFinalizeThreads / 32) + warp;
-    int nq = __ldcg(&P.counters[0]);
-    nq = nq > P.R ? P.R : nq;
-    if (slot >= nq) return;
-    const ResidTask t = P.resid[slot];
-    const int token = sample_from_residual<kElem>(P, t, P.wblk + (long long)slot * P.nblk_r, s_scratch[warp],
-                                                  s_scratch[warp] + kResidBlockBytes, lane);
-    if (lane == 0) P.out_tokens[t.row_t] = token;
+    const int r = blockIdx.x * kFinalizeWarps + warp;
+    if (r >= P.R) return;
+    // issue everything that does not depend on the record together with it: the block values of
+    // this request (residual sums of a rejected position, or masses of the bonus row)
+    const RequestRec rec = P.req[r];
+    const float* wb = P.wblk + (long long)r * P.nblk_r;
+    const bool in_regs = P.nblk_r <= 256;
+    float xr[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { const int i = k * 32 + lane; xr[k] = (in_regs && i < P.nblk_r) ? __ldcg(&wb[i]) : 0.f; }
+    if (rec.kind == kTaskNone) return;
+    Level2Scratch<kElem>& S = s_scr[warp];
+    const double u = (double)rec.u;
+    const unsigned char* trow = P.target + (long long)rec.row_t * P.tstride_bytes;
+    int token = -1;
+    for (int attempt = 0; attempt < 2 && token < 0; ++attempt) {
+        const bool resid = (rec.kind == kTaskResid) && attempt == 0;
+        const int n1 = resid ? P.nblk_r : P.nblk;
+        if (attempt == 1) {
+            // empty residual (p and q agree to rounding): draw from p with the same u; the block masses
+            // of that row are rebuilt from the saved statistics
+            const float2* st = P.stats_t + (long long)rec.row_t * P.nblk;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int i = k * 32 + lane;
+                float m = 0.f;
+                if (i < P.nblk && P.nblk <= 256) { const float2 e = __ldcg(&st[i]); m = e.x > kNegInf ? e.y * ex2_approx(e.x - rec.cp) : 0.f; }
+                xr[k] = m;
+            }
+        }
+        double before, tot;
+        int b;
+        if (n1 <= 256) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) if (k * 32 + lane >= n1) xr[k] = 0.f;   // a bonus row has fewer blocks
+            b = level1_registers(xr, n1, lane, u, before, tot);
+        } else if (attempt == 0) {
+            auto wv = [&](int i) { return __ldcg(&wb[i]); };
+            tot = warp_total(n1, lane, wv);
+            b = level1_memory(n1, lane, wv, u * tot, before);
+        } else {
+            const float2* st = P.stats_t + (long long)rec.row_t * P.nblk;
+            auto mass = [&](int i) { const float2 e = __ldcg(&st[i]); return e.x > kNegInf ? e.y * ex2_approx(e.x - rec.cp) : 0.f; };
+            tot = warp_total(n1, lane, mass);
+            b = level1_memory(n1, lane, mass, u * tot, before);
+        }
+        if (!(tot > 0.0) || !(tot < INFINITY)) {
+            if (!resid) token = 0;                           // cannot happen for a usable row
+            continue;
+        }
+        const double thr_local = u * tot - before;
+        if (resid) {
+            ResidConst K;
+            K.set(P.scale, rec.cp, rec.inv_zp, rec.cq, rec.inv_zq);
+            const int e0 = b * P.epb_r;
+            const int cnt = (P.V - e0) < P.epb_r ? (P.V - e0) : P.epb_r;
+            const unsigned char* drow = P.draft + rec.row_d * P.dstride_bytes;
+            token = e0 + level2_block<kElem, kResidBlockBytes, true>(
+                trow, drow, e0, cnt, lane, thr_local, [&](float xt, float xd) { return resid_elem(xt, xd, K); }, S);
+        } else {
+            // element masses relative to the row reference, like the block masses
+            const float nc = -rec.cp, scale = P.scale;
+            const int e0 = b * P.epb;
+            const int cnt = (P.V - e0) < P.epb ? (P.V - e0) : P.epb;
+            token = e0 + level2_block<kElem, kStatBlockBytes, false>(
+                trow, nullptr, e0, cnt, lane, thr_local,
+                [&](float xt, float) { return ex2_approx(__fmaf_rn(xt, scale, nc)); }, S);
+        }
+    }
+    if (lane == 0) P.out_tokens[rec.row_t] = token;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -1019,7 +1067,7 @@ static void launch_stream(const VerifyParams& P, bool bulk, long long max_units,
 {
     const int sms = device_info().sms;
     if (bulk) {
-        long long g = (long long)sms * 2;
+        long long g = (long long)sms * 3;
         if (g > max_units) g = max_units;
         if (g < 1) g = 1;
         launch_pdl(stream_bulk_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kStreamThreads), kStages * kStageBytes, s, P);
@@ -1039,7 +1087,7 @@ static void launch_stream_dtype(const VerifyParams& P, bool bulk, long long max_
 }
 
 struct Workspace {
-    size_t counters, stats_t, stats_d, resid, wblk, total;
+    size_t counters, stats_t, stats_d, resid, req, wblk, total;
 };
 static Workspace workspace_layout(int R, int n_rows, int V)
 {
@@ -1052,6 +1100,7 @@ static Workspace workspace_layout(int R, int n_rows, int V)
     w.stats_t = o;  o += up((size_t)n_rows * nblk * sizeof(float2));
     w.stats_d = o;  o += up((size_t)n_rows * nblk * sizeof(float2));
     w.resid = o;    o += up((size_t)R * sizeof(ResidTask));
+    w.req = o;      o += up((size_t)R * sizeof(RequestRec));
     w.wblk = o;     o += up((size_t)R * nblk_r * sizeof(float));
     w.total = o;
     return w;
@@ -1095,6 +1144,7 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.stats_t = (float2*)(ws + w.stats_t);
     P.stats_d = (float2*)(ws + w.stats_d);
     P.resid = (ResidTask*)(ws + w.resid);
+    P.req = (RequestRec*)(ws + w.req);
     P.wblk = (float*)(ws + w.wblk);
     return DSPARK_OK;
 }
@@ -1177,8 +1227,7 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_DECIDE, s);
-        if (P.elem == 2) launch_pdl(decide_kernel<2>, dim3(R), dim3(kDecideThreads), 0, s, P);
-        else launch_pdl(decide_kernel<4>, dim3(R), dim3(kDecideThreads), 0, s, P);
+        launch_pdl(decide_kernel, dim3(R), dim3(kDecideThreads), 0, s, P);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
@@ -1188,9 +1237,9 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_FINALIZE, s);
-        const int grid = (R + kFinalizeThreads / 32 - 1) / (kFinalizeThreads / 32);
-        if (P.elem == 2) launch_pdl(finalize_kernel<2>, dim3(grid), dim3(kFinalizeThreads), 0, s, P);
-        else launch_pdl(finalize_kernel<4>, dim3(grid), dim3(kFinalizeThreads), 0, s, P);
+        const int grid = (R + kFinalizeWarps - 1) / kFinalizeWarps;
+        if (P.elem == 2) launch_pdl(finalize_kernel<2>, dim3(grid), dim3(kFinalizeWarps * 32), 0, s, P);
+        else launch_pdl(finalize_kernel<4>, dim3(grid), dim3(kFinalizeWarps * 32), 0, s, P);
     }
     return launch_status();
 }

@@ -25,7 +25,7 @@ def gpu_schedule(sched: W.ScheduleInput, mode: int, topk: int = 0, draft_len=Non
     surv = torch.full((R, gamma), -1.0, dtype=torch.float32, device="cuda") if want_all else None
     exp = torch.full((R,), -1.0, dtype=torch.float32, device="cuda") if want_all else None
     info = torch.zeros(32, dtype=torch.uint8, device="cuda")
-    ws = B.workspace(B.dspark_schedule_workspace_bytes(R, gamma))
+    ws = B.workspace(B.dspark_schedule_workspace_bytes(R, gamma)).fill_(0xFF)     # results must not depend on its content
     dl = None if draft_len is None else torch.as_tensor(draft_len, dtype=torch.int32).cuda()
     B.dspark_schedule(prof, conf, sched.budget_tokens, mode, topk, dl, out_len=out_len, out_row_offsets=off,
                       out_survival=surv, out_expected_len=exp, out_info=info, workspace=ws)
@@ -60,7 +60,7 @@ def gpu_verify_greedy(batch: W.VerifyBatch, n_rows_cap=None):
     acc = torch.full((R,), -7, dtype=torch.int32, device="cuda")
     out = torch.full((cap,), -7, dtype=torch.int32, device="cuda")
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    ws = B.workspace(B.dspark_verify_workspace_bytes(R, cap, batch.V))
+    ws = B.workspace(B.dspark_verify_workspace_bytes(R, cap, batch.V)).fill_(0xFF)
     B.dspark_verify_greedy(batch.target, batch.row_offsets, batch.draft_tokens, accepted_len=acc,
                            out_tokens=out, dev_status=st, workspace=ws, n_rows=cap)
     torch.cuda.synchronize()
@@ -86,7 +86,7 @@ def gpu_verify(batch: W.VerifyBatch, want_probs=True, n_rows_cap=None):
     p = torch.full((cap,), float("nan"), dtype=torch.float32, device="cuda") if want_probs else None
     q = torch.full((cap,), float("nan"), dtype=torch.float32, device="cuda") if want_probs else None
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    ws = B.workspace(B.dspark_verify_workspace_bytes(R, cap, batch.V))
+    ws = B.workspace(B.dspark_verify_workspace_bytes(R, cap, batch.V)).fill_(0xFF)     # poisoned: NaN patterns everywhere
     B.dspark_verify(batch.target, batch.draft, batch.row_offsets, batch.draft_tokens, batch.temperature,
                     batch.seed, draft_row_start=batch.draft_row_start, accepted_len=acc, out_tokens=out,
                     out_p_tok=p, out_q_tok=q, dev_status=st, workspace=ws, n_rows=cap)
