@@ -99,10 +99,11 @@ __device__ __forceinline__ float lg2_approx(float x)
     return y;
 }
 // Programmatic dependent launch: every kernel of the library is launched so that its CTAs may be
-// scheduled while the previous kernel on the stream drains; pdl_wait() returns once that kernel
-// has completed and its writes are visible, and must precede any read of its results.
+// scheduled as soon as the previous kernel on the stream drains (no explicit early trigger: CTAs
+// that arrive early only poll and take issue slots from the kernel they wait for); pdl_wait()
+// returns once that kernel has completed and its writes are visible, and must precede any read of
+// its results.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Packed pairs of fp32 (sm_100 f32x2 arithmetic: one instruction, two IEEE-rounded results).
 __device__ __forceinline__ uint64_t pack2(float a, float b)

@@ -61,7 +61,6 @@ __device__ __forceinline__ unsigned long long fix40(float a)
 // chain and keeps the value of its own position), the mass prefix is a segmented warp scan.
 __global__ void __launch_bounds__(kPrepThreads) sched_prep_kernel(SchedParams P)
 {
-    pdl_launch_dependents();
     pdl_wait();
     if (blockIdx.x == 0 && threadIdx.x == 0) *P.ticket = 0;
     const int lane = threadIdx.x & 31;
@@ -156,7 +155,6 @@ __global__ void __launch_bounds__(kSchedThreads, 1) sched_rank_kernel(SchedParam
     __shared__ unsigned int s_rank[kWarps][32];
     __shared__ unsigned long long s_mass[kWarps][32];
     __shared__ int s_is_last;
-    pdl_launch_dependents();
     pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int tile = blockIdx.x;
@@ -389,7 +387,6 @@ __device__ void sched_final_stage(const SchedParams& P)
 // No candidates at all (gamma = 0): only the final stage runs.
 __global__ void __launch_bounds__(kSchedThreads, 1) sched_final_only_kernel(SchedParams P)
 {
-    pdl_launch_dependents();
     pdl_wait();
     sched_final_stage(P);
 }
@@ -399,7 +396,6 @@ build_offsets_kernel(const int32_t* __restrict__ lengths, int R, int32_t* __rest
 {
     __shared__ unsigned long long s_warp_tot[32];
     __shared__ unsigned long long s_carry;
-    pdl_launch_dependents();
     pdl_wait();
     const int tid = threadIdx.x;
     if (tid == 0) s_carry = 0ull;

@@ -403,7 +403,6 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kConsumerWarps); }
         s_abort = 0;
@@ -481,7 +480,6 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
 {
     using M = ModeCfg<kMode>;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    pdl_launch_dependents();
     pdl_wait();
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
@@ -759,7 +757,6 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     __shared__ float s_fin_C[2];     // [0] target, [1] draft statistics of the row that emits the token
     __shared__ double s_fin_S[2];
 
-    pdl_launch_dependents();
     pdl_wait();
     const int r = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -887,7 +884,6 @@ template <int kElem>
 __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyParams P)
 {
     __shared__ Level2Scratch<kElem> s_scr[kFinalizeWarps];
-    pdl_launch_dependents();
     pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int r = blockIdx.x * kFinalizeWarps + warp;
@@ -963,68 +959,77 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
 }
 
 // ---------------------------------------------------------------------------------------
-// greedy decide: one warp per request, one lane per row (all rows of a request in flight).
+// greedy decide: one CTA per request, one warp per row (eight rows per round): the row argmax
+// from its block statistics, then the first draft token that differs from it.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kDecideThreads) greedy_decide_kernel(VerifyParams P)
 {
-    pdl_launch_dependents();
+    constexpr int kWarps = kDecideThreads / 32;
+    __shared__ int s_bad, s_first, s_am[kWarps], s_neg[kWarps], s_emit, s_status;
     pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * (kDecideThreads / 32) + (threadIdx.x >> 5);
-    if (r >= P.R) return;
+    const int r = blockIdx.x;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
     const int lo = P.row_offsets[r], hi = P.row_offsets[r + 1];
     if (lo < 0 || hi - lo < 1 || hi > n_rows) {
-        if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS); P.accepted_len[r] = 0; }
+        if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS); P.accepted_len[r] = 0; }
         return;
     }
     const int len = hi - lo - 1;
-    int bad = 0;
-    for (int i = lane; i <= len; i += 32) {
+    if (tid == 0) { s_bad = 0; s_first = 0x7fffffff; s_emit = -1; s_status = 0; }
+    __syncthreads();
+    for (int i = tid; i <= len; i += kDecideThreads) {
         P.out_tokens[lo + i] = -1;
-        if (i < len) { const int d = P.draft_tokens[lo + i]; if (d < 0 || d >= P.V) bad = 1; }
+        if (i < len) { const int d = P.draft_tokens[lo + i]; if (d < 0 || d >= P.V) s_bad = 1; }
     }
-    if (__any_sync(0xffffffffu, bad)) {
-        if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN); P.accepted_len[r] = 0; }
+    __syncthreads();
+    if (s_bad) {
+        if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN); P.accepted_len[r] = 0; }
         return;
     }
-    __syncwarp();
-    int n = len, emitted = -1, status = 0;
-    bool done = false;
-    for (int j0 = 0; j0 <= len && !done; j0 += 32) {
-        const int j = j0 + lane;
-        int am = -1, neg = 0;
+    for (int j0 = 0; j0 <= len; j0 += kWarps) {
+        const int j = j0 + warp;
         if (j <= len) {
             const float2* st = P.stats_t + (long long)(lo + j) * P.nblk;
             float best = kNegInf;
             int bi = 0x7fffffff;
-#pragma unroll 4
-            for (int b = 0; b < P.nblk; ++b) {
+            for (int b = lane; b < P.nblk; b += 32) {      // lane-strided: ascending indices per lane
                 const float2 e = __ldcg(&st[b]);
                 const int idx = __float_as_int(e.y);
                 if (e.x > best || (e.x == best && idx < bi)) { best = e.x; bi = idx; }
             }
-            am = bi;
-            if (best == kNegInf) { am = 0; neg = 1; }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+            }
+            if (lane == 0) {
+                const int neg = (best == kNegInf);
+                const int am = neg ? 0 : bi;
+                s_am[warp] = am; s_neg[warp] = neg;
+                // the bonus row always ends the scan; a draft row ends it on a mismatch
+                if (j == len || P.draft_tokens[lo + j] != am) atomicMin(&s_first, j);
+            }
         }
-        const bool ends = (j < len) ? (P.draft_tokens[lo + j] != am) : (j == len);   // mismatch, or the bonus row
-        const unsigned mm = __ballot_sync(0xffffffffu, ends);
-        unsigned negs = __ballot_sync(0xffffffffu, neg);
-        if (mm) {
-            const int src = __ffs(mm) - 1;
-            n = j0 + src;
-            emitted = __shfl_sync(0xffffffffu, am, src);
-            negs &= (src == 31) ? 0xffffffffu : ((2u << src) - 1u);   // only rows up to the one that emits
-            done = true;
+        __syncthreads();
+        const int first = s_first;
+        if (tid == 0) {
+            // rows of this round up to the one that emits may raise the all -inf flag
+            const int last_j = first < j0 + kWarps ? first : j0 + kWarps - 1;
+            for (int w = 0; j0 + w <= last_j && w < kWarps; ++w) if (s_neg[w]) s_status |= DSPARK_DEV_ALL_NEG_INF;
+            if (first < j0 + kWarps) s_emit = s_am[first - j0];
         }
-        if (negs) status |= DSPARK_DEV_ALL_NEG_INF;
+        __syncthreads();
+        if (first < j0 + kWarps) break;
     }
-    for (int i = lane; i < n; i += 32) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
-    if (lane == 0) {
-        P.out_tokens[lo + n] = emitted;
+    const int n = s_first;
+    for (int i = tid; i < n; i += kDecideThreads) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
+    if (tid == 0) {
+        P.out_tokens[lo + n] = s_emit;
         P.accepted_len[r] = n;
-        if (status) atomicOr(P.dev_status, status);
+        if (s_status) atomicOr(P.dev_status, s_status);
     }
 }
 
@@ -1189,8 +1194,7 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_GREEDY_DECIDE, s);
-        const int warps_per_cta = kDecideThreads / 32;
-        launch_pdl(greedy_decide_kernel, dim3((R + warps_per_cta - 1) / warps_per_cta), dim3(kDecideThreads), 0, s, P);
+        launch_pdl(greedy_decide_kernel, dim3(R), dim3(kDecideThreads), 0, s, P);
     }
     return launch_status();
 }
