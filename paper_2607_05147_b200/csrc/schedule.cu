@@ -4,10 +4,12 @@
 // list.  Here nothing is sorted: every request's survival products are already in
 // descending order (a_{r,j} is non-increasing in j), so the position of a candidate in the
 // global order, and the exact expected-accept mass admitted up to it, are sums over all
-// requests of one binary search each.  Two kernels on the caller's stream:
+// requests of one binary search each.  Three kernels on the caller's stream:
 //   prep   one warp per request: a_{r,j} as a left-to-right fp32 product, per-tile inclusive
 //          prefix sums of the fixed-point mass (units of 2^-40, exact integers);
-//   rank   one CTA per tile of 32 candidates, 32 warps each searching a slice of all tiles
+//   select one CTA: histogram of the survival bit patterns, the threshold bin for the admission
+//          cap (budget - R), compaction of the candidates that can possibly be admitted;
+//   rank   one CTA per tile of 32 such candidates, 32 warps each searching a slice of all tiles
 //          (tiles are loaded coalesced and searched with warp shuffles): candidate c gets
 //          rank_c = #{keys <= key_c} and T_c = R*2^40 + mass of those keys, scattered to
 //          by-rank arrays; the CTA that finishes last (a ticket counter, nobody waits) then
@@ -41,7 +43,8 @@ struct SchedParams {
     int32_t* cnt;                   // [R] candidates of request r (bit 30: a confidence was clamped)
     unsigned long long* t_by_rank;  // [N+1] T_i
     int32_t* owner_by_rank;         // [N+1] request of the i-th admitted candidate
-    int* ticket;                    // counts finished rank CTAs (zeroed by the prep kernel)
+    int32_t* cand;                  // [n_tiles*32] entry indices of the candidates worth ranking
+    int* ticket;                    // [0] finished rank CTAs, [1] number of entries in cand (select kernel)
 };
 
 __device__ __forceinline__ float sanitize_conf(float c, int& clamped)
@@ -62,7 +65,7 @@ __device__ __forceinline__ unsigned long long fix40(float a)
 __global__ void __launch_bounds__(kPrepThreads) sched_prep_kernel(SchedParams P)
 {
     pdl_wait();
-    if (blockIdx.x == 0 && threadIdx.x == 0) *P.ticket = 0;
+    if (!P.cand && blockIdx.x == 0 && threadIdx.x == 0) P.ticket[0] = 0;   // else the select kernel does it
     const int lane = threadIdx.x & 31;
     const int wid = blockIdx.x * (kPrepThreads / 32) + (threadIdx.x >> 5);
     const int gamma = P.gamma, gpad = P.gpad, seg = P.seg;
@@ -108,6 +111,75 @@ __global__ void __launch_bounds__(kPrepThreads) sched_prep_kernel(SchedParams P)
         if (real && j < gamma && P.out_surv) P.out_surv[(size_t)r * gamma + j] = mine;
     }
     if (real && k_in_seg == 0) P.cnt[r] = n | (clamped ? (1 << 30) : 0);
+}
+
+// ---- Candidates worth ranking ---------------------------------------------------------------
+// At most cap = budget - R candidates can be admitted, so only the cap largest survival values
+// need a rank.  One CTA histograms the fp32 bit patterns (32 bins per binade, larger a = lower
+// bin), finds the first bin at which the running count reaches the cap, and compacts the entry
+// indices of all candidates up to that bin (the top-M set, M >= min(cap, |E|)).
+constexpr int kSelectBins = 4096;
+__device__ __forceinline__ int select_bin(uint32_t a_bits) { return (int)((0x3F800000u - a_bits) >> 18); }
+
+__global__ void __launch_bounds__(kSchedThreads, 1) sched_select_kernel(SchedParams P)
+{
+    __shared__ int s_hist[kSelectBins];
+    __shared__ int s_warp_tot[32];
+    __shared__ int s_bin_star, s_base;
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_entries = P.n_tiles * 32;
+    long long cap = (long long)P.budget - (long long)P.R;
+    if (cap < 0) cap = 0;
+    for (int b = tid; b < kSelectBins; b += kSchedThreads) s_hist[b] = 0;
+    if (tid == 0) { s_bin_star = kSelectBins - 1; s_base = 0; P.ticket[0] = 0; }
+    __syncthreads();
+    for (int e = tid; e < n_entries; e += kSchedThreads) {
+        const uint32_t a = P.akey[e];
+        if (a) atomicAdd(&s_hist[select_bin(a)], 1);
+    }
+    __syncthreads();
+    // first bin whose inclusive prefix count reaches the cap (4 consecutive bins per thread)
+    {
+        int c[4], sum = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { c[k] = s_hist[tid * 4 + k]; sum += c[k]; }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+        if (lane == 31) s_warp_tot[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int t = s_warp_tot[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(0xffffffffu, t, o); if (lane >= o) t += u; }
+            s_warp_tot[lane] = t;
+        }
+        __syncthreads();
+        long long run = (long long)(incl - sum) + (warp > 0 ? s_warp_tot[warp - 1] : 0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const long long before = run;
+            run += c[k];
+            if (before < cap && run >= cap) s_bin_star = tid * 4 + k;      // exactly one bin crosses the cap
+        }
+    }
+    __syncthreads();
+    const int bin_star = s_bin_star;
+    // compaction: each warp reserves room with one shared-memory atomic (the order of cand does not
+    // matter: every candidate is ranked independently of the others)
+    for (int base = 0; base < n_entries; base += kSchedThreads) {
+        const int e = base + tid;
+        const uint32_t a = e < n_entries ? P.akey[e] : 0u;
+        const bool keep = a != 0u && select_bin(a) <= bin_star;
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        int off = 0;
+        if (lane == 0 && m) off = atomicAdd(&s_base, __popc(m));
+        off = __shfl_sync(0xffffffffu, off, 0);
+        if (keep) P.cand[off + __popc(m & ((1u << lane) - 1u))] = e;
+    }
+    __syncthreads();
+    if (tid == 0) P.ticket[1] = s_base;
 }
 
 // ---- S2 + S3 without a sort: rank and admitted mass of every candidate ------------------------
@@ -157,13 +229,15 @@ __global__ void __launch_bounds__(kSchedThreads, 1) sched_rank_kernel(SchedParam
     __shared__ int s_is_last;
     pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int tile = blockIdx.x;
     const int tiles_per_req = P.gpad > 32 ? P.gpad / 32 : 1;
+    const int n_cand = P.cand ? __ldcg(&P.ticket[1]) : P.n_tiles * 32;   // no selection: every entry
 
-    // my candidate
-    const int e = tile * 32 + lane;            // flat padded entry index
-    const uint32_t a1 = P.akey[e];
-    const int r1 = P.gpad > 32 ? tile / tiles_per_req : e / P.gpad;
+  for (int ctile = blockIdx.x; ctile * 32 < n_cand; ctile += gridDim.x) {
+    // my candidate (one of the compacted entries worth ranking)
+    const int ci = ctile * 32 + lane;
+    const int e = ci < n_cand ? (P.cand ? __ldcg(&P.cand[ci]) : ci) : 0;   // flat padded entry index
+    const uint32_t a1 = ci < n_cand ? P.akey[e] : 0u;
+    const int r1 = e / P.gpad;
     const int j1 = e - r1 * P.gpad;
 
     unsigned int rank = 0;
@@ -197,8 +271,9 @@ __global__ void __launch_bounds__(kSchedThreads, 1) sched_rank_kernel(SchedParam
         P.t_by_rank[rk] = ms;
         P.owner_by_rank[rk] = r1;
     }
+    __syncthreads();                           // s_rank / s_mass are reused by the next candidate tile
+  }
     // the CTA that finishes last walks the path (no CTA ever waits for another)
-    __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         s_is_last = (atomicAdd(P.ticket, 1) == (int)gridDim.x - 1);
@@ -415,7 +490,7 @@ build_offsets_kernel(const int32_t* __restrict__ lengths, int R, int32_t* __rest
 }
 
 // Padded geometry: positions per request, requests after padding, tiles of 32 entries.
-struct SchedGeom { int gpad, seg, R_pad, n_tiles; size_t akey, pfix, cnt, tbr, obr, ticket, total; };
+struct SchedGeom { int gpad, seg, R_pad, n_tiles; size_t akey, pfix, cnt, tbr, obr, cand, ticket, total; };
 static SchedGeom sched_geom(int R, int gamma)
 {
     SchedGeom g;
@@ -434,7 +509,8 @@ static SchedGeom sched_geom(int R, int gamma)
     g.cnt = o;  o += up((size_t)R * sizeof(int32_t));
     g.tbr = o;  o += up((n_entries + 1) * sizeof(unsigned long long));
     g.obr = o;  o += up((n_entries + 1) * sizeof(int32_t));
-    g.ticket = o; o += up(sizeof(int));
+    g.cand = o; o += up(n_entries * sizeof(int32_t));
+    g.ticket = o; o += up(2 * sizeof(int));
     g.total = o;
     return g;
 }
@@ -482,6 +558,12 @@ int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32
     P.cnt = (int32_t*)(ws + g.cnt);
     P.t_by_rank = (unsigned long long*)(ws + g.tbr);
     P.owner_by_rank = (int32_t*)(ws + g.obr);
+    {
+        long long cap0 = (long long)budget_tokens - R;
+        cap0 = cap0 < 0 ? 0 : cap0;
+        const long long n_entries0 = (long long)g.n_tiles * 32;
+        P.cand = (n_entries0 >= 8192 && cap0 * 2 <= n_entries0) ? (int32_t*)(ws + g.cand) : nullptr;
+    }
     P.ticket = (int*)(ws + g.ticket);
 
     cudaStream_t s = (cudaStream_t)stream;
@@ -490,7 +572,18 @@ int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32
     const int prep_ctas = (prep_warps + kPrepThreads / 32 - 1) / (kPrepThreads / 32);
     launch_pdl(sched_prep_kernel, dim3(prep_ctas), dim3(kPrepThreads), 0, s, P);
     if (g.n_tiles > 0 && gamma > 0) {
-        const dim3 grid(g.n_tiles), block(kSchedThreads);
+        // Ranking only the candidates that fit under the cap pays once the candidate set is large and
+        // the cap cuts at least half of it; small problems rank every entry and save the extra kernel.
+        long long cap = (long long)budget_tokens - R;
+        cap = cap < 0 ? 0 : cap;
+        const long long n_entries = (long long)g.n_tiles * 32;
+        const bool select = n_entries >= 8192 && cap * 2 <= n_entries;
+        long long want = g.n_tiles;
+        if (select) {
+            launch_pdl(sched_select_kernel, dim3(1), dim3(kSchedThreads), 0, s, P);
+            want = (cap + n_entries / 16) / 32 + 1;    // the cap plus histogram slack; the kernel loops if more
+        }
+        const dim3 grid((unsigned)(want < g.n_tiles ? want : g.n_tiles)), block(kSchedThreads);
         switch (g.seg) {
             case 1: launch_pdl(sched_rank_kernel<1>, grid, block, 0, s, P); break;
             case 2: launch_pdl(sched_rank_kernel<2>, grid, block, 0, s, P); break;

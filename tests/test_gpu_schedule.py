@@ -86,6 +86,24 @@ def test_edge_cases():
     H.check_schedule(W.ScheduleInput(big[:64], [1, 100], [50.0, 40.0], 10**6, 100), B.DSPARK_SCHED_GLOBAL)
 
 
+def test_selection_path_with_mass_ties():
+    # large candidate set + small cap: the library ranks only the candidates that fit under the cap;
+    # here thousands of candidates share the same survival value, so the cap falls inside a tie group
+    rng = np.random.default_rng(11)
+    R, gamma = 640, 16                                     # 10 240 entries
+    conf = rng.choice([1.0, 0.5, 0.75], size=(R, gamma), p=[0.5, 0.3, 0.2]).astype(np.float32)
+    conf[:, 0] = 1.0
+    for budget in (R + 100, R + 1777, R + 5000):
+        s = W.ScheduleInput(torch.from_numpy(conf), [1, 20000], [100.0, 40.0], budget, max_tokens=20000)
+        for mode in MODES:
+            H.check_schedule(s, mode, topk=1500)
+    # continuous values, cap well below half of the candidates
+    conf = rng.uniform(0.2, 1.0, size=(1024, 16)).astype(np.float32)
+    s = W.ScheduleInput(torch.from_numpy(conf), [1, 4000, 20000], [90.0, 60.0, 10.0], 1024 + 3000, max_tokens=20000)
+    for mode in MODES:
+        H.check_schedule(s, mode, topk=2999)
+
+
 def test_host_side_errors():
     prof = B.Profile([1, 8], [2.0, 1.0], 8)
     conf = torch.rand(4, 4, device="cuda")
