@@ -120,6 +120,27 @@ def schedule(conf, table, budget_tokens: int, mode: int = MODE_EARLY_STOP, topk_
                           info.status, info.tau, info.theta, path)
 
 
+def schedule_async(conf, table, budget_tokens: int, state: np.ndarray, draft_len=None) -> ScheduleResult:
+    """One step of the asynchronous top-K scheduler; `state` (int32[3] = step, K slot 0, K slot 1)
+    is updated in place."""
+    conf = np.ascontiguousarray(conf, dtype=np.float32)
+    R, gamma = conf.shape
+    table = np.ascontiguousarray(table, dtype=np.float64)
+    dl = None if draft_len is None else np.ascontiguousarray(draft_len, dtype=np.int32)
+    assert state.dtype == np.int32 and state.size >= 3 and state.flags.c_contiguous
+    out_len = np.zeros(R, dtype=np.int32)
+    surv = np.zeros((R, max(gamma, 1)), dtype=np.float32)[:, :gamma].copy()
+    exp_len = np.zeros(R, dtype=np.float32)
+    info = _SchedInfo()
+    rc = lib().orc_schedule_async(_p(conf), _p(dl), C.c_int(R), C.c_int(gamma), C.c_int(budget_tokens),
+                                  _p(table), C.c_int(len(table) - 1), _p(state), _p(out_len), _p(surv),
+                                  _p(exp_len), C.byref(info))
+    if rc != 0:
+        raise ValueError(f"orc_schedule_async failed ({rc})")
+    return ScheduleResult(out_len, surv, exp_len, info.B, info.n_admitted, info.n_candidates,
+                          info.status, info.tau, info.theta, np.empty(0))
+
+
 def schedule_bruteforce(conf, table, budget_tokens: int, draft_len=None):
     conf = np.ascontiguousarray(conf, dtype=np.float32)
     R, gamma = conf.shape

@@ -254,6 +254,39 @@ int orc_schedule(const float* conf, const int32_t* draft_len, int R, int gamma,
 }
 
 /*
+ * Asynchronous scheduling (Section 4.2, "Hardware-Aware Prefix Scheduler in Practice").
+ * The capacity K used at step t is the admission count found by the unconstrained (no break)
+ * search on the confidences of step t-2; the candidates admitted at step t are the K most
+ * confident ones by the CURRENT survival products (dynamic top-K), still under the token cap.
+ * state = {t, K slot 0, K slot 1}: slot t mod 2 holds the K of step t-2 until this call
+ * overwrites it with the K found on the current confidences (used at step t+2).
+ * Reading: the first two steps use the K values the caller put into the slots.
+ */
+int orc_schedule_async(const float* conf, const int32_t* draft_len, int R, int gamma,
+                       int budget_tokens, const double* table, int max_tokens, int32_t* state,
+                       int32_t* out_len, float* out_survival, float* out_expected_len,
+                       orc_sched_info_t* info)
+{
+    int32_t* scratch = (int32_t*)malloc((size_t)R * sizeof(int32_t));
+    if (!scratch) return -2;
+    orc_sched_info_t ginfo;
+    /* capacity for step t+2: unconstrained global search on the current confidences */
+    int rc = orc_schedule(conf, draft_len, R, gamma, budget_tokens, ORC_MODE_GLOBAL, 0, table, max_tokens,
+                          scratch, NULL, NULL, &ginfo, NULL);
+    free(scratch);
+    if (rc != 0) return rc;
+    const int slot = 1 + (state[0] & 1);
+    const int K_use = state[slot];
+    /* admission at step t: top-K by current scores with the capacity decided two steps ago */
+    rc = orc_schedule(conf, draft_len, R, gamma, budget_tokens, ORC_MODE_TOPK, K_use < 0 ? 0 : K_use, table,
+                      max_tokens, out_len, out_survival, out_expected_len, info, NULL);
+    if (rc != 0) return rc;
+    state[slot] = ginfo.n_admitted;
+    state[0] += 1;
+    return 0;
+}
+
+/*
  * Exhaustive companion for tiny batches: every schedule l in {0..gamma}^R whose
  * positions are all candidates (a > 0, j < draft_len) and whose admitted count
  * is within the cap; Theta(l) from the same integer tau and the same table.

@@ -212,3 +212,30 @@ def test_draft_len_and_confidence_sanitising():
     np.testing.assert_allclose(res.expected_len, [1 + 0.9 + 0.81, 1.8, 2.0], rtol=1e-6)
     # tau counts one token per request plus the admitted survival mass
     assert res.tau == pytest.approx(3 + 0.9 + 0.81 + 0.8 + 1.0, rel=1e-6)
+
+
+def test_async_topk_uses_the_capacity_of_two_steps_earlier():
+    # Section 4.2: K at step t comes from the no-break search on the confidences of step t-2,
+    # the ranking from the current confidences.  Tiny batches: the capacity is checked against the
+    # exhaustive optimum, the admitted set against an independent top-K by sorting.
+    rng = np.random.default_rng(21)
+    R, gamma, budget = 3, 4, 12
+    table = np.array([0, 9.0, 8.8, 8.5, 8.0, 7.2, 6.5, 5.0, 4.9, 4.8, 3.0, 2.0, 1.0, 0.5])
+    K0 = 2
+    state = np.array([0, K0, K0], dtype=np.int32)
+    confs = [rng.uniform(0.3, 1.0, size=(R, gamma)).astype(np.float32) for _ in range(7)]
+    optimal_counts = []
+    for t, conf in enumerate(confs):
+        _, best_B, _ = oracle.schedule_bruteforce(conf, table, budget)
+        optimal_counts.append(best_B - R)
+        res = oracle.schedule_async(conf, table, budget, state)
+        K_expected = K0 if t < 2 else optimal_counts[t - 2]
+        assert res.n_admitted == min(K_expected, budget - R, R * gamma)
+        surv = np.cumprod(conf, axis=1, dtype=np.float32)
+        rr, jj = np.meshgrid(np.arange(R), np.arange(gamma), indexing="ij")
+        order = np.lexsort((rr.ravel(), jj.ravel(), -surv.ravel().astype(np.float64)))
+        want = np.bincount(rr.ravel()[order[: res.n_admitted]], minlength=R)
+        np.testing.assert_array_equal(res.lengths, want)
+        assert state[0] == t + 1
+    # after the loop the two slots hold the capacities found on the last two steps
+    assert sorted(state[1:3].tolist()) == sorted(optimal_counts[-2:])
