@@ -43,6 +43,8 @@ NCU_TRAFFIC_RATIO = {"cfg4": 1.0135, "cfg5": 1.0165}
 
 # ----------------------------------------------------------------------------- workloads ----
 REQUESTS_OVERRIDE = 0
+ASYNC_TOPK = False
+CUDA_GRAPH = False
 
 
 def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=False):
@@ -68,6 +70,7 @@ def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=Fal
 
     lengths = None
     prof = None
+    steady_K = 0
     if sched is not None:
         # the schedule is fixed by the confidences: run it once to size the logits
         if oracle_schedule:
@@ -81,10 +84,14 @@ def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=Fal
             R, gamma = sched.conf.shape
             out_len = torch.zeros(R, dtype=torch.int32, device=device)
             ws = B.workspace(B.dspark_schedule_workspace_bytes(R, gamma))
-            B.dspark_schedule(prof, sched.conf, sched.budget_tokens, B.DSPARK_SCHED_EARLY_STOP, out_len=out_len,
+            # asynchronous scheduling with constant confidences settles on the global optimum as its capacity
+            mode = B.DSPARK_SCHED_GLOBAL if ASYNC_TOPK else B.DSPARK_SCHED_EARLY_STOP
+            info = torch.zeros(32, dtype=torch.uint8, device=device)
+            B.dspark_schedule(prof, sched.conf, sched.budget_tokens, mode, out_len=out_len, out_info=info,
                               workspace=ws)
             torch.cuda.synchronize()
             lengths = out_len.cpu()
+            steady_K = B.read_sched_info(info).n_admitted
 
     def one(k):
         from paper_2607_05147_b200.replicas import rank_seed
@@ -108,7 +115,7 @@ def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=Fal
         n_sets = max(2, min(8, -(-4 * L2_BYTES // stream_b)))
     for k in range(1, n_sets):
         batches.append(one(k))
-    return dict(name=name, desc=desc, sched=sched, prof=prof, batches=batches, greedy=greedy)
+    return dict(name=name, desc=desc, sched=sched, prof=prof, batches=batches, greedy=greedy, steady_K=steady_K)
 
 
 class Step:
@@ -130,15 +137,38 @@ class Step:
             self.out_len = torch.zeros(R, dtype=torch.int32, device=device)
             self.offsets = torch.zeros(R + 1, dtype=torch.int32, device=device)
             self.sws = B.workspace(B.dspark_schedule_workspace_bytes(R, gamma))
+            if ASYNC_TOPK:
+                self.state = torch.zeros(4, dtype=torch.int32, device=device)
+                B.dspark_async_state_init(self.state, wl["steady_K"])
+        self.graphs = {}
         self.launches_per_step = (2 if self.sched is not None else 0) + (2 if wl["greedy"] else 4)
 
     def run(self, batch, conf=None):
+        """One step; with --cuda-graph the step of every resident batch is captured once and replayed."""
+        if CUDA_GRAPH and conf is None:
+            g = self.graphs.get(id(batch))
+            if g is None:
+                self._launch(batch, None)                      # eager warm-up outside the capture
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    self._launch(batch, None)
+                self.graphs[id(batch)] = g
+            g.replay()
+            return
+        self._launch(batch, conf)
+
+    def _launch(self, batch, conf):
         B = self.B
         offsets = batch.row_offsets
         if self.sched is not None:
-            B.dspark_schedule(self.wl["prof"], self.sched.conf if conf is None else conf, self.sched.budget_tokens,
-                              B.DSPARK_SCHED_EARLY_STOP, out_len=self.out_len, out_row_offsets=self.offsets,
-                              workspace=self.sws)
+            c = self.sched.conf if conf is None else conf
+            if ASYNC_TOPK:
+                B.dspark_schedule_async(self.wl["prof"], c, self.sched.budget_tokens, self.state,
+                                        out_len=self.out_len, out_row_offsets=self.offsets, workspace=self.sws)
+            else:
+                B.dspark_schedule(self.wl["prof"], c, self.sched.budget_tokens, B.DSPARK_SCHED_EARLY_STOP,
+                                  out_len=self.out_len, out_row_offsets=self.offsets, workspace=self.sws)
             offsets = self.offsets            # the verifier reads the schedule's offsets from device memory
         if self.wl["greedy"]:
             B.dspark_verify_greedy(batch.target, offsets, batch.draft_tokens, accepted_len=self.acc,
@@ -289,14 +319,19 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--all-workloads", action="store_true", help="also time the other V=129280 configurations")
+    ap.add_argument("--async-topk", action="store_true",
+                    help="schedule with dspark_schedule_async (capacity from two steps earlier, Section 4.2)")
+    ap.add_argument("--cuda-graph", action="store_true",
+                    help="capture the step (schedule -> verify) in CUDA graphs and time their replay")
     ap.add_argument("--requests", type=int, default=0,
                     help="override the request count of cfg2 / cfg4 (smaller cases for profiler captures)")
     ap.add_argument("--quick", action="store_true",
                     help="timed steps only (no clock probe, per-kernel timing, e2e or CPU legs): for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    global REQUESTS_OVERRIDE
+    global REQUESTS_OVERRIDE, ASYNC_TOPK, CUDA_GRAPH
     REQUESTS_OVERRIDE = args.requests
+    ASYNC_TOPK, CUDA_GRAPH = args.async_topk, args.cuda_graph
 
     from paper_2607_05147_b200 import replicas
     rank, local_rank, world = replicas.env_ranks()
@@ -478,6 +513,9 @@ def main():
                        "logit_dtype": "fp32" if wl["greedy"] else "bf16",
                        "l2": f"inputs larger than L2: {res['n_sets']} distinct batches rotated "
                              f"({res['n_sets'] * stream_bytes / 1e6:.0f} MB of logits)",
+                       "scheduler": ("async top-K, capacity from two steps earlier" if ASYNC_TOPK else "early stop")
+                       if wl["sched"] is not None else None,
+                       "launch": "CUDA graph replay" if CUDA_GRAPH else "stream launches",
                        "parallelism": "replicas only (one engine per GPU, no collective)"},
             "step_algorithmic_bytes": all_bytes,
             "step_effective_gbs": all_bytes / (ms / args.steps * 1e-3) / 1e9,

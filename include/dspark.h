@@ -121,6 +121,28 @@ int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32
                     float* out_expected_len, dspark_sched_info_t* out_info,
                     void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------
+ * dspark_schedule_async -- the scheduler as deployed (Section 4.2): the engine must know the
+ * batch size of the next step before the current one ends, so the capacity K (how many draft
+ * tokens are admitted in total) is taken from the unconstrained, no-break search over the
+ * confidences of TWO STEPS EARLIER, while the candidates themselves are ranked by their current
+ * survival products (a dynamic top-K, still under the token budget).
+ *
+ * state: device int32[4], owned by the caller and kept between steps: {step t, K slot 0,
+ * K slot 1, reserved}.  Each call reads the K stored by step t-2 (slot t mod 2), admits that many
+ * of the most confident current candidates, overwrites the slot with the admission count of the
+ * global search on the CURRENT confidences (to be used at step t+2) and increments t -- all on the
+ * device, so a captured CUDA graph of schedule -> verify can simply be replayed step after step.
+ * dspark_async_state_init sets t = 0 and both slots to initial_K (used by the first two steps).
+ * All other arguments, outputs, limits and errors are those of dspark_schedule.
+ */
+int dspark_async_state_init(int32_t* state, int initial_K, void* stream);
+int dspark_schedule_async(const dspark_profile_t* prof, const float* conf, const int32_t* draft_len,
+                          int R, int gamma, int budget_tokens, int32_t* state,
+                          int32_t* out_len, int32_t* out_row_offsets, float* out_survival,
+                          float* out_expected_len, dspark_sched_info_t* out_info,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
 /* row_offsets[0..R] = exclusive scan of (lengths[r] + 1): the flat ragged layout of
  * Section 4.3 (all verified tokens of all requests flattened).  Device in, device out. */
 int dspark_build_offsets(const int32_t* lengths, int R, int32_t* row_offsets, void* stream);

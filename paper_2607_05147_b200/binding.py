@@ -27,6 +27,7 @@ DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF = 16, 32, 64
 EXPORTS = [
     "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",
     "dspark_schedule_workspace_bytes", "dspark_schedule", "dspark_build_offsets",
+    "dspark_schedule_async", "dspark_async_state_init",
     "dspark_verify_workspace_bytes", "dspark_verify_greedy", "dspark_verify", "dspark_uniforms",
     "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
@@ -61,6 +62,8 @@ def lib() -> C.CDLL:
         L.dspark_schedule_workspace_bytes.restype = sz
         L.dspark_schedule.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_build_offsets.argtypes = [vp, i32, vp, vp]
+        L.dspark_async_state_init.argtypes = [vp, i32, vp]
+        L.dspark_schedule_async.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_verify_workspace_bytes.argtypes = [i32, i32, i32]
         L.dspark_verify_workspace_bytes.restype = sz
         L.dspark_verify_greedy.argtypes = [vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -173,6 +176,33 @@ def dspark_schedule(prof: Profile, conf: torch.Tensor, budget_tokens: int, mode:
                                _dev(out_info, "out_info", torch.uint8), _dev(workspace, "workspace"),
                                workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_schedule")
+
+
+def dspark_async_state_init(state: torch.Tensor, initial_K: int) -> None:
+    """state: CUDA int32[4] kept by the caller between steps."""
+    if state.numel() < 4:
+        raise DsparkError("state must hold 4 int32")
+    _check(lib().dspark_async_state_init(_dev(state, "state", torch.int32), int(initial_K), _stream()),
+           "dspark_async_state_init")
+
+
+def dspark_schedule_async(prof: Profile, conf: torch.Tensor, budget_tokens: int, state: torch.Tensor,
+                          draft_len: Optional[torch.Tensor] = None, *, out_len: torch.Tensor,
+                          out_row_offsets: Optional[torch.Tensor] = None, out_survival: Optional[torch.Tensor] = None,
+                          out_expected_len: Optional[torch.Tensor] = None, out_info: Optional[torch.Tensor] = None,
+                          workspace: torch.Tensor) -> None:
+    if conf.dim() != 2 or not conf.is_contiguous():
+        raise DsparkError("conf must be a contiguous [R, gamma] tensor")
+    R, gamma = conf.shape
+    rc = lib().dspark_schedule_async(prof.handle, _dev(conf, "conf", torch.float32),
+                                     _dev(draft_len, "draft_len", torch.int32), R, gamma, int(budget_tokens),
+                                     _dev(state, "state", torch.int32), _dev(out_len, "out_len", torch.int32),
+                                     _dev(out_row_offsets, "out_row_offsets", torch.int32),
+                                     _dev(out_survival, "out_survival", torch.float32),
+                                     _dev(out_expected_len, "out_expected_len", torch.float32),
+                                     _dev(out_info, "out_info", torch.uint8), _dev(workspace, "workspace"),
+                                     workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_schedule_async")
 
 
 def read_sched_info(out_info: torch.Tensor) -> SchedInfo:

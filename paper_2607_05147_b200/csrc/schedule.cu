@@ -22,6 +22,7 @@ namespace dspark {
 constexpr int kSchedThreads = 1024;
 constexpr int kPrepThreads = 128;
 constexpr int kSmemLenCap = 4096;
+constexpr int kModeAsync = 3;                 // internal: global search for the next K, top-K with the stored K
 
 struct SchedParams {
     const float* conf;
@@ -43,6 +44,7 @@ struct SchedParams {
     int32_t* cnt;                   // [R] candidates of request r (bit 30: a confidence was clamped)
     unsigned long long* t_by_rank;  // [N+1] T_i
     int32_t* owner_by_rank;         // [N+1] request of the i-th admitted candidate
+    int32_t* async_state;           // asynchronous mode: {step, K slot 0, K slot 1} (caller-owned, device)
     int32_t* cand;                  // [n_tiles*32] entry indices of the candidates worth ranking
     int* ticket;                    // [0] finished rank CTAs, [1] number of entries in cand (select kernel)
 };
@@ -376,7 +378,7 @@ __device__ void sched_final_stage(const SchedParams& P)
             const int istar = (fb != 0x7fffffff) ? fb - 1 : (base + kSchedThreads < N ? base + kSchedThreads : N);
             if (valid && i == istar) { s_T_best = Ti; s_theta_best = theta_i; s_istar = i; }
             if (fb != 0x7fffffff && tid == 0) s_done = 1;
-        } else if (P.mode == DSPARK_SCHED_GLOBAL) {
+        } else if (P.mode == DSPARK_SCHED_GLOBAL || P.mode == kModeAsync) {
             // CTA-wide argmax of Theta with the smallest i on ties; NaN never wins
             double bt = (valid && theta_i == theta_i) ? theta_i : -INFINITY;
             int bi = valid ? i : 0x7fffffff;
@@ -412,6 +414,24 @@ __device__ void sched_final_stage(const SchedParams& P)
         if (s_done) break;
     }
     __syncthreads();
+    if (P.mode == kModeAsync) {
+        // Section 4.2: the admission count found on the current confidences becomes the capacity of
+        // the step after next; this step admits the top K by current scores with the capacity that
+        // was stored two steps ago.
+        if (tid == 0) {
+            const int slot = 1 + (P.async_state[0] & 1);
+            int K = P.async_state[slot];
+            K = K < 0 ? 0 : K;
+            const int use = N < K ? N : K;
+            P.async_state[slot] = s_istar;
+            P.async_state[0] += 1;
+            s_istar = use;
+            s_T_best = use > 0 ? P.t_by_rank[use] : T0;
+            const int B = R + use;
+            s_theta_best = __dmul_rn(__ull2double_rn(s_T_best), P.table[B < mt ? B : mt]);
+        }
+        __syncthreads();
+    }
     const int istar = s_istar;
 
     // ---- lengths l*_r = admitted candidates of request r -----------------------------------
@@ -528,15 +548,13 @@ size_t dspark_schedule_workspace_bytes(int R, int gamma)
     return sched_geom(R, gamma).total;
 }
 
-int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32_t* draft_len,
-                    int R, int gamma, int budget_tokens, int mode, int topk_K,
-                    int32_t* out_len, int32_t* out_row_offsets, float* out_survival,
-                    float* out_expected_len, dspark_sched_info_t* out_info,
-                    void* workspace, size_t workspace_bytes, void* stream)
+static int schedule_launch(const dspark_profile_t* prof, const float* conf, const int32_t* draft_len,
+                           int R, int gamma, int budget_tokens, int mode, int topk_K, int32_t* async_state,
+                           int32_t* out_len, int32_t* out_row_offsets, float* out_survival,
+                           float* out_expected_len, dspark_sched_info_t* out_info,
+                           void* workspace, size_t workspace_bytes, void* stream)
 {
     if (!prof || !out_len || (!conf && gamma > 0)) return DSPARK_ERR_INVALID_ARG;
-    if (mode != DSPARK_SCHED_EARLY_STOP && mode != DSPARK_SCHED_GLOBAL && mode != DSPARK_SCHED_TOPK)
-        return DSPARK_ERR_INVALID_ARG;
     if (R < 1 || gamma < 0) return DSPARK_ERR_INVALID_ARG;
     if (R > (1 << 20) || gamma > 4096 || (long long)R * gamma > (1 << 20)) return DSPARK_ERR_SHAPE;
     const SchedGeom g = sched_geom(R, gamma);
@@ -552,6 +570,7 @@ int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32
     P.table = table; P.max_tokens = max_tokens;
     P.out_len = out_len; P.out_offsets = out_row_offsets; P.out_surv = out_survival;
     P.out_exp = out_expected_len; P.info = out_info;
+    P.async_state = async_state;
     P.gpad = g.gpad; P.seg = g.seg; P.n_tiles = g.n_tiles; P.R_pad = g.R_pad;
     P.akey = (uint32_t*)(ws + g.akey);
     P.pfix = (unsigned long long*)(ws + g.pfix);
@@ -596,6 +615,44 @@ int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32
         launch_pdl(sched_final_only_kernel, dim3(1), dim3(kSchedThreads), 0, s, P);
     }
     return launch_status();
+}
+
+int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32_t* draft_len,
+                    int R, int gamma, int budget_tokens, int mode, int topk_K,
+                    int32_t* out_len, int32_t* out_row_offsets, float* out_survival,
+                    float* out_expected_len, dspark_sched_info_t* out_info,
+                    void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (mode != DSPARK_SCHED_EARLY_STOP && mode != DSPARK_SCHED_GLOBAL && mode != DSPARK_SCHED_TOPK)
+        return DSPARK_ERR_INVALID_ARG;
+    return schedule_launch(prof, conf, draft_len, R, gamma, budget_tokens, mode, topk_K, nullptr, out_len,
+                           out_row_offsets, out_survival, out_expected_len, out_info, workspace, workspace_bytes,
+                           stream);
+}
+
+__global__ void async_state_init_kernel(int32_t* state, int K)
+{
+    pdl_wait();
+    if (threadIdx.x == 0) { state[0] = 0; state[1] = K; state[2] = K; state[3] = 0; }
+}
+
+int dspark_async_state_init(int32_t* state, int initial_K, void* stream)
+{
+    if (!state || initial_K < 0) return DSPARK_ERR_INVALID_ARG;
+    launch_pdl(async_state_init_kernel, dim3(1), dim3(32), 0, (cudaStream_t)stream, state, initial_K);
+    return launch_status();
+}
+
+int dspark_schedule_async(const dspark_profile_t* prof, const float* conf, const int32_t* draft_len,
+                          int R, int gamma, int budget_tokens, int32_t* state,
+                          int32_t* out_len, int32_t* out_row_offsets, float* out_survival,
+                          float* out_expected_len, dspark_sched_info_t* out_info,
+                          void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!state) return DSPARK_ERR_INVALID_ARG;
+    return schedule_launch(prof, conf, draft_len, R, gamma, budget_tokens, kModeAsync, 0, state, out_len,
+                           out_row_offsets, out_survival, out_expected_len, out_info, workspace, workspace_bytes,
+                           stream);
 }
 
 int dspark_build_offsets(const int32_t* lengths, int R, int32_t* row_offsets, void* stream)
