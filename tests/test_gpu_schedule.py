@@ -104,6 +104,22 @@ def test_selection_path_with_mass_ties():
         H.check_schedule(s, mode, topk=2999)
 
 
+@pytest.mark.parametrize("R,gamma", [(37, 40), (300, 64), (130, 100), (9, 33)])
+def test_blocks_longer_than_a_tile(R, gamma):
+    # gamma > 32: a request spans several 32-entry tiles
+    rng = np.random.default_rng(R * gamma)
+    conf = rng.uniform(0.55, 1.0, size=(R, gamma)).astype(np.float32)
+    conf[rng.random((R, gamma)) < 0.05] = 1.0
+    conf[rng.random((R, gamma)) < 0.01] = 0.0
+    toks = [1, R, 2 * R, 4 * R, R * (gamma + 1)]
+    s = W.ScheduleInput(torch.from_numpy(conf), toks, [100.0, 90.0, 70.0, 45.0, 5.0],
+                        budget_tokens=R * (gamma // 2), max_tokens=R * (gamma + 1))
+    for mode in MODES:
+        H.check_schedule(s, mode, topk=R * 7)
+    dl = rng.integers(0, gamma + 1, size=R).astype(np.int32)
+    H.check_schedule(s, B.DSPARK_SCHED_EARLY_STOP, draft_len=dl)
+
+
 def test_host_side_errors():
     prof = B.Profile([1, 8], [2.0, 1.0], 8)
     conf = torch.rand(4, 4, device="cuda")

@@ -51,6 +51,12 @@ def test_odd_vocabularies_and_dtypes(V, dtype):
         B.dspark_set_stream_path(0)
 
 
+def test_very_large_vocabulary_and_many_requests():
+    H.check_greedy(W.greedy_batch(torch.tensor([1, 0, 2]), 1_000_003, 8, "cuda", tie_frac=0.5, perturb=0.3))
+    # thousands of requests that verify only their bonus token
+    H.check_greedy(W.greedy_batch(torch.zeros(5000, dtype=torch.int64), 4096, 9, "cuda", perturb=0.0))
+
+
 def test_padded_rows_and_unaligned_views():
     lengths = torch.tensor([2, 4, 0, 1])
     base = W.greedy_batch(lengths, 3000, 5, "cuda", perturb=0.2)

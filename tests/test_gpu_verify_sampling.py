@@ -73,6 +73,16 @@ def test_odd_vocabularies_dtypes_and_paths(V, dtype):
     np.testing.assert_array_equal(g["acc"], g1["acc"])
 
 
+@pytest.mark.parametrize("dtype,V", [(torch.bfloat16, 600_011), (torch.float32, 300_000), (torch.bfloat16, 1_100_000)])
+def test_very_large_vocabularies(dtype, V):
+    # more than 256 statistics / residual blocks per row: the inverse CDF walks memory instead of registers
+    lengths = torch.tensor([2, 0, 3, 1, 0, 2])
+    batch = W.sampling_batch(lengths, V, 5, "cuda", dtype=dtype, temperature=1.1, draft_noise=1.5, verify_seed=V % 97)
+    g, o, mism = H.check_sampling(batch)
+    assert mism == 0
+    assert (g["acc"] < lengths.numpy()).any() and (g["acc"] == lengths.numpy()).any()   # both kinds of draw
+
+
 def test_compact_and_block_layouts_agree():
     lengths = torch.tensor([2, 5, 0, 3, 1, 7])
     a = W.sampling_batch(lengths, 20000, 3, "cuda", verify_seed=5)
