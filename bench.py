@@ -45,6 +45,7 @@ NCU_TRAFFIC_RATIO = {"cfg4": 1.0135, "cfg5": 1.0165}
 REQUESTS_OVERRIDE = 0
 ASYNC_TOPK = False
 CUDA_GRAPH = False
+OVERLAP = False
 
 
 def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=False):
@@ -141,6 +142,15 @@ class Step:
                 self.state = torch.zeros(4, dtype=torch.int32, device=device)
                 B.dspark_async_state_init(self.state, wl["steady_K"])
         self.graphs = {}
+        if OVERLAP and self.sched is not None:
+            # two sets of scheduler outputs: step t+1 is scheduled while step t is still being verified
+            self.side = torch.cuda.Stream(device=device)
+            self.off2 = [self.offsets, torch.zeros_like(self.offsets)]
+            self.len2 = [self.out_len, torch.zeros_like(self.out_len)]
+            self.sched_done = [torch.cuda.Event(), torch.cuda.Event()]
+            self.verify_done = [torch.cuda.Event(), torch.cuda.Event()]
+            self.tick = 0
+            self.primed = False
         self.launches_per_step = (2 if self.sched is not None else 0) + (2 if wl["greedy"] else 4)
 
     def run(self, batch, conf=None):
@@ -158,8 +168,34 @@ class Step:
             return
         self._launch(batch, conf)
 
+    def _schedule_on_side_stream(self, k):
+        B = self.B
+        with torch.cuda.stream(self.side):
+            self.side.wait_event(self.verify_done[k])          # the verifier that last read this slot is done
+            B.dspark_schedule_async(self.wl["prof"], self.sched.conf, self.sched.budget_tokens, self.state,
+                                    out_len=self.len2[k], out_row_offsets=self.off2[k], workspace=self.sws)
+            self.sched_done[k].record(self.side)
+
+    def _launch_overlapped(self, batch):
+        B = self.B
+        main = torch.cuda.current_stream()
+        if not self.primed:
+            self.verify_done[0].record(main); self.verify_done[1].record(main)
+            self._schedule_on_side_stream(0)
+            self.primed = True
+        k = self.tick & 1
+        self._schedule_on_side_stream(k ^ 1)                    # next step's schedule runs beside this verify
+        main.wait_event(self.sched_done[k])
+        B.dspark_verify(batch.target, batch.draft, self.off2[k], batch.draft_tokens, batch.temperature, batch.seed,
+                        draft_row_start=batch.draft_row_start, accepted_len=self.acc, out_tokens=self.out,
+                        dev_status=self.status, workspace=self.ws, n_rows=self.n_rows)
+        self.verify_done[k].record(main)
+        self.tick += 1
+
     def _launch(self, batch, conf):
         B = self.B
+        if OVERLAP and self.sched is not None and conf is None:
+            return self._launch_overlapped(batch)
         offsets = batch.row_offsets
         if self.sched is not None:
             c = self.sched.conf if conf is None else conf
@@ -321,6 +357,9 @@ def main():
     ap.add_argument("--all-workloads", action="store_true", help="also time the other V=129280 configurations")
     ap.add_argument("--async-topk", action="store_true",
                     help="schedule with dspark_schedule_async (capacity from two steps earlier, Section 4.2)")
+    ap.add_argument("--overlap-schedule", action="store_true",
+                    help="with --async-topk: schedule step t+1 on a second stream while step t is verified "
+                         "(the asynchronous scheduler is off the critical path, Section 4.2)")
     ap.add_argument("--cuda-graph", action="store_true",
                     help="capture the step (schedule -> verify) in CUDA graphs and time their replay")
     ap.add_argument("--requests", type=int, default=0,
@@ -329,9 +368,12 @@ def main():
                     help="timed steps only (no clock probe, per-kernel timing, e2e or CPU legs): for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    global REQUESTS_OVERRIDE, ASYNC_TOPK, CUDA_GRAPH
+    global REQUESTS_OVERRIDE, ASYNC_TOPK, CUDA_GRAPH, OVERLAP
     REQUESTS_OVERRIDE = args.requests
     ASYNC_TOPK, CUDA_GRAPH = args.async_topk, args.cuda_graph
+    OVERLAP = args.overlap_schedule
+    if OVERLAP and (not ASYNC_TOPK or CUDA_GRAPH):
+        raise SystemExit("--overlap-schedule needs --async-topk and stream launches")
 
     from paper_2607_05147_b200 import replicas
     rank, local_rank, world = replicas.env_ranks()
@@ -515,7 +557,9 @@ def main():
                              f"({res['n_sets'] * stream_bytes / 1e6:.0f} MB of logits)",
                        "scheduler": ("async top-K, capacity from two steps earlier" if ASYNC_TOPK else "early stop")
                        if wl["sched"] is not None else None,
-                       "launch": "CUDA graph replay" if CUDA_GRAPH else "stream launches",
+                       "launch": "CUDA graph replay" if CUDA_GRAPH else
+                       ("stream launches, scheduler of step t+1 overlapped on a second stream" if OVERLAP
+                        else "stream launches"),
                        "parallelism": "replicas only (one engine per GPU, no collective)"},
             "step_algorithmic_bytes": all_bytes,
             "step_effective_gbs": all_bytes / (ms / args.steps * 1e-3) / 1e9,
