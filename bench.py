@@ -63,9 +63,14 @@ def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=Fal
         desc = "Long-block stress: 512 requests, V=129280, blocks of 32, budget 4096, bf16 sampling T=0.7"
     elif name == "cfg2":
         desc = "Sampling, moderate batch: 64 requests, V=129280, ragged k~U{1..8}, bf16, T=1"
+    elif name == "cfg2_fp32":
+        desc = "cfg2 with fp32 logits (fp32 sampling path): 64 requests, V=129280, ragged k~U{1..8}, T=1"
     elif name == "cfg4":
         greedy = True
         desc = "Large batch greedy: 1024 requests, V=129280, ragged k~U{0..8}, fp32"
+    elif name == "cfg4_bf16":
+        greedy = True
+        desc = "cfg4 with bf16 logits (bf16 greedy path): 1024 requests, V=129280, ragged k~U{0..8}"
     else:
         raise SystemExit(f"unknown workload {name}")
 
@@ -101,14 +106,16 @@ def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=Fal
             return W.sampling_batch(lengths, W.V_FULL, seed, device, temperature=1.0, draft_noise=1.0, verify_seed=2)
         if name == "cfg5":
             return W.sampling_batch(lengths, W.V_FULL, seed, device, temperature=0.7, draft_noise=2.0, verify_seed=4)
-        if name == "cfg2":
+        if name in ("cfg2", "cfg2_fp32"):
             g = torch.Generator(device="cpu"); g.manual_seed(1)
             ln = torch.randint(1, 9, (REQUESTS_OVERRIDE or 64,), generator=g)
-            return W.sampling_batch(ln, W.V_FULL, seed, device, temperature=1.0, draft_noise=1.0, verify_seed=1)
+            return W.sampling_batch(ln, W.V_FULL, seed, device, temperature=1.0, draft_noise=1.0, verify_seed=1,
+                                    dtype=torch.float32 if name == "cfg2_fp32" else torch.bfloat16)
         g = torch.Generator(device="cpu"); g.manual_seed(3)
         ln = torch.randint(0, 9, (REQUESTS_OVERRIDE or 1024,), generator=g)
         return W.greedy_batch(ln, W.V_FULL, seed, device, sigma=4.0, tie_frac=0.01,
-                              match_prob=[0.85 ** (j + 1) for j in range(8)])
+                              match_prob=[0.85 ** (j + 1) for j in range(8)],
+                              dtype=torch.bfloat16 if name == "cfg4_bf16" else torch.float32)
 
     batches = [one(0)]
     if n_sets is None:
@@ -352,7 +359,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg3",
+                    choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2_fp32", "cfg4_bf16"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--all-workloads", action="store_true", help="also time the other V=129280 configurations")
     ap.add_argument("--async-topk", action="store_true",
@@ -552,7 +560,7 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl["desc"], "name": wl["name"], "requests": b0.R, "rows_per_step": res["n_rows"],
                        "draft_rows_per_step": b0.n_rows - b0.R, "rejected_requests": res["n_rejected"],
-                       "logit_dtype": "fp32" if wl["greedy"] else "bf16",
+                       "logit_dtype": str(b0.target.dtype).replace("torch.", ""),
                        "l2": f"inputs larger than L2: {res['n_sets']} distinct batches rotated "
                              f"({res['n_sets'] * stream_bytes / 1e6:.0f} MB of logits)",
                        "scheduler": ("async top-K, capacity from two steps earlier" if ASYNC_TOPK else "early stop")
@@ -575,7 +583,7 @@ def main():
         }
         if args.all_workloads and world == 1:
             others = {}
-            for name in ["cfg2", "cfg3", "cfg4", "cfg5"]:
+            for name in ["cfg2", "cfg3", "cfg4", "cfg5", "cfg2_fp32", "cfg4_bf16"]:
                 if name == args.workload:
                     continue
                 del res, wl
