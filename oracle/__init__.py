@@ -22,6 +22,7 @@ F32, BF16 = 0, 1
 MODE_EARLY_STOP, MODE_GLOBAL, MODE_TOPK = 0, 1, 2
 ST_BAD_OFFSETS, ST_BAD_TOKEN, ST_BAD_ROW = 1, 2, 4
 ST_CONF_CLAMPED, ST_BUDGET_LT_R, ST_ALL_NEG_INF = 16, 32, 64
+ST_BAD_TEMPERATURE = 128
 
 
 def build(force: bool = False) -> str:
@@ -226,7 +227,8 @@ class VerifyResult:
 
 
 def verify(target, draft, row_offsets, draft_tokens, temperature: float, seed: int,
-           draft_row_start=None, eval_all: bool = True, n_threads: int = 1) -> VerifyResult:
+           draft_row_start=None, eval_all: bool = True, n_threads: int = 1, temperatures=None) -> VerifyResult:
+    """temperatures: optional float32[R], one temperature per request (overrides `temperature`)."""
     t, ts = _logits(target)
     d, ds = _logits(draft)
     if t.dtype != d.dtype:
@@ -243,9 +245,10 @@ def verify(target, draft, row_offsets, draft_tokens, temperature: float, seed: i
     am = np.full(n_rows, np.nan)
     tm = np.full(R, np.nan)
     st = np.zeros(R, dtype=np.int32)
+    temps = None if temperatures is None else np.ascontiguousarray(temperatures, dtype=np.float32)
     rc = lib().orc_verify(_p(t), _p(d), C.c_int(_dtype_code(t)), C.c_int64(ts), C.c_int64(ds),
                           C.c_int(t.shape[1]), _p(ro), _p(drs), _p(dt), C.c_int(R),
-                          C.c_double(temperature), C.c_uint64(seed), C.c_int(int(eval_all)),
+                          C.c_double(temperature), _p(temps), C.c_uint64(seed), C.c_int(int(eval_all)),
                           C.c_int(n_threads), _p(acc), _p(out), _p(p), _p(q), _p(am), _p(tm), _p(st))
     if rc != 0:
         raise ValueError("orc_verify rejected its arguments")

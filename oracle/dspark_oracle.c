@@ -34,6 +34,7 @@
 #define ORC_ST_CONF_CLAMPED 16
 #define ORC_ST_BUDGET_LT_R 32
 #define ORC_ST_ALL_NEG_INF 64
+#define ORC_ST_BAD_TEMPERATURE 128
 
 /* ------------------------------------------------------------------------ */
 /* Counter-based RNG.  The paper never names a generator; the reading taken  */
@@ -477,7 +478,7 @@ typedef struct {
     const void* target; const void* draft; int dtype;
     int64_t tstride, dstride; int V;
     const int32_t* row_offsets; const int64_t* draft_row_start; const int32_t* draft_tokens;
-    int R; double T; uint64_t seed; int eval_all;
+    int R; double T; const float* temps; uint64_t seed; int eval_all;
     int32_t* accepted_len; int32_t* out_tokens;
     double* p_tok; double* q_tok; double* accept_margin; double* token_margin;
     int32_t* status;
@@ -492,6 +493,8 @@ static void verify_request(const verify_job_t* J, int r)
     int32_t len = hi - lo - 1;
     int64_t drow0 = J->draft_row_start ? J->draft_row_start[r] : (int64_t)lo - (int64_t)r;
     int32_t st = 0;
+    /* per-request temperature (requests of one batch may use different sampling settings) */
+    const double T = J->temps ? (double)J->temps[r] : J->T;
     for (int32_t i = lo; i < hi; ++i) {
         J->out_tokens[i] = -1;
         if (J->p_tok) J->p_tok[i] = NAN;
@@ -502,18 +505,19 @@ static void verify_request(const verify_job_t* J, int r)
         int32_t d = J->draft_tokens[lo + j];
         if (d < 0 || d >= J->V) st |= ORC_ST_BAD_TOKEN;
     }
+    if (!(T > 0.0) || !isfinite(T)) st |= ORC_ST_BAD_TEMPERATURE;
     if (st) { J->status[r] = st; J->accepted_len[r] = 0; return; }
 
     int32_t n = len;           /* first rejected position, or len */
     for (int32_t j = 0; j < len; ++j) {
         if (n < len && !J->eval_all) break;   /* verification stops at the first rejection */
         double mp, Zp, mq, Zq;
-        int bad = row_softmax_stats(J->target, J->dtype, lo + j, J->tstride, J->V, J->T, &mp, &Zp);
-        bad |= row_softmax_stats(J->draft, J->dtype, drow0 + j, J->dstride, J->V, J->T, &mq, &Zq);
+        int bad = row_softmax_stats(J->target, J->dtype, lo + j, J->tstride, J->V, T, &mp, &Zp);
+        bad |= row_softmax_stats(J->draft, J->dtype, drow0 + j, J->dstride, J->V, T, &mq, &Zq);
         if (bad) { st |= ORC_ST_BAD_ROW; break; }
         int32_t d = J->draft_tokens[lo + j];
-        double p = prob_at(J->target, J->dtype, lo + j, J->tstride, d, J->T, mp, Zp);
-        double q = prob_at(J->draft, J->dtype, drow0 + j, J->dstride, d, J->T, mq, Zq);
+        double p = prob_at(J->target, J->dtype, lo + j, J->tstride, d, T, mp, Zp);
+        double q = prob_at(J->draft, J->dtype, drow0 + j, J->dstride, d, T, mq, Zq);
         if (J->p_tok) J->p_tok[lo + j] = p;
         if (J->q_tok) J->q_tok[lo + j] = q;
         float ua, ur;
@@ -533,18 +537,18 @@ static void verify_request(const verify_job_t* J, int r)
     int32_t tok = -1;
     double margin = 0.0;
     double mp, Zp;
-    if (row_softmax_stats(J->target, J->dtype, lo + n, J->tstride, J->V, J->T, &mp, &Zp)) {
+    if (row_softmax_stats(J->target, J->dtype, lo + n, J->tstride, J->V, T, &mp, &Zp)) {
         J->status[r] = ORC_ST_BAD_ROW; J->accepted_len[r] = 0; return;
     }
     int resampled = 0;
     if (n < len) {
         /* residual norm(max(0, p - q)) at the rejected position */
         double mq, Zq;
-        row_softmax_stats(J->draft, J->dtype, drow0 + n, J->dstride, J->V, J->T, &mq, &Zq);
+        row_softmax_stats(J->draft, J->dtype, drow0 + n, J->dstride, J->V, T, &mq, &Zq);
         double W = 0.0;
         for (int v = 0; v < J->V; ++v) {
-            double pv = prob_at(J->target, J->dtype, lo + n, J->tstride, v, J->T, mp, Zp);
-            double qv = prob_at(J->draft, J->dtype, drow0 + n, J->dstride, v, J->T, mq, Zq);
+            double pv = prob_at(J->target, J->dtype, lo + n, J->tstride, v, T, mp, Zp);
+            double qv = prob_at(J->draft, J->dtype, drow0 + n, J->dstride, v, T, mq, Zq);
             double w = pv - qv;
             if (w > 0.0) W += w;
         }
@@ -553,8 +557,8 @@ static void verify_request(const verify_job_t* J, int r)
             double cum = 0.0;
             int32_t last_pos = -1;
             for (int v = 0; v < J->V; ++v) {
-                double pv = prob_at(J->target, J->dtype, lo + n, J->tstride, v, J->T, mp, Zp);
-                double qv = prob_at(J->draft, J->dtype, drow0 + n, J->dstride, v, J->T, mq, Zq);
+                double pv = prob_at(J->target, J->dtype, lo + n, J->tstride, v, T, mp, Zp);
+                double qv = prob_at(J->draft, J->dtype, drow0 + n, J->dstride, v, T, mq, Zq);
                 double w = pv - qv;
                 if (!(w > 0.0)) continue;
                 double prev = cum;
@@ -573,7 +577,7 @@ static void verify_request(const verify_job_t* J, int r)
     }
     if (!resampled) {
         /* bonus token from p of row n (also the fallback when the residual is empty) */
-        tok = sample_from_p(J->target, J->dtype, lo + n, J->tstride, J->V, J->T, mp, Zp, (double)ur, &margin);
+        tok = sample_from_p(J->target, J->dtype, lo + n, J->tstride, J->V, T, mp, Zp, (double)ur, &margin);
     }
     for (int32_t j = 0; j < n; ++j) J->out_tokens[lo + j] = J->draft_tokens[lo + j];
     J->out_tokens[lo + n] = tok;
@@ -598,18 +602,19 @@ static void* verify_worker(void* arg)
 int orc_verify(const void* target, const void* draft, int dtype,
                int64_t target_row_stride, int64_t draft_row_stride, int V,
                const int32_t* row_offsets, const int64_t* draft_row_start,
-               const int32_t* draft_tokens, int R, double temperature, uint64_t seed,
-               int eval_all, int n_threads,
+               const int32_t* draft_tokens, int R, double temperature, const float* temperatures,
+               uint64_t seed, int eval_all, int n_threads,
                int32_t* accepted_len, int32_t* out_tokens,
                double* p_tok, double* q_tok, double* accept_margin, double* token_margin,
                int32_t* status)
 {
-    if (R <= 0 || V <= 0 || !(temperature > 0.0) || !isfinite(temperature)) return -1;
+    if (R <= 0 || V <= 0) return -1;
+    if (!temperatures && (!(temperature > 0.0) || !isfinite(temperature))) return -1;
     if (n_threads < 1) n_threads = 1;
     if (n_threads > R) n_threads = R;
     if (n_threads > 256) n_threads = 256;
     verify_job_t base = { target, draft, dtype, target_row_stride, draft_row_stride, V,
-                          row_offsets, draft_row_start, draft_tokens, R, temperature, seed, eval_all,
+                          row_offsets, draft_row_start, draft_tokens, R, temperature, temperatures, seed, eval_all,
                           accepted_len, out_tokens, p_tok, q_tok, accept_margin, token_margin,
                           status, 0, R };
     if (n_threads == 1) { verify_worker(&base); return 0; }

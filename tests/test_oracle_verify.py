@@ -281,3 +281,38 @@ def test_threads_and_eval_all_do_not_change_results():
     # non-compact draft layout: rows of request r start at r * L
     c = oracle.verify(x, y, ro, toks, 0.9, seed=4, draft_row_start=np.arange(R) * L)
     np.testing.assert_array_equal(a.out_tokens, c.out_tokens)
+
+
+def test_per_request_temperatures():
+    # every request carries its own temperature: each one's first emitted token must follow
+    # softmax(target / T_r), and the acceptance rate 1 - TV at that temperature
+    rng = np.random.default_rng(12)
+    V, n = 6, 90_000
+    temps = np.array([0.6, 1.0, 1.7], dtype=np.float32)
+    tl = rng.normal(0, 1.5, V).astype(np.float32)
+    ql = rng.normal(0, 1.5, V).astype(np.float32)
+    R = 3 * n
+    Tr = np.tile(temps, n)
+    target = np.broadcast_to(tl, (2 * R, V)); draft = np.broadcast_to(ql, (R, V))
+    ro = (2 * np.arange(R + 1)).astype(np.int32)
+    toks = np.zeros(2 * R, np.int32)
+    for k, T in enumerate(temps):
+        qT = special.softmax(ql.astype(np.float64) / T)
+        toks[0::2][k::3] = rng.choice(V, size=n, p=qT)
+    res = oracle.verify(target, draft, ro, toks, 1.0, seed=31, temperatures=Tr, n_threads=4)
+    for k, T in enumerate(temps):
+        pT = special.softmax(tl.astype(np.float64) / T); qT = special.softmax(ql.astype(np.float64) / T)
+        first = res.out_tokens[0::2][k::3]
+        assert stats.chisquare(np.bincount(first, minlength=V), pT * n).pvalue > 1e-3
+        want = 1 - 0.5 * np.abs(pT - qT).sum()
+        assert abs(res.accepted_len[k::3].mean() - want) < 4 * np.sqrt(want * (1 - want) / n)
+    # a uniform array gives exactly the scalar result; a bad temperature kills only its request
+    a = oracle.verify(target[:40], draft[:20], ro[:21], toks[:40], 0.8, seed=5)
+    b = oracle.verify(target[:40], draft[:20], ro[:21], toks[:40], 123.0, seed=5, temperatures=np.full(20, 0.8, np.float32))
+    np.testing.assert_array_equal(a.out_tokens, b.out_tokens)
+    bad = np.full(20, 0.8, np.float32); bad[3] = 0.0; bad[7] = np.nan
+    c = oracle.verify(target[:40], draft[:20], ro[:21], toks[:40], 1.0, seed=5, temperatures=bad)
+    assert c.status[3] & oracle.ST_BAD_TEMPERATURE and c.status[7] & oracle.ST_BAD_TEMPERATURE
+    assert (c.out_tokens[6:8] == -1).all() and c.accepted_len[3] == 0
+    keep = np.ones(40, bool); keep[6:8] = False; keep[14:16] = False
+    np.testing.assert_array_equal(c.out_tokens[keep], a.out_tokens[keep])
