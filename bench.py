@@ -46,6 +46,7 @@ REQUESTS_OVERRIDE = 0
 ASYNC_TOPK = False
 CUDA_GRAPH = False
 OVERLAP = False
+PER_REQUEST_T = False
 
 
 def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=False):
@@ -216,6 +217,13 @@ class Step:
         if self.wl["greedy"]:
             B.dspark_verify_greedy(batch.target, offsets, batch.draft_tokens, accepted_len=self.acc,
                                    out_tokens=self.out, dev_status=self.status, workspace=self.ws, n_rows=self.n_rows)
+        elif PER_REQUEST_T:
+            if not hasattr(self, "temps"):
+                self.temps = torch.full((self.R,), float(batch.temperature), device=self.acc.device)
+            B.dspark_verify_per_request(batch.target, batch.draft, offsets, batch.draft_tokens, self.temps, batch.seed,
+                                        draft_row_start=batch.draft_row_start, accepted_len=self.acc,
+                                        out_tokens=self.out, dev_status=self.status, workspace=self.ws,
+                                        n_rows=self.n_rows)
         else:
             B.dspark_verify(batch.target, batch.draft, offsets, batch.draft_tokens, batch.temperature, batch.seed,
                             draft_row_start=batch.draft_row_start, accepted_len=self.acc, out_tokens=self.out,
@@ -365,6 +373,8 @@ def main():
     ap.add_argument("--all-workloads", action="store_true", help="also time the other V=129280 configurations")
     ap.add_argument("--async-topk", action="store_true",
                     help="schedule with dspark_schedule_async (capacity from two steps earlier, Section 4.2)")
+    ap.add_argument("--per-request-temperature", action="store_true",
+                    help="verify with dspark_verify_per_request (a device array of R temperatures)")
     ap.add_argument("--overlap-schedule", action="store_true",
                     help="with --async-topk: schedule step t+1 on a second stream while step t is verified "
                          "(the asynchronous scheduler is off the critical path, Section 4.2)")
@@ -376,7 +386,8 @@ def main():
                     help="timed steps only (no clock probe, per-kernel timing, e2e or CPU legs): for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    global REQUESTS_OVERRIDE, ASYNC_TOPK, CUDA_GRAPH, OVERLAP
+    global REQUESTS_OVERRIDE, ASYNC_TOPK, CUDA_GRAPH, OVERLAP, PER_REQUEST_T
+    PER_REQUEST_T = args.per_request_temperature
     REQUESTS_OVERRIDE = args.requests
     ASYNC_TOPK, CUDA_GRAPH = args.async_topk, args.cuda_graph
     OVERLAP = args.overlap_schedule
@@ -565,6 +576,7 @@ def main():
                              f"({res['n_sets'] * stream_bytes / 1e6:.0f} MB of logits)",
                        "scheduler": ("async top-K, capacity from two steps earlier" if ASYNC_TOPK else "early stop")
                        if wl["sched"] is not None else None,
+                       "temperature": "per request (device array)" if PER_REQUEST_T else "one per batch",
                        "launch": "CUDA graph replay" if CUDA_GRAPH else
                        ("stream launches, scheduler of step t+1 overlapped on a second stream" if OVERLAP
                         else "stream launches"),

@@ -59,6 +59,7 @@ typedef enum {
 #define DSPARK_DEV_CONF_CLAMPED 16 /* a confidence was NaN, negative or above 1 (read as 0, 0, 1) */
 #define DSPARK_DEV_BUDGET_LT_R 32  /* token budget below the number of requests: every l*_r = 0 */
 #define DSPARK_DEV_ALL_NEG_INF 64  /* greedy: a row without any element above -inf (index 0 reported) */
+#define DSPARK_DEV_BAD_TEMPERATURE 128 /* a per-request temperature that is not a positive finite number */
 
 /* ------------------------------------------------------------------------------------
  * Engine throughput profile SPS(B), steps per second at B batch tokens (Section 3.2.2:
@@ -238,6 +239,21 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
                   float* out_p_tok, float* out_q_tok, int32_t* dev_status,
                   void* workspace, size_t workspace_bytes, void* stream);
 
+/* dspark_verify_per_request -- dspark_verify with one temperature per request (a serving batch
+ * mixes requests with different sampling settings): temperatures is a device array [R], request
+ * r uses p = softmax(target / T_r), q = softmax(draft / T_r).  A temperature that is not a
+ * positive finite number sets DSPARK_DEV_BAD_TEMPERATURE and voids that request only.
+ * One extra tiny kernel expands T_r to the rows; everything else is dspark_verify.
+ */
+int dspark_verify_per_request(const void* target_logits, const void* draft_logits, int dtype,
+                              int64_t target_row_stride, int64_t draft_row_stride, int V,
+                              const int32_t* row_offsets, const int64_t* draft_row_start,
+                              const int32_t* draft_tokens, int R, int n_rows,
+                              const float* temperatures, uint64_t seed,
+                              int32_t* accepted_len, int32_t* out_tokens,
+                              float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
 /* The two uniforms of (seed, request, position) exactly as the verifier draws them
  * (host computation; for tests and for replaying a step). */
 void dspark_uniforms(uint64_t seed, uint32_t request, uint32_t position,
@@ -254,7 +270,7 @@ typedef struct dspark_ktimer dspark_ktimer_t;
 enum {
     DSPARK_K_SCHEDULE = 0, DSPARK_K_OFFSETS = 1, DSPARK_K_STREAM = 2, DSPARK_K_DECIDE = 3,
     DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6, DSPARK_K_GREEDY_DECIDE = 7,
-    DSPARK_K_COUNT = 8
+    DSPARK_K_ROW_SCALE = 8, DSPARK_K_COUNT = 9
 };
 int dspark_ktimer_create(int capacity, dspark_ktimer_t** out);
 int dspark_ktimer_destroy(dspark_ktimer_t* t);

@@ -20,16 +20,16 @@ _lib: Optional[C.CDLL] = None
 DSPARK_F32, DSPARK_BF16 = 0, 1
 DSPARK_SCHED_EARLY_STOP, DSPARK_SCHED_GLOBAL, DSPARK_SCHED_TOPK = 0, 1, 2
 DEV_BAD_OFFSETS, DEV_BAD_TOKEN, DEV_BAD_ROW, DEV_TIMEOUT = 1, 2, 4, 8
-DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF = 16, 32, 64
+DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF, DEV_BAD_TEMPERATURE = 16, 32, 64, 128
 (K_SCHEDULE, K_OFFSETS, K_STREAM, K_DECIDE, K_RESIDUAL, K_FINALIZE, K_GREEDY_STREAM, K_GREEDY_DECIDE,
- K_COUNT) = range(9)
+ K_ROW_SCALE, K_COUNT) = range(10)
 
 EXPORTS = [
     "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",
     "dspark_schedule_workspace_bytes", "dspark_schedule", "dspark_build_offsets",
     "dspark_schedule_async", "dspark_async_state_init",
     "dspark_verify_workspace_bytes", "dspark_verify_greedy", "dspark_verify", "dspark_uniforms",
-    "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity",
+    "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity", "dspark_verify_per_request",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
     "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
     "dspark_version",
@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
         L.dspark_verify_greedy_static_capacity.restype = sz
         L.dspark_verify.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, C.c_float, u64,
                                     vp, vp, vp, vp, vp, vp, sz, vp]
+        L.dspark_verify_per_request.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, vp, u64,
+                                                vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_uniforms.argtypes = [u64, C.c_uint32, C.c_uint32, C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.dspark_uniforms.restype = None
         L.dspark_ktimer_create.argtypes = [i32, C.POINTER(vp)]
@@ -278,6 +280,33 @@ def dspark_verify(target: torch.Tensor, draft: torch.Tensor, row_offsets: torch.
                              _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
                              workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_verify")
+
+
+def dspark_verify_per_request(target: torch.Tensor, draft: torch.Tensor, row_offsets: torch.Tensor,
+                              draft_tokens: torch.Tensor, temperatures: torch.Tensor, seed: int, *,
+                              draft_row_start: Optional[torch.Tensor] = None,
+                              accepted_len: torch.Tensor, out_tokens: torch.Tensor,
+                              out_p_tok: Optional[torch.Tensor] = None, out_q_tok: Optional[torch.Tensor] = None,
+                              dev_status: Optional[torch.Tensor], workspace: torch.Tensor,
+                              n_rows: Optional[int] = None) -> None:
+    """dspark_verify with a CUDA float32[R] of per-request temperatures."""
+    tp, code, ts = _logits(target, "target")
+    dp, dcode, ds = _logits(draft, "draft")
+    if code != dcode or target.shape[1] != draft.shape[1]:
+        raise DsparkError("target and draft logits must share dtype and vocabulary size")
+    R = row_offsets.numel() - 1
+    if temperatures.numel() != R:
+        raise DsparkError("temperatures must have one entry per request")
+    n_rows = target.shape[0] if n_rows is None else n_rows
+    rc = lib().dspark_verify_per_request(
+        tp, dp, code, ts, ds, target.shape[1], _dev(row_offsets, "row_offsets", torch.int32),
+        _dev(draft_row_start, "draft_row_start", torch.int64), _dev(draft_tokens, "draft_tokens", torch.int32),
+        R, n_rows, _dev(temperatures, "temperatures", torch.float32), int(seed) & 0xFFFFFFFFFFFFFFFF,
+        _dev(accepted_len, "accepted_len", torch.int32), _dev(out_tokens, "out_tokens", torch.int32),
+        _dev(out_p_tok, "out_p_tok", torch.float32), _dev(out_q_tok, "out_q_tok", torch.float32),
+        _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_verify_per_request")
 
 
 def dspark_uniforms(seed: int, request: int, position: int):

@@ -33,7 +33,8 @@ struct __align__(16) ResidTask {     // one rejected request queued for the resi
     int64_t row_d;                   // physical draft row
     float cp, inv_zp, cq, inv_zq;    // row references (log2 domain) and 1 / row sums
     float u;                         // resample uniform of the rejected position
-    int32_t pad[3];
+    float scale;                     // log2(e) / T of this request
+    int32_t pad[2];
 };
 
 struct __align__(16) RequestRec {    // what the finalize kernel needs per request (written by decide)
@@ -42,7 +43,8 @@ struct __align__(16) RequestRec {    // what the finalize kernel needs per reque
     int64_t row_d;                   // physical draft row of the rejected position
     float cp, inv_zp, cq, inv_zq;    // row references (log2 domain) and 1 / row sums
     float u;                         // resample uniform
-    int32_t pad[3];
+    float scale;                     // log2(e) / T of this request
+    int32_t pad[2];
 };
 
 struct VerifyParams {
@@ -56,7 +58,10 @@ struct VerifyParams {
     const int64_t* draft_row_start;
     const int32_t* draft_tokens;
     int R, n_rows_cap;
-    float scale;                              // log2(e) / T
+    float scale;                              // log2(e) / T (one temperature for the batch)
+    const float* req_temp;                    // or: device [R] temperatures, one per request
+    float* row_scale_t;                       // workspace: per target row / per draft row log2(e) / T
+    float* row_scale_d;
     unsigned long long seed;
     int32_t* accepted_len;
     int32_t* out_tokens;
@@ -338,7 +343,7 @@ __device__ __forceinline__ float block_resid(const uint4 (&vt)[kVec], const uint
 // What a consumer warp does with its block of the unit (stream s, piece).
 template <int kElem, int kMode, typename Fetch>
 __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int piece, int n_rows,
-                                              int warp, int lane, const Fetch& f0, const Fetch& f1)
+                                              int warp, int lane, const Fetch& f0, const Fetch& f1, float scale)
 {
     using M = ModeCfg<kMode>;
     const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
@@ -349,7 +354,7 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
     uint4 v[M::kVec];
     load_block<kElem, M::kVec>(f0, nbytes, lane, v);
     if (kMode == kModeStats) {
-        const float2 st = block_stats<kElem, M::kVec>(v, P.scale);
+        const float2 st = block_stats<kElem, M::kVec>(v, scale);
         if (lane == 0) {
             float2* dst = (s < n_rows) ? P.stats_t + (long long)s * nblk : P.stats_d + (long long)(s - n_rows) * nblk;
             dst[b] = st;
@@ -362,10 +367,18 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
         load_block<kElem, M::kVec>(f1, nbytes, lane, vd);
         const ResidTask t = P.resid[s];
         ResidConst K;
-        K.set(P.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
+        K.set(t.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
         const float w = block_resid<kElem, M::kVec>(v, vd, K);
         if (lane == 0) P.wblk[(long long)t.request * nblk + b] = w;
     }
+}
+
+// Exponent scale log2(e)/T of row stream s (per-request temperatures are expanded per row).
+template <int kMode>
+__device__ __forceinline__ float stream_scale(const VerifyParams& P, int s, int n_rows, int n_streams)
+{
+    if (kMode != kModeStats || !P.req_temp || s >= n_streams) return P.scale;
+    return (s < n_rows) ? __ldcg(&P.row_scale_t[s]) : __ldcg(&P.row_scale_d[s - n_rows]);
 }
 
 // Source addresses of a unit (producer / direct path).
@@ -459,13 +472,14 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
             const int st = it % kStages;
             const uint32_t ph = (uint32_t)(it / kStages) & 1u;
             if (*abort_flag) break;
+            const float scale = stream_scale<kMode>(P, cur.s, n_rows, n_streams);   // in flight while we wait for the data
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(&full_bar[st], ph))) {
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
                 break;
             }
             unsigned char* sp = stage_mem + st * kStageBytes + warp * M::kBlockBytes;
             SmemFetch f0{sp}, f1{sp + M::kPieceBytes};
-            consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1);
+            consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1, scale);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);
         }
@@ -497,7 +511,8 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
         unit_sources<kMode>(P, cur.s, cur.piece, n_rows, src0, src1, bytes);
         GlobalFetch<kElem> f0{src0 + warp * M::kBlockBytes};
         GlobalFetch<kElem> f1{(kMode == kModeResid ? src1 : src0) + warp * M::kBlockBytes};
-        consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1);
+        consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1,
+                                    stream_scale<kMode>(P, cur.s, n_rows, n_streams));
     }
 }
 
@@ -743,6 +758,25 @@ __device__ __forceinline__ int level2_block(const unsigned char* trow, const uns
 }
 
 // ---------------------------------------------------------------------------------------
+// Per-request temperatures: expands T_r into one exponent scale log2(e)/T_r per target row and per
+// draft row (the streamed pass walks rows, not requests).  One thread per request.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) row_scale_kernel(VerifyParams P)
+{
+    pdl_wait();
+    const int r = blockIdx.x * 256 + threadIdx.x;
+    if (r >= P.R) return;
+    bool bad_rows;
+    const int n_rows = device_rows(P, &bad_rows);
+    const int lo = P.row_offsets[r], hi = P.row_offsets[r + 1];
+    if (lo < 0 || hi - lo < 1 || hi > n_rows || lo - r < 0 || (hi - 1 - r) > n_rows - P.R) return;
+    const float T = P.req_temp[r];
+    const float scale = (T > 0.0f && T < INFINITY) ? (float)(1.4426950408889634 / (double)T) : 1.0f;
+    for (int i = lo; i < hi; ++i) P.row_scale_t[i] = scale;
+    for (int i = lo - r; i < hi - 1 - r; ++i) P.row_scale_d[i] = scale;
+}
+
+// ---------------------------------------------------------------------------------------
 // decide: one CTA per request, one warp per position (eight per round): row statistics from
 // block statistics, p(x), q(x), accept test, first rejection n_r; the accepted prefix is written.
 // Position j = len is the bonus row (statistics only).  Every request leaves a record for the
@@ -786,7 +820,16 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
         return;
     }
     const bool want_all = (P.out_p != nullptr) || (P.out_q != nullptr);
-    const double scale_d = (double)P.scale;
+    float scale_f = P.scale;
+    if (P.req_temp) {
+        const float T = P.req_temp[r];
+        if (!(T > 0.0f) || !(T < INFINITY)) {
+            if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_TEMPERATURE); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
+            return;
+        }
+        scale_f = (float)(1.4426950408889634 / (double)T);
+    }
+    const double scale_d = (double)scale_f;
 
     for (int j0 = 0; j0 <= len; j0 += kWarps) {
         const int j = j0 + warp;
@@ -846,7 +889,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     const int n = s_first;
     RequestRec rec;
     rec.kind = kTaskNone; rec.row_t = lo + n; rec.row_d = drow0 + n;
-    rec.cp = rec.cq = 0.f; rec.inv_zp = rec.inv_zq = 1.f; rec.u = 0.f; rec.pad[0] = rec.pad[1] = rec.pad[2] = 0;
+    rec.cp = rec.cq = 0.f; rec.inv_zp = rec.inv_zq = 1.f; rec.u = 0.f; rec.scale = scale_f; rec.pad[0] = rec.pad[1] = 0;
     if (s_bad || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
         (n < len && !row_usable(s_fin_C[1], s_fin_S[1]))) {
         atomicOr(P.dev_status, s_bad ? s_bad : DSPARK_DEV_BAD_ROW);
@@ -865,7 +908,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             ResidTask q;
             q.request = r; q.row_t = rec.row_t; q.row_d = rec.row_d;
             q.cp = rec.cp; q.inv_zp = rec.inv_zp; q.cq = rec.cq; q.inv_zq = rec.inv_zq;
-            q.u = ur; q.pad[0] = q.pad[1] = q.pad[2] = 0;
+            q.u = ur; q.scale = scale_f; q.pad[0] = q.pad[1] = 0;
             P.resid[slot] = q;
         } else {
             rec.kind = kTaskBonus;
@@ -939,7 +982,7 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
         const double thr_local = u * tot - before;
         if (resid) {
             ResidConst K;
-            K.set(P.scale, rec.cp, rec.inv_zp, rec.cq, rec.inv_zq);
+            K.set(rec.scale, rec.cp, rec.inv_zp, rec.cq, rec.inv_zq);
             const int e0 = b * P.epb_r;
             const int cnt = (P.V - e0) < P.epb_r ? (P.V - e0) : P.epb_r;
             const unsigned char* drow = P.draft + rec.row_d * P.dstride_bytes;
@@ -947,7 +990,7 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
                 trow, drow, e0, cnt, lane, thr_local, [&](float xt, float xd) { return resid_elem(xt, xd, K); }, S);
         } else {
             // element masses relative to the row reference, like the block masses
-            const float nc = -rec.cp, scale = P.scale;
+            const float nc = -rec.cp, scale = rec.scale;
             const int e0 = b * P.epb;
             const int cnt = (P.V - e0) < P.epb ? (P.V - e0) : P.epb;
             token = e0 + level2_block<kElem, kStatBlockBytes, false>(
@@ -1092,7 +1135,7 @@ static void launch_stream_dtype(const VerifyParams& P, bool bulk, long long max_
 }
 
 struct Workspace {
-    size_t counters, stats_t, stats_d, resid, req, wblk, total;
+    size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, total;
 };
 static Workspace workspace_layout(int R, int n_rows, int V)
 {
@@ -1107,6 +1150,8 @@ static Workspace workspace_layout(int R, int n_rows, int V)
     w.resid = o;    o += up((size_t)R * sizeof(ResidTask));
     w.req = o;      o += up((size_t)R * sizeof(RequestRec));
     w.wblk = o;     o += up((size_t)R * nblk_r * sizeof(float));
+    w.scale_t = o;  o += up((size_t)n_rows * sizeof(float));
+    w.scale_d = o;  o += up((size_t)n_rows * sizeof(float));
     w.total = o;
     return w;
 }
@@ -1151,6 +1196,9 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.resid = (ResidTask*)(ws + w.resid);
     P.req = (RequestRec*)(ws + w.req);
     P.wblk = (float*)(ws + w.wblk);
+    P.req_temp = nullptr;
+    P.row_scale_t = (float*)(ws + w.scale_t);
+    P.row_scale_d = (float*)(ws + w.scale_d);
     return DSPARK_OK;
 }
 
@@ -1199,24 +1247,25 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
     return launch_status();
 }
 
-int dspark_verify(const void* target_logits, const void* draft_logits, int dtype,
-                  int64_t target_row_stride, int64_t draft_row_stride, int V,
-                  const int32_t* row_offsets, const int64_t* draft_row_start,
-                  const int32_t* draft_tokens, int R, int n_rows,
-                  float temperature, uint64_t seed,
-                  int32_t* accepted_len, int32_t* out_tokens,
-                  float* out_p_tok, float* out_q_tok, int32_t* dev_status,
-                  void* workspace, size_t workspace_bytes, void* stream)
+static int verify_launch(const void* target_logits, const void* draft_logits, int dtype,
+                         int64_t target_row_stride, int64_t draft_row_stride, int V,
+                         const int32_t* row_offsets, const int64_t* draft_row_start,
+                         const int32_t* draft_tokens, int R, int n_rows,
+                         float temperature, const float* req_temp, uint64_t seed,
+                         int32_t* accepted_len, int32_t* out_tokens,
+                         float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                         void* workspace, size_t workspace_bytes, void* stream)
 {
     if (!draft_logits) return DSPARK_ERR_INVALID_ARG;
-    if (!(temperature > 0.0f) || !isfinite(temperature)) return DSPARK_ERR_INVALID_ARG;
+    if (!req_temp && (!(temperature > 0.0f) || !isfinite(temperature))) return DSPARK_ERR_INVALID_ARG;
     if (draft_row_stride < V) return DSPARK_ERR_SHAPE;
     VerifyParams P;
     int rc = fill_params(P, target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V,
                          row_offsets, draft_row_start, draft_tokens, R, n_rows, accepted_len, out_tokens,
                          dev_status, workspace, workspace_bytes);
     if (rc != DSPARK_OK) return rc;
-    P.scale = (float)(1.4426950408889634 / (double)temperature);
+    P.scale = req_temp ? 1.0f : (float)(1.4426950408889634 / (double)temperature);
+    P.req_temp = req_temp;
     P.seed = seed;
     P.out_p = out_p_tok;
     P.out_q = out_q_tok;
@@ -1224,6 +1273,10 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
     cudaStream_t s = (cudaStream_t)stream;
     const bool bulk = !g_force_direct && aligned16(P.target, P.tstride_bytes, P.row_bytes) &&
                       aligned16(P.draft, P.dstride_bytes, P.row_bytes);
+    if (req_temp) {
+        KernelTimerScope timer(DSPARK_K_ROW_SCALE, s);
+        launch_pdl(row_scale_kernel, dim3((R + 255) / 256), dim3(256), 0, s, P);
+    }
     {
         KernelTimerScope timer(DSPARK_K_STREAM, s);
         launch_stream_dtype<kModeStats>(P, bulk, (2ll * n_rows - R) * pieces(P.nblk), s);
@@ -1306,6 +1359,35 @@ int dspark_verify_greedy_static(const void* target_logits, int dtype, int64_t ta
     // so nothing left by an earlier call needs clearing
     return dspark_verify_greedy(target_logits, dtype, target_row_stride, V, row_offsets, draft_tokens, R, n_rows,
                                 accepted_len, out_tokens, dev_status, scratch, kStaticScratchBytes, stream);
+}
+
+int dspark_verify(const void* target_logits, const void* draft_logits, int dtype,
+                  int64_t target_row_stride, int64_t draft_row_stride, int V,
+                  const int32_t* row_offsets, const int64_t* draft_row_start,
+                  const int32_t* draft_tokens, int R, int n_rows,
+                  float temperature, uint64_t seed,
+                  int32_t* accepted_len, int32_t* out_tokens,
+                  float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                  void* workspace, size_t workspace_bytes, void* stream)
+{
+    return verify_launch(target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V, row_offsets,
+                         draft_row_start, draft_tokens, R, n_rows, temperature, nullptr, seed, accepted_len,
+                         out_tokens, out_p_tok, out_q_tok, dev_status, workspace, workspace_bytes, stream);
+}
+
+int dspark_verify_per_request(const void* target_logits, const void* draft_logits, int dtype,
+                              int64_t target_row_stride, int64_t draft_row_stride, int V,
+                              const int32_t* row_offsets, const int64_t* draft_row_start,
+                              const int32_t* draft_tokens, int R, int n_rows,
+                              const float* temperatures, uint64_t seed,
+                              int32_t* accepted_len, int32_t* out_tokens,
+                              float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                              void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!temperatures) return DSPARK_ERR_INVALID_ARG;
+    return verify_launch(target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V, row_offsets,
+                         draft_row_start, draft_tokens, R, n_rows, 1.0f, temperatures, seed, accepted_len,
+                         out_tokens, out_p_tok, out_q_tok, dev_status, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

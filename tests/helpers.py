@@ -78,7 +78,7 @@ def check_greedy(batch: W.VerifyBatch, expect_status=None):
     return acc, out, o
 
 
-def gpu_verify(batch: W.VerifyBatch, want_probs=True, n_rows_cap=None):
+def gpu_verify(batch: W.VerifyBatch, want_probs=True, n_rows_cap=None, temperatures=None):
     R = batch.R
     cap = batch.n_rows if n_rows_cap is None else n_rows_cap
     acc = torch.full((R,), -7, dtype=torch.int32, device="cuda")
@@ -87,19 +87,26 @@ def gpu_verify(batch: W.VerifyBatch, want_probs=True, n_rows_cap=None):
     q = torch.full((cap,), float("nan"), dtype=torch.float32, device="cuda") if want_probs else None
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     ws = B.workspace(B.dspark_verify_workspace_bytes(R, cap, batch.V)).fill_(0xFF)     # poisoned: NaN patterns everywhere
-    B.dspark_verify(batch.target, batch.draft, batch.row_offsets, batch.draft_tokens, batch.temperature,
-                    batch.seed, draft_row_start=batch.draft_row_start, accepted_len=acc, out_tokens=out,
-                    out_p_tok=p, out_q_tok=q, dev_status=st, workspace=ws, n_rows=cap)
+    if temperatures is None:
+        B.dspark_verify(batch.target, batch.draft, batch.row_offsets, batch.draft_tokens, batch.temperature,
+                        batch.seed, draft_row_start=batch.draft_row_start, accepted_len=acc, out_tokens=out,
+                        out_p_tok=p, out_q_tok=q, dev_status=st, workspace=ws, n_rows=cap)
+    else:
+        B.dspark_verify_per_request(batch.target, batch.draft, batch.row_offsets, batch.draft_tokens,
+                                    temperatures, batch.seed, draft_row_start=batch.draft_row_start,
+                                    accepted_len=acc, out_tokens=out, out_p_tok=p, out_q_tok=q, dev_status=st,
+                                    workspace=ws, n_rows=cap)
     torch.cuda.synchronize()
     return dict(acc=acc.cpu().numpy(), out=out.cpu().numpy(), status=int(st.item()),
                 p=None if p is None else p.cpu().numpy(), q=None if q is None else q.cpu().numpy())
 
 
-def oracle_verify(batch: W.VerifyBatch, eval_all=True):
+def oracle_verify(batch: W.VerifyBatch, eval_all=True, temperatures=None):
     drs = None if batch.draft_row_start is None else batch.draft_row_start.cpu().numpy()
     return oracle.verify(W.bf16_bits(batch.target), W.bf16_bits(batch.draft), batch.row_offsets.cpu().numpy(),
                          batch.draft_tokens.cpu().numpy(), batch.temperature, batch.seed,
-                         draft_row_start=drs, eval_all=eval_all, n_threads=THREADS)
+                         draft_row_start=drs, eval_all=eval_all, n_threads=THREADS,
+                         temperatures=None if temperatures is None else temperatures.cpu().numpy())
 
 
 def compare_sampling(g: dict, o, row_offsets: np.ndarray, check_probs=True):
@@ -135,8 +142,8 @@ def compare_sampling(g: dict, o, row_offsets: np.ndarray, check_probs=True):
     return mismatches
 
 
-def check_sampling(batch: W.VerifyBatch, want_probs=True):
-    g = gpu_verify(batch, want_probs)
-    o = oracle_verify(batch, eval_all=want_probs)
+def check_sampling(batch: W.VerifyBatch, want_probs=True, temperatures=None):
+    g = gpu_verify(batch, want_probs, temperatures=temperatures)
+    o = oracle_verify(batch, eval_all=want_probs, temperatures=temperatures)
     mism = compare_sampling(g, o, batch.row_offsets.cpu().numpy(), check_probs=want_probs)
     return g, o, mism

@@ -83,6 +83,30 @@ def test_very_large_vocabularies(dtype, V):
     assert (g["acc"] < lengths.numpy()).any() and (g["acc"] == lengths.numpy()).any()   # both kinds of draw
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_per_request_temperatures(dtype):
+    g = torch.Generator(device="cpu"); g.manual_seed(4)
+    lengths = torch.randint(0, 7, (48,), generator=g)
+    batch = W.sampling_batch(lengths, W.V_FULL if dtype == torch.bfloat16 else 40_000, 17, "cuda", dtype=dtype,
+                             draft_noise=1.2, verify_seed=6, block=8)
+    temps = (0.5 + 1.2 * torch.rand(48, generator=g)).float().cuda()
+    gp, o, mism = H.check_sampling(batch, temperatures=temps)
+    assert mism == 0
+    # a uniform temperature array reproduces the scalar entry point bit for bit
+    uni = torch.full((48,), 0.8, device="cuda")
+    a = H.gpu_verify(W.VerifyBatch(batch.target, batch.draft, batch.row_offsets, batch.draft_tokens,
+                                   batch.draft_row_start, 0.8, batch.seed, batch.meta))
+    b = H.gpu_verify(batch, temperatures=uni)
+    for k in ("acc", "out", "p", "q"):
+        np.testing.assert_array_equal(a[k], b[k])
+    # invalid temperatures void only their own requests
+    bad = temps.clone(); bad[5] = 0.0; bad[9] = float("nan"); bad[11] = float("inf")
+    gb, ob, _ = H.check_sampling(batch, temperatures=bad)
+    assert gb["status"] & B.DEV_BAD_TEMPERATURE and (gb["acc"][[5, 9, 11]] == 0).all()
+    keep = np.ones(48, bool); keep[[5, 9, 11]] = False
+    np.testing.assert_array_equal(gb["acc"][keep], gp["acc"][keep])
+
+
 def test_compact_and_block_layouts_agree():
     lengths = torch.tensor([2, 5, 0, 3, 1, 7])
     a = W.sampling_batch(lengths, 20000, 3, "cuda", verify_seed=5)
