@@ -253,3 +253,20 @@ def verify(target, draft, row_offsets, draft_tokens, temperature: float, seed: i
     if rc != 0:
         raise ValueError("orc_verify rejected its arguments")
     return VerifyResult(acc, out, p, q, am, tm, st)
+
+
+def accept_rate(target, draft, row_offsets, temperature: float, draft_row_start=None):
+    """c*_{r,j} = 1 - TV(p, q) at every draft position (NaN at bonus rows); returns (cstar, status)."""
+    t, ts = _logits(target)
+    d, ds = _logits(draft)
+    ro = np.ascontiguousarray(row_offsets, dtype=np.int32)
+    drs = None if draft_row_start is None else np.ascontiguousarray(draft_row_start, dtype=np.int64)
+    R = len(ro) - 1
+    cstar = np.full(t.shape[0], np.nan)
+    st = np.zeros(R, dtype=np.int32)
+    rc = lib().orc_accept_rate(_p(t), _p(d), C.c_int(_dtype_code(t)), C.c_int64(ts), C.c_int64(ds),
+                               C.c_int(t.shape[1]), _p(ro), _p(drs), C.c_int(R), C.c_double(temperature),
+                               _p(cstar), _p(st))
+    if rc != 0:
+        raise ValueError("orc_accept_rate rejected its arguments")
+    return cstar, st

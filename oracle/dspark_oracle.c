@@ -630,6 +630,42 @@ int orc_verify(const void* target, const void* draft, int dtype,
     return 0;
 }
 
+/*
+ * Analytical per-step acceptance rate (Section 3.2.1, Eq. "accept_rate"):
+ *   c*_k = 1 - 1/2 * || p_k^d - p_k^t ||_1
+ * for every draft position of the ragged batch, p = softmax(target/T), q = softmax(draft/T).
+ * cstar has one entry per target row; bonus-row entries are set to NaN.
+ */
+int orc_accept_rate(const void* target, const void* draft, int dtype,
+                    int64_t target_row_stride, int64_t draft_row_stride, int V,
+                    const int32_t* row_offsets, const int64_t* draft_row_start, int R,
+                    double temperature, double* cstar, int32_t* status)
+{
+    if (R <= 0 || V <= 0 || !(temperature > 0.0) || !isfinite(temperature)) return -1;
+    for (int r = 0; r < R; ++r) {
+        int32_t lo = row_offsets[r], hi = row_offsets[r + 1];
+        status[r] = 0;
+        if (lo < 0 || hi - lo < 1) { status[r] = ORC_ST_BAD_OFFSETS; continue; }
+        int32_t len = hi - lo - 1;
+        int64_t drow0 = draft_row_start ? draft_row_start[r] : (int64_t)lo - (int64_t)r;
+        cstar[hi - 1] = NAN;
+        for (int32_t j = 0; j < len; ++j) {
+            double mp, Zp, mq, Zq;
+            int bad = row_softmax_stats(target, dtype, lo + j, target_row_stride, V, temperature, &mp, &Zp);
+            bad |= row_softmax_stats(draft, dtype, drow0 + j, draft_row_stride, V, temperature, &mq, &Zq);
+            if (bad) { status[r] |= ORC_ST_BAD_ROW; cstar[lo + j] = NAN; continue; }
+            double l1 = 0.0;
+            for (int v = 0; v < V; ++v) {
+                double pv = prob_at(target, dtype, lo + j, target_row_stride, v, temperature, mp, Zp);
+                double qv = prob_at(draft, dtype, drow0 + j, draft_row_stride, v, temperature, mq, Zq);
+                l1 += fabs(qv - pv);
+            }
+            cstar[lo + j] = 1.0 - 0.5 * l1;
+        }
+    }
+    return 0;
+}
+
 /* Threaded wrapper for the greedy verifier's timing leg (same results). */
 typedef struct {
     const void* target; int dtype; int64_t stride; int V;

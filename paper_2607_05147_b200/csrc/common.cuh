@@ -92,12 +92,6 @@ __device__ __forceinline__ float ex2_approx(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ float lg2_approx(float x)
-{
-    float y;
-    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 // Programmatic dependent launch: every kernel of the library is launched so that its CTAs may be
 // scheduled as soon as the previous kernel on the stream drains (no explicit early trigger: CTAs
 // that arrive early only poll and take issue slots from the kernel they wait for); pdl_wait()

@@ -316,3 +316,38 @@ def test_per_request_temperatures():
     assert (c.out_tokens[6:8] == -1).all() and c.accepted_len[3] == 0
     keep = np.ones(40, bool); keep[6:8] = False; keep[14:16] = False
     np.testing.assert_array_equal(c.out_tokens[keep], a.out_tokens[keep])
+
+
+def test_accept_rate_label(golden):
+    # Eq. (accept_rate): c* = 1 - 1/2 ||p_d - p_t||_1.  Appendix A pair: 0.8.
+    g = golden("appendix_a.txt")
+    p = np.array([float(x) for x in g["p_target"]]); q = np.array([float(x) for x in g["p_draft"]])
+    tl = np.log(p).astype(np.float32).reshape(1, 2).repeat(2, 0); ql = np.log(q).astype(np.float32).reshape(1, 2)
+    c, st = oracle.accept_rate(tl, ql, [0, 2], 1.0)
+    assert c[0] == pytest.approx(float(g["accept_prob"][0]), abs=1e-7) and np.isnan(c[1]) and st[0] == 0
+    # against numpy on random rows, several temperatures, ragged batch, block layout of the draft rows
+    rng = np.random.default_rng(13)
+    V, lens = 700, np.array([2, 0, 3, 1])
+    ro = np.concatenate([[0], np.cumsum(lens + 1)]).astype(np.int32)
+    x = rng.normal(0, 3, size=(ro[-1], V)).astype(np.float32)
+    y = rng.normal(0, 3, size=(4 * 3, V)).astype(np.float32)              # block layout: request r starts at 3 r
+    for T in (0.7, 1.0, 1.9):
+        c, st = oracle.accept_rate(x, y, ro, T, draft_row_start=np.arange(4) * 3)
+        for r in range(4):
+            for j in range(lens[r]):
+                pp = special.softmax(x[ro[r] + j].astype(np.float64) / T)
+                qq = special.softmax(y[3 * r + j].astype(np.float64) / T)
+                assert c[ro[r] + j] == pytest.approx(1 - 0.5 * np.abs(pp - qq).sum(), abs=1e-12)
+            assert np.isnan(c[ro[r + 1] - 1])
+    # identical distributions: c* = 1; the empirical acceptance frequency of the verifier converges to c*
+    c, _ = oracle.accept_rate(x[:2], x[:1], [0, 2], 1.3)
+    assert c[0] == pytest.approx(1.0, abs=1e-12)
+    n = 100_000
+    pq = rng.dirichlet(np.ones(5), size=2)
+    tl = np.log(pq[0]).astype(np.float32); ql = np.log(pq[1]).astype(np.float32)
+    target = np.broadcast_to(tl, (2 * n, 5)); draft = np.broadcast_to(ql, (n, 5))
+    ro = (2 * np.arange(n + 1)).astype(np.int32)
+    toks = np.zeros(2 * n, np.int32); toks[0::2] = rng.choice(5, size=n, p=_probs_of(ql))
+    res = oracle.verify(target, draft, ro, toks, 1.0, seed=77, n_threads=4)
+    c, _ = oracle.accept_rate(target[:2], draft[:1], [0, 2], 1.0)
+    assert abs(res.accepted_len.mean() - c[0]) < 4 * np.sqrt(c[0] * (1 - c[0]) / n)
