@@ -254,6 +254,26 @@ int dspark_verify_per_request(const void* target_logits, const void* draft_logit
                               float* out_p_tok, float* out_q_tok, int32_t* dev_status,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------
+ * dspark_accept_rate -- the analytical per-step acceptance rate of every draft position,
+ *     c*_{r,j} = 1 - 1/2 * || p^d_{r,j} - p^t_{r,j} ||_1          (Section 3.2.1, Eq. accept_rate),
+ * which the paper uses as the training label of the confidence head; with it an engine can also
+ * watch the calibration of its confidences on live batches.  p = softmax(target/T),
+ * q = softmax(draft/T); same ragged batch layout as the verifiers.
+ *  out_cstar  device [n_rows] fp32: entry row_offsets[r] + j for j < l_r; bonus-row entries and
+ *             positions with an unusable row (NaN, +inf, no finite element; BAD_ROW is set) are NaN.
+ * Reads every target and draft row once for the softmax statistics and the row pairs of all
+ * draft positions a second time (2 x the bytes of dspark_verify's first pass).
+ * workspace: dspark_accept_rate_workspace_bytes(R, n_rows, V), 256-byte aligned.
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE, CUDA.
+ */
+size_t dspark_accept_rate_workspace_bytes(int R, int n_rows, int V);
+int dspark_accept_rate(const void* target_logits, const void* draft_logits, int dtype,
+                       int64_t target_row_stride, int64_t draft_row_stride, int V,
+                       const int32_t* row_offsets, const int64_t* draft_row_start, int R, int n_rows,
+                       float temperature, float* out_cstar, int32_t* dev_status,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
 /* The two uniforms of (seed, request, position) exactly as the verifier draws them
  * (host computation; for tests and for replaying a step). */
 void dspark_uniforms(uint64_t seed, uint32_t request, uint32_t position,

@@ -30,6 +30,7 @@ EXPORTS = [
     "dspark_schedule_async", "dspark_async_state_init",
     "dspark_verify_workspace_bytes", "dspark_verify_greedy", "dspark_verify", "dspark_uniforms",
     "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity", "dspark_verify_per_request",
+    "dspark_accept_rate", "dspark_accept_rate_workspace_bytes",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
     "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
     "dspark_version",
@@ -74,6 +75,9 @@ def lib() -> C.CDLL:
                                     vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_verify_per_request.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, vp, u64,
                                                 vp, vp, vp, vp, vp, vp, sz, vp]
+        L.dspark_accept_rate_workspace_bytes.argtypes = [i32, i32, i32]
+        L.dspark_accept_rate_workspace_bytes.restype = sz
+        L.dspark_accept_rate.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, i32, C.c_float, vp, vp, vp, sz, vp]
         L.dspark_uniforms.argtypes = [u64, C.c_uint32, C.c_uint32, C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.dspark_uniforms.restype = None
         L.dspark_ktimer_create.argtypes = [i32, C.POINTER(vp)]
@@ -307,6 +311,28 @@ def dspark_verify_per_request(target: torch.Tensor, draft: torch.Tensor, row_off
         _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
         workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_verify_per_request")
+
+
+def dspark_accept_rate_workspace_bytes(R: int, n_rows: int, V: int) -> int:
+    return int(lib().dspark_accept_rate_workspace_bytes(R, n_rows, V))
+
+
+def dspark_accept_rate(target: torch.Tensor, draft: torch.Tensor, row_offsets: torch.Tensor, temperature: float, *,
+                       draft_row_start: Optional[torch.Tensor] = None, out_cstar: torch.Tensor,
+                       dev_status: Optional[torch.Tensor], workspace: torch.Tensor,
+                       n_rows: Optional[int] = None) -> None:
+    """c* = 1 - TV(p, q) at every draft position (the confidence head's analytical label)."""
+    tp, code, ts = _logits(target, "target")
+    dp, dcode, ds = _logits(draft, "draft")
+    if code != dcode or target.shape[1] != draft.shape[1]:
+        raise DsparkError("target and draft logits must share dtype and vocabulary size")
+    R = row_offsets.numel() - 1
+    n_rows = target.shape[0] if n_rows is None else n_rows
+    rc = lib().dspark_accept_rate(tp, dp, code, ts, ds, target.shape[1], _dev(row_offsets, "row_offsets", torch.int32),
+                                  _dev(draft_row_start, "draft_row_start", torch.int64), R, n_rows, float(temperature),
+                                  _dev(out_cstar, "out_cstar", torch.float32), _dev(dev_status, "dev_status", torch.int32),
+                                  _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_accept_rate")
 
 
 def dspark_uniforms(seed: int, request: int, position: int):

@@ -34,7 +34,8 @@ struct __align__(16) ResidTask {     // one rejected request queued for the resi
     float cp, inv_zp, cq, inv_zq;    // row references (log2 domain) and 1 / row sums
     float u;                         // resample uniform of the rejected position
     float scale;                     // log2(e) / T of this request
-    int32_t pad[2];
+    int32_t wslot;                   // which row of the block-sum array receives the result
+    int32_t pad;
 };
 
 struct __align__(16) RequestRec {    // what the finalize kernel needs per request (written by decide)
@@ -69,6 +70,7 @@ struct VerifyParams {
     float* out_q;
     int32_t* dev_status;
     // workspace
+    int resid_cap;                            // capacity of the residual queue (R, or rows for c*)
     int* counters;                            // [0] queued residual tasks, [1] dev_status stand-in
     float2* stats_t;
     float2* stats_d;
@@ -117,7 +119,7 @@ __device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
     if (kMode == kModeStats) return n_rows + (n_rows > P.R ? n_rows - P.R : 0);
     if (kMode == kModeGreedy) return n_rows;
     const int nq = __ldcg(&P.counters[0]);
-    return nq > P.R ? P.R : (nq < 0 ? 0 : nq);
+    return nq > P.resid_cap ? P.resid_cap : (nq < 0 ? 0 : nq);
 }
 
 // Walks the units (stream s, piece) owned by this CTA: unit index = s * ppr + piece, advancing by
@@ -369,7 +371,7 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
         ResidConst K;
         K.set(t.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
         const float w = block_resid<kElem, M::kVec>(v, vd, K);
-        if (lane == 0) P.wblk[(long long)t.request * nblk + b] = w;
+        if (lane == 0) P.wblk[(long long)t.wslot * nblk + b] = w;
     }
 }
 
@@ -908,7 +910,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             ResidTask q;
             q.request = r; q.row_t = rec.row_t; q.row_d = rec.row_d;
             q.cp = rec.cp; q.inv_zp = rec.inv_zp; q.cq = rec.cq; q.inv_zq = rec.inv_zq;
-            q.u = ur; q.scale = scale_f; q.pad[0] = q.pad[1] = 0;
+            q.u = ur; q.scale = scale_f; q.wslot = r; q.pad = 0;
             P.resid[slot] = q;
         } else {
             rec.kind = kTaskBonus;
@@ -999,6 +1001,68 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
         }
     }
     if (lane == 0) P.out_tokens[rec.row_t] = token;
+}
+
+// ---------------------------------------------------------------------------------------
+// Analytical acceptance rate c* = 1 - 1/2 ||p_d - p_t||_1 = 1 - sum_v max(0, p_v - q_v)
+// (Section 3.2.1, the confidence head's training label) for every draft position.  Reuses the
+// streamed statistics and the residual pass: every draft position is queued as a residual task
+// (slot = its compact draft index), then one warp per position sums the block values.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kDecideThreads) queue_all_positions_kernel(VerifyParams P, float* out_cstar)
+{
+    constexpr int kWarps = kDecideThreads / 32;
+    pdl_wait();
+    const int r = blockIdx.x;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    bool bad_rows;
+    const int n_rows = device_rows(P, &bad_rows);
+    if (r == 0 && tid == 0) P.counters[0] = n_rows > P.R ? n_rows - P.R : 0;     // every draft position is a task
+    const int lo = P.row_offsets[r], hi = P.row_offsets[r + 1];
+    const bool ok = !(lo < 0 || hi - lo < 1 || hi > n_rows || lo - r < 0 || (hi - 1 - r) > n_rows - P.R);
+    if (!ok) {
+        if (tid == 0) atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS);
+        return;
+    }
+    const int len = hi - lo - 1;
+    const long long drow0 = P.draft_row_start ? P.draft_row_start[r] : (long long)(lo - r);
+    if (tid == 0) out_cstar[hi - 1] = NAN;                                       // bonus row: no draft distribution
+    for (int j = warp; j < len; j += kWarps) {
+        RowAcc A, D;
+        combine_rows(P.stats_t + (long long)(lo + j) * P.nblk, P.stats_d + (long long)(lo - r + j) * P.nblk,
+                     P.nblk, lane, A, D);
+        if (lane == 0) {
+            const bool usable = row_usable(A.C, A.S) && row_usable(D.C, D.S);
+            if (!usable) atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW);
+            ResidTask q;
+            q.request = r; q.row_t = lo + j; q.row_d = drow0 + j;
+            q.cp = A.C; q.cq = D.C;
+            q.inv_zp = usable ? (float)(1.0 / A.S) : NAN;                       // NaN propagates to c*
+            q.inv_zq = usable ? (float)(1.0 / D.S) : NAN;
+            q.u = 0.f; q.scale = P.scale; q.wslot = lo - r + j; q.pad = 0;
+            P.resid[lo - r + j] = q;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kDecideThreads) cstar_reduce_kernel(VerifyParams P, float* out_cstar)
+{
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int slot = blockIdx.x * (kDecideThreads / 32) + (threadIdx.x >> 5);
+    int nq = __ldcg(&P.counters[0]);
+    nq = nq > P.n_rows_cap ? P.n_rows_cap : nq;
+    if (slot >= nq) return;
+    const float* wb = P.wblk + (long long)slot * P.nblk_r;
+    double w = 0.0;
+#pragma unroll 4
+    for (int b = lane; b < P.nblk_r; b += 32) w += (double)__ldcg(&wb[b]);
+    w = warp_sum_f64(w);
+    if (lane == 0) {
+        const ResidTask t = P.resid[slot];
+        const bool usable = t.inv_zp == t.inv_zp && t.inv_zq == t.inv_zq;      // NaN marks an unusable row
+        out_cstar[t.row_t] = usable ? (float)(1.0 - w) : NAN;
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -1196,6 +1260,7 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.resid = (ResidTask*)(ws + w.resid);
     P.req = (RequestRec*)(ws + w.req);
     P.wblk = (float*)(ws + w.wblk);
+    P.resid_cap = R;
     P.req_temp = nullptr;
     P.row_scale_t = (float*)(ws + w.scale_t);
     P.row_scale_d = (float*)(ws + w.scale_d);
@@ -1388,6 +1453,78 @@ int dspark_verify_per_request(const void* target_logits, const void* draft_logit
     return verify_launch(target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V, row_offsets,
                          draft_row_start, draft_tokens, R, n_rows, 1.0f, temperatures, seed, accepted_len,
                          out_tokens, out_p_tok, out_q_tok, dev_status, workspace, workspace_bytes, stream);
+}
+
+static size_t accept_rate_extra(int n_rows, int V, size_t* resid_off, size_t* wblk_off)
+{
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t nblk_r = (size_t)blocks_per_row(V, 4, kResidBlockBytes);
+    size_t o = 0;
+    *resid_off = o; o += up((size_t)n_rows * sizeof(ResidTask));
+    *wblk_off = o;  o += up((size_t)n_rows * nblk_r * sizeof(float));
+    return o;
+}
+
+size_t dspark_accept_rate_workspace_bytes(int R, int n_rows, int V)
+{
+    if (R < 1 || n_rows < R || V < 1) return 0;
+    size_t a, b;
+    return workspace_layout(R, n_rows, V).total + accept_rate_extra(n_rows, V, &a, &b);
+}
+
+int dspark_accept_rate(const void* target_logits, const void* draft_logits, int dtype,
+                       int64_t target_row_stride, int64_t draft_row_stride, int V,
+                       const int32_t* row_offsets, const int64_t* draft_row_start, int R, int n_rows,
+                       float temperature, float* out_cstar, int32_t* dev_status,
+                       void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!draft_logits || !out_cstar) return DSPARK_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || !isfinite(temperature)) return DSPARK_ERR_INVALID_ARG;
+    if (draft_row_stride < V) return DSPARK_ERR_SHAPE;
+    if (R < 1 || n_rows < R || V < 1) return DSPARK_ERR_INVALID_ARG;
+    size_t resid_off, wblk_off;
+    const size_t base = workspace_layout(R, n_rows, V).total;
+    const size_t extra = accept_rate_extra(n_rows, V, &resid_off, &wblk_off);
+    if (!workspace || workspace_bytes < base + extra) return DSPARK_ERR_WORKSPACE;
+    VerifyParams P;
+    // the token / length outputs of the verifier are not produced here: the row_offsets pointer only
+    // stands in for the non-null checks of the shared set-up and is never written through
+    int rc = fill_params(P, target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V,
+                         row_offsets, draft_row_start, row_offsets, R, n_rows,
+                         const_cast<int32_t*>(row_offsets), const_cast<int32_t*>(row_offsets), dev_status,
+                         workspace, workspace_bytes);
+    if (rc != DSPARK_OK) return rc;
+    P.accepted_len = nullptr; P.out_tokens = nullptr; P.draft_tokens = nullptr;
+    P.scale = (float)(1.4426950408889634 / (double)temperature);
+    P.resid = (ResidTask*)((unsigned char*)workspace + base + resid_off);
+    P.wblk = (float*)((unsigned char*)workspace + base + wblk_off);
+    P.resid_cap = n_rows;
+    if (!ensure_attrs()) return launch_status();
+    cudaStream_t s = (cudaStream_t)stream;
+    const bool bulk = !g_force_direct && aligned16(P.target, P.tstride_bytes, P.row_bytes) &&
+                      aligned16(P.draft, P.dstride_bytes, P.row_bytes);
+    {
+        KernelTimerScope timer(DSPARK_K_STREAM, s);
+        launch_stream_dtype<kModeStats>(P, bulk, (2ll * n_rows - R) * pieces(P.nblk), s);
+    }
+    if ((rc = launch_status()) != DSPARK_OK) return rc;
+    {
+        KernelTimerScope timer(DSPARK_K_DECIDE, s);
+        launch_pdl(queue_all_positions_kernel, dim3(R), dim3(kDecideThreads), 0, s, P, out_cstar);
+    }
+    if ((rc = launch_status()) != DSPARK_OK) return rc;
+    {
+        KernelTimerScope timer(DSPARK_K_RESIDUAL, s);
+        launch_stream_dtype<kModeResid>(P, bulk, (long long)(n_rows - R > 0 ? n_rows - R : 1) * pieces(P.nblk_r), s);
+    }
+    if ((rc = launch_status()) != DSPARK_OK) return rc;
+    {
+        KernelTimerScope timer(DSPARK_K_FINALIZE, s);
+        const int warps = kDecideThreads / 32;
+        const int grid = (n_rows - R + warps - 1) / warps;
+        launch_pdl(cstar_reduce_kernel, dim3(grid > 0 ? grid : 1), dim3(kDecideThreads), 0, s, P, out_cstar);
+    }
+    return launch_status();
 }
 
 }  // extern "C"
