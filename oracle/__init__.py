@@ -270,3 +270,36 @@ def accept_rate(target, draft, row_offsets, temperature: float, draft_row_start=
     if rc != 0:
         raise ValueError("orc_accept_rate rejected its arguments")
     return cstar, st
+
+
+def markov_logits(U, W1, W2, x_prev):
+    """Draft logits U + W1[x_prev] @ W2 from bf16 bit patterns (uint16).  Returns (fp64, bf16 bits)."""
+    U = np.asarray(U); W1 = np.ascontiguousarray(W1); W2 = np.ascontiguousarray(W2)
+    assert U.dtype == W1.dtype == W2.dtype == np.uint16 and U.strides[1] == 2
+    R, V = U.shape
+    rank = W1.shape[1]
+    assert W1.shape[0] == V and W2.shape == (rank, V)
+    xp = np.ascontiguousarray(x_prev, dtype=np.int32)
+    f64 = np.empty((R, V), dtype=np.float64)
+    b16 = np.empty((R, V), dtype=np.uint16)
+    rc = lib().orc_markov_logits(_p(U), C.c_int64(U.strides[0] // 2), _p(W1), _p(W2), _p(xp), C.c_int(R), C.c_int(V),
+                                 C.c_int(rank), _p(f64), _p(b16))
+    if rc != 0:
+        raise ValueError(f"orc_markov_logits failed ({rc})")
+    return f64, b16
+
+
+def confidence(H, W1, w, x_prev):
+    """c = sigmoid(w . [h ; W1[x_prev]]): H bf16 bits [R, d], W1 bf16 bits [V, rank], w float32 [d + rank]."""
+    H = np.asarray(H); W1 = np.ascontiguousarray(W1)
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    R, d = H.shape
+    V, rank = W1.shape
+    assert w.size == d + rank
+    xp = np.ascontiguousarray(x_prev, dtype=np.int32)
+    out = np.empty(R, dtype=np.float64)
+    rc = lib().orc_confidence(_p(H), C.c_int64(H.strides[0] // 2), C.c_int(d), _p(W1), C.c_int(rank), C.c_int(V),
+                              _p(w), _p(xp), C.c_int(R), _p(out))
+    if rc != 0:
+        raise ValueError(f"orc_confidence failed ({rc})")
+    return out

@@ -666,6 +666,69 @@ int orc_accept_rate(const void* target, const void* draft, int dtype,
     return 0;
 }
 
+/*
+ * Markov-head draft step (Section 3.1, Eq. "sequential-factorization" and Eq. "markov"):
+ * the draft logits of position k are the backbone's base logits plus a first-order transition
+ * bias from the previously sampled token,
+ *     logits[r, v] = U_k[r, v] + sum_i W1[x_prev[r], i] * W2[i, v],
+ * with W1 in R^{V x rank} (embedding lookup) and W2 in R^{rank x V} (logit projection).
+ * All inputs are bf16 bit patterns; the sum is taken in fp64 in index order.  The result is
+ * returned in fp64 and, rounded to nearest-even, as the bf16 pattern a drafter would store
+ * (the verifier later reads exactly those stored logits as the draft distribution).
+ */
+static inline double bf16_to_f64(uint16_t h)
+{
+    uint32_t bits = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &bits, 4);
+    return (double)f;
+}
+static inline uint16_t f64_to_bf16_rne(double x)
+{
+    float f = (float)x;                 /* fp64 -> fp32 (double rounding is far below a bf16 ulp) */
+    uint32_t bits;
+    memcpy(&bits, &f, 4);
+    if ((bits & 0x7F800000u) == 0x7F800000u) return (uint16_t)(bits >> 16);   /* inf / nan */
+    uint32_t lsb = (bits >> 16) & 1u;
+    bits += 0x7FFFu + lsb;
+    return (uint16_t)(bits >> 16);
+}
+
+int orc_markov_logits(const uint16_t* U, int64_t u_stride, const uint16_t* W1, const uint16_t* W2,
+                      const int32_t* x_prev, int R, int V, int rank, double* out_f64, uint16_t* out_bf16)
+{
+    if (R <= 0 || V <= 0 || rank <= 0) return -1;
+    for (int r = 0; r < R; ++r) {
+        int32_t x = x_prev[r];
+        if (x < 0 || x >= V) return -2;
+        for (int v = 0; v < V; ++v) {
+            double b = 0.0;
+            for (int i = 0; i < rank; ++i)
+                b += bf16_to_f64(W1[(size_t)x * rank + i]) * bf16_to_f64(W2[(size_t)i * V + v]);
+            double l = bf16_to_f64(U[(size_t)r * u_stride + v]) + b;
+            if (out_f64) out_f64[(size_t)r * V + v] = l;
+            if (out_bf16) out_bf16[(size_t)r * V + v] = f64_to_bf16_rne(l);
+        }
+    }
+    return 0;
+}
+
+/* Confidence head (Section 3.2.1, Eq. "confidence"): c = sigmoid(w^T [h ; W1[x_prev]]),
+ * h in R^d (bf16), w in R^{d + rank} (fp32). */
+int orc_confidence(const uint16_t* H, int64_t h_stride, int d, const uint16_t* W1, int rank, int V,
+                   const float* w, const int32_t* x_prev, int R, double* conf)
+{
+    for (int r = 0; r < R; ++r) {
+        int32_t x = x_prev[r];
+        if (x < 0 || x >= V) return -2;
+        double z = 0.0;
+        for (int i = 0; i < d; ++i) z += (double)w[i] * bf16_to_f64(H[(size_t)r * h_stride + i]);
+        for (int i = 0; i < rank; ++i) z += (double)w[d + i] * bf16_to_f64(W1[(size_t)x * rank + i]);
+        conf[r] = 1.0 / (1.0 + exp(-z));
+    }
+    return 0;
+}
+
 /* Threaded wrapper for the greedy verifier's timing leg (same results). */
 typedef struct {
     const void* target; int dtype; int64_t stride; int V;
