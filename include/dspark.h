@@ -274,6 +274,52 @@ int dspark_accept_rate(const void* target_logits, const void* draft_logits, int 
                        float temperature, float* out_cstar, int32_t* dev_status,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------
+ * The Markov-head sequential draft step (Section 3.1, Eq. sequential-factorization and Eq. markov;
+ * confidence head: Section 3.2.1, Eq. confidence).  For block position k and every request r,
+ *     logits[r, :] = U[r, :] + W1[x_prev[r]] W2,   W1 in R^{V x 256}, W2 in R^{256 x V}  (rank 256),
+ *     x[r] ~ softmax(logits[r, :] / T),
+ *     conf[r] = sigmoid(w^T [ H[r, :] ; W1[x_prev[r]] ]).
+ * The bias product runs on the tensor cores (bf16 operands, fp32 accumulation over the 256 terms);
+ * base logits are added in fp32 and the sum is rounded once to bf16 (round to nearest even): the
+ * stored logits are what the draw uses and what a verifier later reads as the draft distribution.
+ *
+ * dspark_markov_pack_w2: one-time re-layout of W2 (device, bf16, row-major [256, V]) into the
+ *   tile order the contraction reads (device, dspark_markov_w2_packed_bytes(V), 16-byte aligned;
+ *   columns past V are zero).  The caller owns both buffers.
+ * dspark_markov_logits:
+ *   U            device bf16 [R, >= V], row stride u_row_stride elements: base logits of position k
+ *   W1           device bf16 [V, 256] row-major, 16-byte aligned
+ *   W2_packed    output of dspark_markov_pack_w2
+ *   x_prev       device int32 [R]: previous token of each request (anchor token at k = 1); a value
+ *                outside [0, V) sets DSPARK_DEV_BAD_TOKEN and contributes a zero embedding
+ *   H, w_conf    device bf16 [R, >= d] (stride h_row_stride) and device fp32 [d + 256]; read only
+ *                when out_conf is non-NULL.  The dot product is accumulated in fp64.
+ *   out_logits   device bf16 [R, >= V], row stride out_row_stride elements
+ *   out_conf     device fp32 [R] or NULL
+ *   workspace    dspark_markov_workspace_bytes(R, V), 256-byte aligned
+ * dspark_markov_draft_step: dspark_markov_logits, then one draw per request exactly as the
+ *   verifier's bonus draw of a request with no draft position: temperature > 0 samples with the
+ *   second uniform of (seed, request r, position 0), temperature == 0 takes the argmax (lowest
+ *   index on ties).  out_tokens device int32 [R].
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, CUDA; a device wait that ran out sets
+ * DSPARK_DEV_TIMEOUT in *dev_status and the affected logits are unspecified.
+ */
+size_t dspark_markov_w2_packed_bytes(int V);
+int dspark_markov_pack_w2(const void* W2, int V, void* W2_packed, void* stream);
+size_t dspark_markov_workspace_bytes(int R, int V);
+int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                         const int32_t* x_prev, int R, int V,
+                         const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                         void* out_logits, int64_t out_row_stride, float* out_conf, int32_t* dev_status,
+                         void* workspace, size_t workspace_bytes, void* stream);
+int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                             const int32_t* x_prev, int R, int V,
+                             const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                             float temperature, uint64_t seed,
+                             void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
+                             int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
+
 /* The two uniforms of (seed, request, position) exactly as the verifier draws them
  * (host computation; for tests and for replaying a step). */
 void dspark_uniforms(uint64_t seed, uint32_t request, uint32_t position,
@@ -290,7 +336,7 @@ typedef struct dspark_ktimer dspark_ktimer_t;
 enum {
     DSPARK_K_SCHEDULE = 0, DSPARK_K_OFFSETS = 1, DSPARK_K_STREAM = 2, DSPARK_K_DECIDE = 3,
     DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6, DSPARK_K_GREEDY_DECIDE = 7,
-    DSPARK_K_ROW_SCALE = 8, DSPARK_K_COUNT = 9
+    DSPARK_K_ROW_SCALE = 8, DSPARK_K_MARKOV_GEMM = 9, DSPARK_K_COUNT = 10
 };
 int dspark_ktimer_create(int capacity, dspark_ktimer_t** out);
 int dspark_ktimer_destroy(dspark_ktimer_t* t);

@@ -22,7 +22,7 @@ DSPARK_SCHED_EARLY_STOP, DSPARK_SCHED_GLOBAL, DSPARK_SCHED_TOPK = 0, 1, 2
 DEV_BAD_OFFSETS, DEV_BAD_TOKEN, DEV_BAD_ROW, DEV_TIMEOUT = 1, 2, 4, 8
 DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF, DEV_BAD_TEMPERATURE = 16, 32, 64, 128
 (K_SCHEDULE, K_OFFSETS, K_STREAM, K_DECIDE, K_RESIDUAL, K_FINALIZE, K_GREEDY_STREAM, K_GREEDY_DECIDE,
- K_ROW_SCALE, K_COUNT) = range(10)
+ K_ROW_SCALE, K_MARKOV_GEMM, K_COUNT) = range(11)
 
 EXPORTS = [
     "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",
@@ -31,6 +31,8 @@ EXPORTS = [
     "dspark_verify_workspace_bytes", "dspark_verify_greedy", "dspark_verify", "dspark_uniforms",
     "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity", "dspark_verify_per_request",
     "dspark_accept_rate", "dspark_accept_rate_workspace_bytes",
+    "dspark_markov_w2_packed_bytes", "dspark_markov_pack_w2", "dspark_markov_workspace_bytes",
+    "dspark_markov_logits", "dspark_markov_draft_step",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
     "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
     "dspark_version",
@@ -78,6 +80,14 @@ def lib() -> C.CDLL:
         L.dspark_accept_rate_workspace_bytes.argtypes = [i32, i32, i32]
         L.dspark_accept_rate_workspace_bytes.restype = sz
         L.dspark_accept_rate.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, i32, C.c_float, vp, vp, vp, sz, vp]
+        L.dspark_markov_w2_packed_bytes.argtypes = [i32]
+        L.dspark_markov_w2_packed_bytes.restype = sz
+        L.dspark_markov_pack_w2.argtypes = [vp, i32, vp, vp]
+        L.dspark_markov_workspace_bytes.argtypes = [i32, i32]
+        L.dspark_markov_workspace_bytes.restype = sz
+        L.dspark_markov_logits.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, vp, i64, vp, vp, vp, sz, vp]
+        L.dspark_markov_draft_step.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, C.c_float, u64,
+                                               vp, i64, vp, vp, vp, vp, sz, vp]
         L.dspark_uniforms.argtypes = [u64, C.c_uint32, C.c_uint32, C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.dspark_uniforms.restype = None
         L.dspark_ktimer_create.argtypes = [i32, C.POINTER(vp)]
@@ -333,6 +343,74 @@ def dspark_accept_rate(target: torch.Tensor, draft: torch.Tensor, row_offsets: t
                                   _dev(out_cstar, "out_cstar", torch.float32), _dev(dev_status, "dev_status", torch.int32),
                                   _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_accept_rate")
+
+
+def dspark_markov_w2_packed_bytes(V: int) -> int:
+    return int(lib().dspark_markov_w2_packed_bytes(V))
+
+
+def dspark_markov_pack_w2(W2: torch.Tensor, W2_packed: torch.Tensor) -> None:
+    """W2: CUDA bf16 [256, V] contiguous; W2_packed: CUDA uint8 of dspark_markov_w2_packed_bytes(V)."""
+    if W2.dim() != 2 or W2.shape[0] != 256 or not W2.is_contiguous():
+        raise DsparkError("W2 must be a contiguous [256, V] tensor")
+    if W2_packed.numel() * W2_packed.element_size() < dspark_markov_w2_packed_bytes(W2.shape[1]):
+        raise DsparkError("W2_packed is too small")
+    _check(lib().dspark_markov_pack_w2(_dev(W2, "W2", torch.bfloat16), W2.shape[1], _dev(W2_packed, "W2_packed"),
+                                       _stream()), "dspark_markov_pack_w2")
+
+
+def dspark_markov_workspace_bytes(R: int, V: int) -> int:
+    return int(lib().dspark_markov_workspace_bytes(R, V))
+
+
+def _markov_args(U, W1, W2_packed, x_prev, H, w_conf, out_logits, out_conf):
+    if U.dim() != 2 or U.stride(1) != 1 or out_logits.dim() != 2 or out_logits.stride(1) != 1:
+        raise DsparkError("U and out_logits must be 2-D with unit inner stride")
+    R, V = U.shape
+    if W1.shape != (V, 256) or not W1.is_contiguous():
+        raise DsparkError("W1 must be a contiguous [V, 256] tensor")
+    if out_logits.shape[0] < R or out_logits.shape[1] < V or x_prev.numel() < R:
+        raise DsparkError("out_logits / x_prev are too small")
+    d = 0
+    if out_conf is not None:
+        if H is None or w_conf is None or H.dim() != 2 or H.stride(1) != 1 or H.shape[0] < R:
+            raise DsparkError("out_conf needs H [R, d] and w_conf [d + 256]")
+        d = H.shape[1]
+        if w_conf.numel() != d + 256 or out_conf.numel() < R:
+            raise DsparkError("w_conf must hold d + 256 weights, out_conf R values")
+    return (_dev(U, "U", torch.bfloat16), U.stride(0), _dev(W1, "W1", torch.bfloat16), _dev(W2_packed, "W2_packed"),
+            _dev(x_prev, "x_prev", torch.int32), R, V, _dev(H, "H", torch.bfloat16) if out_conf is not None else None,
+            H.stride(0) if out_conf is not None else 0, d,
+            _dev(w_conf, "w_conf", torch.float32) if out_conf is not None else None)
+
+
+def dspark_markov_logits(U: torch.Tensor, W1: torch.Tensor, W2_packed: torch.Tensor, x_prev: torch.Tensor, *,
+                         H: Optional[torch.Tensor] = None, w_conf: Optional[torch.Tensor] = None,
+                         out_logits: torch.Tensor, out_conf: Optional[torch.Tensor] = None,
+                         dev_status: torch.Tensor, workspace: torch.Tensor) -> None:
+    head = _markov_args(U, W1, W2_packed, x_prev, H, w_conf, out_logits, out_conf)
+    rc = lib().dspark_markov_logits(*head, _dev(out_logits, "out_logits", torch.bfloat16), out_logits.stride(0),
+                                    _dev(out_conf, "out_conf", torch.float32), _dev(dev_status, "dev_status", torch.int32),
+                                    _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_markov_logits")
+
+
+def dspark_markov_draft_step(U: torch.Tensor, W1: torch.Tensor, W2_packed: torch.Tensor, x_prev: torch.Tensor,
+                             temperature: float, seed: int, *,
+                             H: Optional[torch.Tensor] = None, w_conf: Optional[torch.Tensor] = None,
+                             out_logits: torch.Tensor, out_tokens: torch.Tensor,
+                             out_conf: Optional[torch.Tensor] = None,
+                             dev_status: torch.Tensor, workspace: torch.Tensor) -> None:
+    head = _markov_args(U, W1, W2_packed, x_prev, H, w_conf, out_logits, out_conf)
+    if out_tokens.numel() < head[5]:
+        raise DsparkError("out_tokens is too small")
+    rc = lib().dspark_markov_draft_step(*head, float(temperature), int(seed) & (2**64 - 1),
+                                        _dev(out_logits, "out_logits", torch.bfloat16), out_logits.stride(0),
+                                        _dev(out_tokens, "out_tokens", torch.int32),
+                                        _dev(out_conf, "out_conf", torch.float32),
+                                        _dev(dev_status, "dev_status", torch.int32),
+                                        _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_markov_draft_step")
 
 
 def dspark_uniforms(seed: int, request: int, position: int):

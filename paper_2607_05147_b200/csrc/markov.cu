@@ -1,0 +1,403 @@
+// dspark_markov_*: the Markov-head sequential draft step (Section 3.1, Eq. sequential-factorization
+// and Eq. markov): draft logits of one block position for all requests,
+//     logits[r, :] = U_k[r, :] + W1[x_prev[r]] W2          (rank 256),
+// followed by one draw per request from softmax(logits / T) and the confidence
+//     c[r] = sigmoid(w^T [h_k[r] ; W1[x_prev[r]]])          (Section 3.2.1, Eq. confidence).
+//
+// The bias is a dense [R,256] x [256,V] contraction, so it runs on the 5th-generation tensor cores:
+// one persistent CTA per SM walks 128-column tiles of the vocabulary; a producer thread brings the
+// pre-packed W2 tile and the gathered embedding tiles into shared memory with bulk async copies, one
+// thread issues tcgen05.mma (M = N = 128, K = 16 x 16) into one of two TMEM accumulators, and four
+// epilogue warps read the accumulator back (tcgen05.ld), add the base logits, round to bf16 and
+// store the draft logits.  The draw itself is the verifier's bonus path on those stored logits (a
+// request with no draft position emits one token from p), so what the drafter samples from is
+// bit for bit the distribution the verifier will later read as q.
+#include <cuda_bf16.h>
+#include <cstdio>
+#include <math.h>
+
+#include "common.cuh"
+
+namespace dspark {
+
+constexpr int kRank = 256;                       // r of the low-rank factorization
+constexpr int kTileMN = 128;                     // M and N of one MMA tile
+constexpr int kTileBytes = kTileMN * kRank * 2;  // 64 KB of bf16: one packed operand tile
+constexpr int kKChunks = kRank / 8;              // 16-byte chunks along K
+constexpr int kChunkBytes = kTileMN * 16;        // one K chunk of a tile: 128 rows x 16 B
+constexpr int kGemmThreads = 192;                // producer warp, MMA warp, four epilogue warps
+constexpr int kTmemCols = 256;                   // two fp32 accumulators of 128 columns
+
+// Packed operand tile (K-major, no swizzle): element (row, k) of a 128 x 256 tile lives at
+//   (k / 8) * 2048 + (row / 8) * 128 + (row % 8) * 16 + (k % 8) * 2   bytes,
+// i.e. 8 x 16 B core matrices, 16 of them per K chunk.
+__host__ __device__ inline size_t packed_offset(int row, int k)
+{
+    return (size_t)(k >> 3) * kChunkBytes + (size_t)(row >> 3) * 128 + (size_t)(row & 7) * 16 + (size_t)(k & 7) * 2;
+}
+
+struct MarkovParams {
+    const unsigned char* U; long long u_stride_bytes;
+    const unsigned char* W1;                  // [V, 256] bf16
+    const unsigned char* W2p;                 // packed tiles
+    const int32_t* x_prev;
+    int R, V, n_tiles, m_tiles;
+    const unsigned char* H; long long h_stride_bytes; int d;
+    const float* w_conf;
+    unsigned char* out; long long out_stride_bytes;
+    float* out_conf;
+    int32_t* dev_status;
+    unsigned char* Ap;                        // workspace: gathered embeddings, packed tiles
+};
+
+// ---- one-time packing of W2 [256, V] into per-tile K-major blobs ---------------------------------
+__global__ void markov_pack_w2_kernel(const __nv_bfloat16* __restrict__ W2, int V, int n_tiles, unsigned char* W2p)
+{
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;      // (n, kc)
+    const long long total = (long long)n_tiles * kTileMN * kKChunks;
+    if (idx >= total) return;
+    const int kc = (int)(idx % kKChunks);
+    const long long n = idx / kKChunks;                                         // global column
+    const int tile = (int)(n / kTileMN), nn = (int)(n % kTileMN);
+    __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = n < V ? W2[(size_t)(kc * 8 + i) * V + n] : __float2bfloat16(0.f);
+    *reinterpret_cast<uint4*>(W2p + (size_t)tile * kTileBytes + packed_offset(nn, kc * 8)) = *reinterpret_cast<uint4*>(v);
+}
+
+// ---- per step: gather W1[x_prev] into packed A tiles ----------------------------------------------
+__global__ void markov_gather_kernel(MarkovParams P)
+{
+    pdl_wait();
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;                       // (row, kc)
+    const int total = P.m_tiles * kTileMN * kKChunks;
+    if (idx >= total) return;
+    const int kc = idx % kKChunks, row = idx / kKChunks;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (row < P.R) {
+        const int x = P.x_prev[row];
+        if (x >= 0 && x < P.V) v = __ldg((const uint4*)(P.W1 + ((size_t)x * kRank + kc * 8) * 2));
+        else if (kc == 0) atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN);
+    }
+    *reinterpret_cast<uint4*>(P.Ap + (size_t)(row / kTileMN) * kTileBytes + packed_offset(row % kTileMN, kc * 8)) = v;
+}
+
+// ---- per step: confidence head, one warp per request -------------------------------------------------
+__global__ void markov_confidence_kernel(MarkovParams P)
+{
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (r >= P.R) return;
+    const int x = P.x_prev[r];
+    double z = 0.0;
+    const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(P.H + (long long)r * P.h_stride_bytes);
+    for (int i = lane; i < P.d; i += 32) z += (double)P.w_conf[i] * (double)__bfloat162float(h[i]);
+    if (x >= 0 && x < P.V) {
+        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(P.W1) + (size_t)x * kRank;
+        for (int i = lane; i < kRank; i += 32) z += (double)P.w_conf[P.d + i] * (double)__bfloat162float(e[i]);
+    }
+    z = warp_sum_f64(z);
+    if (lane == 0) P.out_conf[r] = (float)(1.0 / (1.0 + exp(-z)));
+}
+
+// ---- tcgen05 helpers --------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t smem_addr)
+{
+    // start address, leading byte offset (between the two 16 B K chunks of one MMA) = 2048,
+    // stride byte offset (between 8-row groups) = 128, descriptor version 1, no swizzle
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(kChunkBytes >> 4) << 16) |
+           ((uint64_t)(128 >> 4) << 32) | (1ull << 46);
+}
+// D fp32, A and B bf16, both K-major, N = 128, M = 128
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTileMN >> 3) << 17) |
+                                ((uint32_t)(kTileMN >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(kInstrDesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---- the GEMM: logits = U + E W2, bf16 out ------------------------------------------------------------
+__global__ void __launch_bounds__(kGemmThreads, 1) markov_gemm_kernel(MarkovParams P)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned char* sB = smem;                               // one W2 tile
+    unsigned char* sA = smem + kTileBytes;                  // two embedding tiles
+    __shared__ __align__(8) uint64_t b_full, b_empty, a_full[2], a_empty[2], acc_full[2], acc_empty[2];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        mbar_init(&b_full, 1); mbar_init(&b_empty, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1);
+            mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4);
+        }
+        s_abort = 0;
+        mbar_fence_init();
+    }
+    if (warp == 1) {                                        // TMEM: two accumulators of 128 columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&s_tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    pdl_wait();
+    const uint32_t tmem_base = s_tmem_base;
+    volatile int* abort_flag = &s_abort;
+    auto give_up = [&]() { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; };
+
+    if (warp == 0) {
+        // ---------------- producer: bulk copies of the W2 tile and of the embedding tiles ---------------
+        if (lane == 0) {
+            int t = 0, in = 0;
+            for (int nt = blockIdx.x; nt < P.n_tiles && !*abort_flag; nt += gridDim.x, ++in) {
+                if (!mbar_wait_bounded(&b_empty, ((uint32_t)in & 1u) ^ 1u)) { give_up(); break; }
+                mbar_arrive_expect_tx(&b_full, kTileBytes);
+                bulk_g2s(sB, P.W2p + (size_t)nt * kTileBytes, kTileBytes, &b_full);
+                for (int mt = 0; mt < P.m_tiles; ++mt, ++t) {
+                    const int s = t & 1;
+                    if (!mbar_wait_bounded(&a_empty[s], ((uint32_t)(t >> 1) & 1u) ^ 1u)) { give_up(); break; }
+                    mbar_arrive_expect_tx(&a_full[s], kTileBytes);
+                    bulk_g2s(sA + s * kTileBytes, P.Ap + (size_t)mt * kTileBytes, kTileBytes, &a_full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ---------------------------------------------------------------------
+        if (lane == 0) {
+            int t = 0, in = 0;
+            for (int nt = blockIdx.x; nt < P.n_tiles && !*abort_flag; nt += gridDim.x, ++in) {
+                if (!mbar_wait_bounded(&b_full, (uint32_t)in & 1u)) { give_up(); break; }
+                for (int mt = 0; mt < P.m_tiles; ++mt, ++t) {
+                    const int s = t & 1;
+                    const uint32_t ph = (uint32_t)(t >> 1) & 1u;
+                    if (!mbar_wait_bounded(&a_full[s], ph) || !mbar_wait_bounded(&acc_empty[s], ph ^ 1u)) { give_up(); break; }
+                    tc_fence_after();
+                    const uint32_t a0 = smem_u32(sA + s * kTileBytes), b0 = smem_u32(sB);
+#pragma unroll
+                    for (int ks = 0; ks < kRank / 16; ++ks)
+                        umma_bf16(tmem_base + (uint32_t)(s * kTileMN), smem_desc_kmajor(a0 + ks * 2 * kChunkBytes),
+                                  smem_desc_kmajor(b0 + ks * 2 * kChunkBytes), ks > 0 ? 1u : 0u);
+                    umma_commit(&a_empty[s]);               // the embedding tile may be overwritten
+                    umma_commit(&acc_full[s]);              // the accumulator may be read
+                }
+                umma_commit(&b_empty);                      // the W2 tile may be overwritten
+            }
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> registers, + U, round to bf16, store -----------------------
+        const int q = warp & 3;                             // TMEM lane quarter this warp may access
+        int t = 0;
+        for (int nt = blockIdx.x; nt < P.n_tiles && !*abort_flag; nt += gridDim.x) {
+            for (int mt = 0; mt < P.m_tiles; ++mt, ++t) {
+                const int s = t & 1;
+                if (!__all_sync(0xffffffffu, mbar_wait_bounded(&acc_full[s], (uint32_t)(t >> 1) & 1u))) {
+                    if (lane == 0) give_up();
+                    break;
+                }
+                tc_fence_after();
+                const int row = mt * kTileMN + q * 32 + lane;
+                const bool live = row < P.R;
+                const unsigned char* urow = P.U + (long long)row * P.u_stride_bytes;
+                unsigned char* orow = P.out + (long long)row * P.out_stride_bytes;
+#pragma unroll 1
+                for (int c0 = 0; c0 < kTileMN; c0 += 32) {
+                    float acc[32];
+                    tmem_load32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(s * kTileMN + c0), acc);
+                    const int col = nt * kTileMN + c0;
+                    if (!live || col >= P.V) continue;
+                    const unsigned char* up = urow + (long long)col * 2;
+                    unsigned char* op = orow + (long long)col * 2;
+                    if (col + 32 <= P.V && (((uintptr_t)up | (uintptr_t)op) & 15u) == 0) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            const uint4 u = __ldg((const uint4*)(up + 16 * v4));
+                            const uint32_t uw[4] = {u.x, u.y, u.z, u.w};
+                            uint32_t ow[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[v4 * 8 + 2 * i] + bf16lo(uw[i]),
+                                                                                acc[v4 * 8 + 2 * i + 1] + bf16hi(uw[i]));
+                                ow[i] = *reinterpret_cast<const uint32_t*>(&b2);
+                            }
+                            *reinterpret_cast<uint4*>(op + 16 * v4) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            if (col + i >= P.V) continue;
+                            const float u = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(up)[i]);
+                            reinterpret_cast<__nv_bfloat16*>(op)[i] = __float2bfloat16_rn(acc[i] + u);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[s]);
+            }
+        }
+    }
+    // everyone meets here; then the allocating warp returns the tensor memory
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+__global__ void arange_offsets_kernel(int32_t* off, int n)
+{
+    pdl_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i <= n) off[i] = i;
+}
+
+struct MarkovWs { size_t ap, off, toks, verify, total; };
+static MarkovWs markov_layout(int R, int V)
+{
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const int m_tiles = (R + kTileMN - 1) / kTileMN;
+    MarkovWs w;
+    size_t o = 0;
+    w.ap = o;     o += up((size_t)m_tiles * kTileBytes);
+    w.off = o;    o += up((size_t)(R + 1) * 4);
+    w.toks = o;   o += up((size_t)R * 4);
+    w.verify = o; o += up(dspark_verify_workspace_bytes(R, R, V));
+    w.total = o;
+    return w;
+}
+
+static bool g_gemm_attr_set[64] = {};
+
+}  // namespace dspark
+
+using namespace dspark;
+
+extern "C" {
+
+size_t dspark_markov_w2_packed_bytes(int V)
+{
+    if (V < 1) return 0;
+    return (size_t)((V + kTileMN - 1) / kTileMN) * kTileBytes;
+}
+
+int dspark_markov_pack_w2(const void* W2, int V, void* W2_packed, void* stream)
+{
+    if (!W2 || !W2_packed || V < 1) return DSPARK_ERR_INVALID_ARG;
+    if (((uintptr_t)W2_packed & 15u) != 0) return DSPARK_ERR_ALIGNMENT;
+    const int n_tiles = (V + kTileMN - 1) / kTileMN;
+    const long long total = (long long)n_tiles * kTileMN * kKChunks;
+    markov_pack_w2_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+        (const __nv_bfloat16*)W2, V, n_tiles, (unsigned char*)W2_packed);
+    return launch_status();
+}
+
+size_t dspark_markov_workspace_bytes(int R, int V)
+{
+    if (R < 1 || V < 1) return 0;
+    return markov_layout(R, V).total;
+}
+
+int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                         const int32_t* x_prev, int R, int V,
+                         const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                         void* out_logits, int64_t out_row_stride, float* out_conf, int32_t* dev_status,
+                         void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!U || !W1 || !W2_packed || !x_prev || !out_logits || !dev_status) return DSPARK_ERR_INVALID_ARG;
+    if (R < 1 || V < 1 || u_row_stride < V || out_row_stride < V) return DSPARK_ERR_INVALID_ARG;
+    if (out_conf && (!H || !w_conf || d < 0 || h_row_stride < d)) return DSPARK_ERR_INVALID_ARG;
+    const MarkovWs w = markov_layout(R, V);
+    if (!workspace || workspace_bytes < w.total) return DSPARK_ERR_WORKSPACE;
+    if ((((uintptr_t)workspace) & 255u) || (((uintptr_t)W2_packed | (uintptr_t)W1) & 15u)) return DSPARK_ERR_ALIGNMENT;
+    MarkovParams P;
+    P.U = (const unsigned char*)U; P.u_stride_bytes = (long long)u_row_stride * 2;
+    P.W1 = (const unsigned char*)W1; P.W2p = (const unsigned char*)W2_packed; P.x_prev = x_prev;
+    P.R = R; P.V = V; P.n_tiles = (V + kTileMN - 1) / kTileMN; P.m_tiles = (R + kTileMN - 1) / kTileMN;
+    P.H = (const unsigned char*)H; P.h_stride_bytes = (long long)h_row_stride * 2; P.d = d; P.w_conf = w_conf;
+    P.out = (unsigned char*)out_logits; P.out_stride_bytes = (long long)out_row_stride * 2;
+    P.out_conf = out_conf; P.dev_status = dev_status;
+    P.Ap = (unsigned char*)workspace + w.ap;
+
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int smem_bytes = 3 * kTileBytes;
+    if (!g_gemm_attr_set[dev & 63]) {
+        if (cudaFuncSetAttribute(markov_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
+            return launch_status();
+        g_gemm_attr_set[dev & 63] = true;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    const int gather_threads = P.m_tiles * kTileMN * kKChunks;
+    launch_pdl(markov_gather_kernel, dim3((gather_threads + 255) / 256), dim3(256), 0, s, P);
+    if (out_conf) launch_pdl(markov_confidence_kernel, dim3((R + 7) / 8), dim3(256), 0, s, P);
+    {
+        KernelTimerScope timer(DSPARK_K_MARKOV_GEMM, s);
+        launch_pdl(markov_gemm_kernel, dim3(P.n_tiles < sms ? P.n_tiles : sms), dim3(kGemmThreads), (size_t)smem_bytes, s, P);
+    }
+    return launch_status();
+}
+
+int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                             const int32_t* x_prev, int R, int V,
+                             const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                             float temperature, uint64_t seed,
+                             void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
+                             int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!out_tokens) return DSPARK_ERR_INVALID_ARG;
+    int rc = dspark_markov_logits(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf,
+                                  out_logits, out_row_stride, out_conf, dev_status, workspace, workspace_bytes, stream);
+    if (rc != DSPARK_OK) return rc;
+    const MarkovWs w = markov_layout(R, V);
+    unsigned char* ws = (unsigned char*)workspace;
+    int32_t* off = (int32_t*)(ws + w.off);
+    int32_t* acc = (int32_t*)(ws + w.toks);
+    launch_pdl(arange_offsets_kernel, dim3((R + 256) / 256), dim3(256), 0, (cudaStream_t)stream, off, R);
+    // every request owns exactly one row and no draft position: the verifier's bonus path draws one
+    // token per row from softmax(row / T) with the second uniform of (seed, request, position 0);
+    // the draft-token array is never read for such a batch, the offsets stand in for it
+    if (temperature == 0.f)
+        return dspark_verify_greedy(out_logits, DSPARK_BF16, out_row_stride, V, off, off, R, R, acc, out_tokens,
+                                    dev_status, ws + w.verify, workspace_bytes - w.verify, stream);
+    return dspark_verify(out_logits, out_logits, DSPARK_BF16, out_row_stride, out_row_stride, V, off, nullptr,
+                         off, R, R, temperature, seed, acc, out_tokens,
+                         nullptr, nullptr, dev_status, ws + w.verify, workspace_bytes - w.verify, stream);
+}
+
+}  // extern "C"

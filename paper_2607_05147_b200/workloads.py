@@ -241,6 +241,35 @@ def config_5_batch(lengths, device="cpu", V=V_FULL, block=32, seed=1004):
                           verify_seed=4, block=block)
 
 
+
+@dataclass
+class MarkovInput:
+    """Inputs of one Markov-head draft step (Section 3.1): base logits of the block position, the
+    two low-rank factors, previous tokens, hidden states and confidence weights."""
+    U: torch.Tensor        # bf16 [R, V]
+    W1: torch.Tensor       # bf16 [V, 256]
+    W2: torch.Tensor       # bf16 [256, V]
+    x_prev: torch.Tensor   # int32 [R]
+    H: torch.Tensor        # bf16 [R, d]
+    w_conf: torch.Tensor   # fp32 [d + 256]
+
+
+def markov_input(R: int, V: int, seed: int, device, d: int = 1024, sigma: float = 3.0, chunk: int = 8192) -> MarkovInput:
+    """Seeded synthetic head: logit-like base scores (normal, std sigma), embedding rows of std 0.5 and
+    output factors of std 0.12 (a bias of about unit scale after 256 terms), unit hidden states."""
+    g = _gen(seed, device)
+    U = (torch.randn(R, V, generator=g, device=device) * sigma).to(torch.bfloat16)
+    W1 = torch.empty(V, 256, dtype=torch.bfloat16, device=device)
+    for lo in range(0, V, chunk):
+        hi = min(V, lo + chunk)
+        W1[lo:hi] = (torch.randn(hi - lo, 256, generator=g, device=device) * 0.5).to(torch.bfloat16)
+    W2 = (torch.randn(256, V, generator=g, device=device) * 0.12).to(torch.bfloat16)
+    x_prev = torch.randint(0, V, (R,), generator=g, device=device, dtype=torch.int32)
+    H = torch.randn(R, d, generator=g, device=device).to(torch.bfloat16)
+    w_conf = torch.randn(d + 256, generator=g, device=device) / float(d + 256) ** 0.5
+    return MarkovInput(U, W1, W2, x_prev, H, w_conf)
+
+
 def bf16_bits(t: torch.Tensor):
     """Host numpy view of a tensor for the oracle: fp32 as is, bf16 as raw uint16 patterns."""
     import numpy as np

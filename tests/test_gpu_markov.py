@@ -1,0 +1,115 @@
+"""Markov-head draft step on the GPU vs the oracle (Section 3.1, Eq. markov; Section 3.2.1, Eq. confidence).
+
+Logits: the GPU accumulates the 256 products in fp32 on the tensor cores, adds the base logit in fp32
+and rounds once to bf16; the oracle sums in fp64 and rounds once.  Both are a correct rounding of a
+sum whose fp32 error is far below half a bf16 ulp, so the two agree bit for bit except where the
+exact value sits within that fp32 error of a bf16 rounding boundary: there they differ by one ulp.
+The test bounds the distance to the exact value, the size of a difference (one ulp unless the sum
+cancels to nearly zero) and the share of differing elements.
+Draw: the GPU's stored logits are handed to the oracle's sampler, which must pick the same tokens.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_05147_b200 import binding as B
+from paper_2607_05147_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def _run(m: W.MarkovInput, temperature=None, seed=0, out_stride=None, want_conf=True):
+    R, V = m.U.shape
+    packed = torch.empty(B.dspark_markov_w2_packed_bytes(V), dtype=torch.uint8, device="cuda").fill_(0xFF)
+    B.dspark_markov_pack_w2(m.W2, packed)
+    stride = V if out_stride is None else out_stride
+    out_full = torch.full((R, stride), float("nan"), dtype=torch.bfloat16, device="cuda")
+    out = out_full[:, :V]
+    conf = torch.full((R,), -7.0, dtype=torch.float32, device="cuda") if want_conf else None
+    toks = torch.full((R,), -5, dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = B.workspace(B.dspark_markov_workspace_bytes(R, V)).fill_(0xFF)
+    kw = dict(H=m.H if want_conf else None, w_conf=m.w_conf if want_conf else None, out_logits=out, out_conf=conf,
+              dev_status=st, workspace=ws)
+    if temperature is None:
+        B.dspark_markov_logits(m.U, m.W1, packed, m.x_prev, **kw)
+    else:
+        B.dspark_markov_draft_step(m.U, m.W1, packed, m.x_prev, temperature, seed, out_tokens=toks, **kw)
+    torch.cuda.synchronize()
+    if out_stride is not None and stride > V:
+        assert torch.isnan(out_full[:, V:].float()).all(), "columns past V were written"
+    return out, conf, toks, int(st.item())
+
+
+def _check_logits(m: W.MarkovInput, out: torch.Tensor):
+    exact, want_bits = oracle.markov_logits(W.bf16_bits(m.U), W.bf16_bits(m.W1), W.bf16_bits(m.W2), m.x_prev.cpu().numpy())
+    got_bits = W.bf16_bits(out)
+    got = _bf16_to_f64(got_bits)
+    assert np.isfinite(got).all()
+    # a correct rounding is within half a bf16 ulp (2^-9 relative, 2^-8 after binade effects) of the
+    # exact sum; fp32 accumulation of 257 terms of magnitude <= ~20 adds at most ~1e-4
+    assert (np.abs(got - exact) <= np.abs(exact) * 2.0 ** -8 + 2e-4).all()
+    diff = got_bits.astype(np.int32) - want_bits.astype(np.int32)
+    # near zero the sum cancels, a bf16 ulp shrinks below the fp32 error of the accumulation and the bit
+    # patterns may be several ulps apart; there only the absolute bound above applies
+    sizeable = np.abs(exact) >= 2.0 ** -4
+    assert np.abs(diff[sizeable]).max(initial=0) <= 1
+    share = float((diff != 0).mean())
+    assert share <= 2e-3, share
+    return share
+
+
+@pytest.mark.parametrize("R,V", [(8, 256), (128, 1024), (130, 4097), (300, 2000), (1, 129), (16, W.V_FULL)])
+def test_logits_and_confidence(R, V):
+    m = W.markov_input(R, V, 100 + R, "cuda", d=96 if V < 10_000 else 1024)
+    out, conf, _, st = _run(m)
+    assert st == 0
+    share = _check_logits(m, out)
+    want_c = oracle.confidence(W.bf16_bits(m.H), W.bf16_bits(m.W1), m.w_conf.cpu().numpy(), m.x_prev.cpu().numpy())
+    err = np.abs(conf.cpu().numpy().astype(np.float64) - want_c).max()
+    assert err <= 1e-6
+    print(f"[markov] R={R} V={V}: one-ulp share {share:.2e}, confidence max err {err:.1e}")
+
+
+def test_padded_output_rows_and_no_confidence():
+    m = W.markov_input(40, 3000, 7, "cuda", d=64)
+    out, conf, _, st = _run(m, out_stride=3008, want_conf=False)
+    assert st == 0 and conf is None
+    _check_logits(m, out)
+
+
+def test_bad_previous_token_is_flagged():
+    m = W.markov_input(5, 512, 9, "cuda", d=32)
+    m.x_prev[3] = 512
+    out, _, _, st = _run(m)
+    assert st & B.DEV_BAD_TOKEN
+    # the flagged request gets a zero embedding: its logits are the base logits
+    assert torch.equal(out[3], m.U[3])
+
+
+@pytest.mark.parametrize("R,V,T", [(64, 4097, 1.0), (200, 1500, 0.6), (12, W.V_FULL, 1.0), (33, 5000, 0.0)])
+def test_draft_step_draws_like_the_oracle(R, V, T):
+    m = W.markov_input(R, V, 300 + R, "cuda", d=64)
+    seed = 0xD5A9 + R
+    out, conf, toks, st = _run(m, temperature=T, seed=seed)
+    assert st == 0
+    _check_logits(m, out)
+    bits = W.bf16_bits(out)
+    off = np.arange(R + 1, dtype=np.int32)
+    got = toks.cpu().numpy()
+    if T == 0.0:
+        o = oracle.verify_greedy(bits, off, np.zeros(R, dtype=np.int32))
+        np.testing.assert_array_equal(got, o.out_tokens[:R])
+        return
+    o = oracle.verify(bits, bits, off, np.zeros(R, dtype=np.int32), T, seed)
+    assert (o.accepted_len == 0).all()
+    differ = np.nonzero(got != o.out_tokens[:R])[0]
+    for r in differ:
+        assert o.token_margin[r] < 1e-6, (r, got[r], o.out_tokens[r], o.token_margin[r])
+    assert len(differ) <= max(1, R // 50)
+    assert ((got >= 0) & (got < V)).all()
