@@ -362,6 +362,82 @@ def run_reference(args, rank):
 
 
 # --------------------------------------------------------------------------------- main ----
+def bench_markov(args, device, rank, world, dist, barrier):
+    """One Markov-head draft position for R requests: logits = U + W1[x_prev] W2 on the tensor cores, the
+    confidence head, one draw per request.  Reported beside the verification step, not instead of it."""
+    from paper_2607_05147_b200 import binding as B, replicas, workloads as W
+    R = args.requests or 256
+    V = W.V_FULL
+    n_sets = 3                                   # rotate base logits and outputs: 2 x 66 MB x 3 > L2
+    m = W.markov_input(R, V, 4242 + rank, device)
+    Us = [m.U] + [m.U.roll(i, 0).contiguous() for i in range(1, n_sets)]
+    outs = [torch.empty_like(m.U) for _ in range(n_sets)]
+    packed = torch.empty(B.dspark_markov_w2_packed_bytes(V), dtype=torch.uint8, device=device)
+    B.dspark_markov_pack_w2(m.W2, packed)
+    conf = torch.empty(R, dtype=torch.float32, device=device)
+    toks = torch.empty(R, dtype=torch.int32, device=device)
+    st = torch.zeros(1, dtype=torch.int32, device=device)
+    ws = B.workspace(B.dspark_markov_workspace_bytes(R, V))
+
+    def step(i):
+        B.dspark_markov_draft_step(Us[i % n_sets], m.W1, packed, m.x_prev, 1.0, 77 + i, H=m.H, w_conf=m.w_conf,
+                                   out_logits=outs[i % n_sets], out_tokens=toks, out_conf=conf, dev_status=st, workspace=ws)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(device.index or 0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    t_end = time.perf_counter() + 1.0
+    i = 0
+    while time.perf_counter() < t_end:
+        step(i); i += 1
+        if i % 64 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+    timer = B.KernelTimer(args.steps * 8)
+    timer.attach()
+    for i in range(args.steps):
+        step(i)
+    torch.cuda.synchronize()
+    timer.detach()
+    kernels = timer.read()
+    timer.close()
+    (ms,) = replicas.max_over_ranks([ms], dist, device)
+    if rank != 0:
+        return
+    peaks_file = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peaks = json.load(open(peaks_file)) if os.path.exists(peaks_file) else {}
+    peak = float(peaks.get("hbm_gbs", FALLBACK_HBM_GBS))
+    gemm_bytes = 2 * R * V * 2 + 256 * V * 2 + ((R + 127) // 128) * 65536      # U in, logits out, W2, embeddings
+    k = kernels.get("markov_gemm", {"ms": float("nan"), "launches": 1})
+    gemm_ms = k["ms"] / max(1, k["launches"])
+    achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9
+    flops = 2.0 * ((R + 127) // 128 * 128) * 256 * ((V + 127) // 128 * 128)
+    print(json.dumps({
+        "metric": "markov_draft_rows_per_s", "value": replicas.whole_job_rate(R, args.steps, ms, world), "unit": "rows/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32", "data": "synthetic",
+        "config": {"workload": f"Markov-head draft position, R={R}, V={V}, rank 256, T=1, confidence head d=1024",
+                   "l2": f"{n_sets} base-logit / output buffer pairs rotated ({n_sets * 4 * R * V / 1e6:.0f} MB)"},
+        "roofline": {"bound": "hbm", "kernel": "markov_gemm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_launch": gemm_bytes,
+                     "us_per_launch": gemm_ms * 1e3,
+                     "tensor_tflops": flops / (gemm_ms * 1e-3) / 1e12,
+                     "tensor_frac_of_measured_bf16": flops / (gemm_ms * 1e-3) / 1e12 / float(peaks.get("bf16_tflops", 1590.0))},
+        "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in kernels.items()},
+        "clocks": clocks, "dev_status": int(st.item())}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -382,6 +458,9 @@ def main():
                     help="capture the step (schedule -> verify) in CUDA graphs and time their replay")
     ap.add_argument("--requests", type=int, default=0,
                     help="override the request count of cfg2 / cfg4 (smaller cases for profiler captures)")
+    ap.add_argument("--markov-draft", action="store_true",
+                    help="time the Markov-head draft step (Section 3.1) for --requests rows (default 256) instead of "
+                         "the verification step; prints its own JSON line")
     ap.add_argument("--quick", action="store_true",
                     help="timed steps only (no clock probe, per-kernel timing, e2e or CPU legs): for profiler captures")
     args = ap.parse_args()
@@ -417,6 +496,12 @@ def main():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.markov_draft:
+        bench_markov(args, device, rank, world, dist, barrier)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
 
     def time_workload(name, steps, warmup, with_e2e, with_cpu):
         # enough distinct batches that consecutive steps cannot be served from the 126 MB L2

@@ -305,6 +305,11 @@ int dspark_accept_rate(const void* target_logits, const void* draft_logits, int 
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, CUDA; a device wait that ran out sets
  * DSPARK_DEV_TIMEOUT in *dev_status and the affected logits are unspecified.
  */
+/* Diagnostic switch for the epilogue of dspark_markov_logits: 0 = automatic (base logits and draft
+ * logits move through 2-D tensor-map copies when both base addresses are 16-byte aligned and both
+ * row pitches are multiples of 16 bytes, direct loads and stores otherwise), 1 = always direct.
+ * Same results either way.  Process-wide; the paper has no counterpart. */
+int dspark_markov_set_epilogue_path(int path);
 size_t dspark_markov_w2_packed_bytes(int V);
 int dspark_markov_pack_w2(const void* W2, int V, void* W2_packed, void* stream);
 size_t dspark_markov_workspace_bytes(int R, int V);

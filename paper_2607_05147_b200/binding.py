@@ -32,7 +32,7 @@ EXPORTS = [
     "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity", "dspark_verify_per_request",
     "dspark_accept_rate", "dspark_accept_rate_workspace_bytes",
     "dspark_markov_w2_packed_bytes", "dspark_markov_pack_w2", "dspark_markov_workspace_bytes",
-    "dspark_markov_logits", "dspark_markov_draft_step",
+    "dspark_markov_logits", "dspark_markov_draft_step", "dspark_markov_set_epilogue_path",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
     "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
     "dspark_version",
@@ -80,6 +80,7 @@ def lib() -> C.CDLL:
         L.dspark_accept_rate_workspace_bytes.argtypes = [i32, i32, i32]
         L.dspark_accept_rate_workspace_bytes.restype = sz
         L.dspark_accept_rate.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, i32, C.c_float, vp, vp, vp, sz, vp]
+        L.dspark_markov_set_epilogue_path.argtypes = [i32]
         L.dspark_markov_w2_packed_bytes.argtypes = [i32]
         L.dspark_markov_w2_packed_bytes.restype = sz
         L.dspark_markov_pack_w2.argtypes = [vp, i32, vp, vp]
@@ -343,6 +344,10 @@ def dspark_accept_rate(target: torch.Tensor, draft: torch.Tensor, row_offsets: t
                                   _dev(out_cstar, "out_cstar", torch.float32), _dev(dev_status, "dev_status", torch.int32),
                                   _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_accept_rate")
+
+
+def dspark_markov_set_epilogue_path(path: int) -> None:
+    _check(lib().dspark_markov_set_epilogue_path(int(path)), "dspark_markov_set_epilogue_path")
 
 
 def dspark_markov_w2_packed_bytes(V: int) -> int:

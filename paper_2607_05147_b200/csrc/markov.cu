@@ -12,8 +12,10 @@
 // store the draft logits.  The draw itself is the verifier's bonus path on those stored logits (a
 // request with no draft position emits one token from p), so what the drafter samples from is
 // bit for bit the distribution the verifier will later read as q.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cstdio>
+#include <cstring>
 #include <math.h>
 
 #include "common.cuh"
@@ -146,13 +148,51 @@ __device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&v)[32])
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// ---- the GEMM: logits = U + E W2, bf16 out ------------------------------------------------------------
-__global__ void __launch_bounds__(kGemmThreads, 1) markov_gemm_kernel(MarkovParams P)
+// ---- 2-D tensor-map copies of the base-logit / output tiles ---------------------------------------
+// One box is 64 columns x 128 rows of bf16 (128 B x 128) in the 128-byte swizzle: the 16 B chunk j of
+// row r sits at chunk position j ^ (r & 7), so a thread that owns one row reads its chunks without
+// bank conflicts against the seven neighbouring rows.
+constexpr int kBoxCols = 64;
+constexpr int kBoxBytes = kBoxCols * 2 * kTileMN;      // 16 KB
+constexpr int kUTileBytes = 2 * kBoxBytes;             // 128 x 128 bf16
+constexpr int kUBuffers = 3;
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar)
 {
-    extern __shared__ __align__(1024) unsigned char smem[];
-    unsigned char* sB = smem;                               // one W2 tile
-    unsigned char* sA = smem + kTileBytes;                  // two embedding tiles
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(src))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// ---- the GEMM: logits = U + E W2, bf16 out ------------------------------------------------------------
+// Roles: warp 0 brings the W2 tile (64 KB) and the two K halves of each embedding tile (32 KB each) in
+// with 1-D bulk copies; warp 1 owns the tensor memory and issues the MMAs; warps 2..5 run the epilogue.
+// kTma: base-logit tiles arrive by 2-D tensor-map loads in a ring of three buffers, the epilogue adds
+// the accumulator in place and the finished tile leaves by a tensor-map store, so every byte of HBM
+// traffic is moved by the copy engine.  Otherwise (a base address or row pitch that breaks the 16-byte
+// rules) the epilogue threads load and store their rows directly.
+template <bool kTma>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_out)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzle atoms: 1 KB
+    unsigned char* sU = smem;                               // three base-logit / output tiles
+    unsigned char* sB = smem + kUBuffers * kUTileBytes;     // one W2 tile
+    unsigned char* sA = sB + kTileBytes;                    // one embedding tile, as two K halves
     __shared__ __align__(8) uint64_t b_full, b_empty, a_full[2], a_empty[2], acc_full[2], acc_empty[2];
+    __shared__ __align__(8) uint64_t u_full[kUBuffers], epi_done;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -163,6 +203,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) markov_gemm_kernel(MarkovPara
             mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1);
             mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4);
         }
+        for (int s = 0; s < kUBuffers; ++s) mbar_init(&u_full[s], 1);
+        mbar_init(&epi_done, 4);
         s_abort = 0;
         mbar_fence_init();
     }
@@ -178,58 +220,123 @@ __global__ void __launch_bounds__(kGemmThreads, 1) markov_gemm_kernel(MarkovPara
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
     auto give_up = [&]() { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; };
+    const int my_ntiles = blockIdx.x < P.n_tiles ? (P.n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int my_tiles = my_ntiles * P.m_tiles;             // tile t: n-tile blockIdx.x + (t / m_tiles) * gridDim.x
 
     if (warp == 0) {
-        // ---------------- producer: bulk copies of the W2 tile and of the embedding tiles ---------------
+        // ---------------- producer: bulk copies of the W2 tile and of the embedding halves --------------
         if (lane == 0) {
-            int t = 0, in = 0;
-            for (int nt = blockIdx.x; nt < P.n_tiles && !*abort_flag; nt += gridDim.x, ++in) {
+            int t = 0;
+            for (int in = 0; in < my_ntiles && !*abort_flag; ++in) {
+                const int nt = blockIdx.x + in * gridDim.x;
                 if (!mbar_wait_bounded(&b_empty, ((uint32_t)in & 1u) ^ 1u)) { give_up(); break; }
                 mbar_arrive_expect_tx(&b_full, kTileBytes);
                 bulk_g2s(sB, P.W2p + (size_t)nt * kTileBytes, kTileBytes, &b_full);
-                for (int mt = 0; mt < P.m_tiles; ++mt, ++t) {
-                    const int s = t & 1;
-                    if (!mbar_wait_bounded(&a_empty[s], ((uint32_t)(t >> 1) & 1u) ^ 1u)) { give_up(); break; }
-                    mbar_arrive_expect_tx(&a_full[s], kTileBytes);
-                    bulk_g2s(sA + s * kTileBytes, P.Ap + (size_t)mt * kTileBytes, kTileBytes, &a_full[s]);
+                for (int mt = 0; mt < P.m_tiles && !*abort_flag; ++mt, ++t) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (!mbar_wait_bounded(&a_empty[h], ((uint32_t)t & 1u) ^ 1u)) { give_up(); break; }
+                        mbar_arrive_expect_tx(&a_full[h], kTileBytes / 2);
+                        bulk_g2s(sA + h * (kTileBytes / 2), P.Ap + (size_t)mt * kTileBytes + h * (kTileBytes / 2),
+                                 kTileBytes / 2, &a_full[h]);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ---------------------------------------------------------------------
         if (lane == 0) {
-            int t = 0, in = 0;
-            for (int nt = blockIdx.x; nt < P.n_tiles && !*abort_flag; nt += gridDim.x, ++in) {
+            int t = 0;
+            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
+            for (int in = 0; in < my_ntiles && !*abort_flag; ++in) {
                 if (!mbar_wait_bounded(&b_full, (uint32_t)in & 1u)) { give_up(); break; }
-                for (int mt = 0; mt < P.m_tiles; ++mt, ++t) {
+                for (int mt = 0; mt < P.m_tiles && !*abort_flag; ++mt, ++t) {
                     const int s = t & 1;
-                    const uint32_t ph = (uint32_t)(t >> 1) & 1u;
-                    if (!mbar_wait_bounded(&a_full[s], ph) || !mbar_wait_bounded(&acc_empty[s], ph ^ 1u)) { give_up(); break; }
-                    tc_fence_after();
-                    const uint32_t a0 = smem_u32(sA + s * kTileBytes), b0 = smem_u32(sB);
+                    if (!mbar_wait_bounded(&acc_empty[s], ((uint32_t)(t >> 1) & 1u) ^ 1u)) { give_up(); break; }
 #pragma unroll
-                    for (int ks = 0; ks < kRank / 16; ++ks)
-                        umma_bf16(tmem_base + (uint32_t)(s * kTileMN), smem_desc_kmajor(a0 + ks * 2 * kChunkBytes),
-                                  smem_desc_kmajor(b0 + ks * 2 * kChunkBytes), ks > 0 ? 1u : 0u);
-                    umma_commit(&a_empty[s]);               // the embedding tile may be overwritten
+                    for (int h = 0; h < 2; ++h) {
+                        if (!mbar_wait_bounded(&a_full[h], (uint32_t)t & 1u)) { give_up(); break; }
+                        tc_fence_after();
+#pragma unroll
+                        for (int i = 0; i < kRank / 32; ++i) {
+                            const int ks = h * (kRank / 32) + i;
+                            umma_bf16(tmem_base + (uint32_t)(s * kTileMN), smem_desc_kmajor(a0 + ks * 2 * kChunkBytes),
+                                      smem_desc_kmajor(b0 + ks * 2 * kChunkBytes), ks > 0 ? 1u : 0u);
+                        }
+                        umma_commit(&a_empty[h]);           // this half of the embedding tile may be overwritten
+                    }
                     umma_commit(&acc_full[s]);              // the accumulator may be read
                 }
                 umma_commit(&b_empty);                      // the W2 tile may be overwritten
             }
         }
     } else {
-        // ---------------- epilogue: TMEM -> registers, + U, round to bf16, store -----------------------
+        // ---------------- epilogue: accumulator + base logits -> bf16 ------------------------------------
         const int q = warp & 3;                             // TMEM lane quarter this warp may access
-        int t = 0;
-        for (int nt = blockIdx.x; nt < P.n_tiles && !*abort_flag; nt += gridDim.x) {
-            for (int mt = 0; mt < P.m_tiles; ++mt, ++t) {
-                const int s = t & 1;
-                if (!__all_sync(0xffffffffu, mbar_wait_bounded(&acc_full[s], (uint32_t)(t >> 1) & 1u))) {
-                    if (lane == 0) give_up();
-                    break;
+        const int trow = q * 32 + lane;                     // row of the tile this thread owns
+        const bool leader = kTma && warp == 2 && lane == 0;
+        auto issue_u_load = [&](int t) {
+            const int nt = blockIdx.x + (t / P.m_tiles) * gridDim.x, mt = t % P.m_tiles;
+            unsigned char* dst = sU + (t % kUBuffers) * kUTileBytes;
+            mbar_arrive_expect_tx(&u_full[t % kUBuffers], kUTileBytes);
+            tma_load_2d(dst, &map_u, nt * kTileMN, mt * kTileMN, &u_full[t % kUBuffers]);
+            tma_load_2d(dst + kBoxBytes, &map_u, nt * kTileMN + kBoxCols, mt * kTileMN, &u_full[t % kUBuffers]);
+        };
+        if (leader) {
+            if (my_tiles > 0) issue_u_load(0);
+            if (my_tiles > 1) issue_u_load(1);
+        }
+        for (int t = 0; t < my_tiles && !*abort_flag; ++t) {
+            const int nt = blockIdx.x + (t / P.m_tiles) * gridDim.x, mt = t % P.m_tiles;
+            const int s = t & 1, ub = t % kUBuffers;
+            bool ok = mbar_wait_bounded(&acc_full[s], (uint32_t)(t >> 1) & 1u);
+            if (kTma) ok = ok && mbar_wait_bounded(&u_full[ub], (uint32_t)(t / kUBuffers) & 1u);
+            if (!__all_sync(0xffffffffu, ok)) {
+                if (lane == 0) give_up();
+                break;
+            }
+            tc_fence_after();
+            if (kTma) {
+                unsigned char* tile = sU + ub * kUTileBytes;
+#pragma unroll 1
+                for (int c0 = 0; c0 < kTileMN; c0 += 32) {
+                    float acc[32];
+                    tmem_load32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(s * kTileMN + c0), acc);
+                    unsigned char* rowp = tile + (c0 >> 6) * kBoxBytes + trow * 128;
+                    const int j0 = (c0 & 63) >> 3;
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        uint4* cell = reinterpret_cast<uint4*>(rowp + (((j0 + v4) ^ (trow & 7)) << 4));
+                        const uint4 u = *cell;
+                        const uint32_t uw[4] = {u.x, u.y, u.z, u.w};
+                        uint32_t ow[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[v4 * 8 + 2 * i] + bf16lo(uw[i]),
+                                                                            acc[v4 * 8 + 2 * i + 1] + bf16hi(uw[i]));
+                            ow[i] = *reinterpret_cast<const uint32_t*>(&b2);
+                        }
+                        *cell = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                    }
                 }
-                tc_fence_after();
-                const int row = mt * kTileMN + q * 32 + lane;
+                tc_fence_before();
+                fence_proxy_async_smem();                   // the tile is read next by the copy engine
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(&acc_empty[s]); mbar_arrive(&epi_done); }
+                if (leader) {
+                    if (!mbar_wait_bounded(&epi_done, (uint32_t)t & 1u)) {
+                        give_up();                          // the loop condition ends every warp's walk
+                    } else {
+                        tma_store_2d(&map_out, nt * kTileMN, mt * kTileMN, tile);
+                        tma_store_2d(&map_out, nt * kTileMN + kBoxCols, mt * kTileMN, tile + kBoxBytes);
+                        bulk_commit_group();
+                        bulk_wait_group_read<1>();          // the store of tile t-1 has left its buffer
+                        if (t + 2 < my_tiles) issue_u_load(t + 2);
+                    }
+                }
+                __syncwarp();
+            } else {
+                const int row = mt * kTileMN + trow;
                 const bool live = row < P.R;
                 const unsigned char* urow = P.U + (long long)row * P.u_stride_bytes;
                 unsigned char* orow = P.out + (long long)row * P.out_stride_bytes;
@@ -269,6 +376,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) markov_gemm_kernel(MarkovPara
                 if (lane == 0) mbar_arrive(&acc_empty[s]);
             }
         }
+        if (leader) bulk_wait_group_read<0>();              // shared memory stays valid until the stores have read it
     }
     // everyone meets here; then the allocating warp returns the tensor memory
     tc_fence_before();
@@ -302,12 +410,55 @@ static MarkovWs markov_layout(int R, int V)
 }
 
 static bool g_gemm_attr_set[64] = {};
+static int g_markov_path = 0;   // 0: tensor-map epilogue when the 16-byte rules hold, 1: always direct
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against the driver)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool looked = false;
+    if (!looked) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+        else
+            cudaGetLastError();
+        looked = true;
+    }
+    return fn;
+}
+// bf16 matrix [rows, cols] with a row pitch in bytes, boxes of 64 columns x 128 rows, 128-byte swizzle;
+// reads outside the matrix give zeros, writes outside are dropped
+static bool make_tile_map(CUtensorMap* map, const void* base, int rows, int cols, long long pitch_bytes)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || ((uintptr_t)base & 15u) || (pitch_bytes & 15) || pitch_bytes <= 0) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)pitch_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)kBoxCols, (cuuint32_t)kTileMN};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 }  // namespace dspark
 
 using namespace dspark;
 
 extern "C" {
+
+int dspark_markov_set_epilogue_path(int path)
+{
+    if (path != 0 && path != 1) return DSPARK_ERR_INVALID_ARG;
+    g_markov_path = path;
+    return DSPARK_OK;
+}
 
 size_t dspark_markov_w2_packed_bytes(int V)
 {
@@ -356,19 +507,27 @@ int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, co
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int smem_bytes = 3 * kTileBytes;
+    const int smem_bytes = kUBuffers * kUTileBytes + 2 * kTileBytes + 1024;
     if (!g_gemm_attr_set[dev & 63]) {
-        if (cudaFuncSetAttribute(markov_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(markov_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess ||
+            cudaFuncSetAttribute(markov_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
             return launch_status();
         g_gemm_attr_set[dev & 63] = true;
     }
+    CUtensorMap map_u, map_out;
+    memset(&map_u, 0, sizeof map_u);
+    memset(&map_out, 0, sizeof map_out);
+    const bool tma = g_markov_path != 1 && make_tile_map(&map_u, U, R, V, P.u_stride_bytes) &&
+                     make_tile_map(&map_out, out_logits, R, V, P.out_stride_bytes);
     cudaStream_t s = (cudaStream_t)stream;
     const int gather_threads = P.m_tiles * kTileMN * kKChunks;
     launch_pdl(markov_gather_kernel, dim3((gather_threads + 255) / 256), dim3(256), 0, s, P);
     if (out_conf) launch_pdl(markov_confidence_kernel, dim3((R + 7) / 8), dim3(256), 0, s, P);
     {
         KernelTimerScope timer(DSPARK_K_MARKOV_GEMM, s);
-        launch_pdl(markov_gemm_kernel, dim3(P.n_tiles < sms ? P.n_tiles : sms), dim3(kGemmThreads), (size_t)smem_bytes, s, P);
+        const dim3 grid(P.n_tiles < sms ? P.n_tiles : sms);
+        if (tma) launch_pdl(markov_gemm_kernel<true>, grid, dim3(kGemmThreads), (size_t)smem_bytes, s, P, map_u, map_out);
+        else launch_pdl(markov_gemm_kernel<false>, grid, dim3(kGemmThreads), (size_t)smem_bytes, s, P, map_u, map_out);
     }
     return launch_status();
 }

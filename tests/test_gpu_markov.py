@@ -83,6 +83,19 @@ def test_padded_output_rows_and_no_confidence():
     _check_logits(m, out)
 
 
+def test_direct_epilogue_gives_the_same_logits():
+    m = W.markov_input(150, 2048, 11, "cuda", d=64)
+    a, _, _, st_a = _run(m)
+    B.dspark_markov_set_epilogue_path(1)
+    try:
+        b, _, _, st_b = _run(m)
+    finally:
+        B.dspark_markov_set_epilogue_path(0)
+    assert st_a == 0 and st_b == 0
+    assert torch.equal(a, b)
+    _check_logits(m, a)
+
+
 def test_bad_previous_token_is_flagged():
     m = W.markov_input(5, 512, 9, "cuda", d=32)
     m.x_prev[3] = 512
