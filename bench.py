@@ -368,6 +368,7 @@ def bench_markov(args, device, rank, world, dist, barrier):
     from paper_2607_05147_b200 import binding as B, replicas, workloads as W
     R = args.requests or 256
     V = W.V_FULL
+    B.dspark_markov_set_epilogue_path(args.markov_epilogue)
     n_sets = 3                                   # rotate base logits and outputs: 2 x 66 MB x 3 > L2
     m = W.markov_input(R, V, 4242 + rank, device)
     Us = [m.U] + [m.U.roll(i, 0).contiguous() for i in range(1, n_sets)]
@@ -418,9 +419,9 @@ def bench_markov(args, device, rank, world, dist, barrier):
     peaks_file = os.path.join(ROOT, "MEASURED_PEAKS.json")
     peaks = json.load(open(peaks_file)) if os.path.exists(peaks_file) else {}
     peak = float(peaks.get("hbm_gbs", FALLBACK_HBM_GBS))
-    gemm_bytes = 2 * R * V * 2 + 256 * V * 2 + ((R + 127) // 128) * 65536      # U in, logits out, W2, embeddings
+    gemm_bytes = 2 * R * V * 2 + 256 * V * 2 + R * 512       # base logits in, draft logits out, W2 once, embeddings
     k = kernels.get("markov_gemm", {"ms": float("nan"), "launches": 1})
-    gemm_ms = k["ms"] / max(1, k["launches"])
+    gemm_ms = k["ms"] / args.steps              # one launch per group of 256 rows
     achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9
     flops = 2.0 * ((R + 127) // 128 * 128) * 256 * ((V + 127) // 128 * 128)
     print(json.dumps({
@@ -431,7 +432,7 @@ def bench_markov(args, device, rank, world, dist, barrier):
                    "l2": f"{n_sets} base-logit / output buffer pairs rotated ({n_sets * 4 * R * V / 1e6:.0f} MB)"},
         "roofline": {"bound": "hbm", "kernel": "markov_gemm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_launch": gemm_bytes,
-                     "us_per_launch": gemm_ms * 1e3,
+                     "us_per_launch": gemm_ms * 1e3, "launches_per_step": k["launches"] // max(1, args.steps),
                      "tensor_tflops": flops / (gemm_ms * 1e-3) / 1e12,
                      "tensor_frac_of_measured_bf16": flops / (gemm_ms * 1e-3) / 1e12 / float(peaks.get("bf16_tflops", 1590.0))},
         "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in kernels.items()},
@@ -461,6 +462,7 @@ def main():
     ap.add_argument("--markov-draft", action="store_true",
                     help="time the Markov-head draft step (Section 3.1) for --requests rows (default 256) instead of "
                          "the verification step; prints its own JSON line")
+    ap.add_argument("--markov-epilogue", type=int, default=0, help="epilogue path of the Markov GEMM (diagnostic)")
     ap.add_argument("--quick", action="store_true",
                     help="timed steps only (no clock probe, per-kernel timing, e2e or CPU legs): for profiler captures")
     args = ap.parse_args()

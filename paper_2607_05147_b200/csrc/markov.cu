@@ -4,14 +4,23 @@
 // followed by one draw per request from softmax(logits / T) and the confidence
 //     c[r] = sigmoid(w^T [h_k[r] ; W1[x_prev[r]]])          (Section 3.2.1, Eq. confidence).
 //
-// The bias is a dense [R,256] x [256,V] contraction, so it runs on the 5th-generation tensor cores:
-// one persistent CTA per SM walks 128-column tiles of the vocabulary; a producer thread brings the
-// pre-packed W2 tile and the gathered embedding tiles into shared memory with bulk async copies, one
-// thread issues tcgen05.mma (M = N = 128, K = 16 x 16) into one of two TMEM accumulators, and four
-// epilogue warps read the accumulator back (tcgen05.ld), add the base logits, round to bf16 and
-// store the draft logits.  The draw itself is the verifier's bonus path on those stored logits (a
-// request with no draft position emits one token from p), so what the drafter samples from is
-// bit for bit the distribution the verifier will later read as q.
+// The bias is a dense [R,256] x [256,V] contraction, so it runs on the 5th-generation tensor cores,
+// but the step as a whole is bound by HBM (base logits in, draft logits out, W2 once), and the kernel
+// is organised around keeping those three streams in flight:
+//   * one persistent CTA per SM walks 128-column tiles of the vocabulary, 256 rows (two row tiles) per
+//     launch;
+//   * the embedding operand E = W1[x_prev] (gathered once by a small kernel) lives in TENSOR MEMORY for
+//     the whole launch: four loader warps (row tile 0) and the four epilogue warps (row tile 1) write
+//     their rows with tcgen05.st, lane = row, 128 columns of two bf16;
+//   * shared memory then holds the pre-packed W2 tile twice (the next vocabulary tile streams in by one
+//     64 KB bulk copy while the current one is multiplied) and three base-logit tiles;
+//   * one thread issues tcgen05.mma (M = N = 128, 16 steps of K = 16, A from tensor memory, B through a
+//     shared-memory descriptor) into one of two fp32 accumulators in tensor memory;
+//   * base-logit tiles arrive by 2-D tensor-map loads, the epilogue warps read the accumulator back
+//     (tcgen05.ld), add it in place, round to bf16, and the finished tile leaves by a tensor-map store.
+// The draw itself is the verifier's bonus path on the stored logits (a request with no draft position
+// emits one token from p), so what the drafter samples from is bit for bit the distribution the
+// verifier will later read as q.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cstdio>
@@ -24,18 +33,19 @@ namespace dspark {
 
 constexpr int kRank = 256;                       // r of the low-rank factorization
 constexpr int kTileMN = 128;                     // M and N of one MMA tile
-constexpr int kTileBytes = kTileMN * kRank * 2;  // 64 KB of bf16: one packed operand tile
+constexpr int kTileBytes = kTileMN * kRank * 2;  // 64 KB of bf16: one packed W2 tile
 constexpr int kKChunks = kRank / 8;              // 16-byte chunks along K
-constexpr int kChunkBytes = kTileMN * 16;        // one K chunk of a tile: 128 rows x 16 B
-constexpr int kGemmThreads = 192;                // producer warp, MMA warp, four epilogue warps
-constexpr int kTmemCols = 256;                   // two fp32 accumulators of 128 columns
+constexpr int kChunkBytes = kTileMN * 16;        // one K chunk of a tile: 128 columns x 16 B
+constexpr int kGroupRows = 2 * kTileMN;          // rows per launch: two row tiles resident in tensor memory
+constexpr int kGemmThreads = 320;                // producer, MMA, 4 epilogue warps, 4 loader warps
+constexpr int kTmemCols = 512;                   // accumulators: columns 0..255, embedding tiles: 256..511
 
-// Packed operand tile (K-major, no swizzle): element (row, k) of a 128 x 256 tile lives at
-//   (k / 8) * 2048 + (row / 8) * 128 + (row % 8) * 16 + (k % 8) * 2   bytes,
+// Packed W2 tile (K-major, no swizzle): element (n, k) of a 128-column x 256 tile lives at
+//   (k / 8) * 2048 + (n / 8) * 128 + (n % 8) * 16 + (k % 8) * 2   bytes,
 // i.e. 8 x 16 B core matrices, 16 of them per K chunk.
-__host__ __device__ inline size_t packed_offset(int row, int k)
+__host__ __device__ inline size_t packed_offset(int n, int k)
 {
-    return (size_t)(k >> 3) * kChunkBytes + (size_t)(row >> 3) * 128 + (size_t)(row & 7) * 16 + (size_t)(k & 7) * 2;
+    return (size_t)(k >> 3) * kChunkBytes + (size_t)(n >> 3) * 128 + (size_t)(n & 7) * 16 + (size_t)(k & 7) * 2;
 }
 
 struct MarkovParams {
@@ -43,13 +53,16 @@ struct MarkovParams {
     const unsigned char* W1;                  // [V, 256] bf16
     const unsigned char* W2p;                 // packed tiles
     const int32_t* x_prev;
-    int R, V, n_tiles, m_tiles;
+    int R, V, n_tiles, m_tiles;               // for the GEMM: rows and row tiles of this launch's group
     const unsigned char* H; long long h_stride_bytes; int d;
     const float* w_conf;
     unsigned char* out; long long out_stride_bytes;
     float* out_conf;
     int32_t* dev_status;
-    unsigned char* Ap;                        // workspace: gathered embeddings, packed tiles
+    unsigned char* E;                         // workspace: gathered embeddings [rows padded to 128, 256] bf16
+#ifdef DSPARK_MARKOV_TRACE
+    unsigned long long* trace;                // 64 clock stamps per CTA (development aid)
+#endif
 };
 
 // ---- one-time packing of W2 [256, V] into per-tile K-major blobs ---------------------------------
@@ -67,13 +80,12 @@ __global__ void markov_pack_w2_kernel(const __nv_bfloat16* __restrict__ W2, int 
     *reinterpret_cast<uint4*>(W2p + (size_t)tile * kTileBytes + packed_offset(nn, kc * 8)) = *reinterpret_cast<uint4*>(v);
 }
 
-// ---- per step: gather W1[x_prev] into packed A tiles ----------------------------------------------
-__global__ void markov_gather_kernel(MarkovParams P)
+// ---- per step: E = W1[x_prev], rows past R zero -------------------------------------------------------
+__global__ void markov_gather_kernel(MarkovParams P, int rows_padded)
 {
     pdl_wait();
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;                       // (row, kc)
-    const int total = P.m_tiles * kTileMN * kKChunks;
-    if (idx >= total) return;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;                       // (row, 16-byte chunk)
+    if (idx >= rows_padded * kKChunks) return;
     const int kc = idx % kKChunks, row = idx / kKChunks;
     uint4 v = make_uint4(0, 0, 0, 0);
     if (row < P.R) {
@@ -81,7 +93,7 @@ __global__ void markov_gather_kernel(MarkovParams P)
         if (x >= 0 && x < P.V) v = __ldg((const uint4*)(P.W1 + ((size_t)x * kRank + kc * 8) * 2));
         else if (kc == 0) atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN);
     }
-    *reinterpret_cast<uint4*>(P.Ap + (size_t)(row / kTileMN) * kTileBytes + packed_offset(row % kTileMN, kc * 8)) = v;
+    reinterpret_cast<uint4*>(P.E)[idx] = v;
 }
 
 // ---- per step: confidence head, one warp per request -------------------------------------------------
@@ -107,7 +119,7 @@ __global__ void markov_confidence_kernel(MarkovParams P)
 __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t smem_addr)
 {
     // start address, leading byte offset (between the two 16 B K chunks of one MMA) = 2048,
-    // stride byte offset (between 8-row groups) = 128, descriptor version 1, no swizzle
+    // stride byte offset (between 8-column groups) = 128, descriptor version 1, no swizzle
     return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(kChunkBytes >> 4) << 16) |
            ((uint64_t)(128 >> 4) << 32) | (1ull << 46);
 }
@@ -115,12 +127,13 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t smem_addr)
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTileMN >> 3) << 17) |
                                 ((uint32_t)(kTileMN >> 4) << 24);
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
+// D[tmem] (+)= A[tmem] * B[smem descriptor]
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(kInstrDesc), "r"(accumulate)
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(b_desc), "r"(kInstrDesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar)
@@ -130,6 +143,7 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// 32 consecutive fp32 columns of this thread's lane
 __device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&v)[32])
 {
     uint32_t r[32];
@@ -146,6 +160,34 @@ __device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&v)[32])
         : "memory");
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_store32(uint32_t taddr, const uint4 (&w)[8])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(w[0].x), "r"(w[0].y), "r"(w[0].z), "r"(w[0].w), "r"(w[1].x), "r"(w[1].y), "r"(w[1].z), "r"(w[1].w),
+          "r"(w[2].x), "r"(w[2].y), "r"(w[2].z), "r"(w[2].w), "r"(w[3].x), "r"(w[3].y), "r"(w[3].z), "r"(w[3].w),
+          "r"(w[4].x), "r"(w[4].y), "r"(w[4].z), "r"(w[4].w), "r"(w[5].x), "r"(w[5].y), "r"(w[5].z), "r"(w[5].w),
+          "r"(w[6].x), "r"(w[6].y), "r"(w[6].z), "r"(w[6].w), "r"(w[7].x), "r"(w[7].y), "r"(w[7].z), "r"(w[7].w)
+        : "memory");
+}
+
+// One row of an embedding tile: 512 B of E into registers (all 32 loads in flight at once), then into
+// this thread's lane of tensor memory, columns taddr .. taddr + 127 (two bf16 per column, k ascending).
+__device__ __forceinline__ void embedding_row_to_tmem(const unsigned char* E, int row, uint32_t taddr)
+{
+    const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)row * kRank * 2);
+    uint4 w[4][8];
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int v = 0; v < 8; ++v) w[c][v] = src[c * 8 + v];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) tmem_store32(taddr + (uint32_t)(c * 32), w[c]);
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    tc_fence_before();
 }
 
 // ---- 2-D tensor-map copies of the base-logit / output tiles ---------------------------------------
@@ -175,13 +217,23 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_group_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// ---- the GEMM: logits = U + E W2, bf16 out ------------------------------------------------------------
-// Roles: warp 0 brings the W2 tile (64 KB) and the two K halves of each embedding tile (32 KB each) in
-// with 1-D bulk copies; warp 1 owns the tensor memory and issues the MMAs; warps 2..5 run the epilogue.
-// kTma: base-logit tiles arrive by 2-D tensor-map loads in a ring of three buffers, the epilogue adds
-// the accumulator in place and the finished tile leaves by a tensor-map store, so every byte of HBM
-// traffic is moved by the copy engine.  Otherwise (a base address or row pitch that breaks the 16-byte
-// rules) the epilogue threads load and store their rows directly.
+// acc (fp32) + base logits (bf16 pairs) -> bf16 pairs, round to nearest even
+__device__ __forceinline__ uint4 add_round(const float* acc, uint4 u)
+{
+    const uint32_t uw[4] = {u.x, u.y, u.z, u.w};
+    uint32_t ow[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[2 * i] + bf16lo(uw[i]), acc[2 * i + 1] + bf16hi(uw[i]));
+        ow[i] = *reinterpret_cast<const uint32_t*>(&b2);
+    }
+    return make_uint4(ow[0], ow[1], ow[2], ow[3]);
+}
+
+// ---- the GEMM: logits = U + E W2 for one group of at most 256 rows, bf16 out -------------------------
+// kTma: base-logit tiles and finished tiles move through the tensor maps (ring of three buffers, added
+// in place).  Otherwise (a base address or row pitch that breaks the 16-byte rules) the epilogue
+// threads load and store their rows directly.
 template <bool kTma>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_out)
@@ -189,18 +241,17 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzle atoms: 1 KB
     unsigned char* sU = smem;                               // three base-logit / output tiles
-    unsigned char* sB = smem + kUBuffers * kUTileBytes;     // one W2 tile
-    unsigned char* sA = sB + kTileBytes;                    // one embedding tile, as two K halves
-    __shared__ __align__(8) uint64_t b_full, b_empty, a_full[2], a_empty[2], acc_full[2], acc_empty[2];
+    unsigned char* sB = smem + kUBuffers * kUTileBytes;     // two W2 tiles
+    __shared__ __align__(8) uint64_t b_full[2], b_empty[2], a_full[2], acc_full[2], acc_empty[2];
     __shared__ __align__(8) uint64_t u_full[kUBuffers], epi_done;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        mbar_init(&b_full, 1); mbar_init(&b_empty, 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1);
+            mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1);
+            mbar_init(&a_full[s], 4);
             mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4);
         }
         for (int s = 0; s < kUBuffers; ++s) mbar_init(&u_full[s], 1);
@@ -208,7 +259,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
         s_abort = 0;
         mbar_fence_init();
     }
-    if (warp == 1) {                                        // TMEM: two accumulators of 128 columns
+    if (warp == 1) {                                        // the whole tensor memory of this SM
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&s_tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -216,64 +267,74 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    pdl_wait();
+    // The packed W2 is a weight, not a result of the previous kernel on the stream: the producer starts
+    // on it at once; every other role first waits for that kernel (gathered rows, base logits).
+#ifdef DSPARK_MARKOV_TRACE
+    unsigned long long* tr = P.trace + (size_t)blockIdx.x * 64;
+    auto stamp = [&](int slot) { if (slot < 64) tr[slot] = clock64(); };
+#else
+    auto stamp = [](int) {};
+#endif
+    if (tid == 32) stamp(0);
+    if (warp != 0) pdl_wait();
+    if (tid == 32) stamp(1);
     const uint32_t tmem_base = s_tmem_base;
+    const uint32_t tmem_a0 = tmem_base + 2 * kTileMN;       // embedding tile mt: columns 256 + 128 mt ..
     volatile int* abort_flag = &s_abort;
     auto give_up = [&]() { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; };
     const int my_ntiles = blockIdx.x < P.n_tiles ? (P.n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const int my_tiles = my_ntiles * P.m_tiles;             // tile t: n-tile blockIdx.x + (t / m_tiles) * gridDim.x
 
     if (warp == 0) {
-        // ---------------- producer: bulk copies of the W2 tile and of the embedding halves --------------
+        // ---------------- producer: W2 tiles, one ahead ---------------------------------------------------
         if (lane == 0) {
-            int t = 0;
             for (int in = 0; in < my_ntiles && !*abort_flag; ++in) {
-                const int nt = blockIdx.x + in * gridDim.x;
-                if (!mbar_wait_bounded(&b_empty, ((uint32_t)in & 1u) ^ 1u)) { give_up(); break; }
-                mbar_arrive_expect_tx(&b_full, kTileBytes);
-                bulk_g2s(sB, P.W2p + (size_t)nt * kTileBytes, kTileBytes, &b_full);
-                for (int mt = 0; mt < P.m_tiles && !*abort_flag; ++mt, ++t) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (!mbar_wait_bounded(&a_empty[h], ((uint32_t)t & 1u) ^ 1u)) { give_up(); break; }
-                        mbar_arrive_expect_tx(&a_full[h], kTileBytes / 2);
-                        bulk_g2s(sA + h * (kTileBytes / 2), P.Ap + (size_t)mt * kTileBytes + h * (kTileBytes / 2),
-                                 kTileBytes / 2, &a_full[h]);
-                    }
-                }
+                const int nt = blockIdx.x + in * gridDim.x, bs = in & 1;
+                if (!mbar_wait_bounded(&b_empty[bs], ((uint32_t)(in >> 1) & 1u) ^ 1u)) { give_up(); break; }
+                mbar_arrive_expect_tx(&b_full[bs], kTileBytes);
+                bulk_g2s(sB + bs * kTileBytes, P.W2p + (size_t)nt * kTileBytes, kTileBytes, &b_full[bs]);
+                stamp(56 + in);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ---------------------------------------------------------------------
         if (lane == 0) {
             int t = 0;
-            const uint32_t a0 = smem_u32(sA), b0 = smem_u32(sB);
             for (int in = 0; in < my_ntiles && !*abort_flag; ++in) {
-                if (!mbar_wait_bounded(&b_full, (uint32_t)in & 1u)) { give_up(); break; }
+                const int bs = in & 1;
+                if (!mbar_wait_bounded(&b_full[bs], (uint32_t)(in >> 1) & 1u)) { give_up(); break; }
+                const uint32_t b0 = smem_u32(sB + bs * kTileBytes);
+                if (in < 2) stamp(4 + in);
                 for (int mt = 0; mt < P.m_tiles && !*abort_flag; ++mt, ++t) {
                     const int s = t & 1;
-                    if (!mbar_wait_bounded(&acc_empty[s], ((uint32_t)(t >> 1) & 1u) ^ 1u)) { give_up(); break; }
+                    bool ok = mbar_wait_bounded(&acc_empty[s], ((uint32_t)(t >> 1) & 1u) ^ 1u);
+                    if (ok && in == 0) ok = mbar_wait_bounded(&a_full[mt], 0u);      // resident from then on
+                    if (!ok) { give_up(); break; }
+                    tc_fence_after();
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (!mbar_wait_bounded(&a_full[h], (uint32_t)t & 1u)) { give_up(); break; }
-                        tc_fence_after();
-#pragma unroll
-                        for (int i = 0; i < kRank / 32; ++i) {
-                            const int ks = h * (kRank / 32) + i;
-                            umma_bf16(tmem_base + (uint32_t)(s * kTileMN), smem_desc_kmajor(a0 + ks * 2 * kChunkBytes),
-                                      smem_desc_kmajor(b0 + ks * 2 * kChunkBytes), ks > 0 ? 1u : 0u);
-                        }
-                        umma_commit(&a_empty[h]);           // this half of the embedding tile may be overwritten
-                    }
+                    for (int ks = 0; ks < kRank / 16; ++ks)
+                        umma_bf16_ts(tmem_base + (uint32_t)(s * kTileMN), tmem_a0 + (uint32_t)(mt * kTileMN + ks * 8),
+                                     smem_desc_kmajor(b0 + ks * 2 * kChunkBytes), ks > 0 ? 1u : 0u);
                     umma_commit(&acc_full[s]);              // the accumulator may be read
+                    stamp(8 + t);
                 }
-                umma_commit(&b_empty);                      // the W2 tile may be overwritten
+                umma_commit(&b_empty[bs]);                  // the W2 tile may be overwritten
             }
+        }
+    } else if (warp >= 6) {
+        // ---------------- loaders: embedding rows of row tile 0 -> tensor memory -------------------------
+        if (my_tiles > 0) {
+            const int q = warp & 3;
+            embedding_row_to_tmem(P.E, q * 32 + lane, tmem_a0 + ((uint32_t)(q * 32) << 16));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&a_full[0]);
+            if (warp == 6 && lane == 0) stamp(2);
         }
     } else {
         // ---------------- epilogue: accumulator + base logits -> bf16 ------------------------------------
         const int q = warp & 3;                             // TMEM lane quarter this warp may access
         const int trow = q * 32 + lane;                     // row of the tile this thread owns
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const bool leader = kTma && warp == 2 && lane == 0;
         auto issue_u_load = [&](int t) {
             const int nt = blockIdx.x + (t / P.m_tiles) * gridDim.x, mt = t % P.m_tiles;
@@ -282,9 +343,13 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             tma_load_2d(dst, &map_u, nt * kTileMN, mt * kTileMN, &u_full[t % kUBuffers]);
             tma_load_2d(dst + kBoxBytes, &map_u, nt * kTileMN + kBoxCols, mt * kTileMN, &u_full[t % kUBuffers]);
         };
-        if (leader) {
-            if (my_tiles > 0) issue_u_load(0);
-            if (my_tiles > 1) issue_u_load(1);
+        if (leader)
+            for (int t = 0; t < 2 && t < my_tiles; ++t) issue_u_load(t);
+        if (P.m_tiles == 2 && my_tiles > 0) {               // row tile 1, while the pipeline fills
+            embedding_row_to_tmem(P.E, kTileMN + trow, tmem_a0 + lane_base + (uint32_t)kTileMN);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&a_full[1]);
+            if (leader) stamp(3);
         }
         for (int t = 0; t < my_tiles && !*abort_flag; ++t) {
             const int nt = blockIdx.x + (t / P.m_tiles) * gridDim.x, mt = t % P.m_tiles;
@@ -296,27 +361,20 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                 break;
             }
             tc_fence_after();
+            if (leader) stamp(24 + t);
+            const uint32_t acc_addr = tmem_base + lane_base + (uint32_t)(s * kTileMN);
             if (kTma) {
                 unsigned char* tile = sU + ub * kUTileBytes;
 #pragma unroll 1
                 for (int c0 = 0; c0 < kTileMN; c0 += 32) {
                     float acc[32];
-                    tmem_load32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(s * kTileMN + c0), acc);
+                    tmem_load32(acc_addr + (uint32_t)c0, acc);
                     unsigned char* rowp = tile + (c0 >> 6) * kBoxBytes + trow * 128;
                     const int j0 = (c0 & 63) >> 3;
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4) {
                         uint4* cell = reinterpret_cast<uint4*>(rowp + (((j0 + v4) ^ (trow & 7)) << 4));
-                        const uint4 u = *cell;
-                        const uint32_t uw[4] = {u.x, u.y, u.z, u.w};
-                        uint32_t ow[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[v4 * 8 + 2 * i] + bf16lo(uw[i]),
-                                                                            acc[v4 * 8 + 2 * i + 1] + bf16hi(uw[i]));
-                            ow[i] = *reinterpret_cast<const uint32_t*>(&b2);
-                        }
-                        *cell = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                        *cell = add_round(acc + v4 * 8, *cell);
                     }
                 }
                 tc_fence_before();
@@ -332,6 +390,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                         bulk_commit_group();
                         bulk_wait_group_read<1>();          // the store of tile t-1 has left its buffer
                         if (t + 2 < my_tiles) issue_u_load(t + 2);
+                        stamp(40 + t);
                     }
                 }
                 __syncwarp();
@@ -343,25 +402,15 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
 #pragma unroll 1
                 for (int c0 = 0; c0 < kTileMN; c0 += 32) {
                     float acc[32];
-                    tmem_load32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(s * kTileMN + c0), acc);
+                    tmem_load32(acc_addr + (uint32_t)c0, acc);
                     const int col = nt * kTileMN + c0;
                     if (!live || col >= P.V) continue;
                     const unsigned char* up = urow + (long long)col * 2;
                     unsigned char* op = orow + (long long)col * 2;
                     if (col + 32 <= P.V && (((uintptr_t)up | (uintptr_t)op) & 15u) == 0) {
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
-                            const uint4 u = __ldg((const uint4*)(up + 16 * v4));
-                            const uint32_t uw[4] = {u.x, u.y, u.z, u.w};
-                            uint32_t ow[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[v4 * 8 + 2 * i] + bf16lo(uw[i]),
-                                                                                acc[v4 * 8 + 2 * i + 1] + bf16hi(uw[i]));
-                                ow[i] = *reinterpret_cast<const uint32_t*>(&b2);
-                            }
-                            *reinterpret_cast<uint4*>(op + 16 * v4) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-                        }
+                        for (int v4 = 0; v4 < 4; ++v4)
+                            *reinterpret_cast<uint4*>(op + 16 * v4) = add_round(acc + v4 * 8, __ldg((const uint4*)(up + 16 * v4)));
                     } else {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
@@ -381,6 +430,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     // everyone meets here; then the allocating warp returns the tensor memory
     tc_fence_before();
     __syncthreads();
+    if (tid == 32) stamp(63);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
@@ -394,16 +444,20 @@ __global__ void arange_offsets_kernel(int32_t* off, int n)
     if (i <= n) off[i] = i;
 }
 
-struct MarkovWs { size_t ap, off, toks, verify, total; };
+struct MarkovWs { size_t e, off, toks, trace, verify, total; };
 static MarkovWs markov_layout(int R, int V)
 {
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
     const int m_tiles = (R + kTileMN - 1) / kTileMN;
     MarkovWs w;
     size_t o = 0;
-    w.ap = o;     o += up((size_t)m_tiles * kTileBytes);
+    w.e = o;      o += up((size_t)m_tiles * kTileMN * kRank * 2);
     w.off = o;    o += up((size_t)(R + 1) * 4);
     w.toks = o;   o += up((size_t)R * 4);
+    w.trace = o;
+#ifdef DSPARK_MARKOV_TRACE
+    o += up(256 * 64 * 8);
+#endif
     w.verify = o; o += up(dspark_verify_workspace_bytes(R, R, V));
     w.total = o;
     return w;
@@ -502,7 +556,10 @@ int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, co
     P.H = (const unsigned char*)H; P.h_stride_bytes = (long long)h_row_stride * 2; P.d = d; P.w_conf = w_conf;
     P.out = (unsigned char*)out_logits; P.out_stride_bytes = (long long)out_row_stride * 2;
     P.out_conf = out_conf; P.dev_status = dev_status;
-    P.Ap = (unsigned char*)workspace + w.ap;
+    P.E = (unsigned char*)workspace + w.e;
+#ifdef DSPARK_MARKOV_TRACE
+    P.trace = (unsigned long long*)((unsigned char*)workspace + w.trace);
+#endif
 
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
@@ -514,20 +571,28 @@ int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, co
             return launch_status();
         g_gemm_attr_set[dev & 63] = true;
     }
-    CUtensorMap map_u, map_out;
-    memset(&map_u, 0, sizeof map_u);
-    memset(&map_out, 0, sizeof map_out);
-    const bool tma = g_markov_path != 1 && make_tile_map(&map_u, U, R, V, P.u_stride_bytes) &&
-                     make_tile_map(&map_out, out_logits, R, V, P.out_stride_bytes);
     cudaStream_t s = (cudaStream_t)stream;
-    const int gather_threads = P.m_tiles * kTileMN * kKChunks;
-    launch_pdl(markov_gather_kernel, dim3((gather_threads + 255) / 256), dim3(256), 0, s, P);
+    const int rows_padded = P.m_tiles * kTileMN;
+    launch_pdl(markov_gather_kernel, dim3((rows_padded * kKChunks + 255) / 256), dim3(256), 0, s, P, rows_padded);
     if (out_conf) launch_pdl(markov_confidence_kernel, dim3((R + 7) / 8), dim3(256), 0, s, P);
-    {
+    // one launch per group of 256 rows: both row tiles of a group stay in tensor memory while the CTA
+    // walks its vocabulary tiles (W2 is streamed once per group)
+    for (int r0 = 0; r0 < R; r0 += kGroupRows) {
+        MarkovParams G = P;
+        G.R = R - r0 < kGroupRows ? R - r0 : kGroupRows;
+        G.m_tiles = (G.R + kTileMN - 1) / kTileMN;
+        G.U = P.U + (long long)r0 * P.u_stride_bytes;
+        G.out = P.out + (long long)r0 * P.out_stride_bytes;
+        G.E = P.E + (size_t)r0 * kRank * 2;
+        CUtensorMap map_u, map_out;
+        memset(&map_u, 0, sizeof map_u);
+        memset(&map_out, 0, sizeof map_out);
+        const bool tma = g_markov_path != 1 && make_tile_map(&map_u, G.U, G.R, V, P.u_stride_bytes) &&
+                         make_tile_map(&map_out, G.out, G.R, V, P.out_stride_bytes);
         KernelTimerScope timer(DSPARK_K_MARKOV_GEMM, s);
         const dim3 grid(P.n_tiles < sms ? P.n_tiles : sms);
-        if (tma) launch_pdl(markov_gemm_kernel<true>, grid, dim3(kGemmThreads), (size_t)smem_bytes, s, P, map_u, map_out);
-        else launch_pdl(markov_gemm_kernel<false>, grid, dim3(kGemmThreads), (size_t)smem_bytes, s, P, map_u, map_out);
+        if (tma) launch_pdl(markov_gemm_kernel<true>, grid, dim3(kGemmThreads), (size_t)smem_bytes, s, G, map_u, map_out);
+        else launch_pdl(markov_gemm_kernel<false>, grid, dim3(kGemmThreads), (size_t)smem_bytes, s, G, map_u, map_out);
     }
     return launch_status();
 }

@@ -64,7 +64,7 @@ def _check_logits(m: W.MarkovInput, out: torch.Tensor):
     return share
 
 
-@pytest.mark.parametrize("R,V", [(8, 256), (128, 1024), (130, 4097), (300, 2000), (1, 129), (16, W.V_FULL)])
+@pytest.mark.parametrize("R,V", [(8, 256), (128, 1024), (130, 4097), (300, 2000), (1, 129), (600, 4097), (700, 8192), (16, W.V_FULL)])
 def test_logits_and_confidence(R, V):
     m = W.markov_input(R, V, 100 + R, "cuda", d=96 if V < 10_000 else 1024)
     out, conf, _, st = _run(m)
@@ -83,12 +83,13 @@ def test_padded_output_rows_and_no_confidence():
     _check_logits(m, out)
 
 
-def test_direct_epilogue_gives_the_same_logits():
-    m = W.markov_input(150, 2048, 11, "cuda", d=64)
-    a, _, _, st_a = _run(m)
-    B.dspark_markov_set_epilogue_path(1)
+@pytest.mark.parametrize("path,V", [(1, 2048), (1, 3000)])
+def test_epilogue_paths_give_the_same_logits(path, V):
+    m = W.markov_input(150, V, 11, "cuda", d=64)
+    a, _, _, st_a = _run(m, out_stride=3008 if V == 3000 else None)
+    B.dspark_markov_set_epilogue_path(path)
     try:
-        b, _, _, st_b = _run(m)
+        b, _, _, st_b = _run(m, out_stride=3008 if V == 3000 else None)
     finally:
         B.dspark_markov_set_epilogue_path(0)
     assert st_a == 0 and st_b == 0
