@@ -298,10 +298,14 @@ int dspark_accept_rate(const void* target_logits, const void* draft_logits, int 
  *   out_logits   device bf16 [R, >= V], row stride out_row_stride elements
  *   out_conf     device fp32 [R] or NULL
  *   workspace    dspark_markov_workspace_bytes(R, V), 256-byte aligned
- * dspark_markov_draft_step: dspark_markov_logits, then one draw per request exactly as the
- *   verifier's bonus draw of a request with no draft position: temperature > 0 samples with the
- *   second uniform of (seed, request r, position 0), temperature == 0 takes the argmax (lowest
- *   index on ties).  out_tokens device int32 [R].
+ * dspark_markov_draft_step: dspark_markov_logits, then one draw per request with the rule of the
+ *   verifier's bonus draw for a request with no draft position: temperature > 0 inverts the CDF of
+ *   softmax(stored logits / T) in vocabulary order with the second uniform of (seed, request r,
+ *   position 0); temperature == 0 takes the argmax (lowest index on ties, NaN never wins; a row with
+ *   nothing above -inf sets DSPARK_DEV_ALL_NEG_INF and yields 0).  The softmax statistics are taken
+ *   per 128-column tile inside the contraction's epilogue, so the logits are not read a second time.
+ *   A row with NaN, +inf or no finite element sets DSPARK_DEV_BAD_ROW and yields -1.
+ *   out_tokens device int32 [R].
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, CUDA; a device wait that ran out sets
  * DSPARK_DEV_TIMEOUT in *dev_status and the affected logits are unspecified.
  */
@@ -341,7 +345,7 @@ typedef struct dspark_ktimer dspark_ktimer_t;
 enum {
     DSPARK_K_SCHEDULE = 0, DSPARK_K_OFFSETS = 1, DSPARK_K_STREAM = 2, DSPARK_K_DECIDE = 3,
     DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6, DSPARK_K_GREEDY_DECIDE = 7,
-    DSPARK_K_ROW_SCALE = 8, DSPARK_K_MARKOV_GEMM = 9, DSPARK_K_COUNT = 10
+    DSPARK_K_ROW_SCALE = 8, DSPARK_K_MARKOV_GEMM = 9, DSPARK_K_MARKOV_DRAW = 10, DSPARK_K_COUNT = 11
 };
 int dspark_ktimer_create(int capacity, dspark_ktimer_t** out);
 int dspark_ktimer_destroy(dspark_ktimer_t* t);

@@ -60,6 +60,8 @@ struct MarkovParams {
     float* out_conf;
     int32_t* dev_status;
     unsigned char* E;                         // workspace: gathered embeddings [rows padded to 128, 256] bf16
+    float2* stats;                            // workspace: per (row, vocabulary tile) statistics of the stored logits
+    float scale2;                             // log2(e) / T
 #ifdef DSPARK_MARKOV_TRACE
     unsigned long long* trace;                // 64 clock stamps per CTA (development aid)
 #endif
@@ -230,11 +232,67 @@ __device__ __forceinline__ uint4 add_round(const float* acc, uint4 u)
     return make_uint4(ow[0], ow[1], ow[2], ow[3]);
 }
 
+// ---- per-tile statistics of the stored logits, taken in the epilogue --------------------------------
+// kStats = 1 (sampling): m = max of the 128 stored values of (row, tile), s = sum of 2^((x - m) * scale2),
+//   i.e. the tile's softmax mass relative to its own maximum.  A NaN or +inf element makes s NaN; a tile
+//   with no element above -inf has m = -inf, s = 0.
+// kStats = 2 (greedy): m = max, s = the bit pattern of the lowest column index that attains it (-1 if
+//   nothing exceeds -inf; NaN never wins).
+template <int kStats>
+struct TileStats {
+    float m, s;
+    int idx;
+    __device__ __forceinline__ void reset() { m = -INFINITY; s = 0.f; idx = -1; }
+    // 32 stored values (16 words of two bf16) starting at column `col`; columns >= V do not count
+    __device__ __forceinline__ void update(const uint4 (&o)[4], int col, int V, float scale2)
+    {
+        if (kStats != 0) accumulate(o, col, V, scale2);
+    }
+    __device__ __forceinline__ void accumulate(const uint4 (&o)[4], int col, int V, float scale2)
+    {
+        float x[32];
+#pragma unroll
+        for (int v4 = 0; v4 < 4; ++v4) {
+            const uint32_t w[4] = {o[v4].x, o[v4].y, o[v4].z, o[v4].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { x[v4 * 8 + 2 * i] = bf16lo(w[i]); x[v4 * 8 + 2 * i + 1] = bf16hi(w[i]); }
+        }
+        const int nvalid = V - col;                         // >= 32 except in the last tile
+        if (kStats == 2) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < nvalid && x[i] > m) { m = x[i]; idx = col + i; }
+            return;
+        }
+        float cm = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < nvalid) cm = fmaxf(cm, x[i]);           // fmaxf drops NaN: it surfaces in the sum below
+        const float mn = fmaxf(m, cm);
+        if (mn > -INFINITY) {
+            const float off = mn * scale2;
+            float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+                if (i < nvalid) a0 += ex2_approx(fmaf(x[i], scale2, -off));
+                if (i + 1 < nvalid) a1 += ex2_approx(fmaf(x[i + 1], scale2, -off));
+            }
+            s = s * ex2_approx((m - mn) * scale2) + (a0 + a1);
+            m = mn;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < nvalid && x[i] != x[i]) s = x[i];
+        }
+    }
+    __device__ __forceinline__ float2 result() const { return make_float2(m, kStats == 2 ? __int_as_float(idx) : s); }
+};
+
 // ---- the GEMM: logits = U + E W2 for one group of at most 256 rows, bf16 out -------------------------
 // kTma: base-logit tiles and finished tiles move through the tensor maps (ring of three buffers, added
 // in place).  Otherwise (a base address or row pitch that breaks the 16-byte rules) the epilogue
 // threads load and store their rows directly.
-template <bool kTma>
+template <bool kTma, int kStats>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_out)
 {
@@ -363,6 +421,8 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             tc_fence_after();
             if (leader) stamp(24 + t);
             const uint32_t acc_addr = tmem_base + lane_base + (uint32_t)(s * kTileMN);
+            TileStats<kStats> ts;
+            ts.reset();
             if (kTma) {
                 unsigned char* tile = sU + ub * kUTileBytes;
 #pragma unroll 1
@@ -371,12 +431,16 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                     tmem_load32(acc_addr + (uint32_t)c0, acc);
                     unsigned char* rowp = tile + (c0 >> 6) * kBoxBytes + trow * 128;
                     const int j0 = (c0 & 63) >> 3;
+                    uint4 o[4];
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4) {
                         uint4* cell = reinterpret_cast<uint4*>(rowp + (((j0 + v4) ^ (trow & 7)) << 4));
-                        *cell = add_round(acc + v4 * 8, *cell);
+                        o[v4] = add_round(acc + v4 * 8, *cell);
+                        *cell = o[v4];
                     }
+                    ts.update(o, nt * kTileMN + c0, P.V, P.scale2);
                 }
+                if (kStats && mt * kTileMN + trow < P.R) P.stats[(size_t)(mt * kTileMN + trow) * P.n_tiles + nt] = ts.result();
                 tc_fence_before();
                 fence_proxy_async_smem();                   // the tile is read next by the copy engine
                 __syncwarp();
@@ -407,19 +471,32 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                     if (!live || col >= P.V) continue;
                     const unsigned char* up = urow + (long long)col * 2;
                     unsigned char* op = orow + (long long)col * 2;
+                    uint4 o[4];
                     if (col + 32 <= P.V && (((uintptr_t)up | (uintptr_t)op) & 15u) == 0) {
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4)
-                            *reinterpret_cast<uint4*>(op + 16 * v4) = add_round(acc + v4 * 8, __ldg((const uint4*)(up + 16 * v4)));
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            o[v4] = add_round(acc + v4 * 8, __ldg((const uint4*)(up + 16 * v4)));
+                            *reinterpret_cast<uint4*>(op + 16 * v4) = o[v4];
+                        }
                     } else {
+                        uint32_t w[16];
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
-                            if (col + i >= P.V) continue;
-                            const float u = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(up)[i]);
-                            reinterpret_cast<__nv_bfloat16*>(op)[i] = __float2bfloat16_rn(acc[i] + u);
+                            unsigned short b = 0;
+                            if (col + i < P.V) {
+                                const float u = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(up)[i]);
+                                const __nv_bfloat16 r = __float2bfloat16_rn(acc[i] + u);
+                                reinterpret_cast<__nv_bfloat16*>(op)[i] = r;
+                                b = *reinterpret_cast<const unsigned short*>(&r);
+                            }
+                            if (i & 1) w[i >> 1] |= (uint32_t)b << 16; else w[i >> 1] = b;
                         }
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) o[v4] = make_uint4(w[4 * v4], w[4 * v4 + 1], w[4 * v4 + 2], w[4 * v4 + 3]);
                     }
+                    ts.update(o, col, P.V, P.scale2);
                 }
+                if (kStats && live) P.stats[(size_t)row * P.n_tiles + nt] = ts.result();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[s]);
@@ -437,14 +514,122 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     }
 }
 
-__global__ void arange_offsets_kernel(int32_t* off, int n)
+// ---- the draw: one token per request from the tile statistics ---------------------------------------
+// One warp per request.  Sampling (greedy == 0): with M the row maximum and z_i = s_i 2^((m_i - M) scale2)
+// the mass of tile i, the running sum over tiles in vocabulary order gives the total Z; the token is the
+// smallest v whose running sum of 2^((x_v - M) scale2) exceeds u' Z, u' the second uniform of
+// (seed, request, position 0): the tile is located on the tile masses, the element inside it on the 128
+// stored logits of that tile.  A row with NaN, +inf or no finite element sets DSPARK_DEV_BAD_ROW and
+// yields -1.  Greedy: the lowest index of the row maximum; a row with nothing above -inf sets
+// DSPARK_DEV_ALL_NEG_INF and yields 0.
+__global__ void __launch_bounds__(256) markov_draw_kernel(MarkovParams P, int greedy, uint64_t seed, int32_t* out_tokens)
 {
     pdl_wait();
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i <= n) off[i] = i;
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (r >= P.R) return;
+    const float2* st = P.stats + (size_t)r * P.n_tiles;
+    if (greedy) {
+        float best = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int i = lane; i < P.n_tiles; i += 32) {
+            const float2 t = st[i];
+            const int idx = __float_as_int(t.y);
+            if (idx >= 0 && (t.x > best || (t.x == best && idx < bi))) { best = t.x; bi = idx; }
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+        }
+        if (lane == 0) {
+            if (bi == 0x7fffffff) { atomicOr(P.dev_status, DSPARK_DEV_ALL_NEG_INF); bi = 0; }
+            out_tokens[r] = bi;
+        }
+        return;
+    }
+    // row maximum, unusable rows
+    float M = -INFINITY;
+    bool bad = false;
+    for (int i = lane; i < P.n_tiles; i += 32) {
+        const float2 t = st[i];
+        M = fmaxf(M, t.x);
+        bad |= (t.y != t.y);
+    }
+    M = warp_max_f32(M);
+    bad = __any_sync(0xffffffffu, bad) || !(M > -INFINITY) || M == INFINITY;
+    // total mass: inclusive scan over tiles, 32 at a time, in vocabulary order
+    const float offM = M * P.scale2;
+    auto tile_mass = [&](int i) -> float {
+        if (i >= P.n_tiles) return 0.f;
+        const float2 t = st[i];
+        return t.y > 0.f ? t.y * ex2_approx(fmaf(t.x, P.scale2, -offM)) : 0.f;
+    };
+    auto scan32 = [&](float v) -> float {                   // inclusive prefix over the lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float n = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += n;
+        }
+        return v;
+    };
+    float Z = 0.f;
+    if (!bad)
+        for (int i0 = 0; i0 < P.n_tiles; i0 += 32) Z = __shfl_sync(0xffffffffu, Z + scan32(tile_mass(i0 + lane)), 31);
+    if (bad || !(Z > 0.f) || Z == INFINITY) {
+        if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW); out_tokens[r] = -1; }
+        return;
+    }
+    float ua, ur;
+    philox_uniforms(seed, (uint32_t)r, 0u, ua, ur);
+    const float thr = ur * Z;
+    // locate the tile: the first whose inclusive running sum exceeds thr (else the last with mass)
+    int tile = -1, last_pos = -1;
+    float before = 0.f, run = 0.f;
+    for (int i0 = 0; i0 < P.n_tiles && tile < 0; i0 += 32) {
+        const float z = tile_mass(i0 + lane);
+        const float inc = run + scan32(z);
+        const unsigned hit = __ballot_sync(0xffffffffu, inc > thr);
+        const unsigned pos = __ballot_sync(0xffffffffu, z > 0.f);
+        if (pos) last_pos = i0 + 31 - __clz(pos);
+        if (hit) {
+            const int l = __ffs(hit) - 1;
+            tile = i0 + l;
+            before = __shfl_sync(0xffffffffu, inc - z, l);
+        }
+        run = __shfl_sync(0xffffffffu, inc, 31);
+    }
+    float thr_in = thr;
+    if (tile < 0) { tile = last_pos; before = 0.f; thr_in = INFINITY; }   // rounding left the sum at or below thr: the last token with mass
+    // inside the tile: four consecutive columns per lane
+    const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(P.out + (long long)r * P.out_stride_bytes);
+    const int c0 = tile * kTileMN + lane * 4;
+    float e[4];
+    float lsum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        e[i] = c0 + i < P.V ? ex2_approx(fmaf(__bfloat162float(row[c0 + i]), P.scale2, -offM)) : 0.f;
+        lsum += e[i];
+    }
+    const float linc = scan32(lsum);
+    float cum = before + (linc - lsum);
+    int tok = -1, lastp = -1;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        cum += e[i];
+        if (e[i] > 0.f) lastp = c0 + i;
+        if (tok < 0 && cum > thr_in) tok = c0 + i;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, tok >= 0);
+    const unsigned pos = __ballot_sync(0xffffffffu, lastp >= 0);
+    int result;
+    if (hit) result = __shfl_sync(0xffffffffu, tok, __ffs(hit) - 1);
+    else result = pos ? __shfl_sync(0xffffffffu, lastp, 31 - __clz(pos)) : tile * kTileMN;
+    if (lane == 0) out_tokens[r] = result;
 }
 
-struct MarkovWs { size_t e, off, toks, trace, verify, total; };
+struct MarkovWs { size_t e, stats, trace, total; };
 static MarkovWs markov_layout(int R, int V)
 {
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
@@ -452,13 +637,11 @@ static MarkovWs markov_layout(int R, int V)
     MarkovWs w;
     size_t o = 0;
     w.e = o;      o += up((size_t)m_tiles * kTileMN * kRank * 2);
-    w.off = o;    o += up((size_t)(R + 1) * 4);
-    w.toks = o;   o += up((size_t)R * 4);
+    w.stats = o;  o += up((size_t)R * ((V + kTileMN - 1) / kTileMN) * sizeof(float2));
     w.trace = o;
 #ifdef DSPARK_MARKOV_TRACE
     o += up(256 * 64 * 8);
 #endif
-    w.verify = o; o += up(dspark_verify_workspace_bytes(R, R, V));
     w.total = o;
     return w;
 }
@@ -537,11 +720,13 @@ size_t dspark_markov_workspace_bytes(int R, int V)
     return markov_layout(R, V).total;
 }
 
-int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+// gather, confidence head, one GEMM launch per 256-row group; stats_mode 0 none, 1 softmax masses, 2 argmax
+static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
                          const int32_t* x_prev, int R, int V,
                          const void* H, int64_t h_row_stride, int d, const float* w_conf,
                          void* out_logits, int64_t out_row_stride, float* out_conf, int32_t* dev_status,
-                         void* workspace, size_t workspace_bytes, void* stream)
+                         void* workspace, size_t workspace_bytes, cudaStream_t s, int stats_mode, float temperature,
+                         MarkovParams* params_out)
 {
     if (!U || !W1 || !W2_packed || !x_prev || !out_logits || !dev_status) return DSPARK_ERR_INVALID_ARG;
     if (R < 1 || V < 1 || u_row_stride < V || out_row_stride < V) return DSPARK_ERR_INVALID_ARG;
@@ -557,21 +742,28 @@ int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, co
     P.out = (unsigned char*)out_logits; P.out_stride_bytes = (long long)out_row_stride * 2;
     P.out_conf = out_conf; P.dev_status = dev_status;
     P.E = (unsigned char*)workspace + w.e;
+    P.stats = (float2*)((unsigned char*)workspace + w.stats);
+    P.scale2 = stats_mode == 1 ? (float)(1.4426950408889634 / (double)temperature) : 0.f;
 #ifdef DSPARK_MARKOV_TRACE
     P.trace = (unsigned long long*)((unsigned char*)workspace + w.trace);
 #endif
+    if (params_out) *params_out = P;
 
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int smem_bytes = kUBuffers * kUTileBytes + 2 * kTileBytes + 1024;
     if (!g_gemm_attr_set[dev & 63]) {
-        if (cudaFuncSetAttribute(markov_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess ||
-            cudaFuncSetAttribute(markov_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
-            return launch_status();
+        bool ok = true;
+        ok = ok && cudaFuncSetAttribute(markov_gemm_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(markov_gemm_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(markov_gemm_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(markov_gemm_kernel<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(markov_gemm_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(markov_gemm_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) == cudaSuccess;
+        if (!ok) return launch_status();
         g_gemm_attr_set[dev & 63] = true;
     }
-    cudaStream_t s = (cudaStream_t)stream;
     const int rows_padded = P.m_tiles * kTileMN;
     launch_pdl(markov_gather_kernel, dim3((rows_padded * kKChunks + 255) / 256), dim3(256), 0, s, P, rows_padded);
     if (out_conf) launch_pdl(markov_confidence_kernel, dim3((R + 7) / 8), dim3(256), 0, s, P);
@@ -584,17 +776,37 @@ int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, co
         G.U = P.U + (long long)r0 * P.u_stride_bytes;
         G.out = P.out + (long long)r0 * P.out_stride_bytes;
         G.E = P.E + (size_t)r0 * kRank * 2;
+        G.stats = P.stats + (size_t)r0 * P.n_tiles;
         CUtensorMap map_u, map_out;
         memset(&map_u, 0, sizeof map_u);
         memset(&map_out, 0, sizeof map_out);
         const bool tma = g_markov_path != 1 && make_tile_map(&map_u, G.U, G.R, V, P.u_stride_bytes) &&
                          make_tile_map(&map_out, G.out, G.R, V, P.out_stride_bytes);
         KernelTimerScope timer(DSPARK_K_MARKOV_GEMM, s);
-        const dim3 grid(P.n_tiles < sms ? P.n_tiles : sms);
-        if (tma) launch_pdl(markov_gemm_kernel<true>, grid, dim3(kGemmThreads), (size_t)smem_bytes, s, G, map_u, map_out);
-        else launch_pdl(markov_gemm_kernel<false>, grid, dim3(kGemmThreads), (size_t)smem_bytes, s, G, map_u, map_out);
+        const dim3 grid(P.n_tiles < sms ? P.n_tiles : sms), block(kGemmThreads);
+        const size_t sm = (size_t)smem_bytes;
+        if (tma) {
+            if (stats_mode == 0) launch_pdl(markov_gemm_kernel<true, 0>, grid, block, sm, s, G, map_u, map_out);
+            else if (stats_mode == 1) launch_pdl(markov_gemm_kernel<true, 1>, grid, block, sm, s, G, map_u, map_out);
+            else launch_pdl(markov_gemm_kernel<true, 2>, grid, block, sm, s, G, map_u, map_out);
+        } else {
+            if (stats_mode == 0) launch_pdl(markov_gemm_kernel<false, 0>, grid, block, sm, s, G, map_u, map_out);
+            else if (stats_mode == 1) launch_pdl(markov_gemm_kernel<false, 1>, grid, block, sm, s, G, map_u, map_out);
+            else launch_pdl(markov_gemm_kernel<false, 2>, grid, block, sm, s, G, map_u, map_out);
+        }
     }
     return launch_status();
+}
+
+int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                         const int32_t* x_prev, int R, int V,
+                         const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                         void* out_logits, int64_t out_row_stride, float* out_conf, int32_t* dev_status,
+                         void* workspace, size_t workspace_bytes, void* stream)
+{
+    return markov_launch(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf, out_logits,
+                         out_row_stride, out_conf, dev_status, workspace, workspace_bytes, (cudaStream_t)stream, 0, 1.f,
+                         nullptr);
 }
 
 int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
@@ -604,24 +816,18 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
                              void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
                              int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream)
 {
-    if (!out_tokens) return DSPARK_ERR_INVALID_ARG;
-    int rc = dspark_markov_logits(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf,
-                                  out_logits, out_row_stride, out_conf, dev_status, workspace, workspace_bytes, stream);
+    if (!out_tokens || !(temperature >= 0.f) || isinf(temperature)) return DSPARK_ERR_INVALID_ARG;
+    const int greedy = temperature == 0.f;
+    MarkovParams P;
+    const int rc = markov_launch(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf, out_logits,
+                                 out_row_stride, out_conf, dev_status, workspace, workspace_bytes, (cudaStream_t)stream,
+                                 greedy ? 2 : 1, temperature, &P);
     if (rc != DSPARK_OK) return rc;
-    const MarkovWs w = markov_layout(R, V);
-    unsigned char* ws = (unsigned char*)workspace;
-    int32_t* off = (int32_t*)(ws + w.off);
-    int32_t* acc = (int32_t*)(ws + w.toks);
-    launch_pdl(arange_offsets_kernel, dim3((R + 256) / 256), dim3(256), 0, (cudaStream_t)stream, off, R);
-    // every request owns exactly one row and no draft position: the verifier's bonus path draws one
-    // token per row from softmax(row / T) with the second uniform of (seed, request, position 0);
-    // the draft-token array is never read for such a batch, the offsets stand in for it
-    if (temperature == 0.f)
-        return dspark_verify_greedy(out_logits, DSPARK_BF16, out_row_stride, V, off, off, R, R, acc, out_tokens,
-                                    dev_status, ws + w.verify, workspace_bytes - w.verify, stream);
-    return dspark_verify(out_logits, out_logits, DSPARK_BF16, out_row_stride, out_row_stride, V, off, nullptr,
-                         off, R, R, temperature, seed, acc, out_tokens,
-                         nullptr, nullptr, dev_status, ws + w.verify, workspace_bytes - w.verify, stream);
+    {
+        KernelTimerScope timer(DSPARK_K_MARKOV_DRAW, (cudaStream_t)stream);
+        launch_pdl(markov_draw_kernel, dim3((R + 7) / 8), dim3(256), 0, (cudaStream_t)stream, P, greedy, seed, out_tokens);
+    }
+    return launch_status();
 }
 
 }  // extern "C"

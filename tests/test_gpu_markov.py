@@ -127,3 +127,50 @@ def test_draft_step_draws_like_the_oracle(R, V, T):
         assert o.token_margin[r] < 1e-6, (r, got[r], o.out_tokens[r], o.token_margin[r])
     assert len(differ) <= max(1, R // 50)
     assert ((got >= 0) & (got < V)).all()
+
+
+def test_degenerate_rows_in_the_draw():
+    R, V = 6, 1500
+    m = W.markov_input(R, V, 21, "cuda", d=32)
+    m.U[1, 700] = float("nan")
+    m.U[3, :] = float("-inf")
+    m.U[4, 5] = float("inf")
+    for T in (1.0, 0.0):
+        out, _, toks, st = _run(m, temperature=T, seed=5, want_conf=False)
+        bits = W.bf16_bits(out)
+        off = np.arange(R + 1, dtype=np.int32)
+        got = toks.cpu().numpy()
+        if T == 0.0:
+            o = oracle.verify_greedy(bits, off, np.zeros(R, dtype=np.int32))
+            np.testing.assert_array_equal(got, o.out_tokens[:R])
+            assert st == int(np.bitwise_or.reduce(o.status)) == B.DEV_ALL_NEG_INF
+        else:
+            o = oracle.verify(bits, bits, off, np.zeros(R, dtype=np.int32), T, 5)
+            assert st == int(np.bitwise_or.reduce(o.status)) == B.DEV_BAD_ROW
+            for r in range(R):
+                if o.status[r]:
+                    assert got[r] == -1 and r in (1, 3, 4)
+                else:
+                    assert got[r] == o.out_tokens[r] or o.token_margin[r] < 1e-6
+
+
+@pytest.mark.parametrize("T", [0.3, 1.0, 2.5])
+def test_draw_frequencies_follow_the_softmax(T):
+    # many requests share one previous token and one base row: their draws are i.i.d. from one softmax
+    R, V = 2048, 300
+    m = W.markov_input(R, V, 31, "cuda", d=32, sigma=1.5)
+    m.U[:] = m.U[0:1].clone()
+    m.x_prev[:] = m.x_prev[0]
+    out, _, toks, st = _run(m, temperature=T, seed=99, want_conf=False)
+    assert st == 0
+    p = torch.softmax(out[0].double() / T, 0).cpu().numpy()
+    counts = np.bincount(toks.cpu().numpy(), minlength=V).astype(np.float64)
+    # chi-square against the exact probabilities, cells with expectation >= 5 (others pooled)
+    exp = p * R
+    big = exp >= 5
+    chi = ((counts[big] - exp[big]) ** 2 / exp[big]).sum()
+    rest_e, rest_c = exp[~big].sum(), counts[~big].sum()
+    if rest_e > 0:
+        chi += (rest_c - rest_e) ** 2 / rest_e
+    dof = int(big.sum())
+    assert chi < dof + 6 * (2 * dof) ** 0.5, (chi, dof)
