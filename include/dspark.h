@@ -289,7 +289,7 @@ int dspark_accept_rate(const void* target_logits, const void* draft_logits, int 
  *   columns past V are zero).  The caller owns both buffers.
  * dspark_markov_logits:
  *   U            device bf16 [R, >= V], row stride u_row_stride elements: base logits of position k
- *   W1           device bf16 [V, 256] row-major, 16-byte aligned
+ *   W1           device bf16 [V, 256] row-major, 32-byte aligned
  *   W2_packed    output of dspark_markov_pack_w2
  *   x_prev       device int32 [R]: previous token of each request (anchor token at k = 1); a value
  *                outside [0, V) sets DSPARK_DEV_BAD_TOKEN and contributes a zero embedding

@@ -37,7 +37,8 @@ constexpr int kTileBytes = kTileMN * kRank * 2;  // 64 KB of bf16: one packed W2
 constexpr int kKChunks = kRank / 8;              // 16-byte chunks along K
 constexpr int kChunkBytes = kTileMN * 16;        // one K chunk of a tile: 128 columns x 16 B
 constexpr int kGroupRows = 2 * kTileMN;          // rows per launch: two row tiles resident in tensor memory
-constexpr int kGemmThreads = 320;                // producer, MMA, 4 epilogue warps, 4 loader warps
+constexpr int kEpiWarps = 16;                    // four per tensor-memory lane quarter, 32 columns of a tile each
+constexpr int kGemmThreads = (2 + kEpiWarps) * 32; // producer warp, MMA warp, epilogue warps
 constexpr int kTmemCols = 512;                   // accumulators: columns 0..255, embedding tiles: 256..511
 
 // Packed W2 tile (K-major, no swizzle): element (n, k) of a 128-column x 256 tile lives at
@@ -59,7 +60,6 @@ struct MarkovParams {
     unsigned char* out; long long out_stride_bytes;
     float* out_conf;
     int32_t* dev_status;
-    unsigned char* E;                         // workspace: gathered embeddings [rows padded to 128, 256] bf16
     float2* stats;                            // workspace: per (row, vocabulary tile) statistics of the stored logits
     float scale2;                             // log2(e) / T
 #ifdef DSPARK_MARKOV_TRACE
@@ -82,39 +82,34 @@ __global__ void markov_pack_w2_kernel(const __nv_bfloat16* __restrict__ W2, int 
     *reinterpret_cast<uint4*>(W2p + (size_t)tile * kTileBytes + packed_offset(nn, kc * 8)) = *reinterpret_cast<uint4*>(v);
 }
 
-// ---- per step: E = W1[x_prev], rows past R zero -------------------------------------------------------
-__global__ void markov_gather_kernel(MarkovParams P, int rows_padded)
+// ---- confidence head: c = sigmoid(w . [h ; W1[x_prev]]), one CTA per request ---------------------------
+// Every thread takes a strided share of the d + 256 products in fp64 (a handful each), the block adds
+// them up.  All threads of the CTA must call it; thread 0 writes the result.
+__device__ __forceinline__ void block_confidence(const MarkovParams& P, int r, double* s_part)
 {
-    pdl_wait();
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;                       // (row, 16-byte chunk)
-    if (idx >= rows_padded * kKChunks) return;
-    const int kc = idx % kKChunks, row = idx / kKChunks;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (row < P.R) {
-        const int x = P.x_prev[row];
-        if (x >= 0 && x < P.V) v = __ldg((const uint4*)(P.W1 + ((size_t)x * kRank + kc * 8) * 2));
-        else if (kc == 0) atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN);
-    }
-    reinterpret_cast<uint4*>(P.E)[idx] = v;
-}
-
-// ---- per step: confidence head, one warp per request -------------------------------------------------
-__global__ void markov_confidence_kernel(MarkovParams P)
-{
-    pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (r >= P.R) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
     const int x = P.x_prev[r];
     double z = 0.0;
     const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(P.H + (long long)r * P.h_stride_bytes);
-    for (int i = lane; i < P.d; i += 32) z += (double)P.w_conf[i] * (double)__bfloat162float(h[i]);
+    for (int i = tid; i < P.d; i += blockDim.x) z += (double)P.w_conf[i] * (double)__bfloat162float(h[i]);
     if (x >= 0 && x < P.V) {
         const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(P.W1) + (size_t)x * kRank;
-        for (int i = lane; i < kRank; i += 32) z += (double)P.w_conf[P.d + i] * (double)__bfloat162float(e[i]);
+        for (int i = tid; i < kRank; i += blockDim.x) z += (double)P.w_conf[P.d + i] * (double)__bfloat162float(e[i]);
     }
     z = warp_sum_f64(z);
-    if (lane == 0) P.out_conf[r] = (float)(1.0 / (1.0 + exp(-z)));
+    if (lane == 0) s_part[warp] = z;
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < nwarp; ++w) z += s_part[w];
+        P.out_conf[r] = (float)(1.0 / (1.0 + exp(-z)));
+    }
+}
+
+__global__ void __launch_bounds__(256) markov_confidence_kernel(MarkovParams P)
+{
+    __shared__ double s_part[8];
+    pdl_wait();
+    block_confidence(P, blockIdx.x, s_part);
 }
 
 // ---- tcgen05 helpers --------------------------------------------------------------------------------
@@ -176,18 +171,28 @@ __device__ __forceinline__ void tmem_store32(uint32_t taddr, const uint4 (&w)[8]
         : "memory");
 }
 
-// One row of an embedding tile: 512 B of E into registers (all 32 loads in flight at once), then into
-// this thread's lane of tensor memory, columns taddr .. taddr + 127 (two bf16 per column, k ascending).
-__device__ __forceinline__ void embedding_row_to_tmem(const unsigned char* E, int row, uint32_t taddr)
+// Half a row of an embedding tile: 256 B of W1[x_prev] (src; NULL = zeros) into registers by eight 256-bit loads (a full 32 B sector
+// each, all in flight at once), then into this thread's lane of tensor memory, 64 columns from taddr
+// (two bf16 per column, k ascending).
+__device__ __forceinline__ void embedding_half_row_to_tmem(const unsigned char* src, uint32_t taddr)
 {
-    const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)row * kRank * 2);
-    uint4 w[4][8];
+    uint4 w[2][8];
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
+    for (int c = 0; c < 2; ++c)
 #pragma unroll
-        for (int v = 0; v < 8; ++v) w[c][v] = src[c * 8 + v];
+        for (int v = 0; v < 8; ++v) w[c][v] = make_uint4(0, 0, 0, 0);
+    if (src)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) tmem_store32(taddr + (uint32_t)(c * 32), w[c]);
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (int v = 0; v < 8; v += 2)
+            asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(w[c][v].x), "=r"(w[c][v].y), "=r"(w[c][v].z), "=r"(w[c][v].w),
+                           "=r"(w[c][v + 1].x), "=r"(w[c][v + 1].y), "=r"(w[c][v + 1].z), "=r"(w[c][v + 1].w)
+                         : "l"(src + (c * 8 + v) * 16)
+                         : "memory");
+#pragma unroll
+    for (int c = 0; c < 2; ++c) tmem_store32(taddr + (uint32_t)(c * 32), w[c]);
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     tc_fence_before();
 }
@@ -233,8 +238,10 @@ __device__ __forceinline__ uint4 add_round(const float* acc, uint4 u)
 }
 
 // ---- per-tile statistics of the stored logits, taken in the epilogue --------------------------------
-// kStats = 1 (sampling): m = max of the 128 stored values of (row, tile), s = sum of 2^((x - m) * scale2),
-//   i.e. the tile's softmax mass relative to its own maximum.  A NaN or +inf element makes s NaN; a tile
+// One entry per row and 32 columns (four per vocabulary tile, one per epilogue warp of a lane quarter),
+// called a box below.
+// kStats = 1 (sampling): m = max of the 32 stored values of (row, box), s = sum of 2^((x - m) * scale2),
+//   i.e. the box's softmax mass relative to its own maximum.  A NaN or +inf element makes s NaN; a tile
 //   with no element above -inf has m = -inf, s = 0.
 // kStats = 2 (greedy): m = max, s = the bit pattern of the lowest column index that attains it (-1 if
 //   nothing exceeds -inf; NaN never wins).
@@ -301,7 +308,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     unsigned char* sU = smem;                               // three base-logit / output tiles
     unsigned char* sB = smem + kUBuffers * kUTileBytes;     // two W2 tiles
     __shared__ __align__(8) uint64_t b_full[2], b_empty[2], a_full[2], acc_full[2], acc_empty[2];
-    __shared__ __align__(8) uint64_t u_full[kUBuffers], epi_done;
+    __shared__ __align__(8) uint64_t u_full[kUBuffers], epi_done, prefetch_issued;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -309,11 +316,12 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
             mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1);
-            mbar_init(&a_full[s], 4);
-            mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4);
+            mbar_init(&a_full[s], 8);
+            mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], kEpiWarps);
         }
         for (int s = 0; s < kUBuffers; ++s) mbar_init(&u_full[s], 1);
-        mbar_init(&epi_done, 4);
+        mbar_init(&epi_done, kEpiWarps);
+        mbar_init(&prefetch_issued, 2);
         s_abort = 0;
         mbar_fence_init();
     }
@@ -346,12 +354,15 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     if (warp == 0) {
         // ---------------- producer: W2 tiles, one ahead ---------------------------------------------------
         if (lane == 0) {
+            bool told = false;
+            if (my_ntiles == 0) { mbar_arrive(&prefetch_issued); told = true; }
             for (int in = 0; in < my_ntiles && !*abort_flag; ++in) {
                 const int nt = blockIdx.x + in * gridDim.x, bs = in & 1;
                 if (!mbar_wait_bounded(&b_empty[bs], ((uint32_t)(in >> 1) & 1u) ^ 1u)) { give_up(); break; }
                 mbar_arrive_expect_tx(&b_full[bs], kTileBytes);
                 bulk_g2s(sB + bs * kTileBytes, P.W2p + (size_t)nt * kTileBytes, kTileBytes, &b_full[bs]);
                 stamp(56 + in);
+                if (in == 1 || in == my_ntiles - 1) { if (!told) mbar_arrive(&prefetch_issued); told = true; }
             }
         }
     } else if (warp == 1) {
@@ -379,18 +390,14 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                 umma_commit(&b_empty[bs]);                  // the W2 tile may be overwritten
             }
         }
-    } else if (warp >= 6) {
-        // ---------------- loaders: embedding rows of row tile 0 -> tensor memory -------------------------
-        if (my_tiles > 0) {
-            const int q = warp & 3;
-            embedding_row_to_tmem(P.E, q * 32 + lane, tmem_a0 + ((uint32_t)(q * 32) << 16));
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&a_full[0]);
-            if (warp == 6 && lane == 0) stamp(2);
-        }
     } else {
         // ---------------- epilogue: accumulator + base logits -> bf16 ------------------------------------
+        // Sixteen warps: four per tensor-memory lane quarter, each owning 32 columns of every tile.  Before
+        // the first tile each warp brings one (row tile, lane quarter, K half) of the embeddings into
+        // tensor memory.
         const int q = warp & 3;                             // TMEM lane quarter this warp may access
+        const int chunk = (warp - 2) >> 2;                  // which 32 columns of a tile
+        const int c0 = chunk * 32;
         const int trow = q * 32 + lane;                     // row of the tile this thread owns
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const bool leader = kTma && warp == 2 && lane == 0;
@@ -401,13 +408,27 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             tma_load_2d(dst, &map_u, nt * kTileMN, mt * kTileMN, &u_full[t % kUBuffers]);
             tma_load_2d(dst + kBoxBytes, &map_u, nt * kTileMN + kBoxCols, mt * kTileMN, &u_full[t % kUBuffers]);
         };
+        // The first W2 tiles and base-logit tiles are requested before any embedding load: the copy
+        // instructions share the load/store queue with those loads and would wait behind them.
         if (leader)
             for (int t = 0; t < 2 && t < my_tiles; ++t) issue_u_load(t);
-        if (P.m_tiles == 2 && my_tiles > 0) {               // row tile 1, while the pipeline fills
-            embedding_row_to_tmem(P.E, kTileMN + trow, tmem_a0 + lane_base + (uint32_t)kTileMN);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&a_full[1]);
-            if (leader) stamp(3);
+        if (warp == 2 && lane == 0) mbar_arrive(&prefetch_issued);
+        mbar_wait_bounded(&prefetch_issued, 0u);            // a limit that runs out only costs the ordering
+        {
+            const int mt = chunk >> 1, kh = chunk & 1;      // row tile and K half this warp loads
+            if (my_tiles > 0 && mt < P.m_tiles) {
+                const int row = mt * kTileMN + trow;
+                const unsigned char* src = nullptr;         // rows past R and bad tokens: a zero embedding
+                if (row < P.R) {
+                    const int x = P.x_prev[row];
+                    if (x >= 0 && x < P.V) src = P.W1 + ((size_t)x * kRank + kh * (kRank / 2)) * 2;
+                    else if (blockIdx.x == 0 && kh == 0) atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN);
+                }
+                embedding_half_row_to_tmem(src, tmem_a0 + lane_base + (uint32_t)(mt * kTileMN + kh * (kRank / 4)));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&a_full[mt]);
+                if (lane == 0 && q == 2 && kh == 0) stamp(2 + mt);
+            }
         }
         for (int t = 0; t < my_tiles && !*abort_flag; ++t) {
             const int nt = blockIdx.x + (t / P.m_tiles) * gridDim.x, mt = t % P.m_tiles;
@@ -425,8 +446,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             ts.reset();
             if (kTma) {
                 unsigned char* tile = sU + ub * kUTileBytes;
-#pragma unroll 1
-                for (int c0 = 0; c0 < kTileMN; c0 += 32) {
+                {
                     float acc[32];
                     tmem_load32(acc_addr + (uint32_t)c0, acc);
                     unsigned char* rowp = tile + (c0 >> 6) * kBoxBytes + trow * 128;
@@ -440,7 +460,8 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                     }
                     ts.update(o, nt * kTileMN + c0, P.V, P.scale2);
                 }
-                if (kStats && mt * kTileMN + trow < P.R) P.stats[(size_t)(mt * kTileMN + trow) * P.n_tiles + nt] = ts.result();
+                if (kStats && mt * kTileMN + trow < P.R)
+                    P.stats[(size_t)(mt * kTileMN + trow) * (4 * P.n_tiles) + 4 * nt + chunk] = ts.result();
                 tc_fence_before();
                 fence_proxy_async_smem();                   // the tile is read next by the copy engine
                 __syncwarp();
@@ -463,12 +484,11 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                 const bool live = row < P.R;
                 const unsigned char* urow = P.U + (long long)row * P.u_stride_bytes;
                 unsigned char* orow = P.out + (long long)row * P.out_stride_bytes;
-#pragma unroll 1
-                for (int c0 = 0; c0 < kTileMN; c0 += 32) {
+                do {
                     float acc[32];
                     tmem_load32(acc_addr + (uint32_t)c0, acc);
                     const int col = nt * kTileMN + c0;
-                    if (!live || col >= P.V) continue;
+                    if (!live || col >= P.V) break;
                     const unsigned char* up = urow + (long long)col * 2;
                     unsigned char* op = orow + (long long)col * 2;
                     uint4 o[4];
@@ -495,8 +515,8 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                         for (int v4 = 0; v4 < 4; ++v4) o[v4] = make_uint4(w[4 * v4], w[4 * v4 + 1], w[4 * v4 + 2], w[4 * v4 + 3]);
                     }
                     ts.update(o, col, P.V, P.scale2);
-                }
-                if (kStats && live) P.stats[(size_t)row * P.n_tiles + nt] = ts.result();
+                } while (false);
+                if (kStats && live) P.stats[(size_t)row * (4 * P.n_tiles) + 4 * nt + chunk] = ts.result();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[s]);
@@ -514,28 +534,50 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     }
 }
 
-// ---- the draw: one token per request from the tile statistics ---------------------------------------
-// One warp per request.  Sampling (greedy == 0): with M the row maximum and z_i = s_i 2^((m_i - M) scale2)
-// the mass of tile i, the running sum over tiles in vocabulary order gives the total Z; the token is the
-// smallest v whose running sum of 2^((x_v - M) scale2) exceeds u' Z, u' the second uniform of
-// (seed, request, position 0): the tile is located on the tile masses, the element inside it on the 128
-// stored logits of that tile.  A row with NaN, +inf or no finite element sets DSPARK_DEV_BAD_ROW and
-// yields -1.  Greedy: the lowest index of the row maximum; a row with nothing above -inf sets
+// ---- the draw: one token per request from the box statistics -----------------------------------------
+// One CTA of 256 threads per request; thread t owns the kDrawPer consecutive boxes starting at
+// t * per (per = boxes per row / 256, rounded up), so thread order is vocabulary order.
+// Sampling (greedy == 0): with M the row maximum and z_i = s_i 2^((m_i - M) scale2) the mass of box i,
+// the running sum (within a thread, then across threads) gives the total Z; the token is the smallest v
+// whose running sum of 2^((x_v - M) scale2) exceeds u' Z, u' the second uniform of (seed, request,
+// position 0): the box is located on the box masses, the element inside it on the 32 stored logits of
+// that box.  A row with NaN, +inf or no finite element sets DSPARK_DEV_BAD_ROW and yields -1.
+// Greedy: the lowest index of the row maximum; a row with nothing above -inf sets
 // DSPARK_DEV_ALL_NEG_INF and yields 0.
-__global__ void __launch_bounds__(256) markov_draw_kernel(MarkovParams P, int greedy, uint64_t seed, int32_t* out_tokens)
+constexpr int kDrawThreads = 512;
+constexpr int kStatCols = 32;                    // columns per statistics entry
+constexpr int kDrawPer = 16;                     // entries per thread at most: V <= 512 * 16 * 32
+constexpr int kMaxDrawV = kDrawThreads * kDrawPer * kStatCols;
+
+__global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams P, int greedy, uint64_t seed, int32_t* out_tokens)
 {
+    __shared__ float s_red[kDrawThreads / 32];
+    __shared__ int s_redi[kDrawThreads / 32];
+    __shared__ float s_before;
+    __shared__ int s_box, s_last, s_bad;
+    __shared__ double s_part[kDrawThreads / 32];
     pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (r >= P.R) return;
-    const float2* st = P.stats + (size_t)r * P.n_tiles;
+    if (P.out_conf) block_confidence(P, blockIdx.x, s_part);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r = blockIdx.x;
+    const int n_box = 4 * P.n_tiles;
+    const int per = (n_box + kDrawThreads - 1) / kDrawThreads;
+    const float2* st = P.stats + (size_t)r * n_box;
+    float2 e[kDrawPer];
+#pragma unroll
+    for (int k = 0; k < kDrawPer; ++k) {
+        const int i = tid * per + k;
+        e[k] = (k < per && i < n_box) ? st[i] : make_float2(-INFINITY, greedy ? __int_as_float(-1) : 0.f);
+    }
+    if (tid == 0) { s_box = 0x7fffffff; s_last = -1; s_bad = 0; }
+    __syncthreads();
     if (greedy) {
         float best = -INFINITY;
         int bi = 0x7fffffff;
-        for (int i = lane; i < P.n_tiles; i += 32) {
-            const float2 t = st[i];
-            const int idx = __float_as_int(t.y);
-            if (idx >= 0 && (t.x > best || (t.x == best && idx < bi))) { best = t.x; bi = idx; }
+#pragma unroll
+        for (int k = 0; k < kDrawPer; ++k) {
+            const int idx = __float_as_int(e[k].y);
+            if (idx >= 0 && (e[k].x > best || (e[k].x == best && idx < bi))) { best = e[k].x; bi = idx; }
         }
 #pragma unroll
         for (int o = 16; o; o >>= 1) {
@@ -543,7 +585,11 @@ __global__ void __launch_bounds__(256) markov_draw_kernel(MarkovParams P, int gr
             const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
             if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
         }
-        if (lane == 0) {
+        if (lane == 0) { s_red[warp] = best; s_redi[warp] = bi; }
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 1; w < kDrawThreads / 32; ++w)
+                if (s_red[w] > best || (s_red[w] == best && s_redi[w] < bi)) { best = s_red[w]; bi = s_redi[w]; }
             if (bi == 0x7fffffff) { atomicOr(P.dev_status, DSPARK_DEV_ALL_NEG_INF); bi = 0; }
             out_tokens[r] = bi;
         }
@@ -552,92 +598,99 @@ __global__ void __launch_bounds__(256) markov_draw_kernel(MarkovParams P, int gr
     // row maximum, unusable rows
     float M = -INFINITY;
     bool bad = false;
-    for (int i = lane; i < P.n_tiles; i += 32) {
-        const float2 t = st[i];
-        M = fmaxf(M, t.x);
-        bad |= (t.y != t.y);
-    }
-    M = warp_max_f32(M);
-    bad = __any_sync(0xffffffffu, bad) || !(M > -INFINITY) || M == INFINITY;
-    // total mass: inclusive scan over tiles, 32 at a time, in vocabulary order
-    const float offM = M * P.scale2;
-    auto tile_mass = [&](int i) -> float {
-        if (i >= P.n_tiles) return 0.f;
-        const float2 t = st[i];
-        return t.y > 0.f ? t.y * ex2_approx(fmaf(t.x, P.scale2, -offM)) : 0.f;
-    };
-    auto scan32 = [&](float v) -> float {                   // inclusive prefix over the lanes
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float n = __shfl_up_sync(0xffffffffu, v, o);
-            if (lane >= o) v += n;
-        }
-        return v;
-    };
-    float Z = 0.f;
-    if (!bad)
-        for (int i0 = 0; i0 < P.n_tiles; i0 += 32) Z = __shfl_sync(0xffffffffu, Z + scan32(tile_mass(i0 + lane)), 31);
+    for (int k = 0; k < kDrawPer; ++k) { M = fmaxf(M, e[k].x); bad |= (e[k].y != e[k].y); }
+    M = warp_max_f32(M);
+    if (lane == 0) s_red[warp] = M;
+    if (bad) s_bad = 1;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kDrawThreads / 32; ++w) M = fmaxf(M, s_red[w]);
+    bad = s_bad || !(M > -INFINITY) || M == INFINITY;
+    __syncthreads();                                        // s_red is reused below
+    // box masses, running sum inside the thread, exclusive prefix across threads
+    const float offM = M * P.scale2;
+    float z[kDrawPer];
+    float local = 0.f;
+#pragma unroll
+    for (int k = 0; k < kDrawPer; ++k) {
+        z[k] = (!bad && e[k].y > 0.f) ? e[k].y * ex2_approx(fmaf(e[k].x, P.scale2, -offM)) : 0.f;
+        local += z[k];
+    }
+    float inc = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) s_red[warp] = inc;
+    __syncthreads();
+    float wbase = 0.f, Z = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDrawThreads / 32; ++w) { if (w < warp) wbase += s_red[w]; Z += s_red[w]; }
     if (bad || !(Z > 0.f) || Z == INFINITY) {
-        if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW); out_tokens[r] = -1; }
+        if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW); out_tokens[r] = -1; }
         return;
     }
     float ua, ur;
     philox_uniforms(seed, (uint32_t)r, 0u, ua, ur);
     const float thr = ur * Z;
-    // locate the tile: the first whose inclusive running sum exceeds thr (else the last with mass)
-    int tile = -1, last_pos = -1;
-    float before = 0.f, run = 0.f;
-    for (int i0 = 0; i0 < P.n_tiles && tile < 0; i0 += 32) {
-        const float z = tile_mass(i0 + lane);
-        const float inc = run + scan32(z);
-        const unsigned hit = __ballot_sync(0xffffffffu, inc > thr);
-        const unsigned pos = __ballot_sync(0xffffffffu, z > 0.f);
-        if (pos) last_pos = i0 + 31 - __clz(pos);
-        if (hit) {
-            const int l = __ffs(hit) - 1;
-            tile = i0 + l;
-            before = __shfl_sync(0xffffffffu, inc - z, l);
+    const float excl = wbase + (inc - local);
+    // the first box whose inclusive running sum exceeds thr; the last box with mass as a fallback
+    {
+        float run = excl;
+        int mine = 0x7fffffff, lastp = -1;
+#pragma unroll
+        for (int k = 0; k < kDrawPer; ++k) {
+            run += z[k];
+            if (z[k] > 0.f) lastp = tid * per + k;
+            if (mine == 0x7fffffff && z[k] > 0.f && run > thr) mine = tid * per + k;
         }
-        run = __shfl_sync(0xffffffffu, inc, 31);
+        if (mine != 0x7fffffff) atomicMin(&s_box, mine);
+        if (lastp >= 0) atomicMax(&s_last, lastp);
     }
-    float thr_in = thr;
-    if (tile < 0) { tile = last_pos; before = 0.f; thr_in = INFINITY; }   // rounding left the sum at or below thr: the last token with mass
-    // inside the tile: four consecutive columns per lane
+    __syncthreads();
+    const int box = s_box != 0x7fffffff ? s_box : s_last;
+    const bool found = s_box != 0x7fffffff;
+    if (found && box / per == tid) {                        // the owner publishes the sum before its box
+        float run = excl;
+#pragma unroll
+        for (int k = 0; k < kDrawPer; ++k) {
+            if (tid * per + k == box) s_before = run;
+            run += z[k];
+        }
+    }
+    __syncthreads();
+    if (warp != 0) return;
+    // inside the box: one column per lane
+    const float before = found ? s_before : 0.f;
+    const float thr_in = found ? thr : INFINITY;            // rounding left the sum at or below thr: the last token with mass
     const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(P.out + (long long)r * P.out_stride_bytes);
-    const int c0 = tile * kTileMN + lane * 4;
-    float e[4];
-    float lsum = 0.f;
+    const int c = box * kStatCols + lane;
+    const float ev = c < P.V ? ex2_approx(fmaf(__bfloat162float(row[c]), P.scale2, -offM)) : 0.f;
+    float linc = ev;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        e[i] = c0 + i < P.V ? ex2_approx(fmaf(__bfloat162float(row[c0 + i]), P.scale2, -offM)) : 0.f;
-        lsum += e[i];
+    for (int o = 1; o < 32; o <<= 1) {
+        const float n = __shfl_up_sync(0xffffffffu, linc, o);
+        if (lane >= o) linc += n;
     }
-    const float linc = scan32(lsum);
-    float cum = before + (linc - lsum);
-    int tok = -1, lastp = -1;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        cum += e[i];
-        if (e[i] > 0.f) lastp = c0 + i;
-        if (tok < 0 && cum > thr_in) tok = c0 + i;
-    }
+    const int tok = (ev > 0.f && before + linc > thr_in) ? c : -1;
+    const int lastp = ev > 0.f ? c : -1;
     const unsigned hit = __ballot_sync(0xffffffffu, tok >= 0);
     const unsigned pos = __ballot_sync(0xffffffffu, lastp >= 0);
     int result;
     if (hit) result = __shfl_sync(0xffffffffu, tok, __ffs(hit) - 1);
-    else result = pos ? __shfl_sync(0xffffffffu, lastp, 31 - __clz(pos)) : tile * kTileMN;
+    else result = pos ? __shfl_sync(0xffffffffu, lastp, 31 - __clz(pos)) : box * kStatCols;
     if (lane == 0) out_tokens[r] = result;
 }
 
-struct MarkovWs { size_t e, stats, trace, total; };
+struct MarkovWs { size_t stats, trace, total; };
 static MarkovWs markov_layout(int R, int V)
 {
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
-    const int m_tiles = (R + kTileMN - 1) / kTileMN;
     MarkovWs w;
     size_t o = 0;
-    w.e = o;      o += up((size_t)m_tiles * kTileMN * kRank * 2);
-    w.stats = o;  o += up((size_t)R * ((V + kTileMN - 1) / kTileMN) * sizeof(float2));
+    w.stats = o;  o += up((size_t)R * 4 * ((V + kTileMN - 1) / kTileMN) * sizeof(float2));
     w.trace = o;
 #ifdef DSPARK_MARKOV_TRACE
     o += up(256 * 64 * 8);
@@ -720,7 +773,7 @@ size_t dspark_markov_workspace_bytes(int R, int V)
     return markov_layout(R, V).total;
 }
 
-// gather, confidence head, one GEMM launch per 256-row group; stats_mode 0 none, 1 softmax masses, 2 argmax
+// one GEMM launch per 256-row group; stats_mode 0 none, 1 softmax masses, 2 argmax
 static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
                          const int32_t* x_prev, int R, int V,
                          const void* H, int64_t h_row_stride, int d, const float* w_conf,
@@ -733,7 +786,7 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
     if (out_conf && (!H || !w_conf || d < 0 || h_row_stride < d)) return DSPARK_ERR_INVALID_ARG;
     const MarkovWs w = markov_layout(R, V);
     if (!workspace || workspace_bytes < w.total) return DSPARK_ERR_WORKSPACE;
-    if ((((uintptr_t)workspace) & 255u) || (((uintptr_t)W2_packed | (uintptr_t)W1) & 15u)) return DSPARK_ERR_ALIGNMENT;
+    if ((((uintptr_t)workspace) & 255u) || ((uintptr_t)W2_packed & 15u) || ((uintptr_t)W1 & 31u)) return DSPARK_ERR_ALIGNMENT;
     MarkovParams P;
     P.U = (const unsigned char*)U; P.u_stride_bytes = (long long)u_row_stride * 2;
     P.W1 = (const unsigned char*)W1; P.W2p = (const unsigned char*)W2_packed; P.x_prev = x_prev;
@@ -741,7 +794,6 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
     P.H = (const unsigned char*)H; P.h_stride_bytes = (long long)h_row_stride * 2; P.d = d; P.w_conf = w_conf;
     P.out = (unsigned char*)out_logits; P.out_stride_bytes = (long long)out_row_stride * 2;
     P.out_conf = out_conf; P.dev_status = dev_status;
-    P.E = (unsigned char*)workspace + w.e;
     P.stats = (float2*)((unsigned char*)workspace + w.stats);
     P.scale2 = stats_mode == 1 ? (float)(1.4426950408889634 / (double)temperature) : 0.f;
 #ifdef DSPARK_MARKOV_TRACE
@@ -764,9 +816,6 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
         if (!ok) return launch_status();
         g_gemm_attr_set[dev & 63] = true;
     }
-    const int rows_padded = P.m_tiles * kTileMN;
-    launch_pdl(markov_gather_kernel, dim3((rows_padded * kKChunks + 255) / 256), dim3(256), 0, s, P, rows_padded);
-    if (out_conf) launch_pdl(markov_confidence_kernel, dim3((R + 7) / 8), dim3(256), 0, s, P);
     // one launch per group of 256 rows: both row tiles of a group stay in tensor memory while the CTA
     // walks its vocabulary tiles (W2 is streamed once per group)
     for (int r0 = 0; r0 < R; r0 += kGroupRows) {
@@ -775,8 +824,8 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
         G.m_tiles = (G.R + kTileMN - 1) / kTileMN;
         G.U = P.U + (long long)r0 * P.u_stride_bytes;
         G.out = P.out + (long long)r0 * P.out_stride_bytes;
-        G.E = P.E + (size_t)r0 * kRank * 2;
-        G.stats = P.stats + (size_t)r0 * P.n_tiles;
+        G.x_prev = P.x_prev + r0;
+        G.stats = P.stats + (size_t)r0 * 4 * P.n_tiles;
         CUtensorMap map_u, map_out;
         memset(&map_u, 0, sizeof map_u);
         memset(&map_out, 0, sizeof map_out);
@@ -804,9 +853,13 @@ int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, co
                          void* out_logits, int64_t out_row_stride, float* out_conf, int32_t* dev_status,
                          void* workspace, size_t workspace_bytes, void* stream)
 {
-    return markov_launch(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf, out_logits,
-                         out_row_stride, out_conf, dev_status, workspace, workspace_bytes, (cudaStream_t)stream, 0, 1.f,
-                         nullptr);
+    MarkovParams P;
+    const int rc = markov_launch(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf, out_logits,
+                                 out_row_stride, out_conf, dev_status, workspace, workspace_bytes, (cudaStream_t)stream, 0,
+                                 1.f, &P);
+    if (rc != DSPARK_OK || !out_conf) return rc;
+    launch_pdl(markov_confidence_kernel, dim3(R), dim3(256), 0, (cudaStream_t)stream, P);
+    return launch_status();
 }
 
 int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
@@ -817,6 +870,7 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
                              int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream)
 {
     if (!out_tokens || !(temperature >= 0.f) || isinf(temperature)) return DSPARK_ERR_INVALID_ARG;
+    if (V > kMaxDrawV) return DSPARK_ERR_SHAPE;
     const int greedy = temperature == 0.f;
     MarkovParams P;
     const int rc = markov_launch(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf, out_logits,
@@ -825,7 +879,7 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
     if (rc != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_MARKOV_DRAW, (cudaStream_t)stream);
-        launch_pdl(markov_draw_kernel, dim3((R + 7) / 8), dim3(256), 0, (cudaStream_t)stream, P, greedy, seed, out_tokens);
+        launch_pdl(markov_draw_kernel, dim3(R), dim3(kDrawThreads), 0, (cudaStream_t)stream, P, greedy, seed, out_tokens);
     }
     return launch_status();
 }
