@@ -257,14 +257,38 @@ struct TileStats {
     }
     __device__ __forceinline__ void accumulate(const uint4 (&o)[4], int col, int V, float scale2)
     {
+        const uint32_t w[16] = {o[0].x, o[0].y, o[0].z, o[0].w, o[1].x, o[1].y, o[1].z, o[1].w,
+                                o[2].x, o[2].y, o[2].z, o[2].w, o[3].x, o[3].y, o[3].z, o[3].w};
+        const int nvalid = V - col;                         // >= 32 except in the last tile
+        if (kStats == 1 && nvalid >= 32 && m == -INFINITY && s == 0.f) {
+            // whole box, fresh entry: maximum on packed bf16 pairs (NaN dropped, as fmaxf does), then one
+            // packed multiply-add and two exponentials per pair
+            __nv_bfloat162 mx = *reinterpret_cast<const __nv_bfloat162*>(&w[0]);
+#pragma unroll
+            for (int i = 1; i < 16; ++i) mx = __hmax2(mx, *reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+            const uint32_t mb = *reinterpret_cast<const uint32_t*>(&mx);
+            const float cm = fmaxf(bf16lo(mb), bf16hi(mb));
+            if (cm > -INFINITY) {
+                const uint64_t sc = pack2(scale2, scale2), no = pack2(-cm * scale2, -cm * scale2);
+                uint64_t a = pack2(0.f, 0.f), b = pack2(0.f, 0.f);
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    float t0, t1, t2, t3;
+                    unpack2(fma2(pack2(bf16lo(w[i]), bf16hi(w[i])), sc, no), t0, t1);
+                    unpack2(fma2(pack2(bf16lo(w[i + 1]), bf16hi(w[i + 1])), sc, no), t2, t3);
+                    a = add2(a, pack2(ex2_approx(t0), ex2_approx(t1)));
+                    b = add2(b, pack2(ex2_approx(t2), ex2_approx(t3)));
+                }
+                float s0, s1;
+                unpack2(add2(a, b), s0, s1);
+                s = s0 + s1;
+                m = cm;
+                return;
+            }
+        }
         float x[32];
 #pragma unroll
-        for (int v4 = 0; v4 < 4; ++v4) {
-            const uint32_t w[4] = {o[v4].x, o[v4].y, o[v4].z, o[v4].w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { x[v4 * 8 + 2 * i] = bf16lo(w[i]); x[v4 * 8 + 2 * i + 1] = bf16hi(w[i]); }
-        }
-        const int nvalid = V - col;                         // >= 32 except in the last tile
+        for (int i = 0; i < 16; ++i) { x[2 * i] = bf16lo(w[i]); x[2 * i + 1] = bf16hi(w[i]); }
         if (kStats == 2) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
@@ -460,8 +484,6 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                     }
                     ts.update(o, nt * kTileMN + c0, P.V, P.scale2);
                 }
-                if (kStats && mt * kTileMN + trow < P.R)
-                    P.stats[(size_t)(mt * kTileMN + trow) * (4 * P.n_tiles) + 4 * nt + chunk] = ts.result();
                 tc_fence_before();
                 fence_proxy_async_smem();                   // the tile is read next by the copy engine
                 __syncwarp();
@@ -478,6 +500,9 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                         stamp(40 + t);
                     }
                 }
+                // after the arrivals: their release would otherwise wait for this store to be acknowledged
+                if (kStats && mt * kTileMN + trow < P.R)
+                    P.stats[(size_t)(mt * kTileMN + trow) * (4 * P.n_tiles) + 4 * nt + chunk] = ts.result();
                 __syncwarp();
             } else {
                 const int row = mt * kTileMN + trow;
@@ -516,10 +541,10 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                     }
                     ts.update(o, col, P.V, P.scale2);
                 } while (false);
-                if (kStats && live) P.stats[(size_t)row * (4 * P.n_tiles) + 4 * nt + chunk] = ts.result();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[s]);
+                if (kStats && live) P.stats[(size_t)row * (4 * P.n_tiles) + 4 * nt + chunk] = ts.result();
             }
         }
         if (leader) bulk_wait_group_read<0>();              // shared memory stays valid until the stores have read it
