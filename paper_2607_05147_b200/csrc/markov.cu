@@ -171,28 +171,23 @@ __device__ __forceinline__ void tmem_store32(uint32_t taddr, const uint4 (&w)[8]
         : "memory");
 }
 
-// Half a row of an embedding tile: 256 B of W1[x_prev] (src; NULL = zeros) into registers by eight 256-bit loads (a full 32 B sector
-// each, all in flight at once), then into this thread's lane of tensor memory, 64 columns from taddr
-// (two bf16 per column, k ascending).
-__device__ __forceinline__ void embedding_half_row_to_tmem(const unsigned char* src, uint32_t taddr)
+// A quarter row of an embedding tile: 128 B of W1[x_prev] (src; NULL = zeros) into registers by four
+// 256-bit loads (a full 32 B sector each, all in flight at once), then into this thread's lane of tensor
+// memory, 32 columns from taddr (two bf16 per column, k ascending).
+__device__ __forceinline__ void embedding_quarter_row_to_tmem(const unsigned char* src, uint32_t taddr)
 {
-    uint4 w[2][8];
+    uint4 w[8];
 #pragma unroll
-    for (int c = 0; c < 2; ++c)
-#pragma unroll
-        for (int v = 0; v < 8; ++v) w[c][v] = make_uint4(0, 0, 0, 0);
+    for (int v = 0; v < 8; ++v) w[v] = make_uint4(0, 0, 0, 0);
     if (src)
-#pragma unroll
-    for (int c = 0; c < 2; ++c)
 #pragma unroll
         for (int v = 0; v < 8; v += 2)
             asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                         : "=r"(w[c][v].x), "=r"(w[c][v].y), "=r"(w[c][v].z), "=r"(w[c][v].w),
-                           "=r"(w[c][v + 1].x), "=r"(w[c][v + 1].y), "=r"(w[c][v + 1].z), "=r"(w[c][v + 1].w)
-                         : "l"(src + (c * 8 + v) * 16)
+                         : "=r"(w[v].x), "=r"(w[v].y), "=r"(w[v].z), "=r"(w[v].w),
+                           "=r"(w[v + 1].x), "=r"(w[v + 1].y), "=r"(w[v + 1].z), "=r"(w[v + 1].w)
+                         : "l"(src + v * 16)
                          : "memory");
-#pragma unroll
-    for (int c = 0; c < 2; ++c) tmem_store32(taddr + (uint32_t)(c * 32), w[c]);
+    tmem_store32(taddr, w);
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     tc_fence_before();
 }
@@ -340,7 +335,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
             mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1);
-            mbar_init(&a_full[s], 8);
+            mbar_init(&a_full[s], kEpiWarps);
             mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], kEpiWarps);
         }
         for (int s = 0; s < kUBuffers; ++s) mbar_init(&u_full[s], 1);
@@ -369,56 +364,58 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     if (warp != 0) pdl_wait();
     if (tid == 32) stamp(1);
     const uint32_t tmem_base = s_tmem_base;
-    const uint32_t tmem_a0 = tmem_base + 2 * kTileMN;       // embedding tile mt: columns 256 + 128 mt ..
+    const uint32_t tmem_a0 = tmem_base + 2 * kTileMN;       // this CTA's embedding tile: columns 256 .. 383
     volatile int* abort_flag = &s_abort;
     auto give_up = [&]() { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; };
-    const int my_ntiles = blockIdx.x < P.n_tiles ? (P.n_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-    const int my_tiles = my_ntiles * P.m_tiles;             // tile t: n-tile blockIdx.x + (t / m_tiles) * gridDim.x
+    // Work unit u = (vocabulary tile u / m_tiles, row tile u % m_tiles); this CTA takes u = blockIdx.x + k * gridDim.x.
+    // gridDim.x is a multiple of m_tiles, so the row tile is the same for all of them and only that tile's
+    // embeddings are needed (the CTA next door takes the other row tile of the same vocabulary tiles and
+    // finds the W2 tile in L2).
+    const int n_units = P.n_tiles * P.m_tiles;
+    const int my_tiles = (int)blockIdx.x < n_units ? (n_units - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int my_mt = (int)blockIdx.x % P.m_tiles;
+    auto unit_ntile = [&](int k) { return ((int)blockIdx.x + k * (int)gridDim.x) / P.m_tiles; };
 
     if (warp == 0) {
         // ---------------- producer: W2 tiles, one ahead ---------------------------------------------------
         if (lane == 0) {
             bool told = false;
-            if (my_ntiles == 0) { mbar_arrive(&prefetch_issued); told = true; }
-            for (int in = 0; in < my_ntiles && !*abort_flag; ++in) {
-                const int nt = blockIdx.x + in * gridDim.x, bs = in & 1;
-                if (!mbar_wait_bounded(&b_empty[bs], ((uint32_t)(in >> 1) & 1u) ^ 1u)) { give_up(); break; }
+            if (my_tiles == 0) { mbar_arrive(&prefetch_issued); told = true; }
+            for (int k = 0; k < my_tiles && !*abort_flag; ++k) {
+                const int bs = k & 1;
+                if (!mbar_wait_bounded(&b_empty[bs], ((uint32_t)(k >> 1) & 1u) ^ 1u)) { give_up(); break; }
                 mbar_arrive_expect_tx(&b_full[bs], kTileBytes);
-                bulk_g2s(sB + bs * kTileBytes, P.W2p + (size_t)nt * kTileBytes, kTileBytes, &b_full[bs]);
-                stamp(56 + in);
-                if (in == 1 || in == my_ntiles - 1) { if (!told) mbar_arrive(&prefetch_issued); told = true; }
+                bulk_g2s(sB + bs * kTileBytes, P.W2p + (size_t)unit_ntile(k) * kTileBytes, kTileBytes, &b_full[bs]);
+                if (k < 7) stamp(56 + k);
+                if (k == 1 || k == my_tiles - 1) { if (!told) mbar_arrive(&prefetch_issued); told = true; }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ---------------------------------------------------------------------
         if (lane == 0) {
-            int t = 0;
-            for (int in = 0; in < my_ntiles && !*abort_flag; ++in) {
-                const int bs = in & 1;
-                if (!mbar_wait_bounded(&b_full[bs], (uint32_t)(in >> 1) & 1u)) { give_up(); break; }
-                const uint32_t b0 = smem_u32(sB + bs * kTileBytes);
-                if (in < 2) stamp(4 + in);
-                for (int mt = 0; mt < P.m_tiles && !*abort_flag; ++mt, ++t) {
-                    const int s = t & 1;
-                    bool ok = mbar_wait_bounded(&acc_empty[s], ((uint32_t)(t >> 1) & 1u) ^ 1u);
-                    if (ok && in == 0) ok = mbar_wait_bounded(&a_full[mt], 0u);      // resident from then on
-                    if (!ok) { give_up(); break; }
-                    tc_fence_after();
+            for (int k = 0; k < my_tiles && !*abort_flag; ++k) {
+                const int s = k & 1;
+                const uint32_t ph = (uint32_t)(k >> 1) & 1u;
+                bool ok = mbar_wait_bounded(&b_full[s], ph) && mbar_wait_bounded(&acc_empty[s], ph ^ 1u);
+                if (ok && k == 0) ok = mbar_wait_bounded(&a_full[0], 0u);            // resident from then on
+                if (!ok) { give_up(); break; }
+                if (k < 2) stamp(4 + k);
+                tc_fence_after();
+                const uint32_t b0 = smem_u32(sB + s * kTileBytes);
 #pragma unroll
-                    for (int ks = 0; ks < kRank / 16; ++ks)
-                        umma_bf16_ts(tmem_base + (uint32_t)(s * kTileMN), tmem_a0 + (uint32_t)(mt * kTileMN + ks * 8),
-                                     smem_desc_kmajor(b0 + ks * 2 * kChunkBytes), ks > 0 ? 1u : 0u);
-                    umma_commit(&acc_full[s]);              // the accumulator may be read
-                    stamp(8 + t);
-                }
-                umma_commit(&b_empty[bs]);                  // the W2 tile may be overwritten
+                for (int ks = 0; ks < kRank / 16; ++ks)
+                    umma_bf16_ts(tmem_base + (uint32_t)(s * kTileMN), tmem_a0 + (uint32_t)(ks * 8),
+                                 smem_desc_kmajor(b0 + ks * 2 * kChunkBytes), ks > 0 ? 1u : 0u);
+                umma_commit(&acc_full[s]);                  // the accumulator may be read
+                umma_commit(&b_empty[s]);                   // the W2 tile may be overwritten
+                stamp(8 + k);
             }
         }
     } else {
         // ---------------- epilogue: accumulator + base logits -> bf16 ------------------------------------
         // Sixteen warps: four per tensor-memory lane quarter, each owning 32 columns of every tile.  Before
-        // the first tile each warp brings one (row tile, lane quarter, K half) of the embeddings into
-        // tensor memory.
+        // the first tile each warp brings one (lane quarter, K quarter) of the embedding tile into tensor
+        // memory.
         const int q = warp & 3;                             // TMEM lane quarter this warp may access
         const int chunk = (warp - 2) >> 2;                  // which 32 columns of a tile
         const int c0 = chunk * 32;
@@ -426,7 +423,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const bool leader = kTma && warp == 2 && lane == 0;
         auto issue_u_load = [&](int t) {
-            const int nt = blockIdx.x + (t / P.m_tiles) * gridDim.x, mt = t % P.m_tiles;
+            const int nt = unit_ntile(t), mt = my_mt;
             unsigned char* dst = sU + (t % kUBuffers) * kUTileBytes;
             mbar_arrive_expect_tx(&u_full[t % kUBuffers], kUTileBytes);
             tma_load_2d(dst, &map_u, nt * kTileMN, mt * kTileMN, &u_full[t % kUBuffers]);
@@ -438,24 +435,21 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             for (int t = 0; t < 2 && t < my_tiles; ++t) issue_u_load(t);
         if (warp == 2 && lane == 0) mbar_arrive(&prefetch_issued);
         mbar_wait_bounded(&prefetch_issued, 0u);            // a limit that runs out only costs the ordering
-        {
-            const int mt = chunk >> 1, kh = chunk & 1;      // row tile and K half this warp loads
-            if (my_tiles > 0 && mt < P.m_tiles) {
-                const int row = mt * kTileMN + trow;
-                const unsigned char* src = nullptr;         // rows past R and bad tokens: a zero embedding
-                if (row < P.R) {
-                    const int x = P.x_prev[row];
-                    if (x >= 0 && x < P.V) src = P.W1 + ((size_t)x * kRank + kh * (kRank / 2)) * 2;
-                    else if (blockIdx.x == 0 && kh == 0) atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN);
-                }
-                embedding_half_row_to_tmem(src, tmem_a0 + lane_base + (uint32_t)(mt * kTileMN + kh * (kRank / 4)));
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&a_full[mt]);
-                if (lane == 0 && q == 2 && kh == 0) stamp(2 + mt);
+        if (my_tiles > 0) {
+            const int row = my_mt * kTileMN + trow;
+            const unsigned char* src = nullptr;             // rows past R and bad tokens: a zero embedding
+            if (row < P.R) {
+                const int x = P.x_prev[row];
+                if (x >= 0 && x < P.V) src = P.W1 + ((size_t)x * kRank + chunk * (kRank / 4)) * 2;
+                else if ((int)blockIdx.x < P.m_tiles && chunk == 0) atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN);
             }
+            embedding_quarter_row_to_tmem(src, tmem_a0 + lane_base + (uint32_t)(chunk * (kRank / 8)));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&a_full[0]);
+            if (lane == 0 && q == 2 && chunk == 0) stamp(2);
         }
         for (int t = 0; t < my_tiles && !*abort_flag; ++t) {
-            const int nt = blockIdx.x + (t / P.m_tiles) * gridDim.x, mt = t % P.m_tiles;
+            const int nt = unit_ntile(t), mt = my_mt;
             const int s = t & 1, ub = t % kUBuffers;
             bool ok = mbar_wait_bounded(&acc_full[s], (uint32_t)(t >> 1) & 1u);
             if (kTma) ok = ok && mbar_wait_bounded(&u_full[ub], (uint32_t)(t / kUBuffers) & 1u);
@@ -857,7 +851,8 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
         const bool tma = g_markov_path != 1 && make_tile_map(&map_u, G.U, G.R, V, P.u_stride_bytes) &&
                          make_tile_map(&map_out, G.out, G.R, V, P.out_stride_bytes);
         KernelTimerScope timer(DSPARK_K_MARKOV_GEMM, s);
-        const dim3 grid(P.n_tiles < sms ? P.n_tiles : sms), block(kGemmThreads);
+        const int units = P.n_tiles * G.m_tiles, cap = sms - sms % G.m_tiles;     // a multiple of the row tiles
+        const dim3 grid(units < cap ? units : cap), block(kGemmThreads);
         const size_t sm = (size_t)smem_bytes;
         if (tma) {
             if (stats_mode == 0) launch_pdl(markov_gemm_kernel<true, 0>, grid, block, sm, s, G, map_u, map_out);
