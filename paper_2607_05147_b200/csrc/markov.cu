@@ -7,19 +7,23 @@
 // The bias is a dense [R,256] x [256,V] contraction, so it runs on the 5th-generation tensor cores,
 // but the step as a whole is bound by HBM (base logits in, draft logits out, W2 once), and the kernel
 // is organised around keeping those three streams in flight:
-//   * one persistent CTA per SM walks 128-column tiles of the vocabulary, 256 rows (two row tiles) per
-//     launch;
-//   * the embedding operand E = W1[x_prev] (gathered once by a small kernel) lives in TENSOR MEMORY for
-//     the whole launch: four loader warps (row tile 0) and the four epilogue warps (row tile 1) write
-//     their rows with tcgen05.st, lane = row, 128 columns of two bf16;
-//   * shared memory then holds the pre-packed W2 tile twice (the next vocabulary tile streams in by one
-//     64 KB bulk copy while the current one is multiplied) and three base-logit tiles;
+//   * a work unit is one 128-row x 128-column tile of the logits; one persistent CTA per SM walks units
+//     of ONE row tile (the grid is a multiple of the row-tile count, so CTAs that share a vocabulary
+//     tile run side by side and the second reader finds the W2 tile in L2);
+//   * the embedding operand W1[x_prev] of that row tile lives in TENSOR MEMORY for the whole launch: the
+//     sixteen epilogue warps gather their rows from the table (256-bit loads) and write them with
+//     tcgen05.st, lane = row, 128 columns of two bf16;
+//   * shared memory holds the pre-packed W2 tile twice (the next vocabulary tile streams in by one 64 KB
+//     bulk copy while the current one is multiplied) and three base-logit tiles;
 //   * one thread issues tcgen05.mma (M = N = 128, 16 steps of K = 16, A from tensor memory, B through a
 //     shared-memory descriptor) into one of two fp32 accumulators in tensor memory;
-//   * base-logit tiles arrive by 2-D tensor-map loads, the epilogue warps read the accumulator back
-//     (tcgen05.ld), add it in place, round to bf16, and the finished tile leaves by a tensor-map store.
-// The draw itself is the verifier's bonus path on the stored logits (a request with no draft position
-// emits one token from p), so what the drafter samples from is bit for bit the distribution the
+//   * base-logit tiles arrive by 2-D tensor-map loads; each epilogue warp reads 32 accumulator columns of
+//     its lane quarter back (tcgen05.ld), adds them in place, rounds to bf16 and, for a draft step, takes
+//     the softmax (or argmax) statistics of the 32 stored values; the finished tile leaves by a
+//     tensor-map store.
+// The draw is a second, small kernel on those statistics (one CTA per request): no second pass over the
+// logits.  It follows the rule of the verifier's bonus draw for a request with no draft position, applied
+// to the STORED bf16 logits, so what the drafter samples from is bit for bit the distribution the
 // verifier will later read as q.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -36,7 +40,7 @@ constexpr int kTileMN = 128;                     // M and N of one MMA tile
 constexpr int kTileBytes = kTileMN * kRank * 2;  // 64 KB of bf16: one packed W2 tile
 constexpr int kKChunks = kRank / 8;              // 16-byte chunks along K
 constexpr int kChunkBytes = kTileMN * 16;        // one K chunk of a tile: 128 columns x 16 B
-constexpr int kGroupRows = 2 * kTileMN;          // rows per launch: two row tiles resident in tensor memory
+constexpr int kGroupRows = 8 * kTileMN;          // rows per launch (the grid is cut to a multiple of the row tiles)
 constexpr int kEpiWarps = 16;                    // four per tensor-memory lane quarter, 32 columns of a tile each
 constexpr int kGemmThreads = (2 + kEpiWarps) * 32; // producer warp, MMA warp, epilogue warps
 constexpr int kTmemCols = 512;                   // accumulators: columns 0..255, embedding tiles: 256..511
@@ -101,7 +105,7 @@ __device__ __forceinline__ void block_confidence(const MarkovParams& P, int r, d
     __syncthreads();
     if (tid == 0) {
         for (int w = 1; w < nwarp; ++w) z += s_part[w];
-        P.out_conf[r] = (float)(1.0 / (1.0 + exp(-z)));
+        P.out_conf[r] = 1.f / (1.f + expf(-(float)z));      // fp32 exponential: its error is far below the 1e-6 bar
     }
 }
 
@@ -171,6 +175,19 @@ __device__ __forceinline__ void tmem_store32(uint32_t taddr, const uint4 (&w)[8]
         : "memory");
 }
 
+// two / eight consecutive 32-bit columns of this thread's lane
+__device__ __forceinline__ void tmem_store2(uint32_t taddr, uint32_t a, uint32_t b)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};\n\ttcgen05.wait::st.sync.aligned;"
+                 ::"r"(taddr), "r"(a), "r"(b) : "memory");
+}
+__device__ __forceinline__ void tmem_load8(uint32_t taddr, uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];\n\ttcgen05.wait::ld.sync.aligned;"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+}
+
 // A quarter row of an embedding tile: 128 B of W1[x_prev] (src; NULL = zeros) into registers by four
 // 256-bit loads (a full 32 B sector each, all in flight at once), then into this thread's lane of tensor
 // memory, 32 columns from taddr (two bf16 per column, k ascending).
@@ -233,8 +250,8 @@ __device__ __forceinline__ uint4 add_round(const float* acc, uint4 u)
 }
 
 // ---- per-tile statistics of the stored logits, taken in the epilogue --------------------------------
-// One entry per row and 32 columns (four per vocabulary tile, one per epilogue warp of a lane quarter),
-// called a box below.
+// One entry per row and 32 columns (four per vocabulary tile, one per epilogue warp of a lane quarter);
+// merge_entries() below folds the four into the tile's entry.
 // kStats = 1 (sampling): m = max of the 32 stored values of (row, box), s = sum of 2^((x - m) * scale2),
 //   i.e. the box's softmax mass relative to its own maximum.  A NaN or +inf element makes s NaN; a tile
 //   with no element above -inf has m = -inf, s = 0.
@@ -314,7 +331,36 @@ struct TileStats {
     __device__ __forceinline__ float2 result() const { return make_float2(m, kStats == 2 ? __int_as_float(idx) : s); }
 };
 
-// ---- the GEMM: logits = U + E W2 for one group of at most 256 rows, bf16 out -------------------------
+// The four 32-column entries of one (row, tile), as (m, s) pairs in column order, merged into the entry
+// of the 128-column tile.
+template <int kStats>
+__device__ __forceinline__ float2 merge_entries(const uint32_t (&e)[8], float scale2)
+{
+    if (kStats == 2) {
+        float best = -INFINITY;
+        int idx = -1;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float m = __uint_as_float(e[2 * i]);
+            const int id = (int)e[2 * i + 1];
+            if (id >= 0 && m > best) { best = m; idx = id; }   // earlier columns win ties
+        }
+        return make_float2(best, __int_as_float(idx));
+    }
+    float M = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) M = fmaxf(M, __uint_as_float(e[2 * i]));
+    float S = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float m = __uint_as_float(e[2 * i]), s = __uint_as_float(e[2 * i + 1]);
+        // a part without mass (m = -inf, s = 0) adds 0; a NaN sum (NaN or +inf element) carries over
+        S += (s == 0.f) ? 0.f : s * ex2_approx((m - M) * scale2);
+    }
+    return make_float2(M, S);
+}
+
+// ---- the GEMM: logits = U + W1[x_prev] W2 for one group of rows, bf16 out -----------------------------
 // kTma: base-logit tiles and finished tiles move through the tensor maps (ring of three buffers, added
 // in place).  Otherwise (a base address or row pitch that breaks the 16-byte rules) the epilogue
 // threads load and store their rows directly.
@@ -460,6 +506,17 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             tc_fence_after();
             if (leader) stamp(24 + t);
             const uint32_t acc_addr = tmem_base + lane_base + (uint32_t)(s * kTileMN);
+            // Statistics: every warp leaves the (m, s) of its 32 columns in two spare tensor-memory columns of
+            // its lanes (four rotating slots of 8 columns from column 384).  The accumulator of tile t can
+            // only have been produced after all warps released tile t - 2, i.e. after they wrote that
+            // tile's entries: one warp per lane quarter merges them now and stores the tile's entry.
+            const uint32_t stat_base = tmem_base + lane_base + (uint32_t)(3 * kTileMN);
+            if (kStats && t >= 2 && chunk == ((t - 2) & 3)) {
+                uint32_t e[8];
+                tmem_load8(stat_base + (uint32_t)(((t - 2) & 3) * 8), e);
+                const int row = my_mt * kTileMN + trow;
+                if (row < P.R) P.stats[(size_t)row * P.n_tiles + unit_ntile(t - 2)] = merge_entries<kStats>(e, P.scale2);
+            }
             TileStats<kStats> ts;
             ts.reset();
             if (kTma) {
@@ -478,6 +535,10 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                     }
                     ts.update(o, nt * kTileMN + c0, P.V, P.scale2);
                 }
+                if (kStats) {
+                    const float2 r2 = ts.result();
+                    tmem_store2(stat_base + (uint32_t)((t & 3) * 8 + chunk * 2), __float_as_uint(r2.x), __float_as_uint(r2.y));
+                }
                 tc_fence_before();
                 fence_proxy_async_smem();                   // the tile is read next by the copy engine
                 __syncwarp();
@@ -494,9 +555,6 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                         stamp(40 + t);
                     }
                 }
-                // after the arrivals: their release would otherwise wait for this store to be acknowledged
-                if (kStats && mt * kTileMN + trow < P.R)
-                    P.stats[(size_t)(mt * kTileMN + trow) * (4 * P.n_tiles) + 4 * nt + chunk] = ts.result();
                 __syncwarp();
             } else {
                 const int row = mt * kTileMN + trow;
@@ -535,16 +593,34 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                     }
                     ts.update(o, col, P.V, P.scale2);
                 } while (false);
+                if (kStats) {
+                    const float2 r2 = ts.result();
+                    tmem_store2(stat_base + (uint32_t)((t & 3) * 8 + chunk * 2), __float_as_uint(r2.x), __float_as_uint(r2.y));
+                }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[s]);
-                if (kStats && live) P.stats[(size_t)row * (4 * P.n_tiles) + 4 * nt + chunk] = ts.result();
             }
         }
         if (leader) bulk_wait_group_read<0>();              // shared memory stays valid until the stores have read it
     }
-    // everyone meets here; then the allocating warp returns the tensor memory
+    // everyone meets here; the entries of the last two tiles are merged; then the allocating warp returns
+    // the tensor memory
     tc_fence_before();
+    __syncthreads();
+    if (kStats && warp >= 2 && !*abort_flag) {
+        tc_fence_after();
+        const int chunk = (warp - 2) >> 2;
+        const int row = my_mt * kTileMN + (warp & 3) * 32 + lane;
+#pragma unroll 1
+        for (int t = my_tiles > 2 ? my_tiles - 2 : 0; t < my_tiles; ++t) {
+            if (chunk != (t & 3)) continue;
+            uint32_t e[8];
+            tmem_load8(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(3 * kTileMN + (t & 3) * 8), e);
+            if (row < P.R) P.stats[(size_t)row * P.n_tiles + unit_ntile(t)] = merge_entries<kStats>(e, P.scale2);
+        }
+        tc_fence_before();
+    }
     __syncthreads();
     if (tid == 32) stamp(63);
     if (warp == 1) {
@@ -553,19 +629,19 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     }
 }
 
-// ---- the draw: one token per request from the box statistics -----------------------------------------
-// One CTA of 256 threads per request; thread t owns the kDrawPer consecutive boxes starting at
-// t * per (per = boxes per row / 256, rounded up), so thread order is vocabulary order.
-// Sampling (greedy == 0): with M the row maximum and z_i = s_i 2^((m_i - M) scale2) the mass of box i,
+// ---- the draw: one token per request from the tile statistics ---------------------------------------
+// One CTA of 256 threads per request; thread t owns the `per` consecutive tiles starting at t * per
+// (per = tiles per row / 256, rounded up), so thread order is vocabulary order.
+// Sampling (greedy == 0): with M the row maximum and z_i = s_i 2^((m_i - M) scale2) the mass of tile i,
 // the running sum (within a thread, then across threads) gives the total Z; the token is the smallest v
 // whose running sum of 2^((x_v - M) scale2) exceeds u' Z, u' the second uniform of (seed, request,
-// position 0): the box is located on the box masses, the element inside it on the 32 stored logits of
-// that box.  A row with NaN, +inf or no finite element sets DSPARK_DEV_BAD_ROW and yields -1.
+// position 0): the tile is located on the tile masses, the element inside it on the 128 stored logits of
+// that tile.  A row with NaN, +inf or no finite element sets DSPARK_DEV_BAD_ROW and yields -1.
 // Greedy: the lowest index of the row maximum; a row with nothing above -inf sets
 // DSPARK_DEV_ALL_NEG_INF and yields 0.
-constexpr int kDrawThreads = 512;
-constexpr int kStatCols = 32;                    // columns per statistics entry
-constexpr int kDrawPer = 16;                     // entries per thread at most: V <= 512 * 16 * 32
+constexpr int kDrawThreads = 256;
+constexpr int kStatCols = kTileMN;               // columns per statistics entry
+constexpr int kDrawPer = 16;                     // entries per thread at most: V <= 256 * 16 * 128
 constexpr int kMaxDrawV = kDrawThreads * kDrawPer * kStatCols;
 
 __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams P, int greedy, uint64_t seed, int32_t* out_tokens)
@@ -579,7 +655,7 @@ __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams 
     if (P.out_conf) block_confidence(P, blockIdx.x, s_part);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r = blockIdx.x;
-    const int n_box = 4 * P.n_tiles;
+    const int n_box = P.n_tiles;
     const int per = (n_box + kDrawThreads - 1) / kDrawThreads;
     const float2* st = P.stats + (size_t)r * n_box;
     float2 e[kDrawPer];
@@ -665,8 +741,10 @@ __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams 
             if (z[k] > 0.f) lastp = tid * per + k;
             if (mine == 0x7fffffff && z[k] > 0.f && run > thr) mine = tid * per + k;
         }
-        if (mine != 0x7fffffff) atomicMin(&s_box, mine);
-        if (lastp >= 0) atomicMax(&s_last, lastp);
+        mine = __reduce_min_sync(0xffffffffu, mine);          // one shared-memory atomic per warp
+        lastp = __reduce_max_sync(0xffffffffu, lastp);
+        if (lane == 0 && mine != 0x7fffffff) atomicMin(&s_box, mine);
+        if (lane == 0 && lastp >= 0) atomicMax(&s_last, lastp);
     }
     __syncthreads();
     const int box = s_box != 0x7fffffff ? s_box : s_last;
@@ -681,20 +759,32 @@ __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams 
     }
     __syncthreads();
     if (warp != 0) return;
-    // inside the box: one column per lane
+    // inside the tile: four consecutive columns per lane
     const float before = found ? s_before : 0.f;
     const float thr_in = found ? thr : INFINITY;            // rounding left the sum at or below thr: the last token with mass
     const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(P.out + (long long)r * P.out_stride_bytes);
-    const int c = box * kStatCols + lane;
-    const float ev = c < P.V ? ex2_approx(fmaf(__bfloat162float(row[c]), P.scale2, -offM)) : 0.f;
-    float linc = ev;
+    const int c0 = box * kStatCols + lane * 4;
+    float ev[4];
+    float lsum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        ev[i] = c0 + i < P.V ? ex2_approx(fmaf(__bfloat162float(row[c0 + i]), P.scale2, -offM)) : 0.f;
+        lsum += ev[i];
+    }
+    float linc = lsum;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const float n = __shfl_up_sync(0xffffffffu, linc, o);
         if (lane >= o) linc += n;
     }
-    const int tok = (ev > 0.f && before + linc > thr_in) ? c : -1;
-    const int lastp = ev > 0.f ? c : -1;
+    float cum = before + (linc - lsum);
+    int tok = -1, lastp = -1;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        cum += ev[i];
+        if (ev[i] > 0.f) lastp = c0 + i;
+        if (tok < 0 && ev[i] > 0.f && cum > thr_in) tok = c0 + i;
+    }
     const unsigned hit = __ballot_sync(0xffffffffu, tok >= 0);
     const unsigned pos = __ballot_sync(0xffffffffu, lastp >= 0);
     int result;
@@ -709,7 +799,7 @@ static MarkovWs markov_layout(int R, int V)
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
     MarkovWs w;
     size_t o = 0;
-    w.stats = o;  o += up((size_t)R * 4 * ((V + kTileMN - 1) / kTileMN) * sizeof(float2));
+    w.stats = o;  o += up((size_t)R * ((V + kTileMN - 1) / kTileMN) * sizeof(float2));
     w.trace = o;
 #ifdef DSPARK_MARKOV_TRACE
     o += up(256 * 64 * 8);
@@ -792,7 +882,7 @@ size_t dspark_markov_workspace_bytes(int R, int V)
     return markov_layout(R, V).total;
 }
 
-// one GEMM launch per 256-row group; stats_mode 0 none, 1 softmax masses, 2 argmax
+// one GEMM launch per group of rows; stats_mode 0 none, 1 softmax masses, 2 argmax
 static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
                          const int32_t* x_prev, int R, int V,
                          const void* H, int64_t h_row_stride, int d, const float* w_conf,
@@ -835,8 +925,8 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
         if (!ok) return launch_status();
         g_gemm_attr_set[dev & 63] = true;
     }
-    // one launch per group of 256 rows: both row tiles of a group stay in tensor memory while the CTA
-    // walks its vocabulary tiles (W2 is streamed once per group)
+    // one launch per group of up to 1024 rows (8 row tiles): W2 is fetched from HBM once per group, the
+    // CTAs that share a vocabulary tile run side by side and find it in L2
     for (int r0 = 0; r0 < R; r0 += kGroupRows) {
         MarkovParams G = P;
         G.R = R - r0 < kGroupRows ? R - r0 : kGroupRows;
@@ -844,7 +934,7 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
         G.U = P.U + (long long)r0 * P.u_stride_bytes;
         G.out = P.out + (long long)r0 * P.out_stride_bytes;
         G.x_prev = P.x_prev + r0;
-        G.stats = P.stats + (size_t)r0 * 4 * P.n_tiles;
+        G.stats = P.stats + (size_t)r0 * P.n_tiles;
         CUtensorMap map_u, map_out;
         memset(&map_u, 0, sizeof map_u);
         memset(&map_out, 0, sizeof map_out);
