@@ -87,33 +87,37 @@ __global__ void markov_pack_w2_kernel(const __nv_bfloat16* __restrict__ W2, int 
 }
 
 // ---- confidence head: c = sigmoid(w . [h ; W1[x_prev]]), one CTA per request ---------------------------
-// Every thread takes a strided share of the d + 256 products in fp64 (a handful each), the block adds
-// them up.  All threads of the CTA must call it; thread 0 writes the result.
-__device__ __forceinline__ void block_confidence(const MarkovParams& P, int r, double* s_part)
+// Every thread takes a strided share of the d + 256 products (a handful each, fp32 multiply-adds), the
+// warp adds its threads' shares; the caller adds the warps' shares after a __syncthreads and applies
+// the sigmoid.  The fp32 rounding of the ~1300 terms stays two orders below the 1e-6 bar on c.
+__device__ __forceinline__ float confidence_warp_share(const MarkovParams& P, int r)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
+    const int tid = threadIdx.x;
     const int x = P.x_prev[r];
-    double z = 0.0;
+    float z = 0.f;
     const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(P.H + (long long)r * P.h_stride_bytes);
-    for (int i = tid; i < P.d; i += blockDim.x) z += (double)P.w_conf[i] * (double)__bfloat162float(h[i]);
+    for (int i = tid; i < P.d; i += blockDim.x) z = fmaf(P.w_conf[i], __bfloat162float(h[i]), z);
     if (x >= 0 && x < P.V) {
         const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(P.W1) + (size_t)x * kRank;
-        for (int i = tid; i < kRank; i += blockDim.x) z += (double)P.w_conf[P.d + i] * (double)__bfloat162float(e[i]);
+        for (int i = tid; i < kRank; i += blockDim.x) z = fmaf(P.w_conf[P.d + i], __bfloat162float(e[i]), z);
     }
-    z = warp_sum_f64(z);
-    if (lane == 0) s_part[warp] = z;
-    __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < nwarp; ++w) z += s_part[w];
-        P.out_conf[r] = 1.f / (1.f + expf(-(float)z));      // fp32 exponential: its error is far below the 1e-6 bar
-    }
+    return warp_sum_f32(z);
+}
+__device__ __forceinline__ float sigmoid_of_shares(const float* s_part, int nwarp)
+{
+    double z = 0.0;
+    for (int w = 0; w < nwarp; ++w) z += (double)s_part[w];
+    return 1.f / (1.f + expf(-(float)z));
 }
 
 __global__ void __launch_bounds__(256) markov_confidence_kernel(MarkovParams P)
 {
-    __shared__ double s_part[8];
+    __shared__ float s_part[8];
     pdl_wait();
-    block_confidence(P, blockIdx.x, s_part);
+    const float z = confidence_warp_share(P, blockIdx.x);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = z;
+    __syncthreads();
+    if (threadIdx.x == 0) P.out_conf[blockIdx.x] = sigmoid_of_shares(s_part, 8);
 }
 
 // ---- tcgen05 helpers --------------------------------------------------------------------------------
@@ -650,9 +654,8 @@ __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams 
     __shared__ int s_redi[kDrawThreads / 32];
     __shared__ float s_before;
     __shared__ int s_box, s_last, s_bad;
-    __shared__ double s_part[kDrawThreads / 32];
+    __shared__ float s_part[kDrawThreads / 32];
     pdl_wait();
-    if (P.out_conf) block_confidence(P, blockIdx.x, s_part);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r = blockIdx.x;
     const int n_box = P.n_tiles;
@@ -665,7 +668,12 @@ __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams 
         e[k] = (k < per && i < n_box) ? st[i] : make_float2(-INFINITY, greedy ? __int_as_float(-1) : 0.f);
     }
     if (tid == 0) { s_box = 0x7fffffff; s_last = -1; s_bad = 0; }
+    if (P.out_conf) {                                       // its loads overlap the statistics loads above
+        const float zc = confidence_warp_share(P, r);
+        if (lane == 0) s_part[warp] = zc;
+    }
     __syncthreads();
+    if (P.out_conf && tid == 32) P.out_conf[r] = sigmoid_of_shares(s_part, kDrawThreads / 32);
     if (greedy) {
         float best = -INFINITY;
         int bi = 0x7fffffff;
