@@ -303,3 +303,28 @@ def confidence(H, W1, w, x_prev):
     if rc != 0:
         raise ValueError(f"orc_confidence failed ({rc})")
     return out
+
+
+def sts_calibrate(conf, accepted_len, grid, n_bins: int = 15, verified_len=None):
+    """Sequential Temperature Scaling.  conf float32 [N, gamma]; returns (T[gamma] float32, ece_before, ece_after,
+    ece_grid[gamma, G]) with the ECE values in fp64."""
+    c = np.ascontiguousarray(conf, dtype=np.float32)
+    N, gamma = c.shape
+    acc = np.ascontiguousarray(accepted_len, dtype=np.int32)
+    ver = None if verified_len is None else np.ascontiguousarray(verified_len, dtype=np.int32)
+    g = np.ascontiguousarray(grid, dtype=np.float32)
+    T = np.empty(gamma, dtype=np.float32)
+    eb = np.empty(gamma); ea = np.empty(gamma); eg = np.empty((gamma, len(g)))
+    rc = lib().orc_sts_calibrate(_p(c), C.c_int(N), C.c_int(gamma), _p(acc), _p(ver), _p(g), C.c_int(len(g)),
+                                 C.c_int(n_bins), _p(T), _p(eb), _p(ea), _p(eg))
+    if rc != 0:
+        raise ValueError(f"orc_sts_calibrate failed ({rc})")
+    return T, eb, ea, eg
+
+
+def sts_apply(conf, T):
+    c = np.ascontiguousarray(conf, dtype=np.float32)
+    t = np.ascontiguousarray(T, dtype=np.float32)
+    out = np.empty(c.shape)
+    lib().orc_sts_apply(_p(c), C.c_int(c.shape[0]), C.c_int(c.shape[1]), _p(t), _p(out))
+    return out

@@ -767,3 +767,96 @@ int orc_verify_greedy_mt(const void* target, int dtype, int64_t target_row_strid
         if (jobs[t].r_end > jobs[t].r_begin) pthread_join(th[t], NULL);
     return 0;
 }
+
+/* ------------------------------------------------------------------------ */
+/* Sequential Temperature Scaling (Section 3.2.1, "Post-hoc Calibration").   */
+/* From left to right, position k gets the temperature of a 1-D grid that     */
+/* minimises the Expected Calibration Error of the cumulative product         */
+/*   a_{n,k} = prod_{i<=k} sigmoid(logit(c_{n,i}) / T_i)                      */
+/* over held-out blocks n, with T_1..T_{k-1} already fixed.  The label of     */
+/* (n, k) is 1 when the block's draft prefix through k was accepted           */
+/* (accepted_len[n] > k, positions 0-based); a block counts at position k     */
+/* only if that position was verified (k < verified_len[n]; NULL = all).      */
+/* Readings where the paper is silent: temperature scaling acts on the logit  */
+/* of the sigmoid output; a confidence outside (0,1) is clamped to [0,1]       */
+/* (NaN -> 0) and not rescaled; ECE uses n_bins equal-width bins on [0,1],     */
+/*   ECE = (1/N_k) * sum_b | sum_{n in b} y_n - sum_{n in b} a_n |,            */
+/* bin(a) = min(n_bins-1, floor(a*n_bins)); ties take the first grid point;    */
+/* a position nobody verified keeps T = 1.                                     */
+/* ------------------------------------------------------------------------ */
+static double sts_scaled(double c, double T)
+{
+    if (c != c || c <= 0.0) return 0.0;
+    if (c >= 1.0) return 1.0;
+    double z = log(c) - log1p(-c);
+    return 1.0 / (1.0 + exp(-z / T));
+}
+
+static double sts_ece(const double* a, const uint8_t* y, const uint8_t* used, int N, int n_bins)
+{
+    double* sum_a = (double*)calloc((size_t)n_bins, sizeof(double));
+    double* sum_y = (double*)calloc((size_t)n_bins, sizeof(double));
+    long cnt = 0;
+    for (int n = 0; n < N; ++n) {
+        if (!used[n]) continue;
+        int b = (int)floor(a[n] * n_bins);
+        if (b > n_bins - 1) b = n_bins - 1;
+        if (b < 0) b = 0;
+        sum_a[b] += a[n];
+        sum_y[b] += y[n];
+        ++cnt;
+    }
+    double e = 0.0;
+    for (int b = 0; b < n_bins; ++b) e += fabs(sum_y[b] - sum_a[b]);
+    free(sum_a); free(sum_y);
+    return cnt ? e / (double)cnt : 0.0;
+}
+
+int orc_sts_calibrate(const float* conf, int N, int gamma, const int32_t* accepted_len,
+                      const int32_t* verified_len, const float* grid, int G, int n_bins,
+                      float* out_T, double* ece_before, double* ece_after, double* ece_grid)
+{
+    if (N <= 0 || gamma <= 0 || G <= 0 || n_bins <= 0) return -1;
+    for (int g = 0; g < G; ++g) if (!(grid[g] > 0.f) || isinf(grid[g])) return -2;
+    double* a_raw = (double*)malloc(sizeof(double) * (size_t)N);   /* product of raw confidences   */
+    double* a_cal = (double*)malloc(sizeof(double) * (size_t)N);   /* product of calibrated ones   */
+    double* a_try = (double*)malloc(sizeof(double) * (size_t)N);
+    uint8_t* y = (uint8_t*)malloc((size_t)N);
+    uint8_t* used = (uint8_t*)malloc((size_t)N);
+    for (int n = 0; n < N; ++n) a_raw[n] = a_cal[n] = 1.0;
+    for (int k = 0; k < gamma; ++k) {
+        long cnt = 0;
+        for (int n = 0; n < N; ++n) {
+            used[n] = (uint8_t)(!verified_len || k < verified_len[n]);
+            y[n] = (uint8_t)(accepted_len[n] > k);
+            cnt += used[n];
+            a_raw[n] *= sts_scaled((double)conf[(size_t)n * gamma + k], 1.0);
+        }
+        if (ece_before) ece_before[k] = sts_ece(a_raw, y, used, N, n_bins);
+        int best = -1;
+        double best_e = 0.0;
+        for (int g = 0; g < G && cnt > 0; ++g) {
+            for (int n = 0; n < N; ++n)
+                a_try[n] = a_cal[n] * sts_scaled((double)conf[(size_t)n * gamma + k], (double)grid[g]);
+            double e = sts_ece(a_try, y, used, N, n_bins);
+            if (ece_grid) ece_grid[(size_t)k * G + g] = e;
+            if (best < 0 || e < best_e) { best = g; best_e = e; }
+        }
+        if (cnt == 0 && ece_grid) for (int g = 0; g < G; ++g) ece_grid[(size_t)k * G + g] = 0.0;
+        double T = best >= 0 ? (double)grid[best] : 1.0;
+        out_T[k] = (float)T;
+        for (int n = 0; n < N; ++n) a_cal[n] *= sts_scaled((double)conf[(size_t)n * gamma + k], T);
+        if (ece_after) ece_after[k] = sts_ece(a_cal, y, used, N, n_bins);
+    }
+    free(a_raw); free(a_cal); free(a_try); free(y); free(used);
+    return 0;
+}
+
+/* Calibrated confidences for the scheduler: c~ = sigmoid(logit(c) / T_k). */
+int orc_sts_apply(const float* conf, int N, int gamma, const float* T, double* out)
+{
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < gamma; ++k)
+            out[(size_t)n * gamma + k] = sts_scaled((double)conf[(size_t)n * gamma + k], (double)T[k]);
+    return 0;
+}
