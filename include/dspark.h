@@ -329,6 +329,35 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
                              void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
                              int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------
+ * Sequential Temperature Scaling of the confidence head (Section 3.2.1, "Post-hoc Calibration").
+ * From left to right, position k receives the temperature T_k of a caller-given grid that minimises
+ * the Expected Calibration Error of the cumulative product a_{n,k} = prod_{i<=k} sigmoid(logit(c_{n,i}) / T_i)
+ * over N held-out draft blocks, T_1..T_{k-1} already fixed:
+ *     ECE_k = (1/N_k) sum_b | sum_{n in b} y_{n,k} - sum_{n in b} a_{n,k} |,  b = min(n_bins-1, floor(a n_bins)),
+ * y_{n,k} = 1 iff accepted_len[n] > k; block n counts at position k iff k < verified_len[n].
+ *  conf          device fp32 [N, gamma]: raw confidences of the head; a value outside (0,1) is clamped to
+ *                [0,1] (NaN -> 0) and never rescaled
+ *  accepted_len  device int32 [N]: accepted draft tokens of the block (what the verifier returned)
+ *  verified_len  device int32 [N] or NULL (= gamma): how many positions of the block were verified
+ *  grid          device fp32 [G]: candidate temperatures, all > 0 (not checked on the device); ties
+ *                take the first grid point
+ *  n_bins        1..64 equal-width bins
+ *  out_T         device fp32 [gamma]; a position nobody verified gets 1
+ *  out_ece_before / out_ece_after  device fp64 [gamma] or NULL: ECE of the raw and of the calibrated chain
+ *  out_ece_grid  device fp64 [gamma, G] or NULL: ECE of every candidate
+ * The products are fp32, per-bin sums of a are exact integers (a * 2^32 truncated), the ECE is fp64.
+ * dspark_sts_apply writes sigmoid(logit(c) / T_k) for every entry: the confidences to hand to
+ * dspark_schedule.  Temperature scaling keeps the order of the confidences of a position.
+ * workspace: dspark_sts_workspace_bytes(N, gamma, G, n_bins), 256-byte aligned.
+ * Errors: INVALID_ARG, SHAPE (n_bins > 64), WORKSPACE, ALIGNMENT, CUDA.
+ */
+size_t dspark_sts_workspace_bytes(int N, int gamma, int G, int n_bins);
+int dspark_sts_calibrate(const float* conf, int N, int gamma, const int32_t* accepted_len, const int32_t* verified_len,
+                         const float* grid, int G, int n_bins, float* out_T, double* out_ece_before,
+                         double* out_ece_after, double* out_ece_grid, void* workspace, size_t workspace_bytes, void* stream);
+int dspark_sts_apply(const float* conf, int N, int gamma, const float* T, float* out, void* stream);
+
 /* The two uniforms of (seed, request, position) exactly as the verifier draws them
  * (host computation; for tests and for replaying a step). */
 void dspark_uniforms(uint64_t seed, uint32_t request, uint32_t position,

@@ -33,6 +33,7 @@ EXPORTS = [
     "dspark_accept_rate", "dspark_accept_rate_workspace_bytes",
     "dspark_markov_w2_packed_bytes", "dspark_markov_pack_w2", "dspark_markov_workspace_bytes",
     "dspark_markov_logits", "dspark_markov_draft_step", "dspark_markov_set_epilogue_path",
+    "dspark_sts_workspace_bytes", "dspark_sts_calibrate", "dspark_sts_apply",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
     "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
     "dspark_version",
@@ -89,6 +90,10 @@ def lib() -> C.CDLL:
         L.dspark_markov_logits.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, vp, i64, vp, vp, vp, sz, vp]
         L.dspark_markov_draft_step.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, C.c_float, u64,
                                                vp, i64, vp, vp, vp, vp, sz, vp]
+        L.dspark_sts_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        L.dspark_sts_workspace_bytes.restype = sz
+        L.dspark_sts_calibrate.argtypes = [vp, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.dspark_sts_apply.argtypes = [vp, i32, i32, vp, vp, vp]
         L.dspark_uniforms.argtypes = [u64, C.c_uint32, C.c_uint32, C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.dspark_uniforms.restype = None
         L.dspark_ktimer_create.argtypes = [i32, C.POINTER(vp)]
@@ -416,6 +421,44 @@ def dspark_markov_draft_step(U: torch.Tensor, W1: torch.Tensor, W2_packed: torch
                                         _dev(dev_status, "dev_status", torch.int32),
                                         _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_markov_draft_step")
+
+
+def dspark_sts_workspace_bytes(N: int, gamma: int, G: int, n_bins: int) -> int:
+    return int(lib().dspark_sts_workspace_bytes(N, gamma, G, n_bins))
+
+
+def dspark_sts_calibrate(conf: torch.Tensor, accepted_len: torch.Tensor, grid: torch.Tensor, n_bins: int = 15, *,
+                         verified_len: Optional[torch.Tensor] = None, out_T: torch.Tensor,
+                         out_ece_before: Optional[torch.Tensor] = None, out_ece_after: Optional[torch.Tensor] = None,
+                         out_ece_grid: Optional[torch.Tensor] = None, workspace: torch.Tensor) -> None:
+    if conf.dim() != 2 or not conf.is_contiguous():
+        raise DsparkError("conf must be a contiguous [N, gamma] tensor")
+    N, gamma = conf.shape
+    G = grid.numel()
+    if accepted_len.numel() < N or out_T.numel() < gamma or (verified_len is not None and verified_len.numel() < N):
+        raise DsparkError("accepted_len / verified_len need N entries, out_T gamma")
+    for t, n, name in ((out_ece_before, gamma, "out_ece_before"), (out_ece_after, gamma, "out_ece_after"),
+                       (out_ece_grid, gamma * G, "out_ece_grid")):
+        if t is not None and (t.numel() < n or not t.is_contiguous()):
+            raise DsparkError(f"{name} is too small")
+    rc = lib().dspark_sts_calibrate(_dev(conf, "conf", torch.float32), N, gamma,
+                                    _dev(accepted_len, "accepted_len", torch.int32),
+                                    _dev(verified_len, "verified_len", torch.int32), _dev(grid, "grid", torch.float32), G,
+                                    int(n_bins), _dev(out_T, "out_T", torch.float32),
+                                    _dev(out_ece_before, "out_ece_before", torch.float64),
+                                    _dev(out_ece_after, "out_ece_after", torch.float64),
+                                    _dev(out_ece_grid, "out_ece_grid", torch.float64), _dev(workspace, "workspace"),
+                                    workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_sts_calibrate")
+
+
+def dspark_sts_apply(conf: torch.Tensor, T: torch.Tensor, out: torch.Tensor) -> None:
+    if conf.dim() != 2 or not conf.is_contiguous() or out.shape != conf.shape or not out.is_contiguous():
+        raise DsparkError("conf and out must be contiguous [N, gamma] tensors of one shape")
+    if T.numel() < conf.shape[1]:
+        raise DsparkError("T needs gamma entries")
+    _check(lib().dspark_sts_apply(_dev(conf, "conf", torch.float32), conf.shape[0], conf.shape[1],
+                                  _dev(T, "T", torch.float32), _dev(out, "out", torch.float32), _stream()), "dspark_sts_apply")
 
 
 def dspark_uniforms(seed: int, request: int, position: int):

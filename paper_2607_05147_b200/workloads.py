@@ -270,6 +270,28 @@ def markov_input(R: int, V: int, seed: int, device, d: int = 1024, sigma: float 
     return MarkovInput(U, W1, W2, x_prev, H, w_conf)
 
 
+
+def sts_input(N: int, gamma: int, seed: int, device, overconfidence: float = 2.0, partial: bool = True):
+    """Held-out blocks for the calibration of the confidence head: true conditional acceptance
+    probabilities sigmoid(z), z ~ N(1.2 - 0.05 k, 1); the head reports sigmoid(overconfidence * z); a
+    block is verified up to a random length (partial) and accepted up to the first failed draw.
+    Returns (conf [N, gamma] fp32, accepted_len [N] int32, verified_len [N] int32)."""
+    g = _gen(seed, device)
+    k = torch.arange(gamma, device=device, dtype=torch.float32)
+    z = torch.randn(N, gamma, generator=g, device=device) + (1.2 - 0.05 * k)
+    ok = torch.rand(N, gamma, generator=g, device=device) < torch.sigmoid(z)
+    if partial:
+        ver = torch.randint(1, gamma + 1, (N,), generator=g, device=device, dtype=torch.int32)
+    else:
+        ver = torch.full((N,), gamma, device=device, dtype=torch.int32)
+    ok = ok & (k[None, :] < ver[:, None])
+    fail = (~ok).to(torch.int32)
+    acc = torch.where(fail.any(1), fail.argmax(1).to(torch.int32), torch.full((N,), gamma, device=device, dtype=torch.int32))
+    acc = torch.minimum(acc, ver)
+    conf = torch.sigmoid(overconfidence * z).to(torch.float32)
+    return conf.contiguous(), acc.contiguous(), ver.contiguous()
+
+
 def bf16_bits(t: torch.Tensor):
     """Host numpy view of a tensor for the oracle: fp32 as is, bf16 as raw uint16 patterns."""
     import numpy as np
