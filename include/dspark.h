@@ -286,7 +286,10 @@ int dspark_accept_rate(const void* target_logits, const void* draft_logits, int 
  *
  * dspark_markov_pack_w2: one-time re-layout of W2 (device, bf16, row-major [256, V]) into the
  *   tile order the contraction reads (device, dspark_markov_w2_packed_bytes(V), 16-byte aligned;
- *   columns past V are zero).  The caller owns both buffers.
+ *   columns past V are zero).  The caller owns both buffers.  Done once when the weights are loaded:
+ *   the call synchronises `stream` and returns after the re-layout has completed (the contraction
+ *   prefetches the packed weights ahead of its stream dependencies, so they must never be in flight
+ *   while a draft step is enqueued; not capturable in a CUDA graph).
  * dspark_markov_logits:
  *   U            device bf16 [R, >= V], row stride u_row_stride elements: base logits of position k
  *   W1           device bf16 [V, 256] row-major, 32-byte aligned

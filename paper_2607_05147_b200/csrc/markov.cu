@@ -881,7 +881,11 @@ int dspark_markov_pack_w2(const void* W2, int V, void* W2_packed, void* stream)
     const long long total = (long long)n_tiles * kTileMN * kKChunks;
     markov_pack_w2_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
         (const __nv_bfloat16*)W2, V, n_tiles, (unsigned char*)W2_packed);
-    return launch_status();
+    const int rc = launch_status();
+    // The contraction starts fetching the packed weights before it waits for the kernel ahead of it on the
+    // stream, so they must be complete, not merely enqueued, when this call returns.
+    if (rc == DSPARK_OK && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return launch_status();
+    return rc;
 }
 
 size_t dspark_markov_workspace_bytes(int R, int V)
