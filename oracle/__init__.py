@@ -328,3 +328,22 @@ def sts_apply(conf, T):
     out = np.empty(c.shape)
     lib().orc_sts_apply(_p(c), C.c_int(c.shape[0]), C.c_int(c.shape[1]), _p(t), _p(out))
     return out
+
+
+def warp_target(target, row_offsets, top_k=None, top_p=None, temperature: float = 1.0, temperatures=None):
+    """Top-k / top-p truncation of the target rows of a ragged batch: returns (masked copy, tau[n_rows],
+    kept[n_rows], margin[n_rows]).  target: float32 or bf16 bit patterns (uint16), [n_rows, V]."""
+    t = np.array(target, copy=True)
+    tt, stride = _logits(t)
+    ro = np.ascontiguousarray(row_offsets, dtype=np.int32)
+    R = len(ro) - 1
+    k = None if top_k is None else np.ascontiguousarray(top_k, dtype=np.int32)
+    p = None if top_p is None else np.ascontiguousarray(top_p, dtype=np.float32)
+    temps = None if temperatures is None else np.ascontiguousarray(temperatures, dtype=np.float32)
+    n_rows = t.shape[0]
+    tau = np.full(n_rows, -np.inf); kept = np.full(n_rows, t.shape[1], dtype=np.int32); margin = np.full(n_rows, np.inf)
+    rc = lib().orc_warp_target(_p(tt), C.c_int(_dtype_code(tt)), C.c_int64(stride), C.c_int(t.shape[1]), _p(ro), C.c_int(R),
+                               _p(k), _p(p), C.c_double(temperature), _p(temps), _p(tau), _p(kept), _p(margin))
+    if rc != 0:
+        raise ValueError(f"orc_warp_target failed ({rc})")
+    return tt, tau, kept, margin

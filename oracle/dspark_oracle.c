@@ -860,3 +860,95 @@ int orc_sts_apply(const float* conf, int N, int gamma, const float* T, double* o
             out[(size_t)n * gamma + k] = sts_scaled((double)conf[(size_t)n * gamma + k], (double)T[k]);
     return 0;
 }
+
+/* ------------------------------------------------------------------------ */
+/* Top-k / top-p truncation of the target distribution (per-request sampling */
+/* parameters; the paper evaluates with "recommended sampling parameters",    */
+/* Section 4.1, and gives no rule of its own).  Readings:                     */
+/*  - the truncated distribution is obtained by setting the logits of the     */
+/*    excluded tokens to -inf, so that softmax renormalises over the kept set  */
+/*    S and the lossless verifier runs unchanged on the masked rows;           */
+/*  - S is a value cut, S = { v : x_v >= tau }: every token tied with the      */
+/*    threshold value is kept (no dependence on token order);                  */
+/*  - top-k first: tau_k = k-th largest logit (0 or >= V: off); then top-p on  */
+/*    the distribution renormalised over the top-k set: walking the distinct   */
+/*    values downwards, tau_p is the first value at which the cumulative mass  */
+/*    reaches top_p * Z_k (top_p >= 1: off; top_p <= 0: only the maximum);     */
+/*    tau = max(tau_k, tau_p);                                                 */
+/*  - a row with NaN, +inf or no finite element is left as it is (the          */
+/*    verifier reports it).                                                    */
+/* Every target row of request r uses top_k[r], top_p[r] and its temperature.  */
+/* margin[row]: relative distance of top_p * Z_k from the nearest cumulative   */
+/* mass at a value boundary (how close the top-p decision was); +inf if none.  */
+/* ------------------------------------------------------------------------ */
+static int cmp_desc_double(const void* a, const void* b)
+{
+    double x = *(const double*)a, y = *(const double*)b;
+    return x > y ? -1 : (x < y ? 1 : 0);
+}
+
+int orc_warp_target(void* target, int dtype, int64_t stride, int V, const int32_t* row_offsets, int R,
+                    const int32_t* top_k, const float* top_p, double temperature, const float* temperatures,
+                    double* tau_out, int32_t* kept_out, double* margin_out)
+{
+    if (R <= 0 || V <= 0) return -1;
+    double* v = (double*)malloc(sizeof(double) * (size_t)V);
+    for (int r = 0; r < R; ++r) {
+        const double T = temperatures ? (double)temperatures[r] : temperature;
+        const int k = top_k ? top_k[r] : 0;
+        const double pr = top_p ? (double)top_p[r] : 1.0;
+        for (int row = row_offsets[r]; row < row_offsets[r + 1]; ++row) {
+            if (tau_out) tau_out[row] = -INFINITY;
+            if (kept_out) kept_out[row] = V;
+            if (margin_out) margin_out[row] = INFINITY;
+            const int use_k = k > 0 && k < V, use_p = pr < 1.0;
+            if (!use_k && !use_p) continue;
+            if (!(T > 0.0) || isinf(T)) continue;
+            int bad = 0;
+            for (int i = 0; i < V; ++i) { v[i] = logit_at(target, dtype, row, stride, i); if (v[i] != v[i]) bad = 1; }
+            qsort(v, (size_t)V, sizeof(double), cmp_desc_double);
+            const double m = v[0];
+            if (bad || m == INFINITY || m == -INFINITY) continue;
+            double tau_k = -INFINITY;
+            int n_k = V;                                   /* size of the top-k set, ties included */
+            if (use_k) {
+                tau_k = v[k - 1];
+                n_k = k;
+                while (n_k < V && v[n_k] == tau_k) ++n_k;
+            }
+            double tau = tau_k;
+            if (use_p) {
+                double Zk = 0.0;
+                for (int i = 0; i < n_k; ++i) Zk += exp((v[i] - m) / T);
+                const double thr = pr * Zk;
+                double cum = 0.0, margin = INFINITY, tau_p = m;
+                int i = 0;
+                if (pr > 0.0) {
+                    while (i < n_k) {                       /* one group of equal values at a time */
+                        const double val = v[i];
+                        const double before = cum;
+                        while (i < n_k && v[i] == val) { cum += exp((val - m) / T); ++i; }
+                        tau_p = val;
+                        double d0 = fabs(thr - before) / Zk, d1 = fabs(cum - thr) / Zk;
+                        if (d0 < margin) margin = d0;
+                        if (d1 < margin) margin = d1;
+                        if (cum >= thr) break;
+                    }
+                }
+                if (tau_p > tau) tau = tau_p;
+                if (margin_out) margin_out[row] = margin;
+            }
+            int kept = 0;
+            for (int i = 0; i < V; ++i) {
+                double x = logit_at(target, dtype, row, stride, i);
+                if (x >= tau) { ++kept; continue; }
+                if (dtype == ORC_BF16) ((uint16_t*)target)[(size_t)row * stride + i] = 0xFF80u;   /* -inf */
+                else ((float*)target)[(size_t)row * stride + i] = -INFINITY;
+            }
+            if (tau_out) tau_out[row] = tau;
+            if (kept_out) kept_out[row] = kept;
+        }
+    }
+    free(v);
+    return 0;
+}
