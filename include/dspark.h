@@ -333,6 +333,33 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
                              int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------
+ * dspark_truncate_target -- top-k / top-p truncation of the target distribution, per request (Section 4.1
+ * evaluates with the models' recommended sampling parameters; the paper states no rule of its own).
+ * The logits of the excluded tokens of every target row are set to -inf IN PLACE, so that softmax
+ * renormalises over the kept set and dspark_verify / dspark_verify_per_request, run afterwards on the same
+ * rows, are lossless with respect to the truncated target distribution.
+ *   kept set S = { v : x_v >= tau } (a value cut: every token tied with the threshold value is kept);
+ *   top-k first: tau_k = k-th largest logit of the row (top_k[r] <= 0 or >= V: off); then top-p on the
+ *   distribution renormalised over the top-k set: walking the distinct values downwards, tau_p is the first
+ *   value at which the cumulative mass reaches top_p[r] * Z_k (top_p >= 1: off; <= 0: only the maximum);
+ *   tau = max(tau_k, tau_p).  p = softmax(row / T_r).
+ *  target_logits   device bf16 [n_rows, >= V], modified in place; dtype must be DSPARK_BF16 (the threshold
+ *                  is found exactly on the 16-bit keys) -- DSPARK_F32 returns DSPARK_ERR_SHAPE
+ *  row_offsets, R, n_rows   the ragged batch of the verifiers; every row of request r uses r's parameters
+ *  top_k           device int32 [R] or NULL;  top_p  device fp32 [R] or NULL (both NULL: nothing to do)
+ *  temperature / temperatures   one T > 0, or device fp32 [R] (a T that is not positive and finite leaves
+ *                  that request's rows alone)
+ *  out_tau         device fp32 [n_rows] or NULL: threshold value of each row (-inf: untouched)
+ *  out_kept        device int32 [n_rows] or NULL: size of the kept set (V: untouched)
+ * A row with NaN, +inf or no finite element is left as it is (the verifier reports it).  Costs one read of
+ * the row from HBM, two from L2 and one write.  No workspace.  Errors: INVALID_ARG, SHAPE, CUDA.
+ */
+int dspark_truncate_target(void* target_logits, int dtype, int64_t target_row_stride, int V,
+                           const int32_t* row_offsets, int R, int n_rows,
+                           const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
+                           float* out_tau, int32_t* out_kept, int32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------------------
  * Sequential Temperature Scaling of the confidence head (Section 3.2.1, "Post-hoc Calibration").
  * From left to right, position k receives the temperature T_k of a caller-given grid that minimises
  * the Expected Calibration Error of the cumulative product a_{n,k} = prod_{i<=k} sigmoid(logit(c_{n,i}) / T_i)

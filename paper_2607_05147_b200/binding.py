@@ -33,6 +33,7 @@ EXPORTS = [
     "dspark_accept_rate", "dspark_accept_rate_workspace_bytes",
     "dspark_markov_w2_packed_bytes", "dspark_markov_pack_w2", "dspark_markov_workspace_bytes",
     "dspark_markov_logits", "dspark_markov_draft_step", "dspark_markov_set_epilogue_path",
+    "dspark_truncate_target",
     "dspark_sts_workspace_bytes", "dspark_sts_calibrate", "dspark_sts_apply",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
     "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
@@ -90,6 +91,7 @@ def lib() -> C.CDLL:
         L.dspark_markov_logits.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, vp, i64, vp, vp, vp, sz, vp]
         L.dspark_markov_draft_step.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, C.c_float, u64,
                                                vp, i64, vp, vp, vp, vp, sz, vp]
+        L.dspark_truncate_target.argtypes = [vp, i32, i64, i32, vp, i32, i32, vp, vp, C.c_float, vp, vp, vp, vp, vp]
         L.dspark_sts_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.dspark_sts_workspace_bytes.restype = sz
         L.dspark_sts_calibrate.argtypes = [vp, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
@@ -421,6 +423,26 @@ def dspark_markov_draft_step(U: torch.Tensor, W1: torch.Tensor, W2_packed: torch
                                         _dev(dev_status, "dev_status", torch.int32),
                                         _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_markov_draft_step")
+
+
+def dspark_truncate_target(target: torch.Tensor, row_offsets: torch.Tensor, *, top_k: Optional[torch.Tensor] = None,
+                           top_p: Optional[torch.Tensor] = None, temperature: float = 1.0,
+                           temperatures: Optional[torch.Tensor] = None, out_tau: Optional[torch.Tensor] = None,
+                           out_kept: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> None:
+    """Masks the excluded tokens of every target row to -inf in place (bf16 rows)."""
+    tp, code, ts = _logits(target, "target")
+    R = row_offsets.numel() - 1
+    n_rows = target.shape[0]
+    for t, n, name in ((top_k, R, "top_k"), (top_p, R, "top_p"), (temperatures, R, "temperatures"),
+                       (out_tau, n_rows, "out_tau"), (out_kept, n_rows, "out_kept")):
+        if t is not None and t.numel() < n:
+            raise DsparkError(f"{name} is too small")
+    rc = lib().dspark_truncate_target(tp, code, ts, target.shape[1], _dev(row_offsets, "row_offsets", torch.int32), R, n_rows,
+                                      _dev(top_k, "top_k", torch.int32), _dev(top_p, "top_p", torch.float32),
+                                      float(temperature), _dev(temperatures, "temperatures", torch.float32),
+                                      _dev(out_tau, "out_tau", torch.float32), _dev(out_kept, "out_kept", torch.int32),
+                                      _dev(dev_status, "dev_status", torch.int32), _stream())
+    _check(rc, "dspark_truncate_target")
 
 
 def dspark_sts_workspace_bytes(N: int, gamma: int, G: int, n_bins: int) -> int:
