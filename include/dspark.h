@@ -297,7 +297,8 @@ int dspark_accept_rate(const void* target_logits, const void* draft_logits, int 
  *   x_prev       device int32 [R]: previous token of each request (anchor token at k = 1); a value
  *                outside [0, V) sets DSPARK_DEV_BAD_TOKEN and contributes a zero embedding
  *   H, w_conf    device bf16 [R, >= d] (stride h_row_stride) and device fp32 [d + 256]; read only
- *                when out_conf is non-NULL.  The dot product is accumulated in fp64.
+ *                when out_conf is non-NULL.  The d + 256 products are accumulated in fp32 (error far
+ *                below 1e-6 on the confidence).
  *   out_logits   device bf16 [R, >= V], row stride out_row_stride elements
  *   out_conf     device fp32 [R] or NULL
  *   workspace    dspark_markov_workspace_bytes(R, V), 256-byte aligned
@@ -309,8 +310,11 @@ int dspark_accept_rate(const void* target_logits, const void* draft_logits, int 
  *   per 128-column tile inside the contraction's epilogue, so the logits are not read a second time.
  *   A row with NaN, +inf or no finite element sets DSPARK_DEV_BAD_ROW and yields -1.
  *   out_tokens device int32 [R].
- * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, CUDA; a device wait that ran out sets
- * DSPARK_DEV_TIMEOUT in *dev_status and the affected logits are unspecified.
+ * Resources: the contraction runs one CTA per SM with 225 KB of shared memory and allocates all 512
+ * tensor-memory columns of the SM for its lifetime; a concurrent kernel that needs tensor memory waits.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, CUDA; SHAPE from dspark_markov_draft_step when V exceeds
+ * 524 288 (the draw keeps one statistics entry per 128 columns in registers); a device wait that ran out
+ * sets DSPARK_DEV_TIMEOUT in *dev_status and the affected logits are unspecified.
  */
 /* Diagnostic switch for the epilogue of dspark_markov_logits: 0 = automatic (base logits and draft
  * logits move through 2-D tensor-map copies when both base addresses are 16-byte aligned and both

@@ -43,7 +43,7 @@ constexpr int kChunkBytes = kTileMN * 16;        // one K chunk of a tile: 128 c
 constexpr int kGroupRows = 8 * kTileMN;          // rows per launch (the grid is cut to a multiple of the row tiles)
 constexpr int kEpiWarps = 16;                    // four per tensor-memory lane quarter, 32 columns of a tile each
 constexpr int kGemmThreads = (2 + kEpiWarps) * 32; // producer warp, MMA warp, epilogue warps
-constexpr int kTmemCols = 512;                   // accumulators: columns 0..255, embedding tiles: 256..511
+constexpr int kTmemCols = 512;                   // accumulators: columns 0..255, embedding tile: 256..383, statistics: 384..415
 
 // Packed W2 tile (K-major, no swizzle): element (n, k) of a 128-column x 256 tile lives at
 //   (k / 8) * 2048 + (n / 8) * 128 + (n % 8) * 16 + (k % 8) * 2   bytes,
