@@ -81,3 +81,79 @@ def test_schedule_fuzz(seed):
         mode = int(rng.choice([B.DSPARK_SCHED_EARLY_STOP, B.DSPARK_SCHED_GLOBAL, B.DSPARK_SCHED_TOPK]))
         dl = rng.integers(0, gamma + 2, size=R).astype(np.int32) if rng.random() < 0.3 else None
         H.check_schedule(s, mode, topk=int(rng.integers(0, R * gamma + 2)), draft_len=dl)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_truncate_fuzz(seed):
+    import oracle
+    rng = np.random.default_rng(3000 + seed)
+    for _ in range(5):
+        R = int(rng.integers(1, 12))
+        V = int(rng.choice([1, 2, 9, 64, 255, 1000, 4097, 20000]))
+        lengths = rng.integers(0, 4, size=R)
+        off = np.concatenate([[0], np.cumsum(lengths + 1)]).astype(np.int32)
+        n_rows = int(off[-1])
+        kind = rng.integers(0, 3)
+        if kind == 0:
+            t = torch.randn(n_rows, V) * float(rng.uniform(0.2, 6))
+        elif kind == 1:
+            t = torch.from_numpy(rng.integers(-4, 5, (n_rows, V)).astype(np.float32)) * 0.25      # heavy ties
+        else:
+            t = torch.from_numpy(rng.uniform(-30, 30, (n_rows, V)).astype(np.float32))
+        t = _pad_rows(t.to(torch.bfloat16).cuda(), rng)
+        ks = rng.integers(-1, V + 3, size=R).astype(np.int32)
+        ps = rng.choice([0.0, 0.1, 0.5, 0.9, 0.99, 1.0, 1.5], size=R).astype(np.float32)
+        Ts = rng.uniform(0.3, 2.5, size=R).astype(np.float32)
+        got = t.clone()
+        tau = torch.empty(n_rows, device="cuda"); kept = torch.empty(n_rows, dtype=torch.int32, device="cuda")
+        B.dspark_truncate_target(got, torch.from_numpy(off).cuda(), top_k=torch.from_numpy(ks).cuda(),
+                                 top_p=torch.from_numpy(ps).cuda(), temperatures=torch.from_numpy(Ts).cuda(),
+                                 out_tau=tau, out_kept=kept)
+        torch.cuda.synchronize()
+        bits = W.bf16_bits(t)
+        want, otau, okept, margin = oracle.warp_target(bits, off, top_k=ks, top_p=ps, temperatures=Ts)
+        gb = W.bf16_bits(got)
+        for row in range(n_rows):
+            if margin[row] < 1e-5:
+                continue                                  # a top-p decision on its boundary: either neighbour is right
+            np.testing.assert_array_equal(gb[row], want[row], err_msg=f"row {row} V={V} k={ks} p={ps}")
+            assert int(kept[row]) == okept[row]
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_markov_fuzz(seed):
+    import oracle
+    rng = np.random.default_rng(4000 + seed)
+    for _ in range(3):
+        R = int(rng.integers(1, 400))
+        V = int(rng.choice([8, 129, 1000, 2048, 4097, 9000]))
+        T = float(rng.choice([0.0, 0.5, 1.0, 1.7]))
+        m = W.markov_input(R, V, int(rng.integers(0, 10**6)), "cuda", d=int(rng.choice([8, 100, 256])),
+                           sigma=float(rng.uniform(0.5, 4)))
+        packed = torch.empty(B.dspark_markov_w2_packed_bytes(V), dtype=torch.uint8, device="cuda")
+        B.dspark_markov_pack_w2(m.W2, packed)
+        U = _pad_rows(m.U, rng)
+        out = _pad_rows(torch.zeros_like(m.U), rng)
+        conf = torch.empty(R, device="cuda"); toks = torch.empty(R, dtype=torch.int32, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ws = B.workspace(B.dspark_markov_workspace_bytes(R, V)).fill_(0xFF)
+        seed_v = int(rng.integers(0, 2**40))
+        B.dspark_markov_draft_step(U, m.W1, packed, m.x_prev, T, seed_v, H=m.H, w_conf=m.w_conf, out_logits=out,
+                                   out_tokens=toks, out_conf=conf, dev_status=st, workspace=ws)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        exact, bits = oracle.markov_logits(W.bf16_bits(m.U), W.bf16_bits(m.W1), W.bf16_bits(m.W2), m.x_prev.cpu().numpy())
+        got = W.bf16_bits(out.contiguous())
+        diff = np.abs(got.astype(np.int32) - bits.astype(np.int32))
+        assert diff[np.abs(exact) >= 2.0 ** -4].max(initial=0) <= 1 and float((diff != 0).mean()) <= 5e-3
+        want_c = oracle.confidence(W.bf16_bits(m.H), W.bf16_bits(m.W1), m.w_conf.cpu().numpy(), m.x_prev.cpu().numpy())
+        assert np.abs(conf.cpu().numpy() - want_c).max() <= 1e-6
+        off = np.arange(R + 1, dtype=np.int32)
+        tk = toks.cpu().numpy()
+        if T == 0.0:
+            o = oracle.verify_greedy(got, off, np.zeros(R, dtype=np.int32))
+            np.testing.assert_array_equal(tk, o.out_tokens[:R])
+        else:
+            o = oracle.verify(got, got, off, np.zeros(R, dtype=np.int32), T, seed_v)
+            for r in np.nonzero(tk != o.out_tokens[:R])[0]:
+                assert o.token_margin[r] < 1e-6, (r, tk[r], o.out_tokens[r], o.token_margin[r])
