@@ -47,6 +47,7 @@ ASYNC_TOPK = False
 CUDA_GRAPH = False
 OVERLAP = False
 PER_REQUEST_T = False
+TRUNCATE = None          # (top_k, top_p) for every request: dspark_verify_truncated
 
 
 def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=False):
@@ -217,6 +218,14 @@ class Step:
         if self.wl["greedy"]:
             B.dspark_verify_greedy(batch.target, offsets, batch.draft_tokens, accepted_len=self.acc,
                                    out_tokens=self.out, dev_status=self.status, workspace=self.ws, n_rows=self.n_rows)
+        elif TRUNCATE is not None:
+            if not hasattr(self, "top_k"):
+                self.top_k = torch.full((self.R,), int(TRUNCATE[0]), dtype=torch.int32, device=self.acc.device)
+                self.top_p = torch.full((self.R,), float(TRUNCATE[1]), dtype=torch.float32, device=self.acc.device)
+            B.dspark_verify_truncated(batch.target, batch.draft, offsets, batch.draft_tokens, batch.seed,
+                                      temperature=batch.temperature, top_k=self.top_k, top_p=self.top_p,
+                                      draft_row_start=batch.draft_row_start, accepted_len=self.acc, out_tokens=self.out,
+                                      dev_status=self.status, workspace=self.ws, n_rows=self.n_rows)
         elif PER_REQUEST_T:
             if not hasattr(self, "temps"):
                 self.temps = torch.full((self.R,), float(batch.temperature), device=self.acc.device)
@@ -469,6 +478,8 @@ def main():
                     help="schedule with dspark_schedule_async (capacity from two steps earlier, Section 4.2)")
     ap.add_argument("--per-request-temperature", action="store_true",
                     help="verify with dspark_verify_per_request (a device array of R temperatures)")
+    ap.add_argument("--top-k", type=int, default=0, help="verify against the top-k truncated target (every request)")
+    ap.add_argument("--top-p", type=float, default=1.0, help="verify against the top-p truncated target (every request)")
     ap.add_argument("--overlap-schedule", action="store_true",
                     help="with --async-topk: schedule step t+1 on a second stream while step t is verified "
                          "(the asynchronous scheduler is off the critical path, Section 4.2)")
@@ -484,7 +495,9 @@ def main():
                     help="timed steps only (no clock probe, per-kernel timing, e2e or CPU legs): for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    global REQUESTS_OVERRIDE, ASYNC_TOPK, CUDA_GRAPH, OVERLAP, PER_REQUEST_T
+    global REQUESTS_OVERRIDE, ASYNC_TOPK, CUDA_GRAPH, OVERLAP, PER_REQUEST_T, TRUNCATE
+    if args.top_k > 0 or args.top_p < 1.0:
+        TRUNCATE = (args.top_k, args.top_p)
     PER_REQUEST_T = args.per_request_temperature
     REQUESTS_OVERRIDE = args.requests
     ASYNC_TOPK, CUDA_GRAPH = args.async_topk, args.cuda_graph
@@ -681,6 +694,7 @@ def main():
                        "scheduler": ("async top-K, capacity from two steps earlier" if ASYNC_TOPK else "early stop")
                        if wl["sched"] is not None else None,
                        "temperature": "per request (device array)" if PER_REQUEST_T else "one per batch",
+                       "truncation": None if TRUNCATE is None else f"top_k={TRUNCATE[0]}, top_p={TRUNCATE[1]} (dspark_verify_truncated)",
                        "launch": "CUDA graph replay" if CUDA_GRAPH else
                        ("stream launches, scheduler of step t+1 overlapped on a second stream" if OVERLAP
                         else "stream launches"),

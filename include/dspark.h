@@ -363,6 +363,25 @@ int dspark_truncate_target(void* target_logits, int dtype, int64_t target_row_st
                            const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
                            float* out_tau, int32_t* out_kept, int32_t* dev_status, void* stream);
 
+/* dspark_verify_truncated -- dspark_verify / dspark_verify_per_request on the top-k / top-p truncated target
+ * distribution of dspark_truncate_target, without modifying the target rows: after the statistics pass one
+ * kernel finds the threshold tau of every target row (same rule, same exact search on the 16-bit keys) and
+ * replaces the row's block sums by the sums over the kept set; the accept test, the residual pass and the
+ * final draws then treat a target logit below tau as -inf.  The draft distribution q is used as given.
+ * Costs one extra read of the target rows (plus one from L2 / shared memory) instead of the read + write of
+ * dspark_truncate_target.  temperatures / top_k / top_p: device [R] or NULL (temperatures NULL: the scalar
+ * `temperature`; top_k and top_p both NULL: plain dspark_verify).  out_p_tok reports the truncated p(x).
+ * bf16 only (DSPARK_F32 with top_k or top_p: DSPARK_ERR_SHAPE).  Same workspace as dspark_verify.
+ */
+int dspark_verify_truncated(const void* target_logits, const void* draft_logits, int dtype,
+                            int64_t target_row_stride, int64_t draft_row_stride, int V,
+                            const int32_t* row_offsets, const int64_t* draft_row_start,
+                            const int32_t* draft_tokens, int R, int n_rows,
+                            float temperature, const float* temperatures, const int32_t* top_k, const float* top_p,
+                            uint64_t seed, int32_t* accepted_len, int32_t* out_tokens,
+                            float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
 /* ------------------------------------------------------------------------------------
  * Sequential Temperature Scaling of the confidence head (Section 3.2.1, "Post-hoc Calibration").
  * From left to right, position k receives the temperature T_k of a caller-given grid that minimises
@@ -408,7 +427,8 @@ typedef struct dspark_ktimer dspark_ktimer_t;
 enum {
     DSPARK_K_SCHEDULE = 0, DSPARK_K_OFFSETS = 1, DSPARK_K_STREAM = 2, DSPARK_K_DECIDE = 3,
     DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6, DSPARK_K_GREEDY_DECIDE = 7,
-    DSPARK_K_ROW_SCALE = 8, DSPARK_K_MARKOV_GEMM = 9, DSPARK_K_MARKOV_DRAW = 10, DSPARK_K_COUNT = 11
+    DSPARK_K_ROW_SCALE = 8, DSPARK_K_MARKOV_GEMM = 9, DSPARK_K_MARKOV_DRAW = 10, DSPARK_K_TRUNCATE = 11,
+    DSPARK_K_COUNT = 12
 };
 int dspark_ktimer_create(int capacity, dspark_ktimer_t** out);
 int dspark_ktimer_destroy(dspark_ktimer_t* t);

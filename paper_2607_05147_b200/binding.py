@@ -22,7 +22,7 @@ DSPARK_SCHED_EARLY_STOP, DSPARK_SCHED_GLOBAL, DSPARK_SCHED_TOPK = 0, 1, 2
 DEV_BAD_OFFSETS, DEV_BAD_TOKEN, DEV_BAD_ROW, DEV_TIMEOUT = 1, 2, 4, 8
 DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF, DEV_BAD_TEMPERATURE = 16, 32, 64, 128
 (K_SCHEDULE, K_OFFSETS, K_STREAM, K_DECIDE, K_RESIDUAL, K_FINALIZE, K_GREEDY_STREAM, K_GREEDY_DECIDE,
- K_ROW_SCALE, K_MARKOV_GEMM, K_MARKOV_DRAW, K_COUNT) = range(12)
+ K_ROW_SCALE, K_MARKOV_GEMM, K_MARKOV_DRAW, K_TRUNCATE, K_COUNT) = range(13)
 
 EXPORTS = [
     "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",
@@ -33,7 +33,7 @@ EXPORTS = [
     "dspark_accept_rate", "dspark_accept_rate_workspace_bytes",
     "dspark_markov_w2_packed_bytes", "dspark_markov_pack_w2", "dspark_markov_workspace_bytes",
     "dspark_markov_logits", "dspark_markov_draft_step", "dspark_markov_set_epilogue_path",
-    "dspark_truncate_target",
+    "dspark_truncate_target", "dspark_verify_truncated",
     "dspark_sts_workspace_bytes", "dspark_sts_calibrate", "dspark_sts_apply",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
     "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
@@ -91,6 +91,8 @@ def lib() -> C.CDLL:
         L.dspark_markov_logits.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, vp, i64, vp, vp, vp, sz, vp]
         L.dspark_markov_draft_step.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, C.c_float, u64,
                                                vp, i64, vp, vp, vp, vp, sz, vp]
+        L.dspark_verify_truncated.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, C.c_float, vp, vp, vp, u64,
+                                              vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_truncate_target.argtypes = [vp, i32, i64, i32, vp, i32, i32, vp, vp, C.c_float, vp, vp, vp, vp, vp]
         L.dspark_sts_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.dspark_sts_workspace_bytes.restype = sz
@@ -329,6 +331,36 @@ def dspark_verify_per_request(target: torch.Tensor, draft: torch.Tensor, row_off
         _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
         workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_verify_per_request")
+
+
+def dspark_verify_truncated(target: torch.Tensor, draft: torch.Tensor, row_offsets: torch.Tensor,
+                            draft_tokens: torch.Tensor, seed: int, *, temperature: float = 1.0,
+                            temperatures: Optional[torch.Tensor] = None, top_k: Optional[torch.Tensor] = None,
+                            top_p: Optional[torch.Tensor] = None, draft_row_start: Optional[torch.Tensor] = None,
+                            accepted_len: torch.Tensor, out_tokens: torch.Tensor,
+                            out_p_tok: Optional[torch.Tensor] = None, out_q_tok: Optional[torch.Tensor] = None,
+                            dev_status: Optional[torch.Tensor], workspace: torch.Tensor,
+                            n_rows: Optional[int] = None) -> None:
+    """Sampling verification against the top-k / top-p truncated target distribution (rows not modified)."""
+    tp, code, ts = _logits(target, "target")
+    dp, dcode, ds = _logits(draft, "draft")
+    if code != dcode or target.shape[1] != draft.shape[1]:
+        raise DsparkError("target and draft logits must share dtype and vocabulary size")
+    R = row_offsets.numel() - 1
+    for t, name in ((temperatures, "temperatures"), (top_k, "top_k"), (top_p, "top_p")):
+        if t is not None and t.numel() != R:
+            raise DsparkError(f"{name} must have one entry per request")
+    n_rows = target.shape[0] if n_rows is None else n_rows
+    rc = lib().dspark_verify_truncated(
+        tp, dp, code, ts, ds, target.shape[1], _dev(row_offsets, "row_offsets", torch.int32),
+        _dev(draft_row_start, "draft_row_start", torch.int64), _dev(draft_tokens, "draft_tokens", torch.int32),
+        R, n_rows, float(temperature), _dev(temperatures, "temperatures", torch.float32),
+        _dev(top_k, "top_k", torch.int32), _dev(top_p, "top_p", torch.float32), int(seed) & 0xFFFFFFFFFFFFFFFF,
+        _dev(accepted_len, "accepted_len", torch.int32), _dev(out_tokens, "out_tokens", torch.int32),
+        _dev(out_p_tok, "out_p_tok", torch.float32), _dev(out_q_tok, "out_q_tok", torch.float32),
+        _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_verify_truncated")
 
 
 def dspark_accept_rate_workspace_bytes(R: int, n_rows: int, V: int) -> int:

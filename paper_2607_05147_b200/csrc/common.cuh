@@ -192,6 +192,13 @@ struct KernelTimerScope {
 };
 int launch_status();   // maps cudaGetLastError() to DSPARK_OK / DSPARK_ERR_CUDA
 
+// Threshold search of the top-k / top-p truncation run inside the sampling verifier (truncate.cu): writes
+// the threshold of every target row to tau_rows (-inf: no cut) and replaces the block sums of the row's
+// statistics by the sums over the kept set; the rows themselves are not modified.
+int truncate_virtual_launch(const void* target, long long stride_bytes, int V, const int32_t* row_offsets, int R, int n_rows,
+                            const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
+                            float* tau_rows, float2* stats_t, int nblk, int epb, cudaStream_t stream);
+
 // Launch with programmatic stream serialization (the kernel must call pdl_wait() first).
 template <typename... KArgs, typename... Args>
 inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)

@@ -36,6 +36,9 @@ struct TruncParams {
     const int32_t* row_offsets; int R, n_rows;
     const int32_t* top_k; const float* top_p; const float* temperatures; float temperature;
     float* out_tau; int32_t* out_kept; int32_t* dev_status;
+    // virtual mode (inside the verifier): the row is not modified; its statistics blocks receive the sums
+    // restricted to the kept set instead
+    float2* stats; int nblk, epb;
 };
 
 // order-preserving 16-bit key of a bf16 pattern (-0 and +0 share a key; NaN is handled by the caller)
@@ -395,8 +398,50 @@ __device__ void truncate_row(const TruncParams& P, const int row, uint4* cache)
         if (dist_p >= 0 && (dist < 0 || dist_p < dist)) dist = dist_p;
     }
     if (dist < 0) return;                                   // nothing to cut (rounding left the sum below the threshold)
-    // ---- pass 2: mask ------------------------------------------------------------------------------------------
     const uint32_t tau_key = kmax - (uint32_t)dist;
+    if (P.stats) {
+        // ---- virtual mode: block sums of the verifier's statistics, restricted to x >= tau --------------------
+        // (c, s) of a block: c = max * scale, s = sum 2^(x * scale - c); the maximum of the row is always
+        // kept, so only the sums change.  One warp per block; a block whose maximum lies below tau gets 0.
+        const float tau_f = value_of_key(tau_key);
+        const float ctau = __fmul_rn(tau_f, scale2);
+        float2* st = P.stats + (long long)row * P.nblk;
+        const int chunks_per_block = P.epb >> 3;
+        const int n_full = V >> 3, n_cached = (A.vec && n_full < kCacheChunks) ? n_full : (A.vec ? kCacheChunks : 0);
+        for (int b = warp; b < P.nblk; b += kTruncThreads / 32) {
+            const float2 e = st[b];
+            float sum = 0.f;
+            if (e.x >= ctau && e.x > -INFINITY) {
+                const uint64_t sc2 = pack2(scale2, scale2), nc2 = pack2(-e.x, -e.x);
+                uint64_t acc = pack2(0.f, 0.f);
+                for (int i = lane; i < chunks_per_block; i += 32) {
+                    const int c = b * chunks_per_block + i;
+                    if (c * 8 >= V) break;
+                    const uint4 v = c < n_cached ? cache[c] : A.load(c);
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float x0 = bf16lo(w[q]), x1 = bf16hi(w[q]);
+                        x0 = x0 >= tau_f ? x0 : -INFINITY;
+                        x1 = x1 >= tau_f ? x1 : -INFINITY;
+                        float t0, t1;
+                        unpack2(fma2(pack2(x0, x1), sc2, nc2), t0, t1);
+                        acc = add2(acc, pack2(ex2_approx(t0), ex2_approx(t1)));
+                    }
+                }
+                float a0, a1;
+                unpack2(acc, a0, a1);
+                sum = warp_sum_f32(a0 + a1);
+            }
+            if (lane == 0) st[b].y = sum;
+        }
+        if (tid == 0) {
+            if (P.out_tau) P.out_tau[row] = tau_f;
+            if (P.out_kept) P.out_kept[row] = (int32_t)kept;
+        }
+        return;
+    }
+    // ---- pass 2: mask ------------------------------------------------------------------------------------------
     const __nv_bfloat16 tau_b = __float2bfloat16(value_of_key(tau_key));
     const __nv_bfloat162 tau2 = __halves2bfloat162(tau_b, tau_b);
     for_each_chunk<false>(A, cache, [&](int c, uint4 v) {
@@ -427,6 +472,35 @@ __global__ void __launch_bounds__(kTruncThreads) truncate_kernel(TruncParams P)
     truncate_row(P, blockIdx.x, cache);
 }
 
+static int launch_truncate(const TruncParams& P, cudaStream_t stream)
+{
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const size_t smem = (size_t)kCacheChunks * sizeof(uint4);
+    if (!attr_set[dev & 63]) {
+        if (cudaFuncSetAttribute(truncate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return launch_status();
+        attr_set[dev & 63] = true;
+    }
+    launch_pdl(truncate_kernel, dim3(P.n_rows), dim3(kTruncThreads), smem, stream, P);
+    return launch_status();
+}
+
+// Used by the sampling verifier after its statistics pass (virtual truncation: rows stay as they are).
+int truncate_virtual_launch(const void* target, long long stride_bytes, int V, const int32_t* row_offsets, int R, int n_rows,
+                            const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
+                            float* tau_rows, float2* stats_t, int nblk, int epb, cudaStream_t stream)
+{
+    TruncParams P;
+    P.target = (unsigned char*)const_cast<void*>(target); P.stride_bytes = stride_bytes; P.V = V;
+    P.row_offsets = row_offsets; P.R = R; P.n_rows = n_rows;
+    P.top_k = top_k; P.top_p = top_p; P.temperatures = temperatures; P.temperature = temperature;
+    P.out_tau = tau_rows; P.out_kept = nullptr; P.dev_status = nullptr;
+    P.stats = stats_t; P.nblk = nblk; P.epb = epb;
+    return launch_truncate(P, stream);
+}
+
 }  // namespace dspark
 
 using namespace dspark;
@@ -447,17 +521,8 @@ int dspark_truncate_target(void* target_logits, int dtype, int64_t target_row_st
     P.row_offsets = row_offsets; P.R = R; P.n_rows = n_rows;
     P.top_k = top_k; P.top_p = top_p; P.temperatures = temperatures; P.temperature = temperature;
     P.out_tau = out_tau; P.out_kept = out_kept; P.dev_status = dev_status;
-    static bool attr_set[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    const size_t smem = (size_t)kCacheChunks * sizeof(uint4);
-    if (!attr_set[dev & 63]) {
-        if (cudaFuncSetAttribute(truncate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return launch_status();
-        attr_set[dev & 63] = true;
-    }
-    launch_pdl(truncate_kernel, dim3(n_rows), dim3(kTruncThreads), smem, (cudaStream_t)stream, P);
-    return launch_status();
+    P.stats = nullptr; P.nblk = 0; P.epb = 0;
+    return launch_truncate(P, (cudaStream_t)stream);
 }
 
 }  // extern "C"

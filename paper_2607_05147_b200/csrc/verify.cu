@@ -35,7 +35,7 @@ struct __align__(16) ResidTask {     // one rejected request queued for the resi
     float u;                         // resample uniform of the rejected position
     float scale;                     // log2(e) / T of this request
     int32_t wslot;                   // which row of the block-sum array receives the result
-    int32_t pad;
+    float tau;                       // truncation threshold of the target row (-inf: none): p = 0 below it
 };
 
 struct __align__(16) RequestRec {    // what the finalize kernel needs per request (written by decide)
@@ -45,7 +45,8 @@ struct __align__(16) RequestRec {    // what the finalize kernel needs per reque
     float cp, inv_zp, cq, inv_zq;    // row references (log2 domain) and 1 / row sums
     float u;                         // resample uniform
     float scale;                     // log2(e) / T of this request
-    int32_t pad[2];
+    float tau;                       // truncation threshold of the target row (-inf: none)
+    int32_t pad;
 };
 
 struct VerifyParams {
@@ -77,6 +78,7 @@ struct VerifyParams {
     ResidTask* resid;                         // queue of rejected requests (decide -> residual pass)
     RequestRec* req;                          // per request: outcome of decide for the finalize kernel
     float* wblk;                              // per request: residual block sums
+    const float* tau;                         // per target row: top-k / top-p threshold (NULL: no truncation)
 };
 
 template <int kMode> struct ModeCfg {
@@ -290,17 +292,22 @@ __device__ __forceinline__ float2 block_argmax(const uint4 (&v)[kVec], int elem_
 // bit-identical values (the finalize kernel relies on that).
 struct ResidConst {
     uint64_t s2, ncp2, ncq2, izp2, nizq2;
-    float scale, cp, cq, inv_zp, inv_zq;
-    __device__ __forceinline__ void set(float scale_, float cp_, float inv_zp_, float cq_, float inv_zq_)
+    float scale, cp, cq, inv_zp, inv_zq, tau;
+    __device__ __forceinline__ void set(float scale_, float cp_, float inv_zp_, float cq_, float inv_zq_, float tau_)
     {
-        scale = scale_; cp = cp_; cq = cq_; inv_zp = inv_zp_; inv_zq = inv_zq_;
+        scale = scale_; cp = cp_; cq = cq_; inv_zp = inv_zp_; inv_zq = inv_zq_; tau = tau_;
         s2 = pack2(scale, scale); ncp2 = pack2(-cp, -cp); ncq2 = pack2(-cq, -cq);
         izp2 = pack2(inv_zp, inv_zp); nizq2 = pack2(-inv_zq, -inv_zq);
     }
 };
+// A target logit below the truncation threshold of its row counts as -inf (p = 0): top-k / top-p.
+__device__ __forceinline__ float cut_below(float x, float tau) { return x >= tau ? x : kNegInf; }
+
 __device__ __forceinline__ uint64_t resid_pair(uint64_t xt2, uint64_t xd2, const ResidConst& K)
 {
     float a0, a1, b0, b1;
+    unpack2(xt2, a0, a1);
+    xt2 = pack2(cut_below(a0, K.tau), cut_below(a1, K.tau));
     unpack2(fma2(xt2, K.s2, K.ncp2), a0, a1);
     unpack2(fma2(xd2, K.s2, K.ncq2), b0, b1);
     const uint64_t ep2 = pack2(ex2_approx(a0), ex2_approx(a1));
@@ -311,7 +318,7 @@ __device__ __forceinline__ uint64_t resid_pair(uint64_t xt2, uint64_t xd2, const
 }
 __device__ __forceinline__ float resid_elem(float xt, float xd, const ResidConst& K)
 {
-    const float ep = ex2_approx(__fmaf_rn(xt, K.scale, -K.cp));
+    const float ep = ex2_approx(__fmaf_rn(cut_below(xt, K.tau), K.scale, -K.cp));
     const float eq = ex2_approx(__fmaf_rn(xd, K.scale, -K.cq));
     return fmaxf(__fmaf_rn(ep, K.inv_zp, __fmul_rn(eq, -K.inv_zq)), 0.0f);
 }
@@ -369,7 +376,7 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
         load_block<kElem, M::kVec>(f1, nbytes, lane, vd);
         const ResidTask t = P.resid[s];
         ResidConst K;
-        K.set(t.scale, t.cp, t.inv_zp, t.cq, t.inv_zq);
+        K.set(t.scale, t.cp, t.inv_zp, t.cq, t.inv_zq, t.tau);
         const float w = block_resid<kElem, M::kVec>(v, vd, K);
         if (lane == 0) P.wblk[(long long)t.wslot * nblk + b] = w;
     }
@@ -863,7 +870,9 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
                     if (!row_usable(A.C, A.S) || !row_usable(D.C, D.S)) {
                         atomicOr(&s_bad, DSPARK_DEV_BAD_ROW);
                     } else {
-                        const double p = exp2((double)xt * scale_d - (double)A.C) / A.S;
+                        // truncated target (top-k / top-p): the row sum A.S already covers the kept set only
+                        const bool cut = P.tau && xt < P.tau[lo + j];
+                        const double p = cut ? 0.0 : exp2((double)xt * scale_d - (double)A.C) / A.S;
                         const double q = exp2((double)xd * scale_d - (double)D.C) / D.S;
                         if (P.out_p) P.out_p[lo + j] = (float)p;
                         if (P.out_q) P.out_q[lo + j] = (float)q;
@@ -891,7 +900,8 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     const int n = s_first;
     RequestRec rec;
     rec.kind = kTaskNone; rec.row_t = lo + n; rec.row_d = drow0 + n;
-    rec.cp = rec.cq = 0.f; rec.inv_zp = rec.inv_zq = 1.f; rec.u = 0.f; rec.scale = scale_f; rec.pad[0] = rec.pad[1] = 0;
+    rec.cp = rec.cq = 0.f; rec.inv_zp = rec.inv_zq = 1.f; rec.u = 0.f; rec.scale = scale_f; rec.pad = 0;
+    rec.tau = kNegInf;
     if (s_bad || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
         (n < len && !row_usable(s_fin_C[1], s_fin_S[1]))) {
         atomicOr(P.dev_status, s_bad ? s_bad : DSPARK_DEV_BAD_ROW);
@@ -902,6 +912,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
         philox_uniforms(P.seed, (uint32_t)r, (uint32_t)n, ua, ur);
         P.accepted_len[r] = n;
         rec.u = ur;
+        if (P.tau) rec.tau = P.tau[rec.row_t];
         rec.cp = s_fin_C[0]; rec.inv_zp = (float)(1.0 / s_fin_S[0]);
         if (n < len) {
             rec.cq = s_fin_C[1]; rec.inv_zq = (float)(1.0 / s_fin_S[1]);
@@ -910,7 +921,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             ResidTask q;
             q.request = r; q.row_t = rec.row_t; q.row_d = rec.row_d;
             q.cp = rec.cp; q.inv_zp = rec.inv_zp; q.cq = rec.cq; q.inv_zq = rec.inv_zq;
-            q.u = ur; q.scale = scale_f; q.wslot = r; q.pad = 0;
+            q.u = ur; q.scale = scale_f; q.wslot = r; q.tau = rec.tau;
             P.resid[slot] = q;
         } else {
             rec.kind = kTaskBonus;
@@ -984,7 +995,7 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
         const double thr_local = u * tot - before;
         if (resid) {
             ResidConst K;
-            K.set(rec.scale, rec.cp, rec.inv_zp, rec.cq, rec.inv_zq);
+            K.set(rec.scale, rec.cp, rec.inv_zp, rec.cq, rec.inv_zq, rec.tau);
             const int e0 = b * P.epb_r;
             const int cnt = (P.V - e0) < P.epb_r ? (P.V - e0) : P.epb_r;
             const unsigned char* drow = P.draft + rec.row_d * P.dstride_bytes;
@@ -992,12 +1003,12 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
                 trow, drow, e0, cnt, lane, thr_local, [&](float xt, float xd) { return resid_elem(xt, xd, K); }, S);
         } else {
             // element masses relative to the row reference, like the block masses
-            const float nc = -rec.cp, scale = rec.scale;
+            const float nc = -rec.cp, scale = rec.scale, tau = rec.tau;
             const int e0 = b * P.epb;
             const int cnt = (P.V - e0) < P.epb ? (P.V - e0) : P.epb;
             token = e0 + level2_block<kElem, kStatBlockBytes, false>(
                 trow, nullptr, e0, cnt, lane, thr_local,
-                [&](float xt, float) { return ex2_approx(__fmaf_rn(xt, scale, nc)); }, S);
+                [&](float xt, float) { return ex2_approx(__fmaf_rn(cut_below(xt, tau), scale, nc)); }, S);
         }
     }
     if (lane == 0) P.out_tokens[rec.row_t] = token;
@@ -1039,7 +1050,7 @@ __global__ void __launch_bounds__(kDecideThreads) queue_all_positions_kernel(Ver
             q.cp = A.C; q.cq = D.C;
             q.inv_zp = usable ? (float)(1.0 / A.S) : NAN;                       // NaN propagates to c*
             q.inv_zq = usable ? (float)(1.0 / D.S) : NAN;
-            q.u = 0.f; q.scale = P.scale; q.wslot = lo - r + j; q.pad = 0;
+            q.u = 0.f; q.scale = P.scale; q.wslot = lo - r + j; q.tau = kNegInf;
             P.resid[lo - r + j] = q;
         }
     }
@@ -1199,7 +1210,7 @@ static void launch_stream_dtype(const VerifyParams& P, bool bulk, long long max_
 }
 
 struct Workspace {
-    size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, total;
+    size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, tau, total;
 };
 static Workspace workspace_layout(int R, int n_rows, int V)
 {
@@ -1216,6 +1227,7 @@ static Workspace workspace_layout(int R, int n_rows, int V)
     w.wblk = o;     o += up((size_t)R * nblk_r * sizeof(float));
     w.scale_t = o;  o += up((size_t)n_rows * sizeof(float));
     w.scale_d = o;  o += up((size_t)n_rows * sizeof(float));
+    w.tau = o;      o += up((size_t)n_rows * sizeof(float));
     w.total = o;
     return w;
 }
@@ -1262,6 +1274,7 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.wblk = (float*)(ws + w.wblk);
     P.resid_cap = R;
     P.req_temp = nullptr;
+    P.tau = nullptr;
     P.row_scale_t = (float*)(ws + w.scale_t);
     P.row_scale_d = (float*)(ws + w.scale_d);
     return DSPARK_OK;
@@ -1319,9 +1332,12 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
                          float temperature, const float* req_temp, uint64_t seed,
                          int32_t* accepted_len, int32_t* out_tokens,
                          float* out_p_tok, float* out_q_tok, int32_t* dev_status,
-                         void* workspace, size_t workspace_bytes, void* stream)
+                         void* workspace, size_t workspace_bytes, void* stream,
+                         const int32_t* top_k = nullptr, const float* top_p = nullptr)
 {
     if (!draft_logits) return DSPARK_ERR_INVALID_ARG;
+    const bool truncate = top_k || top_p;
+    if (truncate && dtype != DSPARK_BF16) return DSPARK_ERR_SHAPE;   // the threshold search works on 16-bit keys
     if (!req_temp && (!(temperature > 0.0f) || !isfinite(temperature))) return DSPARK_ERR_INVALID_ARG;
     if (draft_row_stride < V) return DSPARK_ERR_SHAPE;
     VerifyParams P;
@@ -1347,6 +1363,17 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
         launch_stream_dtype<kModeStats>(P, bulk, (2ll * n_rows - R) * pieces(P.nblk), s);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
+    if (truncate) {
+        // top-k / top-p of the target distribution without touching the rows: one kernel finds the threshold of
+        // every target row and replaces the row's block sums by the sums over the kept set; from here on a
+        // target logit below the threshold counts as -inf
+        float* tau = (float*)((unsigned char*)workspace + workspace_layout(R, n_rows, V).tau);
+        KernelTimerScope timer(DSPARK_K_TRUNCATE, s);
+        rc = truncate_virtual_launch(P.target, P.tstride_bytes, V, row_offsets, R, n_rows, top_k, top_p, temperature,
+                                     req_temp, tau, P.stats_t, P.nblk, P.epb, s);
+        if (rc != DSPARK_OK) return rc;
+        P.tau = tau;
+    }
     {
         KernelTimerScope timer(DSPARK_K_DECIDE, s);
         launch_pdl(decide_kernel, dim3(R), dim3(kDecideThreads), 0, s, P);
@@ -1453,6 +1480,21 @@ int dspark_verify_per_request(const void* target_logits, const void* draft_logit
     return verify_launch(target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V, row_offsets,
                          draft_row_start, draft_tokens, R, n_rows, 1.0f, temperatures, seed, accepted_len,
                          out_tokens, out_p_tok, out_q_tok, dev_status, workspace, workspace_bytes, stream);
+}
+
+int dspark_verify_truncated(const void* target_logits, const void* draft_logits, int dtype,
+                            int64_t target_row_stride, int64_t draft_row_stride, int V,
+                            const int32_t* row_offsets, const int64_t* draft_row_start,
+                            const int32_t* draft_tokens, int R, int n_rows,
+                            float temperature, const float* temperatures, const int32_t* top_k, const float* top_p,
+                            uint64_t seed, int32_t* accepted_len, int32_t* out_tokens,
+                            float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                            void* workspace, size_t workspace_bytes, void* stream)
+{
+    return verify_launch(target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V, row_offsets,
+                         draft_row_start, draft_tokens, R, n_rows, temperatures ? 1.0f : temperature, temperatures, seed,
+                         accepted_len, out_tokens, out_p_tok, out_q_tok, dev_status, workspace, workspace_bytes, stream,
+                         top_k, top_p);
 }
 
 static size_t accept_rate_extra(int n_rows, int V, size_t* resid_off, size_t* wblk_off)
