@@ -127,9 +127,12 @@ __device__ __forceinline__ double block_sum_f64(double x, double* s_tmp)
     __syncthreads();
     if ((threadIdx.x & 31) == 0) s_tmp[threadIdx.x >> 5] = x;
     __syncthreads();
-    double t = 0.0;
-    for (int w = 0; w < kTruncThreads / 32; ++w) t += s_tmp[w];
-    return t;
+    if (threadIdx.x < 32) {
+        const double t = warp_sum_f64(threadIdx.x < kTruncThreads / 32 ? s_tmp[threadIdx.x] : 0.0);
+        if (threadIdx.x == 0) s_tmp[0] = t;
+    }
+    __syncthreads();
+    return s_tmp[0];
 }
 
 __device__ void truncate_row(const TruncParams& P, const int row, uint4* cache)
@@ -138,6 +141,8 @@ __device__ void truncate_row(const TruncParams& P, const int row, uint4* cache)
     __shared__ double s_tmp[kTruncThreads / 32];
     __shared__ double s_scan[kTruncThreads / 32];
     __shared__ unsigned long long s_scan_c[kTruncThreads / 32];
+    __shared__ unsigned long long s_tot_c;
+    __shared__ double s_tot_m;
     __shared__ int s_req, s_flag, s_hit;
     __shared__ unsigned int s_max;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -290,16 +295,26 @@ __device__ void truncate_row(const TruncParams& P, const int row, uint4* cache)
         __syncthreads();
         if (lane == 31) { s_scan_c[warp] = ic; s_scan[warp] = im; }
         __syncthreads();
-        unsigned long long bc = 0ull, tc = 0ull;
-        double bm = 0.0, tm = 0.0;
-        for (int x = 0; x < kTruncThreads / 32; ++x) {
-            if (x < warp) { bc += s_scan_c[x]; bm += s_scan[x]; }
-            tc += s_scan_c[x]; tm += s_scan[x];
+        if (warp == 0) {                                    // one warp turns the 32 warp totals into exclusive prefixes
+            const unsigned long long wc = lane < kTruncThreads / 32 ? s_scan_c[lane] : 0ull;
+            const double wm = lane < kTruncThreads / 32 ? s_scan[lane] : 0.0;
+            unsigned long long pc = wc;
+            double pm = wm;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long nc = __shfl_up_sync(0xffffffffu, pc, o);
+                const double nm = __shfl_up_sync(0xffffffffu, pm, o);
+                if (lane >= o) { pc += nc; pm += nm; }
+            }
+            if (lane < kTruncThreads / 32) { s_scan_c[lane] = pc - wc; s_scan[lane] = pm - wm; }
+            if (lane == 31) { s_tot_c = pc; s_tot_m = pm; }
         }
-        cnt_excl = bc + (ic - lc);
-        mass_excl = bm + (im - lm);
-        win_cnt = tc;
-        win_mass = tm;
+        __syncthreads();
+        cnt_excl = s_scan_c[warp] + (ic - lc);
+        mass_excl = s_scan[warp] + (im - lm);
+        win_cnt = s_tot_c;
+        win_mass = s_tot_m;
+        __syncthreads();                                    // s_scan is reused by through()
     };
     // first bin of the current window (scanned state) that satisfies pred(count_through, mass_through); the
     // smallest distance over the block, or -1
@@ -463,8 +478,8 @@ __device__ void truncate_row(const TruncParams& P, const int row, uint4* cache)
     }
 }
 
-// one CTA per row (a persistent CTA per SM walking the rows measured slower: the hardware overlaps the tail
-// of one row with the start of the next when they are separate CTAs)
+// One CTA per row.  (A persistent CTA per SM walking its rows, with or without a bulk prefetch of the next row
+// into L2, measured 25 % slower: rows take different times and the hardware's CTA scheduler balances them.)
 __global__ void __launch_bounds__(kTruncThreads) truncate_kernel(TruncParams P)
 {
     extern __shared__ uint4 cache[];                        // kCacheChunks vectors of the row
