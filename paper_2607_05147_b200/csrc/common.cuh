@@ -192,12 +192,25 @@ struct KernelTimerScope {
 };
 int launch_status();   // maps cudaGetLastError() to DSPARK_OK / DSPARK_ERR_CUDA
 
+// Order-preserving 16-bit key of a bf16 pattern (-0 and +0 share a key; NaN is the caller's business) and back.
+__device__ __forceinline__ uint32_t bf16_key(uint32_t b)
+{
+    if (b == 0x8000u) b = 0u;
+    return (b & 0x8000u) ? (0xFFFFu - b) : (b | 0x8000u);
+}
+__device__ __forceinline__ float bf16_key_value(uint32_t k)
+{
+    const uint32_t b = (k & 0x8000u) ? (k & 0x7FFFu) : (0xFFFFu - k);
+    return __uint_as_float(b << 16);
+}
+
 // Threshold search of the top-k / top-p truncation run inside the sampling verifier (truncate.cu): writes
 // the threshold of every target row to tau_rows (-inf: no cut) and replaces the block sums of the row's
 // statistics by the sums over the kept set; the rows themselves are not modified.
 int truncate_virtual_launch(const void* target, long long stride_bytes, int V, const int32_t* row_offsets, int R, int n_rows,
                             const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
-                            float* tau_rows, float2* stats_t, int nblk, int epb, cudaStream_t stream);
+                            float* tau_rows, float2* stats_t, int nblk, int epb, const int32_t* only_flagged,
+                            cudaStream_t stream);
 
 // Launch with programmatic stream serialization (the kernel must call pdl_wait() first).
 template <typename... KArgs, typename... Args>

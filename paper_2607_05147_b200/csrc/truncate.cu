@@ -39,19 +39,11 @@ struct TruncParams {
     // virtual mode (inside the verifier): the row is not modified; its statistics blocks receive the sums
     // restricted to the kept set instead
     float2* stats; int nblk, epb;
+    const int32_t* only_flagged;              // virtual mode: rows whose flag is 0 are somebody else's (NULL: all rows)
 };
 
-// order-preserving 16-bit key of a bf16 pattern (-0 and +0 share a key; NaN is handled by the caller)
-__device__ __forceinline__ uint32_t key_of(uint32_t b)
-{
-    if (b == 0x8000u) b = 0u;
-    return (b & 0x8000u) ? (0xFFFFu - b) : (b | 0x8000u);
-}
-__device__ __forceinline__ float value_of_key(uint32_t k)
-{
-    const uint32_t b = (k & 0x8000u) ? (k & 0x7FFFu) : (0xFFFFu - k);
-    return __uint_as_float(b << 16);
-}
+__device__ __forceinline__ uint32_t key_of(uint32_t b) { return bf16_key(b); }
+__device__ __forceinline__ float value_of_key(uint32_t k) { return bf16_key_value(k); }
 
 // eight consecutive elements starting at element 8c; elements past V read as -inf
 struct RowAccess {
@@ -159,6 +151,7 @@ __device__ void truncate_row(const TruncParams& P, const int row, uint4* cache)
     __syncthreads();
     const int r = s_req;
     if (r < 0) return;
+    if (P.only_flagged && !P.only_flagged[row]) return;
     const int V = P.V;
     const int k = P.top_k ? P.top_k[r] : 0;
     const float pf = P.top_p ? P.top_p[r] : 1.f;
@@ -487,6 +480,29 @@ __global__ void __launch_bounds__(kTruncThreads) truncate_kernel(TruncParams P)
     truncate_row(P, blockIdx.x, cache);
 }
 
+// The verifier's fallback: a few CTAs walk the rows and search only those that the streamed search flagged
+// (usually none, and then this costs a glance at the flags).
+__global__ void __launch_bounds__(kTruncThreads) truncate_flagged_kernel(TruncParams P)
+{
+    extern __shared__ uint4 cache[];
+    __shared__ int s_row;
+    pdl_wait();
+    int* counter = const_cast<int*>(P.only_flagged) + P.n_rows;     // zeroed with the flags
+    for (;;) {
+        // rows are handed out one at a time (they take very different times); unflagged ones are skipped here
+        if (threadIdx.x == 0) {
+            int row;
+            do { row = atomicAdd(counter, 1); } while (row < P.n_rows && !P.only_flagged[row]);
+            s_row = row;
+        }
+        __syncthreads();
+        const int row = s_row;
+        if (row >= P.n_rows) return;
+        truncate_row(P, row, cache);
+        __syncthreads();                                    // the shared state (and s_row) is reused by the next row
+    }
+}
+
 static int launch_truncate(const TruncParams& P, cudaStream_t stream)
 {
     static bool attr_set[64] = {};
@@ -494,25 +510,33 @@ static int launch_truncate(const TruncParams& P, cudaStream_t stream)
     cudaGetDevice(&dev);
     const size_t smem = (size_t)kCacheChunks * sizeof(uint4);
     if (!attr_set[dev & 63]) {
-        if (cudaFuncSetAttribute(truncate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(truncate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+            cudaFuncSetAttribute(truncate_flagged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return launch_status();
         attr_set[dev & 63] = true;
     }
-    launch_pdl(truncate_kernel, dim3(P.n_rows), dim3(kTruncThreads), smem, stream, P);
+    if (P.only_flagged) {
+        int sms = 0;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        launch_pdl(truncate_flagged_kernel, dim3(P.n_rows < sms ? P.n_rows : sms), dim3(kTruncThreads), smem, stream, P);
+    } else {
+        launch_pdl(truncate_kernel, dim3(P.n_rows), dim3(kTruncThreads), smem, stream, P);
+    }
     return launch_status();
 }
 
 // Used by the sampling verifier after its statistics pass (virtual truncation: rows stay as they are).
 int truncate_virtual_launch(const void* target, long long stride_bytes, int V, const int32_t* row_offsets, int R, int n_rows,
                             const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
-                            float* tau_rows, float2* stats_t, int nblk, int epb, cudaStream_t stream)
+                            float* tau_rows, float2* stats_t, int nblk, int epb, const int32_t* only_flagged,
+                            cudaStream_t stream)
 {
     TruncParams P;
     P.target = (unsigned char*)const_cast<void*>(target); P.stride_bytes = stride_bytes; P.V = V;
     P.row_offsets = row_offsets; P.R = R; P.n_rows = n_rows;
     P.top_k = top_k; P.top_p = top_p; P.temperatures = temperatures; P.temperature = temperature;
     P.out_tau = tau_rows; P.out_kept = nullptr; P.dev_status = nullptr;
-    P.stats = stats_t; P.nblk = nblk; P.epb = epb;
+    P.stats = stats_t; P.nblk = nblk; P.epb = epb; P.only_flagged = only_flagged;
     return launch_truncate(P, stream);
 }
 
@@ -536,7 +560,7 @@ int dspark_truncate_target(void* target_logits, int dtype, int64_t target_row_st
     P.row_offsets = row_offsets; P.R = R; P.n_rows = n_rows;
     P.top_k = top_k; P.top_p = top_p; P.temperatures = temperatures; P.temperature = temperature;
     P.out_tau = out_tau; P.out_kept = out_kept; P.dev_status = dev_status;
-    P.stats = nullptr; P.nblk = 0; P.epb = 0;
+    P.stats = nullptr; P.nblk = 0; P.epb = 0; P.only_flagged = nullptr;
     return launch_truncate(P, (cudaStream_t)stream);
 }
 

@@ -22,7 +22,8 @@
 
 namespace dspark {
 
-constexpr int kModeStats = 0, kModeGreedy = 1, kModeResid = 2;
+constexpr int kModeStats = 0, kModeGreedy = 1, kModeResid = 2, kModeHist = 3;
+constexpr int kHistBins = 1024;              // keys next to the row maximum that the streamed threshold search resolves
 constexpr int kTaskNone = 0, kTaskResid = 1, kTaskBonus = 2;
 constexpr int kDecideThreads = 256;
 constexpr float kNegInf = -INFINITY;
@@ -47,6 +48,17 @@ struct __align__(16) RequestRec {    // what the finalize kernel needs per reque
     float scale;                     // log2(e) / T of this request
     float tau;                       // truncation threshold of the target row (-inf: none)
     int32_t pad;
+};
+
+struct __align__(16) TruncRow {      // per target row, for the streamed threshold search of top-k / top-p
+    uint32_t kmax;                   // key of the row maximum
+    uint32_t size;                   // keys in the window next to the maximum (0: row not truncated)
+    uint32_t cut2;                   // lowest value of the window, bf16 pattern in both halves
+    float scale;                     // log2(e) / T
+    float C;                         // row reference (log2 domain) of the statistics
+    float Z;                         // row sum relative to C
+    int32_t k;                       // top-k (0: off)
+    float p;                         // top-p (>= 1: off)
 };
 
 struct VerifyParams {
@@ -79,6 +91,9 @@ struct VerifyParams {
     RequestRec* req;                          // per request: outcome of decide for the finalize kernel
     float* wblk;                              // per request: residual block sums
     const float* tau;                         // per target row: top-k / top-p threshold (NULL: no truncation)
+    TruncRow* trunc_rows;                     // workspace of the streamed threshold search
+    unsigned int* trunc_bins;                 // [n_rows][kHistBins] key counts
+    int32_t* trunc_flag;                      // [n_rows] 1: the window did not resolve the row (per-row search)
 };
 
 template <int kMode> struct ModeCfg {
@@ -119,7 +134,7 @@ template <int kMode>
 __device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
 {
     if (kMode == kModeStats) return n_rows + (n_rows > P.R ? n_rows - P.R : 0);
-    if (kMode == kModeGreedy) return n_rows;
+    if (kMode == kModeGreedy || kMode == kModeHist) return n_rows;
     const int nq = __ldcg(&P.counters[0]);
     return nq > P.resid_cap ? P.resid_cap : (nq < 0 ? 0 : nq);
 }
@@ -371,6 +386,25 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
     } else if (kMode == kModeGreedy) {
         const float2 st = block_argmax<kElem, M::kVec>(v, b * P.epb, lane);
         if (lane == 0) P.stats_t[(long long)s * nblk + b] = st;
+    } else if (kMode == kModeHist) {
+        // bf16 rows only.  Count the keys within the window next to the row maximum: a packed compare rejects
+        // almost every pair, the few tokens of the tail take one atomic each.
+        const TruncRow tr = P.trunc_rows[s];
+        if (tr.size == 0u) return;
+        const __nv_bfloat162 cut2 = *reinterpret_cast<const __nv_bfloat162*>(&tr.cut2);
+        unsigned int* bins = P.trunc_bins + (long long)s * kHistBins;
+#pragma unroll
+        for (int k = 0; k < M::kVec; ++k) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t w = word_of(v[k], i);
+                if (__hge2_mask(*reinterpret_cast<const __nv_bfloat162*>(&w), cut2)) {
+                    const uint32_t d0 = tr.kmax - bf16_key(w & 0xFFFFu), d1 = tr.kmax - bf16_key(w >> 16);
+                    if (d0 < tr.size) atomicAdd(&bins[d0], 1u);
+                    if (d1 < tr.size) atomicAdd(&bins[d1], 1u);
+                }
+            }
+        }
     } else {
         uint4 vd[M::kVec];
         load_block<kElem, M::kVec>(f1, nbytes, lane, vd);
@@ -435,7 +469,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
 
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
-    if (kMode != kModeResid && blockIdx.x == 0 && tid == 0) {
+    if (kMode != kModeResid && kMode != kModeHist && blockIdx.x == 0 && tid == 0) {
         P.counters[0] = 0;                       // residual queue, filled by the decide kernel
         if (bad_rows) atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS);
     }
@@ -506,7 +540,7 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
     pdl_wait();
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
-    if (kMode != kModeResid && blockIdx.x == 0 && tid == 0) {
+    if (kMode != kModeResid && kMode != kModeHist && blockIdx.x == 0 && tid == 0) {
         P.counters[0] = 0;
         if (bad_rows) atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS);
     }
@@ -764,6 +798,248 @@ __device__ __forceinline__ int level2_block(const unsigned char* trow, const uns
     }
     if (found < 0) found = n_src - 1;                     // only by rounding between the two sums
     return src * kPer + found;
+}
+
+// ---------------------------------------------------------------------------------------
+// top-k / top-p truncation of the target distribution inside the verifier (bf16 rows).
+// The kept set of a row is {v : x_v >= tau}; tau is found exactly on the 16-bit keys:
+//   trunc_prep    per target row: row maximum m (recovered exactly from the statistics: the reference
+//                 c = m * scale determines the bf16 value m), the window of keys between m and m - 8 T (at
+//                 most kHistBins keys), zeroed counters;
+//   stream<Hist>  one more streamed pass over the target rows counts the keys inside the window;
+//   trunc_scan    per row: masses count * 2^(value * scale - C), prefix sums, the top-k and top-p
+//                 thresholds; a row whose threshold lies beyond the window is flagged for the per-row
+//                 search of truncate.cu (flat rows: rare);
+//   trunc_sums    per (row, block): the block sum of the statistics restricted to x >= tau (only blocks
+//                 whose maximum reaches tau are read again).
+// ---------------------------------------------------------------------------------------
+struct TruncArgs {
+    const int32_t* top_k; const float* top_p; const float* temperatures; float temperature;
+    float* tau;                       // per target row
+};
+
+__global__ void __launch_bounds__(256) trunc_prep_kernel(VerifyParams P, TruncArgs T)
+{
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    bool bad_rows;
+    const int n_rows = device_rows(P, &bad_rows);
+    if (row >= n_rows) return;
+    int lo = 0, hi = P.R;                                   // largest r with row_offsets[r] <= row
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (P.row_offsets[mid] <= row) lo = mid; else hi = mid;
+    }
+    const int r = lo;
+    const int k = T.top_k ? T.top_k[r] : 0;
+    const float pf = T.top_p ? T.top_p[r] : 1.f;
+    const float temp = T.temperatures ? T.temperatures[r] : T.temperature;
+    RowAcc A, D;
+    combine_rows(P.stats_t + (long long)row * P.nblk, nullptr, P.nblk, lane, A, D);
+    TruncRow tr;
+    tr.kmax = 0u; tr.size = 0u; tr.cut2 = 0u; tr.scale = 0.f; tr.C = A.C; tr.Z = (float)A.S; tr.k = 0; tr.p = 1.f;
+    const bool use_k = k > 0 && k < P.V, use_p = pf < 1.f;
+    if ((use_k || use_p) && temp > 0.f && temp < INFINITY && row_usable(A.C, A.S)) {
+        const float scale = (float)(1.4426950408889634 / (double)temp);
+        const __nv_bfloat16 mb = __float2bfloat16_rn(A.C / scale);      // the bf16 maximum behind c = m * scale
+        const float m = __bfloat162float(mb);
+        const uint32_t kmax = bf16_key((uint32_t)__bfloat16_as_ushort(mb));
+        float lo_val = m - 8.f * temp;
+        if (use_k && k <= P.nblk) {
+            // every block maximum is an element of the row, so the k-th largest logit is at least the k-th
+            // largest block maximum: the window reaches down to it (rank by counting, 64-128 blocks)
+            const float2* st = P.stats_t + (long long)row * P.nblk;
+            float kth = kNegInf;
+            if (P.nblk <= 128) {                             // block references in registers, compared through shuffles
+                float c[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) c[q] = (q * 32 + lane < P.nblk) ? __ldcg(&st[q * 32 + lane]).x : kNegInf;
+                int rank[4] = {0, 0, 0, 0};                  // blocks that come before mine in descending order
+#pragma unroll
+                for (int q2 = 0; q2 < 4; ++q2) {
+                    if (q2 * 32 >= P.nblk) break;
+                    for (int l2 = 0; l2 < 32; ++l2) {
+                        const float cj = __shfl_sync(0xffffffffu, c[q2], l2);
+                        const int j = q2 * 32 + l2;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) rank[q] += (cj > c[q]) || (cj == c[q] && j < q * 32 + lane);
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (q * 32 + lane < P.nblk && rank[q] == k - 1) kth = c[q];
+            } else {
+                for (int b0 = lane; b0 < P.nblk; b0 += 32) {
+                    const float cb = __ldcg(&st[b0]).x;
+                    int rank = 0;
+                    for (int j = 0; j < P.nblk; ++j) {
+                        const float cj = __ldcg(&st[j]).x;
+                        rank += (cj > cb) || (cj == cb && j < b0);
+                    }
+                    if (rank == k - 1) kth = cb;
+                }
+            }
+            kth = warp_max_f32(kth);
+            if (kth > kNegInf) lo_val = fminf(lo_val, __bfloat162float(__float2bfloat16_rn(kth / scale)));
+        }
+        const uint32_t klo = bf16_key((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rd(lo_val)));
+        uint32_t size = kHistBins;
+        if (klo <= kmax && kmax - klo + 1u < (uint32_t)kHistBins) size = kmax - klo + 1u;
+        if (size > kmax + 1u) size = kmax + 1u;                          // keys 0 .. kmax exist
+        const uint32_t cb = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(bf16_key_value(kmax - (size - 1u))));
+        tr.kmax = kmax; tr.size = size; tr.cut2 = cb | (cb << 16); tr.scale = scale;
+        tr.k = use_k ? k : 0; tr.p = use_p ? pf : 1.f;
+        unsigned int* bins = P.trunc_bins + (long long)row * kHistBins;
+        for (uint32_t i = lane; i < size; i += 32) bins[i] = 0u;
+    }
+    if (lane == 0) { P.trunc_rows[row] = tr; T.tau[row] = kNegInf; P.trunc_flag[row] = 0; }
+    if (row == 0 && lane == 0) P.trunc_flag[P.n_rows_cap] = 0;          // work counter of the per-row fallback
+}
+
+constexpr int kScanThreads = 256;
+__global__ void __launch_bounds__(kScanThreads) trunc_scan_kernel(VerifyParams P, TruncArgs T)
+{
+    constexpr int kPer = kHistBins / kScanThreads;
+    __shared__ unsigned long long s_c[kScanThreads / 32];
+    __shared__ double s_m[kScanThreads / 32];
+    __shared__ int s_hit_k, s_hit_p;
+    __shared__ double s_zk;
+    pdl_wait();
+    const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    bool bad_rows;
+    if (row >= device_rows(P, &bad_rows)) return;
+    const TruncRow tr = P.trunc_rows[row];
+    if (tr.size == 0u) return;
+    if (tid == 0) { s_hit_k = 0x7fffffff; s_hit_p = 0x7fffffff; }
+    const unsigned int* bins = P.trunc_bins + (long long)row * kHistBins;
+    unsigned int cnt[kPer];
+    double mass[kPer];
+    unsigned long long lc = 0ull;
+    double lm = 0.0;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+        const uint32_t d = (uint32_t)(tid * kPer + j);
+        cnt[j] = d < tr.size ? __ldcg(&bins[d]) : 0u;
+        // mass of a key relative to the row reference C, as the statistics count it
+        mass[j] = cnt[j] ? (double)cnt[j] * (double)exp2f(__fmaf_rn(bf16_key_value(tr.kmax - d), tr.scale, -tr.C)) : 0.0;
+        lc += cnt[j];
+        lm += mass[j];
+    }
+    unsigned long long ic = lc;
+    double im = lm;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long nc = __shfl_up_sync(0xffffffffu, ic, o);
+        const double nm = __shfl_up_sync(0xffffffffu, im, o);
+        if (lane >= o) { ic += nc; im += nm; }
+    }
+    if (lane == 31) { s_c[warp] = ic; s_m[warp] = im; }
+    __syncthreads();
+    unsigned long long bc = 0ull;
+    double bm = 0.0;
+    for (int x = 0; x < warp; ++x) { bc += s_c[x]; bm += s_m[x]; }
+    const unsigned long long c_excl = bc + (ic - lc);
+    const double m_excl = bm + (im - lm);
+    // top-k: the first key at which the running count reaches k
+    if (tr.k > 0) {
+        unsigned long long c = c_excl;
+        int mine = 0x7fffffff;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            c += cnt[j];
+            if (mine == 0x7fffffff && cnt[j] && c >= (unsigned long long)tr.k) mine = tid * kPer + j;
+        }
+        mine = __reduce_min_sync(0xffffffffu, mine);
+        if (lane == 0 && mine != 0x7fffffff) atomicMin(&s_hit_k, mine);
+    }
+    __syncthreads();
+    const int dk = s_hit_k;
+    if (tr.k > 0 && dk == 0x7fffffff) {                     // the k-th largest key lies beyond the window
+        if (tid == 0) P.trunc_flag[row] = 1;
+        return;
+    }
+    if (tr.k > 0 && dk / kPer == tid) {                     // mass of the top-k set
+        double q = m_excl;
+        for (int j = 0; j <= dk % kPer; ++j) q += mass[j];
+        s_zk = q;
+    }
+    __syncthreads();
+    int dist = tr.k > 0 ? dk : 0x7fffffff;
+    if (tr.p < 1.f) {
+        if (!(tr.p > 0.f)) {
+            dist = 0;                                       // only the maximum
+        } else {
+            const double thr = (double)tr.p * (tr.k > 0 ? s_zk : (double)tr.Z);
+            double q = m_excl;
+            int mine = 0x7fffffff;
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                q += mass[j];
+                if (mine == 0x7fffffff && cnt[j] && q >= thr) mine = tid * kPer + j;
+            }
+            mine = __reduce_min_sync(0xffffffffu, mine);
+            if (lane == 0 && mine != 0x7fffffff) atomicMin(&s_hit_p, mine);
+            __syncthreads();
+            const int dp = s_hit_p;
+            if (dp == 0x7fffffff && tr.k == 0) {            // the nucleus reaches beyond the window
+                if (tid == 0) P.trunc_flag[row] = 1;
+                return;
+            }
+            if (dp < dist) dist = dp;
+        }
+    }
+    if (tid == 0 && dist != 0x7fffffff) T.tau[row] = bf16_key_value(tr.kmax - (uint32_t)dist);
+}
+
+// One warp per (target row, statistics block): s = sum over x >= tau of 2^(x * scale - c).
+__global__ void __launch_bounds__(256) trunc_sums_kernel(VerifyParams P, TruncArgs T)
+{
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x;
+    const int b = blockIdx.y * 8 + (threadIdx.x >> 5);
+    bool bad_rows;
+    if (row >= device_rows(P, &bad_rows) || b >= P.nblk) return;
+    const float tau = T.tau[row];
+    if (!(tau > kNegInf) || P.trunc_flag[row]) return;       // untouched row, or left to the per-row search
+    const TruncRow tr = P.trunc_rows[row];
+    float2* st = P.stats_t + (long long)row * P.nblk + b;
+    const float2 e = *st;
+    float sum = 0.f;
+    if (e.x > kNegInf && e.x >= __fmul_rn(tau, tr.scale)) {
+        const unsigned char* base = P.target + (long long)row * P.tstride_bytes;
+        const int e0 = b * P.epb;
+        const int cnt = (P.V - e0) < P.epb ? (P.V - e0) : P.epb;
+        const uint64_t sc2 = pack2(tr.scale, tr.scale), nc2 = pack2(-e.x, -e.x);
+        uint64_t acc = pack2(0.f, 0.f);
+        const bool vec = (((uintptr_t)(base + (long long)e0 * 2)) & 15u) == 0;
+        for (int i = lane * 8; i < cnt; i += 256) {
+            uint32_t w[4];
+            if (vec && i + 8 <= cnt) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(base + (long long)(e0 + i) * 2));
+                w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+            } else {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int a = i + 2 * q;
+                    const uint32_t l = a < cnt ? reinterpret_cast<const unsigned short*>(base)[e0 + a] : 0xFF80u;
+                    const uint32_t h = a + 1 < cnt ? reinterpret_cast<const unsigned short*>(base)[e0 + a + 1] : 0xFF80u;
+                    w[q] = l | (h << 16);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float t0, t1;
+                unpack2(fma2(pack2(cut_below(bf16lo(w[q]), tau), cut_below(bf16hi(w[q]), tau)), sc2, nc2), t0, t1);
+                acc = add2(acc, pack2(ex2_approx(t0), ex2_approx(t1)));
+            }
+        }
+        float a0, a1;
+        unpack2(acc, a0, a1);
+        sum = warp_sum_f32(a0 + a1);
+    }
+    if (lane == 0) st->y = sum;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -1180,7 +1456,8 @@ static bool ensure_attrs()
     if (d.attrs_set) return true;
     bool ok = set_smem_attr<2, kModeStats>() == cudaSuccess && set_smem_attr<4, kModeStats>() == cudaSuccess &&
               set_smem_attr<2, kModeGreedy>() == cudaSuccess && set_smem_attr<4, kModeGreedy>() == cudaSuccess &&
-              set_smem_attr<2, kModeResid>() == cudaSuccess && set_smem_attr<4, kModeResid>() == cudaSuccess;
+              set_smem_attr<2, kModeResid>() == cudaSuccess && set_smem_attr<4, kModeResid>() == cudaSuccess &&
+              set_smem_attr<2, kModeHist>() == cudaSuccess;
     d.attrs_set = ok;
     return ok;
 }
@@ -1210,7 +1487,7 @@ static void launch_stream_dtype(const VerifyParams& P, bool bulk, long long max_
 }
 
 struct Workspace {
-    size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, tau, total;
+    size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, tau, trunc_rows, trunc_bins, trunc_flag, total;
 };
 static Workspace workspace_layout(int R, int n_rows, int V)
 {
@@ -1228,6 +1505,9 @@ static Workspace workspace_layout(int R, int n_rows, int V)
     w.scale_t = o;  o += up((size_t)n_rows * sizeof(float));
     w.scale_d = o;  o += up((size_t)n_rows * sizeof(float));
     w.tau = o;      o += up((size_t)n_rows * sizeof(float));
+    w.trunc_rows = o; o += up((size_t)n_rows * sizeof(TruncRow));
+    w.trunc_bins = o; o += up((size_t)n_rows * kHistBins * sizeof(unsigned int));
+    w.trunc_flag = o; o += up((size_t)(n_rows + 1) * sizeof(int32_t));   // + the fallback's row counter
     w.total = o;
     return w;
 }
@@ -1275,6 +1555,9 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.resid_cap = R;
     P.req_temp = nullptr;
     P.tau = nullptr;
+    P.trunc_rows = (TruncRow*)(ws + w.trunc_rows);
+    P.trunc_bins = (unsigned int*)(ws + w.trunc_bins);
+    P.trunc_flag = (int32_t*)(ws + w.trunc_flag);
     P.row_scale_t = (float*)(ws + w.scale_t);
     P.row_scale_d = (float*)(ws + w.scale_d);
     return DSPARK_OK;
@@ -1369,8 +1652,15 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
         // target logit below the threshold counts as -inf
         float* tau = (float*)((unsigned char*)workspace + workspace_layout(R, n_rows, V).tau);
         KernelTimerScope timer(DSPARK_K_TRUNCATE, s);
+        TruncArgs T;
+        T.top_k = top_k; T.top_p = top_p; T.temperatures = req_temp; T.temperature = temperature; T.tau = tau;
+        launch_pdl(trunc_prep_kernel, dim3((n_rows + 7) / 8), dim3(256), 0, s, P, T);
+        launch_stream<2, kModeHist>(P, bulk, (long long)n_rows * pieces(P.nblk), s);
+        launch_pdl(trunc_scan_kernel, dim3(n_rows), dim3(kScanThreads), 0, s, P, T);
+        launch_pdl(trunc_sums_kernel, dim3(n_rows, (P.nblk + 7) / 8), dim3(256), 0, s, P, T);
+        // rows whose threshold lies beyond the window (flat rows): the per-row search
         rc = truncate_virtual_launch(P.target, P.tstride_bytes, V, row_offsets, R, n_rows, top_k, top_p, temperature,
-                                     req_temp, tau, P.stats_t, P.nblk, P.epb, s);
+                                     req_temp, tau, P.stats_t, P.nblk, P.epb, P.trunc_flag, s);
         if (rc != DSPARK_OK) return rc;
         P.tau = tau;
     }
