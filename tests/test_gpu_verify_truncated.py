@@ -131,3 +131,26 @@ def test_fp32_is_refused():
     b = W.sampling_batch(lengths, 512, 3, "cuda", dtype=torch.float32)
     with pytest.raises(B.DsparkError):
         _gpu_truncated(b, np.array([3, 3], np.int32), None, None)
+
+
+def test_flat_rows_take_the_per_row_search():
+    # rows without a peak: the top-k threshold and the nucleus lie far below the maximum, beyond the window of
+    # the streamed search, so every row goes through the per-row fallback; results must not change
+    R, V = 12, 20_000
+    g0 = torch.Generator().manual_seed(8)
+    lengths = torch.randint(0, 4, (R,), generator=g0)
+    off = torch.cat([torch.zeros(1, dtype=torch.int64), torch.cumsum(lengths + 1, 0)]).to(torch.int32)
+    n_rows = int(off[-1])
+    target = (torch.rand(n_rows, V, generator=g0) * 2 - 1).to(torch.bfloat16)            # flat, both signs
+    target[1] = (torch.randn(V, generator=g0) * 30).to(torch.bfloat16)                   # very wide
+    draft = (target[: n_rows - R].float() + 0.3 * torch.randn(n_rows - R, V, generator=g0)).to(torch.bfloat16)
+    toks = torch.randint(0, V, (n_rows,), generator=g0, dtype=torch.int32)
+    b = W.VerifyBatch(target.cuda(), draft.cuda(), off.cuda(), toks.cuda(), None, 1.0, 11)
+    ks = np.array([5000, 0, 19000, 200, 0, 70, 3, 0, 12000, 1, 0, 400], dtype=np.int32)
+    # top-k is integer work and exact; on a flat row every top-p decision sits within 1e-5 of a value boundary
+    # (each value carries 1/V of the mass), so only the decisive cases are given a top-p
+    ps = np.array([1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 0.0, 1.0], dtype=np.float32)
+    g = _gpu_truncated(b, ks, ps, None)
+    o, margin = _oracle_pipeline(b, ks, ps, None)
+    mism = H.compare_sampling(g, o, b.row_offsets.cpu().numpy())
+    print(f"[verify_truncated] flat rows: accepted {g['acc'].tolist()}, {mism} boundary mismatches")
