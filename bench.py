@@ -160,7 +160,17 @@ class Step:
             self.verify_done = [torch.cuda.Event(), torch.cuda.Event()]
             self.tick = 0
             self.primed = False
-        self.launches_per_step = (2 if self.sched is not None else 0) + (2 if wl["greedy"] else 4)
+        # kernels of the library per step: scheduler (prep, rank + final stage; a selection kernel when the
+        # candidates are many and the budget admits fewer than half), verifier (stream, decide[, residual
+        # stream, finalize]), row scales for per-request temperatures, five more for the truncation
+        n_sched = 0
+        if self.sched is not None:
+            gamma = self.sched.conf.shape[1]
+            gpad = 1 << max(0, (gamma - 1).bit_length()) if gamma <= 32 else (gamma + 31) // 32 * 32
+            entries = self.R * gpad
+            n_sched = 2 + (1 if entries >= 8192 and 2 * (self.sched.budget_tokens - self.R) <= entries else 0)
+        self.launches_per_step = n_sched + (2 if wl["greedy"] else 4) + (1 if PER_REQUEST_T and not wl["greedy"] else 0) \
+            + (5 if TRUNCATE is not None and not wl["greedy"] else 0)
 
     def run(self, batch, conf=None):
         """One step; with --cuda-graph the step of every resident batch is captured once and replayed."""
