@@ -399,9 +399,13 @@ def bench_markov(args, device, rank, world, dist, barrier):
     st = torch.zeros(1, dtype=torch.int32, device=device)
     ws = B.workspace(B.dspark_markov_workspace_bytes(R, V))
 
+    # sequential drafting: the tokens drawn at one position are the previous tokens of the next one
+    tok2 = [m.x_prev.clone(), toks]
+
     def step(i):
-        B.dspark_markov_draft_step(Us[i % n_sets], m.W1, packed, m.x_prev, 1.0, 77 + i, H=m.H, w_conf=m.w_conf,
-                                   out_logits=outs[i % n_sets], out_tokens=toks, out_conf=conf, dev_status=st, workspace=ws)
+        B.dspark_markov_draft_step(Us[i % n_sets], m.W1, packed, tok2[i & 1], 1.0, 77 + i, H=m.H, w_conf=m.w_conf,
+                                   out_logits=outs[i % n_sets], out_tokens=tok2[(i + 1) & 1], out_conf=conf, dev_status=st,
+                                   workspace=ws)
 
     for i in range(args.warmup):
         step(i)

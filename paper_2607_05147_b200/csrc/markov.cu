@@ -643,6 +643,14 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
 // that tile.  A row with NaN, +inf or no finite element sets DSPARK_DEV_BAD_ROW and yields -1.
 // Greedy: the lowest index of the row maximum; a row with nothing above -inf sets
 // DSPARK_DEV_ALL_NEG_INF and yields 0.
+// The token just drawn is the previous token of the next draft position: its embedding row (512 B of W1) is
+// asked into L2 now, so that the next contraction's gather does not wait for DRAM.  Called by one warp.
+__device__ __forceinline__ void prefetch_embedding(const MarkovParams& P, int token, int lane)
+{
+    if (lane < 4 && token >= 0 && token < P.V)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(P.W1 + (size_t)token * kRank * 2 + lane * 128));
+}
+
 constexpr int kDrawThreads = 256;
 constexpr int kStatCols = kTileMN;               // columns per statistics entry
 constexpr int kDrawPer = 16;                     // entries per thread at most: V <= 256 * 16 * 128
@@ -696,6 +704,7 @@ __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams 
             if (bi == 0x7fffffff) { atomicOr(P.dev_status, DSPARK_DEV_ALL_NEG_INF); bi = 0; }
             out_tokens[r] = bi;
         }
+        if (tid < 32) prefetch_embedding(P, __shfl_sync(0xffffffffu, bi, 0), tid);
         return;
     }
     // row maximum, unusable rows
@@ -799,6 +808,7 @@ __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams 
     if (hit) result = __shfl_sync(0xffffffffu, tok, __ffs(hit) - 1);
     else result = pos ? __shfl_sync(0xffffffffu, lastp, 31 - __clz(pos)) : box * kStatCols;
     if (lane == 0) out_tokens[r] = result;
+    prefetch_embedding(P, result, lane);
 }
 
 struct MarkovWs { size_t stats, trace, total; };
