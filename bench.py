@@ -467,7 +467,11 @@ def bench_markov(args, device, rank, world, dist, barrier):
         "config": {"workload": f"Markov-head draft position, R={R}, V={V}, rank 256, T=1, confidence head d=1024",
                    "l2": f"{n_sets} base-logit / output buffer pairs rotated ({n_sets * 4 * R * V / 1e6:.0f} MB)"},
         "roofline": {"bound": "hbm", "kernel": "markov_gemm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_launch": gemm_bytes,
+                     "frac": achieved / peak,
+                     # dram__bytes_read + write of one launch from the ncu capture summarised under profiles/ (R = 256;
+                     # part of the written tile is still in L2 when the kernel ends)
+                     "traffic": 132_567_040 + 32_054_784 if R == 256 else None,
+                     "algorithmic_bytes_per_launch": gemm_bytes,
                      "us_per_launch": gemm_call_ms * 1e3,
                      "timing": "logits-only calls back to back (statistics off), CUDA events around the whole loop",
                      "us_per_launch_inside_step_with_events": gemm_ms * 1e3,
