@@ -174,3 +174,32 @@ def test_draw_frequencies_follow_the_softmax(T):
         chi += (rest_c - rest_e) ** 2 / rest_e
     dof = int(big.sum())
     assert chi < dof + 6 * (2 * dof) ** 0.5, (chi, dof)
+
+
+@pytest.mark.parametrize("R", [256, 1024])
+def test_bench_configuration_on_sampled_rows(R):
+    # the launch configuration of `bench.py --markov-draft` (V = 129 280); the oracle recomputes a sample of rows
+    # that spans the row tiles (first / last row of a tile, a few in between)
+    V = W.V_FULL
+    m = W.markov_input(R, V, 4242, "cuda")
+    seed = 77
+    out, conf, toks, st = _run(m, temperature=1.0, seed=seed)
+    assert st == 0
+    rows = sorted({0, 127, 128, R // 2 + 3, R - 129, R - 128, R - 1} | {int(x) for x in np.random.default_rng(R).integers(0, R, 5)})
+    idx = torch.tensor(rows, device="cuda")
+    sub = W.MarkovInput(m.U[idx].contiguous(), m.W1, m.W2, m.x_prev[idx].contiguous(), m.H[idx].contiguous(), m.w_conf)
+    share = _check_logits(sub, out[idx].contiguous())
+    want_c = oracle.confidence(W.bf16_bits(sub.H), W.bf16_bits(m.W1), m.w_conf.cpu().numpy(), sub.x_prev.cpu().numpy())
+    assert np.abs(conf[idx].cpu().numpy() - want_c).max() <= 1e-6
+    # the draw of request r uses the uniform of (seed, r, 0): the oracle verifies one request at a time in place r
+    bits = W.bf16_bits(out[idx].contiguous())
+    got = toks[idx].cpu().numpy()
+    for i, r in enumerate(rows):
+        u = oracle.uniforms(seed, r, 0)[1]
+        p, _, _, bad = oracle.softmax_row(bits, i, 1.0)
+        assert not bad
+        cum = np.cumsum(p)
+        want = int(np.searchsorted(cum, u, side="right"))
+        if got[i] != want:
+            assert min(abs(cum[want] - u), abs(u - (cum[want - 1] if want else 0.0))) < 1e-6, (r, got[i], want)
+    print(f"[markov] R={R} V={V}: {len(rows)} sampled rows, one-ulp share {share:.2e}")
