@@ -176,10 +176,11 @@ def test_draw_frequencies_follow_the_softmax(T):
     assert chi < dof + 6 * (2 * dof) ** 0.5, (chi, dof)
 
 
-@pytest.mark.parametrize("R", [256, 1024])
+@pytest.mark.parametrize("R", [256, 1024, 17000])
 def test_bench_configuration_on_sampled_rows(R):
     # the launch configuration of `bench.py --markov-draft` (V = 129 280); the oracle recomputes a sample of rows
-    # that spans the row tiles (first / last row of a tile, a few in between)
+    # that spans the row tiles (first / last row of a tile, a few in between).  R = 17 000: 17 launches, the last
+    # one ragged, and the logits of the last rows lie beyond 4 GiB from the base pointer (64-bit addressing)
     V = W.V_FULL
     m = W.markov_input(R, V, 4242, "cuda")
     seed = 77
