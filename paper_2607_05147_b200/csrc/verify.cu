@@ -6,7 +6,8 @@
 //            4 KB blocks; one warp reduces one block to (reference, sum of 2^(x*scale-ref))
 //            [sampling] or (max, lowest argmax) [greedy].  Persistent CTAs; a producer warp
 //            feeds a ring of 32 KB shared-memory stages with 1-D bulk async copies
-//            (cp.async.bulk + mbarrier), eight consumer warps drain it.
+//            (cp.async.bulk + mbarrier), eight consumer warps drain it.  The 32 KB units are
+//            handed out through a grid-wide counter, so all CTAs finish together.
 //   decide   one CTA per request: combines block statistics into row statistics, gathers
 //            p(x), q(x), runs the accept tests (Philox), finds the first rejection, writes the
 //            accepted prefix, and queues a rejected position for the residual pass.
@@ -15,6 +16,8 @@
 //   finalize one warp per request: inverse CDF over block values (residual sums, or the saved
 //            statistics of the bonus row), then inside the one block that holds the crossing.
 #include <cuda_bf16.h>
+#include <atomic>
+#include <chrono>
 #include <cstdio>
 #include <math.h>
 
@@ -89,6 +92,7 @@ struct VerifyParams {
     float2* stats_d;
     ResidTask* resid;                         // queue of rejected requests (decide -> residual pass)
     RequestRec* req;                          // per request: outcome of decide for the finalize kernel
+    unsigned long long launch_tag;            // unique per call: see unit_counter()
     float* wblk;                              // per request: residual block sums
     const float* tau;                         // per target row: top-k / top-p threshold (NULL: no truncation)
     TruncRow* trunc_rows;                     // workspace of the streamed threshold search
@@ -138,6 +142,34 @@ __device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
     const int nq = __ldcg(&P.counters[0]);
     return nq > P.resid_cap ? P.resid_cap : (nq < 0 ? 0 : nq);
 }
+
+// Unit counters of the bulk-copy passes (64-bit cells behind the two int counters).  The residual and
+// histogram passes find theirs zeroed by the statistics pass of the same call.  The statistics / greedy
+// pass has no kernel of the call before it (a reset kernel would add a kernel boundary, 1.3 us, to every
+// call), so its CTA 0 zeroes the counter and then publishes the call's launch tag -- a 64-bit value no
+// earlier call used -- in the cell next to it; a CTA draws from the counter only after it has seen the tag
+// (its first two units need no draw, so in practice nobody waits).  CTAs are dispatched in index order,
+// CTA 0 is running before any other can ask; the wait is bounded all the same.  The kernel that follows
+// the pass in every call clears the tag, so a replayed CUDA graph (same tag each time) starts clean.
+template <int kMode>
+__device__ __forceinline__ unsigned long long* unit_counter(const VerifyParams& P)
+{
+    return reinterpret_cast<unsigned long long*>(P.counters) + (kMode == kModeResid ? 2 : (kMode == kModeHist ? 3 : 1));
+}
+__device__ __forceinline__ unsigned long long* unit_tag(const VerifyParams& P)
+{
+    return reinterpret_cast<unsigned long long*>(P.counters) + 4;
+}
+__device__ __forceinline__ bool wait_for_tag(const unsigned long long* cell, unsigned long long tag)
+{
+    for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+        unsigned long long v;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(cell) : "memory");
+        if (v == tag) return true;
+    }
+    return false;
+}
+struct UnitSlot { int s, piece; float scale; };   // what the producer tells the consumers about a stage
 
 // Walks the units (stream s, piece) owned by this CTA: unit index = s * ppr + piece, advancing by
 // gridDim.x units per step without divisions.
@@ -456,6 +488,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     extern __shared__ __align__(128) unsigned char stage_mem[];
     __shared__ __align__(8) uint64_t full_bar[kStages];
     __shared__ __align__(8) uint64_t empty_bar[kStages];
+    __shared__ UnitSlot s_unit[kStages];
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -471,36 +504,77 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     const int n_rows = device_rows(P, &bad_rows);
     if (kMode != kModeResid && kMode != kModeHist && blockIdx.x == 0 && tid == 0) {
         P.counters[0] = 0;                       // residual queue, filled by the decide kernel
+        *unit_counter<kModeResid>(P) = 0ull;     // unit counters of the passes that follow this one in the call
+        *unit_counter<kModeHist>(P) = 0ull;
+        *unit_counter<kMode>(P) = 0ull;          // and this pass's own, published by the tag
+        __threadfence();
+        atomicExch(unit_tag(P), P.launch_tag);
         if (bad_rows) atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS);
     }
     const int n_streams = stream_count<kMode>(P, n_rows);
     const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
-    UnitCursor cur;
-    cur.init((nblk + kConsumerWarps - 1) / kConsumerWarps);
+    const int ppr = (nblk + kConsumerWarps - 1) / kConsumerWarps;
+    const long long total = (long long)n_streams * ppr;
     volatile int* abort_flag = &s_abort;
 
     if (warp == kConsumerWarps) {
-        // ---------------- producer warp: lane 0 issues the copies -----------------------
+        // ---------------- producer warp: lane 0 draws the units and issues the copies ----
+        // The first kStages units of a CTA follow from its index; every further one comes from a counter
+        // shared by the grid, so an SM that gets its data sooner takes more units and all CTAs finish
+        // together.  A draw is issued right after the copies of a turn and is needed two turns later.
+        unsigned long long* ctr = unit_counter<kMode>(P);
+        bool counter_ready = (kMode == kModeResid || kMode == kModeHist);    // zeroed by an earlier kernel
         int it = 0;
-        for (; cur.s < n_streams; cur.next(), ++it) {
+        // one turn of the pipeline with the unit held in `mine`; `mine` then receives the unit of the turn after
+        // next (the first kStages units of a CTA are fixed, so the stages fill without waiting for the counter)
+        auto turn = [&](long long& mine) -> bool {
+            const long long u = __shfl_sync(0xffffffffu, mine, 0);
             const int st = it % kStages;
             const uint32_t ph = (uint32_t)(it / kStages) & 1u;
-            if (*abort_flag) break;
+            const bool live = u < total;
+            UnitSlot slot;
+            const unsigned char *src0 = nullptr, *src1 = nullptr;
+            int bytes = 0;
+            if (lane == 0) {
+                if (live) {
+                    slot.s = total <= 0x7fffffffll ? (int)((unsigned)u / (unsigned)ppr) : (int)(u / ppr);
+                    slot.piece = (int)(u - (long long)slot.s * ppr);
+                    unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes);
+                    slot.scale = stream_scale<kMode>(P, slot.s, n_rows, n_streams);
+                } else {
+                    slot.s = -1; slot.piece = 0; slot.scale = 0.f;
+                }
+            }
+            if (*abort_flag) return false;
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(&empty_bar[st], ph ^ 1u))) {
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
-                break;
+                return false;
             }
             if (lane == 0) {
-                const unsigned char *src0, *src1;
-                int bytes;
-                unit_sources<kMode>(P, cur.s, cur.piece, n_rows, src0, src1, bytes);
-                unsigned char* dst = stage_mem + st * kStageBytes;
-                mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(bytes * M::kSrc));
-                bulk_g2s(dst, src0, (uint32_t)bytes, &full_bar[st]);
-                if (M::kSrc == 2) bulk_g2s(dst + M::kPieceBytes, src1, (uint32_t)bytes, &full_bar[st]);
+                s_unit[st] = slot;                 // read by the consumers after the barrier below completes
+                if (live) {
+                    unsigned char* dst = stage_mem + st * kStageBytes;
+                    mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(bytes * M::kSrc));
+                    bulk_g2s(dst, src0, (uint32_t)bytes, &full_bar[st]);
+                    if (M::kSrc == 2) bulk_g2s(dst + M::kPieceBytes, src1, (uint32_t)bytes, &full_bar[st]);
+                    if (!counter_ready && !(counter_ready = wait_for_tag(unit_tag(P), P.launch_tag))) {
+                        atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT);
+                        *abort_flag = 1;
+                        mine = total;
+                    } else {
+                        mine = (long long)gridDim.x * kStages + (long long)atomicAdd(ctr, 1ull);   // needed two turns from now
+                    }
+                } else {
+                    mbar_arrive(&full_bar[st]);    // end marker: no data follows
+                }
             }
             __syncwarp();
-        }
+            if (live) ++it;
+            return live;
+        };
+        static_assert(kStages == 2, "the producer keeps one pending unit per stage");
+        long long unit_a = blockIdx.x, unit_b = (long long)blockIdx.x + gridDim.x;
+        while (turn(unit_a) && turn(unit_b)) {}
         if (*abort_flag) {
             // leave only after every copy already issued has landed (bounded)
             for (int k = 0; k < kStages && k < it; ++k) {
@@ -510,19 +584,19 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
         }
     } else {
         // ---------------- consumer warps --------------------------------------------------
-        int it = 0;
-        for (; cur.s < n_streams; cur.next(), ++it) {
+        for (int it = 0;; ++it) {
             const int st = it % kStages;
             const uint32_t ph = (uint32_t)(it / kStages) & 1u;
             if (*abort_flag) break;
-            const float scale = stream_scale<kMode>(P, cur.s, n_rows, n_streams);   // in flight while we wait for the data
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(&full_bar[st], ph))) {
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
                 break;
             }
+            const UnitSlot slot = s_unit[st];
+            if (slot.s < 0) break;
             unsigned char* sp = stage_mem + st * kStageBytes + warp * M::kBlockBytes;
             SmemFetch f0{sp}, f1{sp + M::kPieceBytes};
-            consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1, scale);
+            consume_block<kElem, kMode>(P, slot.s, slot.piece, n_rows, warp, lane, f0, f1, slot.scale);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);
         }
@@ -1077,6 +1151,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     __shared__ double s_fin_S[2];
 
     pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0) *unit_tag(P) = 0ull;      // the streamed pass of this call is over
     const int r = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -1300,6 +1375,7 @@ __global__ void __launch_bounds__(kDecideThreads) queue_all_positions_kernel(Ver
 {
     constexpr int kWarps = kDecideThreads / 32;
     pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0) *unit_tag(P) = 0ull;      // the streamed pass of this call is over
     const int r = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     bool bad_rows;
@@ -1361,6 +1437,7 @@ __global__ void __launch_bounds__(kDecideThreads) greedy_decide_kernel(VerifyPar
     constexpr int kWarps = kDecideThreads / 32;
     __shared__ int s_bad, s_first, s_am[kWarps], s_neg[kWarps], s_emit, s_status;
     pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0) *unit_tag(P) = 0ull;      // the streamed pass of this call is over
     const int r = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     bool bad_rows;
@@ -1431,6 +1508,20 @@ __global__ void __launch_bounds__(kDecideThreads) greedy_decide_kernel(VerifyPar
 // Host side
 // ---------------------------------------------------------------------------------------
 static int g_force_direct = 0;
+
+// A 64-bit value no earlier call of this process used, and that leftover memory will not hold by chance:
+// a counter started from a hash of the clock and an address of this process image.
+static unsigned long long next_launch_tag()
+{
+    static std::atomic<unsigned long long> counter{[] {
+        unsigned long long x = (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count();
+        x ^= (unsigned long long)(uintptr_t)&g_force_direct * 0x9E3779B97F4A7C15ull;
+        x ^= x >> 31; x *= 0xBF58476D1CE4E5B9ull; x ^= x >> 29;
+        return x | 1ull;
+    }()};
+    unsigned long long t = counter.fetch_add(1, std::memory_order_relaxed);
+    return t ? t : counter.fetch_add(1, std::memory_order_relaxed);     // 0 is what the cell holds between calls
+}
 
 struct DeviceInfo { int sms; bool attrs_set; };
 static DeviceInfo& device_info()
@@ -1546,6 +1637,7 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.scale = 1.0f; P.seed = 0;
     P.accepted_len = accepted_len; P.out_tokens = out_tokens; P.out_p = nullptr; P.out_q = nullptr;
     P.counters = (int*)(ws + w.counters);
+    P.launch_tag = next_launch_tag();
     P.dev_status = dev_status ? dev_status : P.counters + 1;
     P.stats_t = (float2*)(ws + w.stats_t);
     P.stats_d = (float2*)(ws + w.stats_d);

@@ -190,6 +190,52 @@ def test_results_are_reproducible_run_to_run():
             np.testing.assert_array_equal(a[k], b[k])
 
 
+def test_one_workspace_serves_calls_of_different_kinds_and_sizes():
+    # the unit counters of the streamed passes live in the workspace: whatever an earlier call (greedy or
+    # sampling, larger or smaller, many back to back without a host sync) left there must not matter
+    big = W.config_2("cuda", R=24)
+    small = W.sampling_batch(torch.tensor([2, 0, 5]), 40_000, 8, "cuda", verify_seed=4)
+    greedy = W.greedy_batch(torch.tensor([3, 1, 0, 6]), 50_000, 3, "cuda", perturb=0.3)
+    want_big, want_small = H.gpu_verify(big), H.gpu_verify(small)
+    want_greedy = H.gpu_verify_greedy(greedy)
+    nbytes = max(B.dspark_verify_workspace_bytes(b.R, b.n_rows, b.V) for b in (big, small, greedy))
+    ws = B.workspace(nbytes).fill_(0xA5)
+
+    def sampling(b):
+        acc = torch.full((b.R,), -7, dtype=torch.int32, device="cuda")
+        out = torch.full((b.n_rows,), -7, dtype=torch.int32, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.dspark_verify(b.target, b.draft, b.row_offsets, b.draft_tokens, b.temperature, b.seed,
+                        draft_row_start=b.draft_row_start, accepted_len=acc, out_tokens=out, dev_status=st,
+                        workspace=ws, n_rows=b.n_rows)
+        return acc, out, st
+
+    def greedy_call(b):
+        acc = torch.full((b.R,), -7, dtype=torch.int32, device="cuda")
+        out = torch.full((b.n_rows,), -7, dtype=torch.int32, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.dspark_verify_greedy(b.target, b.row_offsets, b.draft_tokens, accepted_len=acc, out_tokens=out,
+                               dev_status=st, workspace=ws, n_rows=b.n_rows)
+        return acc, out, st
+
+    results = []
+    for rep in range(4):                         # all enqueued before the first result is read
+        results.append(("big", sampling(big)))
+        results.append(("greedy", greedy_call(greedy)))
+        results.append(("small", sampling(small)))
+        results.append(("small", sampling(small)))
+    torch.cuda.synchronize()
+    for kind, (acc, out, st) in results:
+        assert int(st.item()) == 0
+        if kind == "greedy":
+            np.testing.assert_array_equal(acc.cpu().numpy(), want_greedy[0])
+            np.testing.assert_array_equal(out.cpu().numpy(), want_greedy[1])
+        else:
+            want = want_big if kind == "big" else want_small
+            np.testing.assert_array_equal(acc.cpu().numpy(), want["acc"])
+            np.testing.assert_array_equal(out.cpu().numpy(), want["out"])
+
+
 def test_host_side_errors():
     b = W.sampling_batch(torch.tensor([1, 2]), 512, 1, "cuda")
     acc = torch.zeros(2, dtype=torch.int32, device="cuda"); out = torch.zeros(5, dtype=torch.int32, device="cuda")
