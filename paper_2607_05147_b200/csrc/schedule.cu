@@ -244,21 +244,36 @@ __global__ void __launch_bounds__(kSchedThreads, 1) sched_rank_kernel(SchedParam
 
     unsigned int rank = 0;
     unsigned long long mass = 0ull;
-    for (int t = warp; t < P.n_tiles; t += kWarps) {
-        const uint32_t ak = P.akey[t * 32 + lane];
-        const unsigned long long pf = P.pfix[t * 32 + lane];
-        const unsigned valid = __ballot_sync(0xffffffffu, ak != 0u);
-        if (valid == 0u) continue;
+    // the tiles of this warp, four at a time: their loads are issued together (one trip to the L2
+    // instead of four in a row), then searched one after the other
+    constexpr int kBatch = 4;
+    for (int t0 = warp; t0 < P.n_tiles; t0 += kBatch * kWarps) {
+        uint32_t akv[kBatch];
+        unsigned long long pfv[kBatch];
 #pragma unroll
-        for (int sgi = 0; sgi < kSegsPerTile; ++sgi) {
-            const int base = sgi * SEG;
-            const unsigned segmask = (SEG == 32) ? 0xffffffffu : (((1u << SEG) - 1u) << base);
-            const int cnt = __popc(valid & segmask);      // candidates form a prefix of the segment
-            const int r2 = P.gpad > 32 ? t / tiles_per_req : (t * 32 + base) / P.gpad;
-            const int j_base = P.gpad > 32 ? (t - r2 * tiles_per_req) * 32 : 0;
-            const int pos = segment_search<SEG>(ak, base, cnt, a1, j1, r1, j_base, r2);
-            const unsigned long long m = __shfl_sync(0xffffffffu, pf, base + (pos > 0 ? pos - 1 : 0));
-            if (pos > 0) { rank += (unsigned)pos; mass += m; }
+        for (int q = 0; q < kBatch; ++q) {
+            const int t = t0 + q * kWarps;
+            akv[q] = t < P.n_tiles ? P.akey[t * 32 + lane] : 0u;
+            pfv[q] = t < P.n_tiles ? P.pfix[t * 32 + lane] : 0ull;
+        }
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) {
+            const int t = t0 + q * kWarps;
+            const uint32_t ak = akv[q];
+            const unsigned long long pf = pfv[q];
+            const unsigned valid = __ballot_sync(0xffffffffu, ak != 0u);
+            if (valid == 0u) continue;                    // also a tile beyond the last one
+#pragma unroll
+            for (int sgi = 0; sgi < kSegsPerTile; ++sgi) {
+                const int base = sgi * SEG;
+                const unsigned segmask = (SEG == 32) ? 0xffffffffu : (((1u << SEG) - 1u) << base);
+                const int cnt = __popc(valid & segmask);      // candidates form a prefix of the segment
+                const int r2 = P.gpad > 32 ? t / tiles_per_req : (t * 32 + base) / P.gpad;
+                const int j_base = P.gpad > 32 ? (t - r2 * tiles_per_req) * 32 : 0;
+                const int pos = segment_search<SEG>(ak, base, cnt, a1, j1, r1, j_base, r2);
+                const unsigned long long m = __shfl_sync(0xffffffffu, pf, base + (pos > 0 ? pos - 1 : 0));
+                if (pos > 0) { rank += (unsigned)pos; mass += m; }
+            }
         }
     }
     s_rank[warp][lane] = rank;
@@ -329,6 +344,22 @@ __device__ void sched_final_stage(const SchedParams& P)
     const bool len_in_smem = R <= kSmemLenCap;
     int* len_arr = len_in_smem ? s_len : P.out_len;
     if (tid == 0) { s_nE = 0; s_status = 0; s_first_bad = 0x7fffffff; s_done = 0; }
+    // This stage is a chain of short steps, each of which would wait for its own trip to the L2: ask now
+    // for what the first round of the path walk and of the length count will read (place tid + 1 on the
+    // path; the by-rank arrays have an entry for every place, what lies beyond the admitted count is
+    // loaded but never used).
+    const int mt = P.max_tokens;
+    const int n_places = P.n_tiles * 32;
+    const int i_first = tid + 1;
+    unsigned long long pre_Ti = 0ull, pre_Tp = 0ull;
+    int pre_owner = 0;
+    if (i_first <= n_places) {
+        pre_Ti = P.t_by_rank[i_first];
+        if (i_first > 1) pre_Tp = P.t_by_rank[i_first - 1];
+        pre_owner = P.owner_by_rank[i_first];
+    }
+    const double pre_tab = P.table[R + i_first < mt ? R + i_first : mt];
+    const double pre_tab_prev = P.table[R + i_first - 1 < mt ? R + i_first - 1 : mt];
     __syncthreads();
     {
         int n = 0, cl = 0;
@@ -348,7 +379,6 @@ __device__ void sched_final_stage(const SchedParams& P)
     if (cap < 0) { cap = 0; if (tid == 0) s_status |= DSPARK_DEV_BUDGET_LT_R; }
     const int N = (int)(nE < cap ? nE : cap);
     const unsigned long long T0 = (unsigned long long)R << 40;
-    const int mt = P.max_tokens;
     if (tid == 0) {
         s_T_best = T0;
         s_theta_best = __dmul_rn(__ull2double_rn(T0), P.table[R < mt ? R : mt]);
@@ -361,16 +391,17 @@ __device__ void sched_final_stage(const SchedParams& P)
         const bool valid = i <= N;
         unsigned long long Ti = 0ull, Tp = 0ull;
         double theta_i = 0.0;
+        const bool first_round = base == 0;
         if (valid) {
-            Ti = P.t_by_rank[i];
-            Tp = (i == 1) ? T0 : P.t_by_rank[i - 1];
+            Ti = first_round ? pre_Ti : P.t_by_rank[i];
+            Tp = (i == 1) ? T0 : (first_round ? pre_Tp : P.t_by_rank[i - 1]);
             const int B = R + i;
-            theta_i = __dmul_rn(__ull2double_rn(Ti), P.table[B < mt ? B : mt]);
+            theta_i = __dmul_rn(__ull2double_rn(Ti), first_round ? pre_tab : P.table[B < mt ? B : mt]);
         }
         if (P.mode == DSPARK_SCHED_EARLY_STOP) {
             if (valid) {
                 const int Bp = R + i - 1;
-                const double theta_prev = __dmul_rn(__ull2double_rn(Tp), P.table[Bp < mt ? Bp : mt]);
+                const double theta_prev = __dmul_rn(__ull2double_rn(Tp), first_round ? pre_tab_prev : P.table[Bp < mt ? Bp : mt]);
                 if (!(theta_i > theta_prev)) atomicMin(&s_first_bad, i);
             }
             __syncthreads();
@@ -435,7 +466,7 @@ __device__ void sched_final_stage(const SchedParams& P)
     const int istar = s_istar;
 
     // ---- lengths l*_r = admitted candidates of request r -----------------------------------
-    for (int k = tid + 1; k <= istar; k += kSchedThreads) atomicAdd(&len_arr[P.owner_by_rank[k]], 1);
+    for (int k = tid + 1; k <= istar; k += kSchedThreads) atomicAdd(&len_arr[k == i_first ? pre_owner : P.owner_by_rank[k]], 1);
     __syncthreads();
     if (len_in_smem)
         for (int r = tid; r < R; r += kSchedThreads) P.out_len[r] = s_len[r];
