@@ -268,8 +268,9 @@ __global__ void __launch_bounds__(kSchedThreads, 1) sched_rank_kernel(SchedParam
                 const int base = sgi * SEG;
                 const unsigned segmask = (SEG == 32) ? 0xffffffffu : (((1u << SEG) - 1u) << base);
                 const int cnt = __popc(valid & segmask);      // candidates form a prefix of the segment
-                const int r2 = P.gpad > 32 ? t / tiles_per_req : (t * 32 + base) / P.gpad;
-                const int j_base = P.gpad > 32 ? (t - r2 * tiles_per_req) * 32 : 0;
+                // a padded block shorter than a tile is exactly one segment (gpad == SEG): no runtime division
+                const int r2 = SEG < 32 ? (t * 32 + base) / SEG : (tiles_per_req == 1 ? t : t / tiles_per_req);
+                const int j_base = SEG < 32 ? 0 : (t - r2 * tiles_per_req) * 32;
                 const int pos = segment_search<SEG>(ak, base, cnt, a1, j1, r1, j_base, r2);
                 const unsigned long long m = __shfl_sync(0xffffffffu, pf, base + (pos > 0 ? pos - 1 : 0));
                 if (pos > 0) { rank += (unsigned)pos; mass += m; }
