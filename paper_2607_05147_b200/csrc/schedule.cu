@@ -199,13 +199,15 @@ template <int SEG>
 __device__ __forceinline__ int segment_search(uint32_t ak, int base, int cnt, uint32_t a1, int j1, int r1,
                                               int j_base, int r2)
 {
+    // entries that are not candidates hold the key 0 and follow the candidates, so "a2 > a1" alone finds
+    // the count: a halving search over places 0 .. SEG-1, then one look at the place it stopped at
     int pos = 0;
 #pragma unroll
-    for (int step = SEG; step >= 1; step >>= 1) {
-        const int probe = pos + step;
-        const uint32_t a2 = __shfl_sync(0xffffffffu, ak, base + (probe <= SEG ? probe : SEG) - 1);
-        if (probe <= cnt && a2 > a1) pos = probe;
+    for (int step = SEG / 2; step >= 1; step >>= 1) {
+        const uint32_t a2 = __shfl_sync(0xffffffffu, ak, base + pos + step - 1);
+        if (a2 > a1) pos += step;
     }
+    if (__shfl_sync(0xffffffffu, ak, base + pos) > a1) ++pos;
     const uint32_t a_next = __shfl_sync(0xffffffffu, ak, base + (pos < SEG ? pos : SEG - 1));
     if (__any_sync(0xffffffffu, pos < cnt && a_next == a1)) {
         pos = 0;
