@@ -169,7 +169,12 @@ __device__ __forceinline__ bool wait_for_tag(const unsigned long long* cell, uns
     }
     return false;
 }
-struct UnitSlot { int s, piece; float scale; };   // what the producer tells the consumers about a stage
+struct __align__(16) UnitSlot {    // what the producer tells the consumers about a stage
+    int s, piece;
+    float scale;
+    int pad;
+    ResidTask task;                // residual pass: the task of stream s (loaded once per unit, not once per warp)
+};
 
 // Walks the units (stream s, piece) owned by this CTA: unit index = s * ppr + piece, advancing by
 // gridDim.x units per step without divisions.
@@ -350,11 +355,14 @@ struct ResidConst {
 // A target logit below the truncation threshold of its row counts as -inf (p = 0): top-k / top-p.
 __device__ __forceinline__ float cut_below(float x, float tau) { return x >= tau ? x : kNegInf; }
 
+template <bool kCut>
 __device__ __forceinline__ uint64_t resid_pair(uint64_t xt2, uint64_t xd2, const ResidConst& K)
 {
     float a0, a1, b0, b1;
-    unpack2(xt2, a0, a1);
-    xt2 = pack2(cut_below(a0, K.tau), cut_below(a1, K.tau));
+    if (kCut) {                    // without truncation (tau = -inf) the cut is the identity on every usable row
+        unpack2(xt2, a0, a1);
+        xt2 = pack2(cut_below(a0, K.tau), cut_below(a1, K.tau));
+    }
     unpack2(fma2(xt2, K.s2, K.ncp2), a0, a1);
     unpack2(fma2(xd2, K.s2, K.ncq2), b0, b1);
     const uint64_t ep2 = pack2(ex2_approx(a0), ex2_approx(a1));
@@ -370,7 +378,7 @@ __device__ __forceinline__ float resid_elem(float xt, float xd, const ResidConst
     return fmaxf(__fmaf_rn(ep, K.inv_zp, __fmul_rn(eq, -K.inv_zq)), 0.0f);
 }
 
-template <int kElem, int kVec>
+template <int kElem, int kVec, bool kCut>
 __device__ __forceinline__ float block_resid(const uint4 (&vt)[kVec], const uint4 (&vd)[kVec], const ResidConst& K)
 {
     uint64_t acc0 = pack2(0.f, 0.f), acc1 = acc0;
@@ -380,13 +388,13 @@ __device__ __forceinline__ float block_resid(const uint4 (&vt)[kVec], const uint
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint32_t a = word_of(vt[k], i), b = word_of(vd[k], i);
-                const uint64_t w2 = resid_pair(pack2(bf16lo(a), bf16hi(a)), pack2(bf16lo(b), bf16hi(b)), K);
+                const uint64_t w2 = resid_pair<kCut>(pack2(bf16lo(a), bf16hi(a)), pack2(bf16lo(b), bf16hi(b)), K);
                 if (i & 1) acc1 = add2(acc1, w2); else acc0 = add2(acc0, w2);
             }
         } else {
-            acc0 = add2(acc0, resid_pair(pack2(__uint_as_float(vt[k].x), __uint_as_float(vt[k].y)),
+            acc0 = add2(acc0, resid_pair<kCut>(pack2(__uint_as_float(vt[k].x), __uint_as_float(vt[k].y)),
                                          pack2(__uint_as_float(vd[k].x), __uint_as_float(vd[k].y)), K));
-            acc1 = add2(acc1, resid_pair(pack2(__uint_as_float(vt[k].z), __uint_as_float(vt[k].w)),
+            acc1 = add2(acc1, resid_pair<kCut>(pack2(__uint_as_float(vt[k].z), __uint_as_float(vt[k].w)),
                                          pack2(__uint_as_float(vd[k].z), __uint_as_float(vd[k].w)), K));
         }
     }
@@ -399,7 +407,8 @@ __device__ __forceinline__ float block_resid(const uint4 (&vt)[kVec], const uint
 // What a consumer warp does with its block of the unit (stream s, piece).
 template <int kElem, int kMode, typename Fetch>
 __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int piece, int n_rows,
-                                              int warp, int lane, const Fetch& f0, const Fetch& f1, float scale)
+                                              int warp, int lane, const Fetch& f0, const Fetch& f1, float scale,
+                                              const ResidTask* task = nullptr)
 {
     using M = ModeCfg<kMode>;
     const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
@@ -440,10 +449,11 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
     } else {
         uint4 vd[M::kVec];
         load_block<kElem, M::kVec>(f1, nbytes, lane, vd);
-        const ResidTask t = P.resid[s];
+        const ResidTask t = task ? *task : P.resid[s];
         ResidConst K;
         K.set(t.scale, t.cp, t.inv_zp, t.cq, t.inv_zq, t.tau);
-        const float w = block_resid<kElem, M::kVec>(v, vd, K);
+        const float w = (t.tau == kNegInf) ? block_resid<kElem, M::kVec, false>(v, vd, K)
+                                           : block_resid<kElem, M::kVec, true>(v, vd, K);
         if (lane == 0) P.wblk[(long long)t.wslot * nblk + b] = w;
     }
 }
@@ -459,7 +469,8 @@ __device__ __forceinline__ float stream_scale(const VerifyParams& P, int s, int 
 // Source addresses of a unit (producer / direct path).
 template <int kMode>
 __device__ __forceinline__ void unit_sources(const VerifyParams& P, int s, int piece, int n_rows,
-                                             const unsigned char*& src0, const unsigned char*& src1, int& bytes)
+                                             const unsigned char*& src0, const unsigned char*& src1, int& bytes,
+                                             const ResidTask* task = nullptr)
 {
     using M = ModeCfg<kMode>;
     const long long off = (long long)piece * M::kPieceBytes;
@@ -467,7 +478,7 @@ __device__ __forceinline__ void unit_sources(const VerifyParams& P, int s, int p
     bytes = (int)(rem < M::kPieceBytes ? rem : M::kPieceBytes);
     src1 = nullptr;
     if (kMode == kModeResid) {
-        const ResidTask t = P.resid[s];
+        const ResidTask t = task ? *task : P.resid[s];
         src0 = P.target + (long long)t.row_t * P.tstride_bytes + off;
         src1 = P.draft + t.row_d * P.dstride_bytes + off;
     } else if (s < n_rows) {
@@ -539,7 +550,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 if (live) {
                     slot.s = total <= 0x7fffffffll ? (int)((unsigned)u / (unsigned)ppr) : (int)(u / ppr);
                     slot.piece = (int)(u - (long long)slot.s * ppr);
-                    unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes);
+                    if (kMode == kModeResid) slot.task = P.resid[slot.s];
+                    unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes, kMode == kModeResid ? &slot.task : nullptr);
                     slot.scale = stream_scale<kMode>(P, slot.s, n_rows, n_streams);
                 } else {
                     slot.s = -1; slot.piece = 0; slot.scale = 0.f;
@@ -551,7 +563,9 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 return false;
             }
             if (lane == 0) {
-                s_unit[st] = slot;                 // read by the consumers after the barrier below completes
+                // read by the consumers after the barrier below completes
+                s_unit[st].s = slot.s; s_unit[st].piece = slot.piece; s_unit[st].scale = slot.scale;
+                if (kMode == kModeResid) s_unit[st].task = slot.task;
                 if (live) {
                     unsigned char* dst = stage_mem + st * kStageBytes;
                     mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(bytes * M::kSrc));
@@ -592,11 +606,13 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
                 break;
             }
-            const UnitSlot slot = s_unit[st];
-            if (slot.s < 0) break;
+            const int unit_s = s_unit[st].s, unit_piece = s_unit[st].piece;
+            const float unit_scale = s_unit[st].scale;
+            if (unit_s < 0) break;
             unsigned char* sp = stage_mem + st * kStageBytes + warp * M::kBlockBytes;
             SmemFetch f0{sp}, f1{sp + M::kPieceBytes};
-            consume_block<kElem, kMode>(P, slot.s, slot.piece, n_rows, warp, lane, f0, f1, slot.scale);
+            consume_block<kElem, kMode>(P, unit_s, unit_piece, n_rows, warp, lane, f0, f1, unit_scale,
+                                        kMode == kModeResid ? &s_unit[st].task : nullptr);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);
         }
