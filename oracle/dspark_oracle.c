@@ -566,7 +566,9 @@ static void verify_request(const verify_job_t* J, int r)
                 last_pos = v;
                 if (cum > thr) {
                     double d0 = thr - prev, d1 = cum - thr;
-                    margin = (d0 < d1 ? d0 : d1) / W;
+                    /* in probability units, like the margin of a draw from p: the fp32 tolerance on p(v) and
+                     * q(v) bounds the running sum of max(0, p - q) absolutely, whatever its total W is */
+                    margin = d0 < d1 ? d0 : d1;
                     tok = v;
                     break;
                 }

@@ -20,7 +20,10 @@ def _pad_rows(t, rng):
     return buf[:, shift:shift + t.shape[1]]
 
 
-@pytest.mark.parametrize("seed", range(12))
+# seed 1416: a request whose target and draft rows agree to about 1e-10 in total variation (temperature 0.43,
+# one token holds almost all the mass) and that is rejected all the same: the residual's total mass is far
+# below what fp32 resolves, the emitted token is decided by rounding (oracle margin 1e-11 in probability)
+@pytest.mark.parametrize("seed", list(range(12)) + [1416])
 def test_sampling_fuzz(seed):
     rng = np.random.default_rng(1000 + seed)
     total_mism = 0
@@ -145,7 +148,8 @@ def test_markov_fuzz(seed):
         exact, bits = oracle.markov_logits(W.bf16_bits(m.U), W.bf16_bits(m.W1), W.bf16_bits(m.W2), m.x_prev.cpu().numpy())
         got = W.bf16_bits(out.contiguous())
         diff = np.abs(got.astype(np.int32) - bits.astype(np.int32))
-        assert diff[np.abs(exact) >= 2.0 ** -4].max(initial=0) <= 1 and float((diff != 0).mean()) <= 5e-3
+        assert diff[np.abs(exact) >= 2.0 ** -4].max(initial=0) <= 1
+        assert int((diff != 0).sum()) <= max(2, int(5e-3 * diff.size))      # rounding boundaries: a few per thousand
         want_c = oracle.confidence(W.bf16_bits(m.H), W.bf16_bits(m.W1), m.w_conf.cpu().numpy(), m.x_prev.cpu().numpy())
         assert np.abs(conf.cpu().numpy() - want_c).max() <= 1e-6
         off = np.arange(R + 1, dtype=np.int32)

@@ -264,6 +264,10 @@ def test_inverse_cdf_against_cumsum_searchsorted():
             want = int(np.searchsorted(cdf, ur * cdf[-1], side="right"))
             if res.token_margin[r] > 1e-9:
                 assert res.out_tokens[2 * r] == want
+                # the margin is the distance of u' W to the nearer end of the chosen token's interval of the
+                # running sum, in probability units (not divided by W)
+                thr, prev = ur * cdf[-1], (cdf[want - 1] if want else 0.0)
+                assert abs(res.token_margin[r] - min(thr - prev, cdf[want] - thr)) < 1e-12
     assert n_rej > 50
 
 
