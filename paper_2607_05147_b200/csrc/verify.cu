@@ -1315,10 +1315,11 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
     // this request (residual sums of a rejected position, or masses of the bonus row)
     const RequestRec rec = P.req[r];
     const float* wb = P.wblk + (long long)r * P.nblk_r;
-    const bool in_regs = P.nblk_r <= 256;
+    // the first 256 block values go to registers whatever the row length: a bonus draw uses the first nblk of
+    // them (nblk <= 256 can go with nblk_r > 256), a residual draw all nblk_r when they fit
     float xr[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) { const int i = k * 32 + lane; xr[k] = (in_regs && i < P.nblk_r) ? __ldcg(&wb[i]) : 0.f; }
+    for (int k = 0; k < 8; ++k) { const int i = k * 32 + lane; xr[k] = i < P.nblk_r ? __ldcg(&wb[i]) : 0.f; }
     if (rec.kind == kTaskNone) return;
     Level2Scratch<kElem>& S = s_scr[warp];
     const double u = (double)rec.u;

@@ -48,6 +48,28 @@ def test_sampling_fuzz(seed):
     assert total_mism <= 1
 
 
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 5006, 5026])
+def test_sampling_fuzz_many_units(seed):
+    # batches large enough that most 32 KB units of the streamed passes are handed out by the grid-wide
+    # counter (more than two units per CTA), with ragged last pieces and both dtypes
+    rng = np.random.default_rng(7000 + seed)
+    R = int(rng.integers(40, 300))
+    V = int(rng.choice([40_000, 65_536, 100_003, W.V_FULL, 200_000]))
+    lengths = torch.from_numpy(rng.integers(0, 9, size=R))
+    dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+    b = W.sampling_batch(lengths, V, int(rng.integers(0, 10**6)), "cuda", dtype=dtype,
+                         sigma=float(rng.uniform(1.0, 4)), draft_noise=float(rng.uniform(0.3, 2.5)),
+                         temperature=float(rng.uniform(0.5, 1.5)), verify_seed=int(rng.integers(0, 2**40)))
+    temps = None
+    if rng.random() < 0.5:
+        temps = torch.from_numpy(rng.uniform(0.5, 1.6, size=R).astype(np.float32)).cuda()
+    g, o, mism = H.check_sampling(b, want_probs=bool(rng.random() < 0.5), temperatures=temps)
+    assert mism <= 3                                       # a few hundred draws over ~1e5 tokens: margins of 1e-9 occur
+    assert (g["acc"] < lengths.numpy()).sum() > 5          # the residual pass had work
+    gb = W.greedy_batch(lengths, V, int(rng.integers(0, 10**6)), "cuda", tie_frac=0.1, perturb=0.3, dtype=dtype)
+    H.check_greedy(gb)
+
+
 @pytest.mark.parametrize("seed", range(6))
 def test_greedy_fuzz(seed):
     rng = np.random.default_rng(2000 + seed)

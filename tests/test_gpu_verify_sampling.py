@@ -73,9 +73,12 @@ def test_odd_vocabularies_dtypes_and_paths(V, dtype):
     np.testing.assert_array_equal(g["acc"], g1["acc"])
 
 
-@pytest.mark.parametrize("dtype,V", [(torch.bfloat16, 600_011), (torch.float32, 300_000), (torch.bfloat16, 1_100_000)])
+@pytest.mark.parametrize("dtype,V", [(torch.bfloat16, 600_011), (torch.float32, 300_000), (torch.bfloat16, 1_100_000),
+                                     (torch.float32, 200_000), (torch.bfloat16, 400_000)])
 def test_very_large_vocabularies(dtype, V):
-    # more than 256 statistics / residual blocks per row: the inverse CDF walks memory instead of registers
+    # more than 256 statistics / residual blocks per row: the inverse CDF walks memory instead of registers.
+    # The last two: at most 256 statistics blocks but more than 256 residual blocks per row, so a bonus draw
+    # still runs from registers while a residual draw walks memory
     lengths = torch.tensor([2, 0, 3, 1, 0, 2])
     batch = W.sampling_batch(lengths, V, 5, "cuda", dtype=dtype, temperature=1.1, draft_noise=1.5, verify_seed=V % 97)
     g, o, mism = H.check_sampling(batch)
