@@ -5,6 +5,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <chrono>
+
 #include "../../include/dspark.h"
 
 namespace dspark {
@@ -98,6 +101,19 @@ __device__ __forceinline__ float ex2_approx(float x)
 // returns once that kernel has completed and its writes are visible, and must precede any read of
 // its results.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Waits (bounded) until a 64-bit cell in global memory holds `tag`: how the CTAs of a grid learn that CTA 0
+// has zeroed the grid's work counters.  The tag is unique per launch (next_launch_tag), so whatever an
+// earlier launch or the caller left in the cell cannot be mistaken for it.
+__device__ __forceinline__ bool wait_for_tag(const unsigned long long* cell, unsigned long long tag)
+{
+    for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+        unsigned long long v;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(cell) : "memory");
+        if (v == tag) return true;
+    }
+    return false;
+}
 
 // Packed pairs of fp32 (sm_100 f32x2 arithmetic: one instruction, two IEEE-rounded results).
 __device__ __forceinline__ uint64_t pack2(float a, float b)
@@ -211,6 +227,21 @@ int truncate_virtual_launch(const void* target, long long stride_bytes, int V, c
                             const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
                             float* tau_rows, float2* stats_t, int nblk, int epb, const int32_t* only_flagged,
                             cudaStream_t stream);
+
+// A nonzero 64-bit value no earlier launch of this process used, and that leftover memory will not hold by
+// chance: a counter started from a hash of the clock and an address of this process image.
+inline unsigned long long next_launch_tag()
+{
+    static std::atomic<unsigned long long> counter{[] {
+        static int anchor;
+        unsigned long long x = (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count();
+        x ^= (unsigned long long)(uintptr_t)&anchor * 0x9E3779B97F4A7C15ull;
+        x ^= x >> 31; x *= 0xBF58476D1CE4E5B9ull; x ^= x >> 29;
+        return x | 1ull;
+    }()};
+    unsigned long long t = counter.fetch_add(1, std::memory_order_relaxed);
+    return t ? t : counter.fetch_add(1, std::memory_order_relaxed);     // 0 is what the cell holds between launches
+}
 
 // Launch with programmatic stream serialization (the kernel must call pdl_wait() first).
 template <typename... KArgs, typename... Args>

@@ -16,8 +16,6 @@
 //   finalize one warp per request: inverse CDF over block values (residual sums, or the saved
 //            statistics of the bonus row), then inside the one block that holds the crossing.
 #include <cuda_bf16.h>
-#include <atomic>
-#include <chrono>
 #include <cstdio>
 #include <math.h>
 
@@ -159,15 +157,6 @@ __device__ __forceinline__ unsigned long long* unit_counter(const VerifyParams& 
 __device__ __forceinline__ unsigned long long* unit_tag(const VerifyParams& P)
 {
     return reinterpret_cast<unsigned long long*>(P.counters) + 4;
-}
-__device__ __forceinline__ bool wait_for_tag(const unsigned long long* cell, unsigned long long tag)
-{
-    for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
-        unsigned long long v;
-        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(cell) : "memory");
-        if (v == tag) return true;
-    }
-    return false;
 }
 struct __align__(16) UnitSlot {    // what the producer tells the consumers about a stage
     int s, piece;
@@ -1525,20 +1514,6 @@ __global__ void __launch_bounds__(kDecideThreads) greedy_decide_kernel(VerifyPar
 // Host side
 // ---------------------------------------------------------------------------------------
 static int g_force_direct = 0;
-
-// A 64-bit value no earlier call of this process used, and that leftover memory will not hold by chance:
-// a counter started from a hash of the clock and an address of this process image.
-static unsigned long long next_launch_tag()
-{
-    static std::atomic<unsigned long long> counter{[] {
-        unsigned long long x = (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count();
-        x ^= (unsigned long long)(uintptr_t)&g_force_direct * 0x9E3779B97F4A7C15ull;
-        x ^= x >> 31; x *= 0xBF58476D1CE4E5B9ull; x ^= x >> 29;
-        return x | 1ull;
-    }()};
-    unsigned long long t = counter.fetch_add(1, std::memory_order_relaxed);
-    return t ? t : counter.fetch_add(1, std::memory_order_relaxed);     // 0 is what the cell holds between calls
-}
 
 struct DeviceInfo { int sms; bool attrs_set; };
 static DeviceInfo& device_info()

@@ -204,3 +204,53 @@ def test_bench_configuration_on_sampled_rows(R):
         if got[i] != want:
             assert min(abs(cum[want] - u), abs(u - (cum[want - 1] if want else 0.0))) < 1e-6, (r, got[i], want)
     print(f"[markov] R={R} V={V}: {len(rows)} sampled rows, one-ulp share {share:.2e}")
+
+
+def test_one_workspace_many_calls_and_graph_replay():
+    # calls of different sizes (one with two launches, R > 1024) back to back on one workspace without a host
+    # sync in between, then a captured call replayed several times: all must give the results of a fresh call
+    V = 9000
+    small, big = W.markov_input(200, V, 11, "cuda"), W.markov_input(1300, V, 12, "cuda")
+    want = {}
+    for name, m in (("small", small), ("big", big)):
+        out, conf, toks, st = _run(m, temperature=0.8, seed=5)
+        assert st == 0
+        want[name] = (out.clone(), toks.clone())
+    ws = B.workspace(max(B.dspark_markov_workspace_bytes(m.U.shape[0], V) for m in (small, big))).fill_(0x5A)
+    packed = {}
+    for name, m in (("small", small), ("big", big)):
+        packed[name] = torch.empty(B.dspark_markov_w2_packed_bytes(V), dtype=torch.uint8, device="cuda")
+        B.dspark_markov_pack_w2(m.W2, packed[name])
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def call(name, m, out, toks):
+        B.dspark_markov_draft_step(m.U, m.W1, packed[name], m.x_prev, 0.8, 5, out_logits=out, out_tokens=toks,
+                                   dev_status=st, workspace=ws)
+
+    results = []
+    for rep in range(3):
+        for name, m in (("big", big), ("small", small), ("small", small)):
+            out = torch.zeros_like(m.U); toks = torch.full((m.U.shape[0],), -9, dtype=torch.int32, device="cuda")
+            call(name, m, out, toks)
+            results.append((name, out, toks))
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    for name, out, toks in results:
+        assert torch.equal(out.view(torch.int16), want[name][0].view(torch.int16))
+        assert torch.equal(toks, want[name][1])
+    # graph replay
+    out = torch.zeros_like(small.U); toks = torch.full((200,), -9, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        call("small", small, out, toks)                       # warm-up on the capture stream
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            call("small", small, out, toks)
+        for rep in range(4):
+            out.zero_(); toks.fill_(-9)
+            g.replay()
+            side.synchronize()
+            assert int(st.item()) == 0
+            assert torch.equal(out.view(torch.int16), want["small"][0].view(torch.int16))
+            assert torch.equal(toks, want["small"][1])

@@ -73,8 +73,14 @@ def test_odd_vocabularies_dtypes_and_paths(V, dtype):
     np.testing.assert_array_equal(g["acc"], g1["acc"])
 
 
+# 256 is the number of block values the finalize kernel keeps in registers; rows of 131 072 / 262 144 / 524 288
+# logits sit exactly at 256 residual or statistics blocks for one of the dtypes
+_BLOCK_COUNT_EDGES = [(dt, V + d) for dt in (torch.bfloat16, torch.float32)
+                      for V in (131_072, 262_144, 524_288) for d in (0, 1)]
+
+
 @pytest.mark.parametrize("dtype,V", [(torch.bfloat16, 600_011), (torch.float32, 300_000), (torch.bfloat16, 1_100_000),
-                                     (torch.float32, 200_000), (torch.bfloat16, 400_000)])
+                                     (torch.float32, 200_000), (torch.bfloat16, 400_000)] + _BLOCK_COUNT_EDGES)
 def test_very_large_vocabularies(dtype, V):
     # more than 256 statistics / residual blocks per row: the inverse CDF walks memory instead of registers.
     # The last two: at most 256 statistics blocks but more than 256 residual blocks per row, so a bonus draw
