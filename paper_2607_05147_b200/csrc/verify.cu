@@ -269,7 +269,20 @@ __device__ __forceinline__ float2 block_stats(const uint4 (&v)[kVec], float scal
         mx = fmaxf(a, b);
     }
     const float wmax = warp_max_f32(mx);
-    if (wmax == kNegInf) return make_float2(kNegInf, 0.0f);
+    if (wmax == kNegInf) {
+        // nothing above -inf in this block: no mass -- unless a NaN hides behind the maximum (max drops NaN
+        // operands; with a finite maximum the NaN would reach the sum below and flag the row by itself)
+        bool nan = false;
+#pragma unroll
+        for (int k = 0; k < kVec; ++k)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t w = word_of(v[k], i);
+                if (kElem == 2) nan |= (w & 0x7FFFu) > 0x7F80u || ((w >> 16) & 0x7FFFu) > 0x7F80u;
+                else nan |= (w & 0x7FFFFFFFu) > 0x7F800000u;
+            }
+        return __any_sync(0xffffffffu, nan) ? make_float2(NAN, NAN) : make_float2(kNegInf, 0.0f);
+    }
     const float c = __fmul_rn(wmax, scale);
     const uint64_t s2 = pack2(scale, scale), nc2 = pack2(-c, -c);
     uint64_t acc0 = pack2(0.f, 0.f), acc1 = acc0;
@@ -1150,6 +1163,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
 {
     constexpr int kWarps = kDecideThreads / 32;
     __shared__ int s_first, s_bad, s_have_fin;
+    __shared__ int s_first_bad;      // first position with an unusable target or draft row among those looked at
     __shared__ float s_Ct[kWarps], s_Cd[kWarps];
     __shared__ double s_St[kWarps], s_Sd[kWarps];
     __shared__ float s_fin_C[2];     // [0] target, [1] draft statistics of the row that emits the token
@@ -1170,7 +1184,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     }
     const int len = hi - lo - 1;
     const long long drow0 = P.draft_row_start ? P.draft_row_start[r] : (long long)(lo - r);
-    if (tid == 0) { s_first = len; s_bad = 0; s_have_fin = 0; }
+    if (tid == 0) { s_first = len; s_bad = 0; s_have_fin = 0; s_first_bad = 0x7fffffff; }
     __syncthreads();
     for (int i = tid; i <= len; i += kDecideThreads) {
         P.out_tokens[lo + i] = -1;
@@ -1180,19 +1194,17 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
         }
     }
     __syncthreads();
-    if (s_bad) {
-        if (tid == 0) { atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
-        return;
-    }
     const bool want_all = (P.out_p != nullptr) || (P.out_q != nullptr);
     float scale_f = P.scale;
+    int bad_request = s_bad;                     // a request reports everything that is wrong with it
     if (P.req_temp) {
         const float T = P.req_temp[r];
-        if (!(T > 0.0f) || !(T < INFINITY)) {
-            if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_TEMPERATURE); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
-            return;
-        }
-        scale_f = (float)(1.4426950408889634 / (double)T);
+        if (!(T > 0.0f) || !(T < INFINITY)) bad_request |= DSPARK_DEV_BAD_TEMPERATURE;
+        else scale_f = (float)(1.4426950408889634 / (double)T);
+    }
+    if (bad_request) {
+        if (tid == 0) { atomicOr(P.dev_status, bad_request); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
+        return;
     }
     const double scale_d = (double)scale_f;
 
@@ -1224,7 +1236,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
                 s_Ct[warp] = A.C; s_St[warp] = A.S; s_Cd[warp] = D.C; s_Sd[warp] = D.S;
                 if (is_draft_pos) {
                     if (!row_usable(A.C, A.S) || !row_usable(D.C, D.S)) {
-                        atomicOr(&s_bad, DSPARK_DEV_BAD_ROW);
+                        atomicMin(&s_first_bad, j);
                     } else {
                         // truncated target (top-k / top-p): the row sum A.S already covers the kept set only
                         const bool cut = P.tau && xt < P.tau[lo + j];
@@ -1247,7 +1259,12 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             s_fin_C[0] = s_Ct[w]; s_fin_S[0] = s_St[w]; s_fin_C[1] = s_Cd[w]; s_fin_S[1] = s_Sd[w];
             s_have_fin = 1;
         }
-        const bool stop = s_bad || (!want_all && first < len);
+        // Which rows void the request: with the probability outputs every draft position is evaluated, and an
+        // unusable row anywhere voids it; without them verification ends at the first rejection, and only an
+        // unusable row before it counts (the warps of this round that looked further do not change the result)
+        const int first_bad = s_first_bad;
+        const bool void_req = want_all ? first_bad != 0x7fffffff : first_bad < first;
+        const bool stop = void_req || (!want_all && first < len);
         __syncthreads();                         // everyone has read the flags before the next round updates them
         if (stop) break;
     }
@@ -1258,9 +1275,10 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     rec.kind = kTaskNone; rec.row_t = lo + n; rec.row_d = drow0 + n;
     rec.cp = rec.cq = 0.f; rec.inv_zp = rec.inv_zq = 1.f; rec.u = 0.f; rec.scale = scale_f; rec.pad = 0;
     rec.tau = kNegInf;
-    if (s_bad || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
+    const bool void_req = want_all ? s_first_bad != 0x7fffffff : s_first_bad < n;
+    if (void_req || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
         (n < len && !row_usable(s_fin_C[1], s_fin_S[1]))) {
-        atomicOr(P.dev_status, s_bad ? s_bad : DSPARK_DEV_BAD_ROW);
+        atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW);
         P.accepted_len[r] = 0;
     } else {
         for (int i = 0; i < n; ++i) P.out_tokens[lo + i] = P.draft_tokens[lo + i];

@@ -170,6 +170,33 @@ def test_degenerate_batches():
     assert g["status"] & B.DEV_BAD_TOKEN
 
 
+def test_which_rows_void_a_request_and_hidden_nan():
+    V = 6000                                        # three 4 KB blocks of bf16 per row
+    lengths = torch.tensor([5, 5, 0, 2])
+    b = W.sampling_batch(lengths, V, 33, "cuda", verify_seed=12, draft_noise=2.0)
+    off = b.row_offsets.cpu().numpy()
+    # (1) a NaN in a block whose other elements are all -inf: the block maximum does not see it
+    t = b.target.clone()
+    t[off[2], :] = float("-inf"); t[off[2], 100] = 3.0; t[off[2], 5000] = float("nan")
+    g, o, _ = H.check_sampling(W.VerifyBatch(t, b.draft, b.row_offsets, b.draft_tokens, None, 1.0, 12, b.meta))
+    assert o.status[2] & B.DEV_BAD_ROW and g["status"] & B.DEV_BAD_ROW and g["out"][off[2]] == -1
+    # (2) an unusable row behind the first rejection: looked at only when the probabilities are asked for
+    base = H.gpu_verify(b, want_probs=False)
+    r = next(r for r in (0, 1) if base["acc"][r] < 4)        # rejected with at least one position behind it
+    t = b.target.clone()
+    t[off[r] + int(base["acc"][r]) + 1, 7] = float("nan")
+    bad = W.VerifyBatch(t, b.draft, b.row_offsets, b.draft_tokens, None, 1.0, 12, b.meta)
+    g0, o0, _ = H.check_sampling(bad, want_probs=False)
+    assert g0["status"] == 0 and g0["acc"][r] == base["acc"][r] and g0["out"][off[r] + g0["acc"][r]] >= 0
+    g1, o1, _ = H.check_sampling(bad, want_probs=True)
+    assert g1["status"] & B.DEV_BAD_ROW and (g1["out"][off[r]:off[r + 1]] == -1).all()
+    # (3) a request with a token out of range AND an invalid temperature reports both
+    toks = b.draft_tokens.clone(); toks[off[0]] = V
+    temps = torch.tensor([float("nan"), 1.0, 1.0, 0.9], device="cuda")
+    g, o, _ = H.check_sampling(W.VerifyBatch(b.target, b.draft, b.row_offsets, toks, None, 1.0, 12, b.meta), temperatures=temps)
+    assert g["status"] == B.DEV_BAD_TOKEN | B.DEV_BAD_TEMPERATURE
+
+
 def test_lossless_invariant_on_the_gpu():
     # first emitted token ~ p whatever q is (chi-square, V = 16, 60k single-position requests)
     rng = np.random.default_rng(5)
