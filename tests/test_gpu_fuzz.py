@@ -183,3 +183,119 @@ def test_markov_fuzz(seed):
             o = oracle.verify(got, got, off, np.zeros(R, dtype=np.int32), T, seed_v)
             for r in np.nonzero(tk != o.out_tokens[:R])[0]:
                 assert o.token_margin[r] < 1e-6, (r, tk[r], o.out_tokens[r], o.token_margin[r])
+
+
+# ---- special values: NaN, +-inf, huge, flat and empty rows, tokens / temperatures / lengths out of range ----
+_SPECIALS = [float("nan"), float("inf"), float("-inf"), 1.0e4, -1.0e4, 0.0, -0.0]
+
+
+def _corrupt(rng, tensors, V, n_max=10):
+    for _ in range(int(rng.integers(0, n_max))):
+        which = tensors[int(rng.integers(0, len(tensors)))]
+        if which.shape[0] == 0:
+            continue
+        r, v = int(rng.integers(0, which.shape[0])), int(rng.integers(0, V))
+        kind = rng.random()
+        if kind < 0.6:
+            which[r, v] = float(rng.choice(_SPECIALS))
+        elif kind < 0.8:
+            which[r, :] = float("-inf")
+        elif kind < 0.9:
+            which[r, :] = float(rng.choice([0.0, 5.0, -7.5]))          # a flat row: every token ties
+        else:
+            which[r, : max(1, V // 2)] = float("-inf")
+
+
+# seeds 20001 / 20022 / 20293: an unusable row behind the first rejection, a request with two things wrong
+# with it, a NaN in a block whose other elements are all -inf (all three once disagreed with the oracle)
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 20001, 20022, 20293])
+def test_special_values_fuzz(seed):
+    import oracle
+    rng = np.random.default_rng([seed, 0])
+    for it in range(1 if seed >= 20000 else 6):
+        R = int(rng.integers(1, 40))
+        lengths = torch.from_numpy(rng.integers(0, 8, size=R))
+        V = int(rng.choice([3, 100, 2049, 5000, 40_000, 129_280]))
+        dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+        b = W.sampling_batch(lengths, V, int(rng.integers(0, 10**6)), "cuda", dtype=dtype, sigma=float(rng.uniform(0.5, 4)),
+                             draft_noise=float(rng.uniform(0.05, 2.5)), temperature=float(rng.uniform(0.3, 2.0)),
+                             verify_seed=int(rng.integers(0, 2**40)), block=(8 if rng.random() < 0.3 else None))
+        t, d, toks = b.target.clone(), b.draft.clone(), b.draft_tokens.clone()
+        for _ in range(int(rng.integers(0, 12))):
+            which = t if rng.random() < 0.6 else d
+            r_, v_ = int(rng.integers(0, which.shape[0])), int(rng.integers(0, V))
+            kind = rng.random()
+            if kind < 0.6:
+                which[r_, v_] = float(rng.choice(_SPECIALS))
+            elif kind < 0.8:
+                which[r_, :] = float("-inf")
+            elif kind < 0.9:
+                which[r_, :] = float(rng.choice([0.0, 5.0, -7.5]))
+            else:
+                which[r_, : max(1, V // 2)] = float("-inf")
+        for _ in range(int(rng.integers(0, 3))):
+            toks[int(rng.integers(0, toks.numel()))] = int(rng.choice([-1, V, V + 5, 2**31 - 1, -2**31]))
+        temps = None
+        if rng.random() < 0.5:
+            tv = rng.uniform(0.4, 1.8, size=R).astype(np.float32)
+            for _ in range(int(rng.integers(0, 3))):
+                tv[int(rng.integers(0, R))] = np.float32(rng.choice([0.0, -1.0, np.nan, np.inf]))
+            temps = torch.from_numpy(tv).cuda()
+        bb = W.VerifyBatch(t, d, b.row_offsets, toks, b.draft_row_start, b.temperature, b.seed, b.meta)
+        want_probs = bool(rng.random() < 0.5)
+        _, _, mism = H.check_sampling(bb, want_probs=want_probs, temperatures=temps)
+        assert mism <= 2
+        H.check_greedy(W.VerifyBatch(t, None, b.row_offsets, toks.clamp(0, V - 1)))
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_special_values_fuzz_other_entry_points(seed):
+    import oracle
+    import test_gpu_accept_rate as AR
+    import test_gpu_verify_truncated as TV
+    rng = np.random.default_rng([seed, 1])
+    for it in range(4):
+        # truncated verification and truncation in place
+        R = int(rng.integers(1, 30))
+        lengths = torch.from_numpy(rng.integers(0, 6, size=R))
+        V = int(rng.choice([3, 100, 2049, 5000, 40_000]))
+        b = W.sampling_batch(lengths, V, int(rng.integers(0, 10**6)), "cuda", temperature=float(rng.uniform(0.5, 1.5)),
+                             sigma=float(rng.uniform(1, 4)), draft_noise=float(rng.uniform(0.3, 2.0)),
+                             verify_seed=int(rng.integers(0, 2**40)))
+        t, d = b.target.clone(), b.draft.clone()
+        _corrupt(rng, [t, d], V)
+        bb = W.VerifyBatch(t, d, b.row_offsets, b.draft_tokens, b.draft_row_start, b.temperature, b.seed, b.meta)
+        ks = rng.choice([-3, 0, 1, 2, 5, 40, V, V + 7], size=R).astype(np.int32)
+        ps = rng.choice([1.0, 0.99, 0.9, 0.5, 0.0, 1.5, -0.5], size=R).astype(np.float32)
+        temps = rng.uniform(0.5, 1.6, size=R).astype(np.float32) if rng.random() < 0.5 else None
+        want_probs = bool(rng.random() < 0.5)
+        g = TV._gpu_truncated(bb, ks, ps, temps, want_probs=want_probs)
+        off = bb.row_offsets.cpu().numpy()
+        masked, tau, kept, margin = oracle.warp_target(W.bf16_bits(bb.target), off, top_k=ks, top_p=ps,
+                                                       temperature=bb.temperature, temperatures=temps)
+        if not (margin < 1e-5).any():
+            o = oracle.verify(masked, W.bf16_bits(bb.draft), off, bb.draft_tokens.cpu().numpy(), bb.temperature, bb.seed,
+                              eval_all=want_probs, n_threads=H.THREADS, temperatures=temps)
+            assert H.compare_sampling(g, o, off, check_probs=want_probs) <= 2
+            got = t.clone()
+            dev = lambda a, dt: torch.as_tensor(a, dtype=dt, device="cuda")
+            B.dspark_truncate_target(got, bb.row_offsets, top_k=dev(ks, torch.int32), top_p=dev(ps, torch.float32),
+                                     temperature=bb.temperature, temperatures=None if temps is None else dev(temps, torch.float32))
+            torch.cuda.synchronize()
+            np.testing.assert_array_equal(W.bf16_bits(got), masked)
+        # acceptance rate
+        if int(lengths.sum()) > 0:
+            AR._check(bb, float(bb.temperature))
+        # scheduler: confidences outside [0, 1], NaN, denormals; lengths and K out of range
+        Rs, gamma = int(rng.integers(1, 300)), int(rng.choice([1, 2, 5, 8, 16, 32, 33]))
+        conf = rng.uniform(0.0, 1.0, size=(Rs, gamma)).astype(np.float32)
+        for _ in range(int(rng.integers(0, 20))):
+            conf[int(rng.integers(0, Rs)), int(rng.integers(0, gamma))] = np.float32(
+                rng.choice([np.nan, np.inf, -np.inf, -0.5, 1.5, 0.0, 1.0, 1e-30, 1e-45, 2.0]))
+        hi = Rs * (gamma + 1) + 5
+        bp = np.sort(rng.choice(np.arange(1, hi), size=min(int(rng.integers(1, 6)), hi - 1), replace=False)).tolist()
+        s = W.ScheduleInput(torch.from_numpy(conf), bp, rng.uniform(1, 100, len(bp)).tolist(), int(rng.integers(0, hi + 10)),
+                            max_tokens=int(rng.integers(1, hi + 1)))
+        mode = int(rng.choice([B.DSPARK_SCHED_EARLY_STOP, B.DSPARK_SCHED_GLOBAL, B.DSPARK_SCHED_TOPK]))
+        dl = rng.integers(-2, gamma + 3, size=Rs).astype(np.int32) if rng.random() < 0.4 else None
+        H.check_schedule(s, mode, topk=int(rng.integers(-2, Rs * gamma + 2)), draft_len=dl)
