@@ -272,6 +272,35 @@ def test_one_workspace_serves_calls_of_different_kinds_and_sizes():
             np.testing.assert_array_equal(out.cpu().numpy(), want["out"])
 
 
+def test_calls_on_several_streams_at_once():
+    # every call has its own workspace; the kernels of different calls share the SMs (so the CTAs of one grid are
+    # not all resident at once) and nothing in the library is shared between them
+    rng = np.random.default_rng(5)
+    jobs = []
+    for i in range(4):
+        R, V = int(rng.integers(20, 200)), int(rng.choice([5000, 40_000, W.V_FULL]))
+        b = W.sampling_batch(torch.from_numpy(rng.integers(0, 8, size=R)), V, 100 + i, "cuda", verify_seed=50 + i, draft_noise=1.5)
+        jobs.append(dict(b=b, ref=H.gpu_verify(b, want_probs=False), stream=torch.cuda.Stream(),
+                         ws=B.workspace(B.dspark_verify_workspace_bytes(b.R, b.n_rows, b.V)).fill_(0xFF),
+                         acc=torch.zeros(b.R, dtype=torch.int32, device="cuda"),
+                         out=torch.zeros(b.n_rows, dtype=torch.int32, device="cuda"),
+                         st=torch.zeros(1, dtype=torch.int32, device="cuda")))
+    torch.cuda.synchronize()
+    for it in range(12):
+        for j in jobs:
+            with torch.cuda.stream(j["stream"]):
+                j["acc"].fill_(-3); j["out"].fill_(-3)
+                b = j["b"]
+                B.dspark_verify(b.target, b.draft, b.row_offsets, b.draft_tokens, b.temperature, b.seed,
+                                draft_row_start=b.draft_row_start, accepted_len=j["acc"], out_tokens=j["out"],
+                                dev_status=j["st"], workspace=j["ws"], n_rows=b.n_rows)
+        torch.cuda.synchronize()
+        for j in jobs:
+            assert int(j["st"].item()) == 0
+            np.testing.assert_array_equal(j["acc"].cpu().numpy(), j["ref"]["acc"])
+            np.testing.assert_array_equal(j["out"].cpu().numpy(), j["ref"]["out"])
+
+
 def test_host_side_errors():
     b = W.sampling_batch(torch.tensor([1, 2]), 512, 1, "cuda")
     acc = torch.zeros(2, dtype=torch.int32, device="cuda"); out = torch.zeros(5, dtype=torch.int32, device="cuda")
