@@ -226,6 +226,13 @@ int dspark_verify_greedy_static(const void* target_logits, int dtype, int64_t ta
  *  out_p_tok/out_q_tok  device [n_rows] fp32 or NULL: p(x), q(x) at every draft position
  *                   (bonus-row entries are not written).  When NULL, positions after the first
  *                   rejection are not evaluated.
+ * Device-side errors void one request (accepted_len 0, its tokens -1) and set a bit of *dev_status; the
+ * others are unaffected.  DSPARK_DEV_BAD_TOKEN: any draft token of the request outside [0, V).
+ * DSPARK_DEV_BAD_ROW: an unusable row (NaN, +inf, no finite element) among the rows that decide the output,
+ * i.e. the target and draft rows of the positions up to the first rejection and the row the emitted token is
+ * drawn from; with out_p_tok / out_q_tok every draft position is evaluated and an unusable row at any of them
+ * voids the request.  A request reports every bit that applies to it.  Logits must be small enough for
+ * x * log2(e) / T to stay finite in fp32 (|x| / T below about 2e38); larger finite values count as infinite.
  * Streams every target and draft row once (online softmax statistics per 4 KB block), then
  * re-reads only the rejected position's row pair of each rejected request.
  * Errors: INVALID_ARG, SHAPE, WORKSPACE, CUDA.
