@@ -536,6 +536,9 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
         // shared by the grid, so an SM that gets its data sooner takes more units and all CTAs finish
         // together.  A draw is issued right after the copies of a turn and is needed two turns later.
         unsigned long long* ctr = unit_counter<kMode>(P);
+        // logit rows are read once (a rejected pair twice): their lines are the first to go, so that what the
+        // short kernels of the step keep re-reading -- statistics, tokens, offsets, scheduler state -- stays in L2
+        const uint64_t pol_first = l2_policy_evict_first();
         bool counter_ready = (kMode == kModeResid || kMode == kModeHist);    // zeroed by an earlier kernel
         int it = 0;
         // one turn of the pipeline with the unit held in `mine`; `mine` then receives the unit of the turn after
@@ -571,8 +574,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 if (live) {
                     unsigned char* dst = stage_mem + st * kStageBytes;
                     mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(bytes * M::kSrc));
-                    bulk_g2s(dst, src0, (uint32_t)bytes, &full_bar[st]);
-                    if (M::kSrc == 2) bulk_g2s(dst + M::kPieceBytes, src1, (uint32_t)bytes, &full_bar[st]);
+                    bulk_g2s_hint(dst, src0, (uint32_t)bytes, &full_bar[st], pol_first);
+                    if (M::kSrc == 2) bulk_g2s_hint(dst + M::kPieceBytes, src1, (uint32_t)bytes, &full_bar[st], pol_first);
                     if (!counter_ready && !(counter_ready = wait_for_tag(unit_tag(P), P.launch_tag))) {
                         atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT);
                         *abort_flag = 1;
