@@ -188,14 +188,15 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
  *
  * Arguments, outputs and device-side error reporting are those of dspark_verify_greedy, minus
  * the workspace.  Differences a caller has to know:
- *  - Size limit.  A batch whose scratch need (dspark_verify_workspace_bytes(R, n_rows, V))
- *    exceeds dspark_verify_greedy_static_capacity() is refused with DSPARK_ERR_STATIC_LIMIT and a
- *    message on stderr; nothing is launched.  8 MiB covers about 8 000 fp32 rows or 16 000
- *    bf16 rows at V = 129 280.
+ *  - Size limit.  A batch whose scratch need, dspark_verify_greedy_static_bytes(R, n_rows, V, dtype) =
+ *    about 8 bytes per 4 KB of logit row plus 12 bytes per row and 8 per request, exceeds
+ *    dspark_verify_greedy_static_capacity() is refused with DSPARK_ERR_STATIC_LIMIT and a message on
+ *    stderr; nothing is launched.  8 MiB covers about 8 000 fp32 rows or 16 000 bf16 rows at V = 129 280.
  *  - First call on a device.  It looks up the device address of the array
  *    (cudaGetSymbolAddress) with that device current and caches it; later calls on that
  *    device do no set-up.  Make that first call during initialisation, before any stream
- *    capture begins.
+ *    capture begins.  On every call the device that owns `stream` must be the current device:
+ *    the array that is used is the current device's copy.
  *  - One array for everybody.  All calls in the process, on every stream, share it, and it keeps
  *    whatever the previous call left.  That is harmless for results (each call rewrites every
  *    entry it later reads), but two calls that overlap in time on the GPU race on it: run them
@@ -204,6 +205,7 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
  */
 #define DSPARK_STATIC_SCRATCH_BYTES (8u << 20)
 size_t dspark_verify_greedy_static_capacity(void);
+size_t dspark_verify_greedy_static_bytes(int R, int n_rows, int V, int dtype);
 int dspark_verify_greedy_static(const void* target_logits, int dtype, int64_t target_row_stride, int V,
                                 const int32_t* row_offsets, const int32_t* draft_tokens, int R, int n_rows,
                                 int32_t* accepted_len, int32_t* out_tokens, int32_t* dev_status,
@@ -435,7 +437,8 @@ enum {
     DSPARK_K_SCHEDULE = 0, DSPARK_K_OFFSETS = 1, DSPARK_K_STREAM = 2, DSPARK_K_DECIDE = 3,
     DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6, DSPARK_K_GREEDY_DECIDE = 7,
     DSPARK_K_ROW_SCALE = 8, DSPARK_K_MARKOV_GEMM = 9, DSPARK_K_MARKOV_DRAW = 10, DSPARK_K_TRUNCATE = 11,
-    DSPARK_K_COUNT = 12
+    DSPARK_K_VERIFY_FUSED = 12, DSPARK_K_GREEDY_FUSED = 13,
+    DSPARK_K_COUNT = 14
 };
 int dspark_ktimer_create(int capacity, dspark_ktimer_t** out);
 int dspark_ktimer_destroy(dspark_ktimer_t* t);
@@ -443,9 +446,10 @@ int dspark_ktimer_attach(dspark_ktimer_t* t);
 int dspark_ktimer_reset(dspark_ktimer_t* t);
 int dspark_ktimer_read(dspark_ktimer_t* t, int kernel_id, float* total_ms, int* launches);
 
-/* Diagnostic switch for the streamed passes: 0 = automatic (bulk-copy pipeline when the
- * 16-byte rules hold, direct loads otherwise), 1 = always direct loads.  Results are the
- * same either way up to fp32 summation order.  Process-wide; the paper has no counterpart. */
+/* Diagnostic switch for the verifiers: 0 = automatic (the single-launch kernel with its bulk-copy
+ * pipeline when the 16-byte rules hold, separate passes with direct loads otherwise), 1 = always
+ * separate passes with direct loads, 2 = separate passes with bulk copies.  Results are the same
+ * up to fp32 summation order.  Process-wide (an atomic); the paper has no counterpart. */
 int dspark_set_stream_path(int path);
 
 const char* dspark_status_string(int status);

@@ -22,14 +22,15 @@ DSPARK_SCHED_EARLY_STOP, DSPARK_SCHED_GLOBAL, DSPARK_SCHED_TOPK = 0, 1, 2
 DEV_BAD_OFFSETS, DEV_BAD_TOKEN, DEV_BAD_ROW, DEV_TIMEOUT = 1, 2, 4, 8
 DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF, DEV_BAD_TEMPERATURE = 16, 32, 64, 128
 (K_SCHEDULE, K_OFFSETS, K_STREAM, K_DECIDE, K_RESIDUAL, K_FINALIZE, K_GREEDY_STREAM, K_GREEDY_DECIDE,
- K_ROW_SCALE, K_MARKOV_GEMM, K_MARKOV_DRAW, K_TRUNCATE, K_COUNT) = range(13)
+ K_ROW_SCALE, K_MARKOV_GEMM, K_MARKOV_DRAW, K_TRUNCATE, K_VERIFY_FUSED, K_GREEDY_FUSED, K_COUNT) = range(15)
 
 EXPORTS = [
     "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",
     "dspark_schedule_workspace_bytes", "dspark_schedule", "dspark_build_offsets",
     "dspark_schedule_async", "dspark_async_state_init",
     "dspark_verify_workspace_bytes", "dspark_verify_greedy", "dspark_verify", "dspark_uniforms",
-    "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity", "dspark_verify_per_request",
+    "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity", "dspark_verify_greedy_static_bytes",
+    "dspark_verify_per_request",
     "dspark_accept_rate", "dspark_accept_rate_workspace_bytes",
     "dspark_markov_w2_packed_bytes", "dspark_markov_pack_w2", "dspark_markov_workspace_bytes",
     "dspark_markov_logits", "dspark_markov_draft_step", "dspark_markov_set_epilogue_path",
@@ -75,6 +76,8 @@ def lib() -> C.CDLL:
         L.dspark_verify_greedy_static.argtypes = [vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp]
         L.dspark_verify_greedy_static_capacity.argtypes = []
         L.dspark_verify_greedy_static_capacity.restype = sz
+        L.dspark_verify_greedy_static_bytes.argtypes = [i32, i32, i32, i32]
+        L.dspark_verify_greedy_static_bytes.restype = sz
         L.dspark_verify.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, C.c_float, u64,
                                     vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_verify_per_request.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, vp, u64,
@@ -263,6 +266,12 @@ def dspark_verify_greedy(target: torch.Tensor, row_offsets: torch.Tensor, draft_
 
 def dspark_verify_greedy_static_capacity() -> int:
     return int(lib().dspark_verify_greedy_static_capacity())
+
+
+def dspark_verify_greedy_static_bytes(R: int, n_rows: int, V: int, dtype: torch.dtype) -> int:
+    """Bytes of the built-in array a batch of this shape would use (0: invalid shape)."""
+    code = DSPARK_BF16 if dtype == torch.bfloat16 else DSPARK_F32
+    return int(lib().dspark_verify_greedy_static_bytes(R, n_rows, V, code))
 
 
 def dspark_verify_greedy_static(target: torch.Tensor, row_offsets: torch.Tensor, draft_tokens: torch.Tensor, *,
