@@ -169,12 +169,9 @@ class Step:
             gpad = 1 << max(0, (gamma - 1).bit_length()) if gamma <= 32 else (gamma + 31) // 32 * 32
             entries = self.R * gpad
             n_sched = 2 + (1 if entries >= 8192 and 2 * (self.sched.budget_tokens - self.R) <= entries else 0)
-        # the verifier is one launch; with truncation it runs as separate passes (row scales, statistics, five
-        # for the threshold search, decide, residual, finalize)
-        if wl["greedy"] or TRUNCATE is None:
-            n_verify = 1
-        else:
-            n_verify = 4 + 5 + (1 if PER_REQUEST_T else 0)
+        # verifier: statistics pass + accept / residual / draw kernel (greedy: argmax pass + decide); row scales for
+        # per-request temperatures, five launches more for the threshold search of a truncated target
+        n_verify = 2 + (1 if PER_REQUEST_T and not wl["greedy"] else 0) + (5 if TRUNCATE is not None and not wl["greedy"] else 0)
         self.launches_per_step = n_sched + n_verify
 
     def run(self, batch, conf=None):
@@ -692,12 +689,10 @@ def main():
         peak, peak_src = float(json.load(open(peaks_file))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     else:
         peak, peak_src = FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
-    fused = TRUNCATE is None
-    dom = ("greedy_fused" if wl["greedy"] else "verify_fused") if fused else "stream_stats"
+    dom = "greedy_stream" if wl["greedy"] else "stream_stats"
     k = res["kernels"].get(dom, {"ms": float("nan"), "launches": 1})
     dom_ms = k["ms"] / max(1, k["launches"])
-    # the single-launch verifier also does the residual re-reads: its algorithmic bytes are those of the call
-    dom_bytes = all_bytes if fused else stream_bytes
+    dom_bytes = stream_bytes
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
@@ -747,10 +742,9 @@ def main():
                 res = time_workload(name, args.steps, args.warmup, False, False)
                 wl = res["wl"]
                 sb, ab = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
-                d = "greedy_fused" if wl["greedy"] else "verify_fused"
+                d = "greedy_stream" if wl["greedy"] else "stream_stats"
                 kk = res["kernels"][d]
                 dms = kk["ms"] / kk["launches"]
-                sb = ab
                 others[name] = {"rows_per_s": res["n_rows"] * args.steps / (res["ms"] * 1e-3),
                                 "ms_per_step": res["ms"] / args.steps,
                                 "step_effective_gbs": ab / (res["ms"] / args.steps * 1e-3) / 1e9,

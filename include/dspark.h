@@ -188,10 +188,11 @@ int dspark_verify_greedy(const void* target_logits, int dtype, int64_t target_ro
  *
  * Arguments, outputs and device-side error reporting are those of dspark_verify_greedy, minus
  * the workspace.  Differences a caller has to know:
- *  - Size limit.  A batch whose scratch need, dspark_verify_greedy_static_bytes(R, n_rows, V, dtype) =
- *    about 8 bytes per 4 KB of logit row plus 12 bytes per row and 8 per request, exceeds
- *    dspark_verify_greedy_static_capacity() is refused with DSPARK_ERR_STATIC_LIMIT and a message on
- *    stderr; nothing is launched.  8 MiB covers about 8 000 fp32 rows or 16 000 bf16 rows at V = 129 280.
+ *  - Size limit.  The array has to hold what greedy verification itself uses: 256 bytes plus 8 bytes per
+ *    4 KB block of every target row (dspark_verify_greedy_static_bytes(R, n_rows, V, dtype) gives the exact
+ *    figure).  A batch that needs more than dspark_verify_greedy_static_capacity() is refused with
+ *    DSPARK_ERR_STATIC_LIMIT and a message on stderr; nothing is launched.  8 MiB covers 8 256 fp32 rows
+ *    or 16 383 bf16 rows at V = 129 280.
  *  - First call on a device.  It looks up the device address of the array
  *    (cudaGetSymbolAddress) with that device current and caches it; later calls on that
  *    device do no set-up.  Make that first call during initialisation, before any stream
@@ -437,8 +438,7 @@ enum {
     DSPARK_K_SCHEDULE = 0, DSPARK_K_OFFSETS = 1, DSPARK_K_STREAM = 2, DSPARK_K_DECIDE = 3,
     DSPARK_K_RESIDUAL = 4, DSPARK_K_FINALIZE = 5, DSPARK_K_GREEDY_STREAM = 6, DSPARK_K_GREEDY_DECIDE = 7,
     DSPARK_K_ROW_SCALE = 8, DSPARK_K_MARKOV_GEMM = 9, DSPARK_K_MARKOV_DRAW = 10, DSPARK_K_TRUNCATE = 11,
-    DSPARK_K_VERIFY_FUSED = 12, DSPARK_K_GREEDY_FUSED = 13,
-    DSPARK_K_COUNT = 14
+    DSPARK_K_COUNT = 12
 };
 int dspark_ktimer_create(int capacity, dspark_ktimer_t** out);
 int dspark_ktimer_destroy(dspark_ktimer_t* t);

@@ -22,7 +22,7 @@ DSPARK_SCHED_EARLY_STOP, DSPARK_SCHED_GLOBAL, DSPARK_SCHED_TOPK = 0, 1, 2
 DEV_BAD_OFFSETS, DEV_BAD_TOKEN, DEV_BAD_ROW, DEV_TIMEOUT = 1, 2, 4, 8
 DEV_CONF_CLAMPED, DEV_BUDGET_LT_R, DEV_ALL_NEG_INF, DEV_BAD_TEMPERATURE = 16, 32, 64, 128
 (K_SCHEDULE, K_OFFSETS, K_STREAM, K_DECIDE, K_RESIDUAL, K_FINALIZE, K_GREEDY_STREAM, K_GREEDY_DECIDE,
- K_ROW_SCALE, K_MARKOV_GEMM, K_MARKOV_DRAW, K_TRUNCATE, K_VERIFY_FUSED, K_GREEDY_FUSED, K_COUNT) = range(15)
+ K_ROW_SCALE, K_MARKOV_GEMM, K_MARKOV_DRAW, K_TRUNCATE, K_COUNT) = range(13)
 
 EXPORTS = [
     "dspark_profile_create", "dspark_profile_destroy", "dspark_profile_table",

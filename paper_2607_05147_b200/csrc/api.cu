@@ -187,8 +187,7 @@ const char* dspark_kernel_name(int id)
 {
     static const char* names[DSPARK_K_COUNT] = {
         "schedule", "build_offsets", "stream_stats", "decide", "residual_stream", "finalize",
-        "greedy_stream", "greedy_decide", "row_scale", "markov_gemm", "markov_draw", "truncate",
-        "verify_fused", "greedy_fused"};
+        "greedy_stream", "greedy_decide", "row_scale", "markov_gemm", "markov_draw", "truncate"};
     return (id >= 0 && id < DSPARK_K_COUNT) ? names[id] : "?";
 }
 

@@ -944,49 +944,6 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     return DSPARK_OK;
 }
 
-// Pointers of the single-launch sampling verifier inside the general workspace.
-static void bind_fused(FusedParams& F, const VerifyParams& P, void* workspace)
-{
-    const Workspace w = workspace_layout(P.R, P.n_rows_cap, P.V);
-    unsigned char* ws = (unsigned char*)workspace;
-    F.P = P;
-    F.gbase_g = P.R > kGbaseSmemMaxR ? (unsigned int*)(ws + w.gbase) : nullptr;
-    F.pos_ticket = (int*)(ws + w.pos_ticket);
-    F.req_ticket = (int*)(ws + w.req_ticket);
-    F.resid_ticket = (int*)(ws + w.resid_ticket);
-    F.pos = (PosRec*)(ws + w.pos);
-    F.xtok = (float*)(ws + w.xtok);
-    F.tasks = (FusedTask*)(ws + w.tasks);
-    F.stream_cap = 2 * P.n_rows_cap;
-}
-
-// Greedy verification needs only the header, the per-block (max, argmax) entries, tickets and per-row outcomes.
-static int greedy_params(FusedParams& F, const void* target, int dtype, int64_t tstride, int V,
-                         const int32_t* row_offsets, const int32_t* draft_tokens, int R, int n_rows,
-                         int32_t* accepted_len, int32_t* out_tokens, int32_t* dev_status,
-                         void* scratch, size_t scratch_bytes)
-{
-    VerifyParams P;
-    int rc = fill_common(P, target, nullptr, dtype, tstride, 0, V, row_offsets, nullptr, draft_tokens, R, n_rows,
-                         accepted_len, out_tokens);
-    if (rc != DSPARK_OK) return rc;
-    const GreedyWorkspace w = greedy_workspace_layout(R, n_rows, V, P.elem);
-    if (!scratch || scratch_bytes < w.total) return DSPARK_ERR_WORKSPACE;
-    if (((uintptr_t)scratch & 255u) != 0) return DSPARK_ERR_ALIGNMENT;
-    unsigned char* ws = (unsigned char*)scratch;
-    P.counters = (int*)(ws + w.counters);
-    P.dev_status = dev_status ? dev_status : P.counters + 1;
-    P.stats_t = (float2*)(ws + w.stats);
-    F = FusedParams{};
-    F.P = P;
-    F.gbase_g = R > kGbaseSmemMaxR ? (unsigned int*)(ws + w.gbase) : nullptr;
-    F.pos_ticket = (int*)(ws + w.pos_ticket);
-    F.req_ticket = (int*)(ws + w.req_ticket);
-    F.pos = (PosRec*)(ws + w.rec);
-    F.stream_cap = n_rows;
-    return DSPARK_OK;
-}
-
 static long long pieces(int nblk) { return (nblk + kConsumerWarps - 1) / kConsumerWarps; }
 
 }  // namespace dspark
@@ -1008,27 +965,26 @@ int dspark_set_stream_path(int path)
     return DSPARK_OK;
 }
 
-// Greedy verification on a scratch region laid out by greedy_workspace_layout (a caller workspace or the
-// built-in array of dspark_verify_greedy_static).
+// Greedy verification on a scratch region laid out by greedy_workspace_layout (the front of a caller workspace,
+// or the built-in array of dspark_verify_greedy_static).
 static int greedy_launch(const void* target_logits, int dtype, int64_t target_row_stride, int V,
                          const int32_t* row_offsets, const int32_t* draft_tokens, int R, int n_rows,
                          int32_t* accepted_len, int32_t* out_tokens, int32_t* dev_status,
                          void* scratch, size_t scratch_bytes, void* stream)
 {
-    FusedParams F;
-    int rc = greedy_params(F, target_logits, dtype, target_row_stride, V, row_offsets, draft_tokens, R, n_rows,
-                           accepted_len, out_tokens, dev_status, scratch, scratch_bytes);
+    VerifyParams P;
+    int rc = fill_common(P, target_logits, nullptr, dtype, target_row_stride, 0, V, row_offsets, nullptr, draft_tokens, R, n_rows,
+                         accepted_len, out_tokens);
     if (rc != DSPARK_OK) return rc;
-    const VerifyParams& P = F.P;
-    cudaStream_t s = (cudaStream_t)stream;
-    const int path = g_stream_path.load(std::memory_order_relaxed);
-    const bool bulk = path != 1 && aligned16(P.target, P.tstride_bytes, P.row_bytes);
-    if (bulk && path == 0) {
-        // one launch: argmax statistics, row argmax and first mismatch
-        KernelTimerScope timer(DSPARK_K_GREEDY_FUSED, s);
-        return fused_verify_launch(F, true, (long long)n_rows * pieces(P.nblk), s);
-    }
+    const GreedyWorkspace w = greedy_workspace_layout(n_rows, V, P.elem);
+    if (!scratch || scratch_bytes < w.total) return DSPARK_ERR_WORKSPACE;
+    if (((uintptr_t)scratch & 255u) != 0) return DSPARK_ERR_ALIGNMENT;
+    P.counters = (int*)((unsigned char*)scratch + w.counters);
+    P.dev_status = dev_status ? dev_status : P.counters + 1;
+    P.stats_t = (float2*)((unsigned char*)scratch + w.stats);
     if (!ensure_attrs()) return launch_status();
+    cudaStream_t s = (cudaStream_t)stream;
+    const bool bulk = g_stream_path.load(std::memory_order_relaxed) != 1 && aligned16(P.target, P.tstride_bytes, P.row_bytes);
     {
         KernelTimerScope timer(DSPARK_K_GREEDY_STREAM, s);
         launch_stream_dtype<kModeGreedy>(P, bulk, (long long)n_rows * pieces(P.nblk), s);
@@ -1082,13 +1038,6 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
     const int path = g_stream_path.load(std::memory_order_relaxed);
     const bool bulk = path != 1 && aligned16(P.target, P.tstride_bytes, P.row_bytes) &&
                       aligned16(P.draft, P.dstride_bytes, P.row_bytes);
-    if (bulk && path == 0 && !truncate && n_rows <= (1 << 29)) {
-        // one launch: statistics, accept tests, residual units and every draw
-        FusedParams F;
-        bind_fused(F, P, workspace);
-        KernelTimerScope timer(DSPARK_K_VERIFY_FUSED, s);
-        return fused_verify_launch(F, false, (2ll * n_rows - R) * pieces(P.nblk), s);
-    }
     if (!ensure_attrs()) return launch_status();
     if (req_temp) {
         KernelTimerScope timer(DSPARK_K_ROW_SCALE, s);
@@ -1180,7 +1129,7 @@ size_t dspark_verify_greedy_static_capacity(void) { return kStaticScratchBytes; 
 size_t dspark_verify_greedy_static_bytes(int R, int n_rows, int V, int dtype)
 {
     if (R < 1 || n_rows < R || V < 1 || (dtype != DSPARK_F32 && dtype != DSPARK_BF16)) return 0;
-    return greedy_workspace_layout(R, n_rows, V, dtype == DSPARK_BF16 ? 2 : 4).total;
+    return greedy_workspace_layout(n_rows, V, dtype == DSPARK_BF16 ? 2 : 4).total;
 }
 
 int dspark_verify_greedy_static(const void* target_logits, int dtype, int64_t target_row_stride, int V,

@@ -1,5 +1,4 @@
-// Device-side building blocks of the verifier kernels (verify.cu: the staged passes, verify_fused.cu: the
-// single-launch verifier): batch parameters, per-block statistics / argmax / residual arithmetic, the
+// Device-side building blocks of the verifier kernels (verify.cu): batch parameters, per-block statistics / argmax / residual arithmetic, the
 // combination of block statistics into row statistics, and the two-level inverse CDF.
 #pragma once
 
@@ -720,52 +719,9 @@ __device__ __forceinline__ int level2_block(const unsigned char* trow, const uns
 }
 
 
-// ---------------------------------------------------------------------------------------
-// Single-launch verifier (verify_fused.cu): records and parameters
-// ---------------------------------------------------------------------------------------
-constexpr int kPosRejected = 1, kPosBad = 2;
-
-struct __align__(16) PosRec {        // outcome of one position (sampling), written by the warp that completes it
-    float cp, inv_zp, cq, inv_zq;    // row references (log2 domain) and 1 / row sums of the target / draft row
-    int32_t flags;                   // kPosRejected, kPosBad
-    int32_t pad[3];
-};
-struct __align__(8) GreedyRec {      // outcome of one target row (greedy)
-    int32_t argmax;
-    int32_t all_neg_inf;
-};
-struct __align__(16) FusedTask {     // a rejected request published for the residual units of the same launch
-    ResidTask t;
-    int32_t sigma_t;                 // statistics row of the rejected position's target row (fallback draw from p)
-    int32_t ready;                   // 0 until the record is complete (written last, with release semantics)
-    int32_t pad[2];
-};
-
-// Ints of the 256-byte workspace header used by the single-launch verifier (cells 0..9 as in the staged passes:
-// [0] queued residual tasks, [1] dev_status stand-in, then the 64-bit unit counters and the launch tag).
-constexpr int kHdrDecided = 16;      // requests whose outcome is settled (dead ones are counted up front)
-constexpr int kHdrExit = 17;         // CTAs that have left the kernel
-constexpr int kHdrAbort = 18;        // nonzero: a bounded wait ran out somewhere, everybody leaves
-constexpr int kHdrTotalFit = 20;     // streams of the batch that fit the workspace (set by CTA 0)
-constexpr int kHdrDead = 21;         // requests without streams (bad offsets)
-constexpr int kGbaseSmemMaxR = 1536; // up to this many requests every CTA keeps the stream prefix in shared memory
-
-struct FusedParams {
-    VerifyParams P;
-    unsigned int* gbase_g;           // [R + 1] stream prefix in global memory (R > kGbaseSmemMaxR), else NULL
-    int* pos_ticket;                 // [stream capacity] blocks done of the position whose target stream this is
-    int* req_ticket;                 // [R] positions done
-    int* resid_ticket;               // [R] residual blocks done
-    PosRec* pos;                     // [stream capacity] (greedy: GreedyRec)
-    float* xtok;                     // [stream capacity] logit at the draft token, captured while the block is on chip
-    FusedTask* tasks;                // [R]
-    int stream_cap;                  // statistics rows available: 2 * n_rows capacity (greedy: n_rows capacity)
-};
-
 // Workspace of the verifiers (caller-provided, any content on entry), offsets in bytes.
 struct Workspace {
     size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, tau, trunc_rows, trunc_bins, trunc_flag;
-    size_t gbase, pos_ticket, req_ticket, resid_ticket, pos, xtok, tasks;       // single-launch verifier
     size_t total;
 };
 inline Workspace workspace_layout(int R, int n_rows, int V)
@@ -787,38 +743,23 @@ inline Workspace workspace_layout(int R, int n_rows, int V)
     w.trunc_rows = o; o += up((size_t)n_rows * sizeof(TruncRow));
     w.trunc_bins = o; o += up((size_t)n_rows * kHistBins * sizeof(unsigned int));
     w.trunc_flag = o; o += up((size_t)(n_rows + 1) * sizeof(int32_t));   // + the fallback's row counter
-    w.gbase = o;        o += up((size_t)(R + 1) * sizeof(unsigned int));
-    w.pos_ticket = o;   o += up((size_t)2 * n_rows * sizeof(int));
-    w.req_ticket = o;   o += up((size_t)R * sizeof(int));
-    w.resid_ticket = o; o += up((size_t)R * sizeof(int));
-    w.pos = o;          o += up((size_t)2 * n_rows * sizeof(PosRec));
-    w.xtok = o;         o += up((size_t)2 * n_rows * sizeof(float));
-    w.tasks = o;        o += up((size_t)R * sizeof(FusedTask));
     w.total = o;
     return w;
 }
 
-// Scratch of the single-launch greedy verifier alone (what dspark_verify_greedy_static must fit into its array):
-// header, per-block (max, argmax) of every target row, tickets, per-row outcomes, stream prefix.
-struct GreedyWorkspace { size_t counters, stats, gbase, pos_ticket, req_ticket, rec, total; };
-inline GreedyWorkspace greedy_workspace_layout(int R, int n_rows, int V, int elem)
+// Scratch of greedy verification alone (what dspark_verify_greedy_static must fit into its array): the header
+// and the per-block (max, argmax) of every target row.
+struct GreedyWorkspace { size_t counters, stats, total; };
+inline GreedyWorkspace greedy_workspace_layout(int n_rows, int V, int elem)
 {
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
     const size_t nblk = (size_t)blocks_per_row(V, elem, kStatBlockBytes);
     GreedyWorkspace w;
     size_t o = 0;
-    w.counters = o;   o += up(64 * sizeof(int));
-    w.stats = o;      o += up((size_t)n_rows * nblk * sizeof(float2));
-    w.gbase = o;      o += up((size_t)(R + 1) * sizeof(unsigned int));
-    w.pos_ticket = o; o += up((size_t)n_rows * sizeof(int));
-    w.req_ticket = o; o += up((size_t)R * sizeof(int));
-    w.rec = o;        o += up((size_t)n_rows * sizeof(GreedyRec));
+    w.counters = o; o += up(64 * sizeof(int));
+    w.stats = o;    o += up((size_t)n_rows * nblk * sizeof(float2));
     w.total = o;
     return w;
 }
-
-// Launches the single-launch verifier (sampling: statistics, accept tests, residual units and all draws;
-// greedy: argmax and first mismatch) on rows that satisfy the 16-byte rules of the bulk copy.
-int fused_verify_launch(const FusedParams& F, bool greedy, long long max_units, cudaStream_t stream);
 
 }  // namespace dspark
