@@ -222,8 +222,10 @@ class VerifyResult:
     p_tok: np.ndarray
     q_tok: np.ndarray
     accept_margin: np.ndarray
-    token_margin: np.ndarray
+    token_margin: np.ndarray          # per request: distance of the draw to the nearer CDF boundary of the distribution drawn from
     status: np.ndarray
+    token_margin_abs: np.ndarray = None   # the same distance in probability units (residual draws: times W)
+    resid_mass: np.ndarray = None         # W = sum max(0, p - q) of a residual draw, NaN for a draw from p
 
 
 def verify(target, draft, row_offsets, draft_tokens, temperature: float, seed: int,
@@ -244,15 +246,17 @@ def verify(target, draft, row_offsets, draft_tokens, temperature: float, seed: i
     q = np.full(n_rows, np.nan)
     am = np.full(n_rows, np.nan)
     tm = np.full(R, np.nan)
+    tma = np.full(R, np.nan)
+    rw = np.full(R, np.nan)
     st = np.zeros(R, dtype=np.int32)
     temps = None if temperatures is None else np.ascontiguousarray(temperatures, dtype=np.float32)
     rc = lib().orc_verify(_p(t), _p(d), C.c_int(_dtype_code(t)), C.c_int64(ts), C.c_int64(ds),
                           C.c_int(t.shape[1]), _p(ro), _p(drs), _p(dt), C.c_int(R),
                           C.c_double(temperature), _p(temps), C.c_uint64(seed), C.c_int(int(eval_all)),
-                          C.c_int(n_threads), _p(acc), _p(out), _p(p), _p(q), _p(am), _p(tm), _p(st))
+                          C.c_int(n_threads), _p(acc), _p(out), _p(p), _p(q), _p(am), _p(tm), _p(tma), _p(rw), _p(st))
     if rc != 0:
         raise ValueError("orc_verify rejected its arguments")
-    return VerifyResult(acc, out, p, q, am, tm, st)
+    return VerifyResult(acc, out, p, q, am, tm, st, tma, rw)
 
 
 def accept_rate(target, draft, row_offsets, temperature: float, draft_row_start=None):

@@ -481,6 +481,7 @@ typedef struct {
     int R; double T; const float* temps; uint64_t seed; int eval_all;
     int32_t* accepted_len; int32_t* out_tokens;
     double* p_tok; double* q_tok; double* accept_margin; double* token_margin;
+    double* token_margin_abs; double* resid_mass;
     int32_t* status;
     int r_begin, r_end;
 } verify_job_t;
@@ -489,6 +490,8 @@ static void verify_request(const verify_job_t* J, int r)
 {
     int32_t lo = J->row_offsets[r], hi = J->row_offsets[r + 1];
     J->token_margin[r] = NAN;
+    if (J->token_margin_abs) J->token_margin_abs[r] = NAN;
+    if (J->resid_mass) J->resid_mass[r] = NAN;
     if (lo < 0 || hi - lo < 1) { J->status[r] = ORC_ST_BAD_OFFSETS; J->accepted_len[r] = 0; return; }
     int32_t len = hi - lo - 1;
     int64_t drow0 = J->draft_row_start ? J->draft_row_start[r] : (int64_t)lo - (int64_t)r;
@@ -535,7 +538,7 @@ static void verify_request(const verify_job_t* J, int r)
     float ua, ur;
     orc_uniforms(J->seed, (uint32_t)r, (uint32_t)n, &ua, &ur);
     int32_t tok = -1;
-    double margin = 0.0;
+    double margin = 0.0, margin_abs = 0.0, resid_W = NAN;
     double mp, Zp;
     if (row_softmax_stats(J->target, J->dtype, lo + n, J->tstride, J->V, T, &mp, &Zp)) {
         J->status[r] = ORC_ST_BAD_ROW; J->accepted_len[r] = 0; return;
@@ -566,25 +569,31 @@ static void verify_request(const verify_job_t* J, int r)
                 last_pos = v;
                 if (cum > thr) {
                     double d0 = thr - prev, d1 = cum - thr;
-                    /* in probability units, like the margin of a draw from p: the fp32 tolerance on p(v) and
-                     * q(v) bounds the running sum of max(0, p - q) absolutely, whatever its total W is */
-                    margin = d0 < d1 ? d0 : d1;
+                    /* distance of u' W to the nearer end of the token's interval of the running sum: kept both in
+                     * probability units and as a fraction of the residual mass W (the distance on the CDF of the
+                     * distribution the token is drawn from) */
+                    margin_abs = d0 < d1 ? d0 : d1;
+                    margin = margin_abs / W;
                     tok = v;
                     break;
                 }
             }
-            if (tok < 0) { tok = last_pos; margin = 0.0; }
+            if (tok < 0) { tok = last_pos; margin = 0.0; margin_abs = 0.0; }
             resampled = 1;
+            resid_W = W;
         }
     }
     if (!resampled) {
         /* bonus token from p of row n (also the fallback when the residual is empty) */
         tok = sample_from_p(J->target, J->dtype, lo + n, J->tstride, J->V, T, mp, Zp, (double)ur, &margin);
+        margin_abs = margin;       /* p sums to one */
     }
     for (int32_t j = 0; j < n; ++j) J->out_tokens[lo + j] = J->draft_tokens[lo + j];
     J->out_tokens[lo + n] = tok;
     J->accepted_len[r] = n;
     J->token_margin[r] = margin;
+    if (J->token_margin_abs) J->token_margin_abs[r] = margin_abs;
+    if (J->resid_mass) J->resid_mass[r] = resid_W;
     J->status[r] = st;
 }
 
@@ -608,7 +617,7 @@ int orc_verify(const void* target, const void* draft, int dtype,
                uint64_t seed, int eval_all, int n_threads,
                int32_t* accepted_len, int32_t* out_tokens,
                double* p_tok, double* q_tok, double* accept_margin, double* token_margin,
-               int32_t* status)
+               double* token_margin_abs, double* resid_mass, int32_t* status)
 {
     if (R <= 0 || V <= 0) return -1;
     if (!temperatures && (!(temperature > 0.0) || !isfinite(temperature))) return -1;
@@ -618,7 +627,7 @@ int orc_verify(const void* target, const void* draft, int dtype,
     verify_job_t base = { target, draft, dtype, target_row_stride, draft_row_stride, V,
                           row_offsets, draft_row_start, draft_tokens, R, temperature, temperatures, seed, eval_all,
                           accepted_len, out_tokens, p_tok, q_tok, accept_margin, token_margin,
-                          status, 0, R };
+                          token_margin_abs, resid_mass, status, 0, R };
     if (n_threads == 1) { verify_worker(&base); return 0; }
     pthread_t th[256];
     verify_job_t jobs[256];

@@ -13,6 +13,23 @@ from paper_2607_05147_b200 import workloads as W
 
 P_REL_TOL = 1e-5        # p(x), q(x): relative agreement with the fp64 oracle
 MARGIN_TOL = 1e-6       # a decision may differ only if the oracle's margin is below this
+# A residual draw is a draw from max(0, p - q) / W.  Its margin is measured on that CDF (normalised), as for
+# every other draw -- except where W itself is below what fp32 resolves: p(v) and q(v) are fp32 numbers with
+# about 1e-7 relative error, so the running sum of max(0, p - q) carries an ABSOLUTE error of about 1e-7
+# whatever W is, and for W < 1e-3 a normalised 1e-6 would ask for 1e-9 absolute.  There (and only there) the
+# margin is taken in probability units.
+SMALL_RESIDUAL_MASS = 1e-3
+MISMATCH_COUNTS = {"accept": 0, "token_normalised": 0, "token_small_mass": 0}   # running totals, printed by the config tests
+
+
+def token_mismatch_allowed(o, r):
+    """Which rule (if any) allows the emitted token of request r to differ from the oracle's."""
+    if o.token_margin[r] < MARGIN_TOL:
+        return "token_normalised"
+    w = o.resid_mass[r]
+    if w == w and w < SMALL_RESIDUAL_MASS and o.token_margin_abs[r] < MARGIN_TOL:
+        return "token_small_mass"
+    return None
 THREADS = max(1, min(32, os.cpu_count() or 1))
 
 
@@ -126,11 +143,15 @@ def compare_sampling(g: dict, o, row_offsets: np.ndarray, check_probs=True):
             j = min(ng, no)
             assert o.accept_margin[lo + j] < MARGIN_TOL, (r, j, ng, no, o.accept_margin[lo + j])
             mismatches += 1
+            MISMATCH_COUNTS["accept"] += 1
             continue
         if not (g["out"][lo:hi] == o.out_tokens[lo:hi]).all():
             assert (g["out"][lo:lo + no] == o.out_tokens[lo:lo + no]).all()
             assert (g["out"][lo + no + 1:hi] == -1).all()
-            assert o.token_margin[r] < MARGIN_TOL, (r, no, g["out"][lo + no], o.out_tokens[lo + no], o.token_margin[r])
+            rule = token_mismatch_allowed(o, r)
+            assert rule is not None, (r, no, g["out"][lo + no], o.out_tokens[lo + no], o.token_margin[r],
+                                      o.token_margin_abs[r], o.resid_mass[r])
+            MISMATCH_COUNTS[rule] += 1
             mismatches += 1
     if check_probs and g["p"] is not None:
         have = ~np.isnan(o.p_tok[:n_rows])

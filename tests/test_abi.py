@@ -46,6 +46,33 @@ def test_uniforms_match_oracle_bit_for_bit():
                 assert B.dspark_uniforms(seed, r, j) == oracle.uniforms(seed, r, j)
 
 
+def test_uniforms_match_oracle_on_a_million_counters():
+    # two independent Philox4x32-10 implementations (the library's and the oracle's), 10^6 (seed, request, position)
+    # counters: low and high key words, requests and positions across several powers of two
+    import ctypes as C
+    import numpy as np
+    import oracle
+    L, O = B.lib(), oracle.lib()
+    rng = np.random.default_rng(123)
+    seeds = [0, 1, 0xFFFFFFFF, 0x100000000, 0xDEADBEEFCAFEF00D] + [int(x) for x in rng.integers(0, 2**63, size=95, dtype=np.uint64)]
+    reqs = [0, 1, 2, 255, 256, 65535, 65536, 2**31 - 1, 2**32 - 1] + [int(x) for x in rng.integers(0, 2**32, size=91, dtype=np.uint64)]
+    poss = [0, 1, 2, 3, 31, 32, 4095, 2**32 - 1] + [int(x) for x in rng.integers(0, 2**20, size=92, dtype=np.uint64)]
+    a, b, c, d = C.c_float(), C.c_float(), C.c_float(), C.c_float()
+    n = 0
+    for seed in seeds:
+        s64 = C.c_uint64(seed)
+        for r in reqs:
+            r32 = C.c_uint32(r)
+            for j in poss:
+                j32 = C.c_uint32(j)
+                L.dspark_uniforms(s64, r32, j32, C.byref(a), C.byref(b))
+                O.orc_uniforms(s64, r32, j32, C.byref(c), C.byref(d))
+                assert a.value == c.value and b.value == d.value, (seed, r, j)
+                assert 0.0 <= a.value < 1.0 and 0.0 <= b.value < 1.0
+                n += 1
+    assert n == 10**6
+
+
 def test_cpu_tensors_are_refused():
     import torch
     with pytest.raises(B.DsparkError):

@@ -17,7 +17,7 @@ def _report(name, batch, g, mism):
     lens = batch.meta["lengths"].cpu().numpy()
     print(f"[{name}] requests={batch.R} rows={batch.n_rows} mean_len={lens.mean():.2f} "
           f"mean_accepted={g['acc'].mean():.2f} rejected={(g['acc'] < lens).mean():.2f} "
-          f"boundary_mismatches={mism} ({mism / batch.R:.2e} per request)")
+          f"boundary_mismatches={mism} ({mism / batch.R:.2e} per request); running totals by rule: {H.MISMATCH_COUNTS}")
 
 
 def test_config_2_reduced():

@@ -181,7 +181,7 @@ def test_config_3_full_size_with_truncation():
             continue
         if not (g["out"][lo:hi] == o.out_tokens[lo:hi]).all():
             assert (g["out"][lo:lo + no] == o.out_tokens[lo:lo + no]).all()
-            assert o.token_margin[r] < H.MARGIN_TOL, (r, g["out"][lo + no], o.out_tokens[lo + no], o.token_margin[r])
+            assert H.token_mismatch_allowed(o, r), (r, g["out"][lo + no], o.out_tokens[lo + no], o.token_margin[r])
             mism += 1
     print(f"[verify_truncated] cfg3: {b.n_rows} rows, mean accepted {g['acc'].mean():.2f}, "
           f"{len(near_req)} requests skipped (top-p decision on its boundary), {mism} boundary mismatches")

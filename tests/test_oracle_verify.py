@@ -262,12 +262,17 @@ def test_inverse_cdf_against_cumsum_searchsorted():
             w = np.maximum(special.softmax(x[2 * r].astype(np.float64)) - special.softmax(y[r].astype(np.float64)), 0)
             cdf = np.cumsum(w)
             want = int(np.searchsorted(cdf, ur * cdf[-1], side="right"))
-            if res.token_margin[r] > 1e-9:
+            # margins against an independent statement: the CDF of the residual distribution itself,
+            # cumsum(max(0, p - q) / W); the absolute margin is that distance times W
+            W = cdf[-1]
+            ncdf = np.cumsum(w / W)
+            prev_n = ncdf[want - 1] if want else 0.0
+            norm = min(ur - prev_n, ncdf[want] - ur)
+            if norm > 1e-9:
                 assert res.out_tokens[2 * r] == want
-                # the margin is the distance of u' W to the nearer end of the chosen token's interval of the
-                # running sum, in probability units (not divided by W)
-                thr, prev = ur * cdf[-1], (cdf[want - 1] if want else 0.0)
-                assert abs(res.token_margin[r] - min(thr - prev, cdf[want] - thr)) < 1e-12
+                assert abs(res.token_margin[r] - norm) < 1e-9
+                assert abs(res.token_margin_abs[r] - norm * W) < 1e-9 * W + 1e-15
+                assert abs(res.resid_mass[r] - W) < 1e-12
     assert n_rej > 50
 
 
@@ -355,3 +360,35 @@ def test_accept_rate_label(golden):
     res = oracle.verify(target, draft, ro, toks, 1.0, seed=77, n_threads=4)
     c, _ = oracle.accept_rate(target[:2], draft[:1], [0, 2], 1.0)
     assert abs(res.accepted_len.mean() - c[0]) < 4 * np.sqrt(c[0] * (1 - c[0]) / n)
+
+
+def test_threaded_greedy_oracle_equals_the_sequential_one():
+    # the threaded variant (what the benchmark times as the CPU baseline) against the sequential one on a ragged
+    # batch with ties, a token out of range and a row without any element above -inf
+    rng = np.random.default_rng(77)
+    V = 513
+    lengths = rng.integers(0, 7, size=37)
+    ro = np.concatenate([[0], np.cumsum(lengths + 1)]).astype(np.int32)
+    n_rows = int(ro[-1])
+    x = np.round(rng.normal(0, 2, size=(n_rows, V))).astype(np.float32)      # rounded: many exact ties
+    x[int(ro[2]), :] = -np.inf                                               # first row of a request: always looked at
+    x[9, 100:] = -np.inf
+    toks = np.argmax(x, axis=1).astype(np.int32)
+    flip = rng.random(n_rows) < 0.3
+    toks[flip] = rng.integers(0, V, size=int(flip.sum()))
+    bad_req = int(np.nonzero(lengths >= 1)[0][3])
+    toks[int(ro[bad_req])] = V + 3                                           # a draft token outside the vocabulary
+    want = oracle.verify_greedy(x, ro, toks)
+    assert want.status[bad_req] & oracle.ST_BAD_TOKEN and (want.accepted_len > 0).any()
+    assert (want.status & oracle.ST_ALL_NEG_INF).any()
+    for threads in (1, 3, 8, 64):
+        acc, out, st = oracle.verify_greedy_mt(x, ro, toks, threads)
+        np.testing.assert_array_equal(acc, want.accepted_len)
+        np.testing.assert_array_equal(out, want.out_tokens)
+        np.testing.assert_array_equal(st, want.status)
+    xb = (x.view(np.uint32) >> 16).astype(np.uint16)                         # the same rows as bf16 patterns
+    wb = oracle.verify_greedy(xb, ro, toks)
+    acc, out, st = oracle.verify_greedy_mt(xb, ro, toks, 5)
+    np.testing.assert_array_equal(acc, wb.accepted_len)
+    np.testing.assert_array_equal(out, wb.out_tokens)
+    np.testing.assert_array_equal(st, wb.status)
