@@ -495,14 +495,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--all-workloads", action="store_true", help="also time the other V=129280 configurations")
     ap.add_argument("--async-topk", action="store_true",
-                    help="schedule with dspark_schedule_async (capacity from two steps earlier, Section 4.2)")
+                    help="schedule with dspark_schedule_async (capacity from two steps earlier, Section 5.2)")
     ap.add_argument("--per-request-temperature", action="store_true",
                     help="verify with dspark_verify_per_request (a device array of R temperatures)")
     ap.add_argument("--top-k", type=int, default=0, help="verify against the top-k truncated target (every request)")
     ap.add_argument("--top-p", type=float, default=1.0, help="verify against the top-p truncated target (every request)")
     ap.add_argument("--overlap-schedule", action="store_true",
                     help="with --async-topk: schedule step t+1 on a second stream while step t is verified "
-                         "(the asynchronous scheduler is off the critical path, Section 4.2)")
+                         "(the asynchronous scheduler is off the critical path, Section 5.2)")
     ap.add_argument("--cuda-graph", action="store_true",
                     help="capture the step (schedule -> verify) in CUDA graphs and time their replay")
     ap.add_argument("--requests", type=int, default=0,

@@ -39,7 +39,8 @@ typedef enum {
     DSPARK_ERR_ALIGNMENT = 3,
     DSPARK_ERR_WORKSPACE = 4,
     DSPARK_ERR_CUDA = 5,
-    DSPARK_ERR_TIMEOUT = 6,
+    /* 6 is not used: no call waits for the device, so a device-side wait that runs out can only be
+     * reported through DSPARK_DEV_TIMEOUT in *dev_status */
     DSPARK_ERR_STATIC_LIMIT = 7
 } dspark_status_t;
 
@@ -47,8 +48,8 @@ typedef enum { DSPARK_F32 = 0, DSPARK_BF16 = 1 } dspark_dtype_t;
 
 typedef enum {
     DSPARK_SCHED_EARLY_STOP = 0, /* Algorithm 1 as printed: stop at the first non-improving admission */
-    DSPARK_SCHED_GLOBAL = 1,     /* Section 4.2: same path without the break, first maximiser wins */
-    DSPARK_SCHED_TOPK = 2        /* Section 4.2: admit the K most confident candidates (K from the caller) */
+    DSPARK_SCHED_GLOBAL = 1,     /* Section 5.2, scheduler in practice: same path without the break, first maximiser wins */
+    DSPARK_SCHED_TOPK = 2        /* Section 5.2: admit the K most confident candidates (K from the caller) */
 } dspark_sched_mode_t;
 
 /* Bits OR-ed into *dev_status (verifier) and into dspark_sched_info_t.status (scheduler). */
@@ -62,8 +63,8 @@ typedef enum {
 #define DSPARK_DEV_BAD_TEMPERATURE 128 /* a per-request temperature that is not a positive finite number */
 
 /* ------------------------------------------------------------------------------------
- * Engine throughput profile SPS(B), steps per second at B batch tokens (Section 3.2.2:
- * "profiled once during engine initialization and stored as a lightweight cost table").
+ * Engine throughput profile SPS(B), steps per second at B batch tokens: a table the engine measures
+ * once when it starts up and only looks up afterwards (Section 3.2.2).
  *
  * bp_tokens / bp_sps: host arrays of n_bp breakpoints, bp_tokens strictly increasing.
  * The library builds a dense fp64 device table SPS[0..max_tokens]: piecewise linear
@@ -92,7 +93,7 @@ typedef struct {
 /* ------------------------------------------------------------------------------------
  * dspark_schedule -- hardware-aware prefix scheduler (Algorithm 1; a, B, tau, Theta as
  * defined in Section 3.2.2; no-break and top-K variants and the capacity limit from
- * Section 4.2).
+ * Section 5.2, "Hardware-Aware Prefix Scheduler in Practice").
  *
  * Computes survival products a_{r,j} = prod_{i<=j} c_{r,i} (fp32, left to right), orders
  * all candidates with a > 0 by (a descending, position ascending, request ascending),
@@ -123,7 +124,7 @@ int dspark_schedule(const dspark_profile_t* prof, const float* conf, const int32
                     void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------
- * dspark_schedule_async -- the scheduler as deployed (Section 4.2): the engine must know the
+ * dspark_schedule_async -- the scheduler as deployed (Section 5.2): the engine must know the
  * batch size of the next step before the current one ends, so the capacity K (how many draft
  * tokens are admitted in total) is taken from the unconstrained, no-break search over the
  * confidences of TWO STEPS EARLIER, while the candidates themselves are ranked by their current
@@ -145,7 +146,8 @@ int dspark_schedule_async(const dspark_profile_t* prof, const float* conf, const
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /* row_offsets[0..R] = exclusive scan of (lengths[r] + 1): the flat ragged layout of
- * Section 4.3 (all verified tokens of all requests flattened).  Device in, device out. */
+ * Section 5.3, "High-Throughput and Low-Latency Inference" (all verified tokens of all requests flattened).
+ * Device in, device out. */
 int dspark_build_offsets(const int32_t* lengths, int R, int32_t* row_offsets, void* stream);
 
 /* ------------------------------------------------------------------------------------
@@ -348,7 +350,7 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
 
 /* ------------------------------------------------------------------------------------
  * dspark_truncate_target -- top-k / top-p truncation of the target distribution, per request (Section 4.1
- * evaluates with the models' recommended sampling parameters; the paper states no rule of its own).
+ * evaluates every model with its own suggested sampling settings; the paper states no rule of its own).
  * The logits of the excluded tokens of every target row are set to -inf IN PLACE, so that softmax
  * renormalises over the kept set and dspark_verify / dspark_verify_per_request, run afterwards on the same
  * rows, are lossless with respect to the truncated target distribution.
@@ -451,6 +453,15 @@ int dspark_ktimer_read(dspark_ktimer_t* t, int kernel_id, float* total_ms, int* 
  * separate passes with direct loads, 2 = separate passes with bulk copies.  Results are the same
  * up to fp32 summation order.  Process-wide (an atomic); the paper has no counterpart. */
 int dspark_set_stream_path(int path);
+
+/* Diagnostic: how many polls the streamed passes of the verifiers spend on an entry wait (a consumer warp
+ * waiting for its data, the producer waiting for a free stage or for the launch tag) before they give up,
+ * set DSPARK_DEV_TIMEOUT in *dev_status and leave.  0 restores the default (about 4 million polls, on the
+ * order of a second); a wait gives up after polls - 1 unsuccessful polls, so 1 makes every such wait run
+ * out at once.  That is how the tests reach the give-up path without hanging anything: a kernel that gives
+ * up still waits, with the long default bound, for the bulk copies it has already issued before it leaves,
+ * and its outputs are unspecified.  Per device (the current one), synchronous; the paper has no counterpart. */
+int dspark_set_wait_poll_limit(unsigned int polls);
 
 const char* dspark_status_string(int status);
 const char* dspark_kernel_name(int kernel_id);

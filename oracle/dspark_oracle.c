@@ -109,7 +109,7 @@ int orc_sps_table(const int32_t* bp_tokens, const double* bp_sps, int n_bp,
 
 /* ------------------------------------------------------------------------ */
 /* Scheduler (Algorithm 1; definitions of a, B, tau, Theta in Section 3.2.2; */
-/* no-break variant and capacity limit in Section 4.2).                      */
+/* no-break variant and capacity limit in Section 5.2).                      */
 /* ------------------------------------------------------------------------ */
 typedef struct {
     float a;
@@ -255,7 +255,7 @@ int orc_schedule(const float* conf, const int32_t* draft_len, int R, int gamma,
 }
 
 /*
- * Asynchronous scheduling (Section 4.2, "Hardware-Aware Prefix Scheduler in Practice").
+ * Asynchronous scheduling (Section 5.2, "Hardware-Aware Prefix Scheduler in Practice").
  * The capacity K used at step t is the admission count found by the unconstrained (no break)
  * search on the confidences of step t-2; the candidates admitted at step t are the K most
  * confident ones by the CURRENT survival products (dynamic top-K), still under the token cap.
@@ -874,8 +874,8 @@ int orc_sts_apply(const float* conf, int N, int gamma, const float* T, double* o
 
 /* ------------------------------------------------------------------------ */
 /* Top-k / top-p truncation of the target distribution (per-request sampling */
-/* parameters; the paper evaluates with "recommended sampling parameters",    */
-/* Section 4.1, and gives no rule of its own).  Readings:                     */
+/* parameters; the evaluation of Section 4.1 takes each model's suggested     */
+/* sampling settings and the paper gives no rule of its own).  Readings:     */
 /*  - the truncated distribution is obtained by setting the logits of the     */
 /*    excluded tokens to -inf, so that softmax renormalises over the kept set  */
 /*    S and the lossless verifier runs unchanged on the masked rows;           */

@@ -37,7 +37,7 @@ EXPORTS = [
     "dspark_truncate_target", "dspark_verify_truncated",
     "dspark_sts_workspace_bytes", "dspark_sts_calibrate", "dspark_sts_apply",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
-    "dspark_ktimer_read", "dspark_set_stream_path", "dspark_status_string", "dspark_kernel_name",
+    "dspark_ktimer_read", "dspark_set_stream_path", "dspark_set_wait_poll_limit", "dspark_status_string", "dspark_kernel_name",
     "dspark_version",
 ]
 
@@ -109,6 +109,7 @@ def lib() -> C.CDLL:
         L.dspark_ktimer_reset.argtypes = [vp]
         L.dspark_ktimer_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_int)]
         L.dspark_set_stream_path.argtypes = [i32]
+        L.dspark_set_wait_poll_limit.argtypes = [C.c_uint]
         L.dspark_status_string.argtypes = [i32]
         L.dspark_status_string.restype = C.c_char_p
         L.dspark_kernel_name.argtypes = [i32]
@@ -532,6 +533,11 @@ def dspark_uniforms(seed: int, request: int, position: int):
 
 def dspark_set_stream_path(path: int) -> None:
     _check(lib().dspark_set_stream_path(path), "dspark_set_stream_path")
+
+
+def dspark_set_wait_poll_limit(polls: int) -> None:
+    """Diagnostic: poll limit of the streamed passes' entry waits (0: default, 1: give up at once)."""
+    _check(lib().dspark_set_wait_poll_limit(polls), "dspark_set_wait_poll_limit")
 
 
 class KernelTimer:

@@ -177,7 +177,6 @@ const char* dspark_status_string(int s)
         case DSPARK_ERR_ALIGNMENT: return "misaligned buffer";
         case DSPARK_ERR_WORKSPACE: return "workspace too small";
         case DSPARK_ERR_CUDA: return "CUDA error";
-        case DSPARK_ERR_TIMEOUT: return "device wait timed out";
         case DSPARK_ERR_STATIC_LIMIT: return "batch exceeds the built-in scratch array";
         default: return "unknown status";
     }

@@ -74,9 +74,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait: false when the poll limit ran out.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit = kWaitPollLimit)
 {
-    for (uint32_t i = 0; i < kWaitPollLimit; ++i)
+    for (uint32_t i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -119,9 +119,9 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 // Waits (bounded) until a 64-bit cell in global memory holds `tag`: how the CTAs of a grid learn that CTA 0
 // has zeroed the grid's work counters.  The tag is unique per launch (next_launch_tag), so whatever an
 // earlier launch or the caller left in the cell cannot be mistaken for it.
-__device__ __forceinline__ bool wait_for_tag(const unsigned long long* cell, unsigned long long tag)
+__device__ __forceinline__ bool wait_for_tag(const unsigned long long* cell, unsigned long long tag, uint32_t limit = kWaitPollLimit)
 {
-    for (uint32_t i = 0; i < kWaitPollLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         unsigned long long v;
         asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(cell) : "memory");
         if (v == tag) return true;

@@ -67,9 +67,6 @@ struct MarkovParams {
     float2* stats;                            // workspace: per (row, vocabulary tile) statistics of the stored logits
     float scale2;                             // log2(e) / T
     int l2_hints;                             // 1: keep W2 in L2, stream the logits through it (small launches only)
-#ifdef DSPARK_MARKOV_TRACE
-    unsigned long long* trace;                // 64 clock stamps per CTA (development aid)
-#endif
 };
 
 // ---- one-time packing of W2 [256, V] into per-tile K-major blobs ---------------------------------
@@ -421,15 +418,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     tc_fence_after();
     // The packed W2 is a weight, not a result of the previous kernel on the stream: the producer starts
     // on it at once; every other role first waits for that kernel (gathered rows, base logits).
-#ifdef DSPARK_MARKOV_TRACE
-    unsigned long long* tr = P.trace + (size_t)blockIdx.x * 64;
-    auto stamp = [&](int slot) { if (slot < 64) tr[slot] = clock64(); };
-#else
-    auto stamp = [](int) {};
-#endif
-    if (tid == 32) stamp(0);
     if (warp != 0) pdl_wait();
-    if (tid == 32) stamp(1);
     const uint32_t tmem_base = s_tmem_base;
     const uint32_t tmem_a0 = tmem_base + 2 * kTileMN;       // this CTA's embedding tile: columns 256 .. 383
     volatile int* abort_flag = &s_abort;
@@ -449,13 +438,18 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             const uint64_t pol_keep = P.l2_hints ? l2_policy_evict_last() : l2_policy_evict_normal();
             bool told = false;
             if (my_tiles == 0) { mbar_arrive(&prefetch_issued); told = true; }
+            int issued = 0;
             for (int k = 0; k < my_tiles && !*abort_flag; ++k) {
                 const int bs = k & 1;
                 if (!mbar_wait_bounded(&b_empty[bs], ((uint32_t)(k >> 1) & 1u) ^ 1u)) { give_up(); break; }
                 mbar_arrive_expect_tx(&b_full[bs], kTileBytes);
                 bulk_g2s_hint(sB + bs * kTileBytes, P.W2p + (size_t)unit_ntile(k) * kTileBytes, kTileBytes, &b_full[bs], pol_keep);
-                if (k < 7) stamp(56 + k);
+                issued = k + 1;
                 if (k == 1 || k == my_tiles - 1) { if (!told) mbar_arrive(&prefetch_issued); told = true; }
+            }
+            if (*abort_flag) {
+                // somebody gave up: leave only after the copies already issued have landed (bounded)
+                for (int k = issued - 1; k >= 0 && k >= issued - 2; --k) mbar_wait_bounded(&b_full[k & 1], (uint32_t)(k >> 1) & 1u);
             }
         }
     } else if (warp == 1) {
@@ -467,7 +461,6 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                 bool ok = mbar_wait_bounded(&b_full[s], ph) && mbar_wait_bounded(&acc_empty[s], ph ^ 1u);
                 if (ok && k == 0) ok = mbar_wait_bounded(&a_full[0], 0u);            // resident from then on
                 if (!ok) { give_up(); break; }
-                if (k < 2) stamp(4 + k);
                 tc_fence_after();
                 const uint32_t b0 = smem_u32(sB + s * kTileBytes);
 #pragma unroll
@@ -476,7 +469,6 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                                  smem_desc_kmajor(b0 + ks * 2 * kChunkBytes), ks > 0 ? 1u : 0u);
                 umma_commit(&acc_full[s]);                  // the accumulator may be read
                 umma_commit(&b_empty[s]);                   // the W2 tile may be overwritten
-                stamp(8 + k);
             }
         }
     } else {
@@ -491,8 +483,10 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const bool leader = kTma && warp == 2 && lane == 0;
         const uint64_t pol_stream = P.l2_hints ? l2_policy_evict_first() : l2_policy_evict_normal();
+        int u_issued = 0;                                   // base-logit tiles requested so far (leader)
         auto issue_u_load = [&](int t) {
             const int nt = unit_ntile(t), mt = my_mt;
+            u_issued = t + 1;
             unsigned char* dst = sU + (t % kUBuffers) * kUTileBytes;
             mbar_arrive_expect_tx(&u_full[t % kUBuffers], kUTileBytes);
             tma_load_2d(dst, &map_u, nt * kTileMN, mt * kTileMN, &u_full[t % kUBuffers], pol_stream);
@@ -515,7 +509,6 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             embedding_quarter_row_to_tmem(src, tmem_a0 + lane_base + (uint32_t)(chunk * (kRank / 8)));
             __syncwarp();
             if (lane == 0) mbar_arrive(&a_full[0]);
-            if (lane == 0 && q == 2 && chunk == 0) stamp(2);
         }
         for (int t = 0; t < my_tiles && !*abort_flag; ++t) {
             const int nt = unit_ntile(t), mt = my_mt;
@@ -527,7 +520,6 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                 break;
             }
             tc_fence_after();
-            if (leader) stamp(24 + t);
             const uint32_t acc_addr = tmem_base + lane_base + (uint32_t)(s * kTileMN);
             // Statistics: every warp leaves the (m, s) of its 32 columns in two spare tensor-memory columns of
             // its lanes (four rotating slots of 8 columns from column 384).  The accumulator of tile t can
@@ -575,7 +567,6 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                         bulk_commit_group();
                         bulk_wait_group_read<1>();          // the store of tile t-1 has left its buffer
                         if (t + 2 < my_tiles) issue_u_load(t + 2);
-                        stamp(40 + t);
                     }
                 }
                 __syncwarp();
@@ -626,6 +617,12 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             }
         }
         if (leader) bulk_wait_group_read<0>();              // shared memory stays valid until the stores have read it
+        if (leader && *abort_flag) {
+            // somebody gave up: the base-logit loads already issued must land before this CTA leaves (bounded);
+            // loads are issued for tiles 0, 1 and then t + 2 after tile t
+            for (int t = 0; t < my_tiles && t < u_issued; ++t)
+                if (t + kUBuffers >= u_issued) mbar_wait_bounded(&u_full[t % kUBuffers], (uint32_t)(t / kUBuffers) & 1u);
+        }
     }
     // everyone meets here; the entries of the last two tiles are merged; then the allocating warp returns
     // the tensor memory
@@ -645,7 +642,6 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
         tc_fence_before();
     }
     __syncthreads();
-    if (tid == 32) stamp(63);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
@@ -838,15 +834,12 @@ static MarkovWs markov_layout(int R, int V)
     size_t o = 0;
     w.stats = o;  o += up((size_t)R * ((V + kTileMN - 1) / kTileMN) * sizeof(float2));
     w.trace = o;
-#ifdef DSPARK_MARKOV_TRACE
-    o += up(256 * 64 * 8);
-#endif
     w.total = o;
     return w;
 }
 
 static bool g_gemm_attr_set[64] = {};
-static int g_markov_path = 0;   // 0: tensor-map epilogue when the 16-byte rules hold, 1: always direct
+static std::atomic<int> g_markov_path{0};   // 0: tensor-map epilogue when the 16-byte rules hold, 1: always direct
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against the driver)
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -892,7 +885,7 @@ extern "C" {
 int dspark_markov_set_epilogue_path(int path)
 {
     if (path != 0 && path != 1) return DSPARK_ERR_INVALID_ARG;
-    g_markov_path = path;
+    g_markov_path.store(path, std::memory_order_relaxed);
     return DSPARK_OK;
 }
 
@@ -947,9 +940,6 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
     P.stats = (float2*)((unsigned char*)workspace + w.stats);
     P.l2_hints = 0;
     P.scale2 = stats_mode == 1 ? (float)(1.4426950408889634 / (double)temperature) : 0.f;
-#ifdef DSPARK_MARKOV_TRACE
-    P.trace = (unsigned long long*)((unsigned char*)workspace + w.trace);
-#endif
     if (params_out) *params_out = P;
 
     int dev = 0, sms = 0, l2_bytes = 0;
@@ -982,7 +972,7 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
         CUtensorMap map_u, map_out;
         memset(&map_u, 0, sizeof map_u);
         memset(&map_out, 0, sizeof map_out);
-        const bool tma = g_markov_path != 1 && make_tile_map(&map_u, G.U, G.R, V, P.u_stride_bytes) &&
+        const bool tma = g_markov_path.load(std::memory_order_relaxed) != 1 && make_tile_map(&map_u, G.U, G.R, V, P.u_stride_bytes) &&
                          make_tile_map(&map_out, G.out, G.R, V, P.out_stride_bytes);
         KernelTimerScope timer(DSPARK_K_MARKOV_GEMM, s);
         const int units = P.n_tiles * G.m_tiles, cap = sms - sms % G.m_tiles;     // a multiple of the row tiles

@@ -1,4 +1,4 @@
-// dspark_schedule: the hardware-aware prefix scheduler (Algorithm 1; Sections 3.2.2, 4.2).
+// dspark_schedule: the hardware-aware prefix scheduler (Algorithm 1; Sections 3.2.2 and 5.2).
 //
 // Algorithm 1 sorts all candidates (r, j) by survival probability and walks the sorted
 // list.  Here nothing is sorted: every request's survival products are already in
@@ -449,7 +449,7 @@ __device__ void sched_final_stage(const SchedParams& P)
     }
     __syncthreads();
     if (P.mode == kModeAsync) {
-        // Section 4.2: the admission count found on the current confidences becomes the capacity of
+        // Section 5.2: the admission count found on the current confidences becomes the capacity of
         // the step after next; this step admits the top K by current scores with the capacity that
         // was stored two steps ago.
         if (tid == 0) {

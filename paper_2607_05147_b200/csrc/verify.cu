@@ -1,5 +1,5 @@
 // dspark_verify / dspark_verify_greedy: the fused ragged-batch speculative verifier
-// (acceptance rule of Section 2.1; bonus token of Section 1; flat ragged rows of Section 4.3).
+// (acceptance rule of Section 2.1; bonus token of Section 1; flat ragged rows of Section 5.3).
 //
 // Pass structure (all on the caller's stream, no host round trip):
 //   stream   every target / draft row is read from HBM exactly once.  A row is cut into
@@ -24,6 +24,12 @@ namespace dspark {
 // ---------------------------------------------------------------------------------------
 // Streamed pass, bulk-copy pipeline: kStages x 32 KB of shared memory per CTA.
 // ---------------------------------------------------------------------------------------
+// Poll limit of the entry waits of the streamed passes (a consumer waiting for data, the producer waiting for a
+// free stage or for the launch tag).  dspark_set_wait_poll_limit shortens it for diagnostics; the producer's
+// wait for copies it has already issued always keeps the long bound, so that no copy can land in the shared
+// memory of a CTA that has left.
+__device__ uint32_t g_entry_poll_limit = kWaitPollLimit;
+
 template <int kElem, int kMode>
 __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyParams P)
 {
@@ -43,6 +49,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     __syncthreads();
     pdl_wait();                                  // everything below reads what earlier kernels wrote
 
+    const uint32_t entry_limit = g_entry_poll_limit;
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
     if (kMode != kModeResid && kMode != kModeHist && blockIdx.x == 0 && tid == 0) {
@@ -93,7 +100,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 }
             }
             if (*abort_flag) return false;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(&empty_bar[st], ph ^ 1u))) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(&empty_bar[st], ph ^ 1u, entry_limit))) {
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
                 return false;
             }
@@ -106,7 +113,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                     mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(bytes * M::kSrc));
                     bulk_g2s_hint(dst, src0, (uint32_t)bytes, &full_bar[st], pol_first);
                     if (M::kSrc == 2) bulk_g2s_hint(dst + M::kPieceBytes, src1, (uint32_t)bytes, &full_bar[st], pol_first);
-                    if (!counter_ready && !(counter_ready = wait_for_tag(unit_tag(P), P.launch_tag))) {
+                    if (!counter_ready && !(counter_ready = wait_for_tag(unit_tag(P), P.launch_tag, entry_limit))) {
                         atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT);
                         *abort_flag = 1;
                         mine = total;
@@ -137,7 +144,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
             const int st = it % kStages;
             const uint32_t ph = (uint32_t)(it / kStages) & 1u;
             if (*abort_flag) break;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(&full_bar[st], ph))) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(&full_bar[st], ph, entry_limit))) {
                 if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
                 break;
             }
@@ -956,6 +963,12 @@ size_t dspark_verify_workspace_bytes(int R, int n_rows, int V)
 {
     if (R < 1 || n_rows < R || V < 1) return 0;
     return workspace_layout(R, n_rows, V).total;
+}
+
+int dspark_set_wait_poll_limit(unsigned int polls)
+{
+    const uint32_t v = polls ? polls - 1u : kWaitPollLimit;     // 1: no poll at all, the wait gives up at once
+    return cudaMemcpyToSymbol(g_entry_poll_limit, &v, sizeof(v)) == cudaSuccess ? DSPARK_OK : launch_status();
 }
 
 int dspark_set_stream_path(int path)

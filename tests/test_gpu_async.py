@@ -1,4 +1,4 @@
-"""Asynchronous top-K scheduling (Section 4.2) on the GPU: device-resident state across steps,
+"""Asynchronous top-K scheduling (Section 5.2) on the GPU: device-resident state across steps,
 bit-exact against the oracle, and the schedule -> verify chain replayed from a CUDA graph."""
 import numpy as np
 import pytest

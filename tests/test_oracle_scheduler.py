@@ -215,7 +215,7 @@ def test_draft_len_and_confidence_sanitising():
 
 
 def test_async_topk_uses_the_capacity_of_two_steps_earlier():
-    # Section 4.2: K at step t comes from the no-break search on the confidences of step t-2,
+    # Section 5.2: K at step t comes from the no-break search on the confidences of step t-2,
     # the ranking from the current confidences.  Tiny batches: the capacity is checked against the
     # exhaustive optimum, the admitted set against an independent top-K by sorting.
     rng = np.random.default_rng(21)
