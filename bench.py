@@ -227,6 +227,14 @@ class Step:
                 B.dspark_schedule(self.wl["prof"], c, self.sched.budget_tokens, B.DSPARK_SCHED_EARLY_STOP,
                                   out_len=self.out_len, out_row_offsets=self.offsets, workspace=self.sws)
             offsets = self.offsets            # the verifier reads the schedule's offsets from device memory
+        self._verify(batch, offsets)
+
+    def verify(self, batch):
+        """The verifier call alone, on the offsets the last schedule left on the device."""
+        self._verify(batch, self.offsets if self.sched is not None else batch.row_offsets)
+
+    def _verify(self, batch, offsets):
+        B = self.B
         if self.wl["greedy"]:
             B.dspark_verify_greedy(batch.target, offsets, batch.draft_tokens, accepted_len=self.acc,
                                    out_tokens=self.out, dev_status=self.status, workspace=self.ws, n_rows=self.n_rows)
@@ -345,6 +353,34 @@ def host_copy(wl):
     wl["host"] = host
 
 
+def workload_config(wl, b0, n_rows, n_rejected, n_sets, stream_bytes):
+    """The `config` object of the JSON line: what the workload is, the same for both arms."""
+    return {"workload": wl["desc"], "name": wl["name"], "requests": b0.R, "rows_per_step": n_rows,
+            "draft_rows_per_step": b0.n_rows - b0.R, "rejected_requests": n_rejected,
+            "logit_dtype": str(b0.target.dtype).replace("torch.", ""),
+            "l2": f"inputs larger than L2: {n_sets} distinct batches rotated "
+                  f"({n_sets * stream_bytes / 1e6:.0f} MB of logits)",
+            "scheduler": ("async top-K, capacity from two steps earlier" if ASYNC_TOPK else "early stop")
+            if wl["sched"] is not None else None,
+            "temperature": "per request (device array)" if PER_REQUEST_T else "one per batch",
+            "truncation": None if TRUNCATE is None else f"top_k={TRUNCATE[0]}, top_p={TRUNCATE[1]} (dspark_verify_truncated)",
+            "launch": "CUDA graph replay" if CUDA_GRAPH else
+            ("stream launches, scheduler of step t+1 overlapped on a second stream" if OVERLAP else "stream launches"),
+            "parallelism": "replicas only (one engine per GPU, no collective)"}
+
+
+def oracle_rejected(wl, batch):
+    """Requests whose first rejection comes before the end of their block, by the oracle."""
+    import oracle
+    host = wl["host"]
+    if wl["greedy"]:
+        return 0
+    o = oracle.verify(host["target"], host["draft"], host["offsets"], host["tokens"], batch.temperature, batch.seed,
+                      eval_all=False, n_threads=os.cpu_count() or 1)
+    lens = host["offsets"][1:] - host["offsets"][:-1] - 1
+    return int((o.accepted_len < lens).sum())
+
+
 def run_reference(args, rank):
     """--impl reference: the CPU oracle, as it stands, on the machine's host cores."""
     from paper_2607_05147_b200 import replicas
@@ -352,30 +388,40 @@ def run_reference(args, rank):
         return                      # under torchrun only rank 0 runs and prints the reference arm
     import oracle
     oracle.build()
-    device = "cuda" if torch.cuda.is_available() else "cpu"     # only to draw the synthetic batch faster
-    wl = make_workload(args.workload, device, 0, 1, oracle_schedule=True)
-    host_copy(wl)
-    b = wl["batches"][0]
+    device = "cuda" if torch.cuda.is_available() else "cpu"     # only to draw the synthetic batches faster
+    wl = make_workload(args.workload, device, 0, None, oracle_schedule=True)
+    n_sets = len(wl["batches"])
+    hosts = []
+    for b in wl["batches"]:                                      # the same rotation of batches as the CUDA arm
+        wl["batches"] = [b]
+        host_copy(wl)
+        hosts.append(wl["host"])
+    b = b0 = wl["batches"][0]
+    wl["host"] = hosts[0]
     threads = os.cpu_count() or 1
+    n_rejected = oracle_rejected(wl, b0)
     t0 = time.perf_counter()
     oracle_step(wl, b, b.R, threads)
     t1 = time.perf_counter() - t0
     budget_s = 150.0
     frac = min(1.0, budget_s / max(1e-9, (args.steps + args.warmup) * t1))
     n_req = max(1, int(b.R * frac))
-    for _ in range(args.warmup):
+    for i in range(args.warmup):
+        wl["host"] = hosts[i % n_sets]
         oracle_step(wl, b, n_req, threads)
     t0 = time.perf_counter()
     rows = 0
-    for _ in range(args.steps):
+    for i in range(args.steps):
+        wl["host"] = hosts[i % n_sets]
         rows += oracle_step(wl, b, n_req, threads)
     dt = time.perf_counter() - t0
     value = rows / dt
+    stream_bytes, _ = algorithmic_bytes(b0, wl["greedy"], 0)
     sample = f"first {n_req} of {b.R} requests per step ({rows // max(1, args.steps)} rows), schedule over all requests"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": wl["desc"], "name": wl["name"]},
+            "data": "synthetic", "config": workload_config(wl, b0, b0.n_rows, n_rejected, n_sets, stream_bytes),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -453,7 +499,7 @@ def bench_markov(args, device, rank, world, dist, barrier):
     gemm_call_ms = ev0.elapsed_time(ev1) / args.steps
     (ms,) = replicas.max_over_ranks([ms], dist, device)
     if rank != 0:
-        return
+        return None
     peaks_file = os.path.join(ROOT, "MEASURED_PEAKS.json")
     peaks = json.load(open(peaks_file)) if os.path.exists(peaks_file) else {}
     peak = float(peaks.get("hbm_gbs", FALLBACK_HBM_GBS))
@@ -462,7 +508,7 @@ def bench_markov(args, device, rank, world, dist, barrier):
     gemm_ms = k["ms"] / args.steps              # one launch per group of 1024 rows
     achieved = gemm_bytes / (gemm_call_ms * 1e-3) / 1e9
     flops = 2.0 * ((R + 127) // 128 * 128) * 256 * ((V + 127) // 128 * 128)
-    print(json.dumps({
+    return {
         "metric": "markov_draft_rows_per_s", "value": replicas.whole_job_rate(R, args.steps, ms, world), "unit": "rows/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32", "data": "synthetic",
@@ -482,7 +528,191 @@ def bench_markov(args, device, rank, world, dist, barrier):
                      "tensor_frac_of_measured_bf16": flops / (gemm_call_ms * 1e-3) / 1e12 / float(peaks.get("bf16_tflops", 1590.0))},
         "step_frac_of_peak": gemm_bytes / (ms / args.steps * 1e-3) / 1e9 / peak,
         "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in kernels.items()},
-        "clocks": clocks, "dev_status": int(st.item())}), flush=True)
+        "clocks": clocks, "dev_status": int(st.item())}
+
+
+def launch_replicas(argv, n):
+    """`bench.py --gpus N` started as one plain process: start N ranks of itself, one per GPU, the way the
+    driver's launcher does (rank 0 prints the line)."""
+    import socket
+    import subprocess
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + argv
+    raise SystemExit(subprocess.call(cmd))
+
+
+def measure_workload(name, args, device, rank, local_rank, world, dist, barrier, with_e2e, with_cpu):
+    """Times one workload: the step (schedule -> verify) as the median over repeats of the --steps loop, the
+    verifier call alone, the kernels one by one, and (main workload only) the end-to-end and CPU legs."""
+    from paper_2607_05147_b200 import binding as B, replicas
+    steps, warmup = args.steps, args.warmup
+    # enough distinct batches that consecutive steps cannot be served from the 126 MB L2
+    wl = make_workload(name, device, rank)
+    step = Step(wl, device)
+    batches = wl["batches"]
+    n_sets = len(batches)
+    for i in range(warmup):
+        step.run(batches[i % n_sets])
+    torch.cuda.synchronize()
+    dev_status = int(step.status.item())
+    n_rows = batches[0].n_rows
+    lens = batches[0].meta["lengths"].to(device)
+    n_rejected = int((step.acc < lens).sum().item()) if not wl["greedy"] else 0
+    if wl["sched"] is not None:
+        assert torch.equal(step.offsets, batches[0].row_offsets), "scheduled offsets differ from the generated batch"
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_loop(fn, k):
+        barrier()
+        ev0.record()
+        for i in range(k):
+            fn(i)
+        ev1.record()
+        barrier()
+        return ev0.elapsed_time(ev1)
+
+    # EXACTLY `steps` steps between a barrier + synchronize on both sides, repeated: one repeat is a millisecond
+    # or two for the small workloads, too short to attribute a few per cent; the line reports the median repeat
+    first = timed_loop(lambda i: step.run(batches[i % n_sets]), steps)
+    if args.quick:
+        sampler.finish()
+        return dict(wl=wl, step=step, ms=first, n_rows=n_rows, n_rejected=n_rejected, quick=True)
+    repeats = max(args.repeats, int(50.0 / max(first, 1e-3)) + 1)
+    repeats = min(repeats, 400)
+    times = [first] + [timed_loop(lambda i: step.run(batches[i % n_sets]), steps) for _ in range(repeats - 1)]
+    times = replicas.max_over_ranks(times, dist, device)                # every repeat: the slowest rank
+    ts = sorted(times)
+    ms, ms_min = ts[len(ts) // 2], ts[0]
+
+    # the verifier call alone (the schedule's offsets stay where the last step left them), un-instrumented
+    def verify_only(i):
+        step.verify(batches[i % n_sets])
+    vt = sorted(timed_loop(verify_only, steps) for _ in range(max(5, repeats // 5)))
+    verify_ms = replicas.max_over_ranks([vt[len(vt) // 2]], dist, device)[0]
+
+    # keep the same load running until the clock sampler has seen enough of it (not timed)
+    t_end = time.perf_counter() + 1.0
+    i = 0
+    while time.perf_counter() < t_end and len(sampler.samples) < 40:
+        step.run(batches[i % n_sets]); i += 1
+        if i % 64 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+
+    # per-kernel timing of the same steps (events around every launch of the library)
+    timer = B.KernelTimer(steps * 12)
+    timer.attach()
+    for i in range(steps):
+        step.run(batches[i % n_sets])
+    torch.cuda.synchronize()
+    timer.detach()
+    kernels = timer.read()
+    timer.close()
+
+    res = dict(wl=wl, step=step, ms=ms, ms_min=ms_min, repeats=repeats, timed_ms=sum(times), verify_ms=verify_ms,
+               n_rows=n_rows, n_rejected=n_rejected, kernels=kernels, clocks=clocks, dev_status=dev_status, n_sets=n_sets)
+
+    if with_e2e:
+        # end to end: inputs start in pinned host memory, results end in host memory, every step
+        b = batches[0]
+        host_in = [t.cpu().pin_memory() for t in (b.target, b.draft, b.draft_tokens) if t is not None]
+        conf_h = wl["sched"].conf.cpu().pin_memory() if wl["sched"] is not None else None
+        off_h = None if wl["sched"] is not None else b.row_offsets.cpu().pin_memory()
+        dev_in = [torch.empty_like(t, device=device) for t in host_in]
+        conf_d = torch.empty_like(wl["sched"].conf) if conf_h is not None else None
+        off_d = torch.empty_like(b.row_offsets) if off_h is not None else None
+        acc_h = torch.empty(step.R, dtype=torch.int32).pin_memory()
+        out_h = torch.empty(step.n_rows, dtype=torch.int32).pin_memory()
+        from paper_2607_05147_b200 import workloads as W
+        h2d = sum(t.numel() * t.element_size() for t in host_in)
+        h2d += conf_h.numel() * 4 if conf_h is not None else off_h.numel() * 4
+        d2h = acc_h.numel() * 4 + out_h.numel() * 4
+
+        def e2e_step(_):
+            for h, d in zip(host_in, dev_in):
+                d.copy_(h, non_blocking=True)
+            if conf_h is not None:
+                conf_d.copy_(conf_h, non_blocking=True)
+            else:
+                off_d.copy_(off_h, non_blocking=True)
+            if wl["greedy"]:
+                eb = W.VerifyBatch(dev_in[0], None, off_d if off_d is not None else b.row_offsets, dev_in[1],
+                                   None, b.temperature, b.seed)
+            else:
+                eb = W.VerifyBatch(dev_in[0], dev_in[1], off_d if off_d is not None else b.row_offsets,
+                                   dev_in[2], None, b.temperature, b.seed)
+            step.run(eb, conf=conf_d)
+            acc_h.copy_(step.acc, non_blocking=True)
+            out_h.copy_(step.out, non_blocking=True)
+
+        e2e_steps = max(3, min(steps, 20))
+        for k in range(3):
+            e2e_step(k)
+        e2e_ms = replicas.max_over_ranks([timed_loop(e2e_step, e2e_steps)], dist, device)[0]
+        res["e2e"] = dict(ms=e2e_ms, steps=e2e_steps, h2d=h2d, d2h=d2h)
+
+    if with_cpu and rank == 0:
+        import oracle
+        oracle.build()
+        host_copy(wl)
+        threads = os.cpu_count() or 1
+        oracle_step(wl, batches[0], batches[0].R, threads)          # first touch of the host copies
+        t0 = time.perf_counter()
+        rows, reps = 0, 0
+        while reps < 3 or (time.perf_counter() - t0 < 2.0 and reps < 200):
+            rows += oracle_step(wl, batches[0], batches[0].R, threads)
+            reps += 1
+        dt = time.perf_counter() - t0
+        res["cpu"] = {"value": rows / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                      "sample": f"whole batch ({batches[0].R} requests, {rows // reps} rows) x {reps} passes in "
+                                f"{dt:.2f} s, pthreads over requests, stops at each first rejection"}
+        # the same oracle on one core: a bounded number of requests (about ten seconds at most)
+        t0 = time.perf_counter()
+        probe = max(1, batches[0].R // 16)
+        r1 = oracle_step(wl, batches[0], probe, 1)
+        t_probe = time.perf_counter() - t0
+        n_req = max(probe, min(batches[0].R, int(probe * 8.0 / max(t_probe, 1e-6))))
+        t0 = time.perf_counter()
+        r1 = oracle_step(wl, batches[0], n_req, 1)
+        dt1 = time.perf_counter() - t0
+        res["cpu"]["single_thread"] = {"value": r1 / dt1, "unit": UNIT, "cores": 1,
+                                       "sample": f"first {n_req} of {batches[0].R} requests ({r1} rows), one pass in {dt1:.2f} s"}
+    return res
+
+
+def roofline_of(res, peak, peak_src):
+    """Dominant kernel of the step against the measured HBM peak (bytes the method must move / its time)."""
+    wl = res["wl"]
+    b0 = wl["batches"][0]
+    stream_bytes, all_bytes = algorithmic_bytes(b0, wl["greedy"], res["n_rejected"])
+    dom = "greedy_stream" if wl["greedy"] else "stream_stats"
+    k = res["kernels"].get(dom, {"ms": float("nan"), "launches": 1})
+    dom_ms = k["ms"] / max(1, k["launches"])
+    achieved = stream_bytes / (dom_ms * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC_BYTES.get(wl["name"]) if not REQUESTS_OVERRIDE else None
+    if traffic is None and wl["name"] in NCU_TRAFFIC_RATIO and not REQUESTS_OVERRIDE:
+        traffic = int(NCU_TRAFFIC_RATIO[wl["name"]] * stream_bytes)
+    return {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": traffic,
+            "peak_source": peak_src, "algorithmic_bytes_per_launch": stream_bytes, "us_per_launch": dom_ms * 1e3}
+
+
+def verify_call_of(res, steps, peak):
+    """The verifier call as a whole (every kernel of dspark_verify / dspark_verify_greedy, no scheduler): the
+    bytes the method must move, re-reads of rejected pairs included, over its un-instrumented time."""
+    wl = res["wl"]
+    _, all_bytes = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
+    us = 1e3 * res["verify_ms"] / steps
+    gbs = all_bytes / (us * 1e-6) / 1e9
+    return {"us_per_call": us, "algorithmic_bytes": all_bytes, "gbs": gbs, "frac": gbs / peak,
+            "timing": "CUDA events around `steps` back-to-back calls, median over repeats, batches rotated"}
 
 
 def main():
@@ -490,10 +720,14 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--repeats", type=int, default=25,
+                    help="how often the timed --steps loop is repeated (the line reports the median and the minimum)")
     ap.add_argument("--workload", default="cfg3",
                     choices=["cfg2", "cfg3", "cfg4", "cfg5", "cfg2_fp32", "cfg4_bf16"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--all-workloads", action="store_true", help="also time the other V=129280 configurations")
+    ap.add_argument("--all-workloads", action="store_true",
+                    help="besides cfg2 / cfg4 / cfg5 and the Markov step also time the fp32 sampling and bf16 greedy variants")
+    ap.add_argument("--only", action="store_true", help="time --workload alone (no other workloads, no Markov step)")
     ap.add_argument("--async-topk", action="store_true",
                     help="schedule with dspark_schedule_async (capacity from two steps earlier, Section 5.2)")
     ap.add_argument("--per-request-temperature", action="store_true",
@@ -525,6 +759,9 @@ def main():
     if OVERLAP and (not ASYNC_TOPK or CUDA_GRAPH):
         raise SystemExit("--overlap-schedule needs --async-topk and stream launches")
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        launch_replicas(sys.argv[1:], args.gpus)
+
     from paper_2607_05147_b200 import replicas
     rank, local_rank, world = replicas.env_ranks()
     if args.impl == "reference":
@@ -550,137 +787,23 @@ def main():
         torch.cuda.synchronize()
 
     if args.markov_draft:
-        bench_markov(args, device, rank, world, dist, barrier)
+        line = bench_markov(args, device, rank, world, dist, barrier)
+        if line is not None:
+            print(json.dumps(line), flush=True)
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    def time_workload(name, steps, warmup, with_e2e, with_cpu):
-        # enough distinct batches that consecutive steps cannot be served from the 126 MB L2
-        wl = make_workload(name, device, rank)
-        step = Step(wl, device)
-        batches = wl["batches"]
-        n_sets = len(batches)
-        for i in range(warmup):
-            step.run(batches[i % n_sets])
-        torch.cuda.synchronize()
-        dev_status = int(step.status.item())
-        n_rows = batches[0].n_rows
-        lens = batches[0].meta["lengths"].to(device)
-        n_rejected = int((step.acc < lens).sum().item()) if not wl["greedy"] else 0
-        if wl["sched"] is not None:
-            assert torch.equal(step.offsets, batches[0].row_offsets), "scheduled offsets differ from the generated batch"
-
-        sampler = ClockSampler(local_rank)
-        sampler.start()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        ev0.record()
-        for i in range(steps):
-            step.run(batches[i % n_sets])
-        ev1.record()
-        barrier()
-        ms = ev0.elapsed_time(ev1)
-        if args.quick:
-            sampler.finish()
-            return dict(wl=wl, step=step, ms=ms, n_rows=n_rows, n_rejected=n_rejected, quick=True)
-        # keep the same load running for ~1.5 s so the clock sampler sees it (not timed)
-        t_end = time.perf_counter() + 1.5
-        i = 0
-        while time.perf_counter() < t_end:
-            step.run(batches[i % n_sets]); i += 1
-            if i % 64 == 0:
-                torch.cuda.synchronize()
-        torch.cuda.synchronize()
-        clocks = sampler.finish()
-
-        # per-kernel timing of the same steps (events around every launch of the library)
-        timer = B.KernelTimer(steps * 8)
-        timer.attach()
-        for i in range(steps):
-            step.run(batches[i % n_sets])
-        torch.cuda.synchronize()
-        timer.detach()
-        kernels = timer.read()
-        timer.close()
-
-        res = dict(wl=wl, step=step, ms=ms, n_rows=n_rows, n_rejected=n_rejected, kernels=kernels,
-                   clocks=clocks, dev_status=dev_status, n_sets=n_sets)
-
-        if with_e2e:
-            # end to end: inputs start in pinned host memory, results end in host memory, every step
-            b = batches[0]
-            host_in = [t.cpu().pin_memory() for t in (b.target, b.draft, b.draft_tokens) if t is not None]
-            conf_h = wl["sched"].conf.cpu().pin_memory() if wl["sched"] is not None else None
-            off_h = None if wl["sched"] is not None else b.row_offsets.cpu().pin_memory()
-            dev_in = [torch.empty_like(t, device=device) for t in host_in]
-            conf_d = torch.empty_like(wl["sched"].conf) if conf_h is not None else None
-            off_d = torch.empty_like(b.row_offsets) if off_h is not None else None
-            acc_h = torch.empty(step.R, dtype=torch.int32).pin_memory()
-            out_h = torch.empty(step.n_rows, dtype=torch.int32).pin_memory()
-            from paper_2607_05147_b200 import workloads as W
-            h2d = sum(t.numel() * t.element_size() for t in host_in)
-            h2d += conf_h.numel() * 4 if conf_h is not None else off_h.numel() * 4
-            d2h = acc_h.numel() * 4 + out_h.numel() * 4
-
-            def e2e_step():
-                for h, d in zip(host_in, dev_in):
-                    d.copy_(h, non_blocking=True)
-                if conf_h is not None:
-                    conf_d.copy_(conf_h, non_blocking=True)
-                else:
-                    off_d.copy_(off_h, non_blocking=True)
-                if wl["greedy"]:
-                    eb = W.VerifyBatch(dev_in[0], None, off_d if off_d is not None else b.row_offsets, dev_in[1],
-                                       None, b.temperature, b.seed)
-                else:
-                    eb = W.VerifyBatch(dev_in[0], dev_in[1], off_d if off_d is not None else b.row_offsets,
-                                       dev_in[2], None, b.temperature, b.seed)
-                step.run(eb, conf=conf_d)
-                acc_h.copy_(step.acc, non_blocking=True)
-                out_h.copy_(step.out, non_blocking=True)
-
-            e2e_steps = max(3, min(steps, 20))
-            for _ in range(3):
-                e2e_step()
-            barrier()
-            ev0.record()
-            for _ in range(e2e_steps):
-                e2e_step()
-            ev1.record()
-            barrier()
-            e2e_ms = ev0.elapsed_time(ev1)
-            res["e2e"] = dict(ms=e2e_ms, steps=e2e_steps, h2d=h2d, d2h=d2h)
-
-        if with_cpu and rank == 0:
-            import oracle
-            oracle.build()
-            host_copy(wl)
-            threads = os.cpu_count() or 1
-            oracle_step(wl, batches[0], batches[0].R, threads)          # first touch of the host copies
-            t0 = time.perf_counter()
-            rows, reps = 0, 0
-            while reps < 3 or (time.perf_counter() - t0 < 2.0 and reps < 200):
-                rows += oracle_step(wl, batches[0], batches[0].R, threads)
-                reps += 1
-            dt = time.perf_counter() - t0
-            res["cpu"] = {"value": rows / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
-                          "sample": f"whole batch ({batches[0].R} requests, {rows // reps} rows) x {reps} passes in "
-                                    f"{dt:.2f} s, pthreads over requests, stops at each first rejection"}
-        return res
-
-    res = time_workload(args.workload, args.steps, args.warmup, True, world == 1 or rank == 0)
+    res = measure_workload(args.workload, args, device, rank, local_rank, world, dist, barrier, True, world == 1 or rank == 0)
     wl = res["wl"]
     if res.get("quick"):
         print(json.dumps({"quick": True, "workload": wl["name"], "ms_per_step": res["ms"] / args.steps,
                           "rows_per_s": res["n_rows"] * args.steps / (res["ms"] * 1e-3)}), flush=True)
         return
 
-    # max over ranks of the device time
-    ms, e2e_ms = replicas.max_over_ranks([res["ms"], res["e2e"]["ms"]], dist, device)
-
     b0 = wl["batches"][0]
     stream_bytes, all_bytes = algorithmic_bytes(b0, wl["greedy"], res["n_rejected"])
+    ms, e2e_ms = res["ms"], res["e2e"]["ms"]
     value = replicas.whole_job_rate(res["n_rows"], args.steps, ms, world)
     e2e_value = replicas.whole_job_rate(res["n_rows"], res["e2e"]["steps"], e2e_ms, world)
 
@@ -689,41 +812,23 @@ def main():
         peak, peak_src = float(json.load(open(peaks_file))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     else:
         peak, peak_src = FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
-    dom = "greedy_stream" if wl["greedy"] else "stream_stats"
-    k = res["kernels"].get(dom, {"ms": float("nan"), "launches": 1})
-    dom_ms = k["ms"] / max(1, k["launches"])
-    dom_bytes = stream_bytes
-    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "traffic": NCU_TRAFFIC_BYTES.get(wl["name"]) if not REQUESTS_OVERRIDE else None,
-                "peak_source": peak_src,
-                "algorithmic_bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3}
 
-    if roofline["traffic"] is None and wl["name"] in NCU_TRAFFIC_RATIO and not REQUESTS_OVERRIDE:
-        roofline["traffic"] = int(NCU_TRAFFIC_RATIO[wl["name"]] * stream_bytes)
+    line = None
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl["desc"], "name": wl["name"], "requests": b0.R, "rows_per_step": res["n_rows"],
-                       "draft_rows_per_step": b0.n_rows - b0.R, "rejected_requests": res["n_rejected"],
-                       "logit_dtype": str(b0.target.dtype).replace("torch.", ""),
-                       "l2": f"inputs larger than L2: {res['n_sets']} distinct batches rotated "
-                             f"({res['n_sets'] * stream_bytes / 1e6:.0f} MB of logits)",
-                       "scheduler": ("async top-K, capacity from two steps earlier" if ASYNC_TOPK else "early stop")
-                       if wl["sched"] is not None else None,
-                       "temperature": "per request (device array)" if PER_REQUEST_T else "one per batch",
-                       "truncation": None if TRUNCATE is None else f"top_k={TRUNCATE[0]}, top_p={TRUNCATE[1]} (dspark_verify_truncated)",
-                       "launch": "CUDA graph replay" if CUDA_GRAPH else
-                       ("stream launches, scheduler of step t+1 overlapped on a second stream" if OVERLAP
-                        else "stream launches"),
-                       "parallelism": "replicas only (one engine per GPU, no collective)"},
+            "config": workload_config(wl, b0, res["n_rows"], res["n_rejected"], res["n_sets"], stream_bytes),
+            "timing": {"repeats": res["repeats"], "ms_per_step_min": res["ms_min"] / args.steps,
+                       "timed_region_ms": res["timed_ms"],
+                       "rule": "ms_per_step is the median over `repeats` repeats of the --steps loop, each between a "
+                               "barrier + synchronize on both sides (max over ranks per repeat)"},
             "step_algorithmic_bytes": all_bytes,
             "step_effective_gbs": all_bytes / (ms / args.steps * 1e-3) / 1e9,
             "step_frac_of_peak": all_bytes / (ms / args.steps * 1e-3) / 1e9 / peak,
-            "roofline": roofline,
+            "roofline": roofline_of(res, peak, peak_src),
+            "verify_call": verify_call_of(res, args.steps, peak),
             "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in res["kernels"].items()},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": res["e2e"]["h2d"],
                     "d2h_bytes_per_step": res["e2e"]["d2h"], "ms_per_step": e2e_ms / res["e2e"]["steps"],
@@ -732,26 +837,40 @@ def main():
             "clocks": res["clocks"], "dev_status": res["dev_status"],
             "cpu_baseline": res.get("cpu"),
         }
-        if args.all_workloads and world == 1:
-            others = {}
-            for name in ["cfg2", "cfg3", "cfg4", "cfg5", "cfg2_fp32", "cfg4_bf16"]:
-                if name == args.workload:
-                    continue
-                del res, wl
-                torch.cuda.empty_cache()
-                res = time_workload(name, args.steps, args.warmup, False, False)
-                wl = res["wl"]
-                sb, ab = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
-                d = "greedy_stream" if wl["greedy"] else "stream_stats"
-                kk = res["kernels"][d]
-                dms = kk["ms"] / kk["launches"]
-                others[name] = {"rows_per_s": res["n_rows"] * args.steps / (res["ms"] * 1e-3),
-                                "ms_per_step": res["ms"] / args.steps,
-                                "step_effective_gbs": ab / (res["ms"] / args.steps * 1e-3) / 1e9,
-                                "dominant_kernel_gbs": sb / (dms * 1e-3) / 1e9,
-                                "dominant_kernel_frac": sb / (dms * 1e-3) / 1e9 / peak,
-                                "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in res["kernels"].items()}}
-            line["other_workloads"] = others
+    if not args.only and world == 1:
+        # the other V = 129 280 configurations and the Markov-head draft step, each with its own clocks
+        names = ["cfg2", "cfg3", "cfg4", "cfg5"] + (["cfg2_fp32", "cfg4_bf16"] if args.all_workloads else [])
+        others = {}
+        for name in names:
+            if name == args.workload:
+                continue
+            del res, wl
+            torch.cuda.empty_cache()
+            res = measure_workload(name, args, device, rank, local_rank, world, dist, barrier, False, False)
+            wl = res["wl"]
+            _, ab = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
+            roof = roofline_of(res, peak, peak_src)
+            step_ms = res["ms"] / args.steps
+            others[name] = {"value": res["n_rows"] * args.steps / (res["ms"] * 1e-3), "unit": UNIT,
+                            "ms_per_step": step_ms, "ms_per_step_min": res["ms_min"] / args.steps, "repeats": res["repeats"],
+                            "rows_per_step": res["n_rows"], "rejected_requests": res["n_rejected"],
+                            "step_algorithmic_bytes": ab, "step_frac_of_peak": ab / (step_ms * 1e-3) / 1e9 / peak,
+                            "dominant_kernel": roof["kernel"], "dominant_kernel_gbs": roof["achieved"],
+                            "dominant_kernel_frac": roof["frac"], "dominant_kernel_us": roof["us_per_launch"],
+                            "verify_call": verify_call_of(res, args.steps, peak),
+                            "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in res["kernels"].items()},
+                            "clocks": res["clocks"], "dev_status": res["dev_status"]}
+        del res, wl
+        torch.cuda.empty_cache()
+        line["other_workloads"] = others
+        margs = argparse.Namespace(**vars(args))
+        margs.requests = 256
+        m = bench_markov(margs, device, rank, world, dist, barrier)
+        line["markov_draft"] = {"requests": 256, "us_per_launch": m["roofline"]["us_per_launch"], "frac": m["roofline"]["frac"],
+                                "gbs": m["roofline"]["achieved"], "tensor_tflops": m["roofline"]["tensor_tflops"],
+                                "step_us": 1e3 * m["ms_per_step"], "algorithmic_bytes_per_launch": m["roofline"]["algorithmic_bytes_per_launch"],
+                                "kernels_us_per_launch": m["kernels_us_per_launch"], "clocks": m["clocks"], "dev_status": m["dev_status"]}
+    if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
