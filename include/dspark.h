@@ -405,8 +405,9 @@ int dspark_verify_truncated(const void* target_logits, const void* draft_logits,
  *                [0,1] (NaN -> 0) and never rescaled
  *  accepted_len  device int32 [N]: accepted draft tokens of the block (what the verifier returned)
  *  verified_len  device int32 [N] or NULL (= gamma): how many positions of the block were verified
- *  grid          device fp32 [G]: candidate temperatures, all > 0 (not checked on the device); ties
- *                take the first grid point
+ *  grid          device fp32 [G]: candidate temperatures; a point that is not a positive finite number is
+ *                never chosen and gets NaN in out_ece_grid (if none is usable the position keeps T = 1);
+ *                ties take the first grid point
  *  n_bins        1..64 equal-width bins
  *  out_T         device fp32 [gamma]; a position nobody verified gets 1
  *  out_ece_before / out_ece_after  device fp64 [gamma] or NULL: ECE of the raw and of the calibrated chain

@@ -100,8 +100,12 @@ sts_pick_kernel(const StsAcc* acc, int k, const float* __restrict__ grid, int G,
         }
         e = cnt ? e / (double)cnt : 0.0;
         if (g == G) { if (ece_before) ece_before[k] = e; continue; }
-        if (ece_grid) ece_grid[(size_t)k * G + g] = e;
-        if (cnt && e < best) { best = e; bg = g; }          // g ascends within a thread: first minimum
+        // a grid point that is not a positive finite temperature is never chosen (its scaled confidences are
+        // meaningless); its entry of the ECE table says so
+        const float Tg = grid[g];
+        const bool usable = Tg > 0.f && Tg < INFINITY;
+        if (ece_grid) ece_grid[(size_t)k * G + g] = usable ? e : NAN;
+        if (usable && cnt && e < best) { best = e; bg = g; }          // g ascends within a thread: first minimum
     }
     s_e[threadIdx.x] = best; s_g[threadIdx.x] = bg;
     __syncthreads();

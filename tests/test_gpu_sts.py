@@ -89,3 +89,23 @@ def test_edge_values_and_unverified_positions():
     torch.cuda.synchronize()
     np.testing.assert_array_equal(out[:, 0].cpu().numpy(), [0.0, 1.0, 0.0, 1.0])
     np.testing.assert_allclose(out[:, 1].cpu().numpy(), [0.5, 0.25, 0.75, 0.5], rtol=1e-6)
+
+
+def test_unusable_grid_temperatures_are_never_chosen():
+    # a grid with a zero, a negative, a NaN and an infinite entry among good ones: the good entries are rated as
+    # without the bad ones, the bad ones are marked NaN and never win
+    rng = np.random.default_rng(3)
+    N, gamma = 5000, 4
+    conf = torch.from_numpy(rng.uniform(0.05, 0.95, size=(N, gamma)).astype(np.float32)).cuda()
+    acc = torch.from_numpy(rng.integers(0, gamma + 1, size=N).astype(np.int32)).cuda()
+    good = [0.5, 0.8, 1.0, 1.5, 2.5]
+    mixed = torch.tensor([0.0, 0.5, -1.0, 0.8, float("nan"), 1.0, float("inf"), 1.5, 2.5], device="cuda")
+    Tg, _, eag, egg = _gpu(conf, acc, None, torch.tensor(good, device="cuda"), 10)
+    Tm, _, eam, egm = _gpu(conf, acc, None, mixed, 10)
+    np.testing.assert_array_equal(Tm, Tg)
+    np.testing.assert_allclose(eam, eag, atol=1e-12)
+    assert np.isnan(egm[:, [0, 2, 4, 6]]).all()
+    np.testing.assert_allclose(egm[:, [1, 3, 5, 7, 8]], egg, atol=1e-12)
+    bad_only = torch.tensor([0.0, float("nan")], device="cuda")
+    Tb, _, _, _ = _gpu(conf, acc, None, bad_only, 10)
+    np.testing.assert_array_equal(Tb, np.ones(gamma, dtype=np.float32))
