@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                     slot.s = total <= 0x7fffffffll ? (int)((unsigned)u / (unsigned)ppr) : (int)(u / ppr);
                     slot.piece = (int)(u - (long long)slot.s * ppr);
                     if (kMode == kModeResid) slot.task = P.resid[slot.s];
+                    if (kMode == kModeHist) slot.trunc = P.trunc_rows[slot.s];
                     unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes, kMode == kModeResid ? &slot.task : nullptr);
                     slot.scale = stream_scale<kMode>(P, slot.s, n_rows, n_streams);
                 } else {
@@ -108,6 +109,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 // read by the consumers after the barrier below completes
                 s_unit[st].s = slot.s; s_unit[st].piece = slot.piece; s_unit[st].scale = slot.scale;
                 if (kMode == kModeResid) s_unit[st].task = slot.task;
+                if (kMode == kModeHist) s_unit[st].trunc = slot.trunc;
                 if (live) {
                     unsigned char* dst = stage_mem + st * kStageBytes;
                     mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(bytes * M::kSrc));
@@ -154,7 +156,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
             unsigned char* sp = stage_mem + st * kStageBytes + warp * M::kBlockBytes;
             SmemFetch f0{sp}, f1{sp + M::kPieceBytes};
             consume_block<kElem, kMode>(P, unit_s, unit_piece, n_rows, warp, lane, f0, f1, unit_scale,
-                                        kMode == kModeResid ? &s_unit[st].task : nullptr);
+                                        kMode == kModeResid ? &s_unit[st].task : nullptr,
+                                        kMode == kModeHist ? &s_unit[st].trunc : nullptr);
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);
         }

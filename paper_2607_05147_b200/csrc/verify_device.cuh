@@ -149,6 +149,7 @@ struct __align__(16) UnitSlot {    // what the producer tells the consumers abou
     float scale;
     int pad;
     ResidTask task;                // residual pass: the task of stream s (loaded once per unit, not once per warp)
+    TruncRow trunc;                // histogram pass: the window of row s (likewise)
 };
 
 // Walks the units (stream s, piece) owned by this CTA: unit index = s * ppr + piece, advancing by
@@ -396,7 +397,7 @@ __device__ __forceinline__ float block_resid(const uint4 (&vt)[kVec], const uint
 template <int kElem, int kMode, typename Fetch>
 __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int piece, int n_rows,
                                               int warp, int lane, const Fetch& f0, const Fetch& f1, float scale,
-                                              const ResidTask* task = nullptr)
+                                              const ResidTask* task = nullptr, const TruncRow* trunc = nullptr)
 {
     using M = ModeCfg<kMode>;
     const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
@@ -418,7 +419,7 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
     } else if (kMode == kModeHist) {
         // bf16 rows only.  Count the keys within the window next to the row maximum: a packed compare rejects
         // almost every pair, the few tokens of the tail take one atomic each.
-        const TruncRow tr = P.trunc_rows[s];
+        const TruncRow tr = trunc ? *trunc : P.trunc_rows[s];
         if (tr.size == 0u) return;
         const __nv_bfloat162 cut2 = *reinterpret_cast<const __nv_bfloat162*>(&tr.cut2);
         unsigned int* bins = P.trunc_bins + (long long)s * kHistBins;
