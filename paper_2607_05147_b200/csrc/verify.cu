@@ -495,18 +495,17 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             if (d < 0 || d >= P.V) atomicOr(&s_bad, DSPARK_DEV_BAD_TOKEN);
         }
     }
-    __syncthreads();
+    // no barrier here: the token check is looked at after the first round of positions, whose barrier covers it
     const bool want_all = (P.out_p != nullptr) || (P.out_q != nullptr);
     float scale_f = P.scale;
-    int bad_request = s_bad;                     // a request reports everything that is wrong with it
     if (P.req_temp) {
         const float T = P.req_temp[r];
-        if (!(T > 0.0f) || !(T < INFINITY)) bad_request |= DSPARK_DEV_BAD_TEMPERATURE;
-        else scale_f = (float)(1.4426950408889634 / (double)T);
-    }
-    if (bad_request) {
-        if (tid == 0) { atomicOr(P.dev_status, bad_request); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
-        return;
+        if (!(T > 0.0f) || !(T < INFINITY)) {
+            __syncthreads();                     // a request reports everything that is wrong with it
+            if (tid == 0) { atomicOr(P.dev_status, s_bad | DSPARK_DEV_BAD_TEMPERATURE); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone; }
+            return;
+        }
+        scale_f = (float)(1.4426950408889634 / (double)T);
     }
     const double scale_d = (double)scale_f;
 
@@ -516,10 +515,14 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             const bool is_draft_pos = j < len;
             // the two logits at the draft token do not depend on the statistics: fetch them first
             float xt = 0.f, xd = 0.f;
+            bool tok_ok = true;
             if (is_draft_pos && lane == 0) {
                 const int d = P.draft_tokens[lo + j];
-                xt = load_logit(P.target, lo + j, P.tstride_bytes, P.elem, d);
-                xd = load_logit(P.draft, drow0 + j, P.dstride_bytes, P.elem, d);
+                tok_ok = d >= 0 && d < P.V;          // a token out of range voids the request (flagged by the scan above)
+                if (tok_ok) {
+                    xt = load_logit(P.target, lo + j, P.tstride_bytes, P.elem, d);
+                    xd = load_logit(P.draft, drow0 + j, P.dstride_bytes, P.elem, d);
+                }
             }
             RowAcc A, D;
             combine_rows(P.stats_t + (long long)(lo + j) * P.nblk,
@@ -536,7 +539,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             }
             if (lane == 0) {
                 s_Ct[warp] = A.C; s_St[warp] = A.S; s_Cd[warp] = D.C; s_Sd[warp] = D.S;
-                if (is_draft_pos) {
+                if (is_draft_pos && tok_ok) {
                     if (!row_usable(A.C, A.S) || !row_usable(D.C, D.S)) {
                         atomicMin(&s_first_bad, j);
                     } else {
@@ -566,12 +569,16 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
         // unusable row before it counts (the warps of this round that looked further do not change the result)
         const int first_bad = s_first_bad;
         const bool void_req = want_all ? first_bad != 0x7fffffff : first_bad < first;
-        const bool stop = void_req || (!want_all && first < len);
+        const bool stop = void_req || (!want_all && first < len) || s_bad != 0;
         __syncthreads();                         // everyone has read the flags before the next round updates them
         if (stop) break;
     }
 
     if (tid != 0) return;
+    if (s_bad) {                                 // a draft token outside the vocabulary
+        atomicOr(P.dev_status, s_bad); P.accepted_len[r] = 0; P.req[r].kind = kTaskNone;
+        return;
+    }
     const int n = s_first;
     RequestRec rec;
     rec.kind = kTaskNone; rec.row_t = lo + n; rec.row_d = drow0 + n;
