@@ -193,9 +193,8 @@ __device__ __forceinline__ void tmem_load8(uint32_t taddr, uint32_t (&r)[8])
 // A quarter row of an embedding tile: 128 B of W1[x_prev] (src; NULL = zeros) into registers by four
 // 256-bit loads (a full 32 B sector each, all in flight at once), then into this thread's lane of tensor
 // memory, 32 columns from taddr (two bf16 per column, k ascending).
-__device__ __forceinline__ void embedding_quarter_row_to_tmem(const unsigned char* src, uint32_t taddr)
+__device__ __forceinline__ void embedding_quarter_row_load(const unsigned char* src, uint4 (&w)[8])
 {
-    uint4 w[8];
 #pragma unroll
     for (int v = 0; v < 8; ++v) w[v] = make_uint4(0, 0, 0, 0);
     if (src)
@@ -206,6 +205,9 @@ __device__ __forceinline__ void embedding_quarter_row_to_tmem(const unsigned cha
                            "=r"(w[v + 1].x), "=r"(w[v + 1].y), "=r"(w[v + 1].z), "=r"(w[v + 1].w)
                          : "l"(src + v * 16)
                          : "memory");
+}
+__device__ __forceinline__ void embedding_quarter_row_store(uint32_t taddr, const uint4 (&w)[8])
+{
     tmem_store32(taddr, w);
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     tc_fence_before();
@@ -391,7 +393,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
     unsigned char* sU = smem;                               // three base-logit / output tiles
     unsigned char* sB = smem + kUBuffers * kUTileBytes;     // two W2 tiles
     __shared__ __align__(8) uint64_t b_full[2], b_empty[2], a_full[2], acc_full[2], acc_empty[2];
-    __shared__ __align__(8) uint64_t u_full[kUBuffers], epi_done, prefetch_issued;
+    __shared__ __align__(8) uint64_t u_full[kUBuffers], epi_done, prefetch_issued, gather_issued;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -405,6 +407,7 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
         for (int s = 0; s < kUBuffers; ++s) mbar_init(&u_full[s], 1);
         mbar_init(&epi_done, kEpiWarps);
         mbar_init(&prefetch_issued, 2);
+        mbar_init(&gather_issued, kEpiWarps);
         s_abort = 0;
         mbar_fence_init();
     }
@@ -442,10 +445,13 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             for (int k = 0; k < my_tiles && !*abort_flag; ++k) {
                 const int bs = k & 1;
                 if (!mbar_wait_bounded(&b_empty[bs], ((uint32_t)(k >> 1) & 1u) ^ 1u)) { give_up(); break; }
+                // the second tile waits until the loads of the embedding rows have been issued: those small loads
+                // would otherwise queue behind it and the first product would start that much later
+                if (k == 1 && !mbar_wait_bounded(&gather_issued, 0u)) { give_up(); break; }
                 mbar_arrive_expect_tx(&b_full[bs], kTileBytes);
                 bulk_g2s_hint(sB + bs * kTileBytes, P.W2p + (size_t)unit_ntile(k) * kTileBytes, kTileBytes, &b_full[bs], pol_keep);
                 issued = k + 1;
-                if (k == 1 || k == my_tiles - 1) { if (!told) mbar_arrive(&prefetch_issued); told = true; }
+                if (!told) { mbar_arrive(&prefetch_issued); told = true; }
             }
             if (*abort_flag) {
                 // somebody gave up: leave only after the copies already issued have landed (bounded)
@@ -492,10 +498,11 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
             tma_load_2d(dst, &map_u, nt * kTileMN, mt * kTileMN, &u_full[t % kUBuffers], pol_stream);
             tma_load_2d(dst + kBoxBytes, &map_u, nt * kTileMN + kBoxCols, mt * kTileMN, &u_full[t % kUBuffers], pol_stream);
         };
-        // The first W2 tiles and base-logit tiles are requested before any embedding load: the copy
-        // instructions share the load/store queue with those loads and would wait behind them.
-        if (leader)
-            for (int t = 0; t < 2 && t < my_tiles; ++t) issue_u_load(t);
+        // Order of the first requests: the first W2 tile and the first base-logit tile (the copy instructions share
+        // the load/store queue with ordinary loads and would wait behind them), then the loads of the embedding
+        // rows, then the second tiles: with both tiles of each ahead of them the embedding rows -- which the first
+        // product needs -- arrived last, behind 28 MB of prefetch.
+        if (leader && my_tiles > 0) issue_u_load(0);
         if (warp == 2 && lane == 0) mbar_arrive(&prefetch_issued);
         mbar_wait_bounded(&prefetch_issued, 0u);            // a limit that runs out only costs the ordering
         if (my_tiles > 0) {
@@ -506,9 +513,15 @@ markov_gemm_kernel(MarkovParams P, const __grid_constant__ CUtensorMap map_u, co
                 if (x >= 0 && x < P.V) src = P.W1 + ((size_t)x * kRank + chunk * (kRank / 4)) * 2;
                 else if ((int)blockIdx.x < P.m_tiles && chunk == 0) atomicOr(P.dev_status, DSPARK_DEV_BAD_TOKEN);
             }
-            embedding_quarter_row_to_tmem(src, tmem_a0 + lane_base + (uint32_t)(chunk * (kRank / 8)));
+            uint4 w[8];
+            embedding_quarter_row_load(src, w);
+            if (lane == 0) mbar_arrive(&gather_issued);     // the loads are on their way: the next tiles may queue behind them
+            if (leader && my_tiles > 1) issue_u_load(1);
+            embedding_quarter_row_store(tmem_a0 + lane_base + (uint32_t)(chunk * (kRank / 8)), w);
             __syncwarp();
             if (lane == 0) mbar_arrive(&a_full[0]);
+        } else if (lane == 0) {
+            mbar_arrive(&gather_issued);
         }
         for (int t = 0; t < my_tiles && !*abort_flag; ++t) {
             const int nt = unit_ntile(t), mt = my_mt;
