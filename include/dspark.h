@@ -359,8 +359,10 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
  *   distribution renormalised over the top-k set: walking the distinct values downwards, tau_p is the first
  *   value at which the cumulative mass reaches top_p[r] * Z_k (top_p >= 1: off; <= 0: only the maximum);
  *   tau = max(tau_k, tau_p).  p = softmax(row / T_r).
- *  target_logits   device bf16 [n_rows, >= V], modified in place; dtype must be DSPARK_BF16 (the threshold
- *                  is found exactly on the 16-bit keys) -- DSPARK_F32 returns DSPARK_ERR_SHAPE
+ *  target_logits   device bf16 or fp32 [n_rows, >= V], modified in place.  bf16: the threshold is found exactly on
+ *                  a histogram of the 16-bit keys.  fp32: by a descent over the 32-bit patterns (a histogram
+ *                  linear in the distance to the row maximum, then 11 bits of the key at a time), masses summed
+ *                  as integers so that the result does not change from run to run; several times slower per row
  *  row_offsets, R, n_rows   the ragged batch of the verifiers; every row of request r uses r's parameters
  *  top_k           device int32 [R] or NULL;  top_p  device fp32 [R] or NULL (both NULL: nothing to do)
  *  temperature / temperatures   one T > 0, or device fp32 [R] (a T that is not positive and finite leaves
@@ -368,7 +370,7 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
  *  out_tau         device fp32 [n_rows] or NULL: threshold value of each row (-inf: untouched)
  *  out_kept        device int32 [n_rows] or NULL: size of the kept set (V: untouched)
  * A row with NaN, +inf or no finite element is left as it is (the verifier reports it).  Costs one read of
- * the row from HBM, two from L2 and one write.  No workspace.  Errors: INVALID_ARG, SHAPE, CUDA.
+ * the row from HBM, two from L2 and one write (fp32: four to six reads).  No workspace.  Errors: INVALID_ARG, CUDA.
  */
 int dspark_truncate_target(void* target_logits, int dtype, int64_t target_row_stride, int V,
                            const int32_t* row_offsets, int R, int n_rows,
@@ -383,7 +385,8 @@ int dspark_truncate_target(void* target_logits, int dtype, int64_t target_row_st
  * Costs one extra read of the target rows (plus one from L2 / shared memory) instead of the read + write of
  * dspark_truncate_target.  temperatures / top_k / top_p: device [R] or NULL (temperatures NULL: the scalar
  * `temperature`; top_k and top_p both NULL: plain dspark_verify).  out_p_tok reports the truncated p(x).
- * bf16 only (DSPARK_F32 with top_k or top_p: DSPARK_ERR_SHAPE).  Same workspace as dspark_verify.
+ * fp32 rows: the threshold of every target row comes from the per-row descent of dspark_truncate_target (no
+ * streamed search), the rest is the same.  Same workspace as dspark_verify.
  */
 int dspark_verify_truncated(const void* target_logits, const void* draft_logits, int dtype,
                             int64_t target_row_stride, int64_t draft_row_stride, int V,

@@ -471,7 +471,7 @@ def dspark_truncate_target(target: torch.Tensor, row_offsets: torch.Tensor, *, t
                            top_p: Optional[torch.Tensor] = None, temperature: float = 1.0,
                            temperatures: Optional[torch.Tensor] = None, out_tau: Optional[torch.Tensor] = None,
                            out_kept: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> None:
-    """Masks the excluded tokens of every target row to -inf in place (bf16 rows)."""
+    """Masks the excluded tokens of every target row to -inf in place (bf16 or fp32 rows)."""
     tp, code, ts = _logits(target, "target")
     R = row_offsets.numel() - 1
     n_rows = target.shape[0]

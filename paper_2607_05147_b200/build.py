@@ -12,7 +12,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libdspark.so")
-SOURCES = ["api.cu", "schedule.cu", "verify.cu", "markov.cu", "sts.cu", "truncate.cu"]
+SOURCES = ["api.cu", "schedule.cu", "verify.cu", "markov.cu", "sts.cu", "truncate.cu", "truncate_f32.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-ffp-contract=off,-fvisibility=default"]
 

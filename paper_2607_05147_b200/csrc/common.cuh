@@ -237,6 +237,13 @@ __device__ __forceinline__ float bf16_key_value(uint32_t k)
 // Threshold search of the top-k / top-p truncation run inside the sampling verifier (truncate.cu): writes
 // the threshold of every target row to tau_rows (-inf: no cut) and replaces the block sums of the row's
 // statistics by the sums over the kept set; the rows themselves are not modified.
+// fp32 rows (truncate_f32.cu): the verifier's virtual truncation of every target row, and the in-place form
+int truncate_f32_virtual_launch(const void* target, long long stride_elems, int V, const int32_t* row_offsets, int R, int n_rows,
+                                const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
+                                float* tau_rows, float2* stats_t, int nblk, int epb, cudaStream_t stream);
+int truncate_f32_in_place(void* target, long long stride_elems, int V, const int32_t* row_offsets, int R, int n_rows,
+                          const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
+                          float* out_tau, int32_t* out_kept, cudaStream_t stream);
 int truncate_virtual_launch(const void* target, long long stride_bytes, int V, const int32_t* row_offsets, int R, int n_rows,
                             const int32_t* top_k, const float* top_p, float temperature, const float* temperatures,
                             float* tau_rows, float2* stats_t, int nblk, int epb, const int32_t* only_flagged,

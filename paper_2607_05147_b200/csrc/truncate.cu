@@ -552,9 +552,12 @@ int dspark_truncate_target(void* target_logits, int dtype, int64_t target_row_st
                            float* out_tau, int32_t* out_kept, int32_t* dev_status, void* stream)
 {
     if (!target_logits || !row_offsets || R < 1 || n_rows < 1 || V < 1 || target_row_stride < V) return DSPARK_ERR_INVALID_ARG;
-    if (dtype != DSPARK_BF16) return DSPARK_ERR_SHAPE;      // the threshold search works on 16-bit keys
+    if (dtype != DSPARK_BF16 && dtype != DSPARK_F32) return DSPARK_ERR_INVALID_ARG;
     if (!top_k && !top_p) return DSPARK_OK;
     if (!temperatures && (!(temperature > 0.f) || isinf(temperature))) return DSPARK_ERR_INVALID_ARG;
+    if (dtype == DSPARK_F32)                                 // 32-bit patterns: a descent instead of a key window
+        return truncate_f32_in_place(target_logits, (long long)target_row_stride, V, row_offsets, R, n_rows, top_k, top_p,
+                                     temperature, temperatures, out_tau, out_kept, (cudaStream_t)stream);
     TruncParams P;
     P.target = (unsigned char*)target_logits; P.stride_bytes = (long long)target_row_stride * 2; P.V = V;
     P.row_offsets = row_offsets; P.R = R; P.n_rows = n_rows;

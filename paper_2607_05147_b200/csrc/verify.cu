@@ -1044,7 +1044,6 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
 {
     if (!draft_logits) return DSPARK_ERR_INVALID_ARG;
     const bool truncate = top_k || top_p;
-    if (truncate && dtype != DSPARK_BF16) return DSPARK_ERR_SHAPE;   // the threshold search works on 16-bit keys
     if (!req_temp && (!(temperature > 0.0f) || !isfinite(temperature))) return DSPARK_ERR_INVALID_ARG;
     if (draft_row_stride < V) return DSPARK_ERR_SHAPE;
     VerifyParams P;
@@ -1071,7 +1070,16 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
         launch_stream_dtype<kModeStats>(P, bulk, (2ll * n_rows - R) * pieces(P.nblk), s);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
-    if (truncate) {
+    if (truncate && dtype == DSPARK_F32) {
+        // fp32 rows: the threshold of every target row by a descent over its 32-bit patterns (one CTA per row),
+        // which also replaces the row's block sums by the sums over the kept set
+        float* tau = (float*)((unsigned char*)workspace + workspace_layout(R, n_rows, V).tau);
+        KernelTimerScope timer(DSPARK_K_TRUNCATE, s);
+        rc = truncate_f32_virtual_launch(P.target, (long long)target_row_stride, V, row_offsets, R, n_rows, top_k, top_p,
+                                         temperature, req_temp, tau, P.stats_t, P.nblk, P.epb, s);
+        if (rc != DSPARK_OK) return rc;
+        P.tau = tau;
+    } else if (truncate) {
         // top-k / top-p of the target distribution without touching the rows: one kernel finds the threshold of
         // every target row and replaces the row's block sums by the sums over the kept set; from here on a
         // target logit below the threshold counts as -inf

@@ -125,7 +125,8 @@ def test_truncate_fuzz(seed):
             t = torch.from_numpy(rng.integers(-4, 5, (n_rows, V)).astype(np.float32)) * 0.25      # heavy ties
         else:
             t = torch.from_numpy(rng.uniform(-30, 30, (n_rows, V)).astype(np.float32))
-        t = _pad_rows(t.to(torch.bfloat16).cuda(), rng)
+        dt = torch.bfloat16 if rng.random() < 0.5 else torch.float32      # 16-bit key window / 32-bit descent
+        t = _pad_rows(t.to(dt).cuda(), rng)
         ks = rng.integers(-1, V + 3, size=R).astype(np.int32)
         ps = rng.choice([0.0, 0.1, 0.5, 0.9, 0.99, 1.0, 1.5], size=R).astype(np.float32)
         Ts = rng.uniform(0.3, 2.5, size=R).astype(np.float32)
