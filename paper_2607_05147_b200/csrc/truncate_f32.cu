@@ -85,6 +85,38 @@ __device__ __forceinline__ void for_each_elem(const float* row, int V, F fn)
     }
 }
 
+// The same walk with the aligned middle of the row handed over four elements at a time: vec(v) for every 16-byte
+// vector, elem(x) for the few elements before and after.  The passes below decide about a whole vector with a handful
+// of instructions (almost every vector of a row lies entirely below the window) and fall back to the element form
+// only for the vectors that do not.
+template <typename FV, typename FE>
+__device__ __forceinline__ void for_each_vec(const float* row, int V, FV vec, FE elem)
+{
+    int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) >> 2);
+    if (head > V) head = V;
+    const int nvec = (V - head) >> 2;
+    const float4* p = reinterpret_cast<const float4*>(row + head);
+    for (int c0 = threadIdx.x; c0 < nvec; c0 += kF32Unroll * kF32Threads) {
+        float4 v[kF32Unroll];
+#pragma unroll
+        for (int u = 0; u < kF32Unroll; ++u) {
+            const int c = c0 + u * kF32Threads;
+            v[u] = c < nvec ? __ldcg(&p[c]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < kF32Unroll; ++u)
+            if (c0 + u * kF32Threads < nvec) vec(v[u]);
+    }
+    const int tail0 = head + 4 * nvec;
+    for (int i = threadIdx.x; i < head + (V - tail0); i += kF32Threads) elem(__ldcg(&row[i < head ? i : tail0 + (i - head)]));
+}
+__device__ __forceinline__ float max_nan(float a, float b)
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+
 struct F32Shared {
     unsigned int cnt[kF32Bins];
     unsigned long long mass[kF32Bins];
@@ -195,10 +227,11 @@ __device__ void truncate_row_f32(const TruncF32Params& P, const int row, F32Shar
 
     // ---- pass 0: maximum, NaN / +inf ------------------------------------------------------------------------
     {
-        float mx = -INFINITY;
-        bool bad = false;
-        for_each_elem(rowp, V, [&](int, float x) { bad |= x != x; mx = fmaxf(mx, x); });
-        mx = warp_max_f32(mx);
+        float mx = -INFINITY;                                // a NaN anywhere survives this maximum
+        for_each_vec(rowp, V, [&](float4 v) { mx = max_nan(mx, max_nan(max_nan(v.x, v.y), max_nan(v.z, v.w))); },
+                     [&](float x) { mx = max_nan(mx, x); });
+        const bool bad = mx != mx;
+        mx = warp_max_f32(bad ? -INFINITY : mx);
         if (bad) S.flag = 1;
         __syncthreads();
         if (lane == 0) S.warp_c[warp] = (unsigned long long)f32_key(mx);
@@ -239,13 +272,33 @@ __device__ void truncate_row_f32(const TruncF32Params& P, const int row, F32Shar
         for (int i = tid; i < kF32Bins; i += kF32Threads) { S.cnt[i] = 0u; S.mass[i] = 0ull; }
         __syncthreads();
         unsigned long long far_c = 0ull, far_m = 0ull;
-        for_each_elem(rowp, V, [&](int, float x) {
+        auto one = [&](float x) {
             const int b = win_bin(x, w);
             if (b < 0) return;
             const unsigned long long fx = mass_of(x);
             if (b == kF32Bins - 1) { ++far_c; far_m += fx; }
             else { atomicAdd(&S.cnt[b], 1u); atomicAdd(&S.mass[b], fx); }
-        });
+        };
+        // a vector entirely below the window: counted, and (top-p) its masses summed in fp32 per vector lane -- every
+        // thread adds its own elements in a fixed order, so these sums are the same from run to run as well
+        const float far_from = (float)((w + 1) * (kF32Bins - 1));
+        unsigned int far_v = 0u;
+        float4 fa = make_float4(0.f, 0.f, 0.f, 0.f);
+        for_each_vec(rowp, V, [&](float4 v) {
+            const float d0 = __fmaf_rn(v.x, -bin_scale, mb), d1 = __fmaf_rn(v.y, -bin_scale, mb);
+            const float d2 = __fmaf_rn(v.z, -bin_scale, mb), d3 = __fmaf_rn(v.w, -bin_scale, mb);
+            if (fminf(fminf(d0, d1), fminf(d2, d3)) >= far_from) {
+                ++far_v;
+                if (use_p) {
+                    fa.x += ex2_approx(__fmaf_rn(v.x, scale2, nm2)); fa.y += ex2_approx(__fmaf_rn(v.y, scale2, nm2));
+                    fa.z += ex2_approx(__fmaf_rn(v.z, scale2, nm2)); fa.w += ex2_approx(__fmaf_rn(v.w, scale2, nm2));
+                }
+            } else {
+                one(v.x); one(v.y); one(v.z); one(v.w);
+            }
+        }, one);
+        far_c += 4ull * far_v;
+        far_m += __double2ull_rz((((double)fa.x + (double)fa.y) + ((double)fa.z + (double)fa.w)) * 1099511627776.0);
         block_sum_pair(S, far_c, far_m);
         if (tid == 0) { S.cnt[kF32Bins - 1] = (unsigned int)S.red_c; S.mass[kF32Bins - 1] = S.red_m; }
         __syncthreads();
@@ -301,13 +354,33 @@ __device__ void truncate_row_f32(const TruncF32Params& P, const int row, F32Shar
         __syncthreads();
         {
             uint32_t lo = 0xFFFFFFFFu, hi = 0u;
-            for_each_elem(rowp, V, [&](int, float x) {
+            // members of an inner bin have Bf <= d < Bf + 1: a vector with all four distances on one side of that has none
+            const float Bf = (float)(bA + w * (kF32Bins - 1));
+            const bool inner = bA != kF32Bins - 1;
+            auto one = [&](float x) {
                 if (lin_bin(x) == bA) {
                     const uint32_t kx = f32_key(x);
                     lo = min(lo, kx); hi = max(hi, kx);
-                    if (listed) S.list[atomicAdd(&S.n_list, 1)] = x;
+                    if (listed) {
+                        // one shared-memory atomic per group of lanes that found a member in the same step
+                        const unsigned act = __activemask();
+                        const int leader = __ffs(act) - 1;
+                        int at = 0;
+                        if (lane == leader) at = atomicAdd(&S.n_list, __popc(act));
+                        at = __shfl_sync(act, at, leader);
+                        S.list[at + __popc(act & ((1u << lane) - 1u))] = x;
+                    }
                 }
-            });
+            };
+            for_each_vec(rowp, V, [&](float4 v) {
+                if (inner) {
+                    const float d0 = __fmaf_rn(v.x, -bin_scale, mb), d1 = __fmaf_rn(v.y, -bin_scale, mb);
+                    const float d2 = __fmaf_rn(v.z, -bin_scale, mb), d3 = __fmaf_rn(v.w, -bin_scale, mb);
+                    if (fminf(fminf(d0, d1), fminf(d2, d3)) >= Bf + 1.0f) return;
+                    if (Bf > 0.0f && fmaxf(fmaxf(d0, d1), fmaxf(d2, d3)) < Bf) return;
+                }
+                one(v.x); one(v.y); one(v.z); one(v.w);
+            }, one);
             lo = __reduce_min_sync(0xffffffffu, lo);
             hi = __reduce_max_sync(0xffffffffu, hi);
             if (lane == 0) { atomicMin(&S.kmin, lo); atomicMax(&S.kmax, hi); }

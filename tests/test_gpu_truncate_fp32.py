@@ -156,25 +156,30 @@ def test_verifier_on_the_truncated_fp32_target_against_the_oracle_pipeline(V, bl
     g0 = torch.Generator().manual_seed(V + 1)
     R = 20
     lengths = torch.randint(0, 7, (R,), generator=g0)
-    b = W.sampling_batch(lengths, V, 47, "cuda", temperature=0.9, draft_noise=1.0, verify_seed=78, block=block,
-                         dtype=torch.float32)
     rng = np.random.default_rng(V + 1)
     ks = rng.choice([0, 1, 5, 40, 500], size=R).astype(np.int32)
     ps = rng.choice([1.0, 0.95, 0.8, 0.5], size=R).astype(np.float32)
     temps = rng.choice([0.7, 1.0, 1.3], size=R).astype(np.float32)
-    off = b.row_offsets.cpu().numpy()
     for use_temps in (False, True):
         t = temps if use_temps else None
+        # a batch on which no top-p decision of the oracle sits on its boundary (there either neighbour is right and
+        # the comparison of the verifier's outputs would say nothing): the first of a few seeds
+        for seed in range(47, 53):
+            b = W.sampling_batch(lengths, V, seed, "cuda", temperature=0.9, draft_noise=1.0, verify_seed=78, block=block,
+                                 dtype=torch.float32)
+            off = b.row_offsets.cpu().numpy()
+            masked, tau, kept, margin = oracle.warp_target(W.bf16_bits(b.target), off, top_k=ks, top_p=ps,
+                                                           temperature=b.temperature, temperatures=t)
+            if not (margin < 1e-5).any():
+                break
+        else:
+            pytest.fail("no seed without a boundary decision")
         g = _gpu_truncated(b, ks, ps, t)
-        masked, tau, kept, margin = oracle.warp_target(W.bf16_bits(b.target), off, top_k=ks, top_p=ps,
-                                                       temperature=b.temperature, temperatures=t)
         drs = None if b.draft_row_start is None else b.draft_row_start.cpu().numpy()
         o = oracle.verify(masked, W.bf16_bits(b.draft), off, b.draft_tokens.cpu().numpy(), b.temperature, b.seed,
                           draft_row_start=drs, eval_all=True, n_threads=H.THREADS, temperatures=t)
-        if (margin < 1e-5).any():
-            pytest.skip("a top-p decision sits on its boundary for this seed")
         mism = H.compare_sampling(g, o, off)
-        print(f"[verify_truncated fp32] V={V} per-request T={use_temps}: accepted {g['acc'].tolist()}, {mism} boundary mismatches")
+        print(f"[verify_truncated fp32] V={V} per-request T={use_temps} seed={seed}: accepted {g['acc'].tolist()}, {mism} boundary mismatches")
 
 
 def test_matches_the_two_step_gpu_pipeline_on_fp32_rows():
