@@ -162,24 +162,27 @@ def test_verifier_on_the_truncated_fp32_target_against_the_oracle_pipeline(V, bl
     temps = rng.choice([0.7, 1.0, 1.3], size=R).astype(np.float32)
     for use_temps in (False, True):
         t = temps if use_temps else None
-        # a batch on which no top-p decision of the oracle sits on its boundary (there either neighbour is right and
-        # the comparison of the verifier's outputs would say nothing): the first of a few seeds
-        for seed in range(47, 53):
-            b = W.sampling_batch(lengths, V, seed, "cuda", temperature=0.9, draft_noise=1.0, verify_seed=78, block=block,
-                                 dtype=torch.float32)
-            off = b.row_offsets.cpu().numpy()
-            masked, tau, kept, margin = oracle.warp_target(W.bf16_bits(b.target), off, top_k=ks, top_p=ps,
+        b = W.sampling_batch(lengths, V, 47, "cuda", temperature=0.9, draft_noise=1.0, verify_seed=78, block=block,
+                             dtype=torch.float32)
+        off = b.row_offsets.cpu().numpy()
+        # Where a top-p decision of the oracle sits on its boundary either neighbour is right and the comparison of
+        # the verifier's outputs would say nothing (on a flat full-vocabulary row a single token carries about 1e-5
+        # of the mass, so this is common): those requests run without top-p here.
+        ps_run = ps.copy()
+        for _ in range(3):
+            masked, tau, kept, margin = oracle.warp_target(W.bf16_bits(b.target), off, top_k=ks, top_p=ps_run,
                                                            temperature=b.temperature, temperatures=t)
-            if not (margin < 1e-5).any():
+            on_boundary = [r for r in range(R) if (margin[off[r]:off[r + 1]] < 1e-5).any()]
+            if not on_boundary:
                 break
-        else:
-            pytest.fail("no seed without a boundary decision")
-        g = _gpu_truncated(b, ks, ps, t)
+            ps_run[on_boundary] = 1.0
+        assert not on_boundary and (ps_run < 1.0).sum() >= 3
+        g = _gpu_truncated(b, ks, ps_run, t)
         drs = None if b.draft_row_start is None else b.draft_row_start.cpu().numpy()
         o = oracle.verify(masked, W.bf16_bits(b.draft), off, b.draft_tokens.cpu().numpy(), b.temperature, b.seed,
                           draft_row_start=drs, eval_all=True, n_threads=H.THREADS, temperatures=t)
         mism = H.compare_sampling(g, o, off)
-        print(f"[verify_truncated fp32] V={V} per-request T={use_temps} seed={seed}: accepted {g['acc'].tolist()}, {mism} boundary mismatches")
+        print(f"[verify_truncated fp32] V={V} per-request T={use_temps}, top-p on {int((ps_run < 1.0).sum())} requests: accepted {g['acc'].tolist()}, {mism} boundary mismatches")
 
 
 def test_matches_the_two_step_gpu_pipeline_on_fp32_rows():
