@@ -198,3 +198,46 @@ def test_matches_the_two_step_gpu_pipeline_on_fp32_rows():
     g2 = H.gpu_verify(mb, temperatures=torch.from_numpy(temps).cuda())
     np.testing.assert_array_equal(g["acc"], g2["acc"])
     np.testing.assert_array_equal(g["out"][:b.n_rows], g2["out"][:b.n_rows])
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_truncated_verifier_replayed_from_a_cuda_graph(dtype):
+    # the call captured once and replayed on other logits in the same buffers gives what the eager call gives
+    lengths = torch.tensor([2, 0, 4, 1, 3, 2, 0, 5])
+    V = 20_000
+    batches = [W.sampling_batch(lengths, V, 300 + i, "cuda", temperature=0.8, draft_noise=1.0, verify_seed=11, dtype=dtype)
+               for i in range(3)]
+    b0 = batches[0]
+    R, cap = b0.R, b0.n_rows
+    ks = torch.full((R,), 30, dtype=torch.int32, device="cuda")
+    ps = torch.full((R,), 0.9, dtype=torch.float32, device="cuda")
+    target = b0.target.clone(); draft = b0.draft.clone()
+    acc = torch.zeros(R, dtype=torch.int32, device="cuda")
+    out = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = B.workspace(B.dspark_verify_workspace_bytes(R, cap, V))
+
+    def call():
+        B.dspark_verify_truncated(target, draft, b0.row_offsets, b0.draft_tokens, b0.seed, temperature=b0.temperature,
+                                  top_k=ks, top_p=ps, accepted_len=acc, out_tokens=out, dev_status=st, workspace=ws)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        call()                                                # eager pass first: sets the kernel attributes
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        call()
+    torch.cuda.synchronize()
+    for b in batches[::-1]:
+        target.copy_(b.target); draft.copy_(b.draft)
+        call()
+        torch.cuda.synchronize()
+        want = (acc.cpu().numpy().copy(), out.cpu().numpy().copy(), int(st.item()))
+        acc.fill_(-5); out.fill_(-5)
+        graph.replay()
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(acc.cpu().numpy(), want[0])
+        np.testing.assert_array_equal(out.cpu().numpy(), want[1])
+        assert int(st.item()) == want[2] == 0
