@@ -161,17 +161,22 @@ class Step:
             self.tick = 0
             self.primed = False
         # kernels of the library per step: scheduler (prep, rank + final stage; a selection kernel when the
-        # candidates are many and the budget admits fewer than half), verifier (stream, decide[, residual
-        # stream, finalize]), row scales for per-request temperatures, five more for the truncation
+        # candidates are many and the budget admits fewer than half)
         n_sched = 0
         if self.sched is not None:
             gamma = self.sched.conf.shape[1]
             gpad = 1 << max(0, (gamma - 1).bit_length()) if gamma <= 32 else (gamma + 31) // 32 * 32
             entries = self.R * gpad
             n_sched = 2 + (1 if entries >= 8192 and 2 * (self.sched.budget_tokens - self.R) <= entries else 0)
-        # verifier: statistics pass + accept / residual / draw kernel (greedy: argmax pass + decide); row scales for
-        # per-request temperatures, five launches more for the threshold search of a truncated target
-        n_verify = 2 + (1 if PER_REQUEST_T and not wl["greedy"] else 0) + (5 if TRUNCATE is not None and not wl["greedy"] else 0)
+        # verifier: statistics pass, accept tests, residual pass, draws (greedy: argmax pass + accept tests); one more
+        # for per-request temperatures; for a truncated target the window preparation, the histogram pass, the
+        # threshold scan, the restricted sums and the per-row fallback (fp32 rows: the per-row descent alone)
+        if wl["greedy"]:
+            n_verify = 2
+        else:
+            n_verify = 4 + (1 if PER_REQUEST_T else 0)
+            if TRUNCATE is not None:
+                n_verify += 1 if b0.target.dtype == torch.float32 else 5
         self.launches_per_step = n_sched + n_verify
 
     def run(self, batch, conf=None):
