@@ -601,6 +601,30 @@ def measure_workload(name, args, device, rank, local_rank, world, dist, barrier,
     vt = sorted(timed_loop(verify_only, steps) for _ in range(max(5, repeats // 5)))
     verify_ms = replicas.max_over_ranks([vt[len(vt) // 2]], dist, device)[0]
 
+    # the same call when the drafter hands over the statistics of its rows (dspark_verify_draft_stats): the pairs are
+    # computed once, outside the timed region, the way a draft step leaves them behind
+    draft_stats_ms = None
+    if not wl["greedy"] and TRUNCATE is None and not PER_REQUEST_T:
+        row_stats = []
+        for b in batches:
+            st_b = torch.empty(b.draft.shape[0], 2, device=device)
+            B.dspark_row_stats(b.draft, b.temperature, out_row_stats=st_b)
+            row_stats.append(st_b)
+        torch.cuda.synchronize()
+        off_now = step.offsets if step.sched is not None else None
+
+        def verify_stats(i):
+            b = batches[i % n_sets]
+            B.dspark_verify_draft_stats(b.target, b.draft, off_now if off_now is not None else b.row_offsets, b.draft_tokens,
+                                        row_stats[i % n_sets], b.seed, temperature=b.temperature,
+                                        draft_row_start=b.draft_row_start, accepted_len=step.acc, out_tokens=step.out,
+                                        dev_status=step.status, workspace=step.ws, n_rows=step.n_rows)
+        for i in range(min(warmup, 5)):
+            verify_stats(i)
+        dt = sorted(timed_loop(verify_stats, steps) for _ in range(max(5, repeats // 5)))
+        draft_stats_ms = replicas.max_over_ranks([dt[len(dt) // 2]], dist, device)[0]
+        assert int(step.status.item()) == dev_status
+
     # keep the same load running until the clock sampler has seen enough of it (not timed)
     t_end = time.perf_counter() + 1.0
     i = 0
@@ -622,6 +646,7 @@ def measure_workload(name, args, device, rank, local_rank, world, dist, barrier,
     timer.close()
 
     res = dict(wl=wl, step=step, ms=ms, ms_min=ms_min, repeats=repeats, timed_ms=sum(times), verify_ms=verify_ms,
+               draft_stats_ms=draft_stats_ms,
                n_rows=n_rows, n_rejected=n_rejected, kernels=kernels, clocks=clocks, dev_status=dev_status, n_sets=n_sets)
 
     if with_e2e:
@@ -718,6 +743,23 @@ def verify_call_of(res, steps, peak):
     gbs = all_bytes / (us * 1e-6) / 1e9
     return {"us_per_call": us, "algorithmic_bytes": all_bytes, "gbs": gbs, "frac": gbs / peak,
             "timing": "CUDA events around `steps` back-to-back calls, median over repeats, batches rotated"}
+
+
+def draft_stats_call_of(res, steps, peak):
+    """The verifier call with the draft rows' statistics supplied by the drafter: the statistics pass streams the
+    target rows alone, so the bytes the method must move shrink by the draft rows."""
+    if res.get("draft_stats_ms") is None:
+        return None
+    wl = res["wl"]
+    b0 = wl["batches"][0]
+    elem = b0.target.element_size()
+    all_bytes = elem * b0.V * b0.n_rows + 2 * elem * b0.V * res["n_rejected"]
+    us = 1e3 * res["draft_stats_ms"] / steps
+    gbs = all_bytes / (us * 1e-6) / 1e9
+    return {"us_per_call": us, "algorithmic_bytes": all_bytes, "gbs": gbs, "frac": gbs / peak,
+            "rows_per_s": b0.n_rows / (us * 1e-6),
+            "what": "dspark_verify_draft_stats: (reference, sum) of every draft row handed over by the drafter "
+                    "(computed outside the timed region, as a draft step leaves them); same timing rule as verify_call"}
 
 
 def main():
@@ -834,6 +876,7 @@ def main():
             "step_frac_of_peak": all_bytes / (ms / args.steps * 1e-3) / 1e9 / peak,
             "roofline": roofline_of(res, peak, peak_src),
             "verify_call": verify_call_of(res, args.steps, peak),
+            "verify_call_draft_stats": draft_stats_call_of(res, args.steps, peak),
             "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in res["kernels"].items()},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": res["e2e"]["h2d"],
                     "d2h_bytes_per_step": res["e2e"]["d2h"], "ms_per_step": e2e_ms / res["e2e"]["steps"],
@@ -863,6 +906,7 @@ def main():
                             "dominant_kernel": roof["kernel"], "dominant_kernel_gbs": roof["achieved"],
                             "dominant_kernel_frac": roof["frac"], "dominant_kernel_us": roof["us_per_launch"],
                             "verify_call": verify_call_of(res, args.steps, peak),
+            "verify_call_draft_stats": draft_stats_call_of(res, args.steps, peak),
                             "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in res["kernels"].items()},
                             "clocks": res["clocks"], "dev_status": res["dev_status"]}
         del res, wl

@@ -348,6 +348,54 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
                              void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
                              int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
 
+/* dspark_verify_draft_stats -- dspark_verify / dspark_verify_per_request for a caller whose drafter kept the softmax
+ * statistics of the draft rows it wrote (Section 2.1: the accept test needs q(x) = 2^(x_d * s - c_q) / Z_q, i.e. of a
+ * draft row only its logit at the draft token and the row's reference and sum).  The statistics pass then streams the
+ * target rows alone: on a batch with as many draft rows as cfg3 a third fewer bytes.  The draft rows themselves are
+ * still read where they are needed: one logit per position, and the whole row of a rejected position.
+ *   draft_row_stats   device fp32 [n_draft_rows_physical][2], 8-byte aligned, indexed like the rows of draft_logits
+ *                     (draft_row_start[r] + j, or the compact index): (c, Z) with s = log2(e) / T of the row's request,
+ *                     c = max(x) * s and Z = sum 2^(x * s - c) -- what dspark_markov_draft_step_stats and
+ *                     dspark_row_stats write.  A row whose entry is not a usable pair (NaN, Z <= 0) counts as a row
+ *                     that cannot be normalised (DSPARK_DEV_BAD_ROW for a request that looks at it).
+ *   temperature / temperatures   one T > 0, or device fp32 [R] (then `temperature` is ignored); the statistics must have
+ *                     been computed with the same temperatures
+ * Everything else as dspark_verify.  Losslessness rests on the statistics being those of the stored draft logits.
+ */
+int dspark_verify_draft_stats(const void* target_logits, const void* draft_logits, int dtype,
+                              int64_t target_row_stride, int64_t draft_row_stride, int V,
+                              const int32_t* row_offsets, const int64_t* draft_row_start,
+                              const int32_t* draft_tokens, const float* draft_row_stats, int R, int n_rows,
+                              float temperature, const float* temperatures, uint64_t seed,
+                              int32_t* accepted_len, int32_t* out_tokens,
+                              float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* dspark_row_stats -- the (c, Z) pair of dspark_verify_draft_stats for every row of a logit matrix, for a producer
+ * that has no statistics of its own: same blocks, block arithmetic and order of combination as the verifier, so the
+ * pair is what the verifier would have computed (Z rounded to fp32).  One read of the rows.
+ *   logits            device fp32 / bf16 [n_rows, >= V], row stride in elements
+ *   temperature / row_temperatures   one T > 0, or device fp32 [n_rows] (one per ROW; a value that is not positive and
+ *                     finite gives (NaN, NaN))
+ *   out_row_stats     device fp32 [n_rows][2], 8-byte aligned
+ * Errors: INVALID_ARG, SHAPE (more than 2 048 blocks of 4 KB per row), ALIGNMENT, CUDA.
+ */
+int dspark_row_stats(const void* logits, int dtype, int64_t row_stride, int V, int n_rows,
+                     float temperature, const float* row_temperatures, float* out_row_stats, void* stream);
+
+/* dspark_markov_draft_step_stats -- dspark_markov_draft_step that also hands out, per request, the statistics of the
+ * draft logits it has just written and drawn from (temperature > 0 only): out_row_stats[r * row_stats_stride] = (c, Z)
+ * as dspark_verify_draft_stats reads them (device fp32 pairs, 8-byte aligned; the stride, in pairs, lets position k of
+ * a block layout [R, block, V] write entry r * block + k).  They are by-products of the draw: nothing is read again.
+ */
+int dspark_markov_draft_step_stats(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                                   const int32_t* x_prev, int R, int V,
+                                   const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                                   float temperature, uint64_t seed,
+                                   void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
+                                   float* out_row_stats, int64_t row_stats_stride,
+                                   int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ------------------------------------------------------------------------------------
  * dspark_truncate_target -- top-k / top-p truncation of the target distribution, per request (Section 4.1
  * evaluates every model with its own suggested sampling settings; the paper states no rule of its own).

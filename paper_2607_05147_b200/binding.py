@@ -30,10 +30,10 @@ EXPORTS = [
     "dspark_schedule_async", "dspark_async_state_init",
     "dspark_verify_workspace_bytes", "dspark_verify_greedy", "dspark_verify", "dspark_uniforms",
     "dspark_verify_greedy_static", "dspark_verify_greedy_static_capacity", "dspark_verify_greedy_static_bytes",
-    "dspark_verify_per_request",
+    "dspark_verify_per_request", "dspark_verify_draft_stats", "dspark_row_stats",
     "dspark_accept_rate", "dspark_accept_rate_workspace_bytes",
     "dspark_markov_w2_packed_bytes", "dspark_markov_pack_w2", "dspark_markov_workspace_bytes",
-    "dspark_markov_logits", "dspark_markov_draft_step", "dspark_markov_set_epilogue_path",
+    "dspark_markov_logits", "dspark_markov_draft_step", "dspark_markov_draft_step_stats", "dspark_markov_set_epilogue_path",
     "dspark_truncate_target", "dspark_verify_truncated",
     "dspark_sts_workspace_bytes", "dspark_sts_calibrate", "dspark_sts_apply",
     "dspark_ktimer_create", "dspark_ktimer_destroy", "dspark_ktimer_attach", "dspark_ktimer_reset",
@@ -82,6 +82,9 @@ def lib() -> C.CDLL:
                                     vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_verify_per_request.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, vp, u64,
                                                 vp, vp, vp, vp, vp, vp, sz, vp]
+        L.dspark_verify_draft_stats.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, vp, i32, i32, C.c_float, vp, u64,
+                                                vp, vp, vp, vp, vp, vp, sz, vp]
+        L.dspark_row_stats.argtypes = [vp, i32, i64, i32, i32, C.c_float, vp, vp, vp]
         L.dspark_accept_rate_workspace_bytes.argtypes = [i32, i32, i32]
         L.dspark_accept_rate_workspace_bytes.restype = sz
         L.dspark_accept_rate.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, i32, i32, C.c_float, vp, vp, vp, sz, vp]
@@ -94,6 +97,8 @@ def lib() -> C.CDLL:
         L.dspark_markov_logits.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, vp, i64, vp, vp, vp, sz, vp]
         L.dspark_markov_draft_step.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, C.c_float, u64,
                                                vp, i64, vp, vp, vp, vp, sz, vp]
+        L.dspark_markov_draft_step_stats.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp, i64, i32, vp, C.c_float, u64,
+                                                     vp, i64, vp, vp, vp, i64, vp, vp, sz, vp]
         L.dspark_verify_truncated.argtypes = [vp, vp, i32, i64, i64, i32, vp, vp, vp, i32, i32, C.c_float, vp, vp, vp, u64,
                                               vp, vp, vp, vp, vp, vp, sz, vp]
         L.dspark_truncate_target.argtypes = [vp, i32, i64, i32, vp, i32, i32, vp, vp, C.c_float, vp, vp, vp, vp, vp]
@@ -465,6 +470,74 @@ def dspark_markov_draft_step(U: torch.Tensor, W1: torch.Tensor, W2_packed: torch
                                         _dev(dev_status, "dev_status", torch.int32),
                                         _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
     _check(rc, "dspark_markov_draft_step")
+
+
+def dspark_markov_draft_step_stats(U: torch.Tensor, W1: torch.Tensor, W2_packed: torch.Tensor, x_prev: torch.Tensor,
+                                   temperature: float, seed: int, *,
+                                   H: Optional[torch.Tensor] = None, w_conf: Optional[torch.Tensor] = None,
+                                   out_logits: torch.Tensor, out_tokens: torch.Tensor,
+                                   out_conf: Optional[torch.Tensor] = None,
+                                   out_row_stats: torch.Tensor, row_stats_stride: int = 1,
+                                   dev_status: torch.Tensor, workspace: torch.Tensor) -> None:
+    """The draft step that also writes (c, Z) of request r's draft row to out_row_stats[r * row_stats_stride] (fp32 pairs)."""
+    head = _markov_args(U, W1, W2_packed, x_prev, H, w_conf, out_logits, out_conf)
+    R = head[5]
+    if out_tokens.numel() < R:
+        raise DsparkError("out_tokens is too small")
+    if out_row_stats.numel() < 2 * ((R - 1) * int(row_stats_stride) + 1):
+        raise DsparkError("out_row_stats is too small")
+    rc = lib().dspark_markov_draft_step_stats(*head, float(temperature), int(seed) & (2**64 - 1),
+                                              _dev(out_logits, "out_logits", torch.bfloat16), out_logits.stride(0),
+                                              _dev(out_tokens, "out_tokens", torch.int32),
+                                              _dev(out_conf, "out_conf", torch.float32),
+                                              _dev(out_row_stats, "out_row_stats", torch.float32), int(row_stats_stride),
+                                              _dev(dev_status, "dev_status", torch.int32),
+                                              _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_markov_draft_step_stats")
+
+
+def dspark_row_stats(logits: torch.Tensor, temperature: float = 1.0, *, row_temperatures: Optional[torch.Tensor] = None,
+                     out_row_stats: torch.Tensor) -> None:
+    """(c, Z) of every row of `logits` as the verifier computes them: out_row_stats is CUDA float32 [n_rows, 2]."""
+    lp, code, ls = _logits(logits, "logits")
+    n_rows = logits.shape[0]
+    if out_row_stats.numel() < 2 * n_rows or (row_temperatures is not None and row_temperatures.numel() < n_rows):
+        raise DsparkError("out_row_stats needs two floats per row, row_temperatures one")
+    rc = lib().dspark_row_stats(lp, code, ls, logits.shape[1], n_rows, float(temperature),
+                                _dev(row_temperatures, "row_temperatures", torch.float32),
+                                _dev(out_row_stats, "out_row_stats", torch.float32), _stream())
+    _check(rc, "dspark_row_stats")
+
+
+def dspark_verify_draft_stats(target: torch.Tensor, draft: torch.Tensor, row_offsets: torch.Tensor,
+                              draft_tokens: torch.Tensor, draft_row_stats: torch.Tensor, seed: int, *,
+                              temperature: float = 1.0, temperatures: Optional[torch.Tensor] = None,
+                              draft_row_start: Optional[torch.Tensor] = None,
+                              accepted_len: torch.Tensor, out_tokens: torch.Tensor,
+                              out_p_tok: Optional[torch.Tensor] = None, out_q_tok: Optional[torch.Tensor] = None,
+                              dev_status: Optional[torch.Tensor], workspace: torch.Tensor,
+                              n_rows: Optional[int] = None) -> None:
+    """Sampling verification with the draft rows' statistics supplied (CUDA float32 [physical draft rows, 2])."""
+    tp, code, ts = _logits(target, "target")
+    dp, dcode, ds = _logits(draft, "draft")
+    if code != dcode or target.shape[1] != draft.shape[1]:
+        raise DsparkError("target and draft logits must share dtype and vocabulary size")
+    R = row_offsets.numel() - 1
+    if temperatures is not None and temperatures.numel() != R:
+        raise DsparkError("temperatures must have one entry per request")
+    if draft_row_stats.numel() < 2 * draft.shape[0]:
+        raise DsparkError("draft_row_stats needs two floats per draft row")
+    n_rows = target.shape[0] if n_rows is None else n_rows
+    rc = lib().dspark_verify_draft_stats(
+        tp, dp, code, ts, ds, target.shape[1], _dev(row_offsets, "row_offsets", torch.int32),
+        _dev(draft_row_start, "draft_row_start", torch.int64), _dev(draft_tokens, "draft_tokens", torch.int32),
+        _dev(draft_row_stats, "draft_row_stats", torch.float32), R, n_rows, float(temperature),
+        _dev(temperatures, "temperatures", torch.float32), int(seed) & 0xFFFFFFFFFFFFFFFF,
+        _dev(accepted_len, "accepted_len", torch.int32), _dev(out_tokens, "out_tokens", torch.int32),
+        _dev(out_p_tok, "out_p_tok", torch.float32), _dev(out_q_tok, "out_q_tok", torch.float32),
+        _dev(dev_status, "dev_status", torch.int32), _dev(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), _stream())
+    _check(rc, "dspark_verify_draft_stats")
 
 
 def dspark_truncate_target(target: torch.Tensor, row_offsets: torch.Tensor, *, top_k: Optional[torch.Tensor] = None,

@@ -66,6 +66,7 @@ struct MarkovParams {
     int32_t* dev_status;
     float2* stats;                            // workspace: per (row, vocabulary tile) statistics of the stored logits
     float scale2;                             // log2(e) / T
+    float2* out_row_stats; long long row_stats_stride;   // optional: (reference, sum) of every stored row for the verifier
     int l2_hints;                             // 1: keep W2 in L2, stream the logits through it (small launches only)
 };
 
@@ -768,6 +769,12 @@ __global__ void __launch_bounds__(kDrawThreads) markov_draw_kernel(MarkovParams 
     float wbase = 0.f, Z = 0.f;
 #pragma unroll
     for (int w = 0; w < kDrawThreads / 32; ++w) { if (w < warp) wbase += s_red[w]; Z += s_red[w]; }
+    // the statistics the sampling verifier would compute from this row: reference max * scale (log2 domain) and the sum
+    // of 2^(x * scale - reference); a row that cannot be normalised hands out NaN and is reported by the verifier too
+    if (tid == 0 && P.out_row_stats) {
+        const bool unusable = bad || !(Z > 0.f) || Z == INFINITY;
+        P.out_row_stats[(long long)r * P.row_stats_stride] = unusable ? make_float2(NAN, NAN) : make_float2(offM, Z);
+    }
     if (bad || !(Z > 0.f) || Z == INFINITY) {
         if (tid == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW); out_tokens[r] = -1; }
         return;
@@ -952,6 +959,7 @@ static int markov_launch(const void* U, int64_t u_row_stride, const void* W1, co
     P.out_conf = out_conf; P.dev_status = dev_status;
     P.stats = (float2*)((unsigned char*)workspace + w.stats);
     P.l2_hints = 0;
+    P.out_row_stats = nullptr; P.row_stats_stride = 0;
     P.scale2 = stats_mode == 1 ? (float)(1.4426950408889634 / (double)temperature) : 0.f;
     if (params_out) *params_out = P;
 
@@ -1019,11 +1027,47 @@ int dspark_markov_logits(const void* U, int64_t u_row_stride, const void* W1, co
     return launch_status();
 }
 
+static int draft_step_launch(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                             const int32_t* x_prev, int R, int V,
+                             const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                             float temperature, uint64_t seed,
+                             void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
+                             float* out_row_stats, int64_t row_stats_stride,
+                             int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
+
 int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
                              const int32_t* x_prev, int R, int V,
                              const void* H, int64_t h_row_stride, int d, const float* w_conf,
                              float temperature, uint64_t seed,
                              void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
+                             int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return draft_step_launch(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf, temperature, seed,
+                             out_logits, out_row_stride, out_tokens, out_conf, nullptr, 0, dev_status, workspace,
+                             workspace_bytes, stream);
+}
+
+int dspark_markov_draft_step_stats(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                                   const int32_t* x_prev, int R, int V,
+                                   const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                                   float temperature, uint64_t seed,
+                                   void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
+                                   float* out_row_stats, int64_t row_stats_stride,
+                                   int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!out_row_stats || row_stats_stride < 1 || !(temperature > 0.f)) return DSPARK_ERR_INVALID_ARG;
+    if (((uintptr_t)out_row_stats & 7u) != 0) return DSPARK_ERR_ALIGNMENT;
+    return draft_step_launch(U, u_row_stride, W1, W2_packed, x_prev, R, V, H, h_row_stride, d, w_conf, temperature, seed,
+                             out_logits, out_row_stride, out_tokens, out_conf, out_row_stats, row_stats_stride, dev_status,
+                             workspace, workspace_bytes, stream);
+}
+
+static int draft_step_launch(const void* U, int64_t u_row_stride, const void* W1, const void* W2_packed,
+                             const int32_t* x_prev, int R, int V,
+                             const void* H, int64_t h_row_stride, int d, const float* w_conf,
+                             float temperature, uint64_t seed,
+                             void* out_logits, int64_t out_row_stride, int32_t* out_tokens, float* out_conf,
+                             float* out_row_stats, int64_t row_stats_stride,
                              int32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream)
 {
     if (!out_tokens || !(temperature >= 0.f) || isinf(temperature)) return DSPARK_ERR_INVALID_ARG;
@@ -1034,6 +1078,7 @@ int dspark_markov_draft_step(const void* U, int64_t u_row_stride, const void* W1
                                  out_row_stride, out_conf, dev_status, workspace, workspace_bytes, (cudaStream_t)stream,
                                  greedy ? 2 : 1, temperature, &P);
     if (rc != DSPARK_OK) return rc;
+    P.out_row_stats = (float2*)out_row_stats; P.row_stats_stride = row_stats_stride;
     {
         KernelTimerScope timer(DSPARK_K_MARKOV_DRAW, (cudaStream_t)stream);
         launch_pdl(markov_draw_kernel, dim3(R), dim3(kDrawThreads), 0, (cudaStream_t)stream, P, greedy, seed, out_tokens);

@@ -437,6 +437,54 @@ __global__ void __launch_bounds__(256) trunc_sums_kernel(VerifyParams P, TruncAr
 }
 
 // ---------------------------------------------------------------------------------------
+// Row statistics on their own (dspark_row_stats): what the statistics pass and the accept kernel compute for a row,
+// (reference, sum) = (max * scale, sum 2^(x * scale - reference)), for a caller that produces logits and wants to hand
+// their statistics to dspark_verify_draft_stats.  One CTA per row; same blocks, same block arithmetic and same order
+// of combination as the verifier, so the result is bit-identical to what the verifier would have computed.
+// ---------------------------------------------------------------------------------------
+constexpr int kRowStatsThreads = 256;
+constexpr int kRowStatsMaxBlocks = 2048;
+template <int kElem>
+__global__ void __launch_bounds__(kRowStatsThreads) row_stats_kernel(const unsigned char* logits, long long stride_bytes, int V,
+                                                                      int n_rows, float temperature, const float* row_temperatures,
+                                                                      float2* out)
+{
+    __shared__ float2 s_e[kRowStatsMaxBlocks];
+    pdl_wait();
+    const int row = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (row >= n_rows) return;
+    const float T = row_temperatures ? row_temperatures[row] : temperature;
+    if (!(T > 0.f) || !(T < INFINITY)) {
+        if (threadIdx.x == 0) out[row] = make_float2(NAN, NAN);
+        return;
+    }
+    const float scale = (float)(1.4426950408889634 / (double)T);
+    const int row_bytes = V * kElem;
+    const int nblk = blocks_per_row(V, kElem, kStatBlockBytes);
+    const unsigned char* base = logits + (long long)row * stride_bytes;
+    for (int b = warp; b < nblk; b += kRowStatsThreads / 32) {
+        const int rem = row_bytes - b * kStatBlockBytes;
+        uint4 v[kStatVec];
+        load_block<kElem, kStatVec>(GlobalFetch<kElem>{base + (long long)b * kStatBlockBytes}, rem < kStatBlockBytes ? rem : kStatBlockBytes, lane, v);
+        const float2 e = block_stats<kElem, kStatVec>(v, scale);
+        if (lane == 0) s_e[b] = e;
+    }
+    __syncthreads();
+    if (warp != 0) return;
+    RowAcc A;
+    A.init();
+    for (int b0 = 0; b0 < nblk; b0 += 128) {
+        float2 e[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { const int i = b0 + k * 32 + lane; e[k] = i < nblk ? s_e[i] : make_float2(kNegInf, 0.f); }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) A.add(e[k]);
+    }
+    A.finish();
+    if (lane == 0) out[row] = make_float2(A.C, (float)A.S);
+}
+
+// ---------------------------------------------------------------------------------------
 // Per-request temperatures: expands T_r into one exponent scale log2(e)/T_r per target row and per
 // draft row (the streamed pass walks rows, not requests).  One thread per request.
 // ---------------------------------------------------------------------------------------
@@ -525,8 +573,16 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
                 }
             }
             RowAcc A, D;
-            combine_rows(P.stats_t + (long long)(lo + j) * P.nblk,
-                         is_draft_pos ? P.stats_d + (long long)(lo - r + j) * P.nblk : nullptr, P.nblk, lane, A, D);
+            if (P.draft_stats) {
+                // the drafter kept the statistics of the rows it wrote: nothing of the draft row was streamed
+                float2 ds = make_float2(kNegInf, 0.f);
+                if (is_draft_pos) ds = __ldg(&P.draft_stats[drow0 + j]);
+                combine_rows(P.stats_t + (long long)(lo + j) * P.nblk, nullptr, P.nblk, lane, A, D);
+                D.C = ds.x; D.S = (double)ds.y;
+            } else {
+                combine_rows(P.stats_t + (long long)(lo + j) * P.nblk,
+                             is_draft_pos ? P.stats_d + (long long)(lo - r + j) * P.nblk : nullptr, P.nblk, lane, A, D);
+            }
             if (!is_draft_pos) {
                 // bonus row: leave its block masses (relative to the row reference) where the finalize
                 // kernel looks for block values; a rejected request overwrites them in the residual pass
@@ -930,6 +986,7 @@ static int fill_common(VerifyParams& P, const void* target, const void* draft, i
     P.resid_cap = R;
     P.req_temp = nullptr;
     P.tau = nullptr;
+    P.draft_stats = nullptr;
     return DSPARK_OK;
 }
 
@@ -1040,7 +1097,7 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
                          int32_t* accepted_len, int32_t* out_tokens,
                          float* out_p_tok, float* out_q_tok, int32_t* dev_status,
                          void* workspace, size_t workspace_bytes, void* stream,
-                         const int32_t* top_k = nullptr, const float* top_p = nullptr)
+                         const int32_t* top_k = nullptr, const float* top_p = nullptr, const float* draft_row_stats = nullptr)
 {
     if (!draft_logits) return DSPARK_ERR_INVALID_ARG;
     const bool truncate = top_k || top_p;
@@ -1056,6 +1113,7 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
     P.seed = seed;
     P.out_p = out_p_tok;
     P.out_q = out_q_tok;
+    P.draft_stats = (const float2*)draft_row_stats;
     cudaStream_t s = (cudaStream_t)stream;
     const int path = g_stream_path.load(std::memory_order_relaxed);
     const bool bulk = path != 1 && aligned16(P.target, P.tstride_bytes, P.row_bytes) &&
@@ -1067,7 +1125,7 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
     }
     {
         KernelTimerScope timer(DSPARK_K_STREAM, s);
-        launch_stream_dtype<kModeStats>(P, bulk, (2ll * n_rows - R) * pieces(P.nblk), s);
+        launch_stream_dtype<kModeStats>(P, bulk, (draft_row_stats ? (long long)n_rows : 2ll * n_rows - R) * pieces(P.nblk), s);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     if (truncate && dtype == DSPARK_F32) {
@@ -1210,6 +1268,42 @@ int dspark_verify_per_request(const void* target_logits, const void* draft_logit
     return verify_launch(target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V, row_offsets,
                          draft_row_start, draft_tokens, R, n_rows, 1.0f, temperatures, seed, accepted_len,
                          out_tokens, out_p_tok, out_q_tok, dev_status, workspace, workspace_bytes, stream);
+}
+
+int dspark_row_stats(const void* logits, int dtype, int64_t row_stride, int V, int n_rows,
+                     float temperature, const float* row_temperatures, float* out_row_stats, void* stream)
+{
+    if (!logits || !out_row_stats || n_rows < 1 || V < 1 || row_stride < V) return DSPARK_ERR_INVALID_ARG;
+    if (dtype != DSPARK_F32 && dtype != DSPARK_BF16) return DSPARK_ERR_INVALID_ARG;
+    if (!row_temperatures && (!(temperature > 0.0f) || !isfinite(temperature))) return DSPARK_ERR_INVALID_ARG;
+    const int elem = dtype == DSPARK_BF16 ? 2 : 4;
+    if ((long long)V * elem >= (1ll << 31) || blocks_per_row(V, elem, kStatBlockBytes) > kRowStatsMaxBlocks) return DSPARK_ERR_SHAPE;
+    if (((uintptr_t)out_row_stats & 7u) != 0 || ((uintptr_t)logits & (uintptr_t)(elem - 1)) != 0) return DSPARK_ERR_ALIGNMENT;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (elem == 2)
+        launch_pdl(row_stats_kernel<2>, dim3(n_rows), dim3(kRowStatsThreads), 0, s, (const unsigned char*)logits,
+                   (long long)row_stride * elem, V, n_rows, temperature, row_temperatures, (float2*)out_row_stats);
+    else
+        launch_pdl(row_stats_kernel<4>, dim3(n_rows), dim3(kRowStatsThreads), 0, s, (const unsigned char*)logits,
+                   (long long)row_stride * elem, V, n_rows, temperature, row_temperatures, (float2*)out_row_stats);
+    return launch_status();
+}
+
+int dspark_verify_draft_stats(const void* target_logits, const void* draft_logits, int dtype,
+                              int64_t target_row_stride, int64_t draft_row_stride, int V,
+                              const int32_t* row_offsets, const int64_t* draft_row_start,
+                              const int32_t* draft_tokens, const float* draft_row_stats, int R, int n_rows,
+                              float temperature, const float* temperatures, uint64_t seed,
+                              int32_t* accepted_len, int32_t* out_tokens,
+                              float* out_p_tok, float* out_q_tok, int32_t* dev_status,
+                              void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!draft_row_stats) return DSPARK_ERR_INVALID_ARG;
+    if (((uintptr_t)draft_row_stats & 7u) != 0) return DSPARK_ERR_ALIGNMENT;
+    return verify_launch(target_logits, draft_logits, dtype, target_row_stride, draft_row_stride, V, row_offsets,
+                         draft_row_start, draft_tokens, R, n_rows, temperatures ? 1.0f : temperature, temperatures, seed,
+                         accepted_len, out_tokens, out_p_tok, out_q_tok, dev_status, workspace, workspace_bytes, stream,
+                         nullptr, nullptr, draft_row_stats);
 }
 
 int dspark_verify_truncated(const void* target_logits, const void* draft_logits, int dtype,

@@ -79,6 +79,8 @@ struct VerifyParams {
     unsigned long long launch_tag;            // unique per call: see unit_counter()
     float* wblk;                              // per request: residual block sums
     const float* tau;                         // per target row: top-k / top-p threshold (NULL: no truncation)
+    const float2* draft_stats;                // per physical draft row: (reference, sum) handed over by the drafter (NULL:
+                                              // the statistics pass streams the draft rows as well)
     TruncRow* trunc_rows;                     // workspace of the streamed threshold search
     unsigned int* trunc_bins;                 // [n_rows][kHistBins] key counts
     int32_t* trunc_flag;                      // [n_rows] 1: the window did not resolve the row (per-row search)
@@ -121,7 +123,7 @@ __device__ __forceinline__ long long draft_phys_row(const VerifyParams& P, int d
 template <int kMode>
 __device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
 {
-    if (kMode == kModeStats) return n_rows + (n_rows > P.R ? n_rows - P.R : 0);
+    if (kMode == kModeStats) return n_rows + ((n_rows > P.R && !P.draft_stats) ? n_rows - P.R : 0);
     if (kMode == kModeGreedy || kMode == kModeHist) return n_rows;
     const int nq = __ldcg(&P.counters[0]);
     return nq > P.resid_cap ? P.resid_cap : (nq < 0 ? 0 : nq);
