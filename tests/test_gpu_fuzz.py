@@ -45,6 +45,13 @@ def test_sampling_fuzz(seed):
             temps = torch.from_numpy(rng.uniform(0.4, 1.8, size=R).astype(np.float32)).cuda()
         _, _, mism = H.check_sampling(b, want_probs=bool(rng.random() < 0.7), temperatures=temps)
         total_mism += mism
+        if temps is None and seed != 1416:
+            # the same batch with the draft rows' statistics handed over instead of streamed
+            import test_gpu_draft_stats as DS
+            want_probs = bool(rng.random() < 0.5)
+            g = DS._verify_with_stats(b, DS._stats(b.draft, b.temperature), want_probs=want_probs)
+            total_mism += H.compare_sampling(g, H.oracle_verify(b, eval_all=want_probs), b.row_offsets.cpu().numpy(),
+                                             check_probs=want_probs)
     assert total_mism <= 1
 
 
