@@ -489,6 +489,7 @@ def bench_markov(args, device, rank, world, dist, barrier):
     timer.detach()
     kernels = timer.read()
     timer.close()
+
     # the contraction kernel alone, launched back to back (no events between launches: an event pair around
     # one launch adds several microseconds of launch latency that the stream normally hides)
     def logits_only(i):
@@ -601,6 +602,27 @@ def measure_workload(name, args, device, rank, local_rank, world, dist, barrier,
     vt = sorted(timed_loop(verify_only, steps) for _ in range(max(5, repeats // 5)))
     verify_ms = replicas.max_over_ranks([vt[len(vt) // 2]], dist, device)[0]
 
+    # keep the same load running until the clock sampler has seen enough of it (not timed)
+    t_end = time.perf_counter() + 1.0
+    i = 0
+    while time.perf_counter() < t_end and len(sampler.samples) < 40:
+        step.run(batches[i % n_sets]); i += 1
+        if i % 64 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+
+    # per-kernel timing of the same steps (events around every launch of the library)
+    n_inst = max(steps, 200)                                 # averages per launch: a short --steps run still sees 200 launches
+    timer = B.KernelTimer(n_inst * 12)
+    timer.attach()
+    for i in range(n_inst):
+        step.run(batches[i % n_sets])
+    torch.cuda.synchronize()
+    timer.detach()
+    kernels = timer.read()
+    timer.close()
+
     # the same call when the drafter hands over the statistics of its rows (dspark_verify_draft_stats): the pairs are
     # computed once, outside the timed region, the way a draft step leaves them behind
     draft_stats_ms = None
@@ -624,26 +646,6 @@ def measure_workload(name, args, device, rank, local_rank, world, dist, barrier,
         dt = sorted(timed_loop(verify_stats, steps) for _ in range(max(5, repeats // 5)))
         draft_stats_ms = replicas.max_over_ranks([dt[len(dt) // 2]], dist, device)[0]
         assert int(step.status.item()) == dev_status
-
-    # keep the same load running until the clock sampler has seen enough of it (not timed)
-    t_end = time.perf_counter() + 1.0
-    i = 0
-    while time.perf_counter() < t_end and len(sampler.samples) < 40:
-        step.run(batches[i % n_sets]); i += 1
-        if i % 64 == 0:
-            torch.cuda.synchronize()
-    torch.cuda.synchronize()
-    clocks = sampler.finish()
-
-    # per-kernel timing of the same steps (events around every launch of the library)
-    timer = B.KernelTimer(steps * 12)
-    timer.attach()
-    for i in range(steps):
-        step.run(batches[i % n_sets])
-    torch.cuda.synchronize()
-    timer.detach()
-    kernels = timer.read()
-    timer.close()
 
     res = dict(wl=wl, step=step, ms=ms, ms_min=ms_min, repeats=repeats, timed_ms=sum(times), verify_ms=verify_ms,
                draft_stats_ms=draft_stats_ms,

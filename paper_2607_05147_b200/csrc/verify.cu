@@ -509,6 +509,8 @@ __global__ void __launch_bounds__(256) row_scale_kernel(VerifyParams P)
 // Position j = len is the bonus row (statistics only).  Every request leaves a record for the
 // finalize kernel; a rejected one is also queued for the residual pass.
 // ---------------------------------------------------------------------------------------
+// kDraftStats: the draft rows' (reference, sum) come from the drafter (P.draft_stats) instead of the statistics pass.
+template <bool kDraftStats>
 __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
 {
     constexpr int kWarps = kDecideThreads / 32;
@@ -573,7 +575,7 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
                 }
             }
             RowAcc A, D;
-            if (P.draft_stats) {
+            if (kDraftStats) {
                 // the drafter kept the statistics of the rows it wrote: nothing of the draft row was streamed
                 float2 ds = make_float2(kNegInf, 0.f);
                 if (is_draft_pos) ds = __ldg(&P.draft_stats[drow0 + j]);
@@ -1157,7 +1159,8 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
     }
     {
         KernelTimerScope timer(DSPARK_K_DECIDE, s);
-        launch_pdl(decide_kernel, dim3(R), dim3(kDecideThreads), 0, s, P);
+        if (P.draft_stats) launch_pdl(decide_kernel<true>, dim3(R), dim3(kDecideThreads), 0, s, P);
+        else launch_pdl(decide_kernel<false>, dim3(R), dim3(kDecideThreads), 0, s, P);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
