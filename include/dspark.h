@@ -238,8 +238,10 @@ int dspark_verify_greedy_static(const void* target_logits, int dtype, int64_t ta
  * drawn from; with out_p_tok / out_q_tok every draft position is evaluated and an unusable row at any of them
  * voids the request.  A request reports every bit that applies to it.  Logits must be small enough for
  * x * log2(e) / T to stay finite in fp32 (|x| / T below about 2e38); larger finite values count as infinite.
- * Streams every target and draft row once (online softmax statistics per 4 KB block), then
- * re-reads only the rejected position's row pair of each rejected request.
+ * Streams the target and draft row of every draft position once (online softmax statistics per 4 KB block),
+ * then in a second pass re-reads the rejected position's row pair of each rejected request and reads the bonus row
+ * of each request that accepted every draft token (the bonus row of a rejected request is never needed and never
+ * read; with a truncated target, direct loads or more than 2 048 requests all bonus rows go through the first pass).
  * Errors: INVALID_ARG, SHAPE, WORKSPACE, CUDA.
  */
 int dspark_verify(const void* target_logits, const void* draft_logits, int dtype,
@@ -500,10 +502,10 @@ int dspark_ktimer_attach(dspark_ktimer_t* t);
 int dspark_ktimer_reset(dspark_ktimer_t* t);
 int dspark_ktimer_read(dspark_ktimer_t* t, int kernel_id, float* total_ms, int* launches);
 
-/* Diagnostic switch for the verifiers: 0 = automatic (the single-launch kernel with its bulk-copy
- * pipeline when the 16-byte rules hold, separate passes with direct loads otherwise), 1 = always
- * separate passes with direct loads, 2 = separate passes with bulk copies.  Results are the same
- * up to fp32 summation order.  Process-wide (an atomic); the paper has no counterpart. */
+/* Diagnostic switch for the verifiers: 0 = automatic (the bulk-copy pipeline when the 16-byte rules hold,
+ * direct loads otherwise), 1 = always direct loads, 2 = bulk copies; add 16 to stream every bonus row in the
+ * statistics pass instead of only the needed ones in the second pass (the earlier order).  Results are the same
+ * (direct loads: up to fp32 summation order).  Process-wide (atomics); the paper has no counterpart. */
 int dspark_set_stream_path(int path);
 
 /* Diagnostic: how many polls the streamed passes of the verifiers spend on an entry wait (a consumer warp

@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     const int n_rows = device_rows(P, &bad_rows);
     if (kMode != kModeResid && kMode != kModeHist && blockIdx.x == 0 && tid == 0) {
         P.counters[0] = 0;                       // residual queue, filled by the decide kernel
+        P.counters[kCtrBonus] = 0;               // and the bonus rows it queues from the back
         *unit_counter<kModeResid>(P) = 0ull;     // unit counters of the passes that follow this one in the call
         *unit_counter<kModeHist>(P) = 0ull;
         *unit_counter<kMode>(P) = 0ull;          // and this pass's own, published by the tag
@@ -64,8 +65,26 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     const int n_streams = stream_count<kMode>(P, n_rows);
     const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
     const int ppr = (nblk + kConsumerWarps - 1) / kConsumerWarps;
-    const long long total = (long long)n_streams * ppr;
+    // the second pass also streams the bonus rows queued from the back of the task array, in 32 KB pieces
+    const int ppr_b = (P.nblk + kConsumerWarps - 1) / kConsumerWarps;
+    int n_bonus = 0;
+    if (kMode == kModeResid && P.skip_bonus) {
+        n_bonus = __ldcg(&P.counters[kCtrBonus]);
+        n_bonus = n_bonus < 0 ? 0 : (n_bonus > P.resid_cap - n_streams ? P.resid_cap - n_streams : n_bonus);
+    }
+    const long long total_first = (long long)n_streams * ppr;
+    const long long total = total_first + (long long)n_bonus * ppr_b;
     volatile int* abort_flag = &s_abort;
+    // Statistics pass without the bonus rows: the target rows that are not bonus rows are, in order, the draft
+    // positions of the batch, so stream s' of them is target row s' + r for the request r it falls into.  Every CTA
+    // keeps row_offsets[r] - r behind its stages (one coalesced read) and finds r by a search in shared memory.
+    int* pref = reinterpret_cast<int*>(stage_mem + kStages * kStageBytes);
+    const bool skip_bonus = kMode == kModeStats && P.skip_bonus;
+    const int nd = n_rows > P.R ? n_rows - P.R : 0;
+    if (skip_bonus) {
+        for (int r = tid; r <= P.R; r += kStreamThreads) pref[r] = P.row_offsets[r] - r;
+        __syncthreads();
+    }
 
     if (warp == kConsumerWarps) {
         // ---------------- producer warp: lane 0 draws the units and issues the copies ----
@@ -89,13 +108,35 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
             const unsigned char *src0 = nullptr, *src1 = nullptr;
             int bytes = 0;
             if (lane == 0) {
-                if (live) {
+                if (live && kMode == kModeResid && u >= total_first) {
+                    // a bonus row: task from the back of the queue, one 32 KB piece of the target row
+                    const long long v = u - total_first;
+                    const int tb = (int)(v / ppr_b);
+                    slot.s = P.resid_cap - 1 - tb;
+                    slot.piece = (int)(v - (long long)tb * ppr_b);
+                    slot.task = P.resid[slot.s];
+                    slot.scale = slot.task.scale;
+                    const long long off = (long long)slot.piece * kStageBytes;
+                    const long long rem = (long long)P.row_bytes - off;
+                    bytes = (int)(rem < kStageBytes ? rem : kStageBytes);
+                    src0 = P.target + (long long)slot.task.row_t * P.tstride_bytes + off;
+                } else if (live) {
                     slot.s = total <= 0x7fffffffll ? (int)((unsigned)u / (unsigned)ppr) : (int)(u / ppr);
                     slot.piece = (int)(u - (long long)slot.s * ppr);
+                    if (skip_bonus) {
+                        if (slot.s < nd) {
+                            int lo = 0, hi = P.R;        // largest r with row_offsets[r] - r <= s'
+                            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (pref[mid] <= slot.s) lo = mid; else hi = mid; }
+                            slot.s += lo;
+                            if (slot.s >= n_rows) slot.s = n_rows - 1;      // only with inconsistent offsets
+                        } else {
+                            slot.s = n_rows + (slot.s - nd);
+                        }
+                    }
                     if (kMode == kModeResid) slot.task = P.resid[slot.s];
                     if (kMode == kModeHist) slot.trunc = P.trunc_rows[slot.s];
                     unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes, kMode == kModeResid ? &slot.task : nullptr);
-                    slot.scale = stream_scale<kMode>(P, slot.s, n_rows, n_streams);
+                    slot.scale = stream_scale<kMode>(P, slot.s, n_rows, n_streams + (skip_bonus ? P.R : 0));
                 } else {
                     slot.s = -1; slot.piece = 0; slot.scale = 0.f;
                 }
@@ -112,9 +153,10 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 if (kMode == kModeHist) s_unit[st].trunc = slot.trunc;
                 if (live) {
                     unsigned char* dst = stage_mem + st * kStageBytes;
-                    mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(bytes * M::kSrc));
+                    const bool two = M::kSrc == 2 && src1 != nullptr;
+                    mbar_arrive_expect_tx(&full_bar[st], (uint32_t)(two ? 2 * bytes : bytes));
                     bulk_g2s_hint(dst, src0, (uint32_t)bytes, &full_bar[st], pol_first);
-                    if (M::kSrc == 2) bulk_g2s_hint(dst + M::kPieceBytes, src1, (uint32_t)bytes, &full_bar[st], pol_first);
+                    if (two) bulk_g2s_hint(dst + M::kPieceBytes, src1, (uint32_t)bytes, &full_bar[st], pol_first);
                     if (!counter_ready && !(counter_ready = wait_for_tag(unit_tag(P), P.launch_tag, entry_limit))) {
                         atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT);
                         *abort_flag = 1;
@@ -559,9 +601,11 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     }
     const double scale_d = (double)scale_f;
 
-    for (int j0 = 0; j0 <= len; j0 += kWarps) {
+    // (P.skip_bonus: the bonus row has not been streamed; it is looked at by the draw kernel if the request gets there)
+    const int last_pos = P.skip_bonus ? len - 1 : len;
+    for (int j0 = 0; j0 <= last_pos; j0 += kWarps) {
         const int j = j0 + warp;
-        if (j <= len) {
+        if (j <= last_pos) {
             const bool is_draft_pos = j < len;
             // the two logits at the draft token do not depend on the statistics: fetch them first
             float xt = 0.f, xd = 0.f;
@@ -643,8 +687,28 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
     rec.cp = rec.cq = 0.f; rec.inv_zp = rec.inv_zq = 1.f; rec.u = 0.f; rec.scale = scale_f; rec.pad = 0;
     rec.tau = kNegInf;
     const bool void_req = want_all ? s_first_bad != 0x7fffffff : s_first_bad < n;
-    if (void_req || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
-        (n < len && !row_usable(s_fin_C[1], s_fin_S[1]))) {
+    const bool bonus_later = P.skip_bonus && n == len;         // every draft token accepted, its bonus row not seen yet
+    if (bonus_later) {
+        if (void_req) {
+            atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW);
+            P.accepted_len[r] = 0;
+        } else {
+            // queue the bonus row for the second pass (one source: row_d < 0); the draw kernel combines its statistics
+            for (int i = 0; i < n; ++i) P.out_tokens[lo + i] = P.draft_tokens[lo + i];
+            float ua, ur;
+            philox_uniforms(P.seed, (uint32_t)r, (uint32_t)n, ua, ur);
+            P.accepted_len[r] = n;
+            rec.u = ur;
+            rec.kind = kTaskBonus;
+            const int slot = P.resid_cap - 1 - atomicAdd(&P.counters[kCtrBonus], 1);
+            ResidTask q;
+            q.request = r; q.row_t = rec.row_t; q.row_d = -1;
+            q.cp = q.cq = 0.f; q.inv_zp = q.inv_zq = 1.f;
+            q.u = ur; q.scale = scale_f; q.wslot = r; q.tau = kNegInf;
+            P.resid[slot] = q;
+        }
+    } else if (void_req || !s_have_fin || !row_usable(s_fin_C[0], s_fin_S[0]) ||
+               (n < len && !row_usable(s_fin_C[1], s_fin_S[1]))) {
         atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW);
         P.accepted_len[r] = 0;
     } else {
@@ -699,7 +763,23 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
     const double u = (double)rec.u;
     const unsigned char* trow = P.target + (long long)rec.row_t * P.tstride_bytes;
     int token = -1;
-    for (int attempt = 0; attempt < 2 && token < 0; ++attempt) {
+    // A bonus row that the second pass has streamed (P.skip_bonus): its row statistics are combined here, and here
+    // it turns out whether the row can be normalised at all; its block masses then come from the saved statistics
+    // exactly as on the second attempt of a rejected row below.
+    const bool late_bonus = P.skip_bonus && rec.kind == kTaskBonus;
+    float cp = rec.cp;
+    if (late_bonus) {
+        RowAcc A, D;
+        combine_rows(P.stats_t + (long long)rec.row_t * P.nblk, nullptr, P.nblk, lane, A, D);
+        if (!row_usable(A.C, A.S)) {
+            const int lo = P.row_offsets[r], hi = P.row_offsets[r + 1];
+            for (int i = lo + lane; i < hi; i += 32) P.out_tokens[i] = -1;
+            if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_BAD_ROW); P.accepted_len[r] = 0; }
+            return;
+        }
+        cp = A.C;
+    }
+    for (int attempt = late_bonus ? 1 : 0; attempt < 2 && token < 0; ++attempt) {
         const bool resid = (rec.kind == kTaskResid) && attempt == 0;
         const int n1 = resid ? P.nblk_r : P.nblk;
         if (attempt == 1) {
@@ -710,7 +790,7 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
             for (int k = 0; k < 8; ++k) {
                 const int i = k * 32 + lane;
                 float m = 0.f;
-                if (i < P.nblk && P.nblk <= 256) { const float2 e = __ldcg(&st[i]); m = e.x > kNegInf ? e.y * ex2_approx(e.x - rec.cp) : 0.f; }
+                if (i < P.nblk && P.nblk <= 256) { const float2 e = __ldcg(&st[i]); m = e.x > kNegInf ? e.y * ex2_approx(e.x - cp) : 0.f; }
                 xr[k] = m;
             }
         }
@@ -726,7 +806,7 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
             b = level1_memory(n1, lane, wv, u * tot, before);
         } else {
             const float2* st = P.stats_t + (long long)rec.row_t * P.nblk;
-            auto mass = [&](int i) { const float2 e = __ldcg(&st[i]); return e.x > kNegInf ? e.y * ex2_approx(e.x - rec.cp) : 0.f; };
+            auto mass = [&](int i) { const float2 e = __ldcg(&st[i]); return e.x > kNegInf ? e.y * ex2_approx(e.x - cp) : 0.f; };
             tot = warp_total(n1, lane, mass);
             b = level1_memory(n1, lane, mass, u * tot, before);
         }
@@ -745,7 +825,7 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
                 trow, drow, e0, cnt, lane, thr_local, [&](float xt, float xd) { return resid_elem(xt, xd, K); }, S);
         } else {
             // element masses relative to the row reference, like the block masses
-            const float nc = -rec.cp, scale = rec.scale, tau = rec.tau;
+            const float nc = -cp, scale = rec.scale, tau = rec.tau;
             const int e0 = b * P.epb;
             const int cnt = (P.V - e0) < P.epb ? (P.V - e0) : P.epb;
             token = e0 + level2_block<kElem, kStatBlockBytes, false>(
@@ -898,6 +978,7 @@ __global__ void __launch_bounds__(kDecideThreads) greedy_decide_kernel(VerifyPar
 // ---------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------
+static std::atomic<int> g_skip_bonus{1};      // diagnostic switch: 0 streams every bonus row in the statistics pass
 static std::atomic<int> g_stream_path{0};     // 0 automatic, 1 direct loads, 2 bulk copies in separate passes
 
 struct DeviceInfo { int sms; bool attrs_set; };
@@ -915,7 +996,7 @@ template <int kElem, int kMode>
 static cudaError_t set_smem_attr()
 {
     return cudaFuncSetAttribute(stream_bulk_kernel<kElem, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                kStages * kStageBytes);
+                                kStages * kStageBytes + (kMode == kModeStats ? (kSkipBonusMaxRequests + 4) * 4 : 0));
 }
 
 static bool ensure_attrs()
@@ -938,7 +1019,9 @@ static void launch_stream(const VerifyParams& P, bool bulk, long long max_units,
         long long g = (long long)sms * 3;
         if (g > max_units) g = max_units;
         if (g < 1) g = 1;
-        launch_pdl(stream_bulk_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kStreamThreads), kStages * kStageBytes, s, P);
+        size_t smem = (size_t)kStages * kStageBytes;
+        if (kMode == kModeStats && P.skip_bonus) smem += (size_t)((P.R + 4) / 4) * 16;
+        launch_pdl(stream_bulk_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kStreamThreads), smem, s, P);
     } else {
         long long g = (long long)sms * 8;
         if (g > max_units) g = max_units;
@@ -989,6 +1072,7 @@ static int fill_common(VerifyParams& P, const void* target, const void* draft, i
     P.req_temp = nullptr;
     P.tau = nullptr;
     P.draft_stats = nullptr;
+    P.skip_bonus = 0;
     return DSPARK_OK;
 }
 
@@ -1042,8 +1126,11 @@ int dspark_set_wait_poll_limit(unsigned int polls)
 
 int dspark_set_stream_path(int path)
 {
-    if (path < 0 || path > 2) return DSPARK_ERR_INVALID_ARG;
-    g_stream_path.store(path, std::memory_order_relaxed);
+    // 0 automatic, 1 direct loads, 2 bulk copies; + 16: every bonus row in the statistics pass (the earlier order)
+    const int base = path & 15;
+    if (path < 0 || path > 31 || base > 2) return DSPARK_ERR_INVALID_ARG;
+    g_stream_path.store(base, std::memory_order_relaxed);
+    g_skip_bonus.store((path & 16) ? 0 : 1, std::memory_order_relaxed);
     return DSPARK_OK;
 }
 
@@ -1121,6 +1208,10 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
     const bool bulk = path != 1 && aligned16(P.target, P.tstride_bytes, P.row_bytes) &&
                       aligned16(P.draft, P.dstride_bytes, P.row_bytes);
     if (!ensure_attrs()) return launch_status();
+    // A rejected request never needs its bonus row: the statistics pass leaves the bonus rows out and the second pass
+    // streams them for the requests that accepted every draft token.  (Not with a truncated target, whose threshold
+    // search wants the statistics of every target row first, nor on the direct-load path.)
+    P.skip_bonus = (bulk && !truncate && g_skip_bonus.load(std::memory_order_relaxed) && R <= kSkipBonusMaxRequests) ? 1 : 0;
     if (req_temp) {
         KernelTimerScope timer(DSPARK_K_ROW_SCALE, s);
         launch_pdl(row_scale_kernel, dim3((R + 255) / 256), dim3(256), 0, s, P);
@@ -1165,7 +1256,8 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {
         KernelTimerScope timer(DSPARK_K_RESIDUAL, s);
-        launch_stream_dtype<kModeResid>(P, bulk, (long long)R * pieces(P.nblk_r), s);
+        const long long per_task = pieces(P.nblk_r) > pieces(P.nblk) ? pieces(P.nblk_r) : pieces(P.nblk);
+        launch_stream_dtype<kModeResid>(P, bulk, (long long)R * per_task, s);
     }
     if ((rc = launch_status()) != DSPARK_OK) return rc;
     {

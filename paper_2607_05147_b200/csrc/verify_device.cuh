@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace dspark {
@@ -12,6 +14,8 @@ namespace dspark {
 constexpr int kModeStats = 0, kModeGreedy = 1, kModeResid = 2, kModeHist = 3;
 constexpr int kHistBins = 1024;              // keys next to the row maximum that the streamed threshold search resolves
 constexpr int kTaskNone = 0, kTaskResid = 1, kTaskBonus = 2;
+constexpr int kCtrBonus = 12;                // header cell: bonus rows queued for the second pass (from the back of the queue)
+constexpr int kSkipBonusMaxRequests = 2048;  // the statistics pass keeps (row_offsets[r] - r) of the batch behind its stages
 constexpr int kDecideThreads = 256;
 constexpr float kNegInf = -INFINITY;
 
@@ -79,6 +83,9 @@ struct VerifyParams {
     unsigned long long launch_tag;            // unique per call: see unit_counter()
     float* wblk;                              // per request: residual block sums
     const float* tau;                         // per target row: top-k / top-p threshold (NULL: no truncation)
+    int skip_bonus;                           // 1: the statistics pass leaves the bonus rows out; the second pass streams
+                                              // them for the requests that accepted every draft token (a rejected
+                                              // request never needs its bonus row)
     const float2* draft_stats;                // per physical draft row: (reference, sum) handed over by the drafter (NULL:
                                               // the statistics pass streams the draft rows as well)
     TruncRow* trunc_rows;                     // workspace of the streamed threshold search
@@ -123,7 +130,10 @@ __device__ __forceinline__ long long draft_phys_row(const VerifyParams& P, int d
 template <int kMode>
 __device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
 {
-    if (kMode == kModeStats) return n_rows + ((n_rows > P.R && !P.draft_stats) ? n_rows - P.R : 0);
+    if (kMode == kModeStats) {
+        const int nd = n_rows > P.R ? n_rows - P.R : 0;           // draft positions = target rows that are not bonus rows
+        return (P.skip_bonus ? nd : n_rows) + (P.draft_stats ? 0 : nd);
+    }
     if (kMode == kModeGreedy || kMode == kModeHist) return n_rows;
     const int nq = __ldcg(&P.counters[0]);
     return nq > P.resid_cap ? P.resid_cap : (nq < 0 ? 0 : nq);
@@ -402,6 +412,21 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
                                               const ResidTask* task = nullptr, const TruncRow* trunc = nullptr)
 {
     using M = ModeCfg<kMode>;
+    if constexpr (kMode == kModeResid && std::is_same<Fetch, SmemFetch>::value) {
+        if (task && task->row_d < 0) {
+            // a bonus row inside the second pass (bulk-copy pipeline only): the stage holds a 32 KB piece of the row,
+            // one 4 KB statistics block per warp (f0 points at this warp's 2 KB residual block)
+            const int b4 = piece * kConsumerWarps + warp;
+            if (b4 >= P.nblk) return;
+            const int rem4 = P.row_bytes - b4 * kStatBlockBytes;
+            uint4 v4[kStatVec];
+            load_block<kElem, kStatVec>(SmemFetch{f0.blk + warp * (kStatBlockBytes - M::kBlockBytes)},
+                                        rem4 < kStatBlockBytes ? rem4 : kStatBlockBytes, lane, v4);
+            const float2 st = block_stats<kElem, kStatVec>(v4, task->scale);
+            if (lane == 0) P.stats_t[(long long)task->row_t * P.nblk + b4] = st;
+            return;
+        }
+    }
     const int nblk = (kMode == kModeResid) ? P.nblk_r : P.nblk;
     const int b = piece * kConsumerWarps + warp;
     if (b >= nblk) return;
@@ -471,7 +496,7 @@ __device__ __forceinline__ void unit_sources(const VerifyParams& P, int s, int p
     if (kMode == kModeResid) {
         const ResidTask t = task ? *task : P.resid[s];
         src0 = P.target + (long long)t.row_t * P.tstride_bytes + off;
-        src1 = P.draft + t.row_d * P.dstride_bytes + off;
+        src1 = t.row_d >= 0 ? P.draft + t.row_d * P.dstride_bytes + off : nullptr;   // a bonus row: the target row alone
     } else if (s < n_rows) {
         src0 = P.target + (long long)s * P.tstride_bytes + off;
     } else {
