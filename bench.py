@@ -33,12 +33,12 @@ NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126 * 1024 * 1024
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/: cfg3 and cfg2 were captured as they are; cfg4 and cfg5 are
-# too large for a multi-pass capture, so their figure is the algorithmic bytes times the
-# traffic / algorithmic ratio of the smaller capture of the same kernel (traffic is proportional to
-# the rows streamed).
-NCU_TRAFFIC_BYTES = {"cfg3": 264811264 + 3869184, "cfg2": 168603136 + 4249856}
-NCU_TRAFFIC_RATIO = {"cfg4": 1.0135, "cfg5": 1.0165}
+# captures summarised under profiles/: cfg3 was captured as it is; cfg4 and cfg5 are too large for a
+# multi-pass capture, so their figure is the algorithmic bytes times the traffic / algorithmic ratio of
+# the smaller capture of the same kernel (traffic is proportional to the rows streamed), and cfg2 takes
+# the ratio of its capture of the earlier form of the pass (every bonus row streamed there as well).
+NCU_TRAFFIC_BYTES = {"cfg3": 198608640 + 3929088}
+NCU_TRAFFIC_RATIO = {"cfg2": 1.025, "cfg4": 1.0135, "cfg5": 1.0165}
 
 
 # ----------------------------------------------------------------------------- workloads ----
@@ -121,7 +121,7 @@ def make_workload(name: str, device, rank: int, n_sets=None, oracle_schedule=Fal
 
     batches = [one(0)]
     if n_sets is None:
-        stream_b, _ = algorithmic_bytes(batches[0], greedy, 0)
+        stream_b = algorithmic_bytes(batches[0], greedy, 0)[0]
         n_sets = max(2, min(8, -(-4 * L2_BYTES // stream_b)))
     for k in range(1, n_sets):
         batches.append(one(k))
@@ -265,12 +265,20 @@ class Step:
 
 
 def algorithmic_bytes(batch, greedy, n_rejected):
-    """Bytes the method must move: every target and draft row once, plus one re-read of the
-    rejected position's row pair per rejected request."""
+    """(bytes the dominant launch streams, bytes the whole call streams, the call's bytes by the formula that counts
+    every row once plus a re-read of each rejected pair).  The sampling verifier streams the target and draft row of
+    every draft position in its statistics pass and, in its second pass, the rejected pairs and the bonus rows of the
+    requests that accepted everything: one row per rejected request fewer than the formula (with a truncated target
+    all bonus rows go through the first pass and the two figures coincide)."""
     elem = batch.target.element_size()
+    row = elem * batch.V
     n_draft = batch.n_rows - batch.R
-    stream = elem * batch.V * (batch.n_rows + (0 if greedy else n_draft))
-    return stream, stream + (0 if greedy else 2 * elem * batch.V * n_rejected)
+    if greedy:
+        return row * batch.n_rows, row * batch.n_rows, row * batch.n_rows
+    formula = row * (batch.n_rows + n_draft + 2 * n_rejected)
+    if TRUNCATE is not None or batch.R > 2048:
+        return row * (batch.n_rows + n_draft), formula, formula
+    return row * 2 * n_draft, row * (2 * n_draft + 2 * n_rejected + (batch.R - n_rejected)), formula
 
 
 # -------------------------------------------------------------------------------- clocks ----
@@ -421,7 +429,7 @@ def run_reference(args, rank):
         rows += oracle_step(wl, b, n_req, threads)
     dt = time.perf_counter() - t0
     value = rows / dt
-    stream_bytes, _ = algorithmic_bytes(b0, wl["greedy"], 0)
+    stream_bytes = algorithmic_bytes(b0, wl["greedy"], 0)[0]
     sample = f"first {n_req} of {b.R} requests per step ({rows // max(1, args.steps)} rows), schedule over all requests"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
@@ -723,7 +731,7 @@ def roofline_of(res, peak, peak_src):
     """Dominant kernel of the step against the measured HBM peak (bytes the method must move / its time)."""
     wl = res["wl"]
     b0 = wl["batches"][0]
-    stream_bytes, all_bytes = algorithmic_bytes(b0, wl["greedy"], res["n_rejected"])
+    stream_bytes, all_bytes, _ = algorithmic_bytes(b0, wl["greedy"], res["n_rejected"])
     dom = "greedy_stream" if wl["greedy"] else "stream_stats"
     k = res["kernels"].get(dom, {"ms": float("nan"), "launches": 1})
     dom_ms = k["ms"] / max(1, k["launches"])
@@ -740,10 +748,11 @@ def verify_call_of(res, steps, peak):
     """The verifier call as a whole (every kernel of dspark_verify / dspark_verify_greedy, no scheduler): the
     bytes the method must move, re-reads of rejected pairs included, over its un-instrumented time."""
     wl = res["wl"]
-    _, all_bytes = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
+    _, all_bytes, formula = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
     us = 1e3 * res["verify_ms"] / steps
     gbs = all_bytes / (us * 1e-6) / 1e9
     return {"us_per_call": us, "algorithmic_bytes": all_bytes, "gbs": gbs, "frac": gbs / peak,
+            "bytes_every_row_once_plus_rejected_pairs": formula, "frac_of_that": formula / (us * 1e-6) / 1e9 / peak,
             "timing": "CUDA events around `steps` back-to-back calls, median over repeats, batches rotated"}
 
 
@@ -755,7 +764,8 @@ def draft_stats_call_of(res, steps, peak):
     wl = res["wl"]
     b0 = wl["batches"][0]
     elem = b0.target.element_size()
-    all_bytes = elem * b0.V * b0.n_rows + 2 * elem * b0.V * res["n_rejected"]
+    # statistics pass: the target rows of the draft positions; second pass: rejected pairs and the bonus rows of the rest
+    all_bytes = elem * b0.V * ((b0.n_rows - b0.R) + 2 * res["n_rejected"] + (b0.R - res["n_rejected"]))
     us = 1e3 * res["draft_stats_ms"] / steps
     gbs = all_bytes / (us * 1e-6) / 1e9
     return {"us_per_call": us, "algorithmic_bytes": all_bytes, "gbs": gbs, "frac": gbs / peak,
@@ -851,7 +861,7 @@ def main():
         return
 
     b0 = wl["batches"][0]
-    stream_bytes, all_bytes = algorithmic_bytes(b0, wl["greedy"], res["n_rejected"])
+    stream_bytes, all_bytes, _ = algorithmic_bytes(b0, wl["greedy"], res["n_rejected"])
     ms, e2e_ms = res["ms"], res["e2e"]["ms"]
     value = replicas.whole_job_rate(res["n_rows"], args.steps, ms, world)
     e2e_value = replicas.whole_job_rate(res["n_rows"], res["e2e"]["steps"], e2e_ms, world)
@@ -898,7 +908,7 @@ def main():
             torch.cuda.empty_cache()
             res = measure_workload(name, args, device, rank, local_rank, world, dist, barrier, False, False)
             wl = res["wl"]
-            _, ab = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
+            _, ab, _ = algorithmic_bytes(wl["batches"][0], wl["greedy"], res["n_rejected"])
             roof = roofline_of(res, peak, peak_src)
             step_ms = res["ms"] / args.steps
             others[name] = {"value": res["n_rows"] * args.steps / (res["ms"] * 1e-3), "unit": UNIT,
