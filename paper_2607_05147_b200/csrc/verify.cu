@@ -38,14 +38,20 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     __shared__ __align__(8) uint64_t full_bar[kStages];
     __shared__ __align__(8) uint64_t empty_bar[kStages];
     __shared__ UnitSlot s_unit[kStages];
+    __shared__ __align__(8) uint64_t hist_bar[2];
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kConsumerWarps); }
+        if (kMode == kModeHist) { mbar_init(&hist_bar[0], kConsumerWarps); mbar_init(&hist_bar[1], kConsumerWarps); }
         s_abort = 0;
         mbar_fence_init();
     }
+    // histogram pass: two histograms of one unit each behind the stages (units alternate between them)
+    unsigned int* unit_bins = reinterpret_cast<unsigned int*>(stage_mem + kStages * kStageBytes);
+    if (kMode == kModeHist)
+        for (int i = tid; i < 2 * kHistBins; i += kStreamThreads) unit_bins[i] = 0u;
     __syncthreads();
     pdl_wait();                                  // everything below reads what earlier kernels wrote
 
@@ -57,6 +63,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
         P.counters[kCtrBonus] = 0;               // and the bonus rows it queues from the back
         *unit_counter<kModeResid>(P) = 0ull;     // unit counters of the passes that follow this one in the call
         *unit_counter<kModeHist>(P) = 0ull;
+        reinterpret_cast<unsigned long long*>(P.counters)[kCellRetryUnits] = 0ull;
+        P.counters[kCtrRetry] = 0;               // rows of the threshold search's second look
         *unit_counter<kMode>(P) = 0ull;          // and this pass's own, published by the tag
         __threadfence();
         atomicExch(unit_tag(P), P.launch_tag);
@@ -134,7 +142,13 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                         }
                     }
                     if (kMode == kModeResid) slot.task = P.resid[slot.s];
-                    if (kMode == kModeHist) slot.trunc = P.trunc_rows[slot.s];
+                    if (kMode == kModeHist) {
+                        if (P.hist_retry) {                  // second look: the rows the first one listed
+                            const int row = __ldcg(&P.retry_rows[slot.s]);
+                            slot.s = row < 0 ? 0 : (row >= n_rows ? n_rows - 1 : row);
+                        }
+                        slot.trunc = P.trunc_rows[slot.s];
+                    }
                     unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes, kMode == kModeResid ? &slot.task : nullptr);
                     slot.scale = stream_scale<kMode>(P, slot.s, n_rows, n_streams + (skip_bonus ? P.R : 0));
                 } else {
@@ -197,11 +211,33 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
             if (unit_s < 0) break;
             unsigned char* sp = stage_mem + st * kStageBytes + warp * M::kBlockBytes;
             SmemFetch f0{sp}, f1{sp + M::kPieceBytes};
-            consume_block<kElem, kMode>(P, unit_s, unit_piece, n_rows, warp, lane, f0, f1, unit_scale,
-                                        kMode == kModeResid ? &s_unit[st].task : nullptr,
-                                        kMode == kModeHist ? &s_unit[st].trunc : nullptr);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[st]);
+            if constexpr (kMode == kModeHist) {
+                // The eight blocks of the unit are counted into one histogram in shared memory; when all consumer
+                // warps have added theirs (a barrier of their own, bounded like every wait), each thread moves
+                // its share of the non-empty bins to the row's counts and leaves them zero for the unit after next.
+                const uint32_t window = s_unit[st].trunc.size;
+                unsigned int* h = unit_bins + (it & 1) * kHistBins;
+                consume_block<kElem, kMode>(P, unit_s, unit_piece, n_rows, warp, lane, f0, f1, unit_scale, nullptr,
+                                            &s_unit[st].trunc, h);
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(&empty_bar[st]); mbar_arrive(&hist_bar[it & 1]); }
+                if (!__all_sync(0xffffffffu, mbar_wait_bounded(&hist_bar[it & 1], (uint32_t)(it >> 1) & 1u, entry_limit))) {
+                    if (lane == 0) { atomicOr(P.dev_status, DSPARK_DEV_TIMEOUT); *abort_flag = 1; }
+                    break;
+                }
+                unsigned int* bins = P.trunc_bins + (long long)unit_s * kHistBins;
+#pragma unroll
+                for (int j = 0; j < kHistBins / (kConsumerWarps * 32); ++j) {
+                    const uint32_t d = (uint32_t)(j * kConsumerWarps * 32 + warp * 32 + lane);
+                    const unsigned int c = d < window ? h[d] : 0u;
+                    if (c) { atomicAdd(&bins[d], c); h[d] = 0u; }
+                }
+            } else {
+                consume_block<kElem, kMode>(P, unit_s, unit_piece, n_rows, warp, lane, f0, f1, unit_scale,
+                                            kMode == kModeResid ? &s_unit[st].task : nullptr, nullptr);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[st]);
+            }
         }
     }
 }
@@ -219,6 +255,7 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
     const int n_rows = device_rows(P, &bad_rows);
     if (kMode != kModeResid && kMode != kModeHist && blockIdx.x == 0 && tid == 0) {
         P.counters[0] = 0;
+        P.counters[kCtrRetry] = 0;
         if (bad_rows) atomicOr(P.dev_status, DSPARK_DEV_BAD_OFFSETS);
     }
     const int n_streams = stream_count<kMode>(P, n_rows);
@@ -228,11 +265,16 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
     for (; cur.s < n_streams; cur.next()) {
         const unsigned char *src0, *src1;
         int bytes;
-        unit_sources<kMode>(P, cur.s, cur.piece, n_rows, src0, src1, bytes);
+        int row = cur.s;
+        if (kMode == kModeHist && P.hist_retry) {            // second look of the threshold search: the listed rows
+            row = __ldcg(&P.retry_rows[cur.s]);
+            row = row < 0 ? 0 : (row >= n_rows ? n_rows - 1 : row);
+        }
+        unit_sources<kMode>(P, row, cur.piece, n_rows, src0, src1, bytes);
         GlobalFetch<kElem> f0{src0 + warp * M::kBlockBytes};
         GlobalFetch<kElem> f1{(kMode == kModeResid ? src1 : src0) + warp * M::kBlockBytes};
-        consume_block<kElem, kMode>(P, cur.s, cur.piece, n_rows, warp, lane, f0, f1,
-                                    stream_scale<kMode>(P, cur.s, n_rows, n_streams));
+        consume_block<kElem, kMode>(P, row, cur.piece, n_rows, warp, lane, f0, f1,
+                                    stream_scale<kMode>(P, row, n_rows, n_streams));
     }
 }
 
@@ -240,9 +282,10 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
 // top-k / top-p truncation of the target distribution inside the verifier (bf16 rows).
 // The kept set of a row is {v : x_v >= tau}; tau is found exactly on the 16-bit keys:
 //   trunc_prep    per target row: row maximum m (recovered exactly from the statistics: the reference
-//                 c = m * scale determines the bf16 value m), the window of keys between m and m - 8 T (at
-//                 most kHistBins keys), zeroed counters;
-//   stream<Hist>  one more streamed pass over the target rows counts the keys inside the window;
+//                 c = m * scale determines the bf16 value m), the window of keys below m (down to the k-th
+//                 largest block maximum for top-k of at most one token per block, else kHistBins keys), zeroed counters;
+//   stream<Hist>  one more streamed pass over the target rows counts the keys inside the window (per 32 KB unit in
+//                 shared memory, non-empty bins added to the row's counts);
 //   trunc_scan    per row: masses count * 2^(value * scale - C), prefix sums, the top-k and top-p
 //                 thresholds; a row whose threshold lies beyond the window is flagged for the per-row
 //                 search of truncate.cu (flat rows: rare);
@@ -253,6 +296,24 @@ struct TruncArgs {
     const int32_t* top_k; const float* top_p; const float* temperatures; float temperature;
     float* tau;                       // per target row
 };
+
+// The window of keys from the row maximum down to lo_val (at most kHistBins keys, and no key below the lowest).
+__device__ __forceinline__ void key_window(float lo_val, uint32_t kmax, uint32_t& size, uint32_t& cut2)
+{
+    const uint32_t klo = bf16_key((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rd(lo_val)));
+    size = kHistBins;
+    if (klo <= kmax && kmax - klo + 1u < (uint32_t)kHistBins) size = kmax - klo + 1u;
+    if (size > kmax + 1u) size = kmax + 1u;                          // keys 0 .. kmax exist
+    const uint32_t cb = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(bf16_key_value(kmax - (size - 1u))));
+    cut2 = cb | (cb << 16);
+}
+
+// Top-p: the tokens below a value v weigh at most V 2^(v scale - C) together, so the nucleus ends above the v at
+// which that is (1 - p) Z.
+__device__ __forceinline__ float nucleus_floor(float C, float Z, float p, float scale, int V)
+{
+    return (C + log2f((1.f - p) * Z / (float)V)) / scale - 0.07f / scale;
+}
 
 __global__ void __launch_bounds__(256) trunc_prep_kernel(VerifyParams P, TruncArgs T)
 {
@@ -281,7 +342,14 @@ __global__ void __launch_bounds__(256) trunc_prep_kernel(VerifyParams P, TruncAr
         const __nv_bfloat16 mb = __float2bfloat16_rn(A.C / scale);      // the bf16 maximum behind c = m * scale
         const float m = __bfloat162float(mb);
         const uint32_t kmax = bf16_key((uint32_t)__bfloat16_as_ushort(mb));
-        float lo_val = m - 8.f * temp;
+        // The window's lower end.  Top-k of at most one token per block: the k-th largest block maximum (tau is at
+        // least tau_k, which cannot lie below it).  Top-k of more tokens: every key the histogram has (for a maximum
+        // of 13 the kHistBins keys below it reach down to 0.05).  Top-p alone: m - 8 T, where a peaked row's nucleus
+        // ends, unless the bound on the nucleus is nearer; a row it does not resolve gets a second look down to
+        // that bound (trunc_scan_kernel).
+        float lo_val = m;
+        if (use_p) lo_val = fmaxf(nucleus_floor(A.C, (float)A.S, pf, scale, P.V), m - 8.f * temp);
+        if (use_k && k > P.nblk) lo_val = -INFINITY;
         if (use_k && k <= P.nblk) {
             // every block maximum is an element of the row, so the k-th largest logit is at least the k-th
             // largest block maximum: the window reaches down to it (rank by counting, 64-128 blocks)
@@ -317,24 +385,46 @@ __global__ void __launch_bounds__(256) trunc_prep_kernel(VerifyParams P, TruncAr
                 }
             }
             kth = warp_max_f32(kth);
-            if (kth > kNegInf) lo_val = fminf(lo_val, __bfloat162float(__float2bfloat16_rn(kth / scale)));
+            if (kth > kNegInf) lo_val = __bfloat162float(__float2bfloat16_rn(kth / scale));
+            else if (!use_p) lo_val = -INFINITY;
         }
-        const uint32_t klo = bf16_key((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rd(lo_val)));
-        uint32_t size = kHistBins;
-        if (klo <= kmax && kmax - klo + 1u < (uint32_t)kHistBins) size = kmax - klo + 1u;
-        if (size > kmax + 1u) size = kmax + 1u;                          // keys 0 .. kmax exist
-        const uint32_t cb = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(bf16_key_value(kmax - (size - 1u))));
-        tr.kmax = kmax; tr.size = size; tr.cut2 = cb | (cb << 16); tr.scale = scale;
+        if (!(lo_val <= m)) lo_val = m;
+        uint32_t size, cut2;
+        key_window(lo_val, kmax, size, cut2);
+        tr.kmax = kmax; tr.size = size; tr.cut2 = cut2; tr.scale = scale;
         tr.k = use_k ? k : 0; tr.p = use_p ? pf : 1.f;
         unsigned int* bins = P.trunc_bins + (long long)row * kHistBins;
         for (uint32_t i = lane; i < size; i += 32) bins[i] = 0u;
     }
-    if (lane == 0) { P.trunc_rows[row] = tr; T.tau[row] = kNegInf; P.trunc_flag[row] = 0; }
+    if (lane == 0) { P.trunc_rows[row] = tr; T.tau[row] = kNegInf; P.trunc_flag[row] = 0; P.trunc_z[row] = -1.0; }
     if (row == 0 && lane == 0) P.trunc_flag[P.n_rows_cap] = 0;          // work counter of the per-row fallback
 }
 
 constexpr int kScanThreads = 256;
-__global__ void __launch_bounds__(kScanThreads) trunc_scan_kernel(VerifyParams P, TruncArgs T)
+// A row its window did not resolve: after the first look it is listed for a second one with the window the bound on
+// its nucleus gives (counts zeroed here), if that is deeper; else (and after the second look) it goes to the per-row
+// search.  Called by all threads of the row's CTA.
+__device__ __forceinline__ void leave_unresolved(const VerifyParams& P, int row, const TruncRow& tr, int retry, int tid)
+{
+    uint32_t size = 0u, cut2 = 0u;
+    if (!retry && tr.k == 0 && tr.p < 1.f && tr.p > 0.f)
+        key_window(nucleus_floor(tr.C, tr.Z, tr.p, tr.scale, P.V), tr.kmax, size, cut2);
+    if (size > tr.size) {
+        unsigned int* bins = P.trunc_bins + (long long)row * kHistBins;
+        for (uint32_t i = tid; i < size; i += kScanThreads) bins[i] = 0u;
+        if (tid == 0) {
+            P.trunc_rows[row].size = size;
+            P.trunc_rows[row].cut2 = cut2;
+            P.trunc_flag[row] = 2;
+            const int slot = atomicAdd(&P.counters[kCtrRetry], 1);
+            if (slot < P.n_rows_cap) P.retry_rows[slot] = row;
+        }
+    } else if (tid == 0) {
+        P.trunc_flag[row] = 1;
+    }
+}
+
+__global__ void __launch_bounds__(kScanThreads) trunc_scan_kernel(VerifyParams P, TruncArgs T, int retry)
 {
     constexpr int kPer = kHistBins / kScanThreads;
     __shared__ unsigned long long s_c[kScanThreads / 32];
@@ -345,6 +435,7 @@ __global__ void __launch_bounds__(kScanThreads) trunc_scan_kernel(VerifyParams P
     const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     bool bad_rows;
     if (row >= device_rows(P, &bad_rows)) return;
+    if (retry && P.trunc_flag[row] != 2) return;            // the second look is for the rows listed by the first
     const TruncRow tr = P.trunc_rows[row];
     if (tr.size == 0u) return;
     if (tid == 0) { s_hit_k = 0x7fffffff; s_hit_p = 0x7fffffff; }
@@ -392,7 +483,7 @@ __global__ void __launch_bounds__(kScanThreads) trunc_scan_kernel(VerifyParams P
     __syncthreads();
     const int dk = s_hit_k;
     if (tr.k > 0 && dk == 0x7fffffff) {                     // the k-th largest key lies beyond the window
-        if (tid == 0) P.trunc_flag[row] = 1;
+        leave_unresolved(P, row, tr, retry, tid);
         return;
     }
     if (tr.k > 0 && dk / kPer == tid) {                     // mass of the top-k set
@@ -419,24 +510,32 @@ __global__ void __launch_bounds__(kScanThreads) trunc_scan_kernel(VerifyParams P
             __syncthreads();
             const int dp = s_hit_p;
             if (dp == 0x7fffffff && tr.k == 0) {            // the nucleus reaches beyond the window
-                if (tid == 0) P.trunc_flag[row] = 1;
+                leave_unresolved(P, row, tr, retry, tid);
                 return;
             }
             if (dp < dist) dist = dp;
         }
     }
     if (tid == 0 && dist != 0x7fffffff) T.tau[row] = bf16_key_value(tr.kmax - (uint32_t)dist);
+    if (tid == 0 && retry) P.trunc_flag[row] = 0;           // resolved by the second look
+    if (dist != 0x7fffffff && dist / kPer == tid) {         // mass of the kept set: what the accept test divides by
+        double q = m_excl;
+        for (int j = 0; j <= dist % kPer; ++j) q += mass[j];
+        P.trunc_z[row] = q;
+    }
 }
 
-// One warp per (target row, statistics block): s = sum over x >= tau of 2^(x * scale - c).
+// One warp per (bonus row, statistics block): s = sum over x >= tau of 2^(x * scale - c).  Only a bonus token is drawn
+// from a target row's block sums; the accept tests take the mass of the kept set from the key counts (trunc_z) and
+// the residual pass sums its own blocks.
 __global__ void __launch_bounds__(256) trunc_sums_kernel(VerifyParams P, TruncArgs T)
 {
     pdl_wait();
     const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x;
+    const int row = P.row_offsets[blockIdx.x + 1] - 1;      // the last row of request blockIdx.x
     const int b = blockIdx.y * 8 + (threadIdx.x >> 5);
     bool bad_rows;
-    if (row >= device_rows(P, &bad_rows) || b >= P.nblk) return;
+    if (row < 0 || row >= device_rows(P, &bad_rows) || b >= P.nblk) return;
     const float tau = T.tau[row];
     if (!(tau > kNegInf) || P.trunc_flag[row]) return;       // untouched row, or left to the per-row search
     const TruncRow tr = P.trunc_rows[row];
@@ -628,6 +727,12 @@ __global__ void __launch_bounds__(kDecideThreads) decide_kernel(VerifyParams P)
             } else {
                 combine_rows(P.stats_t + (long long)(lo + j) * P.nblk,
                              is_draft_pos ? P.stats_d + (long long)(lo - r + j) * P.nblk : nullptr, P.nblk, lane, A, D);
+            }
+            if (P.trunc_z && is_draft_pos) {
+                // truncated target (top-k / top-p) by the streamed search: the mass of the kept set comes from the key
+                // counts (a bonus row, and a row left to the per-row search, carry it in their block sums instead)
+                const double zs = __ldcg(&P.trunc_z[lo + j]);
+                if (zs > 0.0) A.S = zs;
             }
             if (!is_draft_pos) {
                 // bonus row: leave its block masses (relative to the row reference) where the finalize
@@ -996,7 +1101,8 @@ template <int kElem, int kMode>
 static cudaError_t set_smem_attr()
 {
     return cudaFuncSetAttribute(stream_bulk_kernel<kElem, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                kStages * kStageBytes + (kMode == kModeStats ? (kSkipBonusMaxRequests + 4) * 4 : 0));
+                                kStages * kStageBytes + (kMode == kModeStats ? (kSkipBonusMaxRequests + 4) * 4 : 0) +
+                                    (kMode == kModeHist ? 2 * kHistBins * (int)sizeof(unsigned int) : 0));
 }
 
 static bool ensure_attrs()
@@ -1021,6 +1127,7 @@ static void launch_stream(const VerifyParams& P, bool bulk, long long max_units,
         if (g < 1) g = 1;
         size_t smem = (size_t)kStages * kStageBytes;
         if (kMode == kModeStats && P.skip_bonus) smem += (size_t)((P.R + 4) / 4) * 16;
+        if (kMode == kModeHist) smem += 2 * kHistBins * sizeof(unsigned int);
         launch_pdl(stream_bulk_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kStreamThreads), smem, s, P);
     } else {
         long long g = (long long)sms * 8;
@@ -1099,6 +1206,9 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.trunc_rows = (TruncRow*)(ws + w.trunc_rows);
     P.trunc_bins = (unsigned int*)(ws + w.trunc_bins);
     P.trunc_flag = (int32_t*)(ws + w.trunc_flag);
+    P.retry_rows = (int32_t*)(ws + w.retry_rows);
+    P.trunc_z = nullptr;
+    P.hist_retry = 0;
     P.row_scale_t = (float*)(ws + w.scale_t);
     P.row_scale_d = (float*)(ws + w.scale_d);
     return DSPARK_OK;
@@ -1238,10 +1348,16 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
         KernelTimerScope timer(DSPARK_K_TRUNCATE, s);
         TruncArgs T;
         T.top_k = top_k; T.top_p = top_p; T.temperatures = req_temp; T.temperature = temperature; T.tau = tau;
+        P.trunc_z = (double*)((unsigned char*)workspace + workspace_layout(R, n_rows, V).trunc_z);
         launch_pdl(trunc_prep_kernel, dim3((n_rows + 7) / 8), dim3(256), 0, s, P, T);
         launch_stream<2, kModeHist>(P, bulk, (long long)n_rows * pieces(P.nblk), s);
-        launch_pdl(trunc_scan_kernel, dim3(n_rows), dim3(kScanThreads), 0, s, P, T);
-        launch_pdl(trunc_sums_kernel, dim3(n_rows, (P.nblk + 7) / 8), dim3(256), 0, s, P, T);
+        launch_pdl(trunc_scan_kernel, dim3(n_rows), dim3(kScanThreads), 0, s, P, T, 0);
+        // second look at the rows whose nucleus reaches below the first window (flat rows), down to the bound
+        P.hist_retry = 1;
+        launch_stream<2, kModeHist>(P, bulk, (long long)n_rows * pieces(P.nblk), s);
+        P.hist_retry = 0;
+        launch_pdl(trunc_scan_kernel, dim3(n_rows), dim3(kScanThreads), 0, s, P, T, 1);
+        launch_pdl(trunc_sums_kernel, dim3(R, (P.nblk + 7) / 8), dim3(256), 0, s, P, T);
         // rows whose threshold lies beyond the window (flat rows): the per-row search
         rc = truncate_virtual_launch(P.target, P.tstride_bytes, V, row_offsets, R, n_rows, top_k, top_p, temperature,
                                      req_temp, tau, P.stats_t, P.nblk, P.epb, P.trunc_flag, s);

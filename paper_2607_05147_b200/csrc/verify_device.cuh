@@ -15,6 +15,8 @@ constexpr int kModeStats = 0, kModeGreedy = 1, kModeResid = 2, kModeHist = 3;
 constexpr int kHistBins = 1024;              // keys next to the row maximum that the streamed threshold search resolves
 constexpr int kTaskNone = 0, kTaskResid = 1, kTaskBonus = 2;
 constexpr int kCtrBonus = 12;                // header cell: bonus rows queued for the second pass (from the back of the queue)
+constexpr int kCtrRetry = 13;                // header cell: rows the threshold search looks at a second time
+constexpr int kCellRetryUnits = 5;           // 64-bit header cell: unit counter of that second histogram pass
 constexpr int kSkipBonusMaxRequests = 2048;  // the statistics pass keeps (row_offsets[r] - r) of the batch behind its stages
 constexpr int kDecideThreads = 256;
 constexpr float kNegInf = -INFINITY;
@@ -90,7 +92,12 @@ struct VerifyParams {
                                               // the statistics pass streams the draft rows as well)
     TruncRow* trunc_rows;                     // workspace of the streamed threshold search
     unsigned int* trunc_bins;                 // [n_rows][kHistBins] key counts
-    int32_t* trunc_flag;                      // [n_rows] 1: the window did not resolve the row (per-row search)
+    int32_t* trunc_flag;                      // [n_rows] 1: no window resolved the row (per-row search); 2: between the
+                                              // two looks, the row waits for its deeper window
+    int32_t* retry_rows;                      // rows of the second look (their number: counters[kCtrRetry])
+    double* trunc_z;                          // [n_rows] mass of the kept set relative to the row reference, from the key
+                                              // counts (<= 0: take the row's block sums); NULL without the streamed search
+    int hist_retry;                           // histogram pass: 1 = second look, streams retry_rows only
 };
 
 template <int kMode> struct ModeCfg {
@@ -134,6 +141,10 @@ __device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
         const int nd = n_rows > P.R ? n_rows - P.R : 0;           // draft positions = target rows that are not bonus rows
         return (P.skip_bonus ? nd : n_rows) + (P.draft_stats ? 0 : nd);
     }
+    if (kMode == kModeHist && P.hist_retry) {
+        const int nr = __ldcg(&P.counters[kCtrRetry]);
+        return nr < 0 ? 0 : (nr > n_rows ? n_rows : nr);
+    }
     if (kMode == kModeGreedy || kMode == kModeHist) return n_rows;
     const int nq = __ldcg(&P.counters[0]);
     return nq > P.resid_cap ? P.resid_cap : (nq < 0 ? 0 : nq);
@@ -150,7 +161,8 @@ __device__ __forceinline__ int stream_count(const VerifyParams& P, int n_rows)
 template <int kMode>
 __device__ __forceinline__ unsigned long long* unit_counter(const VerifyParams& P)
 {
-    return reinterpret_cast<unsigned long long*>(P.counters) + (kMode == kModeResid ? 2 : (kMode == kModeHist ? 3 : 1));
+    return reinterpret_cast<unsigned long long*>(P.counters) +
+           (kMode == kModeResid ? 2 : (kMode == kModeHist ? (P.hist_retry ? kCellRetryUnits : 3) : 1));
 }
 __device__ __forceinline__ unsigned long long* unit_tag(const VerifyParams& P)
 {
@@ -409,7 +421,8 @@ __device__ __forceinline__ float block_resid(const uint4 (&vt)[kVec], const uint
 template <int kElem, int kMode, typename Fetch>
 __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int piece, int n_rows,
                                               int warp, int lane, const Fetch& f0, const Fetch& f1, float scale,
-                                              const ResidTask* task = nullptr, const TruncRow* trunc = nullptr)
+                                              const ResidTask* task = nullptr, const TruncRow* trunc = nullptr,
+                                              unsigned int* shared_bins = nullptr)
 {
     using M = ModeCfg<kMode>;
     if constexpr (kMode == kModeResid && std::is_same<Fetch, SmemFetch>::value) {
@@ -444,12 +457,13 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
         const float2 st = block_argmax<kElem, M::kVec>(v, b * P.epb, lane);
         if (lane == 0) P.stats_t[(long long)s * nblk + b] = st;
     } else if (kMode == kModeHist) {
-        // bf16 rows only.  Count the keys within the window next to the row maximum: a packed compare rejects
-        // almost every pair, the few tokens of the tail take one atomic each.
+        // bf16 rows only.  Count the keys within the window next to the row maximum: a packed compare rejects the
+        // pairs below it, the others take one atomic per token -- on the unit's histogram in shared memory where the
+        // caller keeps one (it adds the non-empty bins to the row's counts afterwards), else on the row's counts.
         const TruncRow tr = trunc ? *trunc : P.trunc_rows[s];
         if (tr.size == 0u) return;
         const __nv_bfloat162 cut2 = *reinterpret_cast<const __nv_bfloat162*>(&tr.cut2);
-        unsigned int* bins = P.trunc_bins + (long long)s * kHistBins;
+        unsigned int* bins = shared_bins ? shared_bins : P.trunc_bins + (long long)s * kHistBins;
 #pragma unroll
         for (int k = 0; k < M::kVec; ++k) {
 #pragma unroll
@@ -749,7 +763,7 @@ __device__ __forceinline__ int level2_block(const unsigned char* trow, const uns
 
 // Workspace of the verifiers (caller-provided, any content on entry), offsets in bytes.
 struct Workspace {
-    size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, tau, trunc_rows, trunc_bins, trunc_flag;
+    size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, tau, trunc_rows, trunc_bins, trunc_flag, retry_rows, trunc_z;
     size_t total;
 };
 inline Workspace workspace_layout(int R, int n_rows, int V)
@@ -771,6 +785,8 @@ inline Workspace workspace_layout(int R, int n_rows, int V)
     w.trunc_rows = o; o += up((size_t)n_rows * sizeof(TruncRow));
     w.trunc_bins = o; o += up((size_t)n_rows * kHistBins * sizeof(unsigned int));
     w.trunc_flag = o; o += up((size_t)(n_rows + 1) * sizeof(int32_t));   // + the fallback's row counter
+    w.retry_rows = o; o += up((size_t)n_rows * sizeof(int32_t));
+    w.trunc_z = o;    o += up((size_t)n_rows * sizeof(double));
     w.total = o;
     return w;
 }

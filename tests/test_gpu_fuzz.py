@@ -153,6 +153,55 @@ def test_truncate_fuzz(seed):
             assert int(kept[row]) == okept[row]
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_verify_truncated_fuzz(seed):
+    """dspark_verify_truncated (streamed threshold search with its second look on bf16 rows, descent on fp32 rows)
+    against the oracle pipeline warp_target -> verify: peaked, wide, tied and flat rows, top-k / top-p / both / none per
+    request, per-request temperatures, compact and block draft layouts, padded strides."""
+    import oracle
+    rng = np.random.default_rng(9000 + seed)
+    for _ in range(4):
+        R = int(rng.integers(1, 14))
+        V = int(rng.choice([9, 255, 1000, 4097, 20000, 70000]))
+        lengths = torch.from_numpy(rng.integers(0, 5, size=R))
+        dt = torch.bfloat16 if rng.random() < 0.7 else torch.float32
+        kind = int(rng.integers(0, 3))
+        sigma = float(rng.choice([0.5, 1.5, 3.0, 6.0]))
+        block = None if rng.random() < 0.6 else int(lengths.max()) + int(rng.integers(0, 3))
+        T = float(rng.choice([0.5, 1.0, 1.6]))
+        b = W.sampling_batch(lengths, V, int(rng.integers(1 << 30)), "cuda", dtype=dt, sigma=sigma, temperature=T,
+                             draft_noise=float(rng.choice([0.3, 1.0])), verify_seed=int(rng.integers(1 << 30)),
+                             block=block if block else None)
+        if kind == 1:                                          # heavy ties: a coarse grid of values
+            b.target.copy_((b.target.float() * 2).round() / 2)
+        elif kind == 2:                                        # flat rows: no peak at all
+            b.target.copy_(torch.from_numpy(rng.uniform(-2, 2, tuple(b.target.shape)).astype(np.float32)))
+        b.target = _pad_rows(b.target, rng)
+        ks = rng.choice([0, 0, 1, 3, 50, 300, V + 2], size=R).astype(np.int32)
+        ps = rng.choice([1.0, 0.0, 0.3, 0.9, 0.97, 0.999], size=R).astype(np.float32)
+        temps = rng.choice([0.5, 1.0, 1.6], size=R).astype(np.float32) if rng.random() < 0.5 else None
+        acc = torch.full((R,), -7, dtype=torch.int32, device="cuda")
+        out = torch.full((b.n_rows,), -7, dtype=torch.int32, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ws = B.workspace(B.dspark_verify_workspace_bytes(R, b.n_rows, V)).fill_(int(rng.integers(0, 256)))
+        dev = lambda a, d: None if a is None else torch.as_tensor(a, dtype=d, device="cuda")
+        B.dspark_verify_truncated(b.target, b.draft, b.row_offsets, b.draft_tokens, b.seed, temperature=b.temperature,
+                                  temperatures=dev(temps, torch.float32), top_k=dev(ks, torch.int32),
+                                  top_p=dev(ps, torch.float32), draft_row_start=b.draft_row_start, accepted_len=acc,
+                                  out_tokens=out, out_p_tok=None, out_q_tok=None, dev_status=st, workspace=ws)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        off = b.row_offsets.cpu().numpy()
+        bits, dbits = W.bf16_bits(b.target), W.bf16_bits(b.draft)
+        masked, tau, kept, margin = oracle.warp_target(bits, off, top_k=ks, top_p=ps, temperature=b.temperature,
+                                                       temperatures=temps)
+        drs = None if b.draft_row_start is None else b.draft_row_start.cpu().numpy()
+        o = oracle.verify(masked, dbits, off, b.draft_tokens.cpu().numpy(), b.temperature, b.seed, draft_row_start=drs,
+                          eval_all=False, n_threads=H.THREADS, temperatures=temps)
+        g = dict(acc=acc.cpu().numpy(), out=out.cpu().numpy())
+        H.compare_away_from_top_p_boundaries(g, o, margin, off)
+
+
 @pytest.mark.parametrize("seed", range(4))
 def test_markov_fuzz(seed):
     import oracle

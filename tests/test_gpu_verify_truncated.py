@@ -149,6 +149,41 @@ def test_flat_rows_take_the_per_row_search():
     print(f"[verify_truncated] flat rows: accepted {g['acc'].tolist()}, {mism} boundary mismatches")
 
 
+@pytest.mark.parametrize("temperature", [1.0, 0.7])
+def test_a_nucleus_below_the_first_window_gets_a_second_look(temperature):
+    # top-p alone on rows with a wide bulk: the nucleus of most rows ends below m - 8 T, where the first window of
+    # the streamed search stops; those rows are counted a second time down to the bound on their nucleus (p = 0.9 to
+    # 0.99), the others (p = 0.3, 0.5) are resolved by the first look; top-k of more tokens than a row has blocks
+    # takes every key of the histogram at once.  Full-vocabulary rows, so that units of several rows interleave.
+    R, V = 20, W.V_FULL
+    g0 = torch.Generator().manual_seed(31)
+    lengths = torch.randint(0, 5, (R,), generator=g0)
+    b = W.sampling_batch(lengths, V, 53, "cuda", temperature=temperature, draft_noise=1.0, verify_seed=5)
+    ps = np.array([0.9, 0.97, 0.99, 0.5, 0.3, 0.95, 0.9, 1.0, 0.999, 0.9] * 2, dtype=np.float32)
+    ks = np.array([0, 0, 0, 0, 0, 0, 0, 300, 0, 2000] * 2, dtype=np.int32)
+    off = b.row_offsets.cpu().numpy()
+    for want_probs in (True, False):
+        g = _gpu_truncated(b, ks, ps, None, want_probs=want_probs)
+        assert g["status"] == 0
+        o, margin = _oracle_pipeline(b, ks, ps, None)
+        skipped, mism = H.compare_away_from_top_p_boundaries(g, o, margin, off)
+        if want_probs:
+            have = ~np.isnan(g["p"][:b.n_rows]) & (np.asarray(o.p_tok)[:b.n_rows] > 0)
+            np.testing.assert_allclose(g["p"][:b.n_rows][have], np.asarray(o.p_tok)[:b.n_rows][have], rtol=1e-5)
+        print(f"[verify_truncated] second look, T={temperature}: accepted {g['acc'].tolist()}, {skipped} requests on a "
+              f"boundary, {mism} boundary mismatches")
+        # a nucleus that ends in the bulk has many tokens of little mass each next to its boundary: some rows are near
+        assert skipped <= R // 4 and mism <= 1
+    # the two-step pipeline (rows masked in place by the per-row search, then the plain verifier) decides the same
+    masked = b.target.clone()
+    B.dspark_truncate_target(masked, b.row_offsets, temperature=b.temperature,
+                             top_k=torch.as_tensor(ks, device="cuda"), top_p=torch.as_tensor(ps, device="cuda"))
+    b2 = W.VerifyBatch(masked, b.draft, b.row_offsets, b.draft_tokens, b.draft_row_start, b.temperature, b.seed)
+    g2 = H.gpu_verify(b2)
+    g = _gpu_truncated(b, ks, ps, None)
+    assert int((g["acc"] != g2["acc"]).sum()) <= 1           # the kept mass comes from the key counts: equal up to rounding
+
+
 def test_config_3_full_size_with_truncation():
     # the batch and launch configuration that `bench.py --top-k 50 --top-p 0.9` times
     sched = W.config_3_schedule("cuda")
