@@ -39,7 +39,8 @@ struct TruncParams {
     // virtual mode (inside the verifier): the row is not modified; its statistics blocks receive the sums
     // restricted to the kept set instead
     float2* stats; int nblk, epb;
-    const int32_t* only_flagged;              // virtual mode: rows whose flag is 0 are somebody else's (NULL: all rows)
+    const int32_t* only_flagged;              // virtual mode: rows whose flag is 0 are somebody else's (NULL: all rows);
+                                              // [n_rows] work counter, [n_rows + 1] number of flagged rows
 };
 
 __device__ __forceinline__ uint32_t key_of(uint32_t b) { return bf16_key(b); }
@@ -488,6 +489,7 @@ __global__ void __launch_bounds__(kTruncThreads) truncate_flagged_kernel(TruncPa
     __shared__ int s_row;
     pdl_wait();
     int* counter = const_cast<int*>(P.only_flagged) + P.n_rows;     // zeroed with the flags
+    if (P.only_flagged[P.n_rows + 1] == 0) return;                  // nobody flagged a row: the usual case
     for (;;) {
         // rows are handed out one at a time (they take very different times); unflagged ones are skipped here
         if (threadIdx.x == 0) {

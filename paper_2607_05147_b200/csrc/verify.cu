@@ -282,8 +282,9 @@ __global__ void __launch_bounds__(kConsumerWarps * 32, 2) stream_direct_kernel(V
 // top-k / top-p truncation of the target distribution inside the verifier (bf16 rows).
 // The kept set of a row is {v : x_v >= tau}; tau is found exactly on the 16-bit keys:
 //   trunc_prep    per target row: row maximum m (recovered exactly from the statistics: the reference
-//                 c = m * scale determines the bf16 value m), the window of keys below m (down to the k-th
-//                 largest block maximum for top-k of at most one token per block, else kHistBins keys), zeroed counters;
+//                 c = m * scale determines the bf16 value m), the window of keys below m (down to the k-th largest
+//                 block maximum for top-k of at most one token per block; to m - 8 T or the bound on the nucleus for
+//                 top-p alone; else kHistBins keys), zeroed counters;
 //   stream<Hist>  one more streamed pass over the target rows counts the keys inside the window (per 32 KB unit in
 //                 shared memory, non-empty bins added to the row's counts);
 //   trunc_scan    per row: masses count * 2^(value * scale - C), prefix sums, the top-k and top-p
@@ -343,7 +344,8 @@ __global__ void __launch_bounds__(256) trunc_prep_kernel(VerifyParams P, TruncAr
         const float m = __bfloat162float(mb);
         const uint32_t kmax = bf16_key((uint32_t)__bfloat16_as_ushort(mb));
         // The window's lower end.  Top-k of at most one token per block: the k-th largest block maximum (tau is at
-        // least tau_k, which cannot lie below it).  Top-k of more tokens: every key the histogram has (for a maximum
+        // least tau_k, which cannot lie below it; the smallest block maximum would do and needs no ranking, but the
+        // short last block of a row pulls it down, and every token more in the window costs a divergent branch).  Top-k of more tokens: every key the histogram has (for a maximum
         // of 13 the kHistBins keys below it reach down to 0.05).  Top-p alone: m - 8 T, where a peaked row's nucleus
         // ends, unless the bound on the nucleus is nearer; a row it does not resolve gets a second look down to
         // that bound (trunc_scan_kernel).
@@ -397,7 +399,10 @@ __global__ void __launch_bounds__(256) trunc_prep_kernel(VerifyParams P, TruncAr
         for (uint32_t i = lane; i < size; i += 32) bins[i] = 0u;
     }
     if (lane == 0) { P.trunc_rows[row] = tr; T.tau[row] = kNegInf; P.trunc_flag[row] = 0; P.trunc_z[row] = -1.0; }
-    if (row == 0 && lane == 0) P.trunc_flag[P.n_rows_cap] = 0;          // work counter of the per-row fallback
+    if (row == 0 && lane == 0) {                                         // the per-row fallback's work counter and the
+        P.trunc_flag[P.n_rows_cap] = 0;                                  // number of rows left to it
+        P.trunc_flag[P.n_rows_cap + 1] = 0;
+    }
 }
 
 constexpr int kScanThreads = 256;
@@ -421,6 +426,7 @@ __device__ __forceinline__ void leave_unresolved(const VerifyParams& P, int row,
         }
     } else if (tid == 0) {
         P.trunc_flag[row] = 1;
+        atomicAdd(&P.trunc_flag[P.n_rows_cap + 1], 1);
     }
 }
 

@@ -784,7 +784,7 @@ inline Workspace workspace_layout(int R, int n_rows, int V)
     w.tau = o;      o += up((size_t)n_rows * sizeof(float));
     w.trunc_rows = o; o += up((size_t)n_rows * sizeof(TruncRow));
     w.trunc_bins = o; o += up((size_t)n_rows * kHistBins * sizeof(unsigned int));
-    w.trunc_flag = o; o += up((size_t)(n_rows + 1) * sizeof(int32_t));   // + the fallback's row counter
+    w.trunc_flag = o; o += up((size_t)(n_rows + 2) * sizeof(int32_t));   // + the fallback's row counter and row count
     w.retry_rows = o; o += up((size_t)n_rows * sizeof(int32_t));
     w.trunc_z = o;    o += up((size_t)n_rows * sizeof(double));
     w.total = o;
