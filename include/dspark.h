@@ -428,11 +428,12 @@ int dspark_truncate_target(void* target_logits, int dtype, int64_t target_row_st
                            float* out_tau, int32_t* out_kept, int32_t* dev_status, void* stream);
 
 /* dspark_verify_truncated -- dspark_verify / dspark_verify_per_request on the top-k / top-p truncated target
- * distribution of dspark_truncate_target, without modifying the target rows: after the statistics pass one
- * kernel finds the threshold tau of every target row (same rule, same exact search on the 16-bit keys) and
- * replaces the row's block sums by the sums over the kept set; the accept test, the residual pass and the
- * final draws then treat a target logit below tau as -inf.  The draft distribution q is used as given.
- * Costs one extra read of the target rows (plus one from L2 / shared memory) instead of the read + write of
+ * distribution of dspark_truncate_target, without modifying the target rows: after the statistics pass the
+ * threshold tau of every target row is found (same rule, exact on the 16-bit keys: one more streamed pass counts the
+ * keys next to the row maximum, a row that this does not resolve is counted once more over a deeper window, and what
+ * is left goes through the per-row search of dspark_truncate_target) together with the mass of the kept set; the
+ * accept test, the residual pass and the final draws then treat a target logit below tau as -inf.  The draft
+ * distribution q is used as given.  Costs one extra read of the target rows instead of the read + write of
  * dspark_truncate_target.  temperatures / top_k / top_p: device [R] or NULL (temperatures NULL: the scalar
  * `temperature`; top_k and top_p both NULL: plain dspark_verify).  out_p_tok reports the truncated p(x).
  * fp32 rows: the threshold of every target row comes from the per-row descent of dspark_truncate_target (no
