@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 // The eight blocks of the unit are counted into one histogram in shared memory; when all consumer
                 // warps have added theirs (a barrier of their own, bounded like every wait), each thread moves
                 // its share of the non-empty bins to the row's counts and leaves them zero for the unit after next.
-                const uint32_t window = s_unit[st].trunc.size;
+                const uint32_t window = s_unit[st].trunc.size & ~kWindowDense;
                 unsigned int* h = unit_bins + (it & 1) * kHistBins;
                 consume_block<kElem, kMode>(P, unit_s, unit_piece, n_rows, warp, lane, f0, f1, unit_scale, nullptr,
                                             &s_unit[st].trunc, h);
@@ -307,6 +307,8 @@ __device__ __forceinline__ void key_window(float lo_val, uint32_t kmax, uint32_t
     if (size > kmax + 1u) size = kmax + 1u;                          // keys 0 .. kmax exist
     const uint32_t cb = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(bf16_key_value(kmax - (size - 1u))));
     cut2 = cb | (cb << 16);
+    // a wide window of positive values only: counted by the distance of the bit patterns (consume_block)
+    if (size >= 256u && kmax - (size - 1u) > 0x8000u) size |= kWindowDense;
 }
 
 // Top-p: the tokens below a value v weigh at most V 2^(v scale - C) together, so the nucleus ends above the v at
@@ -396,7 +398,7 @@ __global__ void __launch_bounds__(256) trunc_prep_kernel(VerifyParams P, TruncAr
         tr.kmax = kmax; tr.size = size; tr.cut2 = cut2; tr.scale = scale;
         tr.k = use_k ? k : 0; tr.p = use_p ? pf : 1.f;
         unsigned int* bins = P.trunc_bins + (long long)row * kHistBins;
-        for (uint32_t i = lane; i < size; i += 32) bins[i] = 0u;
+        for (uint32_t i = lane; i < (size & ~kWindowDense); i += 32) bins[i] = 0u;
     }
     if (lane == 0) { P.trunc_rows[row] = tr; T.tau[row] = kNegInf; P.trunc_flag[row] = 0; P.trunc_z[row] = -1.0; }
     if (row == 0 && lane == 0) {                                         // the per-row fallback's work counter and the
@@ -414,9 +416,9 @@ __device__ __forceinline__ void leave_unresolved(const VerifyParams& P, int row,
     uint32_t size = 0u, cut2 = 0u;
     if (!retry && tr.k == 0 && tr.p < 1.f && tr.p > 0.f)
         key_window(nucleus_floor(tr.C, tr.Z, tr.p, tr.scale, P.V), tr.kmax, size, cut2);
-    if (size > tr.size) {
+    if ((size & ~kWindowDense) > tr.size) {
         unsigned int* bins = P.trunc_bins + (long long)row * kHistBins;
-        for (uint32_t i = tid; i < size; i += kScanThreads) bins[i] = 0u;
+        for (uint32_t i = tid; i < (size & ~kWindowDense); i += kScanThreads) bins[i] = 0u;
         if (tid == 0) {
             P.trunc_rows[row].size = size;
             P.trunc_rows[row].cut2 = cut2;
@@ -442,7 +444,8 @@ __global__ void __launch_bounds__(kScanThreads) trunc_scan_kernel(VerifyParams P
     bool bad_rows;
     if (row >= device_rows(P, &bad_rows)) return;
     if (retry && P.trunc_flag[row] != 2) return;            // the second look is for the rows listed by the first
-    const TruncRow tr = P.trunc_rows[row];
+    TruncRow tr = P.trunc_rows[row];
+    tr.size &= ~kWindowDense;
     if (tr.size == 0u) return;
     if (tid == 0) { s_hit_k = 0x7fffffff; s_hit_p = 0x7fffffff; }
     const unsigned int* bins = P.trunc_bins + (long long)row * kHistBins;

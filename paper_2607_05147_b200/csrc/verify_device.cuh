@@ -12,6 +12,7 @@
 namespace dspark {
 
 constexpr int kModeStats = 0, kModeGreedy = 1, kModeResid = 2, kModeHist = 3;
+constexpr uint32_t kWindowDense = 0x80000000u;   // flag in TruncRow::size
 constexpr int kHistBins = 1024;              // keys next to the row maximum that the streamed threshold search resolves
 constexpr int kTaskNone = 0, kTaskResid = 1, kTaskBonus = 2;
 constexpr int kCtrBonus = 12;                // header cell: bonus rows queued for the second pass (from the back of the queue)
@@ -45,7 +46,8 @@ struct __align__(16) RequestRec {    // what the finalize kernel needs per reque
 
 struct __align__(16) TruncRow {      // per target row, for the streamed threshold search of top-k / top-p
     uint32_t kmax;                   // key of the row maximum
-    uint32_t size;                   // keys in the window next to the maximum (0: row not truncated)
+    uint32_t size;                   // keys in the window next to the maximum (0: row not truncated); bit 31: a wide
+                                     // window of positive values only (counted without the branch, see consume_block)
     uint32_t cut2;                   // lowest value of the window, bf16 pattern in both halves
     float scale;                     // log2(e) / T
     float C;                         // row reference (log2 domain) of the statistics
@@ -462,8 +464,26 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
         // caller keeps one (it adds the non-empty bins to the row's counts afterwards), else on the row's counts.
         const TruncRow tr = trunc ? *trunc : P.trunc_rows[s];
         if (tr.size == 0u) return;
-        const __nv_bfloat162 cut2 = *reinterpret_cast<const __nv_bfloat162*>(&tr.cut2);
         unsigned int* bins = shared_bins ? shared_bins : P.trunc_bins + (long long)s * kHistBins;
+        if (tr.size & kWindowDense) {
+            // A wide window holds a good part of the row's tokens, and the branch below would be taken by some
+            // thread of the warp for every pair.  All its values are positive, where the key distance is the
+            // distance of the bit patterns: two subtractions, two compares and two predicated adds per pair
+            // (a negative value or a NaN wraps to a distance beyond the window).
+            const uint32_t bmax = tr.kmax & 0x7FFFu, size = tr.size & ~kWindowDense;
+#pragma unroll
+            for (int k = 0; k < M::kVec; ++k) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t w = word_of(v[k], i);
+                    const uint32_t d0 = bmax - (w & 0xFFFFu), d1 = bmax - (w >> 16);
+                    if (d0 < size) atomicAdd(&bins[d0], 1u);
+                    if (d1 < size) atomicAdd(&bins[d1], 1u);
+                }
+            }
+            return;
+        }
+        const __nv_bfloat162 cut2 = *reinterpret_cast<const __nv_bfloat162*>(&tr.cut2);
 #pragma unroll
         for (int k = 0; k < M::kVec; ++k) {
 #pragma unroll
