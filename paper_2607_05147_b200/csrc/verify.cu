@@ -56,6 +56,17 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     pdl_wait();                                  // everything below reads what earlier kernels wrote
 
     const uint32_t entry_limit = g_entry_poll_limit;
+    // Statistics pass without the bonus rows: every CTA keeps row_offsets[r] - r behind its stages (see below).  The
+    // offsets are asked for before anything waits for the row count, so that the prologue costs one trip to the L2.
+    constexpr int kPrefPer = (kSkipBonusMaxRequests + kStreamThreads) / kStreamThreads;
+    int pref_reg[kPrefPer];
+    if (kMode == kModeStats && P.skip_bonus) {
+#pragma unroll
+        for (int k = 0; k < kPrefPer; ++k) {
+            const int r = tid + k * kStreamThreads;
+            pref_reg[k] = r <= P.R ? P.row_offsets[r] - r : 0;
+        }
+    }
     bool bad_rows;
     const int n_rows = device_rows(P, &bad_rows);
     if (kMode != kModeResid && kMode != kModeHist && blockIdx.x == 0 && tid == 0) {
@@ -90,7 +101,11 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     const bool skip_bonus = kMode == kModeStats && P.skip_bonus;
     const int nd = n_rows > P.R ? n_rows - P.R : 0;
     if (skip_bonus) {
-        for (int r = tid; r <= P.R; r += kStreamThreads) pref[r] = P.row_offsets[r] - r;
+#pragma unroll
+        for (int k = 0; k < kPrefPer; ++k) {
+            const int r = tid + k * kStreamThreads;
+            if (r <= P.R) pref[r] = pref_reg[k];
+        }
         __syncthreads();
     }
 
