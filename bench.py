@@ -169,14 +169,15 @@ class Step:
             entries = self.R * gpad
             n_sched = 2 + (1 if entries >= 8192 and 2 * (self.sched.budget_tokens - self.R) <= entries else 0)
         # verifier: statistics pass, accept tests, residual pass, draws (greedy: argmax pass + accept tests); one more
-        # for per-request temperatures; for a truncated target the window preparation, the histogram pass, the
-        # threshold scan, the restricted sums and the per-row fallback (fp32 rows: the per-row descent alone)
+        # for per-request temperatures; for a truncated target the window preparation, the histogram pass and the
+        # threshold scan, both a second time for the rows of the second look, the restricted sums of the bonus rows
+        # and the per-row fallback (fp32 rows: the per-row descent alone)
         if wl["greedy"]:
             n_verify = 2
         else:
             n_verify = 4 + (1 if PER_REQUEST_T else 0)
             if TRUNCATE is not None:
-                n_verify += 1 if b0.target.dtype == torch.float32 else 5
+                n_verify += 1 if b0.target.dtype == torch.float32 else 7
         self.launches_per_step = n_sched + n_verify
 
     def run(self, batch, conf=None):
@@ -924,6 +925,28 @@ def main():
         del res, wl
         torch.cuda.empty_cache()
         line["other_workloads"] = others
+        # the option rows on cfg3 (each is what `bench.py --only <flags>` prints as its own line): the step with
+        # top-k / top-p truncation inside the verifier, with one temperature per request, with the asynchronous
+        # top-K scheduler
+        if args.workload == "cfg3" and TRUNCATE is None and not (PER_REQUEST_T or ASYNC_TOPK or CUDA_GRAPH or OVERLAP):
+            variants = {}
+            for label, setting in (("top_k50_top_p0.9", {"TRUNCATE": (50, 0.9)}), ("top_p0.9", {"TRUNCATE": (0, 0.9)}),
+                                   ("top_k50", {"TRUNCATE": (50, 1.0)}), ("per_request_temperature", {"PER_REQUEST_T": True}),
+                                   ("async_topk", {"ASYNC_TOPK": True})):
+                saved = {k: globals()[k] for k in setting}
+                globals().update(setting)
+                try:
+                    res = measure_workload("cfg3", args, device, rank, local_rank, world, dist, barrier, False, False)
+                finally:
+                    globals().update(saved)
+                variants[label] = {"ms_per_step": res["ms"] / args.steps, "ms_per_step_min": res["ms_min"] / args.steps,
+                                   "verify_call_us": verify_call_of(res, args.steps, peak)["us_per_call"],
+                                   "kernels_us_per_launch": {n: 1e3 * v["ms"] / v["launches"] for n, v in res["kernels"].items()},
+                                   "gpu_launches_per_step": res["step"].launches_per_step,
+                                   "clocks": res["clocks"], "dev_status": res["dev_status"]}
+                del res
+                torch.cuda.empty_cache()
+            line["variants_cfg3"] = variants
         margs = argparse.Namespace(**vars(args))
         margs.requests = 256
         m = bench_markov(margs, device, rank, world, dist, barrier)
