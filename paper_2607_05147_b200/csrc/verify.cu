@@ -100,6 +100,10 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     int* pref = reinterpret_cast<int*>(stage_mem + kStages * kStageBytes);
     const bool skip_bonus = kMode == kModeStats && P.skip_bonus;
     const int nd = n_rows > P.R ? n_rows - P.R : 0;
+    // Where it fits behind that array: the request of every draft position, so that a unit costs its producer one
+    // look-up instead of a search (and a draft unit no search through global memory for its physical row).
+    unsigned short* req_of = reinterpret_cast<unsigned short*>(pref + ((P.R + 4) & ~3));
+    const bool have_req_of = skip_bonus && P.req_table;
     if (skip_bonus) {
 #pragma unroll
         for (int k = 0; k < kPrefPer; ++k) {
@@ -107,6 +111,14 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
             if (r <= P.R) pref[r] = pref_reg[k];
         }
         __syncthreads();
+        if (have_req_of) {
+            for (int r = tid; r < P.R; r += kStreamThreads) {
+                int a = pref[r], b = pref[r + 1];
+                a = a < 0 ? 0 : a; b = b > P.req_table ? P.req_table : b;
+                for (int i = a; i < b; ++i) req_of[i] = (unsigned short)r;
+            }
+            __syncthreads();
+        }
     }
 
     if (warp == kConsumerWarps) {
@@ -146,14 +158,29 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                 } else if (live) {
                     slot.s = total <= 0x7fffffffll ? (int)((unsigned)u / (unsigned)ppr) : (int)(u / ppr);
                     slot.piece = (int)(u - (long long)slot.s * ppr);
+                    long long draft_row = -2;                // physical draft row, where it is found here
                     if (skip_bonus) {
+                        // draft position ds of the batch (target stream s' = ds, draft stream s' = nd + ds) belongs to
+                        // the largest r with row_offsets[r] - r <= ds
+                        const int ds = slot.s < nd ? slot.s : slot.s - nd;
+                        int lo = 0;
+                        if (have_req_of && ds < P.req_table) {
+                            lo = req_of[ds];
+                            if (lo >= P.R) lo = P.R - 1;                    // only with inconsistent offsets
+                        } else if (slot.s < nd) {
+                            int hi = P.R;
+                            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (pref[mid] <= ds) lo = mid; else hi = mid; }
+                        }
                         if (slot.s < nd) {
-                            int lo = 0, hi = P.R;        // largest r with row_offsets[r] - r <= s'
-                            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (pref[mid] <= slot.s) lo = mid; else hi = mid; }
-                            slot.s += lo;
+                            slot.s = ds + lo;
                             if (slot.s >= n_rows) slot.s = n_rows - 1;      // only with inconsistent offsets
                         } else {
-                            slot.s = n_rows + (slot.s - nd);
+                            slot.s = n_rows + ds;
+                            if (have_req_of && ds < P.req_table) {
+                                const int j = ds - pref[lo], len = pref[lo + 1] - pref[lo];
+                                draft_row = !P.draft_row_start ? (long long)ds
+                                                               : ((j >= 0 && j < len) ? P.draft_row_start[lo] + j : -1);
+                            }
                         }
                     }
                     if (kMode == kModeResid) slot.task = P.resid[slot.s];
@@ -164,7 +191,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                         }
                         slot.trunc = P.trunc_rows[slot.s];
                     }
-                    unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes, kMode == kModeResid ? &slot.task : nullptr);
+                    unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes, kMode == kModeResid ? &slot.task : nullptr,
+                                        draft_row);
                     slot.scale = stream_scale<kMode>(P, slot.s, n_rows, n_streams + (skip_bonus ? P.R : 0));
                 } else {
                     slot.s = -1; slot.piece = 0; slot.scale = 0.f;
@@ -1125,7 +1153,7 @@ template <int kElem, int kMode>
 static cudaError_t set_smem_attr()
 {
     return cudaFuncSetAttribute(stream_bulk_kernel<kElem, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                kStages * kStageBytes + (kMode == kModeStats ? (kSkipBonusMaxRequests + 4) * 4 : 0) +
+                                kStages * kStageBytes + (kMode == kModeStats ? kSkipBonusSmemBytes : 0) +
                                     (kMode == kModeHist ? 2 * kHistBins * (int)sizeof(unsigned int) : 0));
 }
 
@@ -1150,7 +1178,7 @@ static void launch_stream(const VerifyParams& P, bool bulk, long long max_units,
         if (g > max_units) g = max_units;
         if (g < 1) g = 1;
         size_t smem = (size_t)kStages * kStageBytes;
-        if (kMode == kModeStats && P.skip_bonus) smem += (size_t)((P.R + 4) / 4) * 16;
+        if (kMode == kModeStats && P.skip_bonus) smem += (size_t)((P.R + 4) / 4) * 16 + (size_t)((P.req_table + 7) / 8) * 16;
         if (kMode == kModeHist) smem += 2 * kHistBins * sizeof(unsigned int);
         launch_pdl(stream_bulk_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kStreamThreads), smem, s, P);
     } else {
@@ -1346,6 +1374,10 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
     // streams them for the requests that accepted every draft token.  (Not with a truncated target, whose threshold
     // search wants the statistics of every target row first, nor on the direct-load path.)
     P.skip_bonus = (bulk && !truncate && g_skip_bonus.load(std::memory_order_relaxed) && R <= kSkipBonusMaxRequests) ? 1 : 0;
+    // the request of every draft position rides along in shared memory when it fits beside the offsets (16-bit entries)
+    P.req_table = 0;
+    if (P.skip_bonus && R <= 65535 && (size_t)((R + 4) / 4) * 16 + (size_t)((n_rows - R + 7) / 8) * 16 <= (size_t)kSkipBonusSmemBytes)
+        P.req_table = n_rows - R;
     if (req_temp) {
         KernelTimerScope timer(DSPARK_K_ROW_SCALE, s);
         launch_pdl(row_scale_kernel, dim3((R + 255) / 256), dim3(256), 0, s, P);

@@ -16,6 +16,7 @@ constexpr uint32_t kWindowDense = 0x80000000u;   // flag in TruncRow::size
 constexpr int kHistBins = 1024;              // keys next to the row maximum that the streamed threshold search resolves
 constexpr int kTaskNone = 0, kTaskResid = 1, kTaskBonus = 2;
 constexpr int kCtrBonus = 12;                // header cell: bonus rows queued for the second pass (from the back of the queue)
+constexpr int kSkipBonusSmemBytes = 9 * 1024;    // shared memory behind the stages for the offsets and that table
 constexpr int kCtrRetry = 13;                // header cell: rows the threshold search looks at a second time
 constexpr int kCellRetryUnits = 5;           // 64-bit header cell: unit counter of that second histogram pass
 constexpr int kSkipBonusMaxRequests = 2048;  // the statistics pass keeps (row_offsets[r] - r) of the batch behind its stages
@@ -87,6 +88,8 @@ struct VerifyParams {
     unsigned long long launch_tag;            // unique per call: see unit_counter()
     float* wblk;                              // per request: residual block sums
     const float* tau;                         // per target row: top-k / top-p threshold (NULL: no truncation)
+    int req_table;                            // statistics pass without the bonus rows: entries of the request-of-position
+                                              // table kept in shared memory (0: none, the request is searched for)
     int skip_bonus;                           // 1: the statistics pass leaves the bonus rows out; the second pass streams
                                               // them for the requests that accepted every draft token (a rejected
                                               // request never needs its bonus row)
@@ -520,7 +523,7 @@ __device__ __forceinline__ float stream_scale(const VerifyParams& P, int s, int 
 template <int kMode>
 __device__ __forceinline__ void unit_sources(const VerifyParams& P, int s, int piece, int n_rows,
                                              const unsigned char*& src0, const unsigned char*& src1, int& bytes,
-                                             const ResidTask* task = nullptr)
+                                             const ResidTask* task = nullptr, long long draft_row = -2)
 {
     using M = ModeCfg<kMode>;
     const long long off = (long long)piece * M::kPieceBytes;
@@ -534,7 +537,8 @@ __device__ __forceinline__ void unit_sources(const VerifyParams& P, int s, int p
     } else if (s < n_rows) {
         src0 = P.target + (long long)s * P.tstride_bytes + off;
     } else {
-        const long long phys = draft_phys_row(P, s - n_rows);
+        // draft_row: the physical row where the caller has found it already (-1: inconsistent offsets), else -2
+        const long long phys = draft_row != -2 ? draft_row : draft_phys_row(P, s - n_rows);
         src0 = (phys >= 0 ? P.draft + phys * P.dstride_bytes : P.target) + off;
     }
 }
