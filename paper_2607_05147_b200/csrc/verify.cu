@@ -915,6 +915,15 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
     float xr[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) { const int i = k * 32 + lane; xr[k] = i < P.nblk_r ? __ldcg(&wb[i]) : 0.f; }
+    // and, where the second pass streams the bonus rows, the block statistics it left for this request (up to 256
+    // blocks in registers; whether the request drew a bonus token at all is in the record)
+    const float2* sb = P.stats_b + (long long)r * P.nblk;
+    float2 eb[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int i = k * 32 + lane;
+        eb[k] = (P.skip_bonus && i < P.nblk) ? __ldcg(&sb[i]) : make_float2(kNegInf, 0.f);
+    }
     if (rec.kind == kTaskNone) return;
     Level2Scratch<kElem>& S = s_scr[warp];
     const double u = (double)rec.u;
@@ -927,7 +936,14 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
     float cp = rec.cp;
     if (late_bonus) {
         RowAcc A, D;
-        combine_rows(P.stats_t + (long long)rec.row_t * P.nblk, nullptr, P.nblk, lane, A, D);
+        if (P.nblk <= 256) {                   // the entries in the order combine_rows takes them
+            A.init();
+#pragma unroll
+            for (int k = 0; k < 8; ++k) A.add(eb[k]);
+            A.finish();
+        } else {
+            combine_rows(sb, nullptr, P.nblk, lane, A, D);
+        }
         if (!row_usable(A.C, A.S)) {
             const int lo = P.row_offsets[r], hi = P.row_offsets[r + 1];
             for (int i = lo + lane; i < hi; i += 32) P.out_tokens[i] = -1;
@@ -947,7 +963,10 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
             for (int k = 0; k < 8; ++k) {
                 const int i = k * 32 + lane;
                 float m = 0.f;
-                if (i < P.nblk && P.nblk <= 256) { const float2 e = __ldcg(&st[i]); m = e.x > kNegInf ? e.y * ex2_approx(e.x - cp) : 0.f; }
+                if (i < P.nblk && P.nblk <= 256) {
+                    const float2 e = late_bonus ? eb[k] : __ldcg(&st[i]);
+                    m = e.x > kNegInf ? e.y * ex2_approx(e.x - cp) : 0.f;
+                }
                 xr[k] = m;
             }
         }
@@ -962,7 +981,7 @@ __global__ void __launch_bounds__(kFinalizeWarps * 32) finalize_kernel(VerifyPar
             tot = warp_total(n1, lane, wv);
             b = level1_memory(n1, lane, wv, u * tot, before);
         } else {
-            const float2* st = P.stats_t + (long long)rec.row_t * P.nblk;
+            const float2* st = late_bonus ? sb : P.stats_t + (long long)rec.row_t * P.nblk;
             auto mass = [&](int i) { const float2 e = __ldcg(&st[i]); return e.x > kNegInf ? e.y * ex2_approx(e.x - cp) : 0.f; };
             tot = warp_total(n1, lane, mass);
             b = level1_memory(n1, lane, mass, u * tot, before);
@@ -1252,6 +1271,7 @@ static int fill_params(VerifyParams& P, const void* target, const void* draft, i
     P.dev_status = dev_status ? dev_status : P.counters + 1;
     P.stats_t = (float2*)(ws + w.stats_t);
     P.stats_d = (float2*)(ws + w.stats_d);
+    P.stats_b = (float2*)(ws + w.stats_b);
     P.resid = (ResidTask*)(ws + w.resid);
     P.req = (RequestRec*)(ws + w.req);
     P.wblk = (float*)(ws + w.wblk);

@@ -83,6 +83,8 @@ struct VerifyParams {
     int* counters;                            // [0] queued residual tasks, [1] dev_status stand-in
     float2* stats_t;
     float2* stats_d;
+    float2* stats_b;                          // [R][nblk]: block statistics of a bonus row streamed by the second pass, by
+                                              // request (the draw kernel asks for them before it knows the row)
     ResidTask* resid;                         // queue of rejected requests (decide -> residual pass)
     RequestRec* req;                          // per request: outcome of decide for the finalize kernel
     unsigned long long launch_tag;            // unique per call: see unit_counter()
@@ -441,7 +443,7 @@ __device__ __forceinline__ void consume_block(const VerifyParams& P, int s, int 
             load_block<kElem, kStatVec>(SmemFetch{f0.blk + warp * (kStatBlockBytes - M::kBlockBytes)},
                                         rem4 < kStatBlockBytes ? rem4 : kStatBlockBytes, lane, v4);
             const float2 st = block_stats<kElem, kStatVec>(v4, task->scale);
-            if (lane == 0) P.stats_t[(long long)task->row_t * P.nblk + b4] = st;
+            if (lane == 0) P.stats_b[(long long)task->wslot * P.nblk + b4] = st;
             return;
         }
     }
@@ -787,7 +789,7 @@ __device__ __forceinline__ int level2_block(const unsigned char* trow, const uns
 
 // Workspace of the verifiers (caller-provided, any content on entry), offsets in bytes.
 struct Workspace {
-    size_t counters, stats_t, stats_d, resid, req, wblk, scale_t, scale_d, tau, trunc_rows, trunc_bins, trunc_flag, retry_rows, trunc_z;
+    size_t counters, stats_t, stats_d, stats_b, resid, req, wblk, scale_t, scale_d, tau, trunc_rows, trunc_bins, trunc_flag, retry_rows, trunc_z;
     size_t total;
 };
 inline Workspace workspace_layout(int R, int n_rows, int V)
@@ -800,6 +802,7 @@ inline Workspace workspace_layout(int R, int n_rows, int V)
     w.counters = o; o += up(64 * sizeof(int));
     w.stats_t = o;  o += up((size_t)n_rows * nblk * sizeof(float2));
     w.stats_d = o;  o += up((size_t)n_rows * nblk * sizeof(float2));
+    w.stats_b = o;  o += up((size_t)R * nblk * sizeof(float2));
     w.resid = o;    o += up((size_t)R * sizeof(ResidTask));
     w.req = o;      o += up((size_t)R * sizeof(RequestRec));
     w.wblk = o;     o += up((size_t)R * nblk_r * sizeof(float));
