@@ -402,11 +402,30 @@ __global__ void __launch_bounds__(256) trunc_prep_kernel(VerifyParams P, TruncAr
             // largest block maximum: the window reaches down to it (rank by counting, 64-128 blocks)
             const float2* st = P.stats_t + (long long)row * P.nblk;
             float kth = kNegInf;
-            if (P.nblk <= 128) {                             // block references in registers, compared through shuffles
+            if (P.nblk <= 64) {                              // two block references per lane, compared through shuffles
+                float c[2];
+#pragma unroll
+                for (int q = 0; q < 2; ++q) c[q] = (q * 32 + lane < P.nblk) ? __ldcg(&st[q * 32 + lane]).x : kNegInf;
+                int rank[2] = {0, 0};                        // blocks that come before mine in descending order
+#pragma unroll
+                for (int q2 = 0; q2 < 2; ++q2) {
+                    if (q2 * 32 >= P.nblk) break;
+#pragma unroll 8
+                    for (int l2 = 0; l2 < 32; ++l2) {
+                        const float cj = __shfl_sync(0xffffffffu, c[q2], l2);
+                        const int j = q2 * 32 + l2;
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) rank[q] += (cj > c[q]) || (cj == c[q] && j < q * 32 + lane);
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 2; ++q)
+                    if (q * 32 + lane < P.nblk && rank[q] == k - 1) kth = c[q];
+            } else if (P.nblk <= 128) {                      // four per lane
                 float c[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) c[q] = (q * 32 + lane < P.nblk) ? __ldcg(&st[q * 32 + lane]).x : kNegInf;
-                int rank[4] = {0, 0, 0, 0};                  // blocks that come before mine in descending order
+                int rank[4] = {0, 0, 0, 0};
 #pragma unroll
                 for (int q2 = 0; q2 < 4; ++q2) {
                     if (q2 * 32 >= P.nblk) break;
