@@ -33,12 +33,11 @@ NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126 * 1024 * 1024
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/: cfg3 was captured as it is; cfg4 and cfg5 are too large for a
-# multi-pass capture, so their figure is the algorithmic bytes times the traffic / algorithmic ratio of
-# the smaller capture of the same kernel (traffic is proportional to the rows streamed), and cfg2 takes
-# the ratio of its capture of the earlier form of the pass (every bonus row streamed there as well).
-NCU_TRAFFIC_BYTES = {"cfg3": 198608640 + 3929088}
-NCU_TRAFFIC_RATIO = {"cfg2": 1.025, "cfg4": 1.0135, "cfg5": 1.0165}
+# captures summarised under profiles/: cfg2 and cfg3 were captured as they are; cfg4 and cfg5 are too large
+# for a multi-pass capture, so their figure is the algorithmic bytes times the traffic / algorithmic ratio of
+# the smaller capture of the same kernel (traffic is proportional to the rows streamed).
+NCU_TRAFFIC_BYTES = {"cfg3": 198612480 + 3035136, "cfg2": 152069376 + 3132160}
+NCU_TRAFFIC_RATIO = {"cfg4": 1.0135, "cfg5": 1.0165}
 
 
 # ----------------------------------------------------------------------------- workloads ----
