@@ -495,6 +495,9 @@ static void verify_request(const verify_job_t* J, int r)
     if (lo < 0 || hi - lo < 1) { J->status[r] = ORC_ST_BAD_OFFSETS; J->accepted_len[r] = 0; return; }
     int32_t len = hi - lo - 1;
     int64_t drow0 = J->draft_row_start ? J->draft_row_start[r] : (int64_t)lo - (int64_t)r;
+    /* compact layout (Section 5.3, flat ragged rows): the draft rows of request r follow those of the requests
+       before it, at lo - r; an earlier request without a row of its own would put them before the array */
+    if (drow0 < 0) { J->status[r] = ORC_ST_BAD_OFFSETS; J->accepted_len[r] = 0; return; }
     int32_t st = 0;
     /* per-request temperature (requests of one batch may use different sampling settings) */
     const double T = J->temps ? (double)J->temps[r] : J->T;
@@ -659,6 +662,7 @@ int orc_accept_rate(const void* target, const void* draft, int dtype,
         if (lo < 0 || hi - lo < 1) { status[r] = ORC_ST_BAD_OFFSETS; continue; }
         int32_t len = hi - lo - 1;
         int64_t drow0 = draft_row_start ? draft_row_start[r] : (int64_t)lo - (int64_t)r;
+        if (drow0 < 0) { status[r] = ORC_ST_BAD_OFFSETS; continue; }   /* see verify_request */
         cstar[hi - 1] = NAN;
         for (int32_t j = 0; j < len; ++j) {
             double mp, Zp, mq, Zq;

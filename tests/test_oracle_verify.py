@@ -232,8 +232,13 @@ def test_degenerate_cases():
     ok = np.log(p).astype(np.float32).reshape(1, V).repeat(2, 0)
     r = oracle.verify(ok, ok[:1], [0, 2], [V, 0], 1.0, seed=3)
     assert r.status[0] & oracle.ST_BAD_TOKEN and (r.out_tokens == -1).all()
+    # a request without a row of its own: reported; in the compact layout the draft rows of the next request would
+    # start before the array (off[1] - 1 = -1), so it is reported too and nothing is read; with explicit draft row
+    # starts the next request is verified as usual
     r = oracle.verify(ok, ok[:1], [0, 0, 2], [0, 0], 1.0, seed=3)
-    assert r.status[0] & oracle.ST_BAD_OFFSETS and r.status[1] == 0
+    assert r.status[0] & oracle.ST_BAD_OFFSETS and r.status[1] & oracle.ST_BAD_OFFSETS and (r.out_tokens == -1).all()
+    r = oracle.verify(ok, ok[:1], [0, 0, 2], [0, 0], 1.0, seed=3, draft_row_start=np.array([0, 0], dtype=np.int64))
+    assert r.status[0] & oracle.ST_BAD_OFFSETS and r.status[1] == 0 and r.out_tokens[1] >= 0
 
 
 def test_inverse_cdf_against_cumsum_searchsorted():
