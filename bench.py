@@ -739,9 +739,17 @@ def roofline_of(res, peak, peak_src):
     traffic = NCU_TRAFFIC_BYTES.get(wl["name"]) if not REQUESTS_OVERRIDE else None
     if traffic is None and wl["name"] in NCU_TRAFFIC_RATIO and not REQUESTS_OVERRIDE:
         traffic = int(NCU_TRAFFIC_RATIO[wl["name"]] * stream_bytes)
+    if wl["greedy"]:
+        rows = "every target row once"
+    elif TRUNCATE is not None or b0.R > 2048:
+        rows = "every target row and every draft row once"
+    else:
+        rows = ("the target and the draft row of every draft position (the bonus rows are left to the second pass, which "
+                "streams them only for requests that accepted every draft token)")
     return {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": traffic,
-            "peak_source": peak_src, "algorithmic_bytes_per_launch": stream_bytes, "us_per_launch": dom_ms * 1e3}
+            "peak_source": peak_src, "algorithmic_bytes_per_launch": stream_bytes, "us_per_launch": dom_ms * 1e3,
+            "rows_per_launch": stream_bytes // (b0.target.element_size() * b0.V), "launch_streams": rows}
 
 
 def verify_call_of(res, steps, peak):
