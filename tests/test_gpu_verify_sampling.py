@@ -73,6 +73,49 @@ def test_odd_vocabularies_dtypes_and_paths(V, dtype):
     np.testing.assert_array_equal(g["acc"], g1["acc"])
 
 
+@pytest.mark.parametrize("V,dtype,block", [(W.V_FULL, torch.bfloat16, 8), (50_000, torch.float32, None), (4097, torch.bfloat16, None)])
+def test_bonus_rows_in_the_second_pass_change_nothing(V, dtype, block):
+    # the verifier leaves the bonus rows out of its statistics pass and streams them in the second pass for the requests
+    # that accepted every draft token; the earlier order (every bonus row in the statistics pass) stays behind the
+    # diagnostic switch: same accepted lengths, tokens and probabilities, bit for bit -- also with the draft rows'
+    # statistics handed over, with per-request temperatures, and for requests without a draft token
+    g0 = torch.Generator().manual_seed(V)
+    R = 40
+    lengths = torch.randint(0, 7, (R,), generator=g0)
+    lengths[:4] = 0
+    b = W.sampling_batch(lengths, V, 90, "cuda", dtype=dtype, temperature=0.8, draft_noise=0.5, verify_seed=17, block=block)
+    temps = torch.tensor(np.random.default_rng(V).choice([0.6, 1.0, 1.4], size=R), dtype=torch.float32, device="cuda")
+    stats = torch.empty(b.draft.shape[0], 2, device="cuda")
+    B.dspark_row_stats(b.draft, b.temperature, out_row_stats=stats)
+
+    def run_all():
+        res = [H.gpu_verify(b), H.gpu_verify(b, temperatures=temps)]
+        acc = torch.full((R,), -7, dtype=torch.int32, device="cuda")
+        out = torch.full((b.n_rows,), -7, dtype=torch.int32, device="cuda")
+        p = torch.full((b.n_rows,), float("nan"), device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ws = B.workspace(B.dspark_verify_workspace_bytes(R, b.n_rows, V))
+        B.dspark_verify_draft_stats(b.target, b.draft, b.row_offsets, b.draft_tokens, stats, b.seed, temperature=b.temperature,
+                                    draft_row_start=b.draft_row_start, accepted_len=acc, out_tokens=out, out_p_tok=p,
+                                    out_q_tok=None, dev_status=st, workspace=ws)
+        torch.cuda.synchronize()
+        res.append(dict(acc=acc.cpu().numpy(), out=out.cpu().numpy(), p=p.cpu().numpy(), status=int(st.item())))
+        return res
+
+    new = run_all()
+    B.dspark_set_stream_path(16)
+    try:
+        old = run_all()
+    finally:
+        B.dspark_set_stream_path(0)
+    assert (new[0]["acc"] == lengths.numpy()).any() and (new[0]["acc"] < lengths.numpy()).any()    # both kinds of request
+    for a, c in zip(new, old):
+        assert a["status"] == 0 and c["status"] == 0
+        np.testing.assert_array_equal(a["acc"], c["acc"])
+        np.testing.assert_array_equal(a["out"], c["out"])
+        np.testing.assert_array_equal(a["p"], c["p"])          # NaN where not evaluated, on both sides
+
+
 # 256 is the number of block values the finalize kernel keeps in registers; rows of 131 072 / 262 144 / 524 288
 # logits sit exactly at 256 residual or statistics blocks for one of the dtypes
 _BLOCK_COUNT_EDGES = [(dt, V + d) for dt in (torch.bfloat16, torch.float32)
