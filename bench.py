@@ -168,13 +168,19 @@ class Step:
             entries = self.R * gpad
             n_sched = 2 + (1 if entries >= 8192 and 2 * (self.sched.budget_tokens - self.R) <= entries else 0)
         # verifier: statistics pass, accept tests, residual pass, draws (greedy: argmax pass + accept tests); one more
-        # for per-request temperatures; for a truncated target the window preparation, the histogram pass and the
+        # for per-request temperatures on large batches; for a truncated target the window preparation, the histogram pass and the
         # threshold scan, both a second time for the rows of the second look, the restricted sums of the bonus rows
         # and the per-row fallback (fp32 rows: the per-row descent alone)
         if wl["greedy"]:
             n_verify = 2
         else:
-            n_verify = 4 + (1 if PER_REQUEST_T else 0)
+            n_verify = 4
+            if PER_REQUEST_T:
+                # the kernel that expands the temperatures to rows runs only when the requests' scales do not fit in
+                # the statistics pass's shared memory beside its request table (the library's rule, restated)
+                R, nd = self.R, self.n_rows - self.R
+                fits = R <= 2048 and ((R + 4) // 4) * 16 + ((nd + 7) // 8) * 16 + ((R + 3) // 4) * 16 <= 9 * 1024
+                n_verify += 0 if (fits and TRUNCATE is None) else 1
             if TRUNCATE is not None:
                 n_verify += 1 if b0.target.dtype == torch.float32 else 7
         self.launches_per_step = n_sched + n_verify

@@ -30,7 +30,9 @@ namespace dspark {
 // memory of a CTA that has left.
 __device__ uint32_t g_entry_poll_limit = kWaitPollLimit;
 
-template <int kElem, int kMode>
+// kReqScale (statistics pass only): one temperature per request, and every request's exponent scale kept in shared
+// memory beside the request table (P.req_scale_smem); an instantiation of its own, so that the plain pass keeps its code.
+template <int kElem, int kMode, bool kReqScale = false>
 __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyParams P)
 {
     using M = ModeCfg<kMode>;
@@ -60,11 +62,13 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     // offsets are asked for before anything waits for the row count, so that the prologue costs one trip to the L2.
     constexpr int kPrefPer = (kSkipBonusMaxRequests + kStreamThreads) / kStreamThreads;
     int pref_reg[kPrefPer];
+    float temp_reg[kPrefPer];                    // one temperature per request: they ride along (P.req_scale_smem)
     if (kMode == kModeStats && P.skip_bonus) {
 #pragma unroll
         for (int k = 0; k < kPrefPer; ++k) {
             const int r = tid + k * kStreamThreads;
             pref_reg[k] = r <= P.R ? P.row_offsets[r] - r : 0;
+            temp_reg[k] = (kReqScale && r < P.R) ? P.req_temp[r] : 1.0f;
         }
     }
     bool bad_rows;
@@ -104,11 +108,19 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
     // look-up instead of a search (and a draft unit no search through global memory for its physical row).
     unsigned short* req_of = reinterpret_cast<unsigned short*>(pref + ((P.R + 4) & ~3));
     const bool have_req_of = skip_bonus && P.req_table;
+    // and, with one temperature per request, every request's exponent scale log2(e)/T behind that table (no kernel
+    // that expands the temperatures to rows is needed then: the producer knows each unit's request)
+    float* scale_of = reinterpret_cast<float*>(req_of + ((P.req_table + 7) & ~7));
+    const bool have_scale_of = kReqScale && have_req_of;
     if (skip_bonus) {
 #pragma unroll
         for (int k = 0; k < kPrefPer; ++k) {
             const int r = tid + k * kStreamThreads;
             if (r <= P.R) pref[r] = pref_reg[k];
+            if (have_scale_of && r < P.R) {
+                const float T = temp_reg[k];
+                scale_of[r] = (T > 0.0f && T < INFINITY) ? (float)(1.4426950408889634 / (double)T) : 1.0f;
+            }
         }
         __syncthreads();
         if (have_req_of) {
@@ -159,6 +171,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                     slot.s = total <= 0x7fffffffll ? (int)((unsigned)u / (unsigned)ppr) : (int)(u / ppr);
                     slot.piece = (int)(u - (long long)slot.s * ppr);
                     long long draft_row = -2;                // physical draft row, where it is found here
+                    float own_scale = 0.f;                   // exponent scale of the unit's request, where it is known here
                     if (skip_bonus) {
                         // draft position ds of the batch (target stream s' = ds, draft stream s' = nd + ds) belongs to
                         // the largest r with row_offsets[r] - r <= ds
@@ -167,6 +180,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                         if (have_req_of && ds < P.req_table) {
                             lo = req_of[ds];
                             if (lo >= P.R) lo = P.R - 1;                    // only with inconsistent offsets
+                            if (have_scale_of) own_scale = scale_of[lo];
                         } else if (slot.s < nd) {
                             int hi = P.R;
                             while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (pref[mid] <= ds) lo = mid; else hi = mid; }
@@ -193,7 +207,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) stream_bulk_kernel(VerifyPa
                     }
                     unit_sources<kMode>(P, slot.s, slot.piece, n_rows, src0, src1, bytes, kMode == kModeResid ? &slot.task : nullptr,
                                         draft_row);
-                    slot.scale = stream_scale<kMode>(P, slot.s, n_rows, n_streams + (skip_bonus ? P.R : 0));
+                    slot.scale = have_scale_of ? (own_scale != 0.f ? own_scale : 1.0f)     // (no per-row scales exist then)
+                                               : stream_scale<kMode>(P, slot.s, n_rows, n_streams + (skip_bonus ? P.R : 0));
                 } else {
                     slot.s = -1; slot.piece = 0; slot.scale = 0.f;
                 }
@@ -1187,10 +1202,10 @@ static DeviceInfo& device_info()
     return d;
 }
 
-template <int kElem, int kMode>
+template <int kElem, int kMode, bool kReqScale = false>
 static cudaError_t set_smem_attr()
 {
-    return cudaFuncSetAttribute(stream_bulk_kernel<kElem, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(stream_bulk_kernel<kElem, kMode, kReqScale>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 kStages * kStageBytes + (kMode == kModeStats ? kSkipBonusSmemBytes : 0) +
                                     (kMode == kModeHist ? 2 * kHistBins * (int)sizeof(unsigned int) : 0));
 }
@@ -1202,7 +1217,8 @@ static bool ensure_attrs()
     bool ok = set_smem_attr<2, kModeStats>() == cudaSuccess && set_smem_attr<4, kModeStats>() == cudaSuccess &&
               set_smem_attr<2, kModeGreedy>() == cudaSuccess && set_smem_attr<4, kModeGreedy>() == cudaSuccess &&
               set_smem_attr<2, kModeResid>() == cudaSuccess && set_smem_attr<4, kModeResid>() == cudaSuccess &&
-              set_smem_attr<2, kModeHist>() == cudaSuccess;
+              set_smem_attr<2, kModeHist>() == cudaSuccess &&
+              set_smem_attr<2, kModeStats, true>() == cudaSuccess && set_smem_attr<4, kModeStats, true>() == cudaSuccess;
     d.attrs_set = ok;
     return ok;
 }
@@ -1216,9 +1232,13 @@ static void launch_stream(const VerifyParams& P, bool bulk, long long max_units,
         if (g > max_units) g = max_units;
         if (g < 1) g = 1;
         size_t smem = (size_t)kStages * kStageBytes;
-        if (kMode == kModeStats && P.skip_bonus) smem += (size_t)((P.R + 4) / 4) * 16 + (size_t)((P.req_table + 7) / 8) * 16;
+        if (kMode == kModeStats && P.skip_bonus)
+            smem += (size_t)((P.R + 4) / 4) * 16 + (size_t)((P.req_table + 7) / 8) * 16 + (P.req_scale_smem ? (size_t)((P.R + 3) / 4) * 16 : 0);
         if (kMode == kModeHist) smem += 2 * kHistBins * sizeof(unsigned int);
-        launch_pdl(stream_bulk_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kStreamThreads), smem, s, P);
+        if (kMode == kModeStats && P.req_scale_smem)
+            launch_pdl(stream_bulk_kernel<kElem, kMode, kMode == kModeStats>, dim3((unsigned)g), dim3(kStreamThreads), smem, s, P);
+        else
+            launch_pdl(stream_bulk_kernel<kElem, kMode>, dim3((unsigned)g), dim3(kStreamThreads), smem, s, P);
     } else {
         long long g = (long long)sms * 8;
         if (g > max_units) g = max_units;
@@ -1417,7 +1437,13 @@ static int verify_launch(const void* target_logits, const void* draft_logits, in
     P.req_table = 0;
     if (P.skip_bonus && R <= 65535 && (size_t)((R + 4) / 4) * 16 + (size_t)((n_rows - R + 7) / 8) * 16 <= (size_t)kSkipBonusSmemBytes)
         P.req_table = n_rows - R;
-    if (req_temp) {
+    // with one temperature per request and that table in place, the requests' exponent scales ride along as well, and
+    // the kernel that expands the temperatures to rows is not needed
+    P.req_scale_smem = 0;
+    if (req_temp && P.req_table > 0 &&
+        (size_t)((R + 4) / 4) * 16 + (size_t)((P.req_table + 7) / 8) * 16 + (size_t)((R + 3) / 4) * 16 <= (size_t)kSkipBonusSmemBytes)
+        P.req_scale_smem = 1;
+    if (req_temp && !P.req_scale_smem) {
         KernelTimerScope timer(DSPARK_K_ROW_SCALE, s);
         launch_pdl(row_scale_kernel, dim3((R + 255) / 256), dim3(256), 0, s, P);
     }

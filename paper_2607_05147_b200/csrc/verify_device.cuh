@@ -90,6 +90,8 @@ struct VerifyParams {
     unsigned long long launch_tag;            // unique per call: see unit_counter()
     float* wblk;                              // per request: residual block sums
     const float* tau;                         // per target row: top-k / top-p threshold (NULL: no truncation)
+    int req_scale_smem;                       // 1: with that table, the requests' exponent scales are kept beside it and the
+                                              // statistics pass needs no per-row scales (one temperature per request)
     int req_table;                            // statistics pass without the bonus rows: entries of the request-of-position
                                               // table kept in shared memory (0: none, the request is searched for)
     int skip_bonus;                           // 1: the statistics pass leaves the bonus rows out; the second pass streams
