@@ -257,7 +257,8 @@ int dspark_verify(const void* target_logits, const void* draft_logits, int dtype
  * mixes requests with different sampling settings): temperatures is a device array [R], request
  * r uses p = softmax(target / T_r), q = softmax(draft / T_r).  A temperature that is not a
  * positive finite number sets DSPARK_DEV_BAD_TEMPERATURE and voids that request only.
- * One extra tiny kernel expands T_r to the rows; everything else is dspark_verify.
+ * The statistics pass takes each unit's exponent scale from its request (on very large batches, and with a truncated
+ * target, one extra tiny kernel expands T_r to the rows first); everything else is dspark_verify.
  */
 int dspark_verify_per_request(const void* target_logits, const void* draft_logits, int dtype,
                               int64_t target_row_stride, int64_t draft_row_stride, int V,
